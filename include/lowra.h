@@ -1,0 +1,155 @@
+/*
+ * lowra.h -- C ABI of the B200 (sm_100a) hot path of LowRA's quantized-LoRA linear layer.
+ *
+ * Data model (paper Section 4.1): a frozen base weight W [N, K] (N output channels = rows,
+ * K input features) is quantised per output channel: row r has its own precision
+ * b_r in {1, 2, 4} bits ("Per-Output-Channel Quantization"), its own 2^b_r mapping values and
+ * its own 2^b_r - 1 sorted thresholds ("Per-Output-Channel Thresholds and Mappings"), and is
+ * normalised in blocks of 64 consecutive elements by the block's maximum magnitude
+ * ("Groupwise Normalization").  The quantised state is: the per-row precisions (`Precs` in
+ * Appendix A), the packed codes, one fp32 absmax per 64-block, the mapping table and the
+ * threshold table.
+ *
+ * Storage order: rows are grouped by precision (all 1-bit rows, then 2-bit, then 4-bit),
+ * ascending original index inside a group.  `perm[p]` is the original row of stored row p.
+ * Stored row p of class c (bits b) with rank q inside its class starts at byte
+ *     seg_off[c] + q * K * b / 8
+ * of the packed buffer; element k of the row occupies bits [k*b, k*b + b) of the row's
+ * little-endian bitstream (bit i of the stream = bit (i % 8) of byte i / 8).  No padding:
+ * packed_bytes = K * (n_1 + 2 n_2 + 4 n_4) / 8.
+ *
+ * Tables: `maps` and `thresholds` are fp32 [N, 16], row r = original row r, first 2^b (resp.
+ * 2^b - 1) entries valid.  `absmax` is fp32 [N, K / 64] in STORED row order.
+ *
+ * Conventions for every call:
+ *   - pointers named *_dev are DEVICE pointers owned by the caller, 16-byte aligned; pointers
+ *     named *_host are host pointers; the library never allocates, frees or synchronises
+ *     (except lowra_device_status, which synchronises the given stream);
+ *   - work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = default stream);
+ *   - the return value is a lowra_status; arguments are validated on the host before any launch;
+ *   - inputs are read-only, outputs are fully overwritten;
+ *   - there is no CPU fallback: on a device that is not sm_100 the calls return LOWRA_ERR_ARCH.
+ * Not checked on the device (preconditions): precisions in {1,2,4}, thresholds non-decreasing in
+ * their valid prefix, finite weights.
+ */
+#ifndef LOWRA_H
+#define LOWRA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LOWRA_OK = 0,
+    LOWRA_ERR_NULL = 1,      /* a required pointer is NULL */
+    LOWRA_ERR_SHAPE = 2,     /* N < 1, K % 128 != 0, block != 64, M < 1, r not in {16,32,...,128} */
+    LOWRA_ERR_ALIGN = 3,     /* a device pointer is not 16-byte aligned */
+    LOWRA_ERR_PREC = 4,      /* a precision outside {1,2,4}, or counts that do not sum to N */
+    LOWRA_ERR_WORKSPACE = 5, /* workspace smaller than lowra_workspace_bytes() */
+    LOWRA_ERR_CUDA = 6,      /* a CUDA runtime / driver call failed */
+    LOWRA_ERR_TIMEOUT = 7,   /* a bounded device-side wait ran out (read via lowra_device_status) */
+    LOWRA_ERR_ARCH = 8       /* current device is not compute capability 10.x */
+} lowra_status;
+
+const char* lowra_status_string(lowra_status st);
+
+/* Immutable description of one quantised weight (host struct, device arrays inside). */
+typedef struct {
+    int32_t N, K, block;         /* block must be 64; K % 128 == 0; N >= 1 */
+    int32_t counts[3];           /* rows with 1, 2, 4 bits */
+    uint64_t seg_off[3];         /* byte offset of each precision class in the packed buffer */
+    uint64_t packed_bytes;
+    const uint8_t* precs_dev;    /* [N] bits per row, original order */
+    const int32_t* perm_dev;     /* [N] stored position -> original row */
+    const int32_t* inv_perm_dev; /* [N] original row -> stored position */
+} lowra_layout;
+
+/*
+ * Storage planner (host only; Appendix A.1: packed rows are written "at the appropriate offset",
+ * A.2: the offset follows from the channel's bit precision).  Reads precs_host[N]; writes
+ * perm_host[N], inv_perm_host[N], counts[3], seg_off[3], *packed_bytes.  The caller uploads
+ * perm / inv_perm / precs and fills a lowra_layout.
+ * Errors: NULL pointer -> ERR_NULL; N < 1 or K % 128 != 0 -> ERR_SHAPE; bad precision -> ERR_PREC.
+ */
+lowra_status lowra_plan(int32_t N, int32_t K, const uint8_t* precs_host, int32_t* perm_host,
+                        int32_t* inv_perm_host, int32_t counts[3], uint64_t seg_off[3],
+                        uint64_t* packed_bytes);
+
+/*
+ * Quantize (Appendix A.1): for each 64-block of W compute the maximum magnitude and store it;
+ * normalise each value with it (n = x * fl(1/absmax) in fp32, n = 0 for an all-zero block);
+ * quantise n with the row's thresholds at the row's precision
+ * (code = number of valid thresholds <= n, so a value on a threshold takes the upper bucket);
+ * pack the codes and write them at the row's offset.
+ *   W_dev          fp32 [N, K] row-major, original row order          (in)
+ *   thresholds_dev fp32 [N, 16], original row order                   (in)
+ *   packed_dev     uint8 [layout->packed_bytes]                       (out)
+ *   absmax_dev     fp32 [N, K/64], stored row order                   (out)
+ */
+lowra_status lowra_encode(const lowra_layout* layout, const float* W_dev, const float* thresholds_dev,
+                          uint8_t* packed_dev, float* absmax_dev, void* stream);
+
+/*
+ * Dequantize (Appendix A.2): unpack each row's 1/2/4-bit codes, look them up in the row's mapping
+ * table, multiply by the block's absmax in fp32 and round to bf16 (nearest even).
+ *   W_bf16_dev     bf16 bit patterns [N, K] row-major, original row order   (out)
+ */
+lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* packed_dev, const float* absmax_dev,
+                          const float* maps_dev, uint16_t* W_bf16_dev, void* stream);
+
+/* Bytes of device scratch that lowra_lora_forward / lowra_lora_backward_input need for M tokens and
+ * LoRA rank r (0 if the arguments are invalid).  The first 256 bytes hold the device status word. */
+size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r);
+
+/*
+ * Forward of the quantized-LoRA linear layer (Section 3: the fine-tuning module recovers the base
+ * weights with the dequantize kernel; frozen base plus trainable low-rank factors):
+ *     Y = X . deq(Wq)^T + s * (X . A) . B
+ * deq(Wq) is exactly what lowra_decode produces, formed on the fly in the operand stage of the
+ * tensor-core contraction and never written to memory.  fp32 accumulation, bf16 output.
+ *   X_dev bf16 [M, K];  A_dev bf16 [K, r];  B_dev bf16 [r, N];  Y_dev bf16 [M, N], original
+ *   channel order; all row-major.  r in {16, 32, ..., 128}.  X . A is rounded to bf16 once.
+ *   workspace_dev: >= lowra_workspace_bytes(layout, M, r) bytes, 256-byte aligned, contents
+ *   overwritten.  Calls that share a workspace must not overlap on the device.
+ */
+lowra_status lowra_lora_forward(const lowra_layout* layout, const uint8_t* packed_dev,
+                                const float* absmax_dev, const float* maps_dev, const uint16_t* X_dev,
+                                int32_t M, const uint16_t* A_dev, const uint16_t* B_dev, int32_t r,
+                                float s, uint16_t* Y_dev, void* workspace_dev, size_t workspace_bytes,
+                                void* stream);
+
+/*
+ * Input gradient of the same layer (the base weights are frozen, Section 3, so the only gradient
+ * through the quantised weight is the one with respect to the input):
+ *     dX = dY . deq(Wq) + s * (dY . B^T) . A^T
+ *   dY_dev bf16 [M, N];  dX_dev bf16 [M, K];  other arguments as in lowra_lora_forward.
+ */
+lowra_status lowra_lora_backward_input(const lowra_layout* layout, const uint8_t* packed_dev,
+                                       const float* absmax_dev, const float* maps_dev,
+                                       const uint16_t* dY_dev, int32_t M, const uint16_t* A_dev,
+                                       const uint16_t* B_dev, int32_t r, float s, uint16_t* dX_dev,
+                                       void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/*
+ * Synchronises `stream` and returns the status word that the last forward / backward call wrote
+ * into its workspace: LOWRA_OK, or LOWRA_ERR_TIMEOUT if a bounded wait inside a kernel ran out
+ * (the kernel then released its resources and returned; the output is not valid).
+ */
+lowra_status lowra_device_status(const void* workspace_dev, void* stream);
+
+/*
+ * Diagnostic, not part of the method: C = P . Q^T with P bf16 [M, K], Q bf16 [N, K] (both
+ * row-major, K % 64 == 0), C bf16 [M, N], run through the same tensor-core pipeline as the fused
+ * kernels but with both operands fetched as plain bf16 tiles.  Used to compare "decode, then dense
+ * product" against the fused path.  workspace as above (only the status word is used).
+ */
+lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_dev, int32_t M, int32_t N, int32_t K,
+                            uint16_t* C_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LOWRA_H */

@@ -1,0 +1,262 @@
+"""Thin Python binding of the LowRA B200 hot-path library (``liblowra.so``).
+
+Argument marshalling only: every step of the path (encode, decode, fused dequant + LoRA products)
+runs in the CUDA kernels behind the C ABI declared in ``include/lowra.h``.  PyTorch is used for
+device memory and streams, nothing else.  There is no CPU fallback: if the shared library has
+not been built, or the device is not a B200, the calls raise.
+
+Function names are those of the C ABI.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "liblowra.so")
+
+LOWRA_OK = 0
+(LOWRA_ERR_NULL, LOWRA_ERR_SHAPE, LOWRA_ERR_ALIGN, LOWRA_ERR_PREC, LOWRA_ERR_WORKSPACE,
+ LOWRA_ERR_CUDA, LOWRA_ERR_TIMEOUT, LOWRA_ERR_ARCH) = range(1, 9)
+
+EXPORTS = (
+    "lowra_status_string", "lowra_plan", "lowra_encode", "lowra_decode", "lowra_workspace_bytes",
+    "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
+)
+
+
+class LowraError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+class _CLayout(ctypes.Structure):
+    _fields_ = [
+        ("N", ctypes.c_int32), ("K", ctypes.c_int32), ("block", ctypes.c_int32),
+        ("counts", ctypes.c_int32 * 3),
+        ("seg_off", ctypes.c_uint64 * 3),
+        ("packed_bytes", ctypes.c_uint64),
+        ("precs_dev", ctypes.c_void_p), ("perm_dev", ctypes.c_void_p), ("inv_perm_dev", ctypes.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2502_08141_b200.build` "
+                "(there is no fallback path)")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32, u64p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_uint64)
+        lp = ctypes.POINTER(_CLayout)
+        L.lowra_status_string.argtypes = [ctypes.c_int]
+        L.lowra_status_string.restype = ctypes.c_char_p
+        L.lowra_plan.argtypes = [i32, i32, vp, vp, vp, vp, vp, u64p]
+        L.lowra_plan.restype = ctypes.c_int
+        L.lowra_encode.argtypes = [lp, vp, vp, vp, vp, vp]
+        L.lowra_encode.restype = ctypes.c_int
+        L.lowra_decode.argtypes = [lp, vp, vp, vp, vp, vp]
+        L.lowra_decode.restype = ctypes.c_int
+        L.lowra_workspace_bytes.argtypes = [lp, i32, i32]
+        L.lowra_workspace_bytes.restype = ctypes.c_size_t
+        gemm_args = [lp, vp, vp, vp, vp, i32, vp, vp, i32, ctypes.c_float, vp, vp, ctypes.c_size_t, vp]
+        L.lowra_lora_forward.argtypes = gemm_args
+        L.lowra_lora_forward.restype = ctypes.c_int
+        L.lowra_lora_backward_input.argtypes = gemm_args
+        L.lowra_lora_backward_input.restype = ctypes.c_int
+        L.lowra_device_status.argtypes = [vp, vp]
+        L.lowra_device_status.restype = ctypes.c_int
+        L.lowra_dense_nt.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
+        L.lowra_dense_nt.restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().lowra_status_string(int(code)).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != LOWRA_OK:
+        raise LowraError(code, where)
+
+
+def _stream(stream) -> ctypes.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _ptr(t: Optional[torch.Tensor]) -> ctypes.c_void_p:
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+    if t.dtype != dtype:
+        raise ValueError(f"{name} must be {dtype}, got {t.dtype}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t
+
+
+# ---------------------------------------------------------------------------------------------
+def lowra_plan(precs_host: np.ndarray, K: int) -> dict:
+    """Host-side storage planner. -> dict(perm, inv_perm, counts, seg_off, packed_bytes)."""
+    precs = np.ascontiguousarray(precs_host, dtype=np.uint8)
+    N = int(precs.shape[0])
+    perm = np.empty(max(N, 1), dtype=np.int32)
+    inv = np.empty(max(N, 1), dtype=np.int32)
+    counts = (ctypes.c_int32 * 3)()
+    seg = (ctypes.c_uint64 * 3)()
+    total = ctypes.c_uint64(0)
+    code = lib().lowra_plan(N, int(K), precs.ctypes.data, perm.ctypes.data, inv.ctypes.data,
+                            ctypes.addressof(counts), ctypes.addressof(seg), ctypes.byref(total))
+    _check(code, "lowra_plan")
+    return dict(perm=perm[:N], inv_perm=inv[:N], counts=[int(c) for c in counts],
+                seg_off=[int(s) for s in seg], packed_bytes=int(total.value))
+
+
+class Layout:
+    """A ``lowra_layout`` plus the device arrays it points to (kept alive here)."""
+
+    def __init__(self, precs_host: np.ndarray, K: int, device="cuda"):
+        self.precs_host = np.ascontiguousarray(precs_host, dtype=np.uint8)
+        self.N, self.K = int(self.precs_host.shape[0]), int(K)
+        self.plan = lowra_plan(self.precs_host, K)
+        self.device = torch.device(device)
+        self.precs = torch.from_numpy(self.precs_host).to(self.device)
+        self.perm = torch.from_numpy(self.plan["perm"]).to(self.device)
+        self.inv_perm = torch.from_numpy(self.plan["inv_perm"]).to(self.device)
+        self.packed_bytes = self.plan["packed_bytes"]
+        c = _CLayout()
+        c.N, c.K, c.block = self.N, self.K, 64
+        for i in range(3):
+            c.counts[i] = self.plan["counts"][i]
+            c.seg_off[i] = self.plan["seg_off"][i]
+        c.packed_bytes = self.packed_bytes
+        c.precs_dev = self.precs.data_ptr()
+        c.perm_dev = self.perm.data_ptr()
+        c.inv_perm_dev = self.inv_perm.data_ptr()
+        self.c = c
+
+    @property
+    def ref(self):
+        return ctypes.byref(self.c)
+
+
+def lowra_encode(layout: Layout, W: torch.Tensor, thresholds: torch.Tensor,
+                 packed: Optional[torch.Tensor] = None, absmax: Optional[torch.Tensor] = None,
+                 stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """W fp32 [N,K], thresholds fp32 [N,16] -> packed uint8 [packed_bytes], absmax fp32 [N,K/64]."""
+    _dev(W, torch.float32, "W")
+    _dev(thresholds, torch.float32, "thresholds")
+    if tuple(W.shape) != (layout.N, layout.K) or tuple(thresholds.shape) != (layout.N, 16):
+        raise ValueError("shape mismatch")
+    if packed is None:
+        packed = torch.empty(max(layout.packed_bytes, 16), dtype=torch.uint8, device=W.device)
+    if absmax is None:
+        absmax = torch.empty((layout.N, layout.K // 64), dtype=torch.float32, device=W.device)
+    _dev(packed, torch.uint8, "packed")
+    _dev(absmax, torch.float32, "absmax")
+    code = lib().lowra_encode(layout.ref, _ptr(W), _ptr(thresholds), _ptr(packed), _ptr(absmax), _stream(stream))
+    _check(code, "lowra_encode")
+    return packed, absmax
+
+
+def lowra_decode(layout: Layout, packed: torch.Tensor, absmax: torch.Tensor, maps: torch.Tensor,
+                 out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """-> bf16 [N, K], original row order."""
+    _dev(packed, torch.uint8, "packed")
+    _dev(absmax, torch.float32, "absmax")
+    _dev(maps, torch.float32, "maps")
+    if out is None:
+        out = torch.empty((layout.N, layout.K), dtype=torch.bfloat16, device=packed.device)
+    _dev(out, torch.bfloat16, "out")
+    code = lib().lowra_decode(layout.ref, _ptr(packed), _ptr(absmax), _ptr(maps), _ptr(out), _stream(stream))
+    _check(code, "lowra_decode")
+    return out
+
+
+def lowra_workspace_bytes(layout: Layout, M: int, r: int) -> int:
+    return int(lib().lowra_workspace_bytes(layout.ref, int(M), int(r)))
+
+
+def _workspace(layout: Layout, M: int, r: int, device) -> torch.Tensor:
+    n = lowra_workspace_bytes(layout, M, r)
+    if n == 0:
+        raise LowraError(LOWRA_ERR_SHAPE, "lowra_workspace_bytes")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def lowra_lora_forward(layout: Layout, packed, absmax, maps, X, A, B, s: float,
+                       Y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                       stream=None) -> torch.Tensor:
+    """Y = X . deq(Wq)^T + s (X . A) . B ; X bf16 [M,K], A bf16 [K,r], B bf16 [r,N] -> Y bf16 [M,N]."""
+    for t, n in ((X, "X"), (A, "A"), (B, "B")):
+        _dev(t, torch.bfloat16, n)
+    M, r = int(X.shape[0]), int(A.shape[1])
+    if tuple(X.shape) != (M, layout.K) or tuple(A.shape) != (layout.K, r) or tuple(B.shape) != (r, layout.N):
+        raise ValueError("shape mismatch")
+    if Y is None:
+        Y = torch.empty((M, layout.N), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = _workspace(layout, M, r, X.device)
+    code = lib().lowra_lora_forward(layout.ref, _ptr(packed), _ptr(absmax), _ptr(maps), _ptr(X), M, _ptr(A),
+                                    _ptr(B), r, ctypes.c_float(s), _ptr(Y), _ptr(workspace),
+                                    workspace.numel(), _stream(stream))
+    _check(code, "lowra_lora_forward")
+    return Y
+
+
+def lowra_lora_backward_input(layout: Layout, packed, absmax, maps, dY, A, B, s: float,
+                              dX: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                              stream=None) -> torch.Tensor:
+    """dX = dY . deq(Wq) + s (dY . B^T) . A^T ; dY bf16 [M,N] -> dX bf16 [M,K]."""
+    for t, n in ((dY, "dY"), (A, "A"), (B, "B")):
+        _dev(t, torch.bfloat16, n)
+    M, r = int(dY.shape[0]), int(A.shape[1])
+    if tuple(dY.shape) != (M, layout.N) or tuple(A.shape) != (layout.K, r) or tuple(B.shape) != (r, layout.N):
+        raise ValueError("shape mismatch")
+    if dX is None:
+        dX = torch.empty((M, layout.K), dtype=torch.bfloat16, device=dY.device)
+    if workspace is None:
+        workspace = _workspace(layout, M, r, dY.device)
+    code = lib().lowra_lora_backward_input(layout.ref, _ptr(packed), _ptr(absmax), _ptr(maps), _ptr(dY), M,
+                                           _ptr(A), _ptr(B), r, ctypes.c_float(s), _ptr(dX), _ptr(workspace),
+                                           workspace.numel(), _stream(stream))
+    _check(code, "lowra_lora_backward_input")
+    return dX
+
+
+def lowra_device_status(workspace: torch.Tensor, stream=None) -> int:
+    """Synchronises the stream and returns the status word of the last fused call."""
+    return int(lib().lowra_device_status(_ptr(workspace), _stream(stream)))
+
+
+def lowra_dense_nt(P: torch.Tensor, Q: torch.Tensor, C: Optional[torch.Tensor] = None,
+                   workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Diagnostic: C = P . Q^T through the same tensor-core pipeline (both operands plain bf16)."""
+    _dev(P, torch.bfloat16, "P")
+    _dev(Q, torch.bfloat16, "Q")
+    M, K = P.shape
+    N = Q.shape[0]
+    if C is None:
+        C = torch.empty((M, N), dtype=torch.bfloat16, device=P.device)
+    if workspace is None:
+        workspace = torch.empty(256, dtype=torch.uint8, device=P.device)
+    code = lib().lowra_dense_nt(_ptr(P), _ptr(Q), int(M), int(N), int(K), _ptr(C), _ptr(workspace),
+                                workspace.numel(), _stream(stream))
+    _check(code, "lowra_dense_nt")
+    return C

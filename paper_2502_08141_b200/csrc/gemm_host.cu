@@ -1,0 +1,205 @@
+// Host side of lowra_lora_forward / lowra_lora_backward_input / lowra_dense_nt: validation, workspace
+// carve-up, TMA descriptors, launches.
+#include <cudaTypedefs.h>
+#include <string.h>
+
+#include "gemm_params.cuh"
+
+namespace lowra {
+
+namespace {
+
+constexpr size_t kStatusBytes = 256;
+
+size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+struct Workspace {
+    size_t off_T, off_F2, off_info, total;
+    int rp;
+};
+
+bool rank_ok(int r) { return r >= 16 && r <= 128 && r % 16 == 0; }
+
+Workspace plan_workspace(int N, int K, int M, int r) {
+    Workspace w;
+    w.rp = (r + 63) / 64 * 64;
+    const int big = N > K ? N : K;
+    w.off_T = kStatusBytes;
+    w.off_F2 = w.off_T + align256((size_t)M * w.rp * 2);
+    w.off_info = w.off_F2 + align256((size_t)big * w.rp * 2);
+    w.total = w.off_info + align256((size_t)((N + 127) / 128 * 128) * 4);
+    return w;
+}
+
+PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
+    static PFN_cuTensorMapEncodeTiled_v12000 fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(p);
+    }
+    return fn;
+}
+
+// bf16 matrix [rows, cols] row-major with pitch `ld` elements; box = 64 columns x box_rows rows,
+// 128-byte swizzle, out-of-range elements read as zero.
+bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, uint64_t ld, uint32_t box_rows) {
+    PFN_cuTensorMapEncodeTiled_v12000 fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kTileC, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult rc = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS;
+}
+
+lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* packed, const float* absmax,
+                      const float* maps, const uint16_t* act, int32_t M, const uint16_t* A, const uint16_t* B,
+                      int32_t r, float s, uint16_t* out, void* workspace, size_t workspace_bytes, void* stream_v) {
+    lowra_status st = check_layout(layout);
+    if (st != LOWRA_OK) return st;
+    if (!packed || !absmax || !maps || !act || !A || !B || !out || !workspace) return LOWRA_ERR_NULL;
+    const int N = layout->N, K = layout->K;
+    if (M < 1 || !rank_ok(r) || N % 8 != 0 || N >= (1 << 23)) return LOWRA_ERR_SHAPE;
+    if (!aligned16(packed) || !aligned16(absmax) || !aligned16(maps) || !aligned16(act) || !aligned16(A) ||
+        !aligned16(B) || !aligned16(out))
+        return LOWRA_ERR_ALIGN;
+    const Workspace w = plan_workspace(N, K, M, r);
+    if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LOWRA_ERR_WORKSPACE;
+    st = check_device();
+    if (st != LOWRA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
+    uint16_t* F2 = reinterpret_cast<uint16_t*>(ws + w.off_F2);
+    uint32_t* rowinfo = reinterpret_cast<uint32_t*>(ws + w.off_info);
+    uint32_t* status = reinterpret_cast<uint32_t*>(ws);
+
+    // ---- prologue
+    PrepParams P;
+    memset(&P, 0, sizeof(P));
+    P.In = act;
+    P.M = M;
+    P.r = r;
+    P.rp = w.rp;
+    P.s = s;
+    P.T = T;
+    P.Dst = F2;
+    P.precs = layout->precs_dev;
+    P.inv_perm = layout->inv_perm_dev;
+    P.rowinfo = rowinfo;
+    P.N = N;
+    P.status = status;
+    if (!backward) {
+        P.C = K; P.F = A; P.f_is_A = 1;            // T = s X A
+        P.Src = B; P.R = N; P.src_transposed = 1;  // Bt[n, j] = B[j, n]
+        P.group = 128;
+    } else {
+        P.C = N; P.F = B; P.f_is_A = 0;            // U = s dY B^T
+        P.Src = A; P.R = K; P.src_transposed = 0;  // Ap[k, j] = A[k, j]
+        P.group = 64;
+    }
+    P.blocksA = (M + kPrepTokens - 1) / kPrepTokens;
+    P.blocksB = 32;
+    P.blocksC = ((N + P.group - 1) / P.group + 3) / 4;
+    st = launch_prep(P, stream);
+    if (st != LOWRA_OK) return st;
+
+    // ---- fused kernel
+    GemmParams G;
+    memset(&G, 0, sizeof(G));
+    G.L = make_row_layout(layout);
+    G.packed = packed;
+    G.absmax = absmax;
+    G.maps = maps;
+    G.rowinfo = rowinfo;
+    G.out = out;
+    G.status = status;
+    G.M = M;
+    G.R = backward ? K : N;
+    G.C = backward ? N : K;
+    G.ld_out = G.R;
+    G.main_blocks = (G.C + kTileC - 1) / kTileC;
+    G.lora_blocks = w.rp / kTileC;
+    G.tiles_r = (G.R + kTileR - 1) / kTileR;
+    G.tiles_t = (M + kTileT - 1) / kTileT;
+    CUtensorMap tmB, tmB2, tmA2;
+    if (!make_map(&tmB, act, (uint64_t)M, (uint64_t)G.C, (uint64_t)G.C, kTileT)) return LOWRA_ERR_CUDA;
+    if (!make_map(&tmB2, T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
+    if (!make_map(&tmA2, F2, (uint64_t)G.R, (uint64_t)w.rp, (uint64_t)w.rp, kTileR)) return LOWRA_ERR_CUDA;
+    return launch_fused(backward ? kModeBackward : kModeForward, G, tmB, tmB2, tmA2, stream);
+}
+
+__global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
+
+}  // namespace
+}  // namespace lowra
+
+extern "C" size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r) {
+    using namespace lowra;
+    if (!layout || layout->N < 1 || layout->K < 1 || M < 1 || !rank_ok(r)) return 0;
+    return plan_workspace(layout->N, layout->K, M, r).total;
+}
+
+extern "C" lowra_status lowra_lora_forward(const lowra_layout* layout, const uint8_t* packed_dev,
+                                           const float* absmax_dev, const float* maps_dev, const uint16_t* X_dev,
+                                           int32_t M, const uint16_t* A_dev, const uint16_t* B_dev, int32_t r, float s,
+                                           uint16_t* Y_dev, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    return lowra::run_lora(false, layout, packed_dev, absmax_dev, maps_dev, X_dev, M, A_dev, B_dev, r, s, Y_dev,
+                           workspace_dev, workspace_bytes, stream);
+}
+
+extern "C" lowra_status lowra_lora_backward_input(const lowra_layout* layout, const uint8_t* packed_dev,
+                                                  const float* absmax_dev, const float* maps_dev,
+                                                  const uint16_t* dY_dev, int32_t M, const uint16_t* A_dev,
+                                                  const uint16_t* B_dev, int32_t r, float s, uint16_t* dX_dev,
+                                                  void* workspace_dev, size_t workspace_bytes, void* stream) {
+    return lowra::run_lora(true, layout, packed_dev, absmax_dev, maps_dev, dY_dev, M, A_dev, B_dev, r, s, dX_dev,
+                           workspace_dev, workspace_bytes, stream);
+}
+
+extern "C" lowra_status lowra_device_status(const void* workspace_dev, void* stream) {
+    if (!workspace_dev) return LOWRA_ERR_NULL;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return LOWRA_ERR_CUDA;
+    uint32_t word = 0;
+    if (cudaMemcpy(&word, workspace_dev, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return LOWRA_ERR_CUDA;
+    return (lowra_status)word;
+}
+
+extern "C" lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_dev, int32_t M, int32_t N, int32_t K,
+                                       uint16_t* C_dev, void* workspace_dev, size_t workspace_bytes, void* stream_v) {
+    using namespace lowra;
+    if (!P_dev || !Q_dev || !C_dev || !workspace_dev) return LOWRA_ERR_NULL;
+    if (M < 1 || N < 1 || K < 64 || K % 64 != 0) return LOWRA_ERR_SHAPE;
+    if (!aligned16(P_dev) || !aligned16(Q_dev) || !aligned16(C_dev)) return LOWRA_ERR_ALIGN;
+    if (workspace_bytes < kStatusBytes || (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) != 0)
+        return LOWRA_ERR_WORKSPACE;
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    uint32_t* status = reinterpret_cast<uint32_t*>(workspace_dev);
+    clear_status_kernel<<<1, 1, 0, stream>>>(status);
+
+    GemmParams G;
+    memset(&G, 0, sizeof(G));
+    G.out = C_dev;
+    G.status = status;
+    G.M = M;
+    G.R = N;
+    G.C = K;
+    G.ld_out = N;
+    G.main_blocks = K / kTileC;
+    G.lora_blocks = 0;
+    G.tiles_r = (N + kTileR - 1) / kTileR;
+    G.tiles_t = (M + kTileT - 1) / kTileT;
+    CUtensorMap tmB, tmA2;
+    if (!make_map(&tmB, P_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, kTileT)) return LOWRA_ERR_CUDA;
+    if (!make_map(&tmA2, Q_dev, (uint64_t)N, (uint64_t)K, (uint64_t)K, kTileR)) return LOWRA_ERR_CUDA;
+    return launch_fused(kModeDense, G, tmB, tmB, tmA2, stream);
+}

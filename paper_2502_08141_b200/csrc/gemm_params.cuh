@@ -1,0 +1,78 @@
+// Launch parameters shared by the prologue kernel, the fused tensor-core kernel and their host code.
+#pragma once
+
+#include <cuda.h>
+
+#include "lowra_common.cuh"
+
+namespace lowra {
+
+// ---- prologue ------------------------------------------------------------------------------
+constexpr int kPrepThreads = 128;
+constexpr int kPrepTokens = 32;   // tokens per down-projection CTA
+
+struct PrepParams {
+    // (A) T[m, j] = bf16(s * sum_c In[m, c] * F(c, j)),  T is [M, rp]
+    const uint16_t* In;   // [M, C] bf16
+    const uint16_t* F;    // f_is_A: A [C, r] (F(c,j) = F[c*r + j]);  else B [r, C] (F(c,j) = F[j*C + c])
+    uint16_t* T;
+    int M, C, r, rp, f_is_A;
+    float s;
+    // (B) Dst [R, rp]: src_transposed: Dst[n, j] = Src[j*R + n];  else Dst[k, j] = Src[k*r + j]
+    const uint16_t* Src;
+    uint16_t* Dst;
+    int R, src_transposed;
+    // (C) per-group precision order: rowinfo[g * group + i] describes the i-th row of group g in
+    // precision order: bits 0-6 row offset inside the group, 7-8 class (3 = past N), 9-31 stored position
+    const uint8_t* precs;
+    const int32_t* inv_perm;
+    uint32_t* rowinfo;    // [ceil(N / group) * group]
+    int N, group;
+    uint32_t* status;
+    int blocksA, blocksB, blocksC;
+};
+
+lowra_status launch_prep(const PrepParams& P, cudaStream_t stream);
+
+// ---- fused kernel --------------------------------------------------------------------------
+constexpr int kTileR = 128;       // rows of the MMA A operand per tile (output channels fwd, input features bwd)
+constexpr int kTileT = 256;       // tokens per tile (MMA N)
+constexpr int kTileC = 64;        // contraction elements per pipeline stage (= one absmax block, = 128 bytes of bf16)
+constexpr int kStages = 4;
+constexpr int kProducerWarps = 8;
+constexpr int kFirstEpilogueWarp = 2;
+constexpr int kFirstProducerWarp = 6;
+constexpr int kGemmThreads = 32 * (kFirstProducerWarp + kProducerWarps);
+constexpr int kTmemCols = 512;    // two 128 x 256 fp32 accumulators
+
+constexpr int kModeForward = 0, kModeBackward = 1, kModeDense = 2;
+
+struct GemmParams {
+    RowLayout L;
+    const uint8_t* packed;
+    const float* absmax;
+    const float* maps;
+    const uint32_t* rowinfo;  // from the prologue
+    uint16_t* out;          // [M, ld_out] bf16
+    uint32_t* status;
+    int M;                  // tokens
+    int R;                  // A-operand rows in total: N (forward, dense) or K (backward)
+    int C;                  // main contraction length: K (forward, dense) or N (backward)
+    int ld_out;             // = R
+    int main_blocks;        // ceil(C / 64)
+    int lora_blocks;        // rp / 64 (0 in dense mode)
+    int tiles_r, tiles_t;
+};
+
+constexpr uint32_t kSmemA = kTileR * kTileC * 2;   // 16 KB
+constexpr uint32_t kSmemB = kTileT * kTileC * 2;   // 32 KB
+constexpr uint32_t kSmemStage = kSmemA + kSmemB;
+constexpr uint32_t kSmemOut = 32 * kTileR * 2;     // epilogue staging: 32 tokens x 128 channels bf16
+constexpr uint32_t kSmemLut4 = 16 * kProducerWarps * 32 * 4;  // per-thread 16-entry fp32 tables
+constexpr uint32_t kSmemBarriers = 1024;
+constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kStages * kSmemStage + kSmemOut + kSmemLut4 + kSmemBarriers;
+
+lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmB2,
+                          const CUtensorMap& tmA2, cudaStream_t stream);
+
+}  // namespace lowra

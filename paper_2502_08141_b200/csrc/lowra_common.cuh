@@ -1,0 +1,65 @@
+// Shared declarations of the CUDA path: launch-parameter structs, host-side validation helpers and
+// a few device intrinsics.  Nothing in here is used by, or taken from, the CPU oracle.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "lowra.h"
+
+namespace lowra {
+
+constexpr int kBlock = 64;        // elements per absmax block (Section 4.1, groupwise normalisation)
+constexpr int kTableStride = 16;  // fp32 entries per row in the mapping / threshold tables
+constexpr int kNumSMs = 148;      // B200
+
+// Everything a kernel needs to find a stored row; passed by value as a kernel argument.
+struct RowLayout {
+    int32_t N, K, nb;             // nb = K / 64
+    int32_t class_start[4];       // first stored row of each precision class; [3] = N
+    uint64_t seg_off[3];          // byte offset of each class in the packed buffer
+    const uint8_t* precs;         // [N] original order
+    const int32_t* perm;          // stored -> original
+    const int32_t* inv_perm;      // original -> stored
+};
+
+lowra_status check_layout(const lowra_layout* L);
+lowra_status check_device();
+RowLayout make_row_layout(const lowra_layout* L);
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// -------------------------------------------------------------------------------------------
+// device helpers
+// -------------------------------------------------------------------------------------------
+__device__ __forceinline__ int class_of_stored_row(const RowLayout& L, int p) {
+    return (p >= L.class_start[1]) + (p >= L.class_start[2]);
+}
+
+// Two fp32 -> packed bf16x2, round to nearest even; `lo` lands in bits [0,16).
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ float4 ld_stream_f4(const void* p) {
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+
+__device__ __forceinline__ void st_stream_v4(void* p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+}  // namespace lowra

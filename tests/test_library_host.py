@@ -1,0 +1,99 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every declared symbol, and its host
+logic (storage planner, argument validation that happens before any device work) behaves."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2502_08141_b200 import build
+    build.build()
+    import paper_2502_08141_b200 as lw
+    return lw
+
+
+def test_library_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "lowra.h")).read()
+    declared = set(re.findall(r"\b(lowra_[a-z_]+)\s*\(", header))
+    assert declared == set(lib.EXPORTS)
+    L = lib.lib()
+    for name in declared:
+        assert hasattr(L, name), name
+
+
+def test_status_strings(lib):
+    assert lib.status_string(0) == "ok"
+    assert len({lib.status_string(c) for c in range(9)}) == 9
+
+
+def test_plan_matches_oracle_layout(lib):
+    for N, K, mix, mid in ((1000, 256, {1: 0.3, 2: 0.5, 4: 0.2}, 1), (77, 128, {4: 1.0}, 2),
+                           (512, 512, {1: 0.5, 2: 0.5}, 3), (5, 1280, {2: 1.0}, 4)):
+        precs = si.precisions(N, mix, matrix_id=mid)
+        got = lib.lowra_plan(precs, K)
+        want = oracle.plan(precs, K)
+        assert np.array_equal(got["perm"], want["perm"])
+        assert np.array_equal(got["inv_perm"], want["inv_perm"])
+        assert got["counts"] == list(want["counts"])
+        assert got["seg_off"] == [int(x) for x in want["seg_off"]]
+        assert got["packed_bytes"] == want["packed_bytes"] == sum(K * int(b) // 8 for b in precs)
+
+
+def test_plan_rejects_bad_input(lib):
+    with pytest.raises(lib.LowraError) as e:
+        lib.lowra_plan(np.array([1, 2, 3], np.uint8), 128)
+    assert e.value.code == lib.LOWRA_ERR_PREC
+    with pytest.raises(lib.LowraError) as e:
+        lib.lowra_plan(np.array([1, 2, 4], np.uint8), 100)
+    assert e.value.code == lib.LOWRA_ERR_SHAPE
+    with pytest.raises(lib.LowraError) as e:
+        lib.lowra_plan(np.zeros(0, np.uint8), 128)
+    assert e.value.code == lib.LOWRA_ERR_SHAPE
+
+
+def test_validation_runs_before_any_device_work(lib):
+    """Null pointers / bad shapes are refused on the host, so this needs no GPU."""
+    L = lib.lib()
+    lay = lib._CLayout()
+    lay.N, lay.K, lay.block = 8, 128, 64
+    lay.counts[0] = 8
+    lay.packed_bytes = 8 * 128 // 8
+    lay.seg_off[1] = lay.seg_off[2] = lay.packed_bytes
+    # null device arrays in the layout
+    assert L.lowra_decode(ctypes.byref(lay), None, None, None, None, None) == lib.LOWRA_ERR_NULL
+    lay.precs_dev = lay.perm_dev = lay.inv_perm_dev = 4096   # fake, never dereferenced
+    assert L.lowra_decode(ctypes.byref(lay), None, None, None, None, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_encode(ctypes.byref(lay), 4096, 4096, 4096 + 8, 4096, None) == lib.LOWRA_ERR_ALIGN
+    lay.block = 32
+    assert L.lowra_decode(ctypes.byref(lay), 4096, 4096, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
+    lay.block = 64
+    lay.counts[0] = 7
+    assert L.lowra_decode(ctypes.byref(lay), 4096, 4096, 4096, 4096, None) == lib.LOWRA_ERR_PREC
+    lay.counts[0] = 8
+    assert L.lowra_workspace_bytes(ctypes.byref(lay), 16, 16) > 256
+    assert L.lowra_workspace_bytes(ctypes.byref(lay), 16, 24) == 0      # rank must be a multiple of 16
+    assert L.lowra_workspace_bytes(ctypes.byref(lay), 0, 16) == 0
+    args = [ctypes.byref(lay), 4096, 4096, 4096, 4096, 16, 4096, 4096, 24, ctypes.c_float(1.0), 4096, 4096, 1 << 20, None]
+    assert L.lowra_lora_forward(*args) == lib.LOWRA_ERR_SHAPE
+    args[8] = 16
+    args[12] = 16                                                        # workspace too small
+    assert L.lowra_lora_forward(*args) == lib.LOWRA_ERR_WORKSPACE
+    assert L.lowra_lora_backward_input(*args) == lib.LOWRA_ERR_WORKSPACE
+    assert L.lowra_device_status(None, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_dense_nt(4096, 4096, 16, 16, 100, 4096, 4096, 256, None) == lib.LOWRA_ERR_SHAPE
+
+
+def test_missing_library_fails_loudly(lib, monkeypatch, tmp_path):
+    monkeypatch.setattr(lib, "_lib", None)
+    monkeypatch.setattr(lib, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(RuntimeError, match="no fallback"):
+        lib.lib()
