@@ -1,0 +1,443 @@
+#!/usr/bin/env python
+"""Benchmark of the LowRA quantized-LoRA hot path on B200.
+
+A *step* is one pass of the whole hot path over one Llama-7B-shaped decoder layer (seven weight
+matrices, 4096 tokens, LoRA rank 64, precision mix averaging 1.5 bits): for every matrix
+lowra_encode, lowra_decode, lowra_lora_forward and lowra_lora_backward_input, through the C ABI.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line.  `value` is the fused dequant+LoRA product throughput of the step (algorithmic
+FLOPs of the 7 forward + 7 backward products divided by the time of the WHOLE step, encode and decode
+included), measured with CUDA events and inputs resident in HBM; `phases` breaks the step down
+(encode / decode in GB/s, forward / backward in TFLOP/s); `e2e` repeats the step with host buffers and
+the host<->device copies inside the timed region; `roofline` is for the dominant kernel (the fused
+tensor-core kernel); `cpu_baseline` times the CPU oracle on a bounded sample of the same workload.
+
+With N > 1 (torchrun) every rank runs the same layer shapes on its own seeded weights (independent
+problems, no data-path collective; weak scaling) and rank 0 reports the aggregate.
+
+`--impl reference` times the CPU oracle alone (there is no reference code for this paper).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import synth_inputs as si  # noqa: E402
+
+WORKLOAD = 3  # Llama-7B decoder layer, 4096 tokens, avg 1.5 bits
+METRIC = "fused dequant+LoRA fwd+bwd throughput over one Llama-7B layer step (encode+decode+fwd+bwd)"
+UNIT = "TFLOP/s"
+
+
+def gemm_flops(M, N, K, r):
+    """Algorithmic FLOPs of one forward (or one backward-input) call."""
+    return 2.0 * M * N * K + 2.0 * M * r * (K + N)
+
+
+def decode_bytes(N, K, bits):
+    return N * K * (bits / 8.0 + 4.0 / 64.0 + 2.0)   # packed codes + absmax in, bf16 out (tables: < 0.1 %, not counted)
+
+
+def encode_bytes(N, K, bits):
+    return N * K * (4.0 + bits / 8.0 + 4.0 / 64.0)
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm=float(p["hbm_gbs"]), tensor_burst=float(p["bf16_tflops"]),
+                    tensor_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm=6650.0, tensor_burst=1590.0, tensor_sustained=1400.0, source="fallback")
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks sampling
+# --------------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        for ts, line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                clk, mx = float(parts[1]), float(parts[2])
+            except ValueError:
+                continue
+            if t0 - 0.05 <= ts <= t1 + 0.15:
+                sm.append(clk)
+                smax.append(mx)
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        if not sm:  # region shorter than the sampling period: take everything seen
+            for ts, line in self.lines:
+                parts = [p.strip() for p in line.split(",")]
+                try:
+                    sm.append(float(parts[1])); smax.append(float(parts[2]))
+                except Exception:
+                    pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------------
+# workload
+# --------------------------------------------------------------------------------------------------
+def make_host_inputs(cfg, rank: int):
+    """Seeded host inputs of one layer (matrix ids offset by the rank, so ranks hold different layers)."""
+    M, r = cfg.tokens[0], cfg.rank
+
+    def one(mat):
+        mid = mat.matrix_id + 7 * rank
+        W = si.weights(mat.N, mat.K, matrix_id=mid, kind=cfg.weight_kind)
+        precs = si.precisions(mat.N, cfg.mix, matrix_id=mid)
+        maps, thr = si.standin_codebooks(precs, matrix_id=mid)
+        A, B = si.lora_factors(mat.K, mat.N, r, matrix_id=mid)
+        return dict(name=mat.name, N=mat.N, K=mat.K, W=W, precs=precs, maps=maps, thr=thr, A=A, B=B)
+
+    with ThreadPoolExecutor(max_workers=min(8, len(cfg.matrices))) as ex:
+        mats = list(ex.map(one, cfg.matrices))
+    # one activation / gradient buffer per distinct width, shared by the matrices of that width
+    acts = {}
+    for m in mats:
+        if m["K"] not in acts:
+            acts[m["K"]] = si.activations(M, m["K"], matrix_id=100 + rank)
+        if m["N"] not in acts:
+            acts[m["N"]] = si.activations(M, m["N"], matrix_id=100 + rank)
+    return mats, acts
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2502_08141_b200 as lw
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    lw.lib()
+
+    cfg = si.config(WORKLOAD)
+    M, r, s = cfg.tokens[0], cfg.rank, cfg.s
+    bits = si.avg_bits(cfg.mix)
+    mats, acts = make_host_inputs(cfg, rank)
+
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    bfv = lambda t: t.view(torch.bfloat16)
+    # ---- device-resident problem
+    dev = []
+    for m in mats:
+        layout = lw.Layout(m["precs"], m["K"])
+        d = dict(m=m, layout=layout,
+                 W=torch.from_numpy(m["W"]).cuda(), thr=torch.from_numpy(m["thr"]).cuda(),
+                 maps=torch.from_numpy(m["maps"]).cuda(),
+                 A=bfv(torch.from_numpy(m["A"].view(np.int16)).cuda()), B=bfv(torch.from_numpy(m["B"].view(np.int16)).cuda()),
+                 packed=torch.empty(max(layout.packed_bytes, 16), dtype=torch.uint8, device="cuda"),
+                 absmax=torch.empty((m["N"], m["K"] // 64), dtype=torch.float32, device="cuda"),
+                 What=torch.empty((m["N"], m["K"]), dtype=torch.bfloat16, device="cuda"),
+                 Y=torch.empty((M, m["N"]), dtype=torch.bfloat16, device="cuda"),
+                 dX=torch.empty((M, m["K"]), dtype=torch.bfloat16, device="cuda"),
+                 ws=torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda"))
+        dev.append(d)
+    act_dev = {k: bfv(torch.from_numpy(v.view(np.int16)).cuda()) for k, v in acts.items()}
+    stream = torch.cuda.current_stream()
+
+    def step(record=None):
+        """One pass; `record` (a list) receives (phase, event_start, event_end) per call."""
+        def timed(phase, fn):
+            if record is None:
+                fn()
+                return
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream); fn(); e1.record(stream)
+            record.append((phase, e0, e1))
+        for d in dev:
+            timed("encode", lambda: lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"]))
+        for d in dev:
+            timed("decode", lambda: lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"]))
+        for d in dev:
+            timed("forward", lambda: lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"],
+                                                           act_dev[d["m"]["K"]], d["A"], d["B"], s, Y=d["Y"], workspace=d["ws"]))
+        for d in dev:
+            timed("backward", lambda: lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"],
+                                                                   act_dev[d["m"]["N"]], d["A"], d["B"], s, dX=d["dX"],
+                                                                   workspace=d["ws"]))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    for d in dev:
+        st = lw.lowra_device_status(d["ws"])
+        if st != 0:
+            raise SystemExit(f"device status {st} after warm-up")
+
+    # ---- timed region: exactly K steps, device timing with CUDA events, max over ranks
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    barrier()
+    records = []
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    ev0.record(stream)
+    for _ in range(args.steps):
+        step(records)
+    ev1.record(stream)
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    total_ms = ev0.elapsed_time(ev1)
+    if world > 1:
+        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+
+    flops_step = sum(2 * gemm_flops(M, d["m"]["N"], d["m"]["K"], r) for d in dev)
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+
+    phase_ms = {}
+    for phase, e0, e1 in records:
+        phase_ms[phase] = phase_ms.get(phase, 0.0) + e0.elapsed_time(e1)
+    for k in phase_ms:
+        phase_ms[k] /= args.steps
+    elems = sum(d["m"]["N"] * d["m"]["K"] for d in dev)
+    P = peaks()
+    dec_gbs = sum(decode_bytes(d["m"]["N"], d["m"]["K"], bits) for d in dev) / (phase_ms["decode"] * 1e-3) / 1e9
+    enc_gbs = sum(encode_bytes(d["m"]["N"], d["m"]["K"], bits) for d in dev) / (phase_ms["encode"] * 1e-3) / 1e9
+    fwd_tf = flops_step / 2 / (phase_ms["forward"] * 1e-3) / 1e12
+    bwd_tf = flops_step / 2 / (phase_ms["backward"] * 1e-3) / 1e12
+    phases = {
+        "encode": {"ms": phase_ms["encode"], "GB/s": enc_gbs, "frac_hbm": enc_gbs / P["hbm"]},
+        "decode": {"ms": phase_ms["decode"], "GB/s": dec_gbs, "frac_hbm": dec_gbs / P["hbm"]},
+        "forward": {"ms": phase_ms["forward"], "TFLOP/s": fwd_tf, "frac_tensor_burst": fwd_tf / P["tensor_burst"]},
+        "backward_input": {"ms": phase_ms["backward"], "TFLOP/s": bwd_tf, "frac_tensor_burst": bwd_tf / P["tensor_burst"]},
+    }
+    # dominant kernel: the fused tensor-core kernel (forward + backward launches), timed as whole calls
+    fused_ms = phase_ms["forward"] + phase_ms["backward"]
+    achieved = flops_step / (fused_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "kernel": "fused_kernel (forward + backward-input calls, prologue included)",
+                "achieved": achieved, "peak": P["tensor_sustained"], "unit": "TFLOP/s",
+                "frac": achieved / P["tensor_sustained"], "peak_burst": P["tensor_burst"],
+                "frac_burst": achieved / P["tensor_burst"], "peak_source": P["source"] + " (sustained: timed inside a long step)",
+                "traffic": None}
+
+    # ---- end to end: host buffers, pinned, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        host = []
+        for m in mats:
+            host.append(dict(W=pin(m["W"]), thr=pin(m["thr"]), maps=pin(m["maps"]), A=pin(m["A"].view(np.int16)),
+                             B=pin(m["B"].view(np.int16)),
+                             Y=torch.empty((M, m["N"]), dtype=torch.bfloat16).pin_memory(),
+                             dX=torch.empty((M, m["K"]), dtype=torch.bfloat16).pin_memory()))
+        act_host = {k: pin(v.view(np.int16)) for k, v in acts.items()}
+        h2d = sum(h[k].numel() * h[k].element_size() for h in host for k in ("W", "thr", "maps", "A", "B")) \
+            + sum(2 * act_host[d["m"]["K"]].numel() + 2 * act_host[d["m"]["N"]].numel() for d in dev)
+        d2h = sum(h[k].numel() * h[k].element_size() for h in host for k in ("Y", "dX"))
+
+        def e2e_step():
+            for d, h in zip(dev, host):
+                d["W"].copy_(h["W"], non_blocking=True); d["thr"].copy_(h["thr"], non_blocking=True)
+                d["maps"].copy_(h["maps"], non_blocking=True)
+                d["A"].view(torch.int16).copy_(h["A"], non_blocking=True); d["B"].view(torch.int16).copy_(h["B"], non_blocking=True)
+                x = act_dev[d["m"]["K"]]; x.view(torch.int16).copy_(act_host[d["m"]["K"]], non_blocking=True)
+                g = act_dev[d["m"]["N"]]; g.view(torch.int16).copy_(act_host[d["m"]["N"]], non_blocking=True)
+                lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"])
+                lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"])
+                lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], x, d["A"], d["B"], s, Y=d["Y"], workspace=d["ws"])
+                lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], g, d["A"], d["B"], s, dX=d["dX"], workspace=d["ws"])
+                h["Y"].copy_(d["Y"], non_blocking=True); h["dX"].copy_(d["dX"], non_blocking=True)
+
+        e2e_step()
+        barrier()
+        n_e2e = max(1, min(args.steps, 3))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        ms = a.elapsed_time(b) / n_e2e
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        e2e = {"value": world * flops_step / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e}
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu:
+        cpu = cpu_baseline_sample()
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"config {WORKLOAD}: {cfg.name}, 7 matrices, {M} tokens, rank {r}, "
+                                   f"mix {cfg.mix} (avg {bits:.2f} bits), stand-in codebooks",
+                       "elements": elems, "l2": "inputs larger than L2 (about 2.7 GB touched per step)"},
+            "phases": phases, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "gpu_launches": args.steps * len(dev) * 6, "clocks": clocks,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# --------------------------------------------------------------------------------------------------
+# CPU oracle arm
+# --------------------------------------------------------------------------------------------------
+SAMPLE_TOKENS = 512
+
+
+def oracle_sample_step(problem):
+    """The oracle on the bounded sample: q_proj-shaped matrix, encode + decode in full, forward +
+    backward-input on SAMPLE_TOKENS token rows.  Returns per-phase seconds."""
+    import oracle
+    W, precs, maps, thr, X, dY, A, B, s = problem
+    K = W.shape[1]
+    t = {}
+    t0 = time.time(); packed, a = oracle.encode(W, precs, thr); t["encode"] = time.time() - t0
+    t0 = time.time(); what = oracle.decode(packed, a, maps, precs, K); t["decode"] = time.time() - t0
+    t0 = time.time(); oracle.lora_forward(what, X, A, B, s); t["forward"] = time.time() - t0
+    t0 = time.time(); oracle.lora_backward_input(what, dY, A, B, s); t["backward"] = time.time() - t0
+    return t
+
+
+def make_sample_problem():
+    cfg = si.config(WORKLOAD)
+    mat = cfg.matrices[0]
+    W = si.weights(mat.N, mat.K, matrix_id=mat.matrix_id)
+    precs = si.precisions(mat.N, cfg.mix, matrix_id=mat.matrix_id)
+    maps, thr = si.standin_codebooks(precs, matrix_id=mat.matrix_id)
+    X = si.activations(SAMPLE_TOKENS, mat.K, matrix_id=100)
+    dY = si.activations(SAMPLE_TOKENS, mat.N, matrix_id=101)
+    A, B = si.lora_factors(mat.K, mat.N, cfg.rank, matrix_id=mat.matrix_id)
+    return (W, precs, maps, thr, X, dY, A, B, cfg.s), mat, cfg
+
+
+def cpu_baseline_sample(reps: int = 3):
+    import oracle
+    problem, mat, cfg = make_sample_problem()
+    oracle_sample_step(problem)  # warm
+    ts = [oracle_sample_step(problem) for _ in range(reps)]
+    tot = min(sum(t.values()) for t in ts)
+    best = min(ts, key=lambda t: sum(t.values()))
+    flops = 2 * gemm_flops(SAMPLE_TOKENS, mat.N, mat.K, cfg.rank)
+    el = mat.N * mat.K
+    return {"value": flops / tot / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{mat.name} {mat.N}x{mat.K}: oracle encode + decode in full, forward + backward-input on "
+                      f"{SAMPLE_TOKENS} of {cfg.tokens[0]} token rows (fp64); same value definition as the GPU arm",
+            "seconds_per_sample_step": tot,
+            "encode_ns_per_element": best["encode"] / el * 1e9, "decode_ns_per_element": best["decode"] / el * 1e9,
+            "gemm_fp64_gflops": flops / (best["forward"] + best["backward"]) / 1e9}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    problem, mat, cfg = make_sample_problem()
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_step(problem)
+    t0 = time.time()
+    for _ in range(args.steps):
+        oracle_sample_step(problem)
+    dt = (time.time() - t0) / args.steps
+    flops = 2 * gemm_flops(SAMPLE_TOKENS, mat.N, mat.K, cfg.rank)
+    value = flops / dt / 1e12
+    sample = (f"each step = the CPU oracle on {mat.name} {mat.N}x{mat.K}: encode + decode in full, forward + "
+              f"backward-input on {SAMPLE_TOKENS} of {cfg.tokens[0]} token rows (fp64)")
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+           "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": min(args.warmup, 1),
+           "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+           "dtype": "f64", "data": "synthetic",
+           "config": {"workload": f"config {WORKLOAD}: {cfg.name} (bounded sample: {sample})"},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -21,6 +21,7 @@ namespace {
 
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 constexpr uint32_t kIdesc = ptx::umma_idesc_bf16(kTileR, kTileT);
+constexpr uint32_t kIdescAmn = kIdesc | (1u << 15);   // A operand MN-major
 
 struct Barriers {
     uint64_t full_x[kStages];   // TMA bytes of a stage have landed
@@ -33,87 +34,121 @@ struct Barriers {
     uint32_t abort;
 };
 
-// rowinfo word written by the prologue: bits 0-6 row offset inside its group, 7-8 class (3 = past N),
-// 9-31 stored position.
+// fields of the per-thread row word written by the prologue (see kIdleItem below)
 __device__ __forceinline__ int info_row(uint32_t w) { return (int)(w & 127u); }
 __device__ __forceinline__ int info_class(uint32_t w) { return (int)((w >> 7) & 3u); }
 __device__ __forceinline__ int info_pos(uint32_t w) { return (int)(w >> 9); }
 
-// ---- dequantisation of 8 consecutive elements to 8 bf16 (one 16-byte chunk) ----------------------
-// 1 bit: LH = {level0 * absmax, level1 * absmax} as bf16x2; each output word picks two halves.
-__device__ __forceinline__ uint4 deq8_b1(uint32_t bits8, uint32_t LH) {
-    uint32_t o[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const uint32_t v = (bits8 >> (2 * j)) & 3u;
-        const uint32_t sel = ((v * 0x1122u) & 0x2222u) | 0x1010u;
-        o[j] = __byte_perm(LH, LH, sel);
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-
-// 2 bits: E01 = {level0, level1} * absmax, E23 = {level2, level3} * absmax, bf16x2 each.
-__device__ __forceinline__ uint4 deq8_b2(uint32_t bits16, uint32_t E01, uint32_t E23) {
-    uint32_t o[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const uint32_t y = bits16 >> (4 * j);
-        const uint32_t t = (y & 3u) | ((y << 6) & 0x300u);
-        const uint32_t sel = t * 0x22u + 0x1010u;
-        o[j] = __byte_perm(E01, E23, sel);
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-
-// 4 bits: per-thread table of the 16 unscaled fp32 levels in shared memory (entry e at lut[e * stride]).
-__device__ __forceinline__ uint4 deq8_b4(uint32_t bits32, const float* lut, int stride, float a) {
-    uint32_t o[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-        const uint32_t c0 = (bits32 >> (8 * j)) & 15u;
-        const uint32_t c1 = (bits32 >> (8 * j + 4)) & 15u;
-        o[j] = pack_bf16x2(__fmul_rn(lut[c0 * stride], a), __fmul_rn(lut[c1 * stride], a));
-    }
-    return make_uint4(o[0], o[1], o[2], o[3]);
-}
-
-// Packed bits of `nbits` (32, 64 or 128) starting at p.
-__device__ __forceinline__ uint4 load_bits(const uint8_t* p, int cls) {
-    uint4 q = make_uint4(0u, 0u, 0u, 0u);
-    if (cls == 0) {
-        q.x = __ldg(reinterpret_cast<const uint32_t*>(p));
-    } else if (cls == 1) {
-        const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
-        q.x = t.x;
-        q.y = t.y;
-    } else if (cls == 2) {
-        q = __ldg(reinterpret_cast<const uint4*>(p));
-    }
-    return q;
-}
-
-// The 8 elements number x (0..3) of a thread's 32 elements.
-__device__ __forceinline__ uint32_t chunk_bits(const uint4& q, int cls, int x) {
-    if (cls == 0) return (q.x >> (8 * x)) & 0xFFu;
-    if (cls == 1) return (((x & 2) ? q.y : q.x) >> ((x & 1) * 16)) & 0xFFFFu;
-    return x == 0 ? q.x : x == 1 ? q.y : x == 2 ? q.z : q.w;
-}
-
-struct RowState {
-    const uint8_t* bits_ptr;   // this thread's first packed byte of the row (block 0)
-    const float* absmax_ptr;
-    float m0, m1, m2, m3;      // levels for 1- and 2-bit rows
-    int cls;                   // 0,1,2 = 1,2,4 bits; 3 = row past the end
+// ---- dequantisation of one 64-element block to 64 bf16 (one 128-byte operand row) -----------------
+// Packed codes of one 64-element block (8, 16 or 32 bytes) plus the block's absmax.
+struct Block {
+    uint4 lo, hi;
+    float a;
 };
 
-__device__ __forceinline__ uint4 deq_chunk(const RowState& rs, const uint4& q, int x, float a, uint32_t LH,
-                                           uint32_t E01, uint32_t E23, const float* lut, int lut_stride) {
-    const uint32_t bits = chunk_bits(q, rs.cls, x);
-    if (rs.cls == 0) return deq8_b1(bits, LH);
-    if (rs.cls == 1) return deq8_b2(bits, E01, E23);
-    if (rs.cls == 2) return deq8_b4(bits, lut, lut_stride, a);
-    return make_uint4(0u, 0u, 0u, 0u);
+__device__ __forceinline__ void load_block(Block& blk, const uint8_t* p, const float* absmax, int cls) {
+    if (cls == 0) {
+        const uint2 t = __ldg(reinterpret_cast<const uint2*>(p));
+        blk.lo.x = t.x;
+        blk.lo.y = t.y;
+    } else if (cls == 1) {
+        blk.lo = __ldg(reinterpret_cast<const uint4*>(p));
+    } else if (cls == 2) {
+        blk.lo = __ldg(reinterpret_cast<const uint4*>(p));
+        blk.hi = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+    }
+    if (cls < 3) blk.a = __ldg(absmax);
 }
+
+struct Levels { float m0, m1, m2, m3; };
+
+// Chunk t (elements 8t .. 8t+7) of the row goes to physical 16-byte slot t ^ swz (128B swizzle).
+__device__ __forceinline__ void store_chunk(uint32_t row_addr, int swz, int t, uint32_t o0, uint32_t o1, uint32_t o2,
+                                            uint32_t o3) {
+    ptx::st_shared_v4(row_addr + (uint32_t)((t ^ swz) << 4), make_uint4(o0, o1, o2, o3));
+}
+
+// 1 bit.  L, H = bf16(level0 * absmax), bf16(level1 * absmax) as 16-bit patterns; BB = min(L,H) in both
+// halves, d = |H - L|, f = 0x10001 if L > H else 0.  A half takes min + d exactly when its (possibly
+// flipped) code bit is set, so one multiply-add forms two elements without any carry between halves.
+// 16 code bits h are spread once (z = h | h << 15) so that pair j sits at bits 0 and 16 of z >> 2j.
+__device__ __noinline__ void dequant_block_1bit(uint32_t w0, uint32_t w1, float m0, float m1, float a,
+                                                uint32_t row_addr, int swz) {
+    const uint32_t LH = pack_bf16x2(__fmul_rn(m0, a), __fmul_rn(m1, a));
+    const uint32_t L = LH & 0xFFFFu, H = LH >> 16;
+    const uint32_t lo = min(L, H);
+    const uint32_t BB = lo * 0x10001u, d = max(L, H) - lo, f = (L > H) ? 0x10001u : 0u;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {  // 16 elements = two chunks per iteration
+        const uint32_t w = (q < 2) ? w0 : w1;
+        const uint32_t h = (q & 1) ? (w >> 16) : (w & 0xFFFFu);
+        const uint32_t z = h | (h << 15);
+        uint32_t o[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) o[j] = (((z >> (2 * j)) & 0x10001u) ^ f) * d + BB;
+        store_chunk(row_addr, swz, 2 * q, o[0], o[1], o[2], o[3]);
+        store_chunk(row_addr, swz, 2 * q + 1, o[4], o[5], o[6], o[7]);
+    }
+}
+
+// 2 bits: E01 = {level0, level1} * absmax, E23 = {level2, level3} * absmax, bf16x2 each; a byte
+// permute picks the two 16-bit entries named by a pair of codes.
+__device__ __noinline__ void dequant_block_2bit(uint4 w, Levels lv, float a, uint32_t row_addr, int swz) {
+    const uint32_t E01 = pack_bf16x2(__fmul_rn(lv.m0, a), __fmul_rn(lv.m1, a));
+    const uint32_t E23 = pack_bf16x2(__fmul_rn(lv.m2, a), __fmul_rn(lv.m3, a));
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {  // one 32-bit word = 16 elements = two chunks
+        const uint32_t x = q == 0 ? w.x : q == 1 ? w.y : q == 2 ? w.z : w.w;
+        uint32_t o[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t y = x >> (4 * j);
+            const uint32_t t = (y & 3u) | ((y << 6) & 0x300u);
+            o[j] = __byte_perm(E01, E23, t * 0x22u + 0x1010u);
+        }
+        store_chunk(row_addr, swz, 2 * q, o[0], o[1], o[2], o[3]);
+        store_chunk(row_addr, swz, 2 * q + 1, o[4], o[5], o[6], o[7]);
+    }
+}
+
+__device__ __noinline__ void zero_row(uint32_t row_addr) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) ptx::st_shared_v4(row_addr + 16u * t, make_uint4(0u, 0u, 0u, 0u));
+}
+
+// 4 bits.  The 16 levels are scaled by the block's absmax and rounded to bf16 exactly as the decode
+// kernel does, into a per-lane table in shared memory (entry e of lane l at slut[e * 32 + l], so the
+// warp's lookups never collide on a bank); each code is then one shift/mask and one 16-bit load.
+struct Levels16 { float v[16]; };
+__device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, Levels16 lv, uint32_t slut_addr,
+                                                uint32_t row_addr, int swz) {
+#pragma unroll
+    for (int e = 0; e < 16; e += 2) {
+        const uint32_t two = pack_bf16x2(__fmul_rn(lv.v[e], a), __fmul_rn(lv.v[e + 1], a));
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(slut_addr + (uint32_t)e * 128u), "r"(two & 0xFFFFu) : "memory");
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(slut_addr + (uint32_t)(e + 1) * 128u), "r"(two >> 16) : "memory");
+    }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {  // one 32-bit word = 8 elements = one chunk
+        const uint32_t w = q == 0 ? lo.x : q == 1 ? lo.y : q == 2 ? lo.z : q == 3 ? lo.w
+                         : q == 4 ? hi.x : q == 5 ? hi.y : q == 6 ? hi.z : hi.w;
+        uint32_t v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            // byte offset of entry c = (w >> 4j) & 15 is c * 128
+            const uint32_t off = (j == 0) ? ((w << 7) & 0x780u) : (j == 1) ? ((w << 3) & 0x780u)
+                                                                           : ((w >> (j < 2 ? 0 : 4 * j - 7)) & 0x780u);
+            asm("ld.shared.u32 %0, [%1];" : "=r"(v[j]) : "r"(slut_addr + off));
+        }
+        store_chunk(row_addr, swz, q, __byte_perm(v[0], v[1], 0x5410), __byte_perm(v[2], v[3], 0x5410),
+                    __byte_perm(v[4], v[5], 0x5410), __byte_perm(v[6], v[7], 0x5410));
+    }
+}
+
+// word written by the prologue for every dequant thread and every row group: bits 0-6 row offset inside
+// the group, 7-8 class (0,1,2 = 1,2,4 bits; 3 = row past N, to be zero-filled), 9-31 stored position;
+// all ones = this thread has no row in this group.  All rows of one warp have the same class.
+constexpr uint32_t kIdleItem = 0xFFFFFFFFu;
 
 }  // namespace
 
@@ -125,7 +160,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     const uint32_t raw_addr = ptx::smem_u32(smem_raw);
     unsigned char* base = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
     unsigned char* out_s = base + kStages * kSmemStage;
-    float* lut4 = reinterpret_cast<float*>(out_s + kSmemOut);
+    unsigned char* slut_all = out_s + kSmemOut;   // [8 warps][16 entries][32 lanes] u32: scaled 4-bit tables
     Barriers* bars = reinterpret_cast<Barriers*>(out_s + kSmemOut + kSmemLut4);
     volatile uint32_t* abort_flag = &bars->abort;
 
@@ -211,11 +246,19 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         if (!ptx::mbar_wait(&bars->full_w[s], ph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                     ptx::tc_fence_after();
                     const uint32_t a_addr = ptx::smem_u32(base + s * kSmemStage);
-                    const uint64_t adesc = ptx::umma_desc_k_sw128(a_addr);
                     const uint64_t bdesc = ptx::umma_desc_k_sw128(a_addr + kSmemA);
+                    if (MODE == kModeBackward && kb >= P.lora_blocks) {
+                        // weights tile is MN-major: 16 contraction rows = two 1024-byte groups per MMA
+                        const uint64_t adesc = ptx::umma_desc_mn_sw128(a_addr, 8192u);
 #pragma unroll
-                    for (int kk = 0; kk < kTileC / 16; ++kk)  // 16 elements = 32 bytes along K per MMA
-                        ptx::umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+                        for (int kk = 0; kk < kTileC / 16; ++kk)
+                            ptx::umma_bf16(d_tmem, adesc + 128u * kk, bdesc + 2u * kk, kIdescAmn, (kb | kk) != 0 ? 1u : 0u);
+                    } else {
+                        const uint64_t adesc = ptx::umma_desc_k_sw128(a_addr);
+#pragma unroll
+                        for (int kk = 0; kk < kTileC / 16; ++kk)  // 16 elements = 32 bytes along K per MMA
+                            ptx::umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+                    }
                     ptx::umma_commit(&bars->empty[s]);
                 }
                 if (failed) break;
@@ -278,164 +321,201 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         }
     } else if (MODE != kModeDense) {
         // ================================================================== dequant producers
+        // All eight warps work on every stage.  The prologue has dealt the rows of every group to the 256
+        // threads so that a warp only ever holds rows of one precision (chunks of at most 32 rows forward,
+        // 16 rows x 2 feature halves backward), so no warp runs more than one code path.  Each thread
+        // dequantises one 64-element absmax block per stage; the packed codes of the next two stages are
+        // already in registers (a two-deep ring with static indices, so no load is waited on early).
         const int pt = threadIdx.x - kFirstProducerWarp * 32;  // 0..255
-        const float* lut = lut4 + pt;
-        constexpr int kLutStride = kProducerWarps * 32;
+        const uint32_t slut_addr = ptx::smem_u32(slut_all) + (uint32_t)((pt >> 5) * 2048 + lane * 4);
         const int K = P.L.K;
-        uint32_t it = 0;
-        for (int tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
+        uint32_t it0 = 0;                                       // running stage index at the start of the tile
+        for (int tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x, it0 += total_blocks) {
             const int rt = tile % P.tiles_r;
             const int r0 = rt * kTileR;
             if (MODE == kModeForward) {
-                // ------------------------------------------------------------ forward: row = channel
-                // thread pair (2 lanes) per row, each 32 of the 64 elements of a stage
-                const int slot = pt >> 1, h = pt & 1, jq = (lane >> 1) & 3;
-                const uint32_t info = __ldg(P.rowinfo + (size_t)rt * kTileR + slot);
-                const int row_local = info_row(info);
-                RowState rs;
-                rs.cls = info_class(info);
-                rs.m0 = rs.m1 = rs.m2 = rs.m3 = 0.0f;
-                rs.bits_ptr = P.packed;
-                rs.absmax_ptr = P.absmax;
+                // ---------------------------------------------------------------- forward
+                // thread = one output channel of the tile, 64 input features per stage; operand tile is
+                // [128 channels][64 features], K-major.
+                const uint32_t item = __ldg(P.items + (size_t)rt * 256 + pt);
+                const int nch = (int)__ldg(P.n_chunks + rt);
+                const int turn_mask = 8 / nch - 1;            // k - 1, k = warps per chunk (a power of two)
+                const int phase = (pt >> 5) / nch;            // this warp serves main blocks mb with (mb & turn_mask) == phase
+                const bool active = item != kIdleItem;
+                const int cls = active ? info_class(item) : 4;
+                const int wcls = __shfl_sync(0xffffffffu, cls, 0);   // lane 0 always holds a row if the warp does
+                const int row_local = info_row(item);
+                Levels lv = {0.f, 0.f, 0.f, 0.f};
+                const uint8_t* bits_ptr = P.packed;
+                const float* absmax_ptr = P.absmax;
+                const float* mrow = P.maps;
                 int bits_stride = 0;  // packed bytes per 64-element block
-                if (rs.cls < 3) {
-                    const int p = info_pos(info);
-                    const int b = 1 << rs.cls;
-                    const int r = r0 + row_local;
+                if (cls < 3) {
+                    const int p = info_pos(item);
+                    const int b = 1 << cls;
                     bits_stride = 8 * b;
-                    rs.bits_ptr = P.packed + P.L.seg_off[rs.cls] +
-                                  (size_t)(p - P.L.class_start[rs.cls]) * ((size_t)K * b / 8) + h * (4 * b);
-                    rs.absmax_ptr = P.absmax + (size_t)p * P.L.nb;
-                    const float* mrow = P.maps + (size_t)r * kTableStride;
-                    if (rs.cls == 0) {
-                        rs.m0 = __ldg(mrow); rs.m1 = __ldg(mrow + 1);
-                    } else if (rs.cls == 1) {
-                        rs.m0 = __ldg(mrow); rs.m1 = __ldg(mrow + 1); rs.m2 = __ldg(mrow + 2); rs.m3 = __ldg(mrow + 3);
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 16; ++e) lut4[e * kLutStride + pt] = __ldg(mrow + e);
+                    bits_ptr = P.packed + P.L.seg_off[cls] + (size_t)(p - P.L.class_start[cls]) * ((size_t)K * b / 8);
+                    absmax_ptr = P.absmax + (size_t)p * P.L.nb;
+                    mrow = P.maps + (size_t)(r0 + row_local) * kTableStride;
+                    if (cls == 0) {
+                        lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
+                    } else if (cls == 1) {
+                        lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
                     }
                 }
                 const uint32_t row_off = (uint32_t)row_local * 128u;
                 const int swz = row_local & 7;
-                // two blocks of look-ahead
-                uint4 q0 = make_uint4(0, 0, 0, 0), q1 = q0;
-                float a0 = 0.0f, a1 = 0.0f;
-                if (rs.cls < 3) {
-                    q0 = load_bits(rs.bits_ptr, rs.cls);
-                    a0 = __ldg(rs.absmax_ptr);
-                    if (P.main_blocks > 1) {
-                        q1 = load_bits(rs.bits_ptr + bits_stride, rs.cls);
-                        a1 = __ldg(rs.absmax_ptr + 1);
-                    }
-                }
-                for (int kb = 0; kb < total_blocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
-                    if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
-                    if (kb >= P.lora_blocks) {
-                        const int mb = kb - P.lora_blocks;
-                        uint4 q2 = make_uint4(0, 0, 0, 0);
-                        float a2 = 0.0f;
-                        if (rs.cls < 3 && mb + 2 < P.main_blocks) {
-                            q2 = load_bits(rs.bits_ptr + (size_t)(mb + 2) * bits_stride, rs.cls);
-                            a2 = __ldg(rs.absmax_ptr + mb + 2);
-                        }
-                        const uint32_t a_s = ptx::smem_u32(base + s * kSmemStage) + row_off;
-                        uint32_t LH = 0, E01 = 0, E23 = 0;
-                        if (rs.cls == 0) {
-                            LH = pack_bf16x2(__fmul_rn(rs.m0, a0), __fmul_rn(rs.m1, a0));
-                        } else if (rs.cls == 1) {
-                            E01 = pack_bf16x2(__fmul_rn(rs.m0, a0), __fmul_rn(rs.m1, a0));
-                            E23 = pack_bf16x2(__fmul_rn(rs.m2, a0), __fmul_rn(rs.m3, a0));
-                        }
+                Block ring[2];
+                ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
+                ring[0].a = ring[1].a = 0.0f;
 #pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            // rotate the chunk order so that the 8 lanes of a quarter-warp hit 8 distinct
-                            // 16-byte bank groups whatever rows they own
-                            const int x = ((jq + t) & 3) ^ (row_local & 3);
-                            const uint4 val = deq_chunk(rs, q0, x, a0, LH, E01, E23, lut, kLutStride);
-                            const int chunk_phys = (4 * h + x) ^ swz;
-                            ptx::st_shared_v4(a_s + (uint32_t)chunk_phys * 16u, val);
+                for (int u = 0; u < 2; ++u) {   // ring slot u serves the stages kb with kb % 2 == u
+                    const int mb = ((P.lora_blocks + 1 - u) & ~1) + u - P.lora_blocks;  // first main block of slot u
+                    if (cls < 3 && mb < P.main_blocks && (mb & turn_mask) == phase)
+                        load_block(ring[u], bits_ptr + (size_t)mb * bits_stride, absmax_ptr + mb, cls);
+                }
+                for (int kb0 = 0; kb0 < total_blocks && !failed; kb0 += 2) {
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int kb = kb0 + u;
+                        if (kb >= total_blocks) break;
+                        const uint32_t it = it0 + (uint32_t)kb;
+                        const int s = it % kStages;
+                        const uint32_t ph = (it / kStages) & 1u;
+                        if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
+                            failed = true; bars->abort = 1u; break;
                         }
-                        q0 = q1; q1 = q2; a0 = a1; a1 = a2;
-                        ptx::fence_proxy_async_smem();
+                        const int mb = kb - P.lora_blocks;
+                        if (mb >= 0 && wcls < 4 && (mb & turn_mask) == phase) {
+                            if (active) {
+                                const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + row_off;
+                                if (wcls == 0) {
+                                    dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lv.m0, lv.m1, ring[u].a, row_addr, swz);
+                                } else if (wcls == 1) {
+                                    dequant_block_2bit(ring[u].lo, lv, ring[u].a, row_addr, swz);
+                                } else if (wcls == 2) {
+                                    Levels16 l16;
+                                    const float4* m4 = reinterpret_cast<const float4*>(mrow);   // stays in L1
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) {
+                                        const float4 t = __ldg(m4 + e);
+                                        l16.v[4 * e] = t.x; l16.v[4 * e + 1] = t.y; l16.v[4 * e + 2] = t.z; l16.v[4 * e + 3] = t.w;
+                                    }
+                                    dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, l16, slut_addr, row_addr, swz);
+                                } else {
+                                    zero_row(row_addr);
+                                }
+                                ptx::fence_proxy_async_smem();
+                            }
+                        }
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
+                        const int nb = mb + 2;   // this ring slot's next stage
+                        if (cls < 3 && mb >= 0 && nb < P.main_blocks && (nb & turn_mask) == phase)
+                            load_block(ring[u], bits_ptr + (size_t)nb * bits_stride, absmax_ptr + nb, cls);
                     }
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
                 }
             } else {
-                // ------------------------------------------------------------ backward: row = contraction index
-                // every stage brings 64 new channels; 4 threads per channel, 32 input features each
-                const int qslot = pt & 63, kq = pt >> 6;
-                const int k_first = r0 + 32 * kq;       // first input feature of this thread
-                const bool k_ok = k_first < K;          // K % 128 == 0, so all 32 are in range or none
-                const uint32_t* infos = P.rowinfo;
-                uint32_t info_next = (P.main_blocks > 0) ? __ldg(infos + qslot) : (3u << 7);
-                for (int kb = 0; kb < total_blocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
-                    uint4 q = make_uint4(0, 0, 0, 0);
-                    float a = 0.0f;
-                    RowState rs;
-                    rs.cls = 3;
-                    rs.m0 = rs.m1 = rs.m2 = rs.m3 = 0.0f;
-                    int col = qslot;
-                    if (kb >= P.lora_blocks) {
-                        // fetch this stage's row before waiting for the slot (hides the load latency)
+                // ---------------------------------------------------------------- backward
+                // every stage brings 64 new channels (the contraction index); thread = one channel x 64 of
+                // the tile's 128 input features = one absmax block.  Operand tile is MN-major:
+                // [feature half][64 channels][64 features], so the block is one 128-byte row and is
+                // written exactly as in the forward case.
+                const int half = (lane >> 4) & 1;
+                const int k_first = r0 + 64 * half;
+                const uint32_t* items = P.items + pt;
+                uint32_t info_ring[2];
+                Block ring[2];
+                Levels lvr[2];
+                ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
+                ring[0].a = ring[1].a = 0.0f;
+                lvr[0] = lvr[1] = Levels{0.f, 0.f, 0.f, 0.f};
+                uint32_t cur_info[2] = {kIdleItem, kIdleItem};
+                Levels16 m16;
+#pragma unroll
+                for (int e = 0; e < 16; ++e) m16.v[e] = 0.0f;
+
+                // fetch everything block mb needs except a 4-bit table: codes, absmax, 1/2-bit levels
+                auto fetch = [&](Block& blk, Levels& lv, uint32_t info, int mb) {
+                    const int cls = (info == kIdleItem) ? 4 : info_class(info);
+                    if (cls < 3) {
+                        const int p = info_pos(info);
+                        const int b = 1 << cls;
+                        load_block(blk,
+                                   P.packed + P.L.seg_off[cls] + (size_t)(p - P.L.class_start[cls]) * ((size_t)K * b / 8) +
+                                       (size_t)k_first * b / 8,
+                                   P.absmax + (size_t)p * P.L.nb + k_first / kBlock, cls);
+                        const float* mrow = P.maps + (size_t)(mb * kTileC + info_row(info)) * kTableStride;
+                        if (cls == 0) {
+                            lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
+                        } else if (cls == 1) {
+                            lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
+                        }
+                    }
+                };
+                auto fetch_table = [&](uint32_t info, int mb) {
+                    if (info != kIdleItem && info_class(info) == 2) {
+                        const float4* m4 = reinterpret_cast<const float4*>(
+                            P.maps + (size_t)(mb * kTileC + info_row(info)) * kTableStride);
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float4 t = __ldg(m4 + e);
+                            m16.v[4 * e] = t.x; m16.v[4 * e + 1] = t.y; m16.v[4 * e + 2] = t.z; m16.v[4 * e + 3] = t.w;
+                        }
+                    }
+                };
+
+                // prologue: first two main blocks fully, row descriptors of the next two
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int mb = ((P.lora_blocks + 1 - u) & ~1) + u - P.lora_blocks;  // first main block of slot u
+                    if (mb < P.main_blocks) {
+                        cur_info[u] = __ldg(items + (size_t)mb * 256);
+                        fetch(ring[u], lvr[u], cur_info[u], mb);
+                    }
+                    info_ring[u] = (mb + 2 < P.main_blocks) ? __ldg(items + (size_t)(mb + 2) * 256) : kIdleItem;
+                }
+                if (P.main_blocks > 0) fetch_table(cur_info[P.lora_blocks & 1], 0);
+                for (int kb0 = 0; kb0 < total_blocks && !failed; kb0 += 2) {
+#pragma unroll
+                    for (int u = 0; u < 2; ++u) {
+                        const int kb = kb0 + u;
+                        if (kb >= total_blocks) break;
+                        const uint32_t it = it0 + (uint32_t)kb;
+                        const int s = it % kStages;
+                        const uint32_t ph = (it / kStages) & 1u;
+                        if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
+                            failed = true; bars->abort = 1u; break;
+                        }
                         const int mb = kb - P.lora_blocks;
-                        const uint32_t info = info_next;
-                        if (mb + 1 < P.main_blocks) info_next = __ldg(infos + (size_t)(mb + 1) * kTileC + qslot);
-                        col = info_row(info);
-                        rs.cls = k_ok ? info_class(info) : 3;
-                        if (rs.cls < 3) {
-                            const int p = info_pos(info);
-                            const int b = 1 << rs.cls;
-                            const int n = mb * kTileC + col;
-                            q = load_bits(P.packed + P.L.seg_off[rs.cls] +
-                                              (size_t)(p - P.L.class_start[rs.cls]) * ((size_t)K * b / 8) +
-                                              (size_t)k_first * b / 8,
-                                          rs.cls);
-                            a = __ldg(P.absmax + (size_t)p * P.L.nb + k_first / kBlock);
-                            const float* mrow = P.maps + (size_t)n * kTableStride;
-                            if (rs.cls == 0) {
-                                rs.m0 = __ldg(mrow); rs.m1 = __ldg(mrow + 1);
-                            } else if (rs.cls == 1) {
-                                rs.m0 = __ldg(mrow); rs.m1 = __ldg(mrow + 1); rs.m2 = __ldg(mrow + 2); rs.m3 = __ldg(mrow + 3);
-                            } else {
-#pragma unroll
-                                for (int e = 0; e < 16; ++e) lut4[e * kLutStride + pt] = __ldg(mrow + e);
+                        if (mb >= 0) {
+                            const uint32_t info = cur_info[u];
+                            const bool active = info != kIdleItem;
+                            const int wcls = __shfl_sync(0xffffffffu, active ? info_class(info) : 4, 0);
+                            if (active) {
+                                const int col = info_row(info);   // channel inside the stage = K index of the tile
+                                const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + (uint32_t)half * 8192u +
+                                                          (uint32_t)col * 128u;
+                                if (wcls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lvr[u].m0, lvr[u].m1, ring[u].a, row_addr, col & 7);
+                                else if (wcls == 1) dequant_block_2bit(ring[u].lo, lvr[u], ring[u].a, row_addr, col & 7);
+                                else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, m16, slut_addr, row_addr, col & 7);
+                                else zero_row(row_addr);
+                                ptx::fence_proxy_async_smem();
                             }
                         }
-                    }
-                    if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
-                    if (kb >= P.lora_blocks) {
-                        uint32_t LH = 0, E01 = 0, E23 = 0;
-                        if (rs.cls == 0) {
-                            LH = pack_bf16x2(__fmul_rn(rs.m0, a), __fmul_rn(rs.m1, a));
-                        } else if (rs.cls == 1) {
-                            E01 = pack_bf16x2(__fmul_rn(rs.m0, a), __fmul_rn(rs.m1, a));
-                            E23 = pack_bf16x2(__fmul_rn(rs.m2, a), __fmul_rn(rs.m3, a));
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
+                        // refill this ring slot for its next stage (block mb + 2), fetch the 4-bit table of the
+                        // very next stage (block mb + 1, other slot), look two stages further ahead for the row
+                        const int nb = mb + 2;
+                        if (mb >= 0) {
+                            cur_info[u] = info_ring[u];
+                            if (nb < P.main_blocks) fetch(ring[u], lvr[u], cur_info[u], nb);
+                            info_ring[u] = (nb + 2 < P.main_blocks) ? __ldg(items + (size_t)(nb + 2) * 256) : kIdleItem;
                         }
-                        // operand tile is [128 features][64 channels], K-major: this thread owns column `col`
-                        const uint32_t a_s = ptx::smem_u32(base + s * kSmemStage);
-                        const uint32_t col_chunk = (uint32_t)col >> 3, col_in = ((uint32_t)col & 7u) * 2u;
-#pragma unroll
-                        for (int x = 0; x < 4; ++x) {
-                            const uint4 val = deq_chunk(rs, q, x, a, LH, E01, E23, lut, kLutStride);
-                            const uint32_t w[4] = {val.x, val.y, val.z, val.w};
-#pragma unroll
-                            for (int e = 0; e < 8; ++e) {
-                                const uint32_t krow = (uint32_t)(32 * kq + 8 * x + e);
-                                const uint32_t addr = a_s + krow * 128u + ((col_chunk ^ (krow & 7u)) << 4) + col_in;
-                                const uint16_t hv = (uint16_t)((e & 1) ? (w[e >> 1] >> 16) : (w[e >> 1] & 0xFFFFu));
-                                asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(hv) : "memory");
-                            }
-                        }
-                        ptx::fence_proxy_async_smem();
+                        const int tb = mb + 1;
+                        if (tb >= 1 && tb < P.main_blocks) fetch_table(cur_info[u ^ 1], tb);
                     }
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
                 }
             }
         }

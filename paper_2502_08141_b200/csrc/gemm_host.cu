@@ -14,7 +14,7 @@ constexpr size_t kStatusBytes = 256;
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Workspace {
-    size_t off_T, off_F2, off_info, total;
+    size_t off_T, off_F2, off_info, off_meta, total;
     int rp;
 };
 
@@ -27,7 +27,8 @@ Workspace plan_workspace(int N, int K, int M, int r) {
     w.off_T = kStatusBytes;
     w.off_F2 = w.off_T + align256((size_t)M * w.rp * 2);
     w.off_info = w.off_F2 + align256((size_t)big * w.rp * 2);
-    w.total = w.off_info + align256((size_t)((N + 127) / 128 * 128) * 4);
+    w.off_meta = w.off_info + align256((size_t)((N + 63) / 64) * 256 * 4);
+    w.total = w.off_meta + align256((size_t)((N + 63) / 64) * 4);
     return w;
 }
 
@@ -78,7 +79,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
     uint16_t* F2 = reinterpret_cast<uint16_t*>(ws + w.off_F2);
-    uint32_t* rowinfo = reinterpret_cast<uint32_t*>(ws + w.off_info);
+    uint32_t* items = reinterpret_cast<uint32_t*>(ws + w.off_info);
     uint32_t* status = reinterpret_cast<uint32_t*>(ws);
 
     // ---- prologue
@@ -93,7 +94,8 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     P.Dst = F2;
     P.precs = layout->precs_dev;
     P.inv_perm = layout->inv_perm_dev;
-    P.rowinfo = rowinfo;
+    P.items = items;
+    P.n_chunks = reinterpret_cast<uint32_t*>(ws + w.off_meta);
     P.N = N;
     P.status = status;
     if (!backward) {
@@ -118,7 +120,8 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.packed = packed;
     G.absmax = absmax;
     G.maps = maps;
-    G.rowinfo = rowinfo;
+    G.items = items;
+    G.n_chunks = reinterpret_cast<uint32_t*>(ws + w.off_meta);
     G.out = out;
     G.status = status;
     G.M = M;

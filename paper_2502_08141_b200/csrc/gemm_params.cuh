@@ -22,11 +22,13 @@ struct PrepParams {
     const uint16_t* Src;
     uint16_t* Dst;
     int R, src_transposed;
-    // (C) per-group precision order: rowinfo[g * group + i] describes the i-th row of group g in
-    // precision order: bits 0-6 row offset inside the group, 7-8 class (3 = past N), 9-31 stored position
+    // (C) deal of the rows of every group (128 rows forward, 64 backward) to the 256 dequant threads of
+    // the main kernel, one precision per warp: items[g * 256 + thread] = row offset (bits 0-6) | class
+    // (bits 7-8, 3 = row past N) | stored position (bits 9-31), or all ones for "no row"
     const uint8_t* precs;
     const int32_t* inv_perm;
-    uint32_t* rowinfo;    // [ceil(N / group) * group]
+    uint32_t* items;      // [ceil(N / group) * 256]
+    uint32_t* n_chunks;   // [ceil(N / group)] number of chunks the group was cut into (1..7)
     int N, group;
     uint32_t* status;
     int blocksA, blocksB, blocksC;
@@ -52,7 +54,8 @@ struct GemmParams {
     const uint8_t* packed;
     const float* absmax;
     const float* maps;
-    const uint32_t* rowinfo;  // from the prologue
+    const uint32_t* items;    // from the prologue: [row groups][256 dequant threads]
+    const uint32_t* n_chunks; // from the prologue: [row groups]
     uint16_t* out;          // [M, ld_out] bf16
     uint32_t* status;
     int M;                  // tokens
@@ -68,7 +71,7 @@ constexpr uint32_t kSmemA = kTileR * kTileC * 2;   // 16 KB
 constexpr uint32_t kSmemB = kTileT * kTileC * 2;   // 32 KB
 constexpr uint32_t kSmemStage = kSmemA + kSmemB;
 constexpr uint32_t kSmemOut = 32 * kTileR * 2;     // epilogue staging: 32 tokens x 128 channels bf16
-constexpr uint32_t kSmemLut4 = 16 * kProducerWarps * 32 * 4;  // per-thread 16-entry fp32 tables
+constexpr uint32_t kSmemLut4 = kProducerWarps * 32 * 16 * 4;  // per dequant lane: 16 scaled bf16 levels (one word each)
 constexpr uint32_t kSmemBarriers = 1024;
 constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kStages * kSmemStage + kSmemOut + kSmemLut4 + kSmemBarriers;
 

@@ -3,9 +3,8 @@
 //       with warp-level tensor-core MMAs, rounded once to bf16, zero-padded to a multiple of 64 columns;
 //   (B) writes the other LoRA factor as a K-major, zero-padded bf16 matrix that TMA can fetch:
 //       Bt[n, j] = B[j, n] (forward)  or  Ap[k, j] = A[k, j] (backward);
-//   (C) for every group of 128 (forward) or 64 (backward) consecutive output channels, lists the rows
-//       of the group ordered by precision (stable), so that the dequant warps of the main kernel can
-//       give rows of equal precision to neighbouring threads;
+//   (C) deals the rows of every group of 128 (forward) or 64 (backward) consecutive output channels to the
+//       256 dequant threads of the main kernel so that each warp only holds rows of one precision;
 //   and clears the device status word.
 #include "gemm_params.cuh"
 #include "ptx.cuh"
@@ -155,13 +154,22 @@ __device__ void pad_factor(const PrepParams& P, int blk) {
 }
 
 // ------------------------------------------------------------------------------------------ role C
-// One warp per group of G rows: stable sort of the group's rows by precision class
-// (1 bit, 2 bits, 4 bits, then rows past N); entry i of the group describes its i-th row in that order.
-__device__ void order_groups(const PrepParams& P, int blk) {
+// One warp per group of G rows (128 forward, 64 backward).  The rows are ordered by precision class
+// (1 bit, 2 bits, 4 bits, rows past N; stable) and cut into chunks of CH rows of one class (32 forward;
+// 16 backward, where every row is handled by two threads, one per 64-feature half), so that no warp of
+// the main kernel ever sees two precisions.  At most G / CH + 3 = 7 chunks exist and the kernel has 8
+// dequant warps: with n chunks, k = 8 / n warps share a chunk and take turns over the stages
+// (warp c + j * n serves chunk c at the stages whose index is congruent to j mod k).
+__device__ void deal_rows(const PrepParams& P, int blk) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = P.group, per = G / 32;
+    const int CH = (G == 128) ? 32 : 16;
     const int n_groups = (P.N + G - 1) / G;
     for (int grp = blk * (kPrepThreads / 32) + warp; grp < n_groups; grp += P.blocksC * (kPrepThreads / 32)) {
+        uint32_t* out = P.items + (size_t)grp * 256;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) out[i * 32 + lane] = 0xFFFFFFFFu;
+        __syncwarp();
         int cls[4];
         unsigned mask[4][4];
         int total[4] = {0, 0, 0, 0};
@@ -178,22 +186,34 @@ __device__ void order_groups(const PrepParams& P, int blk) {
                 total[c] += __popc(mask[i][c]);
             }
         }
-        int base[4];
-        base[0] = 0;
-        base[1] = total[0];
-        base[2] = total[0] + total[1];
-        base[3] = base[2] + total[2];
+        int chunk_base[4];
+        chunk_base[0] = 0;
+#pragma unroll
+        for (int c = 1; c < 4; ++c) chunk_base[c] = chunk_base[c - 1] + (total[c - 1] + CH - 1) / CH;
+        const int n_chunks = chunk_base[3] + (total[3] + CH - 1) / CH;
+        const int k = 8 / n_chunks;
+        if (lane == 0) P.n_chunks[grp] = (uint32_t)n_chunks;
         int before[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             if (i < per) {
-                int pos = 0;
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    if (cls[i] == c) pos = base[c] + before[c] + __popc(mask[i][c] & ((1u << lane) - 1u));
-                const int off = i * 32 + lane, row = grp * G + off;
-                const uint32_t p = (cls[i] < 3) ? (uint32_t)P.inv_perm[row] : 0u;
-                P.rowinfo[(size_t)grp * G + pos] = (uint32_t)off | ((uint32_t)cls[i] << 7) | (p << 9);
+                for (int c = 0; c < 4; ++c) {
+                    if (cls[i] == c) {
+                        const int q = before[c] + __popc(mask[i][c] & ((1u << lane) - 1u));  // rank inside the class
+                        const int off = i * 32 + lane, row = grp * G + off;
+                        const uint32_t p = (c < 3) ? (uint32_t)P.inv_perm[row] : 0u;
+                        const uint32_t word = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
+                        for (int j = 0; j < k; ++j) {
+                            // backward: the group index is the stage index, so only the warp whose turn it
+                            // is gets the row; forward: all k warps get it and take turns over the stages
+                            if (CH == 16 && j != (grp & (k - 1))) continue;
+                            const int thread = (chunk_base[c] + q / CH + j * n_chunks) * 32 + q % CH;
+                            out[thread] = word;
+                            if (CH == 16) out[thread + 16] = word;
+                        }
+                    }
+                }
 #pragma unroll
                 for (int c = 0; c < 4; ++c) before[c] += __popc(mask[i][c]);
             }
@@ -209,7 +229,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const PrepParams P) 
     if (b == 0 && threadIdx.x == 0) *P.status = 0u;
     if (b < P.blocksA) down_projection(P, b, smem_raw);
     else if (b < P.blocksA + P.blocksB) pad_factor(P, b - P.blocksA);
-    else order_groups(P, b - P.blocksA - P.blocksB);
+    else deal_rows(P, b - P.blocksA - P.blocksB);
 }
 
 static size_t prep_smem_bytes(int rp) {

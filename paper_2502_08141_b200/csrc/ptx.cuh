@@ -69,11 +69,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     }
 }
 
-// Same, executed by a whole warp with one common answer.
+// Same for a whole warp with one common answer: only lane 0 polls (256 threads spinning on a barrier
+// would compete with the tensor core for shared-memory bandwidth), the others wait at the warp barrier.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort,
                                                uint64_t limit_ns) {
-    const bool ok = mbar_wait(bar, parity, abort, limit_ns);
-    return __all_sync(0xffffffffu, ok) != 0;
+    uint32_t ok = 1u;
+    if ((threadIdx.x & 31u) == 0u) ok = mbar_wait(bar, parity, abort, limit_ns) ? 1u : 0u;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0u;
 }
 
 // ---------------------------------------------------------------------------------- fences
@@ -120,6 +122,19 @@ __device__ __forceinline__ uint64_t umma_desc_k_sw128(uint32_t saddr) {
     d |= (uint64_t)(1024u >> 4) << 32;               // stride byte offset between 8-row groups
     d |= (uint64_t)1u << 46;                         // descriptor version (sm_100)
     d |= (uint64_t)2u << 61;                         // SWIZZLE_128B
+    return d;
+}
+
+// Shared-memory operand descriptor: MN-major tile with 128B swizzle.  Every contraction index is a
+// 128-byte row of 64 consecutive M (or N) elements; eight such rows form a 1024-byte swizzle group
+// (stride byte offset); the next 64 M elements start `mn_block_bytes` further (leading byte offset).
+__device__ __forceinline__ uint64_t umma_desc_mn_sw128(uint32_t saddr, uint32_t mn_block_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((mn_block_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024u >> 4) << 32;
+    d |= (uint64_t)1u << 46;
+    d |= (uint64_t)2u << 61;
     return d;
 }
 
