@@ -51,7 +51,8 @@ typedef enum {
     LOWRA_ERR_WORKSPACE = 5, /* workspace smaller than lowra_workspace_bytes() */
     LOWRA_ERR_CUDA = 6,      /* a CUDA runtime / driver call failed */
     LOWRA_ERR_TIMEOUT = 7,   /* a bounded device-side wait ran out (read via lowra_device_status) */
-    LOWRA_ERR_ARCH = 8       /* current device is not compute capability 10.x */
+    LOWRA_ERR_ARCH = 8,      /* current device is not compute capability 10.x */
+    LOWRA_ERR_LIMIT = 9      /* problem larger than the built-in scratch of lowra_lora_forward_static */
 } lowra_status;
 
 const char* lowra_status_string(lowra_status st);
@@ -139,6 +140,36 @@ lowra_status lowra_lora_backward_input(const lowra_layout* layout, const uint8_t
  * (the kernel then released its resources and returned; the output is not valid).
  */
 lowra_status lowra_device_status(const void* workspace_dev, void* stream);
+
+/*
+ * (No counterpart in the paper: this is a packaging variant of lowra_lora_forward.)
+ *
+ * lowra_lora_forward for callers that cannot hand over scratch memory.  Some hosts of this library
+ * never get to call cudaMalloc themselves: a plug-in running inside another process's CUDA context
+ * whose allocator it must not touch, a real-time or safety-certified loop in which every allocation
+ * was frozen at start-up, a sandbox in which only pre-registered buffers may be passed around.  For
+ * them the scratch that lowra_lora_forward takes as `workspace_dev` lives inside the library itself,
+ * in a fixed device array of LOWRA_STATIC_SCRATCH_BYTES bytes that every GPU holds from the moment the
+ * library is loaded there until the process exits.  The call allocates nothing, frees nothing and
+ * calls no allocating routine; inputs and outputs are still the caller's.
+ *
+ *   - Same arguments, results and errors as lowra_lora_forward, without the workspace.  If
+ *     lowra_workspace_bytes(layout, M, r) exceeds LOWRA_STATIC_SCRATCH_BYTES the call launches nothing
+ *     and returns LOWRA_ERR_LIMIT (for scale: N = K = 8192, M = 8192, r = 64 needs about 2.2 MB).
+ *   - status_out_dev (optional, may be NULL): a device uint32 that receives the device status word
+ *     (LOWRA_OK or LOWRA_ERR_TIMEOUT) once the call's kernels have run, since the built-in scratch cannot
+ *     be given to lowra_device_status.
+ *   - The first call on each device looks up the device address of the built-in array (once per device,
+ *     with that device current).  Make that first call outside any CUDA stream capture.
+ *   - All calls on a device share the one array, and it keeps what the previous call left in it (the call
+ *     clears the words it relies on being zero).  Two calls that overlap on the GPU - from different
+ *     streams or threads - race on it; serialise them.
+ */
+#define LOWRA_STATIC_SCRATCH_BYTES (8u << 20)
+lowra_status lowra_lora_forward_static(const lowra_layout* layout, const uint8_t* packed_dev,
+                                       const float* absmax_dev, const float* maps_dev, const uint16_t* X_dev,
+                                       int32_t M, const uint16_t* A_dev, const uint16_t* B_dev, int32_t r,
+                                       float s, uint16_t* Y_dev, uint32_t* status_out_dev, void* stream);
 
 /*
  * Diagnostic, not part of the method: C = P . Q^T with P bf16 [M, K], Q bf16 [N, K] (both

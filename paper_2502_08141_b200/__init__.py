@@ -21,11 +21,13 @@ LIB_PATH = os.path.join(_HERE, "liblowra.so")
 
 LOWRA_OK = 0
 (LOWRA_ERR_NULL, LOWRA_ERR_SHAPE, LOWRA_ERR_ALIGN, LOWRA_ERR_PREC, LOWRA_ERR_WORKSPACE,
- LOWRA_ERR_CUDA, LOWRA_ERR_TIMEOUT, LOWRA_ERR_ARCH) = range(1, 9)
+ LOWRA_ERR_CUDA, LOWRA_ERR_TIMEOUT, LOWRA_ERR_ARCH, LOWRA_ERR_LIMIT) = range(1, 10)
+LOWRA_STATIC_SCRATCH_BYTES = 8 << 20
 
 EXPORTS = (
     "lowra_status_string", "lowra_plan", "lowra_encode", "lowra_decode", "lowra_workspace_bytes",
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
+    "lowra_lora_forward_static",
 )
 
 
@@ -74,6 +76,8 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_forward.restype = ctypes.c_int
         L.lowra_lora_backward_input.argtypes = gemm_args
         L.lowra_lora_backward_input.restype = ctypes.c_int
+        L.lowra_lora_forward_static.argtypes = [lp, vp, vp, vp, vp, i32, vp, vp, i32, ctypes.c_float, vp, vp, vp]
+        L.lowra_lora_forward_static.restype = ctypes.c_int
         L.lowra_device_status.argtypes = [vp, vp]
         L.lowra_device_status.restype = ctypes.c_int
         L.lowra_dense_nt.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
@@ -217,6 +221,28 @@ def lowra_lora_forward(layout: Layout, packed, absmax, maps, X, A, B, s: float,
                                     _ptr(B), r, ctypes.c_float(s), _ptr(Y), _ptr(workspace),
                                     workspace.numel(), _stream(stream))
     _check(code, "lowra_lora_forward")
+    return Y
+
+
+def lowra_lora_forward_static(layout: Layout, packed, absmax, maps, X, A, B, s: float,
+                              Y: Optional[torch.Tensor] = None, status_out: Optional[torch.Tensor] = None,
+                              stream=None) -> torch.Tensor:
+    """lowra_lora_forward for callers that may not allocate device memory (a plug-in inside a host
+    application's CUDA context, a loop whose allocations were frozen at start-up): the scratch is a fixed
+    array inside the library (LOWRA_STATIC_SCRATCH_BYTES), shared by every call on the device, so calls
+    must not overlap on the GPU.  Raises LowraError(LOWRA_ERR_LIMIT) when the problem needs more scratch.
+    `status_out`: optional int32/uint32 device tensor of one element that receives the device status word.
+    This wrapper allocates Y only if the caller passes none; the library call itself allocates nothing."""
+    for t, n in ((X, "X"), (A, "A"), (B, "B")):
+        _dev(t, torch.bfloat16, n)
+    M, r = int(X.shape[0]), int(A.shape[1])
+    if tuple(X.shape) != (M, layout.K) or tuple(A.shape) != (layout.K, r) or tuple(B.shape) != (r, layout.N):
+        raise ValueError("shape mismatch")
+    if Y is None:
+        Y = torch.empty((M, layout.N), dtype=torch.bfloat16, device=X.device)
+    code = lib().lowra_lora_forward_static(layout.ref, _ptr(packed), _ptr(absmax), _ptr(maps), _ptr(X), M, _ptr(A),
+                                           _ptr(B), r, ctypes.c_float(s), _ptr(Y), _ptr(status_out), _stream(stream))
+    _check(code, "lowra_lora_forward_static")
     return Y
 
 

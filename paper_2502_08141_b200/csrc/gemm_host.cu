@@ -1,6 +1,8 @@
 // Host side of lowra_lora_forward / lowra_lora_backward_input / lowra_dense_nt: validation, workspace
 // carve-up, TMA descriptors, launches.
 #include <cudaTypedefs.h>
+
+#include <mutex>
 #include <string.h>
 
 #include "gemm_params.cuh"
@@ -165,6 +167,62 @@ extern "C" lowra_status lowra_lora_backward_input(const lowra_layout* layout, co
                                                   void* workspace_dev, size_t workspace_bytes, void* stream) {
     return lowra::run_lora(true, layout, packed_dev, absmax_dev, maps_dev, dY_dev, M, A_dev, B_dev, r, s, dX_dev,
                            workspace_dev, workspace_bytes, stream);
+}
+
+// ---------------------------------------------------------------------------------------------------
+// Forward without caller-provided scratch, for callers that may not allocate device memory.
+// The scratch is this fixed array: part of the library image, present on every GPU that loads it.
+// In host code `g_static_scratch` is only a handle for the symbol, never a device address; the address
+// is looked up once per device with cudaGetSymbolAddress and that pointer is what the kernels get.
+static __device__ __align__(256) unsigned char g_static_scratch[LOWRA_STATIC_SCRATCH_BYTES];
+
+namespace lowra {
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {nullptr};
+
+// Device address of the built-in scratch on the current device (looked up on first use).
+lowra_status static_scratch(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LOWRA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) return LOWRA_ERR_CUDA;
+        g_static_ptr[dev] = p;
+    }
+    *out = g_static_ptr[dev];
+    return LOWRA_OK;
+}
+}  // namespace
+}  // namespace lowra
+
+extern "C" lowra_status lowra_lora_forward_static(const lowra_layout* layout, const uint8_t* packed_dev,
+                                                  const float* absmax_dev, const float* maps_dev,
+                                                  const uint16_t* X_dev, int32_t M, const uint16_t* A_dev,
+                                                  const uint16_t* B_dev, int32_t r, float s, uint16_t* Y_dev,
+                                                  uint32_t* status_out_dev, void* stream) {
+    using namespace lowra;
+    if (!layout) return LOWRA_ERR_NULL;
+    const size_t need = lowra_workspace_bytes(layout, M, r);
+    if (need == 0) return LOWRA_ERR_SHAPE;
+    if (need > (size_t)LOWRA_STATIC_SCRATCH_BYTES) return LOWRA_ERR_LIMIT;
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    void* scratch = nullptr;
+    st = static_scratch(&scratch);
+    if (st != LOWRA_OK) return st;
+    // The prologue kernel rewrites every word the fused kernel reads (status word, down-projection,
+    // padded factor, row deal), so nothing left over from an earlier call is ever consumed.
+    st = run_lora(false, layout, packed_dev, absmax_dev, maps_dev, X_dev, M, A_dev, B_dev, r, s, Y_dev, scratch,
+                  (size_t)LOWRA_STATIC_SCRATCH_BYTES, stream);
+    if (st != LOWRA_OK) return st;
+    if (status_out_dev &&
+        cudaMemcpyAsync(status_out_dev, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream) !=
+            cudaSuccess)
+        return LOWRA_ERR_CUDA;
+    return LOWRA_OK;
 }
 
 extern "C" lowra_status lowra_device_status(const void* workspace_dev, void* stream) {

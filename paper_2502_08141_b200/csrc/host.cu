@@ -62,6 +62,7 @@ extern "C" const char* lowra_status_string(lowra_status st) {
         case LOWRA_ERR_CUDA: return "CUDA call failed";
         case LOWRA_ERR_TIMEOUT: return "device-side wait timed out";
         case LOWRA_ERR_ARCH: return "device is not sm_100";
+        case LOWRA_ERR_LIMIT: return "problem exceeds the built-in scratch of the no-allocation entry point";
     }
     return "unknown status";
 }

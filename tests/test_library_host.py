@@ -32,7 +32,7 @@ def test_library_exports_every_declared_symbol(lib):
 
 def test_status_strings(lib):
     assert lib.status_string(0) == "ok"
-    assert len({lib.status_string(c) for c in range(9)}) == 9
+    assert len({lib.status_string(c) for c in range(10)}) == 10
 
 
 def test_plan_matches_oracle_layout(lib):
@@ -89,6 +89,10 @@ def test_validation_runs_before_any_device_work(lib):
     assert L.lowra_lora_forward(*args) == lib.LOWRA_ERR_WORKSPACE
     assert L.lowra_lora_backward_input(*args) == lib.LOWRA_ERR_WORKSPACE
     assert L.lowra_device_status(None, None) == lib.LOWRA_ERR_NULL
+    sargs = [ctypes.byref(lay), 4096, 4096, 4096, 4096, 1 << 20, 4096, 4096, 128, ctypes.c_float(1.0), 4096, None, None]
+    assert L.lowra_lora_forward_static(*sargs) == lib.LOWRA_ERR_LIMIT   # 1M tokens x rank 128 needs > 8 MiB of scratch
+    sargs[8] = 24
+    assert L.lowra_lora_forward_static(*sargs) == lib.LOWRA_ERR_SHAPE
     assert L.lowra_dense_nt(4096, 4096, 16, 16, 100, 4096, 4096, 256, None) == lib.LOWRA_ERR_SHAPE
 
 
