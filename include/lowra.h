@@ -155,7 +155,7 @@ lowra_status lowra_device_status(const void* workspace_dev, void* stream);
  *
  *   - Same arguments, results and errors as lowra_lora_forward, without the workspace.  If
  *     lowra_workspace_bytes(layout, M, r) exceeds LOWRA_STATIC_SCRATCH_BYTES the call launches nothing
- *     and returns LOWRA_ERR_LIMIT (for scale: N = K = 8192, M = 8192, r = 64 needs about 2.2 MB).
+ *     and returns LOWRA_ERR_LIMIT (for scale: N = K = 8192, M = 8192, r = 64 needs about 1.2 MB).
  *   - status_out_dev (optional, may be NULL): a device uint32 that receives the device status word
  *     (LOWRA_OK or LOWRA_ERR_TIMEOUT) once the call's kernels have run, since the built-in scratch cannot
  *     be given to lowra_device_status.

@@ -7,8 +7,13 @@
 // eight dequant warps straight from the packed codes (never from HBM as bf16); the 256-token operand
 // (activations / output gradients) is the B operand and arrives by TMA.  The accumulator lives in
 // TMEM (two 128 x 256 fp32 buffers, so the epilogue of one tile overlaps the main loop of the next).
-// The LoRA term is folded into the same accumulator as extra contraction blocks whose operands
-// (the padded factor and the down-projected activations from the prologue) both arrive by TMA.
+// The LoRA term is folded into the same accumulator as extra contraction blocks at the end of every
+// tile, whose operands both arrive by TMA: the up-projection factor straight from the caller's matrix
+// and the down-projected activations T = s X A (resp. U = s dY B^T).  T itself is produced by this same
+// kernel: for every token tile there is one extra "T tile" whose 128 operand rows are the LoRA ranks
+// (factor fetched by TMA, no dequant); T tiles come first in the tile order, their epilogue publishes a
+// per-token-tile flag, and the TMA producer of a regular tile waits (bounded) for that flag before it
+// fetches T.  All CTAs are co-resident and walk the tiles in increasing order, so the wait cannot deadlock.
 //
 // Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, 6-13 = dequant.
 // All mbarrier waits are bounded; a wait that runs out sets the status word and every role leaves.
@@ -152,10 +157,17 @@ constexpr uint32_t kIdleItem = 0xFFFFFFFFu;
 
 }  // namespace
 
+// Decoded position of a tile in the persistent schedule.
+struct TileInfo {
+    bool is_t;     // a LoRA down-projection tile (operand rows = ranks) rather than a weight tile
+    int rt, mt;    // row tile, token tile
+    int blocks;    // contraction blocks of this tile
+};
+
 template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmB2,
-             const __grid_constant__ CUtensorMap tmA2) {
+fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmT,
+             const __grid_constant__ CUtensorMap tmFt, const __grid_constant__ CUtensorMap tmFl) {
     extern __shared__ unsigned char smem_raw[];
     const uint32_t raw_addr = ptx::smem_u32(smem_raw);
     unsigned char* base = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
@@ -165,8 +177,19 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     volatile uint32_t* abort_flag = &bars->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int total_blocks = P.lora_blocks + P.main_blocks;
-    const int n_tiles = P.tiles_r * P.tiles_t;
+    const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? P.tiles_t : 0;
+    const int n_tiles = n_t_tiles + P.tiles_r * P.tiles_t;
+    auto decode_tile = [&](int g) {
+        TileInfo t;
+        t.is_t = g < n_t_tiles;
+        if (t.is_t) {
+            t.rt = 0; t.mt = g; t.blocks = P.main_blocks;
+        } else {
+            const int idx = g - n_t_tiles;
+            t.mt = idx / P.tiles_r; t.rt = idx - t.mt * P.tiles_r; t.blocks = P.main_blocks + P.lora_blocks;
+        }
+        return t;
+    };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -182,8 +205,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         bars->abort = 0u;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmB);
-        if (P.lora_blocks > 0) ptx::prefetch_tensormap(&tmB2);
-        if (P.lora_blocks > 0 || MODE == kModeDense) ptx::prefetch_tensormap(&tmA2);
+        if (P.lora_blocks > 0) { ptx::prefetch_tensormap(&tmT); ptx::prefetch_tensormap(&tmFt); }
+        if (P.lora_blocks > 0 || MODE == kModeDense) ptx::prefetch_tensormap(&tmFl);
     }
     if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, kTmemCols);
     ptx::tc_fence_before();
@@ -197,27 +220,51 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // ================================================================== TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x) {
-                const int r0 = (tile % P.tiles_r) * kTileR, m0 = (tile / P.tiles_r) * kTileT;
-                for (int kb = 0; kb < total_blocks; ++kb, ++it) {
+            for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x) {
+                const TileInfo t = decode_tile(g);
+                const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
+                for (int kb = 0; kb < t.blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!ptx::mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                     unsigned char* a_s = base + s * kSmemStage;
                     unsigned char* b_s = a_s + kSmemA;
-                    if (kb < P.lora_blocks) {
-                        ptx::mbar_arrive_expect_tx(&bars->full_x[s], kSmemA + kSmemB);
-                        ptx::tma_load_2d(a_s, &tmA2, kb * kTileC, r0, &bars->full_x[s]);
-                        ptx::tma_load_2d(b_s, &tmB2, kb * kTileC, m0, &bars->full_x[s]);
-                    } else {
-                        const int c0 = (kb - P.lora_blocks) * kTileC;
-                        if (MODE == kModeDense) {
-                            ptx::mbar_arrive_expect_tx(&bars->full_x[s], kSmemA + kSmemB);
-                            ptx::tma_load_2d(a_s, &tmA2, c0, r0, &bars->full_x[s]);
-                        } else {
-                            ptx::mbar_arrive_expect_tx(&bars->full_x[s], kSmemB);
+                    uint64_t* bar = &bars->full_x[s];
+                    if (t.is_t) {
+                        const int c0 = kb * kTileC;
+                        if (MODE == kModeForward) {   // ranks x features from A [K, r]: one 64x64 box per 64 ranks
+                            ptx::mbar_arrive_expect_tx(bar, (uint32_t)P.lora_blocks * 8192u + kSmemB);
+                            for (int jb = 0; jb < P.lora_blocks; ++jb) ptx::tma_load_2d(a_s + jb * 8192, &tmFt, jb * 64, c0, bar);
+                        } else {                      // ranks x channels from B [r, N]: one 64 x 128 box
+                            ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
+                            ptx::tma_load_2d(a_s, &tmFt, c0, 0, bar);
                         }
-                        ptx::tma_load_2d(b_s, &tmB, c0, m0, &bars->full_x[s]);
+                        ptx::tma_load_2d(b_s, &tmB, c0, m0, bar);
+                    } else if (kb < P.main_blocks) {
+                        const int c0 = kb * kTileC;
+                        if (MODE == kModeDense) {
+                            ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
+                            ptx::tma_load_2d(a_s, &tmFl, c0, r0, bar);
+                        } else {
+                            ptx::mbar_arrive_expect_tx(bar, kSmemB);
+                        }
+                        ptx::tma_load_2d(b_s, &tmB, c0, m0, bar);
+                    } else {
+                        const int lb = kb - P.main_blocks;
+                        if (lb == 0) {
+                            // T of this token tile is written by another CTA: wait for its flag, then make
+                            // those generic-proxy writes visible to the TMA (async proxy) reads below
+                            if (!ptx::flag_wait(P.flags + t.mt, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                            ptx::fence_proxy_async_all();
+                        }
+                        ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
+                        if (MODE == kModeForward) {   // channels x ranks from B [r, N], MN-major: two 64-channel boxes
+                            ptx::tma_load_2d(a_s, &tmFl, r0, lb * 64, bar);
+                            ptx::tma_load_2d(a_s + 8192, &tmFl, r0 + 64, lb * 64, bar);
+                        } else {                      // features x ranks from A [K, r], K-major: one 64 x 128 box
+                            ptx::tma_load_2d(a_s, &tmFl, lb * 64, r0, bar);
+                        }
+                        ptx::tma_load_2d(b_s, &tmT, lb * 64, m0, bar);
                     }
                 }
             }
@@ -233,12 +280,13 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // ================================================================== MMA issuer
         if (lane == 0) {
             uint32_t it = 0, tile_iter = 0;
-            for (int tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x, ++tile_iter) {
+            for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x, ++tile_iter) {
+                const TileInfo t = decode_tile(g);
                 const uint32_t acc = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
                 if (!ptx::mbar_wait(&bars->tmem_empty[acc], aph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileT;
-                for (int kb = 0; kb < total_blocks; ++kb, ++it) {
+                for (int kb = 0; kb < t.blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!ptx::mbar_wait(&bars->full_x[s], ph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
@@ -247,8 +295,14 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     ptx::tc_fence_after();
                     const uint32_t a_addr = ptx::smem_u32(base + s * kSmemStage);
                     const uint64_t bdesc = ptx::umma_desc_k_sw128(a_addr + kSmemA);
-                    if (MODE == kModeBackward && kb >= P.lora_blocks) {
-                        // weights tile is MN-major: 16 contraction rows = two 1024-byte groups per MMA
+                    // which operand tiles are MN-major (a contraction index is a 128-byte row of 64 operand
+                    // rows): forward - the factor tiles fetched from A [K, r] and B [r, N]; backward - the
+                    // dequantised weight tile
+                    const bool lora_blk = !t.is_t && kb >= P.main_blocks;
+                    const bool a_mn = (MODE == kModeForward) ? (t.is_t || lora_blk)
+                                                             : (MODE == kModeBackward && !t.is_t && !lora_blk);
+                    if (a_mn) {
+                        // 16 contraction rows = two 1024-byte groups per MMA
                         const uint64_t adesc = ptx::umma_desc_mn_sw128(a_addr, 8192u);
 #pragma unroll
                         for (int kk = 0; kk < kTileC / 16; ++kk)
@@ -274,10 +328,16 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         const int et = (warp - kFirstEpilogueWarp) * 32 + lane;
         uint16_t* out16 = reinterpret_cast<uint16_t*>(out_s);
-        const bool vec_ok = (P.ld_out % 8) == 0;
         uint32_t tile_iter = 0;
-        for (int tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x, ++tile_iter) {
-            const int r0 = (tile % P.tiles_r) * kTileR, m0 = (tile / P.tiles_r) * kTileT;
+        for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x, ++tile_iter) {
+            const TileInfo t = decode_tile(g);
+            const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
+            // a T tile writes the down-projected activations [M, rp] (scaled by s); a weight tile writes Y / dX
+            uint16_t* out = t.is_t ? P.T : P.out;
+            const int ld = t.is_t ? P.rp : P.ld_out;
+            const int R = t.is_t ? P.rp : P.R;
+            const float scale = t.is_t ? P.s : 1.0f;
+            const bool vec_ok = (ld % 8) == 0;
             const uint32_t acc = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
             // the four epilogue warps share named barriers, so they must agree on leaving
             if (!ptx::mbar_wait_warp(&bars->tmem_full[acc], aph, abort_flag, kWaitLimitNs)) bars->abort = 1u;
@@ -293,7 +353,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // thread = operand row (channel), v[j] = token j: transpose through shared memory
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    const uint32_t two = pack_bf16x2(__uint_as_float(v[j]), 0.0f);
+                    const uint32_t two = pack_bf16x2(scale * __uint_as_float(v[j]), 0.0f);
                     out16[j * kTileR + q * 32 + lane] = (uint16_t)two;
                 }
                 ptx::named_barrier_sync(1, 128);
@@ -302,14 +362,14 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     const int idx = i * 128 + et;
                     const int row = idx >> 4, ch = idx & 15;
                     const int m = m0 + chunk * 32 + row, n = r0 + ch * 8;
-                    if (m < P.M && n < P.R) {
+                    if (m < P.M && n < R) {
                         const uint4 val = *reinterpret_cast<const uint4*>(out16 + row * kTileR + ch * 8);
-                        uint16_t* dst = P.out + (size_t)m * P.ld_out + n;
-                        if (vec_ok && n + 8 <= P.R) {
+                        uint16_t* dst = out + (size_t)m * ld + n;
+                        if (vec_ok && n + 8 <= R) {
                             *reinterpret_cast<uint4*>(dst) = val;
                         } else {
                             const uint16_t* e = reinterpret_cast<const uint16_t*>(&val);
-                            for (int t = 0; t < 8 && n + t < P.R; ++t) dst[t] = e[t];
+                            for (int k = 0; k < 8 && n + k < R; ++k) dst[k] = e[k];
                         }
                     }
                 }
@@ -318,29 +378,49 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(&bars->tmem_empty[acc]);
+            if (t.is_t) {
+                // publish T of this token tile: every writer fences, then one thread raises the flag
+                __threadfence();
+                ptx::named_barrier_sync(1, 128);
+                if (et == 0) {
+                    ptx::fence_proxy_async_all();
+                    ptx::flag_release(P.flags + t.mt, 1u);
+                }
+            }
         }
     } else if (MODE != kModeDense) {
         // ================================================================== dequant producers
-        // All eight warps work on every stage.  The prologue has dealt the rows of every group to the 256
-        // threads so that a warp only ever holds rows of one precision (chunks of at most 32 rows forward,
-        // 16 rows x 2 feature halves backward), so no warp runs more than one code path.  Each thread
-        // dequantises one 64-element absmax block per stage; the packed codes of the next two stages are
-        // already in registers (a two-deep ring with static indices, so no load is waited on early).
+        // All eight warps take part in every stage.  The prologue has dealt the rows of every group to the
+        // 256 threads so that a warp only ever holds rows of one precision (chunks of at most 32 rows
+        // forward, 16 rows x 2 feature halves backward); with n chunks, 8 / n warps share a chunk and take
+        // turns.  Each thread dequantises one 64-element absmax block per turn; the packed codes of the next
+        // two stages are already in registers (a two-deep ring with static indices, so no load is waited
+        // on early).
         const int pt = threadIdx.x - kFirstProducerWarp * 32;  // 0..255
         const uint32_t slut_addr = ptx::smem_u32(slut_all) + (uint32_t)((pt >> 5) * 2048 + lane * 4);
         const int K = P.L.K;
         uint32_t it0 = 0;                                       // running stage index at the start of the tile
-        for (int tile = blockIdx.x; tile < n_tiles && !failed; tile += gridDim.x, it0 += total_blocks) {
-            const int rt = tile % P.tiles_r;
-            const int r0 = rt * kTileR;
-            if (MODE == kModeForward) {
+        for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x) {
+            const TileInfo t = decode_tile(g);
+            const int r0 = t.rt * kTileR;
+            if (t.is_t) {
+                // nothing to dequantise: keep the stage barriers in step
+                for (int kb = 0; kb < t.blocks; ++kb) {
+                    const uint32_t it = it0 + (uint32_t)kb;
+                    const int s = it % kStages;
+                    if (!ptx::mbar_wait_warp(&bars->empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                        failed = true; bars->abort = 1u; break;
+                    }
+                    if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
+                }
+            } else if (MODE == kModeForward) {
                 // ---------------------------------------------------------------- forward
                 // thread = one output channel of the tile, 64 input features per stage; operand tile is
                 // [128 channels][64 features], K-major.
-                const uint32_t item = __ldg(P.items + (size_t)rt * 256 + pt);
-                const int nch = (int)__ldg(P.n_chunks + rt);
+                const uint32_t item = __ldg(P.items + (size_t)t.rt * 256 + pt);
+                const int nch = (int)__ldg(P.n_chunks + t.rt);
                 const int turn_mask = 8 / nch - 1;            // k - 1, k = warps per chunk (a power of two)
-                const int phase = (pt >> 5) / nch;            // this warp serves main blocks mb with (mb & turn_mask) == phase
+                const int phase = (pt >> 5) / nch;            // this warp serves the blocks mb with (mb & turn_mask) == phase
                 const bool active = item != kIdleItem;
                 const int cls = active ? info_class(item) : 4;
                 const int wcls = __shfl_sync(0xffffffffu, cls, 0);   // lane 0 always holds a row if the warp does
@@ -369,49 +449,45 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
                 ring[0].a = ring[1].a = 0.0f;
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {   // ring slot u serves the stages kb with kb % 2 == u
-                    const int mb = ((P.lora_blocks + 1 - u) & ~1) + u - P.lora_blocks;  // first main block of slot u
-                    if (cls < 3 && mb < P.main_blocks && (mb & turn_mask) == phase)
-                        load_block(ring[u], bits_ptr + (size_t)mb * bits_stride, absmax_ptr + mb, cls);
-                }
-                for (int kb0 = 0; kb0 < total_blocks && !failed; kb0 += 2) {
+                for (int u = 0; u < 2; ++u)   // ring slot u serves the blocks mb with mb % 2 == u
+                    if (cls < 3 && u < P.main_blocks && (u & turn_mask) == phase)
+                        load_block(ring[u], bits_ptr + (size_t)u * bits_stride, absmax_ptr + u, cls);
+                for (int kb0 = 0; kb0 < t.blocks && !failed; kb0 += 2) {
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const int kb = kb0 + u;
-                        if (kb >= total_blocks) break;
-                        const uint32_t it = it0 + (uint32_t)kb;
+                        const int mb = kb0 + u;
+                        if (mb >= t.blocks) break;
+                        const uint32_t it = it0 + (uint32_t)mb;
                         const int s = it % kStages;
                         const uint32_t ph = (it / kStages) & 1u;
                         if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
                             failed = true; bars->abort = 1u; break;
                         }
-                        const int mb = kb - P.lora_blocks;
-                        if (mb >= 0 && wcls < 4 && (mb & turn_mask) == phase) {
-                            if (active) {
-                                const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + row_off;
-                                if (wcls == 0) {
-                                    dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lv.m0, lv.m1, ring[u].a, row_addr, swz);
-                                } else if (wcls == 1) {
-                                    dequant_block_2bit(ring[u].lo, lv, ring[u].a, row_addr, swz);
-                                } else if (wcls == 2) {
-                                    Levels16 l16;
-                                    const float4* m4 = reinterpret_cast<const float4*>(mrow);   // stays in L1
+                        const bool my_turn = mb < P.main_blocks && wcls < 4 && (mb & turn_mask) == phase;
+                        if (my_turn && active) {
+                            const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + row_off;
+                            if (wcls == 0) {
+                                dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lv.m0, lv.m1, ring[u].a, row_addr, swz);
+                            } else if (wcls == 1) {
+                                dequant_block_2bit(ring[u].lo, lv, ring[u].a, row_addr, swz);
+                            } else if (wcls == 2) {
+                                Levels16 l16;
+                                const float4* m4 = reinterpret_cast<const float4*>(mrow);   // stays in L1
 #pragma unroll
-                                    for (int e = 0; e < 4; ++e) {
-                                        const float4 t = __ldg(m4 + e);
-                                        l16.v[4 * e] = t.x; l16.v[4 * e + 1] = t.y; l16.v[4 * e + 2] = t.z; l16.v[4 * e + 3] = t.w;
-                                    }
-                                    dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, l16, slut_addr, row_addr, swz);
-                                } else {
-                                    zero_row(row_addr);
+                                for (int e = 0; e < 4; ++e) {
+                                    const float4 f = __ldg(m4 + e);
+                                    l16.v[4 * e] = f.x; l16.v[4 * e + 1] = f.y; l16.v[4 * e + 2] = f.z; l16.v[4 * e + 3] = f.w;
                                 }
-                                ptx::fence_proxy_async_smem();
+                                dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, l16, slut_addr, row_addr, swz);
+                            } else {
+                                zero_row(row_addr);
                             }
+                            ptx::fence_proxy_async_smem();
                         }
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
                         const int nb = mb + 2;   // this ring slot's next stage
-                        if (cls < 3 && mb >= 0 && nb < P.main_blocks && (nb & turn_mask) == phase)
+                        if (cls < 3 && nb < P.main_blocks && (nb & turn_mask) == phase)
                             load_block(ring[u], bits_ptr + (size_t)nb * bits_stride, absmax_ptr + nb, cls);
                     }
                 }
@@ -420,7 +496,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // every stage brings 64 new channels (the contraction index); thread = one channel x 64 of
                 // the tile's 128 input features = one absmax block.  Operand tile is MN-major:
                 // [feature half][64 channels][64 features], so the block is one 128-byte row and is
-                // written exactly as in the forward case.
+                // written exactly as in the forward case.  The deal (and the turn-taking) is per stage.
                 const int half = (lane >> 4) & 1;
                 const int k_first = r0 + 64 * half;
                 const uint32_t* items = P.items + pt;
@@ -459,36 +535,34 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             P.maps + (size_t)(mb * kTileC + info_row(info)) * kTableStride);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
-                            const float4 t = __ldg(m4 + e);
-                            m16.v[4 * e] = t.x; m16.v[4 * e + 1] = t.y; m16.v[4 * e + 2] = t.z; m16.v[4 * e + 3] = t.w;
+                            const float4 f = __ldg(m4 + e);
+                            m16.v[4 * e] = f.x; m16.v[4 * e + 1] = f.y; m16.v[4 * e + 2] = f.z; m16.v[4 * e + 3] = f.w;
                         }
                     }
                 };
 
-                // prologue: first two main blocks fully, row descriptors of the next two
+                // prologue: blocks 0 and 1 fully, row descriptors of blocks 2 and 3
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    const int mb = ((P.lora_blocks + 1 - u) & ~1) + u - P.lora_blocks;  // first main block of slot u
-                    if (mb < P.main_blocks) {
-                        cur_info[u] = __ldg(items + (size_t)mb * 256);
-                        fetch(ring[u], lvr[u], cur_info[u], mb);
+                    if (u < P.main_blocks) {
+                        cur_info[u] = __ldg(items + (size_t)u * 256);
+                        fetch(ring[u], lvr[u], cur_info[u], u);
                     }
-                    info_ring[u] = (mb + 2 < P.main_blocks) ? __ldg(items + (size_t)(mb + 2) * 256) : kIdleItem;
+                    info_ring[u] = (u + 2 < P.main_blocks) ? __ldg(items + (size_t)(u + 2) * 256) : kIdleItem;
                 }
-                if (P.main_blocks > 0) fetch_table(cur_info[P.lora_blocks & 1], 0);
-                for (int kb0 = 0; kb0 < total_blocks && !failed; kb0 += 2) {
+                if (P.main_blocks > 0) fetch_table(cur_info[0], 0);
+                for (int kb0 = 0; kb0 < t.blocks && !failed; kb0 += 2) {
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const int kb = kb0 + u;
-                        if (kb >= total_blocks) break;
-                        const uint32_t it = it0 + (uint32_t)kb;
+                        const int mb = kb0 + u;
+                        if (mb >= t.blocks) break;
+                        const uint32_t it = it0 + (uint32_t)mb;
                         const int s = it % kStages;
                         const uint32_t ph = (it / kStages) & 1u;
                         if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
                             failed = true; bars->abort = 1u; break;
                         }
-                        const int mb = kb - P.lora_blocks;
-                        if (mb >= 0) {
+                        if (mb < P.main_blocks) {
                             const uint32_t info = cur_info[u];
                             const bool active = info != kIdleItem;
                             const int wcls = __shfl_sync(0xffffffffu, active ? info_class(info) : 4, 0);
@@ -508,16 +582,14 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         // refill this ring slot for its next stage (block mb + 2), fetch the 4-bit table of the
                         // very next stage (block mb + 1, other slot), look two stages further ahead for the row
                         const int nb = mb + 2;
-                        if (mb >= 0) {
-                            cur_info[u] = info_ring[u];
-                            if (nb < P.main_blocks) fetch(ring[u], lvr[u], cur_info[u], nb);
-                            info_ring[u] = (nb + 2 < P.main_blocks) ? __ldg(items + (size_t)(nb + 2) * 256) : kIdleItem;
-                        }
-                        const int tb = mb + 1;
-                        if (tb >= 1 && tb < P.main_blocks) fetch_table(cur_info[u ^ 1], tb);
+                        cur_info[u] = info_ring[u];
+                        if (nb < P.main_blocks) fetch(ring[u], lvr[u], cur_info[u], nb);
+                        info_ring[u] = (nb + 2 < P.main_blocks) ? __ldg(items + (size_t)(nb + 2) * 256) : kIdleItem;
+                        if (mb + 1 < P.main_blocks) fetch_table(cur_info[u ^ 1], mb + 1);
                     }
                 }
             }
+            it0 += (uint32_t)t.blocks;
         }
     }
 
@@ -532,8 +604,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
 }
 
 template <int MODE>
-static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmB2,
-                                const CUtensorMap& tmA2, cudaStream_t stream) {
+static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
+                                const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
     static bool configured = false;
     if (!configured) {
         if (cudaFuncSetAttribute(fused_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -541,17 +613,17 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
             return LOWRA_ERR_CUDA;
         configured = true;
     }
-    const int n_tiles = G.tiles_r * G.tiles_t;
+    const int n_tiles = G.tiles_r * G.tiles_t + ((MODE != kModeDense && G.lora_blocks > 0) ? G.tiles_t : 0);
     const int grid = n_tiles < kNumSMs ? n_tiles : kNumSMs;
-    fused_kernel<MODE><<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(G, tmB, tmB2, tmA2);
+    fused_kernel<MODE><<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(G, tmB, tmT, tmFt, tmFl);
     return cudaGetLastError() == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
 }
 
-lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmB2,
-                          const CUtensorMap& tmA2, cudaStream_t stream) {
-    if (mode == kModeForward) return launch_mode<kModeForward>(G, tmB, tmB2, tmA2, stream);
-    if (mode == kModeBackward) return launch_mode<kModeBackward>(G, tmB, tmB2, tmA2, stream);
-    return launch_mode<kModeDense>(G, tmB, tmB2, tmA2, stream);
+lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
+                          const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
+    if (mode == kModeForward) return launch_mode<kModeForward>(G, tmB, tmT, tmFt, tmFl, stream);
+    if (mode == kModeBackward) return launch_mode<kModeBackward>(G, tmB, tmT, tmFt, tmFl, stream);
+    return launch_mode<kModeDense>(G, tmB, tmT, tmFt, tmFl, stream);
 }
 
 }  // namespace lowra

@@ -16,21 +16,22 @@ constexpr size_t kStatusBytes = 256;
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Workspace {
-    size_t off_T, off_F2, off_info, off_meta, total;
+    size_t off_T, off_flags, off_items, off_meta, total;
     int rp;
 };
 
 bool rank_ok(int r) { return r >= 16 && r <= 128 && r % 16 == 0; }
 
 Workspace plan_workspace(int N, int K, int M, int r) {
+    (void)K;
     Workspace w;
     w.rp = (r + 63) / 64 * 64;
-    const int big = N > K ? N : K;
+    const size_t groups = (size_t)(N + 63) / 64;   // backward has the most row groups
     w.off_T = kStatusBytes;
-    w.off_F2 = w.off_T + align256((size_t)M * w.rp * 2);
-    w.off_info = w.off_F2 + align256((size_t)big * w.rp * 2);
-    w.off_meta = w.off_info + align256((size_t)((N + 63) / 64) * 256 * 4);
-    w.total = w.off_meta + align256((size_t)((N + 63) / 64) * 4);
+    w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);
+    w.off_items = w.off_flags + align256((size_t)((M + kTileT - 1) / kTileT) * 4);
+    w.off_meta = w.off_items + align256(groups * 256 * 4);
+    w.total = w.off_meta + align256(groups * 4);
     return w;
 }
 
@@ -79,43 +80,30 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     cudaStream_t stream = (cudaStream_t)stream_v;
 
     unsigned char* ws = static_cast<unsigned char*>(workspace);
-    uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
-    uint16_t* F2 = reinterpret_cast<uint16_t*>(ws + w.off_F2);
-    uint32_t* items = reinterpret_cast<uint32_t*>(ws + w.off_info);
     uint32_t* status = reinterpret_cast<uint32_t*>(ws);
+    uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
+    uint32_t* flags = reinterpret_cast<uint32_t*>(ws + w.off_flags);
+    uint32_t* items = reinterpret_cast<uint32_t*>(ws + w.off_items);
+    uint32_t* n_chunks = reinterpret_cast<uint32_t*>(ws + w.off_meta);
+    const int tiles_t = (M + kTileT - 1) / kTileT;
 
-    // ---- prologue
+    // ---- prologue: clear status and flags, deal the rows
     PrepParams P;
     memset(&P, 0, sizeof(P));
-    P.In = act;
-    P.M = M;
-    P.r = r;
-    P.rp = w.rp;
-    P.s = s;
-    P.T = T;
-    P.Dst = F2;
     P.precs = layout->precs_dev;
     P.inv_perm = layout->inv_perm_dev;
     P.items = items;
-    P.n_chunks = reinterpret_cast<uint32_t*>(ws + w.off_meta);
+    P.n_chunks = n_chunks;
     P.N = N;
+    P.group = backward ? 64 : 128;
     P.status = status;
-    if (!backward) {
-        P.C = K; P.F = A; P.f_is_A = 1;            // T = s X A
-        P.Src = B; P.R = N; P.src_transposed = 1;  // Bt[n, j] = B[j, n]
-        P.group = 128;
-    } else {
-        P.C = N; P.F = B; P.f_is_A = 0;            // U = s dY B^T
-        P.Src = A; P.R = K; P.src_transposed = 0;  // Ap[k, j] = A[k, j]
-        P.group = 64;
-    }
-    P.blocksA = (M + kPrepTokens - 1) / kPrepTokens;
-    P.blocksB = 32;
-    P.blocksC = ((N + P.group - 1) / P.group + 3) / 4;
+    P.flags = flags;
+    P.n_flags = tiles_t;
+    P.blocks = ((N + P.group - 1) / P.group + 3) / 4;
     st = launch_prep(P, stream);
     if (st != LOWRA_OK) return st;
 
-    // ---- fused kernel
+    // ---- fused kernel (its first tiles compute T = s X A, resp. U = s dY B^T)
     GemmParams G;
     memset(&G, 0, sizeof(G));
     G.L = make_row_layout(layout);
@@ -123,9 +111,13 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.absmax = absmax;
     G.maps = maps;
     G.items = items;
-    G.n_chunks = reinterpret_cast<uint32_t*>(ws + w.off_meta);
+    G.n_chunks = n_chunks;
     G.out = out;
+    G.T = T;
+    G.flags = flags;
     G.status = status;
+    G.s = s;
+    G.rp = w.rp;
     G.M = M;
     G.R = backward ? K : N;
     G.C = backward ? N : K;
@@ -133,12 +125,20 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.main_blocks = (G.C + kTileC - 1) / kTileC;
     G.lora_blocks = w.rp / kTileC;
     G.tiles_r = (G.R + kTileR - 1) / kTileR;
-    G.tiles_t = (M + kTileT - 1) / kTileT;
-    CUtensorMap tmB, tmB2, tmA2;
+    G.tiles_t = tiles_t;
+    CUtensorMap tmB, tmT, tmFt, tmFl;
     if (!make_map(&tmB, act, (uint64_t)M, (uint64_t)G.C, (uint64_t)G.C, kTileT)) return LOWRA_ERR_CUDA;
-    if (!make_map(&tmB2, T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
-    if (!make_map(&tmA2, F2, (uint64_t)G.R, (uint64_t)w.rp, (uint64_t)w.rp, kTileR)) return LOWRA_ERR_CUDA;
-    return launch_fused(backward ? kModeBackward : kModeForward, G, tmB, tmB2, tmA2, stream);
+    if (!make_map(&tmT, T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
+    if (!backward) {
+        // T tiles take ranks x features from A [K, r] (64 x 64 boxes); LoRA blocks take channels x ranks from B [r, N]
+        if (!make_map(&tmFt, A, (uint64_t)K, (uint64_t)r, (uint64_t)r, 64)) return LOWRA_ERR_CUDA;
+        if (!make_map(&tmFl, B, (uint64_t)r, (uint64_t)N, (uint64_t)N, 64)) return LOWRA_ERR_CUDA;
+    } else {
+        // T tiles take ranks x channels from B [r, N]; LoRA blocks take features x ranks from A [K, r] (64 x 128 boxes)
+        if (!make_map(&tmFt, B, (uint64_t)r, (uint64_t)N, (uint64_t)N, kTileR)) return LOWRA_ERR_CUDA;
+        if (!make_map(&tmFl, A, (uint64_t)K, (uint64_t)r, (uint64_t)r, kTileR)) return LOWRA_ERR_CUDA;
+    }
+    return launch_fused(backward ? kModeBackward : kModeForward, G, tmB, tmT, tmFt, tmFl, stream);
 }
 
 __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
@@ -259,8 +259,8 @@ extern "C" lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_
     G.lora_blocks = 0;
     G.tiles_r = (N + kTileR - 1) / kTileR;
     G.tiles_t = (M + kTileT - 1) / kTileT;
-    CUtensorMap tmB, tmA2;
+    CUtensorMap tmB, tmFl;
     if (!make_map(&tmB, P_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, kTileT)) return LOWRA_ERR_CUDA;
-    if (!make_map(&tmA2, Q_dev, (uint64_t)N, (uint64_t)K, (uint64_t)K, kTileR)) return LOWRA_ERR_CUDA;
-    return launch_fused(kModeDense, G, tmB, tmB, tmA2, stream);
+    if (!make_map(&tmFl, Q_dev, (uint64_t)N, (uint64_t)K, (uint64_t)K, kTileR)) return LOWRA_ERR_CUDA;
+    return launch_fused(kModeDense, G, tmB, tmB, tmB, tmFl, stream);
 }

@@ -9,29 +9,20 @@ namespace lowra {
 
 // ---- prologue ------------------------------------------------------------------------------
 constexpr int kPrepThreads = 128;
-constexpr int kPrepTokens = 32;   // tokens per down-projection CTA
 
 struct PrepParams {
-    // (A) T[m, j] = bf16(s * sum_c In[m, c] * F(c, j)),  T is [M, rp]
-    const uint16_t* In;   // [M, C] bf16
-    const uint16_t* F;    // f_is_A: A [C, r] (F(c,j) = F[c*r + j]);  else B [r, C] (F(c,j) = F[j*C + c])
-    uint16_t* T;
-    int M, C, r, rp, f_is_A;
-    float s;
-    // (B) Dst [R, rp]: src_transposed: Dst[n, j] = Src[j*R + n];  else Dst[k, j] = Src[k*r + j]
-    const uint16_t* Src;
-    uint16_t* Dst;
-    int R, src_transposed;
-    // (C) deal of the rows of every group (128 rows forward, 64 backward) to the 256 dequant threads of
-    // the main kernel, one precision per warp: items[g * 256 + thread] = row offset (bits 0-6) | class
+    // deal of the rows of every group (128 rows forward, 64 backward) to the 256 dequant threads of the
+    // main kernel, one precision per warp: items[g * 256 + thread] = row offset (bits 0-6) | class
     // (bits 7-8, 3 = row past N) | stored position (bits 9-31), or all ones for "no row"
     const uint8_t* precs;
     const int32_t* inv_perm;
     uint32_t* items;      // [ceil(N / group) * 256]
     uint32_t* n_chunks;   // [ceil(N / group)] number of chunks the group was cut into (1..7)
     int N, group;
-    uint32_t* status;
-    int blocksA, blocksB, blocksC;
+    uint32_t* status;     // device status word, cleared
+    uint32_t* flags;      // [n_flags] "T of this token tile is ready" flags, cleared
+    int n_flags;
+    int blocks;
 };
 
 lowra_status launch_prep(const PrepParams& P, cudaStream_t stream);
@@ -57,7 +48,11 @@ struct GemmParams {
     const uint32_t* items;    // from the prologue: [row groups][256 dequant threads]
     const uint32_t* n_chunks; // from the prologue: [row groups]
     uint16_t* out;          // [M, ld_out] bf16
+    uint16_t* T;            // [M, rp] bf16: s * X . A (forward) or s * dY . B^T (backward), written by the T tiles
+    uint32_t* flags;        // [tiles_t] raised when T of a token tile is complete
     uint32_t* status;
+    float s;
+    int rp;                 // LoRA rank rounded up to 64
     int M;                  // tokens
     int R;                  // A-operand rows in total: N (forward, dense) or K (backward)
     int C;                  // main contraction length: K (forward, dense) or N (backward)
@@ -75,7 +70,7 @@ constexpr uint32_t kSmemLut4 = kProducerWarps * 32 * 16 * 4;  // per dequant lan
 constexpr uint32_t kSmemBarriers = 1024;
 constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kStages * kSmemStage + kSmemOut + kSmemLut4 + kSmemBarriers;
 
-lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmB2,
-                          const CUtensorMap& tmA2, cudaStream_t stream);
+lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
+                          const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream);
 
 }  // namespace lowra

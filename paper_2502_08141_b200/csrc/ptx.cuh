@@ -83,6 +83,27 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
+// generic <-> async proxy fence over every state space (used around TMA reads of data that another
+// CTA wrote to global memory with ordinary stores)
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Global-memory flag between CTAs: release store / bounded acquire poll.
+__device__ __forceinline__ void flag_release(uint32_t* flag, uint32_t value) {
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
+}
+__device__ __forceinline__ bool flag_wait(const uint32_t* flag, volatile uint32_t* abort, uint64_t limit_ns) {
+    const uint64_t t0 = globaltimer_ns();
+#pragma unroll 1
+    for (;;) {
+        uint32_t v;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+        if (v != 0u) return true;
+        __nanosleep(64);
+        if (abort != nullptr && *abort != 0u) return false;
+        if (globaltimer_ns() - t0 > limit_ns) return false;
+    }
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
