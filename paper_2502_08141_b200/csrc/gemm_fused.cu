@@ -27,6 +27,9 @@ namespace {
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 constexpr uint32_t kIdesc = ptx::umma_idesc_bf16(kTileR, kTileT);
 constexpr uint32_t kIdescAmn = kIdesc | (1u << 15);   // A operand MN-major
+// Forward keeps the dequantised weights in tensor memory: one 128 x 256 accumulator (columns 0-255) and one
+// 32-column operand slot per pipeline stage behind it.
+constexpr uint32_t kTmemASlots = 256;
 
 struct Barriers {
     uint64_t full_x[kStages];   // TMA bytes of a stage have landed
@@ -67,66 +70,49 @@ __device__ __forceinline__ void load_block(Block& blk, const uint8_t* p, const f
 
 struct Levels { float m0, m1, m2, m3; };
 
-// Chunk t (elements 8t .. 8t+7) of the row goes to physical 16-byte slot t ^ swz (128B swizzle).
-__device__ __forceinline__ void store_chunk(uint32_t row_addr, int swz, int t, uint32_t o0, uint32_t o1, uint32_t o2,
-                                            uint32_t o3) {
-    ptx::st_shared_v4(row_addr + (uint32_t)((t ^ swz) << 4), make_uint4(o0, o1, o2, o3));
-}
-
+// ---- cores: one 64-element block -> 32 words of bf16 pairs (element 2i in the low half of o[i]) --------
 // 1 bit.  L, H = bf16(level0 * absmax), bf16(level1 * absmax) as 16-bit patterns; BB = min(L,H) in both
 // halves, d = |H - L|, f = 0x10001 if L > H else 0.  A half takes min + d exactly when its (possibly
 // flipped) code bit is set, so one multiply-add forms two elements without any carry between halves.
 // 16 code bits h are spread once (z = h | h << 15) so that pair j sits at bits 0 and 16 of z >> 2j.
-__device__ __noinline__ void dequant_block_1bit(uint32_t w0, uint32_t w1, float m0, float m1, float a,
-                                                uint32_t row_addr, int swz) {
+__device__ __forceinline__ void deq64_1bit(uint32_t w0, uint32_t w1, float m0, float m1, float a, uint32_t (&o)[32]) {
     const uint32_t LH = pack_bf16x2(__fmul_rn(m0, a), __fmul_rn(m1, a));
     const uint32_t L = LH & 0xFFFFu, H = LH >> 16;
     const uint32_t lo = min(L, H);
     const uint32_t BB = lo * 0x10001u, d = max(L, H) - lo, f = (L > H) ? 0x10001u : 0u;
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {  // 16 elements = two chunks per iteration
+    for (int q = 0; q < 4; ++q) {  // 16 elements per iteration
         const uint32_t w = (q < 2) ? w0 : w1;
         const uint32_t h = (q & 1) ? (w >> 16) : (w & 0xFFFFu);
         const uint32_t z = h | (h << 15);
-        uint32_t o[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) o[j] = (((z >> (2 * j)) & 0x10001u) ^ f) * d + BB;
-        store_chunk(row_addr, swz, 2 * q, o[0], o[1], o[2], o[3]);
-        store_chunk(row_addr, swz, 2 * q + 1, o[4], o[5], o[6], o[7]);
+        for (int j = 0; j < 8; ++j) o[8 * q + j] = (((z >> (2 * j)) & 0x10001u) ^ f) * d + BB;
     }
 }
 
 // 2 bits: E01 = {level0, level1} * absmax, E23 = {level2, level3} * absmax, bf16x2 each; a byte
 // permute picks the two 16-bit entries named by a pair of codes.
-__device__ __noinline__ void dequant_block_2bit(uint4 w, Levels lv, float a, uint32_t row_addr, int swz) {
+__device__ __forceinline__ void deq64_2bit(const uint4& w, const Levels& lv, float a, uint32_t (&o)[32]) {
     const uint32_t E01 = pack_bf16x2(__fmul_rn(lv.m0, a), __fmul_rn(lv.m1, a));
     const uint32_t E23 = pack_bf16x2(__fmul_rn(lv.m2, a), __fmul_rn(lv.m3, a));
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {  // one 32-bit word = 16 elements = two chunks
+    for (int q = 0; q < 4; ++q) {  // one 32-bit word = 16 elements
         const uint32_t x = q == 0 ? w.x : q == 1 ? w.y : q == 2 ? w.z : w.w;
-        uint32_t o[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint32_t y = x >> (4 * j);
             const uint32_t t = (y & 3u) | ((y << 6) & 0x300u);
-            o[j] = __byte_perm(E01, E23, t * 0x22u + 0x1010u);
+            o[8 * q + j] = __byte_perm(E01, E23, t * 0x22u + 0x1010u);
         }
-        store_chunk(row_addr, swz, 2 * q, o[0], o[1], o[2], o[3]);
-        store_chunk(row_addr, swz, 2 * q + 1, o[4], o[5], o[6], o[7]);
     }
-}
-
-__device__ __noinline__ void zero_row(uint32_t row_addr) {
-#pragma unroll
-    for (int t = 0; t < 8; ++t) ptx::st_shared_v4(row_addr + 16u * t, make_uint4(0u, 0u, 0u, 0u));
 }
 
 // 4 bits.  The 16 levels are scaled by the block's absmax and rounded to bf16 exactly as the decode
 // kernel does, into a per-lane table in shared memory (entry e of lane l at slut[e * 32 + l], so the
-// warp's lookups never collide on a bank); each code is then one shift/mask and one 16-bit load.
+// warp's lookups never collide on a bank); each code is then one shift/mask and one load.
 struct Levels16 { float v[16]; };
-__device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, Levels16 lv, uint32_t slut_addr,
-                                                uint32_t row_addr, int swz) {
+__device__ __forceinline__ void deq64_4bit(const uint4& lo, const uint4& hi, float a, const Levels16& lv,
+                                           uint32_t slut_addr, uint32_t (&o)[32]) {
 #pragma unroll
     for (int e = 0; e < 16; e += 2) {
         const uint32_t two = pack_bf16x2(__fmul_rn(lv.v[e], a), __fmul_rn(lv.v[e + 1], a));
@@ -134,7 +120,7 @@ __device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, Lev
         asm volatile("st.shared.u32 [%0], %1;" ::"r"(slut_addr + (uint32_t)(e + 1) * 128u), "r"(two >> 16) : "memory");
     }
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {  // one 32-bit word = 8 elements = one chunk
+    for (int q = 0; q < 8; ++q) {  // one 32-bit word = 8 elements
         const uint32_t w = q == 0 ? lo.x : q == 1 ? lo.y : q == 2 ? lo.z : q == 3 ? lo.w
                          : q == 4 ? hi.x : q == 5 ? hi.y : q == 6 ? hi.z : hi.w;
         uint32_t v[8];
@@ -143,11 +129,88 @@ __device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, Lev
             // byte offset of entry c = (w >> 4j) & 15 is c * 128
             const uint32_t off = (j == 0) ? ((w << 7) & 0x780u) : (j == 1) ? ((w << 3) & 0x780u)
                                                                            : ((w >> (j < 2 ? 0 : 4 * j - 7)) & 0x780u);
-            asm("ld.shared.u32 %0, [%1];" : "=r"(v[j]) : "r"(slut_addr + off));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[j]) : "r"(slut_addr + off) : "memory");
         }
-        store_chunk(row_addr, swz, q, __byte_perm(v[0], v[1], 0x5410), __byte_perm(v[2], v[3], 0x5410),
-                    __byte_perm(v[4], v[5], 0x5410), __byte_perm(v[6], v[7], 0x5410));
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[4 * q + j] = __byte_perm(v[2 * j], v[2 * j + 1], 0x5410);
     }
+}
+
+// ---- shared-memory operand (backward): the block is one 128-byte row of the swizzled tile ----------
+// Chunk t (elements 8t .. 8t+7) of the row goes to physical 16-byte slot t ^ swz (128B swizzle).
+__device__ __forceinline__ void store_row(uint32_t row_addr, int swz, const uint32_t (&o)[32]) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t)
+        ptx::st_shared_v4(row_addr + (uint32_t)((t ^ swz) << 4), make_uint4(o[4 * t], o[4 * t + 1], o[4 * t + 2], o[4 * t + 3]));
+}
+
+// Deliberately not inlined: the hot code of the dequant warps must stay small.
+__device__ __noinline__ void dequant_block_1bit(uint32_t w0, uint32_t w1, float m0, float m1, float a,
+                                                uint32_t row_addr, int swz) {
+    uint32_t o[32];
+    deq64_1bit(w0, w1, m0, m1, a, o);
+    store_row(row_addr, swz, o);
+}
+__device__ __noinline__ void dequant_block_2bit(uint4 w, Levels lv, float a, uint32_t row_addr, int swz) {
+    uint32_t o[32];
+    deq64_2bit(w, lv, a, o);
+    store_row(row_addr, swz, o);
+}
+__device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, Levels16 lv, uint32_t slut_addr,
+                                                uint32_t row_addr, int swz) {
+    uint32_t o[32];
+    deq64_4bit(lo, hi, a, lv, slut_addr, o);
+    store_row(row_addr, swz, o);
+}
+__device__ __noinline__ void zero_row(uint32_t row_addr) {
+#pragma unroll
+    for (int t = 0; t < 8; ++t) ptx::st_shared_v4(row_addr + 16u * t, make_uint4(0u, 0u, 0u, 0u));
+}
+
+// ---- tensor-memory operand (forward): thread = operand row = TMEM lane -----------------------------
+// The whole warp writes its 32 lanes x 32 columns (64 bf16 per row) with one tcgen05.st; rows of different
+// precision in the warp take their own branch first (at most two classes meet in a warp, see the deal).
+__device__ __noinline__ void produce_block_tmem(Block blk, int cls, Levels lv, const float* mrow, uint32_t slut_addr,
+                                                uint32_t taddr) {
+    uint32_t o[32];
+    if (cls == 0) {
+        deq64_1bit(blk.lo.x, blk.lo.y, lv.m0, lv.m1, blk.a, o);
+    } else if (cls == 1) {
+        deq64_2bit(blk.lo, lv, blk.a, o);
+    } else if (cls == 2) {
+        Levels16 l16;
+        const float4* m4 = reinterpret_cast<const float4*>(mrow);   // stays in L1 for the whole tile
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const float4 f = __ldg(m4 + e);
+            l16.v[4 * e] = f.x; l16.v[4 * e + 1] = f.y; l16.v[4 * e + 2] = f.z; l16.v[4 * e + 3] = f.w;
+        }
+        deq64_4bit(blk.lo, blk.hi, blk.a, l16, slut_addr, o);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = 0u;
+    }
+    __syncwarp();
+    ptx::tmem_st_32x32(taddr, o);
+    ptx::tmem_st_wait();
+}
+
+// LoRA up-projection factor for the forward pass: row = output channel n, 64 ranks starting at j0, read
+// down a column of B [r, N] (the channels of a warp lie within one 128-wide window, so the 2-byte loads of
+// a warp share a few sectors).  Ranks >= r and channels >= N give zeros.
+__device__ __noinline__ void produce_lora_tmem(const uint16_t* B, int N, int r, int n, int j0, uint32_t taddr) {
+    uint32_t o[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const int j = j0 + 2 * i;
+        uint32_t lo = 0u, hi = 0u;
+        if (n < N && j < r) lo = __ldg(B + (size_t)j * N + n);
+        if (n < N && j + 1 < r) hi = __ldg(B + (size_t)(j + 1) * N + n);
+        o[i] = lo | (hi << 16);
+    }
+    __syncwarp();
+    ptx::tmem_st_32x32(taddr, o);
+    ptx::tmem_st_wait();
 }
 
 // word written by the prologue for every dequant thread and every row group: bits 0-6 row offset inside
@@ -194,7 +257,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(&bars->full_x[s], 1);
-            ptx::mbar_init(&bars->full_w[s], kProducerWarps);
+            ptx::mbar_init(&bars->full_w[s], MODE == kModeForward ? kProducerWarps / 2 : kProducerWarps);
             ptx::mbar_init(&bars->empty[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -257,11 +320,10 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             if (!ptx::flag_wait(P.flags + t.mt, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                             ptx::fence_proxy_async_all();
                         }
-                        ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
-                        if (MODE == kModeForward) {   // channels x ranks from B [r, N], MN-major: two 64-channel boxes
-                            ptx::tma_load_2d(a_s, &tmFl, r0, lb * 64, bar);
-                            ptx::tma_load_2d(a_s + 8192, &tmFl, r0 + 64, lb * 64, bar);
+                        if (MODE == kModeForward) {   // the up-projection rows are written to tensor memory by the dequant warps
+                            ptx::mbar_arrive_expect_tx(bar, kSmemB);
                         } else {                      // features x ranks from A [K, r], K-major: one 64 x 128 box
+                            ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
                             ptx::tma_load_2d(a_s, &tmFl, lb * 64, r0, bar);
                         }
                         ptx::tma_load_2d(b_s, &tmT, lb * 64, m0, bar);
@@ -282,7 +344,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             uint32_t it = 0, tile_iter = 0;
             for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x, ++tile_iter) {
                 const TileInfo t = decode_tile(g);
-                const uint32_t acc = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
+                // forward has a single accumulator, the other modes alternate between two
+                const uint32_t acc = (MODE == kModeForward) ? 0u : (tile_iter & 1u);
+                const uint32_t aph = (MODE == kModeForward) ? (tile_iter & 1u) : ((tile_iter >> 1) & 1u);
                 if (!ptx::mbar_wait(&bars->tmem_empty[acc], aph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileT;
@@ -295,13 +359,18 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     ptx::tc_fence_after();
                     const uint32_t a_addr = ptx::smem_u32(base + s * kSmemStage);
                     const uint64_t bdesc = ptx::umma_desc_k_sw128(a_addr + kSmemA);
-                    // which operand tiles are MN-major (a contraction index is a 128-byte row of 64 operand
-                    // rows): forward - the factor tiles fetched from A [K, r] and B [r, N]; backward - the
-                    // dequantised weight tile
+                    // which shared-memory operand tiles are MN-major (a contraction index is a 128-byte row of
+                    // 64 operand rows): forward - the factor tile of a T tile, fetched from A [K, r];
+                    // backward - the dequantised weight tile
                     const bool lora_blk = !t.is_t && kb >= P.main_blocks;
-                    const bool a_mn = (MODE == kModeForward) ? (t.is_t || lora_blk)
-                                                             : (MODE == kModeBackward && !t.is_t && !lora_blk);
-                    if (a_mn) {
+                    const bool a_mn = (MODE == kModeForward) ? t.is_t : (MODE == kModeBackward && !t.is_t && !lora_blk);
+                    if (MODE == kModeForward && !t.is_t) {
+                        // weights (and the LoRA up-projection rows) come from tensor memory: 8 columns per MMA
+                        const uint32_t a_tmem = tmem_base + kTmemASlots + 32u * (uint32_t)s;
+#pragma unroll
+                        for (int kk = 0; kk < kTileC / 16; ++kk)
+                            ptx::umma_bf16_ts(d_tmem, a_tmem + 8u * kk, bdesc + 2u * kk, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+                    } else if (a_mn) {
                         // 16 contraction rows = two 1024-byte groups per MMA
                         const uint64_t adesc = ptx::umma_desc_mn_sw128(a_addr, 8192u);
 #pragma unroll
@@ -338,7 +407,12 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             const int R = t.is_t ? P.rp : P.R;
             const float scale = t.is_t ? P.s : 1.0f;
             const bool vec_ok = (ld % 8) == 0;
-            const uint32_t acc = tile_iter & 1u, aph = (tile_iter >> 1) & 1u;
+            const uint32_t acc = (MODE == kModeForward) ? 0u : (tile_iter & 1u);
+            const uint32_t aph = (MODE == kModeForward) ? (tile_iter & 1u) : ((tile_iter >> 1) & 1u);
+            // forward weight tiles hold their rows in precision order: this lane's accumulator row belongs to
+            // the channel that the deal put at this position
+            int my_row = q * 32 + lane;
+            if (MODE == kModeForward && !t.is_t) my_row = info_row(__ldg(P.items + (size_t)t.rt * 256 + q * 32 + lane));
             // the four epilogue warps share named barriers, so they must agree on leaving
             if (!ptx::mbar_wait_warp(&bars->tmem_full[acc], aph, abort_flag, kWaitLimitNs)) bars->abort = 1u;
             ptx::named_barrier_sync(1, 128);
@@ -354,7 +428,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     const uint32_t two = pack_bf16x2(scale * __uint_as_float(v[j]), 0.0f);
-                    out16[j * kTileR + q * 32 + lane] = (uint16_t)two;
+                    out16[j * kTileR + my_row] = (uint16_t)two;
                 }
                 ptx::named_barrier_sync(1, 128);
 #pragma unroll
@@ -404,8 +478,10 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             const TileInfo t = decode_tile(g);
             const int r0 = t.rt * kTileR;
             if (t.is_t) {
-                // nothing to dequantise: keep the stage barriers in step
-                for (int kb = 0; kb < t.blocks; ++kb) {
+                // nothing to dequantise: keep the stage barriers in step (forward: the warps whose turn it is)
+                const int first = (MODE == kModeForward) ? ((pt >> 7) & 1) : 0;
+                const int step = (MODE == kModeForward) ? 2 : 1;
+                for (int kb = first; kb < t.blocks; kb += step) {
                     const uint32_t it = it0 + (uint32_t)kb;
                     const int s = it % kStages;
                     if (!ptx::mbar_wait_warp(&bars->empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
@@ -415,16 +491,15 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 }
             } else if (MODE == kModeForward) {
                 // ---------------------------------------------------------------- forward
-                // thread = one output channel of the tile, 64 input features per stage; operand tile is
-                // [128 channels][64 features], K-major.
-                const uint32_t item = __ldg(P.items + (size_t)t.rt * 256 + pt);
-                const int nch = (int)__ldg(P.n_chunks + t.rt);
-                const int turn_mask = 8 / nch - 1;            // k - 1, k = warps per chunk (a power of two)
-                const int phase = (pt >> 5) / nch;            // this warp serves the blocks mb with (mb & turn_mask) == phase
-                const bool active = item != kIdleItem;
-                const int cls = active ? info_class(item) : 4;
-                const int wcls = __shfl_sync(0xffffffffu, cls, 0);   // lane 0 always holds a row if the warp does
+                // thread = one output channel = one tensor-memory lane (rows of the tile in precision order, so
+                // at most two precisions meet in a warp); 64 input features per stage, written with tcgen05.st
+                // into the stage's 32-column operand slot.  The two warps that own a lane quarter take turns.
+                const int q = warp & 3;                              // lane quarter this warp may touch
+                const int turn = (pt >> 7) & 1;                      // this warp serves the blocks kb with kb % 2 == turn
+                const uint32_t item = __ldg(P.items + (size_t)t.rt * 256 + q * 32 + lane);
+                const int cls = info_class(item);
                 const int row_local = info_row(item);
+                const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + kTmemASlots;
                 Levels lv = {0.f, 0.f, 0.f, 0.f};
                 const uint8_t* bits_ptr = P.packed;
                 const float* absmax_ptr = P.absmax;
@@ -443,51 +518,38 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
                     }
                 }
-                const uint32_t row_off = (uint32_t)row_local * 128u;
-                const int swz = row_local & 7;
                 Block ring[2];
                 ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
                 ring[0].a = ring[1].a = 0.0f;
 #pragma unroll
-                for (int u = 0; u < 2; ++u)   // ring slot u serves the blocks mb with mb % 2 == u
-                    if (cls < 3 && u < P.main_blocks && (u & turn_mask) == phase)
-                        load_block(ring[u], bits_ptr + (size_t)u * bits_stride, absmax_ptr + u, cls);
-                for (int kb0 = 0; kb0 < t.blocks && !failed; kb0 += 2) {
+                for (int u = 0; u < 2; ++u) {   // ring slot u serves this warp's turns number u, u + 2, ...
+                    const int mb = turn + 2 * u;
+                    if (cls < 3 && mb < P.main_blocks)
+                        load_block(ring[u], bits_ptr + (size_t)mb * bits_stride, absmax_ptr + mb, cls);
+                }
+                for (int kb0 = turn; kb0 < t.blocks && !failed; kb0 += 4) {
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const int mb = kb0 + u;
-                        if (mb >= t.blocks) break;
-                        const uint32_t it = it0 + (uint32_t)mb;
+                        const int kb = kb0 + 2 * u;
+                        if (kb >= t.blocks) break;
+                        const uint32_t it = it0 + (uint32_t)kb;
                         const int s = it % kStages;
                         const uint32_t ph = (it / kStages) & 1u;
                         if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
                             failed = true; bars->abort = 1u; break;
                         }
-                        const bool my_turn = mb < P.main_blocks && wcls < 4 && (mb & turn_mask) == phase;
-                        if (my_turn && active) {
-                            const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + row_off;
-                            if (wcls == 0) {
-                                dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lv.m0, lv.m1, ring[u].a, row_addr, swz);
-                            } else if (wcls == 1) {
-                                dequant_block_2bit(ring[u].lo, lv, ring[u].a, row_addr, swz);
-                            } else if (wcls == 2) {
-                                Levels16 l16;
-                                const float4* m4 = reinterpret_cast<const float4*>(mrow);   // stays in L1
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    const float4 f = __ldg(m4 + e);
-                                    l16.v[4 * e] = f.x; l16.v[4 * e + 1] = f.y; l16.v[4 * e + 2] = f.z; l16.v[4 * e + 3] = f.w;
-                                }
-                                dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, l16, slut_addr, row_addr, swz);
-                            } else {
-                                zero_row(row_addr);
-                            }
-                            ptx::fence_proxy_async_smem();
+                        ptx::tc_fence_after();
+                        const uint32_t taddr = lane_addr + 32u * (uint32_t)s;
+                        if (kb < P.main_blocks) {
+                            produce_block_tmem(ring[u], cls, lv, mrow, slut_addr, taddr);
+                        } else {
+                            produce_lora_tmem(P.lora_up, P.L.N, P.r, r0 + row_local, (kb - P.main_blocks) * 64, taddr);
                         }
+                        ptx::tc_fence_before();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
-                        const int nb = mb + 2;   // this ring slot's next stage
-                        if (cls < 3 && nb < P.main_blocks && (nb & turn_mask) == phase)
+                        const int nb = kb + 4;   // this ring slot's next turn
+                        if (cls < 3 && nb < P.main_blocks)
                             load_block(ring[u], bits_ptr + (size_t)nb * bits_stride, absmax_ptr + nb, cls);
                     }
                 }

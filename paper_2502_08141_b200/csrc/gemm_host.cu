@@ -118,6 +118,8 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.status = status;
     G.s = s;
     G.rp = w.rp;
+    G.r = r;
+    G.lora_up = B;
     G.M = M;
     G.R = backward ? K : N;
     G.C = backward ? N : K;

@@ -53,6 +53,8 @@ struct GemmParams {
     uint32_t* status;
     float s;
     int rp;                 // LoRA rank rounded up to 64
+    int r;                  // LoRA rank
+    const uint16_t* lora_up;  // forward: B [r, N] (read by the dequant warps for the LoRA blocks)
     int M;                  // tokens
     int R;                  // A-operand rows in total: N (forward, dense) or K (backward)
     int C;                  // main contraction length: K (forward, dense) or N (backward)

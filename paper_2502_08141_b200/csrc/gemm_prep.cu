@@ -10,11 +10,13 @@ namespace lowra {
 namespace {
 
 // One warp per group of G rows (128 forward, 64 backward).  The rows are ordered by precision class
-// (1 bit, 2 bits, 4 bits, rows past N; stable) and cut into chunks of CH rows of one class (32 forward;
-// 16 backward, where every row is handled by two threads, one per 64-feature half), so that no warp of
-// the main kernel ever sees two precisions.  At most G / CH + 3 = 7 chunks exist and the kernel has 8
-// dequant warps: with n chunks, k = 8 / n warps share a chunk and take turns over the stages
-// (warp c + j * n serves chunk c at the stages whose index is congruent to j mod k).
+// (1 bit, 2 bits, 4 bits, rows past N; stable).
+//   forward : entry i of the group is the i-th row in that order = the row held by tensor-memory lane i of
+//             the main kernel, so that at most two precisions meet in a warp (32 consecutive lanes);
+//   backward: the ordered rows are cut into chunks of 16 rows of one class (every row is handled by two
+//             threads, one per 64-feature half), so that no warp ever sees two precisions.  At most
+//             64 / 16 + 3 = 7 chunks exist and the kernel has 8 dequant warps: with n chunks, k = 8 / n warps
+//             share a chunk and take turns (warp c + j * n serves chunk c in the groups congruent to j mod k).
 __device__ void deal_rows(const PrepParams& P, int blk) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int G = P.group, per = G / 32;
@@ -45,6 +47,10 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
         chunk_base[0] = 0;
 #pragma unroll
         for (int c = 1; c < 4; ++c) chunk_base[c] = chunk_base[c - 1] + (total[c - 1] + CH - 1) / CH;
+        int class_base[4];
+        class_base[0] = 0;
+#pragma unroll
+        for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total[c - 1];
         const int n_chunks = chunk_base[3] + (total[3] + CH - 1) / CH;
         const int k = 8 / n_chunks;
         if (lane == 0) P.n_chunks[grp] = (uint32_t)n_chunks;
@@ -59,13 +65,16 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
                         const int off = i * 32 + lane, row = grp * G + off;
                         const uint32_t p = (c < 3) ? (uint32_t)P.inv_perm[row] : 0u;
                         const uint32_t word = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
-                        for (int j = 0; j < k; ++j) {
-                            // backward: the group index is the stage index, so only the warp whose turn it
-                            // is gets the row; forward: all k warps get it and take turns over the stages
-                            if (CH == 16 && j != (grp & (k - 1))) continue;
+                        if (CH == 32) {
+                            // forward: position in precision order = tensor-memory lane of the row
+                            out[class_base[c] + q] = word;
+                        } else {
+                            // backward: the group index is the stage index; of the k warps that share the
+                            // chunk, the one whose turn it is gets the row (for both feature halves)
+                            const int j = grp & (k - 1);
                             const int thread = (chunk_base[c] + q / CH + j * n_chunks) * 32 + q % CH;
                             out[thread] = word;
-                            if (CH == 16) out[thread + 16] = word;
+                            out[thread + 16] = word;
                         }
                     }
                 }
