@@ -31,10 +31,15 @@ constexpr uint32_t kIdescAmn = kIdesc | (1u << 15);   // A operand MN-major
 // 32-column operand slot per pipeline stage behind it.
 constexpr uint32_t kTmemASlots = 256;
 
+// Forward keeps the weight operand in tensor memory, in a ring of its own that is deeper than the
+// shared-memory ring of the token operand, so the dequant warps can run further ahead of the tensor core.
+constexpr int kWSlots = 8;
+
 struct Barriers {
     uint64_t full_x[kStages];   // TMA bytes of a stage have landed
-    uint64_t full_w[kStages];   // dequant warps have written (or skipped) a stage
-    uint64_t empty[kStages];    // the MMAs reading a stage have completed
+    uint64_t full_w[kWSlots];   // dequant warps have written (or skipped) a stage (forward: 8 slots, else kStages)
+    uint64_t empty[kStages];    // the MMAs reading a shared-memory stage have completed
+    uint64_t empty_w[kWSlots];  // forward: the MMAs reading a tensor-memory weight slot have completed
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
@@ -195,17 +200,18 @@ __device__ __noinline__ void produce_block_tmem(Block blk, int cls, Levels lv, c
     ptx::tmem_st_wait();
 }
 
-// LoRA up-projection factor for the forward pass: row = output channel n, 64 ranks starting at j0, read
-// down a column of B [r, N] (the channels of a warp lie within one 128-wide window, so the 2-byte loads of
-// a warp share a few sectors).  Ranks >= r and channels >= N give zeros.
-__device__ __noinline__ void produce_lora_tmem(const uint16_t* B, int N, int r, int n, int j0, uint32_t taddr) {
+// LoRA up-projection factor for the forward pass: the tile [64 ranks][128 channels] lies in shared memory as
+// TMA delivered it from B [r, N] (per 64-channel half: one 128-byte row per rank, 128B swizzle); this lane
+// copies the column of its channel into its tensor-memory row (rank 2i in the low half of word i).
+__device__ __noinline__ void produce_lora_tmem(uint32_t tile_addr, int channel, uint32_t taddr) {
+    const uint32_t col = tile_addr + (uint32_t)(channel >> 6) * 8192u + (uint32_t)(channel & 7) * 2u;
+    const uint32_t chunk = (uint32_t)(channel & 63) >> 3;
     uint32_t o[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-        const int j = j0 + 2 * i;
-        uint32_t lo = 0u, hi = 0u;
-        if (n < N && j < r) lo = __ldg(B + (size_t)j * N + n);
-        if (n < N && j + 1 < r) hi = __ldg(B + (size_t)(j + 1) * N + n);
+        uint32_t lo, hi;   // ranks 2i and 2i + 1: rows 2i, 2i + 1 of the tile, chunk index swizzled by the row
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(col + (uint32_t)(2 * i) * 128u + ((chunk ^ (uint32_t)((2 * i) & 7)) << 4)));
+        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(col + (uint32_t)(2 * i + 1) * 128u + ((chunk ^ (uint32_t)((2 * i + 1) & 7)) << 4)));
         o[i] = lo | (hi << 16);
     }
     __syncwarp();
@@ -257,8 +263,11 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) {
             ptx::mbar_init(&bars->full_x[s], 1);
-            ptx::mbar_init(&bars->full_w[s], MODE == kModeForward ? kProducerWarps / 2 : kProducerWarps);
             ptx::mbar_init(&bars->empty[s], 1);
+        }
+        for (int s = 0; s < kWSlots; ++s) {
+            ptx::mbar_init(&bars->full_w[s], MODE == kModeForward ? kProducerWarps / 2 : kProducerWarps);
+            ptx::mbar_init(&bars->empty_w[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(&bars->tmem_full[a], 1);
@@ -320,10 +329,12 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             if (!ptx::flag_wait(P.flags + t.mt, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                             ptx::fence_proxy_async_all();
                         }
-                        if (MODE == kModeForward) {   // the up-projection rows are written to tensor memory by the dequant warps
-                            ptx::mbar_arrive_expect_tx(bar, kSmemB);
+                        ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
+                        if (MODE == kModeForward) {   // channels x ranks from B [r, N]: two 64-channel boxes; the dequant
+                                                      // warps move the rows into tensor memory in their own row order
+                            ptx::tma_load_2d(a_s, &tmFl, r0, lb * 64, bar);
+                            ptx::tma_load_2d(a_s + 8192, &tmFl, r0 + 64, lb * 64, bar);
                         } else {                      // features x ranks from A [K, r], K-major: one 64 x 128 box
-                            ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
                             ptx::tma_load_2d(a_s, &tmFl, lb * 64, r0, bar);
                         }
                         ptx::tma_load_2d(b_s, &tmT, lb * 64, m0, bar);
@@ -354,8 +365,10 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!ptx::mbar_wait(&bars->full_x[s], ph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                    const int sw = (MODE == kModeForward) ? (int)(it % kWSlots) : s;              // weight slot
+                    const uint32_t phw = (MODE == kModeForward) ? ((it / kWSlots) & 1u) : ph;
                     if (MODE != kModeDense)
-                        if (!ptx::mbar_wait(&bars->full_w[s], ph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                        if (!ptx::mbar_wait(&bars->full_w[sw], phw, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                     ptx::tc_fence_after();
                     const uint32_t a_addr = ptx::smem_u32(base + s * kSmemStage);
                     const uint64_t bdesc = ptx::umma_desc_k_sw128(a_addr + kSmemA);
@@ -366,7 +379,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     const bool a_mn = (MODE == kModeForward) ? t.is_t : (MODE == kModeBackward && !t.is_t && !lora_blk);
                     if (MODE == kModeForward && !t.is_t) {
                         // weights (and the LoRA up-projection rows) come from tensor memory: 8 columns per MMA
-                        const uint32_t a_tmem = tmem_base + kTmemASlots + 32u * (uint32_t)s;
+                        const uint32_t a_tmem = tmem_base + kTmemASlots + 32u * (uint32_t)sw;
 #pragma unroll
                         for (int kk = 0; kk < kTileC / 16; ++kk)
                             ptx::umma_bf16_ts(d_tmem, a_tmem + 8u * kk, bdesc + 2u * kk, kIdesc, (kb | kk) != 0 ? 1u : 0u);
@@ -383,6 +396,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             ptx::umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, kIdesc, (kb | kk) != 0 ? 1u : 0u);
                     }
                     ptx::umma_commit(&bars->empty[s]);
+                    if (MODE == kModeForward) ptx::umma_commit(&bars->empty_w[sw]);
                 }
                 if (failed) break;
                 ptx::umma_commit(&bars->tmem_full[acc]);
@@ -483,8 +497,10 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const int step = (MODE == kModeForward) ? 2 : 1;
                 for (int kb = first; kb < t.blocks; kb += step) {
                     const uint32_t it = it0 + (uint32_t)kb;
-                    const int s = it % kStages;
-                    if (!ptx::mbar_wait_warp(&bars->empty[s], ((it / kStages) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                    const int ring = (MODE == kModeForward) ? kWSlots : kStages;
+                    const int s = it % ring;
+                    uint64_t* eb = (MODE == kModeForward) ? &bars->empty_w[s] : &bars->empty[s];
+                    if (!ptx::mbar_wait_warp(eb, ((it / ring) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         failed = true; bars->abort = 1u; break;
                     }
                     if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
@@ -533,9 +549,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         const int kb = kb0 + 2 * u;
                         if (kb >= t.blocks) break;
                         const uint32_t it = it0 + (uint32_t)kb;
-                        const int s = it % kStages;
-                        const uint32_t ph = (it / kStages) & 1u;
-                        if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
+                        const int s = it % kWSlots;
+                        const uint32_t ph = (it / kWSlots) & 1u;
+                        if (!ptx::mbar_wait_warp(&bars->empty_w[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
                             failed = true; bars->abort = 1u; break;
                         }
                         ptx::tc_fence_after();
@@ -543,7 +559,18 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         if (kb < P.main_blocks) {
                             produce_block_tmem(ring[u], cls, lv, mrow, slut_addr, taddr);
                         } else {
-                            produce_lora_tmem(P.lora_up, P.L.N, P.r, r0 + row_local, (kb - P.main_blocks) * 64, taddr);
+                            // LoRA block: the factor tile (channels x 64 ranks, natural channel order) has been
+                            // fetched by TMA into the stage's weight region; copy this lane's channel row
+                            // (the weight ring is deeper than the shared-memory ring: first make sure the tensor
+                            // core is done with the previous use of this shared-memory stage, so that the parity
+                            // of the "landed" barrier below cannot be mistaken for an older phase)
+                            const int sx = it % kStages;
+                            const uint32_t phx = (it / kStages) & 1u;
+                            if (!ptx::mbar_wait_warp(&bars->empty[sx], phx ^ 1u, abort_flag, kWaitLimitNs) ||
+                                !ptx::mbar_wait_warp(&bars->full_x[sx], phx, abort_flag, kWaitLimitNs)) {
+                                failed = true; bars->abort = 1u; break;
+                            }
+                            produce_lora_tmem(ptx::smem_u32(base + sx * kSmemStage), row_local, taddr);
                         }
                         ptx::tc_fence_before();
                         __syncwarp();

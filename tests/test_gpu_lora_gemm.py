@@ -84,22 +84,29 @@ def test_forward_and_backward_input(lw, N, K, M, r, mix, kind):
     assert emax <= MAX_TOL and efro <= FRO_TOL, ("backward", emax, efro)
 
 
-def test_lora_term_is_really_there(lw):
-    """With large LoRA factors the low-rank term dominates: a path that dropped it, or applied the
-    wrong scale, would fail by far."""
-    N, K, M, r = 256, 256, 128, 64
-    case = make_case(N, K, {1: 0.5, 2: 0.5}, matrix_id=5)
+@pytest.mark.parametrize("N,K,M,r", [(256, 256, 128, 64), (640, 1152, 515, 96), (128, 1152, 256, 128),
+                                     (1024, 2048, 700, 64)])
+def test_lora_term_is_really_there(lw, N, K, M, r):
+    """With large LoRA factors the low-rank term dominates: a path that dropped it, applied the wrong
+    scale, or picked up a stale operand tile (long contractions, several LoRA blocks, several tiles per
+    CTA) would fail by far.  Both directions."""
+    case = make_case(N, K, {1: 0.5, 2: 0.3, 4: 0.2}, matrix_id=5)
     layout = lw.Layout(case.precs, K)
     X = si.activations(M, K, matrix_id=9)
+    dY = si.out_grads(M, N, matrix_id=9)
     A = si.bf16_normal((K, r), 0.5, stream=50)
     B = si.bf16_normal((r, N), 0.5, stream=51)
     packed, absmax, maps = _dev(case.packed), _dev(case.absmax), _dev(case.maps)
     for s in (0.0, 0.25, -3.0):
         Y = lw.lowra_lora_forward(layout, packed, absmax, maps, _bf(X), _bf(A), _bf(B), s)
+        dX = lw.lowra_lora_backward_input(layout, packed, absmax, maps, _bf(dY), _bf(A), _bf(B), s)
         torch.cuda.synchronize()
         ref = oracle.lora_forward(case.W_hat, X, A, B, s)
         emax, efro = gemm_errors(si.bf16_bits_to_f32(_bits(Y)), ref)
-        assert emax <= MAX_TOL and efro <= FRO_TOL, (s, emax, efro)
+        assert emax <= MAX_TOL and efro <= FRO_TOL, ("forward", s, emax, efro)
+        ref = oracle.lora_backward_input(case.W_hat, dY, A, B, s)
+        emax, efro = gemm_errors(si.bf16_bits_to_f32(_bits(dX)), ref)
+        assert emax <= MAX_TOL and efro <= FRO_TOL, ("backward", s, emax, efro)
 
 
 def test_fused_weights_equal_decoded_weights(lw):
