@@ -96,7 +96,7 @@ lowra_status lowra_encode(const lowra_layout* layout, const float* W_dev, const 
 /*
  * Dequantize (Appendix A.2): unpack each row's 1/2/4-bit codes, look them up in the row's mapping
  * table, multiply by the block's absmax in fp32 and round to bf16 (nearest even).
- *   W_bf16_dev     bf16 bit patterns [N, K] row-major, original row order   (out)
+ *   W_bf16_dev     bf16 bit patterns [N, K] row-major, original row order, 32-byte aligned   (out)
  */
 lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* packed_dev, const float* absmax_dev,
                           const float* maps_dev, uint16_t* W_bf16_dev, void* stream);

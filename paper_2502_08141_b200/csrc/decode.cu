@@ -1,9 +1,18 @@
 // lowra_decode: packed 1/2/4-bit codes -> bf16 weights (paper Appendix A.2).
 //
-// HBM-bound: 2 bytes written per element against b/8 + 1/16 bytes read.  One warp handles one
-// 512-byte piece of one stored row: every lane fetches 16 packed bytes with a single 128-bit load,
-// the row's mapping table is staged in shared memory, and the codes are redistributed with warp
-// shuffles so that every store instruction of the warp writes 512 contiguous bytes of the output.
+// HBM-bound: 2 bytes written per element against b/8 + 1/16 bytes read, so the kernel must spend very few
+// instructions per element and every store instruction must fill whole 128-byte lines.
+// One warp handles one 512-byte piece of one stored row.  Every lane fetches 16 packed bytes with a single
+// 128-bit load; the piece and its absmax values are parked in the warp's slice of shared memory, and the warp
+// then walks over the piece 512 elements at a time: lane l expands elements 16 l .. 16 l + 15 (four lanes
+// per 64-element absmax block) and writes them with one 32-byte vector store, so a store instruction of
+// the warp writes 1 KB of contiguous output.
+//   1 bit : the two levels are scaled by the block's absmax and rounded to bf16 once; a pair of elements is
+//           then one multiply-add (min + bit * |H - L| in both 16-bit halves);
+//   2 bits: the four scaled levels sit in two registers, a pair of elements is one byte permute;
+//   4 bits: the row's 16 fp32 levels are staged in shared memory; per element one load, one multiply,
+//           half a convert.
+// Results are bit-identical to table[code] * absmax rounded to bf16 (round to nearest even).
 #include "lowra_common.cuh"
 
 namespace lowra {
@@ -21,71 +30,93 @@ struct DecodeParams {
     uint32_t task_start[4];      // first task of each class; [3] = number of tasks
 };
 
-// One 512-byte piece of a B-bit row: 4096 / B elements, written as 16 / B warp-wide stores.
+__device__ __forceinline__ void st_stream_v8(void* p, const uint32_t (&v)[8]) {
+    asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]),
+                 "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+
+struct WarpStage {
+    uint4 packed[32];    // the 512-byte piece
+    float absmax[64];    // absmax of the piece's blocks (64 at 1 bit, 32 at 2 bits, 16 at 4 bits)
+    float lut[16];       // 4-bit rows: the row's levels
+};
+
 template <int B>
-__device__ __forceinline__ void decode_piece(const DecodeParams& P, int p, int piece, int lane, float* lut) {
-    constexpr int c = B >> 1;         // class index of B bits
-    constexpr int kElems = 4096 / B;  // elements in the piece
-    constexpr int kIters = 16 / B;    // 256 elements (512 output bytes) per iteration
-    constexpr int kUnits = 16 / B;    // 8-element units held by one lane's 16 bytes
-    constexpr uint32_t kMask = (1u << B) - 1u;
+__device__ __forceinline__ void decode_piece(const DecodeParams& P, int p, int piece, int lane, WarpStage* ws) {
+    constexpr int c = B >> 1;              // class index of B bits
+    constexpr int kElemsPiece = 4096 / B;  // elements in a full piece
+    constexpr int kIters = 8 / B;          // 512 elements per iteration
+    constexpr int kBlocks = kElemsPiece / kBlock;
     const int K = P.L.K;
     const int r = __ldg(P.L.perm + p);
     const size_t row_bytes = (size_t)K * B / 8;
     const uint8_t* row = P.packed + P.L.seg_off[c] + (size_t)(p - P.L.class_start[c]) * row_bytes;
-
     const size_t byte0 = (size_t)piece * 512 + (size_t)lane * 16;
-    uint4 q = make_uint4(0u, 0u, 0u, 0u);
-    if (byte0 < row_bytes) q = ld_stream_v4(row + byte0);
+    const int e0 = piece * kElemsPiece;                         // first element of the piece
+    const float* arow = P.absmax + (size_t)p * P.L.nb + e0 / kBlock;
+    const int blocks_left = P.L.nb - e0 / kBlock;               // blocks of the row from e0 on
+    const float* mrow = P.maps + (size_t)r * kTableStride;
 
-    if (lane < (1 << B)) lut[lane] = __ldg(P.maps + (size_t)r * kTableStride + lane);
-
-    const int e0 = piece * kElems;  // first element of the piece
-    const int blk0 = e0 / kBlock;
-    const float* arow = P.absmax + (size_t)p * P.L.nb;
-    float av0 = (blk0 + lane < P.L.nb) ? __ldg(arow + blk0 + lane) : 0.0f;
-    float av1 = 0.0f;
-    if (B == 1 && blk0 + 32 + lane < P.L.nb) av1 = __ldg(arow + blk0 + 32 + lane);
+    // stage the piece
+    ws->packed[lane] = (byte0 < row_bytes) ? ld_stream_v4(row + byte0) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+    for (int i = 0; i < kBlocks; i += 32)
+        if (i + lane < kBlocks) ws->absmax[i + lane] = (i + lane < blocks_left) ? __ldg(arow + i + lane) : 0.0f;
+    float m0 = 0.f, m1 = 0.f, m2 = 0.f, m3 = 0.f;
+    if (B == 4) {
+        if (lane < 16) ws->lut[lane] = __ldg(mrow + lane);
+    } else {
+        m0 = __ldg(mrow); m1 = __ldg(mrow + 1);
+        if (B == 2) { m2 = __ldg(mrow + 2); m3 = __ldg(mrow + 3); }
+    }
     __syncwarp();
 
-    uint16_t* orow = P.out + (size_t)r * K;
+    uint16_t* dst = P.out + (size_t)r * K + e0 + lane * 16;
+    const unsigned char* bytes = reinterpret_cast<const unsigned char*>(ws->packed);
 #pragma unroll
     for (int j = 0; j < kIters; ++j) {
-        // This lane writes elements e0 + 256 j + 8 lane .. +8, i.e. 8-element unit u = 32 j + lane
-        // of the piece; that unit sits in lane u / kUnits, 32-bit word (u % kUnits) * B / 4.
-        const int u = 32 * j + lane;
-        const int src = u / kUnits;
-        const int sub = u % kUnits;
-        const int w = (sub * B) >> 2;
-        const uint32_t x0 = __shfl_sync(0xffffffffu, q.x, src);
-        const uint32_t x1 = __shfl_sync(0xffffffffu, q.y, src);
-        const uint32_t x2 = __shfl_sync(0xffffffffu, q.z, src);
-        const uint32_t x3 = __shfl_sync(0xffffffffu, q.w, src);
-        const uint32_t word = (w == 0) ? x0 : (w == 1) ? x1 : (w == 2) ? x2 : x3;
-        const uint32_t bits = word >> ((sub * 8 * B) & 31);
-        // 256 elements = 4 absmax blocks per iteration, 8 lanes per block
-        const int blk = 4 * j + (lane >> 3);
-        const float a = __shfl_sync(0xffffffffu, (B == 1 && j >= 8) ? av1 : av0, blk & 31);
-        uint32_t o[4];
+        // lane l: elements e0 + 512 j + 16 l .. + 15, i.e. bits [(512 j + 16 l) B, + 16 B) of the piece
+        const int e = e0 + 512 * j + 16 * lane;
+        const float a = ws->absmax[8 * j + (lane >> 2)];
+        uint32_t o[8];
+        if (B == 1) {
+            const uint32_t h = *reinterpret_cast<const uint16_t*>(bytes + 64 * j + 2 * lane);
+            const uint32_t LH = pack_bf16x2(__fmul_rn(m0, a), __fmul_rn(m1, a));
+            const uint32_t L = LH & 0xFFFFu, H = LH >> 16;
+            const uint32_t lo = min(L, H);
+            const uint32_t BB = lo * 0x10001u, d = max(L, H) - lo, f = (L > H) ? 0x10001u : 0u;
+            const uint32_t z = h | (h << 15);   // pair i at bits 0 and 16 of z >> 2i
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const uint32_t c0 = (bits >> (2 * i * B)) & kMask;
-            const uint32_t c1 = (bits >> ((2 * i + 1) * B)) & kMask;
-            const float f0 = __fmul_rn(lut[c0], a);
-            const float f1 = __fmul_rn(lut[c1], a);
-            o[i] = pack_bf16x2(f0, f1);
+            for (int i = 0; i < 8; ++i) o[i] = (((z >> (2 * i)) & 0x10001u) ^ f) * d + BB;
+        } else if (B == 2) {
+            const uint32_t w = *reinterpret_cast<const uint32_t*>(bytes + 128 * j + 4 * lane);
+            const uint32_t E01 = pack_bf16x2(__fmul_rn(m0, a), __fmul_rn(m1, a));
+            const uint32_t E23 = pack_bf16x2(__fmul_rn(m2, a), __fmul_rn(m3, a));
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t y = w >> (4 * i);
+                const uint32_t t = (y & 3u) | ((y << 6) & 0x300u);
+                o[i] = __byte_perm(E01, E23, t * 0x22u + 0x1010u);
+            }
+        } else {
+            const uint2 w = *reinterpret_cast<const uint2*>(bytes + 256 * j + 8 * lane);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint32_t x = ((i < 4) ? w.x : w.y) >> (8 * (i & 3));
+                o[i] = pack_bf16x2(__fmul_rn(ws->lut[x & 15u], a), __fmul_rn(ws->lut[(x >> 4) & 15u], a));
+            }
         }
-        const int e = e0 + 256 * j + 8 * lane;
-        if (e < K) st_stream_v4(orow + e, make_uint4(o[0], o[1], o[2], o[3]));
+        if (e < K) st_stream_v8(dst + 512 * j, o);
     }
-    __syncwarp();  // the table slot is reused by the warp's next piece
+    __syncwarp();  // the stage is reused by the warp's next piece
 }
 
 __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const DecodeParams P) {
-    __shared__ float lut_all[kDecodeWarps][kTableStride];
+    __shared__ __align__(16) WarpStage stage_all[kDecodeWarps];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
-    float* lut = lut_all[warp];
+    WarpStage* ws = &stage_all[warp];
     const uint32_t n_tasks = P.task_start[3];
     const uint32_t stride = gridDim.x * kDecodeWarps;
     for (uint32_t t = blockIdx.x * kDecodeWarps + warp; t < n_tasks; t += stride) {
@@ -95,9 +126,9 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const DecodePara
         const int q = local / ppr;
         const int piece = local - q * ppr;
         const int p = P.L.class_start[c] + q;
-        if (c == 0) decode_piece<1>(P, p, piece, lane, lut);
-        else if (c == 1) decode_piece<2>(P, p, piece, lane, lut);
-        else decode_piece<4>(P, p, piece, lane, lut);
+        if (c == 0) decode_piece<1>(P, p, piece, lane, ws);
+        else if (c == 1) decode_piece<2>(P, p, piece, lane, ws);
+        else decode_piece<4>(P, p, piece, lane, ws);
     }
 }
 
@@ -110,7 +141,8 @@ extern "C" lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* 
     lowra_status st = check_layout(layout);
     if (st != LOWRA_OK) return st;
     if (!packed_dev || !absmax_dev || !maps_dev || !W_bf16_dev) return LOWRA_ERR_NULL;
-    if (!aligned16(packed_dev) || !aligned16(absmax_dev) || !aligned16(maps_dev) || !aligned16(W_bf16_dev))
+    if (!aligned16(packed_dev) || !aligned16(absmax_dev) || !aligned16(maps_dev) ||
+        (reinterpret_cast<uintptr_t>(W_bf16_dev) & 31u) != 0)
         return LOWRA_ERR_ALIGN;
     st = check_device();
     if (st != LOWRA_OK) return st;

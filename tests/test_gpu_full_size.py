@@ -1,0 +1,75 @@
+"""Parity at benchmark sizes, in the launch configuration that bench.py times (4096 tokens, rank 64).
+
+Encode and decode are compared bit for bit on the whole matrix.  The two products are computed in full
+on the GPU and compared with the fp64 oracle on 128 sampled token rows (always rows 0, 127, 128 and
+M - 1, the rest seeded): the oracle evaluates exactly those rows, all N (resp. K) outputs of each.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from helpers import FRO_TOL, MAX_TOL, gemm_errors, make_case
+
+pytestmark = pytest.mark.gpu
+
+CASES = [
+    # name, N, K, mix, matrix id  -- shapes of configs 3 and 4
+    ("gate_proj-7b", 11008, 4096, {1: 0.60, 2: 0.35, 4: 0.05}, 4),
+    ("down_proj-7b", 4096, 11008, {1: 0.60, 2: 0.35, 4: 0.05}, 6),
+    ("q_proj-13b", 5120, 5120, {1: 0.85, 2: 0.15}, 0),
+]
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _bf(bits):
+    return _dev(bits.view(np.int16)).view(torch.bfloat16)
+
+
+def _bits(t):
+    return t.view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+@pytest.mark.parametrize("name,N,K,mix,mid", CASES)
+def test_full_size_matrix(name, N, K, mix, mid):
+    import paper_2502_08141_b200 as lw
+
+    M, r, s = 4096, 64, 2.0
+    case = make_case(N, K, mix, matrix_id=mid)
+    layout = lw.Layout(case.precs, K)
+
+    packed, absmax = lw.lowra_encode(layout, _dev(case.W), _dev(case.thr))
+    what = lw.lowra_decode(layout, packed, absmax, _dev(case.maps))
+    torch.cuda.synchronize()
+    assert np.array_equal(packed.cpu().numpy()[:layout.packed_bytes], case.packed)
+    assert np.array_equal(absmax.cpu().numpy().view(np.uint32), case.absmax.view(np.uint32))
+    assert np.array_equal(_bits(what), case.W_hat)
+    del what
+
+    X = si.activations(M, K, matrix_id=300 + mid)
+    dY = si.out_grads(M, N, matrix_id=300 + mid)
+    A, B = si.lora_factors(K, N, r, matrix_id=mid)
+    rng = np.random.default_rng(mid)
+    rows = np.unique(np.concatenate([[0, 127, 128, M - 1], rng.choice(M, 124, replace=False)]))
+    ws = torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")
+
+    Y = lw.lowra_lora_forward(layout, packed, absmax, _dev(case.maps), _bf(X), _bf(A), _bf(B), s, workspace=ws)
+    assert lw.lowra_device_status(ws) == lw.LOWRA_OK
+    got = si.bf16_bits_to_f32(_bits(Y[torch.from_numpy(rows).cuda()]))
+    ref = oracle.lora_forward(case.W_hat, X[rows], A, B, s)
+    emax, efro = gemm_errors(got, ref)
+    assert emax <= MAX_TOL and efro <= FRO_TOL, ("forward", name, emax, efro)
+    assert torch.isfinite(Y.float()).all()
+    del Y
+
+    dX = lw.lowra_lora_backward_input(layout, packed, absmax, _dev(case.maps), _bf(dY), _bf(A), _bf(B), s, workspace=ws)
+    assert lw.lowra_device_status(ws) == lw.LOWRA_OK
+    got = si.bf16_bits_to_f32(_bits(dX[torch.from_numpy(rows).cuda()]))
+    ref = oracle.lora_backward_input(case.W_hat, dY[rows], A, B, s)
+    emax, efro = gemm_errors(got, ref)
+    assert emax <= MAX_TOL and efro <= FRO_TOL, ("backward", name, emax, efro)
+    assert torch.isfinite(dX.float()).all()
