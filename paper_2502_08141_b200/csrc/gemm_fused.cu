@@ -34,6 +34,7 @@ constexpr uint32_t kTmemASlots = 256;
 // Forward keeps the weight operand in tensor memory, in a ring of its own that is deeper than the
 // shared-memory ring of the token operand, so the dequant warps can run further ahead of the tensor core.
 constexpr int kWSlots = 8;
+constexpr int kTurns = kProducerWarps / 4;   // forward: warps that share a tensor-memory lane quarter and take turns
 
 struct Barriers {
     uint64_t full_x[kStages];   // TMA bytes of a stage have landed
@@ -149,7 +150,6 @@ __device__ __forceinline__ void store_row(uint32_t row_addr, int swz, const uint
         ptx::st_shared_v4(row_addr + (uint32_t)((t ^ swz) << 4), make_uint4(o[4 * t], o[4 * t + 1], o[4 * t + 2], o[4 * t + 3]));
 }
 
-// Deliberately not inlined: the hot code of the dequant warps must stay small.
 __device__ __noinline__ void dequant_block_1bit(uint32_t w0, uint32_t w1, float m0, float m1, float a,
                                                 uint32_t row_addr, int swz) {
     uint32_t o[32];
@@ -266,7 +266,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             ptx::mbar_init(&bars->empty[s], 1);
         }
         for (int s = 0; s < kWSlots; ++s) {
-            ptx::mbar_init(&bars->full_w[s], MODE == kModeForward ? kProducerWarps / 2 : kProducerWarps);
+            ptx::mbar_init(&bars->full_w[s], MODE == kModeForward ? 4 : kProducerWarps);
             ptx::mbar_init(&bars->empty_w[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -426,7 +426,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             // forward weight tiles hold their rows in precision order: this lane's accumulator row belongs to
             // the channel that the deal put at this position
             int my_row = q * 32 + lane;
-            if (MODE == kModeForward && !t.is_t) my_row = info_row(__ldg(P.items + (size_t)t.rt * 256 + q * 32 + lane));
+            if (MODE == kModeForward && !t.is_t) my_row = info_row(__ldg(P.items + (size_t)t.rt * kItemStride + q * 32 + lane));
             // the four epilogue warps share named barriers, so they must agree on leaving
             if (!ptx::mbar_wait_warp(&bars->tmem_full[acc], aph, abort_flag, kWaitLimitNs)) bars->abort = 1u;
             ptx::named_barrier_sync(1, 128);
@@ -493,8 +493,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             const int r0 = t.rt * kTileR;
             if (t.is_t) {
                 // nothing to dequantise: keep the stage barriers in step (forward: the warps whose turn it is)
-                const int first = (MODE == kModeForward) ? ((pt >> 7) & 1) : 0;
-                const int step = (MODE == kModeForward) ? 2 : 1;
+                const int first = (MODE == kModeForward) ? (pt >> 7) : 0;
+                const int step = (MODE == kModeForward) ? kTurns : 1;
                 for (int kb = first; kb < t.blocks; kb += step) {
                     const uint32_t it = it0 + (uint32_t)kb;
                     const int ring = (MODE == kModeForward) ? kWSlots : kStages;
@@ -511,8 +511,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // at most two precisions meet in a warp); 64 input features per stage, written with tcgen05.st
                 // into the stage's 32-column operand slot.  The two warps that own a lane quarter take turns.
                 const int q = warp & 3;                              // lane quarter this warp may touch
-                const int turn = (pt >> 7) & 1;                      // this warp serves the blocks kb with kb % 2 == turn
-                const uint32_t item = __ldg(P.items + (size_t)t.rt * 256 + q * 32 + lane);
+                const int turn = pt >> 7;                            // this warp serves the blocks kb with kb % kTurns == turn
+                const uint32_t item = __ldg(P.items + (size_t)t.rt * kItemStride + q * 32 + lane);
                 const int cls = info_class(item);
                 const int row_local = info_row(item);
                 const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + kTmemASlots;
@@ -539,14 +539,14 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 ring[0].a = ring[1].a = 0.0f;
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {   // ring slot u serves this warp's turns number u, u + 2, ...
-                    const int mb = turn + 2 * u;
+                    const int mb = turn + kTurns * u;
                     if (cls < 3 && mb < P.main_blocks)
                         load_block(ring[u], bits_ptr + (size_t)mb * bits_stride, absmax_ptr + mb, cls);
                 }
-                for (int kb0 = turn; kb0 < t.blocks && !failed; kb0 += 4) {
+                for (int kb0 = turn; kb0 < t.blocks && !failed; kb0 += 2 * kTurns) {
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const int kb = kb0 + 2 * u;
+                        const int kb = kb0 + kTurns * u;
                         if (kb >= t.blocks) break;
                         const uint32_t it = it0 + (uint32_t)kb;
                         const int s = it % kWSlots;
@@ -575,7 +575,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         ptx::tc_fence_before();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
-                        const int nb = kb + 4;   // this ring slot's next turn
+                        const int nb = kb + 2 * kTurns;   // this ring slot's next turn
                         if (cls < 3 && nb < P.main_blocks)
                             load_block(ring[u], bits_ptr + (size_t)nb * bits_stride, absmax_ptr + nb, cls);
                     }
@@ -634,10 +634,10 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     if (u < P.main_blocks) {
-                        cur_info[u] = __ldg(items + (size_t)u * 256);
+                        cur_info[u] = __ldg(items + (size_t)u * kItemStride);
                         fetch(ring[u], lvr[u], cur_info[u], u);
                     }
-                    info_ring[u] = (u + 2 < P.main_blocks) ? __ldg(items + (size_t)(u + 2) * 256) : kIdleItem;
+                    info_ring[u] = (u + 2 < P.main_blocks) ? __ldg(items + (size_t)(u + 2) * kItemStride) : kIdleItem;
                 }
                 if (P.main_blocks > 0) fetch_table(cur_info[0], 0);
                 for (int kb0 = 0; kb0 < t.blocks && !failed; kb0 += 2) {
@@ -673,7 +673,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         const int nb = mb + 2;
                         cur_info[u] = info_ring[u];
                         if (nb < P.main_blocks) fetch(ring[u], lvr[u], cur_info[u], nb);
-                        info_ring[u] = (nb + 2 < P.main_blocks) ? __ldg(items + (size_t)(nb + 2) * 256) : kIdleItem;
+                        info_ring[u] = (nb + 2 < P.main_blocks) ? __ldg(items + (size_t)(nb + 2) * kItemStride) : kIdleItem;
                         if (mb + 1 < P.main_blocks) fetch_table(cur_info[u ^ 1], mb + 1);
                     }
                 }

@@ -30,7 +30,7 @@ Workspace plan_workspace(int N, int K, int M, int r) {
     w.off_T = kStatusBytes;
     w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);
     w.off_items = w.off_flags + align256((size_t)((M + kTileT - 1) / kTileT) * 4);
-    w.off_meta = w.off_items + align256(groups * 256 * 4);
+    w.off_meta = w.off_items + align256(groups * kItemStride * 4);
     w.total = w.off_meta + align256(groups * 4);
     return w;
 }

@@ -9,14 +9,16 @@ namespace lowra {
 
 // ---- prologue ------------------------------------------------------------------------------
 constexpr int kPrepThreads = 128;
+constexpr int kProducerWarps = 12;            // dequant warps of the main kernel: three per tensor-memory lane quarter
+constexpr int kItemStride = 512;              // entries per row group in the deal table (>= 32 * kProducerWarps)
 
 struct PrepParams {
     // deal of the rows of every group (128 rows forward, 64 backward) to the 256 dequant threads of the
-    // main kernel, one precision per warp: items[g * 256 + thread] = row offset (bits 0-6) | class
+    // main kernel, one precision per warp: items[g * kItemStride + thread] = row offset (bits 0-6) | class
     // (bits 7-8, 3 = row past N) | stored position (bits 9-31), or all ones for "no row"
     const uint8_t* precs;
     const int32_t* inv_perm;
-    uint32_t* items;      // [ceil(N / group) * 256]
+    uint32_t* items;      // [ceil(N / group) * kItemStride]
     uint32_t* n_chunks;   // [ceil(N / group)] number of chunks the group was cut into (1..7)
     int N, group;
     uint32_t* status;     // device status word, cleared
@@ -32,7 +34,6 @@ constexpr int kTileR = 128;       // rows of the MMA A operand per tile (output 
 constexpr int kTileT = 256;       // tokens per tile (MMA N)
 constexpr int kTileC = 64;        // contraction elements per pipeline stage (= one absmax block, = 128 bytes of bf16)
 constexpr int kStages = 4;
-constexpr int kProducerWarps = 8;
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstProducerWarp = 6;
 constexpr int kGemmThreads = 32 * (kFirstProducerWarp + kProducerWarps);
@@ -45,7 +46,7 @@ struct GemmParams {
     const uint8_t* packed;
     const float* absmax;
     const float* maps;
-    const uint32_t* items;    // from the prologue: [row groups][256 dequant threads]
+    const uint32_t* items;    // from the prologue: [row groups][kItemStride]
     const uint32_t* n_chunks; // from the prologue: [row groups]
     uint16_t* out;          // [M, ld_out] bf16
     uint16_t* T;            // [M, rp] bf16: s * X . A (forward) or s * dY . B^T (backward), written by the T tiles

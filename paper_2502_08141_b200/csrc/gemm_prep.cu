@@ -15,7 +15,7 @@ namespace {
 //             the main kernel, so that at most two precisions meet in a warp (32 consecutive lanes);
 //   backward: the ordered rows are cut into chunks of 16 rows of one class (every row is handled by two
 //             threads, one per 64-feature half), so that no warp ever sees two precisions.  At most
-//             64 / 16 + 3 = 7 chunks exist and the kernel has 8 dequant warps: with n chunks, k = 8 / n warps
+//             64 / 16 + 3 = 7 chunks exist and the kernel has 12 dequant warps: with n chunks, k = 12 / n warps
 //             share a chunk and take turns (warp c + j * n serves chunk c in the groups congruent to j mod k).
 __device__ void deal_rows(const PrepParams& P, int blk) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -23,9 +23,9 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
     const int CH = (G == 128) ? 32 : 16;
     const int n_groups = (P.N + G - 1) / G;
     for (int grp = blk * (kPrepThreads / 32) + warp; grp < n_groups; grp += P.blocks * (kPrepThreads / 32)) {
-        uint32_t* out = P.items + (size_t)grp * 256;
+        uint32_t* out = P.items + (size_t)grp * kItemStride;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) out[i * 32 + lane] = 0xFFFFFFFFu;
+        for (int i = 0; i < kItemStride / 32; ++i) out[i * 32 + lane] = 0xFFFFFFFFu;
         __syncwarp();
         int cls[4];
         unsigned mask[4][4];
@@ -52,7 +52,7 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
 #pragma unroll
         for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total[c - 1];
         const int n_chunks = chunk_base[3] + (total[3] + CH - 1) / CH;
-        const int k = 8 / n_chunks;
+        const int k = kProducerWarps / n_chunks;   // warps that share a chunk (backward)
         if (lane == 0) P.n_chunks[grp] = (uint32_t)n_chunks;
         int before[4] = {0, 0, 0, 0};
 #pragma unroll
@@ -70,9 +70,27 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
                             out[class_base[c] + q] = word;
                         } else {
                             // backward: the group index is the stage index; of the k warps that share the
-                            // chunk, the one whose turn it is gets the row (for both feature halves)
-                            const int j = grp & (k - 1);
-                            const int thread = (chunk_base[c] + q / CH + j * n_chunks) * 32 + q % CH;
+                            // chunk, the one whose turn it is gets the row (for both feature halves).
+                            // Inside the class the rows are taken round-robin over (row offset mod 8), so that
+                            // eight neighbouring lanes hold eight different residues: their 16-byte stores into
+                            // the swizzled operand tile then fall into eight different bank groups.
+                            const unsigned res_mask = 0x01010101u << (lane & 7);
+                            int b = 0;   // rank of this row among the rows of its class with the same residue
+#pragma unroll
+                            for (int i2 = 0; i2 < 4; ++i2)
+                                if (i2 < i) b += __popc(mask[i2][c] & res_mask);
+                            b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
+                            int pos = 0;  // rows taken before this one
+#pragma unroll
+                            for (int res = 0; res < 8; ++res) {
+                                int cnt = 0;
+#pragma unroll
+                                for (int i2 = 0; i2 < 4; ++i2)
+                                    if (i2 < per) cnt += __popc(mask[i2][c] & (0x01010101u << res));
+                                pos += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
+                            }
+                            const int j = grp % k;
+                            const int thread = (chunk_base[c] + pos / CH + j * n_chunks) * 32 + pos % CH;
                             out[thread] = word;
                             out[thread + 16] = word;
                         }
