@@ -159,6 +159,24 @@ def make_host_inputs(cfg, rank: int):
     return mats, acts
 
 
+# DRAM traffic of one fused_kernel launch measured with ncu on the small profiling case (N = K = 4096,
+# 2048 tokens, rank 64, 1.5 bits on average): forward 22.35 MB, backward-input 22.40 MB, almost all of it reads
+# (the bf16 output is still in L2 when the kernel ends).  That equals the case's input bytes (activations +
+# packed codes + absmax + tables + LoRA factors = 22.1 MB), so traffic is scaled in proportion to input bytes.
+NCU_CASE = dict(N=4096, K=4096, M=2048, r=64, bits=1.5, dram_bytes=0.5 * (22.35e6 + 22.40e6))
+
+
+def fused_input_bytes(N, K, M, r, bits):
+    return 2.0 * M * K + N * K * (bits / 8 + 4 / 64) + 64.0 * N + 2.0 * (K + N) * r
+
+
+def fused_traffic_per_launch(dev, M, r, bits):
+    case = fused_input_bytes(NCU_CASE["N"], NCU_CASE["K"], NCU_CASE["M"], NCU_CASE["r"], NCU_CASE["bits"])
+    per = [fused_input_bytes(d["m"]["N"], d["m"]["K"], M, r, bits) for d in dev] + \
+          [fused_input_bytes(d["m"]["K"], d["m"]["N"], M, r, bits) for d in dev]   # backward reads dY [M, N]
+    return NCU_CASE["dram_bytes"] / case * sum(per) / len(per)
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
@@ -283,7 +301,10 @@ def run_gpu(args):
                 "achieved": achieved, "peak": P["tensor_sustained"], "unit": "TFLOP/s",
                 "frac": achieved / P["tensor_sustained"], "peak_burst": P["tensor_burst"],
                 "frac_burst": achieved / P["tensor_burst"], "peak_source": P["source"] + " (sustained: timed inside a long step)",
-                "traffic": None}
+                "traffic": fused_traffic_per_launch(dev, M, r, bits),
+                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one fused_kernel launch at "
+                                  "N=K=4096, 2048 tokens (profiles/fused_*_4096x4096_m2048.md), scaled by the input "
+                                  "bytes of an average launch of this workload"}
 
     # ---- end to end: host buffers, pinned, copies inside the timed region
     e2e = None

@@ -1,0 +1,56 @@
+"""Small, self-contained launches of one kernel family, sized for an `ncu --set full` capture.
+
+    python -m paper_2502_08141_b200.profile_case forward     # fused forward,  N = K = 4096, 2048 tokens, rank 64
+    python -m paper_2502_08141_b200.profile_case backward    # fused backward-input, same shapes
+    python -m paper_2502_08141_b200.profile_case codec       # decode + encode of an 11008 x 4096 matrix
+
+Each case runs its call three times on seeded synthetic inputs (config-3 precision mix) and checks the
+device status word; a few hundred MB on the device at most.
+"""
+from __future__ import annotations
+
+import sys
+
+import torch
+
+import synth_inputs as si
+
+from . import (Layout, lowra_decode, lowra_device_status, lowra_encode, lowra_lora_backward_input,
+               lowra_lora_forward, lowra_workspace_bytes)
+
+
+def main(case: str) -> None:
+    cfg = si.config(3)
+    N, K = (11008, 4096) if case == "codec" else (4096, 4096)
+    M, r, s = 2048, cfg.rank, cfg.s
+    precs = si.precisions(N, cfg.mix)
+    maps, thr = si.standin_codebooks(precs)
+    layout = Layout(precs, K)
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    W = torch.randn(N, K, device="cuda", generator=gen) * 0.02
+    maps_d, thr_d = torch.from_numpy(maps).cuda(), torch.from_numpy(thr).cuda()
+    packed, absmax = lowra_encode(layout, W, thr_d)
+    if case == "codec":
+        out = torch.empty(N, K, dtype=torch.bfloat16, device="cuda")
+        for _ in range(3):
+            lowra_decode(layout, packed, absmax, maps_d, out=out)
+            lowra_encode(layout, W, thr_d, packed=packed, absmax=absmax)
+        torch.cuda.synchronize()
+        print("codec ok")
+        return
+    act_cols = K if case == "forward" else N
+    act = torch.randn(M, act_cols, device="cuda", generator=gen).bfloat16()
+    A = (torch.randn(K, r, device="cuda", generator=gen) * 0.01).bfloat16()
+    B = (torch.randn(r, N, device="cuda", generator=gen) * 0.01).bfloat16()
+    ws = torch.empty(lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")
+    fn = lowra_lora_forward if case == "forward" else lowra_lora_backward_input
+    for _ in range(3):
+        fn(layout, packed, absmax, maps_d, act, A, B, s, workspace=ws)
+    status = lowra_device_status(ws)
+    print(case, "status", status)
+    if status != 0:
+        raise SystemExit(1)
+
+
+if __name__ == "__main__":
+    main(sys.argv[1] if len(sys.argv) > 1 else "forward")
