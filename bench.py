@@ -140,7 +140,7 @@ def make_host_inputs(cfg, rank: int):
     M, r = cfg.tokens[0], cfg.rank
 
     def one(mat):
-        mid = mat.matrix_id + 7 * rank
+        mid = rank_matrix_id(mat.matrix_id, rank)
         W = si.weights(mat.N, mat.K, matrix_id=mid, kind=cfg.weight_kind)
         precs = si.precisions(mat.N, cfg.mix, matrix_id=mid)
         maps, thr = si.standin_codebooks(precs, matrix_id=mid)
@@ -175,6 +175,27 @@ def fused_traffic_per_launch(dev, M, r, bits):
     per = [fused_input_bytes(d["m"]["N"], d["m"]["K"], M, r, bits) for d in dev] + \
           [fused_input_bytes(d["m"]["K"], d["m"]["N"], M, r, bits) for d in dev]   # backward reads dY [M, N]
     return NCU_CASE["dram_bytes"] / case * sum(per) / len(per)
+
+
+def max_over_ranks(ms: float, world: int, device="cuda") -> float:
+    """Slowest rank's time: the job is done when its last rank is (all-reduce MAX over the process group)."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_tflops(flops_per_rank_step: float, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank does one layer step per step (weak scaling)."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
+
+
+def rank_matrix_id(matrix_id: int, rank: int, per_layer: int = 7) -> int:
+    """Ranks hold different layers: the seed stream of matrix j on rank q is that of matrix j + 7 q."""
+    return matrix_id + per_layer * rank
 
 
 def run_gpu(args):
@@ -268,14 +289,11 @@ def run_gpu(args):
     t1 = time.time()
     clocks = sampler.stop(t0, t1)
     total_ms = ev0.elapsed_time(ev1)
-    if world > 1:
-        t = torch.tensor([total_ms], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world)
     ms_per_step = total_ms / args.steps
 
     flops_step = sum(2 * gemm_flops(M, d["m"]["N"], d["m"]["K"], r) for d in dev)
-    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+    value = aggregate_tflops(flops_step, world, ms_per_step)
 
     phase_ms = {}
     for phase, e0, e1 in records:
@@ -343,11 +361,8 @@ def run_gpu(args):
         b.record(stream)
         barrier()
         ms = a.elapsed_time(b) / n_e2e
-        if world > 1:
-            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        e2e = {"value": world * flops_step / (ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": ms,
+        ms = max_over_ranks(ms, world)
+        e2e = {"value": aggregate_tflops(flops_step, world, ms), "unit": UNIT, "ms_per_step": ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e}
 
     cpu = None
