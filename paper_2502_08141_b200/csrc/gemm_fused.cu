@@ -3,19 +3,20 @@
 // One persistent CTA per SM walks over output tiles of 128 "operand rows" x 256 tokens:
 //   forward : operand rows = output channels n;  Y^T tile [128 n x 256 m]  = W_hat[n, :] . X[m, :]
 //   backward: operand rows = input features k;   dX^T tile [128 k x 256 m] = W_hat[:, k] . dY[m, :]
-// The 128-row operand (the weights) is the A operand of tcgen05.mma and is produced in shared memory by
-// eight dequant warps straight from the packed codes (never from HBM as bf16); the 256-token operand
-// (activations / output gradients) is the B operand and arrives by TMA.  The accumulator lives in
-// TMEM (two 128 x 256 fp32 buffers, so the epilogue of one tile overlaps the main loop of the next).
+// The 128-row operand (the weights) is the A operand of tcgen05.mma and is produced by twelve dequant warps
+// straight from the packed codes (never from HBM as bf16): into tensor memory in the forward pass (a thread
+// owns one output channel = one TMEM lane for the whole tile), into shared memory (MN-major) in the backward
+// pass, where every stage brings 64 new channels.  The 256-token operand (activations / output gradients)
+// is the B operand and arrives by TMA.  Accumulators live in TMEM.
 // The LoRA term is folded into the same accumulator as extra contraction blocks at the end of every
-// tile, whose operands both arrive by TMA: the up-projection factor straight from the caller's matrix
-// and the down-projected activations T = s X A (resp. U = s dY B^T).  T itself is produced by this same
+// tile: the up-projection factor comes by TMA straight from the caller's matrix, the down-projected
+// activations T = s X A (resp. U = s dY B^T) by TMA from the workspace.  T itself is produced by this same
 // kernel: for every token tile there is one extra "T tile" whose 128 operand rows are the LoRA ranks
 // (factor fetched by TMA, no dequant); T tiles come first in the tile order, their epilogue publishes a
 // per-token-tile flag, and the TMA producer of a regular tile waits (bounded) for that flag before it
 // fetches T.  All CTAs are co-resident and walk the tiles in increasing order, so the wait cannot deadlock.
 //
-// Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, 6-13 = dequant.
+// Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, 6-17 = dequant.
 // All mbarrier waits are bounded; a wait that runs out sets the status word and every role leaves.
 #include "gemm_params.cuh"
 #include "ptx.cuh"
@@ -46,6 +47,7 @@ struct Barriers {
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort;
+    uint32_t free_upto;         // backward: stages 0 .. free_upto - 1 have been found free by the TMA producer
 };
 
 // fields of the per-thread row word written by the prologue (see kIdleItem below)
@@ -266,7 +268,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             ptx::mbar_init(&bars->empty[s], 1);
         }
         for (int s = 0; s < kWSlots; ++s) {
-            ptx::mbar_init(&bars->full_w[s], MODE == kModeForward ? 4 : kProducerWarps);
+            ptx::mbar_init(&bars->full_w[s], MODE == kModeForward ? 4 : kStageArrivals);
             ptx::mbar_init(&bars->empty_w[s], 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -275,6 +277,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         }
         ptx::mbar_init(&bars->drain, 1);
         bars->abort = 0u;
+        bars->free_upto = 0u;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmB);
         if (P.lora_blocks > 0) { ptx::prefetch_tensormap(&tmT); ptx::prefetch_tensormap(&tmFt); }
@@ -299,6 +302,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!ptx::mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                    if (MODE == kModeBackward) ptx::st_release_shared(&bars->free_upto, it + 1u);
                     unsigned char* a_s = base + s * kSmemStage;
                     unsigned char* b_s = a_s + kSmemA;
                     uint64_t* bar = &bars->full_x[s];
@@ -478,32 +482,58 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         }
     } else if (MODE != kModeDense) {
         // ================================================================== dequant producers
-        // All eight warps take part in every stage.  The prologue has dealt the rows of every group to the
-        // 256 threads so that a warp only ever holds rows of one precision (chunks of at most 32 rows
-        // forward, 16 rows x 2 feature halves backward); with n chunks, 8 / n warps share a chunk and take
-        // turns.  Each thread dequantises one 64-element absmax block per turn; the packed codes of the next
-        // two stages are already in registers (a two-deep ring with static indices, so no load is waited
-        // on early).
+        // The prologue has dealt the rows to these warps (see gemm_prep.cu).  Each thread dequantises one
+        // 64-element absmax block per visit of a stage.
         const int pt = threadIdx.x - kFirstProducerWarp * 32;  // 0..255
         const uint32_t slut_addr = ptx::smem_u32(slut_all) + (uint32_t)((pt >> 5) * 2048 + lane * 4);
         const int K = P.L.K;
+        const int pw = warp - kFirstProducerWarp;               // 0 .. kProducerWarps - 1
         uint32_t it0 = 0;                                       // running stage index at the start of the tile
+        // Backward: a warp only visits the stages it has work on, so it can be several ring revolutions behind
+        // or ahead of a stage's "empty" barrier, where a parity wait says nothing.  The TMA producer visits every
+        // stage in order and publishes how many stages it has found free (bars->free_upto); the dequant warps
+        // follow that counter instead (lane 0 polls, bounded).
+        uint32_t seen_free = 0;
+        auto stage_free = [&](uint32_t it) -> bool {
+            if (it < seen_free) return true;
+            uint32_t v = 0;
+            if (lane == 0) {
+                uint64_t t_start = 0;
+#pragma unroll 1
+                for (uint32_t spin = 0;; ++spin) {
+                    v = ptx::ld_acquire_shared(&bars->free_upto);
+                    if (v > it) break;
+                    __nanosleep(20);
+                    if ((spin & 255u) == 255u) {
+                        if (t_start == 0) t_start = ptx::globaltimer_ns();
+                        if (*abort_flag != 0u || ptx::globaltimer_ns() - t_start > kWaitLimitNs) { v = 0; break; }
+                    }
+                }
+            }
+            v = __shfl_sync(0xffffffffu, v, 0);
+            if (v <= it) return false;
+            seen_free = v;
+            return true;
+        };
         for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x) {
             const TileInfo t = decode_tile(g);
             const int r0 = t.rt * kTileR;
-            if (t.is_t) {
-                // nothing to dequantise: keep the stage barriers in step (forward: the warps whose turn it is)
-                const int first = (MODE == kModeForward) ? (pt >> 7) : 0;
-                const int step = (MODE == kModeForward) ? kTurns : 1;
-                for (int kb = first; kb < t.blocks; kb += step) {
+            if (t.is_t && MODE == kModeForward) {
+                // nothing to dequantise: the warps whose turn it is keep the stage barriers in step
+                for (int kb = pt >> 7; kb < t.blocks; kb += kTurns) {
                     const uint32_t it = it0 + (uint32_t)kb;
-                    const int ring = (MODE == kModeForward) ? kWSlots : kStages;
-                    const int s = it % ring;
-                    uint64_t* eb = (MODE == kModeForward) ? &bars->empty_w[s] : &bars->empty[s];
-                    if (!ptx::mbar_wait_warp(eb, ((it / ring) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
+                    const int s = it % kWSlots;
+                    if (!ptx::mbar_wait_warp(&bars->empty_w[s], ((it / kWSlots) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
                         failed = true; bars->abort = 1u; break;
                     }
                     if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
+                }
+            } else if (t.is_t) {
+                // backward: the warps take the stages in turn and arrive for everybody
+                for (int kb = pw; kb < t.blocks; kb += kProducerWarps) {
+                    const uint32_t it = it0 + (uint32_t)kb;
+                    if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
+                    if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % kStages], kStageArrivals);
                 }
             } else if (MODE == kModeForward) {
                 // ---------------------------------------------------------------- forward
@@ -584,25 +614,28 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // ---------------------------------------------------------------- backward
                 // every stage brings 64 new channels (the contraction index); thread = one channel x 64 of
                 // the tile's 128 input features = one absmax block.  Operand tile is MN-major:
-                // [feature half][64 channels][64 features], so the block is one 128-byte row and is
-                // written exactly as in the forward case.  The deal (and the turn-taking) is per stage.
+                // [feature half][64 channels][64 features], so the block is one 128-byte row.
+                // The warp walks its own work list (written by the prologue): entry = (stage, 16 rows of one
+                // precision); entries two ahead are already in registers (codes, absmax, levels), in a
+                // two-deep ring with static indices so that no load is waited on early.
                 const int half = (lane >> 4) & 1;
                 const int k_first = r0 + 64 * half;
-                const uint32_t* items = P.items + pt;
-                uint32_t info_ring[2];
+                const uint32_t* heads = P.heads + pw;                       // entry j of this warp: heads[j * kProducerWarps]
+                const uint32_t* items = P.items + (size_t)pw * 32 + lane;   // and items[j * kProducerWarps * 32]
+                constexpr uint32_t kEnd = 0xFFFFFFFFu;
+                uint32_t head_cur[2], head_nxt[2], item_cur[2], item_nxt[2];
                 Block ring[2];
                 Levels lvr[2];
                 ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
                 ring[0].a = ring[1].a = 0.0f;
                 lvr[0] = lvr[1] = Levels{0.f, 0.f, 0.f, 0.f};
-                uint32_t cur_info[2] = {kIdleItem, kIdleItem};
                 Levels16 m16;
 #pragma unroll
                 for (int e = 0; e < 16; ++e) m16.v[e] = 0.0f;
 
-                // fetch everything block mb needs except a 4-bit table: codes, absmax, 1/2-bit levels
-                auto fetch = [&](Block& blk, Levels& lv, uint32_t info, int mb) {
-                    const int cls = (info == kIdleItem) ? 4 : info_class(info);
+                // fetch everything an entry needs except a 4-bit table: codes, absmax, 1/2-bit levels
+                auto fetch = [&](Block& blk, Levels& lv, uint32_t head, uint32_t info) {
+                    const int cls = (head == kEnd || info == kIdleItem) ? 4 : info_class(info);
                     if (cls < 3) {
                         const int p = info_pos(info);
                         const int b = 1 << cls;
@@ -610,7 +643,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                                    P.packed + P.L.seg_off[cls] + (size_t)(p - P.L.class_start[cls]) * ((size_t)K * b / 8) +
                                        (size_t)k_first * b / 8,
                                    P.absmax + (size_t)p * P.L.nb + k_first / kBlock, cls);
-                        const float* mrow = P.maps + (size_t)(mb * kTileC + info_row(info)) * kTableStride;
+                        const float* mrow = P.maps + (size_t)((head & 0xFFFFFFu) * kTileC + info_row(info)) * kTableStride;
                         if (cls == 0) {
                             lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
                         } else if (cls == 1) {
@@ -618,10 +651,10 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         }
                     }
                 };
-                auto fetch_table = [&](uint32_t info, int mb) {
-                    if (info != kIdleItem && info_class(info) == 2) {
+                auto fetch_table = [&](uint32_t head, uint32_t info) {
+                    if (head != kEnd && info != kIdleItem && info_class(info) == 2) {
                         const float4* m4 = reinterpret_cast<const float4*>(
-                            P.maps + (size_t)(mb * kTileC + info_row(info)) * kTableStride);
+                            P.maps + (size_t)((head & 0xFFFFFFu) * kTileC + info_row(info)) * kTableStride);
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float4 f = __ldg(m4 + e);
@@ -630,52 +663,58 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     }
                 };
 
-                // prologue: blocks 0 and 1 fully, row descriptors of blocks 2 and 3
+                // prologue: entries 0 and 1 in full, heads and row words of entries 2 and 3
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    if (u < P.main_blocks) {
-                        cur_info[u] = __ldg(items + (size_t)u * kItemStride);
-                        fetch(ring[u], lvr[u], cur_info[u], u);
-                    }
-                    info_ring[u] = (u + 2 < P.main_blocks) ? __ldg(items + (size_t)(u + 2) * kItemStride) : kIdleItem;
+                    head_cur[u] = __ldg(heads + (size_t)u * kProducerWarps);
+                    item_cur[u] = __ldg(items + (size_t)u * kProducerWarps * 32);
+                    fetch(ring[u], lvr[u], head_cur[u], item_cur[u]);
+                    head_nxt[u] = __ldg(heads + (size_t)(u + 2) * kProducerWarps);
+                    item_nxt[u] = __ldg(items + (size_t)(u + 2) * kProducerWarps * 32);
                 }
-                if (P.main_blocks > 0) fetch_table(cur_info[0], 0);
-                for (int kb0 = 0; kb0 < t.blocks && !failed; kb0 += 2) {
+                fetch_table(head_cur[0], item_cur[0]);
+                bool list_end = false;
+                for (uint32_t j0 = 0; !list_end && !failed; j0 += 2) {
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const int mb = kb0 + u;
-                        if (mb >= t.blocks) break;
-                        const uint32_t it = it0 + (uint32_t)mb;
+                        const uint32_t head = head_cur[u];
+                        if (head == kEnd) { list_end = true; break; }
+                        const uint32_t mb = head & 0xFFFFFFu;
+                        const uint32_t it = it0 + mb;
                         const int s = it % kStages;
-                        const uint32_t ph = (it / kStages) & 1u;
-                        if (!ptx::mbar_wait_warp(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
-                            failed = true; bars->abort = 1u; break;
-                        }
-                        if (mb < P.main_blocks) {
-                            const uint32_t info = cur_info[u];
-                            const bool active = info != kIdleItem;
-                            const int wcls = __shfl_sync(0xffffffffu, active ? info_class(info) : 4, 0);
-                            if (active) {
-                                const int col = info_row(info);   // channel inside the stage = K index of the tile
-                                const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + (uint32_t)half * 8192u +
-                                                          (uint32_t)col * 128u;
-                                if (wcls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lvr[u].m0, lvr[u].m1, ring[u].a, row_addr, col & 7);
-                                else if (wcls == 1) dequant_block_2bit(ring[u].lo, lvr[u], ring[u].a, row_addr, col & 7);
-                                else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, m16, slut_addr, row_addr, col & 7);
-                                else zero_row(row_addr);
-                                ptx::fence_proxy_async_smem();
-                            }
+                        if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
+                        const uint32_t info = item_cur[u];
+                        const bool active = info != kIdleItem;
+                        const int wcls = __shfl_sync(0xffffffffu, active ? info_class(info) : 4, 0);
+                        if (active) {
+                            const int col = info_row(info);   // channel inside the stage = K index of the tile
+                            const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + (uint32_t)half * 8192u +
+                                                      (uint32_t)col * 128u;
+                            if (wcls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lvr[u].m0, lvr[u].m1, ring[u].a, row_addr, col & 7);
+                            else if (wcls == 1) dequant_block_2bit(ring[u].lo, lvr[u], ring[u].a, row_addr, col & 7);
+                            else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, m16, slut_addr, row_addr, col & 7);
+                            else zero_row(row_addr);
+                            ptx::fence_proxy_async_smem();
                         }
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
-                        // refill this ring slot for its next stage (block mb + 2), fetch the 4-bit table of the
-                        // very next stage (block mb + 1, other slot), look two stages further ahead for the row
-                        const int nb = mb + 2;
-                        cur_info[u] = info_ring[u];
-                        if (nb < P.main_blocks) fetch(ring[u], lvr[u], cur_info[u], nb);
-                        info_ring[u] = (nb + 2 < P.main_blocks) ? __ldg(items + (size_t)(nb + 2) * kItemStride) : kIdleItem;
-                        if (mb + 1 < P.main_blocks) fetch_table(cur_info[u ^ 1], mb + 1);
+                        if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[s], head >> 24);
+                        // refill this ring slot with the entry after next, fetch the 4-bit table of the next
+                        // entry (other slot), look two entries further ahead for head and row word
+                        head_cur[u] = head_nxt[u];
+                        item_cur[u] = item_nxt[u];
+                        fetch(ring[u], lvr[u], head_cur[u], item_cur[u]);
+                        if (head_cur[u] != kEnd) {   // the lists end with kListSlack all-ones heads
+                            head_nxt[u] = __ldg(heads + (size_t)(j0 + u + 4) * kProducerWarps);
+                            item_nxt[u] = __ldg(items + (size_t)(j0 + u + 4) * kProducerWarps * 32);
+                        }
+                        fetch_table(head_cur[u ^ 1], item_cur[u ^ 1]);
                     }
+                }
+                // LoRA blocks: operands come by TMA; the warps take the stages in turn and arrive for everybody
+                for (int kb = P.main_blocks + pw; kb < t.blocks && !failed; kb += kProducerWarps) {
+                    const uint32_t it = it0 + (uint32_t)kb;
+                    if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
+                    if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % kStages], kStageArrivals);
                 }
             }
             it0 += (uint32_t)t.blocks;

@@ -26,12 +26,15 @@ Workspace plan_workspace(int N, int K, int M, int r) {
     (void)K;
     Workspace w;
     w.rp = (r + 63) / 64 * 64;
-    const size_t groups = (size_t)(N + 63) / 64;   // backward has the most row groups
+    // forward: 128 row words per group of 128 channels; backward: at most 7 work-list entries (a head and
+    // 32 row words each) per group of 64 channels, plus the end markers
+    const size_t entries = 7 * ((size_t)(N + 63) / 64) + kListSlack;
+    const size_t fwd_words = (size_t)((N + 127) / 128) * kItemStride;
     w.off_T = kStatusBytes;
     w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);
     w.off_items = w.off_flags + align256((size_t)((M + kTileT - 1) / kTileT) * 4);
-    w.off_meta = w.off_items + align256(groups * kItemStride * 4);
-    w.total = w.off_meta + align256(groups * 4);
+    w.off_meta = w.off_items + align256((entries * 32 > fwd_words ? entries * 32 : fwd_words) * 4);
+    w.total = w.off_meta + align256(entries * 4);
     return w;
 }
 
@@ -69,7 +72,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     if (st != LOWRA_OK) return st;
     if (!packed || !absmax || !maps || !act || !A || !B || !out || !workspace) return LOWRA_ERR_NULL;
     const int N = layout->N, K = layout->K;
-    if (M < 1 || !rank_ok(r) || N % 8 != 0 || N >= (1 << 23)) return LOWRA_ERR_SHAPE;
+    if (M < 1 || !rank_ok(r) || N % 8 != 0 || N > 64 * kMaxGroups64) return LOWRA_ERR_SHAPE;
     if (!aligned16(packed) || !aligned16(absmax) || !aligned16(maps) || !aligned16(act) || !aligned16(A) ||
         !aligned16(B) || !aligned16(out))
         return LOWRA_ERR_ALIGN;
@@ -84,7 +87,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
     uint32_t* flags = reinterpret_cast<uint32_t*>(ws + w.off_flags);
     uint32_t* items = reinterpret_cast<uint32_t*>(ws + w.off_items);
-    uint32_t* n_chunks = reinterpret_cast<uint32_t*>(ws + w.off_meta);
+    uint32_t* heads = reinterpret_cast<uint32_t*>(ws + w.off_meta);
     const int tiles_t = (M + kTileT - 1) / kTileT;
 
     // ---- prologue: clear status and flags, deal the rows
@@ -93,7 +96,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     P.precs = layout->precs_dev;
     P.inv_perm = layout->inv_perm_dev;
     P.items = items;
-    P.n_chunks = n_chunks;
+    P.heads = heads;
     P.N = N;
     P.group = backward ? 64 : 128;
     P.status = status;
@@ -111,7 +114,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.absmax = absmax;
     G.maps = maps;
     G.items = items;
-    G.n_chunks = n_chunks;
+    G.heads = heads;
     G.out = out;
     G.T = T;
     G.flags = flags;

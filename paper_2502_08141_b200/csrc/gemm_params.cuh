@@ -10,16 +10,20 @@ namespace lowra {
 // ---- prologue ------------------------------------------------------------------------------
 constexpr int kPrepThreads = 128;
 constexpr int kProducerWarps = 12;            // dequant warps of the main kernel: three per tensor-memory lane quarter
-constexpr int kItemStride = 512;              // entries per row group in the deal table (>= 32 * kProducerWarps)
+constexpr int kItemStride = 128;              // forward: entries per group of 128 rows in the deal table
+constexpr int kStageArrivals = 8;             // backward: arrivals a stage barrier expects from the dequant warps (>= 7 chunks)
+constexpr int kListSlack = 48;                // backward: all-ones heads written behind the last work-list entry
+constexpr int kMaxGroups64 = 8192;            // backward: at most this many groups of 64 output channels (N <= 524288)
 
 struct PrepParams {
-    // deal of the rows of every group (128 rows forward, 64 backward) to the 256 dequant threads of the
-    // main kernel, one precision per warp: items[g * kItemStride + thread] = row offset (bits 0-6) | class
-    // (bits 7-8, 3 = row past N) | stored position (bits 9-31), or all ones for "no row"
+    // deal of the rows to the dequant threads of the main kernel.  Row word = row offset inside its group
+    // (bits 0-6) | class (bits 7-8, 3 = row past N) | stored position (bits 9-31), all ones for "no row".
+    //   forward (group 128): items[g * kItemStride + i] = i-th row of group g in precision order
+    //   backward (group 64): per-warp work lists, see deal_backward
     const uint8_t* precs;
     const int32_t* inv_perm;
-    uint32_t* items;      // [ceil(N / group) * kItemStride]
-    uint32_t* n_chunks;   // [ceil(N / group)] number of chunks the group was cut into (1..7)
+    uint32_t* items;
+    uint32_t* heads;      // backward: [7 * ceil(N / 64) + kListSlack] work-list heads
     int N, group;
     uint32_t* status;     // device status word, cleared
     uint32_t* flags;      // [n_flags] "T of this token tile is ready" flags, cleared
@@ -46,8 +50,8 @@ struct GemmParams {
     const uint8_t* packed;
     const float* absmax;
     const float* maps;
-    const uint32_t* items;    // from the prologue: [row groups][kItemStride]
-    const uint32_t* n_chunks; // from the prologue: [row groups]
+    const uint32_t* items;    // from the prologue: row words (forward: per tile; backward: per work-list entry)
+    const uint32_t* heads;    // from the prologue (backward): work-list heads
     uint16_t* out;          // [M, ld_out] bf16
     uint16_t* T;            // [M, rp] bf16: s * X . A (forward) or s * dY . B^T (backward), written by the T tiles
     uint32_t* flags;        // [tiles_t] raised when T of a token tile is complete

@@ -1,7 +1,7 @@
 // Prologue of the fused forward / backward-input calls: one small launch that clears the device status
 // word and the "T ready" flags, and deals the rows of every group of 128 (forward) or 64 (backward)
-// consecutive output channels to the 256 dequant threads of the main kernel so that each warp only holds
-// rows of one precision.
+// consecutive output channels to the dequant threads of the main kernel so that a warp holds rows of one
+// precision wherever the counts allow.
 #include "gemm_params.cuh"
 #include "ptx.cuh"
 
@@ -9,99 +9,161 @@ namespace lowra {
 
 namespace {
 
-// One warp per group of G rows (128 forward, 64 backward).  The rows are ordered by precision class
-// (1 bit, 2 bits, 4 bits, rows past N; stable).
-//   forward : entry i of the group is the i-th row in that order = the row held by tensor-memory lane i of
-//             the main kernel, so that at most two precisions meet in a warp (32 consecutive lanes);
-//   backward: the ordered rows are cut into chunks of 16 rows of one class (every row is handled by two
-//             threads, one per 64-feature half), so that no warp ever sees two precisions.  At most
-//             64 / 16 + 3 = 7 chunks exist and the kernel has 12 dequant warps: with n chunks, k = 12 / n warps
-//             share a chunk and take turns (warp c + j * n serves chunk c in the groups congruent to j mod k).
+// Forward: one warp per group of 128 consecutive output channels (one weight tile of the main kernel).  The
+// rows are ordered by precision class (1 bit, 2 bits, 4 bits, rows past N; stable); entry i of the group is the
+// i-th row in that order = the row held by tensor-memory lane i of the main kernel, so that at most two
+// precisions meet in a warp (32 consecutive lanes).
 __device__ void deal_rows(const PrepParams& P, int blk) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int G = P.group, per = G / 32;
-    const int CH = (G == 128) ? 32 : 16;
+    constexpr int G = 128, per = G / 32;
     const int n_groups = (P.N + G - 1) / G;
     for (int grp = blk * (kPrepThreads / 32) + warp; grp < n_groups; grp += P.blocks * (kPrepThreads / 32)) {
         uint32_t* out = P.items + (size_t)grp * kItemStride;
-#pragma unroll
-        for (int i = 0; i < kItemStride / 32; ++i) out[i * 32 + lane] = 0xFFFFFFFFu;
-        __syncwarp();
-        int cls[4];
-        unsigned mask[4][4];
+        int cls[per];
+        unsigned mask[per][4];
         int total[4] = {0, 0, 0, 0};
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            cls[i] = 3;
-            if (i < per) {
-                const int row = grp * G + i * 32 + lane;
-                if (row < P.N) cls[i] = P.precs[row] >> 1;
-            }
+        for (int i = 0; i < per; ++i) {
+            const int row = grp * G + i * 32 + lane;
+            cls[i] = (row < P.N) ? (P.precs[row] >> 1) : 3;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                mask[i][c] = (i < per) ? __ballot_sync(0xffffffffu, cls[i] == c) : 0u;
+                mask[i][c] = __ballot_sync(0xffffffffu, cls[i] == c);
                 total[c] += __popc(mask[i][c]);
+            }
+        }
+        int class_base[4];
+        class_base[0] = 0;
+#pragma unroll
+        for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total[c - 1];
+        int before[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int i = 0; i < per; ++i) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                if (cls[i] == c) {
+                    const int q = before[c] + __popc(mask[i][c] & ((1u << lane) - 1u));  // rank inside the class
+                    const int off = i * 32 + lane, row = grp * G + off;
+                    const uint32_t p = (c < 3) ? (uint32_t)P.inv_perm[row] : 0u;
+                    out[class_base[c] + q] = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) before[c] += __popc(mask[i][c]);
+        }
+    }
+}
+
+// Backward-input: every pipeline stage of the main kernel brings a group of 64 consecutive output channels.
+// The rows of a group are ordered by precision class and cut into chunks of at most 16 rows of one class; a
+// chunk is the work of one dequant warp on one stage (32 lanes = 16 rows x 2 halves of the tile's 128
+// features).  Chunks are numbered through the whole matrix (group after group) and chunk g goes to warp
+// g % kProducerWarps as entry g / kProducerWarps of that warp's work list, so a warp only ever visits the
+// stages it has work on:
+//   heads[e]          = group index (bits 0-23) | number of arrivals this entry owes the stage barrier (bits 24-31)
+//   items[e * 32 + l] = row word of lane l (see deal_rows), all ones for "no row"
+// with e = entry * kProducerWarps + warp.  The stage barrier expects kStageArrivals arrivals; the first chunk
+// of a group also arrives for the chunks the group does not have.  The lists end with an all-ones head.
+__device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint32_t* wsum) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
+    constexpr int kWarps = kPrepThreads / 32;
+    const int n_groups = (P.N + 63) / 64;
+    // ---- chunks per group (every block computes all of them: the numbering needs the running sum)
+    for (int grp = warp; grp < n_groups; grp += kWarps) {
+        const int r0 = grp * 64 + lane, r1 = r0 + 32;
+        const int c0 = (r0 < P.N) ? (P.precs[r0] >> 1) : 3, c1 = (r1 < P.N) ? (P.precs[r1] >> 1) : 3;
+        int n = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            n += (__popc(__ballot_sync(0xffffffffu, c0 == c)) + __popc(__ballot_sync(0xffffffffu, c1 == c)) + 15) / 16;
+        if (lane == 0) pre[grp] = (uint16_t)n;
+    }
+    __syncthreads();
+    // ---- exclusive running sum over the groups
+    const int seg = (n_groups + kPrepThreads - 1) / kPrepThreads;
+    const int begin = min(tid * seg, n_groups), end = min(begin + seg, n_groups);
+    uint32_t mine = 0;
+    for (int i = begin; i < end; ++i) mine += pre[i];
+    uint32_t incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
+        if (lane >= d) incl += v;
+    }
+    if (lane == 31) wsum[warp] = incl;
+    __syncthreads();
+    uint32_t run = incl - mine;
+    uint32_t total = 0;
+#pragma unroll
+    for (int w2 = 0; w2 < kWarps; ++w2) {
+        if (w2 < warp) run += wsum[w2];
+        total += wsum[w2];
+    }
+    for (int i = begin; i < end; ++i) {
+        const uint32_t n = pre[i];
+        pre[i] = (uint16_t)run;
+        run += n;
+    }
+    __syncthreads();
+    if (blk == 0)
+        for (int i = tid; i < kListSlack; i += kPrepThreads) P.heads[total + i] = 0xFFFFFFFFu;
+
+    // ---- the deal proper: one warp per group
+    for (int grp = blk * kWarps + warp; grp < n_groups; grp += P.blocks * kWarps) {
+        const uint32_t g0 = pre[grp];
+        int cls[2];
+        unsigned mask[2][4];
+        int total_c[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int row = grp * 64 + i * 32 + lane;
+            cls[i] = (row < P.N) ? (P.precs[row] >> 1) : 3;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                mask[i][c] = __ballot_sync(0xffffffffu, cls[i] == c);
+                total_c[c] += __popc(mask[i][c]);
             }
         }
         int chunk_base[4];
         chunk_base[0] = 0;
 #pragma unroll
-        for (int c = 1; c < 4; ++c) chunk_base[c] = chunk_base[c - 1] + (total[c - 1] + CH - 1) / CH;
-        int class_base[4];
-        class_base[0] = 0;
+        for (int c = 1; c < 4; ++c) chunk_base[c] = chunk_base[c - 1] + (total_c[c - 1] + 15) / 16;
+        const int n_chunks = chunk_base[3] + (total_c[3] + 15) / 16;
+        auto entry_of = [&](int ci) { return g0 + (uint32_t)ci; };   // the warps' lists interleave: e = chunk number
+        for (int ci = 0; ci < n_chunks; ++ci) P.items[(size_t)entry_of(ci) * 32 + lane] = 0xFFFFFFFFu;
+        if (lane < n_chunks)
+            P.heads[entry_of(lane)] = (uint32_t)grp | ((uint32_t)(lane == 0 ? kStageArrivals - n_chunks + 1 : 1) << 24);
+        __syncwarp();
 #pragma unroll
-        for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total[c - 1];
-        const int n_chunks = chunk_base[3] + (total[3] + CH - 1) / CH;
-        const int k = kProducerWarps / n_chunks;   // warps that share a chunk (backward)
-        if (lane == 0) P.n_chunks[grp] = (uint32_t)n_chunks;
-        int before[4] = {0, 0, 0, 0};
+        for (int i = 0; i < 2; ++i) {
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            if (i < per) {
+            for (int c = 0; c < 4; ++c) {
+                if (cls[i] == c) {
+                    const int off = i * 32 + lane, row = grp * 64 + off;
+                    const uint32_t p = (c < 3) ? (uint32_t)P.inv_perm[row] : 0u;
+                    const uint32_t word = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
+                    // inside the class the rows are taken round-robin over (row offset mod 8), so that eight
+                    // neighbouring lanes hold eight different residues: their 16-byte stores into the swizzled
+                    // operand tile then fall into eight different bank groups
+                    const unsigned res_mask = 0x01010101u << (lane & 7);
+                    int b = 0;   // rank of this row among the rows of its class with the same residue
+                    if (i == 1) b += __popc(mask[0][c] & res_mask);
+                    b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
+                    int pos = 0;  // rows taken before this one
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    if (cls[i] == c) {
-                        const int q = before[c] + __popc(mask[i][c] & ((1u << lane) - 1u));  // rank inside the class
-                        const int off = i * 32 + lane, row = grp * G + off;
-                        const uint32_t p = (c < 3) ? (uint32_t)P.inv_perm[row] : 0u;
-                        const uint32_t word = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
-                        if (CH == 32) {
-                            // forward: position in precision order = tensor-memory lane of the row
-                            out[class_base[c] + q] = word;
-                        } else {
-                            // backward: the group index is the stage index; of the k warps that share the
-                            // chunk, the one whose turn it is gets the row (for both feature halves).
-                            // Inside the class the rows are taken round-robin over (row offset mod 8), so that
-                            // eight neighbouring lanes hold eight different residues: their 16-byte stores into
-                            // the swizzled operand tile then fall into eight different bank groups.
-                            const unsigned res_mask = 0x01010101u << (lane & 7);
-                            int b = 0;   // rank of this row among the rows of its class with the same residue
-#pragma unroll
-                            for (int i2 = 0; i2 < 4; ++i2)
-                                if (i2 < i) b += __popc(mask[i2][c] & res_mask);
-                            b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
-                            int pos = 0;  // rows taken before this one
-#pragma unroll
-                            for (int res = 0; res < 8; ++res) {
-                                int cnt = 0;
-#pragma unroll
-                                for (int i2 = 0; i2 < 4; ++i2)
-                                    if (i2 < per) cnt += __popc(mask[i2][c] & (0x01010101u << res));
-                                pos += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
-                            }
-                            const int j = grp % k;
-                            const int thread = (chunk_base[c] + pos / CH + j * n_chunks) * 32 + pos % CH;
-                            out[thread] = word;
-                            out[thread + 16] = word;
-                        }
+                    for (int res = 0; res < 8; ++res) {
+                        const int cnt = __popc(mask[0][c] & (0x01010101u << res)) + __popc(mask[1][c] & (0x01010101u << res));
+                        pos += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
                     }
+                    uint32_t* dst = P.items + (size_t)entry_of(chunk_base[c] + pos / 16) * 32 + pos % 16;
+                    dst[0] = word;
+                    dst[16] = word;
                 }
-#pragma unroll
-                for (int c = 0; c < 4; ++c) before[c] += __popc(mask[i][c]);
             }
         }
     }
 }
+
 
 }  // namespace
 
@@ -110,7 +172,13 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const PrepParams P) 
         if (threadIdx.x == 0) *P.status = 0u;
         for (int i = threadIdx.x; i < P.n_flags; i += kPrepThreads) P.flags[i] = 0u;
     }
-    deal_rows(P, blockIdx.x);
+    if (P.group == 64) {
+        __shared__ uint16_t pre[kMaxGroups64];
+        __shared__ uint32_t wsum[kPrepThreads / 32];
+        deal_backward(P, blockIdx.x, pre, wsum);
+    } else {
+        deal_rows(P, blockIdx.x);
+    }
 }
 
 lowra_status launch_prep(const PrepParams& P, cudaStream_t stream) {
