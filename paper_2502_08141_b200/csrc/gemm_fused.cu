@@ -163,8 +163,15 @@ __device__ __noinline__ void dequant_block_2bit(uint4 w, Levels lv, float a, uin
     deq64_2bit(w, lv, a, o);
     store_row(row_addr, swz, o);
 }
-__device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, Levels16 lv, uint32_t slut_addr,
+__device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, const float* mrow, uint32_t slut_addr,
                                                 uint32_t row_addr, int swz) {
+    Levels16 lv;   // the row's 16 levels (the caller has prefetched the line)
+    const float4* m4 = reinterpret_cast<const float4*>(mrow);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const float4 f = __ldg(m4 + e);
+        lv.v[4 * e] = f.x; lv.v[4 * e + 1] = f.y; lv.v[4 * e + 2] = f.z; lv.v[4 * e + 3] = f.w;
+    }
     uint32_t o[32];
     deq64_4bit(lo, hi, a, lv, slut_addr, o);
     store_row(row_addr, swz, o);
@@ -621,93 +628,69 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const int half = (lane >> 4) & 1;
                 const int k_first = r0 + 64 * half;
                 const uint32_t* heads = P.heads + pw;                       // entry j of this warp: heads[j * kProducerWarps]
-                const uint32_t* items = P.items + (size_t)pw * 32 + lane;   // and items[j * kProducerWarps * 32]
+                const uint4* rows = reinterpret_cast<const uint4*>(P.items) + (size_t)pw * 32 + lane;   // rows[j * kProducerWarps * 32]
                 constexpr uint32_t kEnd = 0xFFFFFFFFu;
-                uint32_t head_cur[2], head_nxt[2], item_cur[2], item_nxt[2];
+                uint32_t head_cur[2];
+                uint4 rec_cur[2];
                 Block ring[2];
                 Levels lvr[2];
                 ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
                 ring[0].a = ring[1].a = 0.0f;
                 lvr[0] = lvr[1] = Levels{0.f, 0.f, 0.f, 0.f};
-                Levels16 m16;
-#pragma unroll
-                for (int e = 0; e < 16; ++e) m16.v[e] = 0.0f;
 
-                // fetch everything an entry needs except a 4-bit table: codes, absmax, 1/2-bit levels
-                auto fetch = [&](Block& blk, Levels& lv, uint32_t head, uint32_t info) {
-                    const int cls = (head == kEnd || info == kIdleItem) ? 4 : info_class(info);
+                // fetch what an entry needs: codes, absmax, 1/2-bit levels (a 4-bit table is only prefetched)
+                auto fetch = [&](Block& blk, Levels& lv, uint32_t head, const uint4& rec) {
+                    const int cls = (head == kEnd || rec.w == kIdleItem) ? 4 : (int)((head >> 28) & 3u);
                     if (cls < 3) {
-                        const int p = info_pos(info);
-                        const int b = 1 << cls;
-                        load_block(blk,
-                                   P.packed + P.L.seg_off[cls] + (size_t)(p - P.L.class_start[cls]) * ((size_t)K * b / 8) +
-                                       (size_t)k_first * b / 8,
-                                   P.absmax + (size_t)p * P.L.nb + k_first / kBlock, cls);
-                        const float* mrow = P.maps + (size_t)((head & 0xFFFFFFu) * kTileC + info_row(info)) * kTableStride;
+                        load_block(blk, P.packed + ((size_t)rec.x << 4) + (((size_t)k_first << cls) >> 3),
+                                   P.absmax + rec.y + (k_first >> 6), cls);
+                        const float* mrow = P.maps + rec.z;
                         if (cls == 0) {
                             lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
                         } else if (cls == 1) {
                             lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
-                        }
-                    }
-                };
-                auto fetch_table = [&](uint32_t head, uint32_t info) {
-                    if (head != kEnd && info != kIdleItem && info_class(info) == 2) {
-                        const float4* m4 = reinterpret_cast<const float4*>(
-                            P.maps + (size_t)((head & 0xFFFFFFu) * kTileC + info_row(info)) * kTableStride);
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float4 f = __ldg(m4 + e);
-                            m16.v[4 * e] = f.x; m16.v[4 * e + 1] = f.y; m16.v[4 * e + 2] = f.z; m16.v[4 * e + 3] = f.w;
+                        } else {
+                            ptx::prefetch_l1(mrow);
                         }
                     }
                 };
 
-                // prologue: entries 0 and 1 in full, heads and row words of entries 2 and 3
+                // prologue: entries 0 and 1
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
                     head_cur[u] = __ldg(heads + (size_t)u * kProducerWarps);
-                    item_cur[u] = __ldg(items + (size_t)u * kProducerWarps * 32);
-                    fetch(ring[u], lvr[u], head_cur[u], item_cur[u]);
-                    head_nxt[u] = __ldg(heads + (size_t)(u + 2) * kProducerWarps);
-                    item_nxt[u] = __ldg(items + (size_t)(u + 2) * kProducerWarps * 32);
+                    rec_cur[u] = __ldg(rows + (size_t)u * kProducerWarps * 32);
                 }
-                fetch_table(head_cur[0], item_cur[0]);
+#pragma unroll
+                for (int u = 0; u < 2; ++u) fetch(ring[u], lvr[u], head_cur[u], rec_cur[u]);
                 bool list_end = false;
                 for (uint32_t j0 = 0; !list_end && !failed; j0 += 2) {
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
                         const uint32_t head = head_cur[u];
                         if (head == kEnd) { list_end = true; break; }
-                        const uint32_t mb = head & 0xFFFFFFu;
-                        const uint32_t it = it0 + mb;
+                        const uint32_t col = rec_cur[u].w;   // channel inside the stage = K index of the tile
+                        const float* mrow = P.maps + rec_cur[u].z;
+                        // head and row record of the entry after next (this ring slot's next use) are asked for
+                        // now and consumed after this visit; the lists end with kListSlack all-ones heads
+                        head_cur[u] = __ldg(heads + (size_t)(j0 + u + 2) * kProducerWarps);
+                        rec_cur[u] = __ldg(rows + (size_t)(j0 + u + 2) * kProducerWarps * 32);
+                        const uint32_t it = it0 + (head & 0xFFFFFFu);
                         const int s = it % kStages;
                         if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
-                        const uint32_t info = item_cur[u];
-                        const bool active = info != kIdleItem;
-                        const int wcls = __shfl_sync(0xffffffffu, active ? info_class(info) : 4, 0);
-                        if (active) {
-                            const int col = info_row(info);   // channel inside the stage = K index of the tile
-                            const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + (uint32_t)half * 8192u +
-                                                      (uint32_t)col * 128u;
+                        if (col != kIdleItem) {
+                            const int wcls = (int)((head >> 28) & 3u);   // the same for the whole warp
+                            const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + (uint32_t)half * 8192u + col * 128u;
                             if (wcls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lvr[u].m0, lvr[u].m1, ring[u].a, row_addr, col & 7);
                             else if (wcls == 1) dequant_block_2bit(ring[u].lo, lvr[u], ring[u].a, row_addr, col & 7);
-                            else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, m16, slut_addr, row_addr, col & 7);
+                            else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, slut_addr, row_addr, col & 7);
                             else zero_row(row_addr);
                             ptx::fence_proxy_async_smem();
                         }
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[s], head >> 24);
-                        // refill this ring slot with the entry after next, fetch the 4-bit table of the next
-                        // entry (other slot), look two entries further ahead for head and row word
-                        head_cur[u] = head_nxt[u];
-                        item_cur[u] = item_nxt[u];
-                        fetch(ring[u], lvr[u], head_cur[u], item_cur[u]);
-                        if (head_cur[u] != kEnd) {   // the lists end with kListSlack all-ones heads
-                            head_nxt[u] = __ldg(heads + (size_t)(j0 + u + 4) * kProducerWarps);
-                            item_nxt[u] = __ldg(items + (size_t)(j0 + u + 4) * kProducerWarps * 32);
-                        }
-                        fetch_table(head_cur[u ^ 1], item_cur[u ^ 1]);
+                        if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[s], (head >> 24) & 15u);
+                        // refill this ring slot
+                        fetch(ring[u], lvr[u], head_cur[u], rec_cur[u]);
                     }
                 }
                 // LoRA blocks: operands come by TMA; the warps take the stages in turn and arrive for everybody

@@ -27,13 +27,13 @@ Workspace plan_workspace(int N, int K, int M, int r) {
     Workspace w;
     w.rp = (r + 63) / 64 * 64;
     // forward: 128 row words per group of 128 channels; backward: at most 7 work-list entries (a head and
-    // 32 row words each) per group of 64 channels, plus the end markers
+    // 32 row records of 16 bytes each) per group of 64 channels, plus the end markers
     const size_t entries = 7 * ((size_t)(N + 63) / 64) + kListSlack;
     const size_t fwd_words = (size_t)((N + 127) / 128) * kItemStride;
     w.off_T = kStatusBytes;
     w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);
     w.off_items = w.off_flags + align256((size_t)((M + kTileT - 1) / kTileT) * 4);
-    w.off_meta = w.off_items + align256((entries * 32 > fwd_words ? entries * 32 : fwd_words) * 4);
+    w.off_meta = w.off_items + align256((entries * 32 * 4 > fwd_words ? entries * 32 * 4 : fwd_words) * 4);
     w.total = w.off_meta + align256(entries * 4);
     return w;
 }
@@ -72,7 +72,8 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     if (st != LOWRA_OK) return st;
     if (!packed || !absmax || !maps || !act || !A || !B || !out || !workspace) return LOWRA_ERR_NULL;
     const int N = layout->N, K = layout->K;
-    if (M < 1 || !rank_ok(r) || N % 8 != 0 || N > 64 * kMaxGroups64) return LOWRA_ERR_SHAPE;
+    if (M < 1 || !rank_ok(r) || N % 8 != 0 || N > 64 * kMaxGroups64 || (uint64_t)N * (uint64_t)(K / 64) >= (1ull << 32))
+        return LOWRA_ERR_SHAPE;
     if (!aligned16(packed) || !aligned16(absmax) || !aligned16(maps) || !aligned16(act) || !aligned16(A) ||
         !aligned16(B) || !aligned16(out))
         return LOWRA_ERR_ALIGN;
@@ -93,6 +94,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     // ---- prologue: clear status and flags, deal the rows
     PrepParams P;
     memset(&P, 0, sizeof(P));
+    P.L = make_row_layout(layout);
     P.precs = layout->precs_dev;
     P.inv_perm = layout->inv_perm_dev;
     P.items = items;

@@ -20,9 +20,10 @@ struct PrepParams {
     // (bits 0-6) | class (bits 7-8, 3 = row past N) | stored position (bits 9-31), all ones for "no row".
     //   forward (group 128): items[g * kItemStride + i] = i-th row of group g in precision order
     //   backward (group 64): per-warp work lists, see deal_backward
+    RowLayout L;
     const uint8_t* precs;
     const int32_t* inv_perm;
-    uint32_t* items;
+    uint32_t* items;      // forward: row words; backward: 16-byte row records of the work-list entries
     uint32_t* heads;      // backward: [7 * ceil(N / 64) + kListSlack] work-list heads
     int N, group;
     uint32_t* status;     // device status word, cleared

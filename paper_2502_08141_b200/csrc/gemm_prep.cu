@@ -60,8 +60,12 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
 // features).  Chunks are numbered through the whole matrix (group after group) and chunk g goes to warp
 // g % kProducerWarps as entry g / kProducerWarps of that warp's work list, so a warp only ever visits the
 // stages it has work on:
-//   heads[e]          = group index (bits 0-23) | number of arrivals this entry owes the stage barrier (bits 24-31)
-//   items[e * 32 + l] = row word of lane l (see deal_rows), all ones for "no row"
+//   heads[e]         = group index (bits 0-23) | arrivals this entry owes the stage barrier (bits 24-27) |
+//                      precision class of the chunk (bits 28-29; 3 = rows past N, to be zero-filled)
+//   rows[e * 32 + l] = what lane l needs to find its row, ready to use (16 bytes):
+//                      x = byte offset of the row in the packed buffer / 16, y = index of the row's first absmax,
+//                      z = index of the row's first level in the maps table, w = channel inside the group
+//                      (all ones: this lane has no row)
 // with e = entry * kProducerWarps + warp.  The stage barrier expects kStageArrivals arrivals; the first chunk
 // of a group also arrives for the chunks the group does not have.  The lists end with an all-ones head.
 __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint32_t* wsum) {
@@ -130,9 +134,14 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
         for (int c = 1; c < 4; ++c) chunk_base[c] = chunk_base[c - 1] + (total_c[c - 1] + 15) / 16;
         const int n_chunks = chunk_base[3] + (total_c[3] + 15) / 16;
         auto entry_of = [&](int ci) { return g0 + (uint32_t)ci; };   // the warps' lists interleave: e = chunk number
-        for (int ci = 0; ci < n_chunks; ++ci) P.items[(size_t)entry_of(ci) * 32 + lane] = 0xFFFFFFFFu;
-        if (lane < n_chunks)
-            P.heads[entry_of(lane)] = (uint32_t)grp | ((uint32_t)(lane == 0 ? kStageArrivals - n_chunks + 1 : 1) << 24);
+        uint4* rows = reinterpret_cast<uint4*>(P.items);
+        for (int ci = 0; ci < n_chunks; ++ci)
+            rows[(size_t)entry_of(ci) * 32 + lane] = make_uint4(0u, 0u, 0u, 0xFFFFFFFFu);
+        if (lane < n_chunks) {
+            const int c = (lane >= chunk_base[1]) + (lane >= chunk_base[2]) + (lane >= chunk_base[3]);   // class of chunk `lane`
+            P.heads[entry_of(lane)] = (uint32_t)grp | ((uint32_t)(lane == 0 ? kStageArrivals - n_chunks + 1 : 1) << 24) |
+                                      ((uint32_t)c << 28);
+        }
         __syncwarp();
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
@@ -140,8 +149,14 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
             for (int c = 0; c < 4; ++c) {
                 if (cls[i] == c) {
                     const int off = i * 32 + lane, row = grp * 64 + off;
-                    const uint32_t p = (c < 3) ? (uint32_t)P.inv_perm[row] : 0u;
-                    const uint32_t word = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
+                    uint4 rec = make_uint4(0u, 0u, 0u, (uint32_t)off);
+                    if (c < 3) {
+                        const uint32_t sp = (uint32_t)P.inv_perm[row];   // stored position
+                        const uint64_t row_bytes = ((uint64_t)P.L.K << c) >> 3;
+                        rec.x = (uint32_t)((P.L.seg_off[c] + (uint64_t)(sp - (uint32_t)P.L.class_start[c]) * row_bytes) >> 4);
+                        rec.y = sp * (uint32_t)P.L.nb;
+                        rec.z = (uint32_t)row * (uint32_t)kTableStride;
+                    }
                     // inside the class the rows are taken round-robin over (row offset mod 8), so that eight
                     // neighbouring lanes hold eight different residues: their 16-byte stores into the swizzled
                     // operand tile then fall into eight different bank groups
@@ -155,9 +170,9 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
                         const int cnt = __popc(mask[0][c] & (0x01010101u << res)) + __popc(mask[1][c] & (0x01010101u << res));
                         pos += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
                     }
-                    uint32_t* dst = P.items + (size_t)entry_of(chunk_base[c] + pos / 16) * 32 + pos % 16;
-                    dst[0] = word;
-                    dst[16] = word;
+                    uint4* dst = rows + (size_t)entry_of(chunk_base[c] + pos / 16) * 32 + pos % 16;
+                    dst[0] = rec;
+                    dst[16] = rec;
                 }
             }
         }

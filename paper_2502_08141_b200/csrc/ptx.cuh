@@ -109,6 +109,8 @@ __device__ __forceinline__ bool flag_wait(const uint32_t* flag, volatile uint32_
     }
 }
 
+__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+
 // Shared-memory word between the warps of a CTA: release store / acquire load.
 __device__ __forceinline__ void st_release_shared(uint32_t* p, uint32_t v) {
     asm volatile("st.release.cta.shared::cta.u32 [%0], %1;" ::"r"(smem_u32(p)), "r"(v) : "memory");
