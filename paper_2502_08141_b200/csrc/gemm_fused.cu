@@ -47,7 +47,9 @@ struct Barriers {
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort;
-    uint32_t free_upto;         // backward: stages 0 .. free_upto - 1 have been found free by the TMA producer
+    uint32_t produced[kStages];        // backward: arrivals of this CTA's dequant warps on the stage being filled
+    uint32_t free_upto[kClusterBwd];   // backward: stages 0 .. free_upto[c] - 1 have been found free by the TMA
+                                       // producer of CTA c of the cluster (every CTA holds a copy of all counters)
 };
 
 // fields of the per-thread row word written by the prologue (see kIdleItem below)
@@ -255,16 +257,23 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     volatile uint32_t* abort_flag = &bars->abort;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? P.tiles_t : 0;
-    const int n_tiles = n_t_tiles + P.tiles_r * P.tiles_t;
+    // Backward: the CTAs of a cluster work on the same weight rows and on neighbouring token tiles, in lock step:
+    // every dequantised weight tile is produced once per cluster and written into the shared memory of all its CTAs.
+    constexpr int CL = (MODE == kModeBackward) ? kClusterBwd : 1;
+    const uint32_t crank = (CL > 1) ? ptx::cluster_ctarank() : 0u;
+    const int first_tile = (int)blockIdx.x / CL, tile_step = (int)gridDim.x / CL;
+    const int super_t = (P.tiles_t + CL - 1) / CL;          // groups of CL token tiles
+    const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? super_t : 0;
+    const int n_tiles = n_t_tiles + P.tiles_r * super_t;    // per cluster
     auto decode_tile = [&](int g) {
         TileInfo t;
         t.is_t = g < n_t_tiles;
         if (t.is_t) {
-            t.rt = 0; t.mt = g; t.blocks = P.main_blocks;
+            t.rt = 0; t.mt = g * CL + (int)crank; t.blocks = P.main_blocks;
         } else {
             const int idx = g - n_t_tiles;
-            t.mt = idx / P.tiles_r; t.rt = idx - t.mt * P.tiles_r; t.blocks = P.main_blocks + P.lora_blocks;
+            const int st = idx / P.tiles_r;
+            t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank; t.blocks = P.main_blocks + P.lora_blocks;
         }
         return t;
     };
@@ -284,7 +293,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         }
         ptx::mbar_init(&bars->drain, 1);
         bars->abort = 0u;
-        bars->free_upto = 0u;
+        for (int c = 0; c < kClusterBwd; ++c) bars->free_upto[c] = 0u;
+        for (int c = 0; c < kStages; ++c) bars->produced[c] = 0u;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmB);
         if (P.lora_blocks > 0) { ptx::prefetch_tensormap(&tmT); ptx::prefetch_tensormap(&tmFt); }
@@ -293,6 +303,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, kTmemCols);
     ptx::tc_fence_before();
     __syncthreads();
+    if (CL > 1) ptx::cluster_sync();   // the peers' barriers and counters exist before anybody touches them
     ptx::tc_fence_after();
     const uint32_t tmem_base = bars->tmem_base;
 
@@ -302,14 +313,18 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // ================================================================== TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x) {
+            for (int g = first_tile; g < n_tiles && !failed; g += tile_step) {
                 const TileInfo t = decode_tile(g);
                 const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
                 for (int kb = 0; kb < t.blocks; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!ptx::mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
-                    if (MODE == kModeBackward) ptx::st_release_shared(&bars->free_upto, it + 1u);
+                    if (MODE == kModeBackward) {   // tell the dequant warps of every CTA of the cluster
+#pragma unroll
+                        for (int c = 0; c < CL; ++c)
+                            ptx::st_relaxed_cluster(ptx::map_to_cta(ptx::smem_u32(&bars->free_upto[crank]), (uint32_t)c), it + 1u);
+                    }
                     unsigned char* a_s = base + s * kSmemStage;
                     unsigned char* b_s = a_s + kSmemA;
                     uint64_t* bar = &bars->full_x[s];
@@ -364,7 +379,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // ================================================================== MMA issuer
         if (lane == 0) {
             uint32_t it = 0, tile_iter = 0;
-            for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x, ++tile_iter) {
+            for (int g = first_tile; g < n_tiles && !failed; g += tile_step, ++tile_iter) {
                 const TileInfo t = decode_tile(g);
                 // forward has a single accumulator, the other modes alternate between two
                 const uint32_t acc = (MODE == kModeForward) ? 0u : (tile_iter & 1u);
@@ -423,7 +438,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         const int et = (warp - kFirstEpilogueWarp) * 32 + lane;
         uint16_t* out16 = reinterpret_cast<uint16_t*>(out_s);
         uint32_t tile_iter = 0;
-        for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x, ++tile_iter) {
+        for (int g = first_tile; g < n_tiles && !failed; g += tile_step, ++tile_iter) {
             const TileInfo t = decode_tile(g);
             const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
             // a T tile writes the down-projected activations [M, rp] (scaled by s); a weight tile writes Y / dX
@@ -508,7 +523,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 uint64_t t_start = 0;
 #pragma unroll 1
                 for (uint32_t spin = 0;; ++spin) {
-                    v = ptx::ld_acquire_shared(&bars->free_upto);
+                    v = ptx::ld_relaxed_cluster(&bars->free_upto[0]);
+#pragma unroll
+                    for (int c = 1; c < CL; ++c) v = min(v, ptx::ld_relaxed_cluster(&bars->free_upto[c]));
                     if (v > it) break;
                     __nanosleep(20);
                     if ((spin & 255u) == 255u) {
@@ -522,7 +539,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             seen_free = v;
             return true;
         };
-        for (int g = blockIdx.x; g < n_tiles && !failed; g += gridDim.x) {
+        for (int g = first_tile; g < n_tiles && !failed; g += tile_step) {
             const TileInfo t = decode_tile(g);
             const int r0 = t.rt * kTileR;
             if (t.is_t && MODE == kModeForward) {
@@ -627,8 +644,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // two-deep ring with static indices so that no load is waited on early.
                 const int half = (lane >> 4) & 1;
                 const int k_first = r0 + 64 * half;
-                const uint32_t* heads = P.heads + pw;                       // entry j of this warp: heads[j * kProducerWarps]
-                const uint4* rows = reinterpret_cast<const uint4*>(P.items) + (size_t)pw * 32 + lane;   // rows[j * kProducerWarps * 32]
+                const int list = pw * CL + (int)crank;                      // this warp's work list among the cluster's
+                const uint32_t* heads = P.heads + list;                     // entry j of this warp: heads[j * kListWarps]
+                const uint4* rows = reinterpret_cast<const uint4*>(P.items) + (size_t)list * 32 + lane;   // rows[j * kListWarps * 32]
                 constexpr uint32_t kEnd = 0xFFFFFFFFu;
                 uint32_t head_cur[2];
                 uint4 rec_cur[2];
@@ -658,8 +676,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // prologue: entries 0 and 1
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
-                    head_cur[u] = __ldg(heads + (size_t)u * kProducerWarps);
-                    rec_cur[u] = __ldg(rows + (size_t)u * kProducerWarps * 32);
+                    head_cur[u] = __ldg(heads + (size_t)u * kListWarps);
+                    rec_cur[u] = __ldg(rows + (size_t)u * kListWarps * 32);
                 }
 #pragma unroll
                 for (int u = 0; u < 2; ++u) fetch(ring[u], lvr[u], head_cur[u], rec_cur[u]);
@@ -673,8 +691,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         const float* mrow = P.maps + rec_cur[u].z;
                         // head and row record of the entry after next (this ring slot's next use) are asked for
                         // now and consumed after this visit; the lists end with kListSlack all-ones heads
-                        head_cur[u] = __ldg(heads + (size_t)(j0 + u + 2) * kProducerWarps);
-                        rec_cur[u] = __ldg(rows + (size_t)(j0 + u + 2) * kProducerWarps * 32);
+                        head_cur[u] = __ldg(heads + (size_t)(j0 + u + 2) * kListWarps);
+                        rec_cur[u] = __ldg(rows + (size_t)(j0 + u + 2) * kListWarps * 32);
                         const uint32_t it = it0 + (head & 0xFFFFFFu);
                         const int s = it % kStages;
                         if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
@@ -685,10 +703,31 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             else if (wcls == 1) dequant_block_2bit(ring[u].lo, lvr[u], ring[u].a, row_addr, col & 7);
                             else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, slut_addr, row_addr, col & 7);
                             else zero_row(row_addr);
-                            ptx::fence_proxy_async_smem();
+                            ptx::fence_proxy_async_smem();   // the tensor core and the copy below read the row
                         }
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[s], (head >> 24) & 15u);
+                        if (lane == 0) {
+                            const uint32_t cnt = (head >> 24) & 15u;
+                            // the warp that completes the operand tile of the stage hands a copy to every peer CTA
+                            const bool last = CL > 1 && ptx::atom_add_acq_rel_shared(&bars->produced[s], cnt) + cnt == (uint32_t)kStageArrivals;
+                            if (last) bars->produced[s] = 0u;   // for the next use of the slot (ordered by the arrival below)
+                            ptx::mbar_arrive_n(&bars->full_w[s], cnt);
+                            if (last) {
+                                // one asynchronous 16 KB copy per peer, counted in bytes on the peer's stage
+                                // barrier, plus the arrivals that barrier expects
+                                ptx::fence_proxy_async_smem();
+                                const uint32_t tile = ptx::smem_u32(base + s * kSmemStage);
+                                const uint32_t bar = ptx::smem_u32(&bars->full_w[s]);
+#pragma unroll
+                                for (int c = 1; c < CL; ++c) {
+                                    const uint32_t peer = (crank + (uint32_t)c) % CL;
+                                    const uint32_t rbar = ptx::map_to_cta(bar, peer);
+                                    ptx::mbar_expect_tx_cluster(rbar, kSmemA);
+                                    ptx::bulk_copy_to_cta(ptx::map_to_cta(tile, peer), tile, kSmemA, rbar);
+                                    ptx::mbar_arrive_cluster(rbar, (uint32_t)kStageArrivals);
+                                }
+                            }
+                        }
                         // refill this ring slot
                         fetch(ring[u], lvr[u], head_cur[u], rec_cur[u]);
                     }
@@ -708,6 +747,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     // ---------------------------------------------------------------------- teardown
     ptx::tc_fence_before();
     __syncthreads();
+    if (CL > 1) ptx::cluster_sync();   // no peer writes into this CTA's shared memory (or arrives on its barriers) any more
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
@@ -717,17 +757,40 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
 template <int MODE>
 static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
                                 const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
+    constexpr int CL = (MODE == kModeBackward) ? kClusterBwd : 1;
     static bool configured = false;
+    static int max_clusters = 0;   // clusters (CL = 1: CTAs) that can be resident at the same time
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = CL;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(kGemmThreads, 1, 1);
+    cfg.dynamicSmemBytes = kGemmSmemBytes;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
     if (!configured) {
         if (cudaFuncSetAttribute(fused_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kGemmSmemBytes) != cudaSuccess)
             return LOWRA_ERR_CUDA;
+        max_clusters = kNumSMs / CL;
+        if (CL > 1) {
+            // the persistent schedule needs every cluster of the grid resident (a tile waits for T of another)
+            cfg.gridDim = dim3(kNumSMs / CL * CL, 1, 1);
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, fused_kernel<MODE>, &cfg) != cudaSuccess || n < 1) return LOWRA_ERR_CUDA;
+            if (n < max_clusters) max_clusters = n;
+        }
         configured = true;
     }
-    const int n_tiles = G.tiles_r * G.tiles_t + ((MODE != kModeDense && G.lora_blocks > 0) ? G.tiles_t : 0);
-    const int grid = n_tiles < kNumSMs ? n_tiles : kNumSMs;
-    fused_kernel<MODE><<<grid, kGemmThreads, kGemmSmemBytes, stream>>>(G, tmB, tmT, tmFt, tmFl);
-    return cudaGetLastError() == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+    const int super_t = (G.tiles_t + CL - 1) / CL;
+    const int n_tiles = G.tiles_r * super_t + ((MODE != kModeDense && G.lora_blocks > 0) ? super_t : 0);
+    const int clusters = n_tiles < max_clusters ? n_tiles : max_clusters;
+    cfg.gridDim = dim3((unsigned)(clusters * CL), 1, 1);
+    if (cudaLaunchKernelEx(&cfg, fused_kernel<MODE>, G, tmB, tmT, tmFt, tmFl) != cudaSuccess) return LOWRA_ERR_CUDA;
+    return LOWRA_OK;
 }
 
 lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,

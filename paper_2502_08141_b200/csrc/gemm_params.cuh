@@ -12,7 +12,9 @@ constexpr int kPrepThreads = 128;
 constexpr int kProducerWarps = 12;            // dequant warps of the main kernel: three per tensor-memory lane quarter
 constexpr int kItemStride = 128;              // forward: entries per group of 128 rows in the deal table
 constexpr int kStageArrivals = 8;             // backward: arrivals a stage barrier expects from the dequant warps (>= 7 chunks)
-constexpr int kListSlack = 48;                // backward: all-ones heads written behind the last work-list entry
+constexpr int kClusterBwd = 2;                // backward: CTAs per cluster; they share every dequantised weight tile
+constexpr int kListWarps = kProducerWarps * kClusterBwd;   // backward: work lists (one per dequant warp of the cluster)
+constexpr int kListSlack = 4 * kProducerWarps;  // backward: all-ones heads written behind the last entry of a CTA's lists
 constexpr int kMaxGroups64 = 8192;            // backward: at most this many groups of 64 output channels (N <= 524288)
 
 struct PrepParams {

@@ -55,24 +55,29 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
 }
 
 // Backward-input: every pipeline stage of the main kernel brings a group of 64 consecutive output channels.
-// The rows of a group are ordered by precision class and cut into chunks of at most 16 rows of one class; a
-// chunk is the work of one dequant warp on one stage (32 lanes = 16 rows x 2 halves of the tile's 128
-// features).  Chunks are numbered through the whole matrix (group after group) and chunk g goes to warp
-// g % kProducerWarps as entry g / kProducerWarps of that warp's work list, so a warp only ever visits the
-// stages it has work on:
+// The CTAs of a cluster take the groups in turn (group g is dequantised by CTA g % kClusterBwd, which then copies
+// the finished operand tile to its peers).  The rows of a group are ordered by precision class and cut into
+// chunks of at most 16 rows of one class; a chunk is the work of one dequant warp on one stage (32 lanes =
+// 16 rows x 2 halves of the tile's 128 features).  The chunks of the groups of one CTA are numbered through the
+// whole matrix and chunk n goes to warp n % kProducerWarps of that CTA as entry n / kProducerWarps of the
+// warp's work list, so a warp only ever visits the stages it has work on:
 //   heads[e]         = group index (bits 0-23) | arrivals this entry owes the stage barrier (bits 24-27) |
 //                      precision class of the chunk (bits 28-29; 3 = rows past N, to be zero-filled)
 //   rows[e * 32 + l] = what lane l needs to find its row, ready to use (16 bytes):
 //                      x = byte offset of the row in the packed buffer / 16, y = index of the row's first absmax,
 //                      z = index of the row's first level in the maps table, w = channel inside the group
 //                      (all ones: this lane has no row)
-// with e = entry * kProducerWarps + warp.  The stage barrier expects kStageArrivals arrivals; the first chunk
-// of a group also arrives for the chunks the group does not have.  The lists end with an all-ones head.
+// with e = entry * kListWarps + warp * kClusterBwd + CTA.  The stage barrier expects kStageArrivals arrivals; the
+// first chunk of a group also arrives for the chunks the group does not have.  Every list ends with all-ones heads.
+__device__ __forceinline__ uint32_t list_slot(uint32_t n, int cta) {
+    return (n / kProducerWarps) * kListWarps + (n % kProducerWarps) * kClusterBwd + (uint32_t)cta;
+}
+
 __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint32_t* wsum) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
     constexpr int kWarps = kPrepThreads / 32;
     const int n_groups = (P.N + 63) / 64;
-    // ---- chunks per group (every block computes all of them: the numbering needs the running sum)
+    // ---- chunks per group (every block computes all of them: the numbering needs the running sums)
     for (int grp = warp; grp < n_groups; grp += kWarps) {
         const int r0 = grp * 64 + lane, r1 = r0 + 32;
         const int c0 = (r0 < P.N) ? (P.precs[r0] >> 1) : 3, c1 = (r1 < P.N) ? (P.precs[r1] >> 1) : 3;
@@ -83,34 +88,37 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
         if (lane == 0) pre[grp] = (uint16_t)n;
     }
     __syncthreads();
-    // ---- exclusive running sum over the groups
-    const int seg = (n_groups + kPrepThreads - 1) / kPrepThreads;
-    const int begin = min(tid * seg, n_groups), end = min(begin + seg, n_groups);
-    uint32_t mine = 0;
-    for (int i = begin; i < end; ++i) mine += pre[i];
-    uint32_t incl = mine;
+    // ---- exclusive running sums, one per CTA of the cluster (over the groups g with g % kClusterBwd == cta)
+    for (int cta = 0; cta < kClusterBwd; ++cta) {
+        const int n_mine = (n_groups - cta + kClusterBwd - 1) / kClusterBwd;   // groups of this CTA
+        const int seg = (n_mine + kPrepThreads - 1) / kPrepThreads;
+        const int begin = min(tid * seg, n_mine), end = min(begin + seg, n_mine);
+        uint32_t mine = 0;
+        for (int i = begin; i < end; ++i) mine += pre[i * kClusterBwd + cta];
+        uint32_t incl = mine;
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) {
-        const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
-        if (lane >= d) incl += v;
-    }
-    if (lane == 31) wsum[warp] = incl;
-    __syncthreads();
-    uint32_t run = incl - mine;
-    uint32_t total = 0;
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += v;
+        }
+        if (lane == 31) wsum[warp] = incl;
+        __syncthreads();
+        uint32_t run = incl - mine;
+        uint32_t total = 0;
 #pragma unroll
-    for (int w2 = 0; w2 < kWarps; ++w2) {
-        if (w2 < warp) run += wsum[w2];
-        total += wsum[w2];
+        for (int w2 = 0; w2 < kWarps; ++w2) {
+            if (w2 < warp) run += wsum[w2];
+            total += wsum[w2];
+        }
+        for (int i = begin; i < end; ++i) {
+            const uint32_t n = pre[i * kClusterBwd + cta];
+            pre[i * kClusterBwd + cta] = (uint16_t)run;
+            run += n;
+        }
+        if (blk == 0)
+            for (int i = tid; i < kListSlack; i += kPrepThreads) P.heads[list_slot(total + (uint32_t)i, cta)] = 0xFFFFFFFFu;
+        __syncthreads();
     }
-    for (int i = begin; i < end; ++i) {
-        const uint32_t n = pre[i];
-        pre[i] = (uint16_t)run;
-        run += n;
-    }
-    __syncthreads();
-    if (blk == 0)
-        for (int i = tid; i < kListSlack; i += kPrepThreads) P.heads[total + i] = 0xFFFFFFFFu;
 
     // ---- the deal proper: one warp per group
     for (int grp = blk * kWarps + warp; grp < n_groups; grp += P.blocks * kWarps) {
@@ -133,7 +141,7 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
 #pragma unroll
         for (int c = 1; c < 4; ++c) chunk_base[c] = chunk_base[c - 1] + (total_c[c - 1] + 15) / 16;
         const int n_chunks = chunk_base[3] + (total_c[3] + 15) / 16;
-        auto entry_of = [&](int ci) { return g0 + (uint32_t)ci; };   // the warps' lists interleave: e = chunk number
+        auto entry_of = [&](int ci) { return list_slot(g0 + (uint32_t)ci, grp % kClusterBwd); };
         uint4* rows = reinterpret_cast<uint4*>(P.items);
         for (int ci = 0; ci < n_chunks; ++ci)
             rows[(size_t)entry_of(ci) * 32 + lane] = make_uint4(0u, 0u, 0u, 0xFFFFFFFFu);
