@@ -47,7 +47,7 @@ struct Barriers {
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort;
-    uint32_t produced[kStages];        // backward: arrivals of this CTA's dequant warps on the stage being filled
+    uint32_t produced[kMaxStagesA];        // backward: arrivals of this CTA's dequant warps on the stage being filled
     uint32_t free_upto[kClusterBwd];   // backward: stages 0 .. free_upto[c] - 1 have been found free by the TMA
                                        // producer of CTA c of the cluster (every CTA holds a copy of all counters)
 };
@@ -261,6 +261,11 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     // every dequantised weight tile is produced once per cluster and written into the shared memory of all its CTAs.
     constexpr int CL = (MODE == kModeBackward) ? kClusterBwd : 1;
     const uint32_t crank = (CL > 1) ? ptx::cluster_ctarank() : 0u;
+    // ring geometry: SA weight-operand slots of 16 KB, then SB token-operand slots of 32 KB
+    constexpr int SA = (MODE == kModeBackward) ? kStagesA_bwd : kStages;
+    constexpr int SB = (MODE == kModeBackward) ? kStagesB_bwd : kStages;
+    auto a_slot = [&](uint32_t it) { return base + (it % SA) * kSmemA; };
+    auto b_slot = [&](uint32_t it) { return base + SA * kSmemA + (it % SB) * kSmemB; };
     const int first_tile = (int)blockIdx.x / CL, tile_step = (int)gridDim.x / CL;
     const int super_t = (P.tiles_t + CL - 1) / CL;          // groups of CL token tiles
     const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? super_t : 0;
@@ -294,7 +299,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         ptx::mbar_init(&bars->drain, 1);
         bars->abort = 0u;
         for (int c = 0; c < kClusterBwd; ++c) bars->free_upto[c] = 0u;
-        for (int c = 0; c < kStages; ++c) bars->produced[c] = 0u;
+        for (int c = 0; c < kMaxStagesA; ++c) bars->produced[c] = 0u;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmB);
         if (P.lora_blocks > 0) { ptx::prefetch_tensormap(&tmT); ptx::prefetch_tensormap(&tmFt); }
@@ -317,16 +322,16 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const TileInfo t = decode_tile(g);
                 const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
                 for (int kb = 0; kb < t.blocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
+                    const int s = it % SB;
+                    const uint32_t ph = (it / SB) & 1u;
                     if (!ptx::mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                     if (MODE == kModeBackward) {   // tell the dequant warps of every CTA of the cluster
 #pragma unroll
                         for (int c = 0; c < CL; ++c)
                             ptx::st_relaxed_cluster(ptx::map_to_cta(ptx::smem_u32(&bars->free_upto[crank]), (uint32_t)c), it + 1u);
                     }
-                    unsigned char* a_s = base + s * kSmemStage;
-                    unsigned char* b_s = a_s + kSmemA;
+                    unsigned char* a_s = a_slot(it);   // free as well: its last readers were the MMAs of stage it - SA
+                    unsigned char* b_s = b_slot(it);
                     uint64_t* bar = &bars->full_x[s];
                     if (t.is_t) {
                         const int c0 = kb * kTileC;
@@ -369,9 +374,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             }
             if (failed) {
                 // let this thread's own copies land before the CTA's shared memory is released
-                for (uint32_t back = 1; back <= (uint32_t)kStages && back <= it; ++back) {
+                for (uint32_t back = 1; back <= (uint32_t)SB && back <= it; ++back) {
                     const uint32_t j = it - back;
-                    ptx::mbar_wait(&bars->full_x[j % kStages], (j / kStages) & 1u, nullptr, 2000000ull);
+                    ptx::mbar_wait(&bars->full_x[j % SB], (j / SB) & 1u, nullptr, 2000000ull);
                 }
             }
         }
@@ -388,16 +393,16 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileT;
                 for (int kb = 0; kb < t.blocks; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
+                    const int s = it % SB;
+                    const uint32_t ph = (it / SB) & 1u;
                     if (!ptx::mbar_wait(&bars->full_x[s], ph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
-                    const int sw = (MODE == kModeForward) ? (int)(it % kWSlots) : s;              // weight slot
-                    const uint32_t phw = (MODE == kModeForward) ? ((it / kWSlots) & 1u) : ph;
+                    const int sw = (MODE == kModeForward) ? (int)(it % kWSlots) : (int)(it % SA);              // weight slot
+                    const uint32_t phw = (MODE == kModeForward) ? ((it / kWSlots) & 1u) : ((it / SA) & 1u);
                     if (MODE != kModeDense)
                         if (!ptx::mbar_wait(&bars->full_w[sw], phw, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                     ptx::tc_fence_after();
-                    const uint32_t a_addr = ptx::smem_u32(base + s * kSmemStage);
-                    const uint64_t bdesc = ptx::umma_desc_k_sw128(a_addr + kSmemA);
+                    const uint32_t a_addr = ptx::smem_u32(a_slot(it));
+                    const uint64_t bdesc = ptx::umma_desc_k_sw128(ptx::smem_u32(b_slot(it)));
                     // which shared-memory operand tiles are MN-major (a contraction index is a 128-byte row of
                     // 64 operand rows): forward - the factor tile of a T tile, fetched from A [K, r];
                     // backward - the dequantised weight tile
@@ -526,7 +531,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     v = ptx::ld_relaxed_cluster(&bars->free_upto[0]);
 #pragma unroll
                     for (int c = 1; c < CL; ++c) v = min(v, ptx::ld_relaxed_cluster(&bars->free_upto[c]));
-                    if (v > it) break;
+                    if (v + (uint32_t)(SA - SB) > it) break;
                     __nanosleep(20);
                     if ((spin & 255u) == 255u) {
                         if (t_start == 0) t_start = ptx::globaltimer_ns();
@@ -535,8 +540,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 }
             }
             v = __shfl_sync(0xffffffffu, v, 0);
-            if (v <= it) return false;
-            seen_free = v;
+            if (v + (uint32_t)(SA - SB) <= it) return false;
+            seen_free = v + (uint32_t)(SA - SB);
             return true;
         };
         for (int g = first_tile; g < n_tiles && !failed; g += tile_step) {
@@ -557,7 +562,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 for (int kb = pw; kb < t.blocks; kb += kProducerWarps) {
                     const uint32_t it = it0 + (uint32_t)kb;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
-                    if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % kStages], kStageArrivals);
+                    if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % SA], kStageArrivals);
                 }
             } else if (MODE == kModeForward) {
                 // ---------------------------------------------------------------- forward
@@ -618,13 +623,13 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             // (the weight ring is deeper than the shared-memory ring: first make sure the tensor
                             // core is done with the previous use of this shared-memory stage, so that the parity
                             // of the "landed" barrier below cannot be mistaken for an older phase)
-                            const int sx = it % kStages;
-                            const uint32_t phx = (it / kStages) & 1u;
+                            const int sx = it % SB;
+                            const uint32_t phx = (it / SB) & 1u;
                             if (!ptx::mbar_wait_warp(&bars->empty[sx], phx ^ 1u, abort_flag, kWaitLimitNs) ||
                                 !ptx::mbar_wait_warp(&bars->full_x[sx], phx, abort_flag, kWaitLimitNs)) {
                                 failed = true; bars->abort = 1u; break;
                             }
-                            produce_lora_tmem(ptx::smem_u32(base + sx * kSmemStage), row_local, taddr);
+                            produce_lora_tmem(ptx::smem_u32(a_slot(it)), row_local, taddr);
                         }
                         ptx::tc_fence_before();
                         __syncwarp();
@@ -694,11 +699,11 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         head_cur[u] = __ldg(heads + (size_t)(j0 + u + 2) * kListWarps);
                         rec_cur[u] = __ldg(rows + (size_t)(j0 + u + 2) * kListWarps * 32);
                         const uint32_t it = it0 + (head & 0xFFFFFFu);
-                        const int s = it % kStages;
+                        const int s = it % SA;
                         if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
                         if (col != kIdleItem) {
                             const int wcls = (int)((head >> 28) & 3u);   // the same for the whole warp
-                            const uint32_t row_addr = ptx::smem_u32(base + s * kSmemStage) + (uint32_t)half * 8192u + col * 128u;
+                            const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)half * 8192u + col * 128u;
                             if (wcls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lvr[u].m0, lvr[u].m1, ring[u].a, row_addr, col & 7);
                             else if (wcls == 1) dequant_block_2bit(ring[u].lo, lvr[u], ring[u].a, row_addr, col & 7);
                             else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, slut_addr, row_addr, col & 7);
@@ -716,7 +721,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                                 // one asynchronous 16 KB copy per peer, counted in bytes on the peer's stage
                                 // barrier, plus the arrivals that barrier expects
                                 ptx::fence_proxy_async_smem();
-                                const uint32_t tile = ptx::smem_u32(base + s * kSmemStage);
+                                const uint32_t tile = ptx::smem_u32(a_slot(it));
                                 const uint32_t bar = ptx::smem_u32(&bars->full_w[s]);
 #pragma unroll
                                 for (int c = 1; c < CL; ++c) {
@@ -736,7 +741,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 for (int kb = P.main_blocks + pw; kb < t.blocks && !failed; kb += kProducerWarps) {
                     const uint32_t it = it0 + (uint32_t)kb;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
-                    if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % kStages], kStageArrivals);
+                    if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % SA], kStageArrivals);
                 }
             }
             it0 += (uint32_t)t.blocks;

@@ -40,7 +40,12 @@ lowra_status launch_prep(const PrepParams& P, cudaStream_t stream);
 constexpr int kTileR = 128;       // rows of the MMA A operand per tile (output channels fwd, input features bwd)
 constexpr int kTileT = 256;       // tokens per tile (MMA N)
 constexpr int kTileC = 64;        // contraction elements per pipeline stage (= one absmax block, = 128 bytes of bf16)
-constexpr int kStages = 4;
+constexpr int kStages = 4;        // token-operand (B) slots = weight-operand (A) slots, forward and dense
+// Backward: the dequant warps (and the copies between the CTAs of a cluster) need to run further ahead of the
+// tensor core than the TMA loads do, so the ring is split: more, smaller weight slots and fewer token slots
+// in the same 192 KB.  A weight slot is free once the MMAs of kStagesA stages earlier are complete.
+constexpr int kStagesA_bwd = 6, kStagesB_bwd = 3;
+constexpr int kMaxStagesA = 6;
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstProducerWarp = 6;
 constexpr int kGemmThreads = 32 * (kFirstProducerWarp + kProducerWarps);
@@ -75,6 +80,7 @@ struct GemmParams {
 constexpr uint32_t kSmemA = kTileR * kTileC * 2;   // 16 KB
 constexpr uint32_t kSmemB = kTileT * kTileC * 2;   // 32 KB
 constexpr uint32_t kSmemStage = kSmemA + kSmemB;
+static_assert(kStagesA_bwd * kSmemA + kStagesB_bwd * kSmemB == kStages * kSmemStage, "both ring layouts fill the same space");
 constexpr uint32_t kSmemOut = 32 * kTileR * 2;     // epilogue staging: 32 tokens x 128 channels bf16
 constexpr uint32_t kSmemLut4 = kProducerWarps * 32 * 16 * 4;  // per dequant lane: 16 scaled bf16 levels (one word each)
 constexpr uint32_t kSmemBarriers = 1024;
