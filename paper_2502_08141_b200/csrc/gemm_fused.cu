@@ -1,13 +1,18 @@
 // Fused dequant + LoRA tensor-core kernel (forward, backward-input, and a dense diagnostic mode).
 //
-// One persistent CTA per SM walks over output tiles of 128 "operand rows" x 256 tokens:
+// Persistent CTAs, one per SM, in clusters of two, walk over output tiles of 128 "operand rows" x 256 tokens:
 //   forward : operand rows = output channels n;  Y^T tile [128 n x 256 m]  = W_hat[n, :] . X[m, :]
 //   backward: operand rows = input features k;   dX^T tile [128 k x 256 m] = W_hat[:, k] . dY[m, :]
-// The 128-row operand (the weights) is the A operand of tcgen05.mma and is produced by twelve dequant warps
-// straight from the packed codes (never from HBM as bf16): into tensor memory in the forward pass (a thread
-// owns one output channel = one TMEM lane for the whole tile), into shared memory (MN-major) in the backward
-// pass, where every stage brings 64 new channels.  The 256-token operand (activations / output gradients)
-// is the B operand and arrives by TMA.  Accumulators live in TMEM.
+// The 128-row operand (the weights) is the A operand of tcgen05.mma.  Twelve dequant warps produce it in shared
+// memory straight from the packed codes (never from HBM as bf16), one 128-byte row per 64-element absmax
+// block: K-major in the forward pass (a thread keeps one output channel for the whole tile), MN-major in the
+// backward pass (every stage brings 64 new channels, dealt to the warps by the prologue).  The two CTAs of a
+// cluster work on the same weight rows and on neighbouring token tiles, in lock step: they take the stages in
+// turn, and the CTA that has dequantised a stage's operand tile sends a copy into its peer's shared memory
+// (one asynchronous 16 KB copy, counted on the peer's stage barrier), so every weight is dequantised once
+// per 512 tokens.  The 256-token operand (activations / output gradients) is the B operand and arrives by
+// TMA.  Shared memory holds six weight slots and three token slots.  Accumulators live in TMEM (two, so the
+// epilogue of a tile overlaps the main loop of the next).
 // The LoRA term is folded into the same accumulator as extra contraction blocks at the end of every
 // tile: the up-projection factor comes by TMA straight from the caller's matrix, the down-projected
 // activations T = s X A (resp. U = s dY B^T) by TMA from the workspace.  T itself is produced by this same
@@ -28,27 +33,18 @@ namespace {
 constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
 constexpr uint32_t kIdesc = ptx::umma_idesc_bf16(kTileR, kTileT);
 constexpr uint32_t kIdescAmn = kIdesc | (1u << 15);   // A operand MN-major
-// Forward keeps the dequantised weights in tensor memory: one 128 x 256 accumulator (columns 0-255) and one
-// 32-column operand slot per pipeline stage behind it.
-constexpr uint32_t kTmemASlots = 256;
-
-// Forward keeps the weight operand in tensor memory, in a ring of its own that is deeper than the
-// shared-memory ring of the token operand, so the dequant warps can run further ahead of the tensor core.
-constexpr int kWSlots = 8;
-constexpr int kTurns = kProducerWarps / 4;   // forward: warps that share a tensor-memory lane quarter and take turns
 
 struct Barriers {
     uint64_t full_x[kStages];   // TMA bytes of a stage have landed
-    uint64_t full_w[kWSlots];   // dequant warps have written (or skipped) a stage (forward: 8 slots, else kStages)
+    uint64_t full_w[kMaxStagesA];   // the weight operand of a stage is complete (dequant warps, or a copy from a peer CTA)
     uint64_t empty[kStages];    // the MMAs reading a shared-memory stage have completed
-    uint64_t empty_w[kWSlots];  // forward: the MMAs reading a tensor-memory weight slot have completed
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
     uint32_t tmem_base;
     uint32_t abort;
-    uint32_t produced[kMaxStagesA];        // backward: arrivals of this CTA's dequant warps on the stage being filled
-    uint32_t free_upto[kClusterBwd];   // backward: stages 0 .. free_upto[c] - 1 have been found free by the TMA
+    uint32_t produced[kMaxStagesA];    // arrivals of this CTA's dequant warps on the stage being filled
+    uint32_t free_upto[kCluster];   // stages 0 .. free_upto[c] - 1 have been found free by the TMA
                                        // producer of CTA c of the cluster (every CTA holds a copy of all counters)
 };
 
@@ -183,53 +179,6 @@ __device__ __noinline__ void zero_row(uint32_t row_addr) {
     for (int t = 0; t < 8; ++t) ptx::st_shared_v4(row_addr + 16u * t, make_uint4(0u, 0u, 0u, 0u));
 }
 
-// ---- tensor-memory operand (forward): thread = operand row = TMEM lane -----------------------------
-// The whole warp writes its 32 lanes x 32 columns (64 bf16 per row) with one tcgen05.st; rows of different
-// precision in the warp take their own branch first (at most two classes meet in a warp, see the deal).
-__device__ __noinline__ void produce_block_tmem(Block blk, int cls, Levels lv, const float* mrow, uint32_t slut_addr,
-                                                uint32_t taddr) {
-    uint32_t o[32];
-    if (cls == 0) {
-        deq64_1bit(blk.lo.x, blk.lo.y, lv.m0, lv.m1, blk.a, o);
-    } else if (cls == 1) {
-        deq64_2bit(blk.lo, lv, blk.a, o);
-    } else if (cls == 2) {
-        Levels16 l16;
-        const float4* m4 = reinterpret_cast<const float4*>(mrow);   // stays in L1 for the whole tile
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            const float4 f = __ldg(m4 + e);
-            l16.v[4 * e] = f.x; l16.v[4 * e + 1] = f.y; l16.v[4 * e + 2] = f.z; l16.v[4 * e + 3] = f.w;
-        }
-        deq64_4bit(blk.lo, blk.hi, blk.a, l16, slut_addr, o);
-    } else {
-#pragma unroll
-        for (int i = 0; i < 32; ++i) o[i] = 0u;
-    }
-    __syncwarp();
-    ptx::tmem_st_32x32(taddr, o);
-    ptx::tmem_st_wait();
-}
-
-// LoRA up-projection factor for the forward pass: the tile [64 ranks][128 channels] lies in shared memory as
-// TMA delivered it from B [r, N] (per 64-channel half: one 128-byte row per rank, 128B swizzle); this lane
-// copies the column of its channel into its tensor-memory row (rank 2i in the low half of word i).
-__device__ __noinline__ void produce_lora_tmem(uint32_t tile_addr, int channel, uint32_t taddr) {
-    const uint32_t col = tile_addr + (uint32_t)(channel >> 6) * 8192u + (uint32_t)(channel & 7) * 2u;
-    const uint32_t chunk = (uint32_t)(channel & 63) >> 3;
-    uint32_t o[32];
-#pragma unroll
-    for (int i = 0; i < 32; ++i) {
-        uint32_t lo, hi;   // ranks 2i and 2i + 1: rows 2i, 2i + 1 of the tile, chunk index swizzled by the row
-        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(col + (uint32_t)(2 * i) * 128u + ((chunk ^ (uint32_t)((2 * i) & 7)) << 4)));
-        asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(col + (uint32_t)(2 * i + 1) * 128u + ((chunk ^ (uint32_t)((2 * i + 1) & 7)) << 4)));
-        o[i] = lo | (hi << 16);
-    }
-    __syncwarp();
-    ptx::tmem_st_32x32(taddr, o);
-    ptx::tmem_st_wait();
-}
-
 // word written by the prologue for every dequant thread and every row group: bits 0-6 row offset inside
 // the group, 7-8 class (0,1,2 = 1,2,4 bits; 3 = row past N, to be zero-filled), 9-31 stored position;
 // all ones = this thread has no row in this group.  All rows of one warp have the same class.
@@ -259,11 +208,11 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Backward: the CTAs of a cluster work on the same weight rows and on neighbouring token tiles, in lock step:
     // every dequantised weight tile is produced once per cluster and written into the shared memory of all its CTAs.
-    constexpr int CL = (MODE == kModeBackward) ? kClusterBwd : 1;
+    constexpr int CL = (MODE == kModeDense) ? 1 : kCluster;
     const uint32_t crank = (CL > 1) ? ptx::cluster_ctarank() : 0u;
     // ring geometry: SA weight-operand slots of 16 KB, then SB token-operand slots of 32 KB
-    constexpr int SA = (MODE == kModeBackward) ? kStagesA_bwd : kStages;
-    constexpr int SB = (MODE == kModeBackward) ? kStagesB_bwd : kStages;
+    constexpr int SA = (MODE == kModeDense) ? kStages : kStagesA;
+    constexpr int SB = (MODE == kModeDense) ? kStages : kStagesB;
     auto a_slot = [&](uint32_t it) { return base + (it % SA) * kSmemA; };
     auto b_slot = [&](uint32_t it) { return base + SA * kSmemA + (it % SB) * kSmemB; };
     const int first_tile = (int)blockIdx.x / CL, tile_step = (int)gridDim.x / CL;
@@ -288,17 +237,14 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             ptx::mbar_init(&bars->full_x[s], 1);
             ptx::mbar_init(&bars->empty[s], 1);
         }
-        for (int s = 0; s < kWSlots; ++s) {
-            ptx::mbar_init(&bars->full_w[s], MODE == kModeForward ? 4 : kStageArrivals);
-            ptx::mbar_init(&bars->empty_w[s], 1);
-        }
+        for (int s = 0; s < kMaxStagesA; ++s) ptx::mbar_init(&bars->full_w[s], kStageArrivals);
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(&bars->tmem_full[a], 1);
             ptx::mbar_init(&bars->tmem_empty[a], 4);
         }
         ptx::mbar_init(&bars->drain, 1);
         bars->abort = 0u;
-        for (int c = 0; c < kClusterBwd; ++c) bars->free_upto[c] = 0u;
+        for (int c = 0; c < kCluster; ++c) bars->free_upto[c] = 0u;
         for (int c = 0; c < kMaxStagesA; ++c) bars->produced[c] = 0u;
         ptx::fence_barrier_init();
         ptx::prefetch_tensormap(&tmB);
@@ -325,7 +271,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     const int s = it % SB;
                     const uint32_t ph = (it / SB) & 1u;
                     if (!ptx::mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
-                    if (MODE == kModeBackward) {   // tell the dequant warps of every CTA of the cluster
+                    if (MODE != kModeDense) {   // tell the dequant warps of every CTA of the cluster
 #pragma unroll
                         for (int c = 0; c < CL; ++c)
                             ptx::st_relaxed_cluster(ptx::map_to_cta(ptx::smem_u32(&bars->free_upto[crank]), (uint32_t)c), it + 1u);
@@ -386,9 +332,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             uint32_t it = 0, tile_iter = 0;
             for (int g = first_tile; g < n_tiles && !failed; g += tile_step, ++tile_iter) {
                 const TileInfo t = decode_tile(g);
-                // forward has a single accumulator, the other modes alternate between two
-                const uint32_t acc = (MODE == kModeForward) ? 0u : (tile_iter & 1u);
-                const uint32_t aph = (MODE == kModeForward) ? (tile_iter & 1u) : ((tile_iter >> 1) & 1u);
+                const uint32_t acc = tile_iter & 1u;            // two accumulators take turns
+                const uint32_t aph = (tile_iter >> 1) & 1u;
                 if (!ptx::mbar_wait(&bars->tmem_empty[acc], aph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileT;
@@ -396,25 +341,19 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     const int s = it % SB;
                     const uint32_t ph = (it / SB) & 1u;
                     if (!ptx::mbar_wait(&bars->full_x[s], ph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
-                    const int sw = (MODE == kModeForward) ? (int)(it % kWSlots) : (int)(it % SA);              // weight slot
-                    const uint32_t phw = (MODE == kModeForward) ? ((it / kWSlots) & 1u) : ((it / SA) & 1u);
+                    const int sw = (int)(it % SA);              // weight slot
+                    const uint32_t phw = (it / SA) & 1u;
                     if (MODE != kModeDense)
                         if (!ptx::mbar_wait(&bars->full_w[sw], phw, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                     ptx::tc_fence_after();
                     const uint32_t a_addr = ptx::smem_u32(a_slot(it));
                     const uint64_t bdesc = ptx::umma_desc_k_sw128(ptx::smem_u32(b_slot(it)));
-                    // which shared-memory operand tiles are MN-major (a contraction index is a 128-byte row of
-                    // 64 operand rows): forward - the factor tile of a T tile, fetched from A [K, r];
+                    // which weight-operand tiles are MN-major (a contraction index is a 128-byte row of 64 operand
+                    // rows): forward - the factor tiles, fetched from A [K, r] (T tiles) and B [r, N] (LoRA blocks);
                     // backward - the dequantised weight tile
                     const bool lora_blk = !t.is_t && kb >= P.main_blocks;
-                    const bool a_mn = (MODE == kModeForward) ? t.is_t : (MODE == kModeBackward && !t.is_t && !lora_blk);
-                    if (MODE == kModeForward && !t.is_t) {
-                        // weights (and the LoRA up-projection rows) come from tensor memory: 8 columns per MMA
-                        const uint32_t a_tmem = tmem_base + kTmemASlots + 32u * (uint32_t)sw;
-#pragma unroll
-                        for (int kk = 0; kk < kTileC / 16; ++kk)
-                            ptx::umma_bf16_ts(d_tmem, a_tmem + 8u * kk, bdesc + 2u * kk, kIdesc, (kb | kk) != 0 ? 1u : 0u);
-                    } else if (a_mn) {
+                    const bool a_mn = (MODE == kModeForward) ? (t.is_t || lora_blk) : (MODE == kModeBackward && !t.is_t && !lora_blk);
+                    if (a_mn) {
                         // 16 contraction rows = two 1024-byte groups per MMA
                         const uint64_t adesc = ptx::umma_desc_mn_sw128(a_addr, 8192u);
 #pragma unroll
@@ -427,7 +366,6 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             ptx::umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, kIdesc, (kb | kk) != 0 ? 1u : 0u);
                     }
                     ptx::umma_commit(&bars->empty[s]);
-                    if (MODE == kModeForward) ptx::umma_commit(&bars->empty_w[sw]);
                 }
                 if (failed) break;
                 ptx::umma_commit(&bars->tmem_full[acc]);
@@ -452,12 +390,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             const int R = t.is_t ? P.rp : P.R;
             const float scale = t.is_t ? P.s : 1.0f;
             const bool vec_ok = (ld % 8) == 0;
-            const uint32_t acc = (MODE == kModeForward) ? 0u : (tile_iter & 1u);
-            const uint32_t aph = (MODE == kModeForward) ? (tile_iter & 1u) : ((tile_iter >> 1) & 1u);
-            // forward weight tiles hold their rows in precision order: this lane's accumulator row belongs to
-            // the channel that the deal put at this position
-            int my_row = q * 32 + lane;
-            if (MODE == kModeForward && !t.is_t) my_row = info_row(__ldg(P.items + (size_t)t.rt * kItemStride + q * 32 + lane));
+            const uint32_t acc = tile_iter & 1u;
+            const uint32_t aph = (tile_iter >> 1) & 1u;
+            const int my_row = q * 32 + lane;
             // the four epilogue warps share named barriers, so they must agree on leaving
             if (!ptx::mbar_wait_warp(&bars->tmem_full[acc], aph, abort_flag, kWaitLimitNs)) bars->abort = 1u;
             ptx::named_barrier_sync(1, 128);
@@ -544,21 +479,34 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             seen_free = v + (uint32_t)(SA - SB);
             return true;
         };
+        // One lane per visit: `cnt` arrivals on the stage's barrier of this CTA.  The warp that completes the
+        // operand tile of the stage (kStageArrivals arrivals in all) hands a copy to every peer CTA of the cluster:
+        // one asynchronous 16 KB copy per peer, counted in bytes on the peer's stage barrier, plus the arrivals
+        // that barrier expects.
+        auto finish_stage = [&](uint32_t it, int s, uint32_t cnt) {
+            const bool last = CL > 1 && ptx::atom_add_acq_rel_shared(&bars->produced[s], cnt) + cnt == (uint32_t)kStageArrivals;
+            if (last) bars->produced[s] = 0u;   // for the next use of the slot (ordered by the arrival below)
+            ptx::mbar_arrive_n(&bars->full_w[s], cnt);
+            if (last) {
+                ptx::fence_proxy_async_smem();
+                const uint32_t tile = ptx::smem_u32(a_slot(it));
+                const uint32_t bar = ptx::smem_u32(&bars->full_w[s]);
+#pragma unroll
+                for (int c = 1; c < CL; ++c) {
+                    const uint32_t peer = (crank + (uint32_t)c) % CL;
+                    const uint32_t rbar = ptx::map_to_cta(bar, peer);
+                    ptx::mbar_expect_tx_cluster(rbar, kSmemA);
+                    ptx::bulk_copy_to_cta(ptx::map_to_cta(tile, peer), tile, kSmemA, rbar);
+                    ptx::mbar_arrive_cluster(rbar, (uint32_t)kStageArrivals);
+                }
+            }
+        };
         for (int g = first_tile; g < n_tiles && !failed; g += tile_step) {
             const TileInfo t = decode_tile(g);
             const int r0 = t.rt * kTileR;
-            if (t.is_t && MODE == kModeForward) {
-                // nothing to dequantise: the warps whose turn it is keep the stage barriers in step
-                for (int kb = pt >> 7; kb < t.blocks; kb += kTurns) {
-                    const uint32_t it = it0 + (uint32_t)kb;
-                    const int s = it % kWSlots;
-                    if (!ptx::mbar_wait_warp(&bars->empty_w[s], ((it / kWSlots) & 1u) ^ 1u, abort_flag, kWaitLimitNs)) {
-                        failed = true; bars->abort = 1u; break;
-                    }
-                    if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
-                }
-            } else if (t.is_t) {
-                // backward: the warps take the stages in turn and arrive for everybody
+            if (t.is_t) {
+                // nothing to dequantise (the operand comes by TMA): the warps take the stages in turn and arrive
+                // for everybody
                 for (int kb = pw; kb < t.blocks; kb += kProducerWarps) {
                     const uint32_t it = it0 + (uint32_t)kb;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
@@ -566,15 +514,16 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 }
             } else if (MODE == kModeForward) {
                 // ---------------------------------------------------------------- forward
-                // thread = one output channel = one tensor-memory lane (rows of the tile in precision order, so
-                // at most two precisions meet in a warp); 64 input features per stage, written with tcgen05.st
-                // into the stage's 32-column operand slot.  The two warps that own a lane quarter take turns.
-                const int q = warp & 3;                              // lane quarter this warp may touch
-                const int turn = pt >> 7;                            // this warp serves the blocks kb with kb % kTurns == turn
+                // The operand tile of a stage is [128 channels][64 input features], K-major: a channel's
+                // 64-element absmax block is one 128-byte row.  The CTAs of the cluster take the stages in turn
+                // (stage kb is produced by CTA kb % CL and copied to the peers); inside the CTA the three groups
+                // of four warps take this CTA's stages in turn, and warp q of a group holds rows 32 q .. 32 q + 31
+                // of the tile in precision order (at most two precisions meet in a warp).  A thread keeps its
+                // channel for the whole tile; the packed codes of its next two blocks are already in registers.
+                const int q = pw & 3, wgrp = pw >> 2;
                 const uint32_t item = __ldg(P.items + (size_t)t.rt * kItemStride + q * 32 + lane);
                 const int cls = info_class(item);
                 const int row_local = info_row(item);
-                const uint32_t lane_addr = tmem_base + ((uint32_t)(q * 32) << 16) + kTmemASlots;
                 Levels lv = {0.f, 0.f, 0.f, 0.f};
                 const uint8_t* bits_ptr = P.packed;
                 const float* absmax_ptr = P.absmax;
@@ -593,51 +542,43 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
                     }
                 }
+                constexpr int kStep = CL * (kProducerWarps / 4);     // distance between two stages of this warp
+                const int kb_first = (int)crank + CL * wgrp;
                 Block ring[2];
                 ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
                 ring[0].a = ring[1].a = 0.0f;
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {   // ring slot u serves this warp's turns number u, u + 2, ...
-                    const int mb = turn + kTurns * u;
+                for (int u = 0; u < 2; ++u) {   // ring slot u serves this warp's visits number u, u + 2, ...
+                    const int mb = kb_first + kStep * u;
                     if (cls < 3 && mb < P.main_blocks)
                         load_block(ring[u], bits_ptr + (size_t)mb * bits_stride, absmax_ptr + mb, cls);
                 }
-                for (int kb0 = turn; kb0 < t.blocks && !failed; kb0 += 2 * kTurns) {
+                for (int kb0 = kb_first; kb0 < P.main_blocks && !failed; kb0 += 2 * kStep) {
 #pragma unroll
                     for (int u = 0; u < 2; ++u) {
-                        const int kb = kb0 + kTurns * u;
-                        if (kb >= t.blocks) break;
+                        const int kb = kb0 + kStep * u;
+                        if (kb >= P.main_blocks) break;
                         const uint32_t it = it0 + (uint32_t)kb;
-                        const int s = it % kWSlots;
-                        const uint32_t ph = (it / kWSlots) & 1u;
-                        if (!ptx::mbar_wait_warp(&bars->empty_w[s], ph ^ 1u, abort_flag, kWaitLimitNs)) {
-                            failed = true; bars->abort = 1u; break;
-                        }
-                        ptx::tc_fence_after();
-                        const uint32_t taddr = lane_addr + 32u * (uint32_t)s;
-                        if (kb < P.main_blocks) {
-                            produce_block_tmem(ring[u], cls, lv, mrow, slut_addr, taddr);
-                        } else {
-                            // LoRA block: the factor tile (channels x 64 ranks, natural channel order) has been
-                            // fetched by TMA into the stage's weight region; copy this lane's channel row
-                            // (the weight ring is deeper than the shared-memory ring: first make sure the tensor
-                            // core is done with the previous use of this shared-memory stage, so that the parity
-                            // of the "landed" barrier below cannot be mistaken for an older phase)
-                            const int sx = it % SB;
-                            const uint32_t phx = (it / SB) & 1u;
-                            if (!ptx::mbar_wait_warp(&bars->empty[sx], phx ^ 1u, abort_flag, kWaitLimitNs) ||
-                                !ptx::mbar_wait_warp(&bars->full_x[sx], phx, abort_flag, kWaitLimitNs)) {
-                                failed = true; bars->abort = 1u; break;
-                            }
-                            produce_lora_tmem(ptx::smem_u32(a_slot(it)), row_local, taddr);
-                        }
-                        ptx::tc_fence_before();
+                        const int s = it % SA;
+                        if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
+                        const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)row_local * 128u;
+                        if (cls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lv.m0, lv.m1, ring[u].a, row_addr, row_local & 7);
+                        else if (cls == 1) dequant_block_2bit(ring[u].lo, lv, ring[u].a, row_addr, row_local & 7);
+                        else if (cls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, slut_addr, row_addr, row_local & 7);
+                        else zero_row(row_addr);
+                        ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
                         __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(&bars->full_w[s]);
-                        const int nb = kb + 2 * kTurns;   // this ring slot's next turn
+                        if (lane == 0) finish_stage(it, s, kStageArrivals / 4);
+                        const int nb = kb + 2 * kStep;   // this ring slot's next visit
                         if (cls < 3 && nb < P.main_blocks)
                             load_block(ring[u], bits_ptr + (size_t)nb * bits_stride, absmax_ptr + nb, cls);
                     }
+                }
+                // LoRA blocks: operands come by TMA; the warps take the stages in turn and arrive for everybody
+                for (int kb = P.main_blocks + pw; kb < t.blocks && !failed; kb += kProducerWarps) {
+                    const uint32_t it = it0 + (uint32_t)kb;
+                    if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
+                    if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % SA], kStageArrivals);
                 }
             } else {
                 // ---------------------------------------------------------------- backward
@@ -711,28 +652,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             ptx::fence_proxy_async_smem();   // the tensor core and the copy below read the row
                         }
                         __syncwarp();
-                        if (lane == 0) {
-                            const uint32_t cnt = (head >> 24) & 15u;
-                            // the warp that completes the operand tile of the stage hands a copy to every peer CTA
-                            const bool last = CL > 1 && ptx::atom_add_acq_rel_shared(&bars->produced[s], cnt) + cnt == (uint32_t)kStageArrivals;
-                            if (last) bars->produced[s] = 0u;   // for the next use of the slot (ordered by the arrival below)
-                            ptx::mbar_arrive_n(&bars->full_w[s], cnt);
-                            if (last) {
-                                // one asynchronous 16 KB copy per peer, counted in bytes on the peer's stage
-                                // barrier, plus the arrivals that barrier expects
-                                ptx::fence_proxy_async_smem();
-                                const uint32_t tile = ptx::smem_u32(a_slot(it));
-                                const uint32_t bar = ptx::smem_u32(&bars->full_w[s]);
-#pragma unroll
-                                for (int c = 1; c < CL; ++c) {
-                                    const uint32_t peer = (crank + (uint32_t)c) % CL;
-                                    const uint32_t rbar = ptx::map_to_cta(bar, peer);
-                                    ptx::mbar_expect_tx_cluster(rbar, kSmemA);
-                                    ptx::bulk_copy_to_cta(ptx::map_to_cta(tile, peer), tile, kSmemA, rbar);
-                                    ptx::mbar_arrive_cluster(rbar, (uint32_t)kStageArrivals);
-                                }
-                            }
-                        }
+                        if (lane == 0) finish_stage(it, s, (head >> 24) & 15u);
                         // refill this ring slot
                         fetch(ring[u], lvr[u], head_cur[u], rec_cur[u]);
                     }
@@ -762,7 +682,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
 template <int MODE>
 static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
                                 const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
-    constexpr int CL = (MODE == kModeBackward) ? kClusterBwd : 1;
+    constexpr int CL = (MODE == kModeDense) ? 1 : kCluster;
     static bool configured = false;
     static int max_clusters = 0;   // clusters (CL = 1: CTAs) that can be resident at the same time
     cudaLaunchConfig_t cfg = {};

@@ -28,12 +28,12 @@ Workspace plan_workspace(int N, int K, int M, int r) {
     w.rp = (r + 63) / 64 * 64;
     // forward: 128 row words per group of 128 channels; backward: at most 7 work-list entries (a head and
     // 32 row records of 16 bytes each) per group of 64 channels, plus the end markers
-    const size_t groups_per_cta = ((size_t)(N + 63) / 64 + kClusterBwd - 1) / kClusterBwd;
-    const size_t entries = kClusterBwd * (7 * groups_per_cta + kListSlack + kProducerWarps);
+    const size_t groups_per_cta = ((size_t)(N + 63) / 64 + kCluster - 1) / kCluster;
+    const size_t entries = kCluster * (7 * groups_per_cta + kListSlack + kProducerWarps);
     const size_t fwd_words = (size_t)((N + 127) / 128) * kItemStride;
     w.off_T = kStatusBytes;
     w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);
-    w.off_items = w.off_flags + align256((size_t)((M + kTileT - 1) / kTileT + kClusterBwd) * 4);
+    w.off_items = w.off_flags + align256((size_t)((M + kTileT - 1) / kTileT + kCluster) * 4);
     w.off_meta = w.off_items + align256((entries * 32 * 4 > fwd_words ? entries * 32 * 4 : fwd_words) * 4);
     w.total = w.off_meta + align256(entries * 4);
     return w;
@@ -104,7 +104,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     P.group = backward ? 64 : 128;
     P.status = status;
     P.flags = flags;
-    P.n_flags = tiles_t + kClusterBwd;   // a cluster's last token tiles may lie past M
+    P.n_flags = tiles_t + kCluster;   // a cluster's last token tiles may lie past M
     P.blocks = ((N + P.group - 1) / P.group + 3) / 4;
     st = launch_prep(P, stream);
     if (st != LOWRA_OK) return st;

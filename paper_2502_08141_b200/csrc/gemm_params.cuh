@@ -12,8 +12,8 @@ constexpr int kPrepThreads = 128;
 constexpr int kProducerWarps = 12;            // dequant warps of the main kernel: three per tensor-memory lane quarter
 constexpr int kItemStride = 128;              // forward: entries per group of 128 rows in the deal table
 constexpr int kStageArrivals = 8;             // backward: arrivals a stage barrier expects from the dequant warps (>= 7 chunks)
-constexpr int kClusterBwd = 2;                // backward: CTAs per cluster; they share every dequantised weight tile
-constexpr int kListWarps = kProducerWarps * kClusterBwd;   // backward: work lists (one per dequant warp of the cluster)
+constexpr int kCluster = 2;                // backward: CTAs per cluster; they share every dequantised weight tile
+constexpr int kListWarps = kProducerWarps * kCluster;   // backward: work lists (one per dequant warp of the cluster)
 constexpr int kListSlack = 4 * kProducerWarps;  // backward: all-ones heads written behind the last entry of a CTA's lists
 constexpr int kMaxGroups64 = 8192;            // backward: at most this many groups of 64 output channels (N <= 524288)
 
@@ -44,7 +44,7 @@ constexpr int kStages = 4;        // token-operand (B) slots = weight-operand (A
 // Backward: the dequant warps (and the copies between the CTAs of a cluster) need to run further ahead of the
 // tensor core than the TMA loads do, so the ring is split: more, smaller weight slots and fewer token slots
 // in the same 192 KB.  A weight slot is free once the MMAs of kStagesA stages earlier are complete.
-constexpr int kStagesA_bwd = 6, kStagesB_bwd = 3;
+constexpr int kStagesA = 6, kStagesB = 3;
 constexpr int kMaxStagesA = 6;
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstProducerWarp = 6;
@@ -80,7 +80,7 @@ struct GemmParams {
 constexpr uint32_t kSmemA = kTileR * kTileC * 2;   // 16 KB
 constexpr uint32_t kSmemB = kTileT * kTileC * 2;   // 32 KB
 constexpr uint32_t kSmemStage = kSmemA + kSmemB;
-static_assert(kStagesA_bwd * kSmemA + kStagesB_bwd * kSmemB == kStages * kSmemStage, "both ring layouts fill the same space");
+static_assert(kStagesA * kSmemA + kStagesB * kSmemB == kStages * kSmemStage, "both ring layouts fill the same space");
 constexpr uint32_t kSmemOut = 32 * kTileR * 2;     // epilogue staging: 32 tokens x 128 channels bf16
 constexpr uint32_t kSmemLut4 = kProducerWarps * 32 * 16 * 4;  // per dequant lane: 16 scaled bf16 levels (one word each)
 constexpr uint32_t kSmemBarriers = 1024;

@@ -55,7 +55,7 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
 }
 
 // Backward-input: every pipeline stage of the main kernel brings a group of 64 consecutive output channels.
-// The CTAs of a cluster take the groups in turn (group g is dequantised by CTA g % kClusterBwd, which then copies
+// The CTAs of a cluster take the groups in turn (group g is dequantised by CTA g % kCluster, which then copies
 // the finished operand tile to its peers).  The rows of a group are ordered by precision class and cut into
 // chunks of at most 16 rows of one class; a chunk is the work of one dequant warp on one stage (32 lanes =
 // 16 rows x 2 halves of the tile's 128 features).  The chunks of the groups of one CTA are numbered through the
@@ -67,10 +67,10 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
 //                      x = byte offset of the row in the packed buffer / 16, y = index of the row's first absmax,
 //                      z = index of the row's first level in the maps table, w = channel inside the group
 //                      (all ones: this lane has no row)
-// with e = entry * kListWarps + warp * kClusterBwd + CTA.  The stage barrier expects kStageArrivals arrivals; the
+// with e = entry * kListWarps + warp * kCluster + CTA.  The stage barrier expects kStageArrivals arrivals; the
 // first chunk of a group also arrives for the chunks the group does not have.  Every list ends with all-ones heads.
 __device__ __forceinline__ uint32_t list_slot(uint32_t n, int cta) {
-    return (n / kProducerWarps) * kListWarps + (n % kProducerWarps) * kClusterBwd + (uint32_t)cta;
+    return (n / kProducerWarps) * kListWarps + (n % kProducerWarps) * kCluster + (uint32_t)cta;
 }
 
 __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint32_t* wsum) {
@@ -88,13 +88,13 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
         if (lane == 0) pre[grp] = (uint16_t)n;
     }
     __syncthreads();
-    // ---- exclusive running sums, one per CTA of the cluster (over the groups g with g % kClusterBwd == cta)
-    for (int cta = 0; cta < kClusterBwd; ++cta) {
-        const int n_mine = (n_groups - cta + kClusterBwd - 1) / kClusterBwd;   // groups of this CTA
+    // ---- exclusive running sums, one per CTA of the cluster (over the groups g with g % kCluster == cta)
+    for (int cta = 0; cta < kCluster; ++cta) {
+        const int n_mine = (n_groups - cta + kCluster - 1) / kCluster;   // groups of this CTA
         const int seg = (n_mine + kPrepThreads - 1) / kPrepThreads;
         const int begin = min(tid * seg, n_mine), end = min(begin + seg, n_mine);
         uint32_t mine = 0;
-        for (int i = begin; i < end; ++i) mine += pre[i * kClusterBwd + cta];
+        for (int i = begin; i < end; ++i) mine += pre[i * kCluster + cta];
         uint32_t incl = mine;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -111,8 +111,8 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
             total += wsum[w2];
         }
         for (int i = begin; i < end; ++i) {
-            const uint32_t n = pre[i * kClusterBwd + cta];
-            pre[i * kClusterBwd + cta] = (uint16_t)run;
+            const uint32_t n = pre[i * kCluster + cta];
+            pre[i * kCluster + cta] = (uint16_t)run;
             run += n;
         }
         if (blk == 0)
@@ -141,7 +141,7 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
 #pragma unroll
         for (int c = 1; c < 4; ++c) chunk_base[c] = chunk_base[c - 1] + (total_c[c - 1] + 15) / 16;
         const int n_chunks = chunk_base[3] + (total_c[3] + 15) / 16;
-        auto entry_of = [&](int ci) { return list_slot(g0 + (uint32_t)ci, grp % kClusterBwd); };
+        auto entry_of = [&](int ci) { return list_slot(g0 + (uint32_t)ci, grp % kCluster); };
         uint4* rows = reinterpret_cast<uint4*>(P.items);
         for (int ci = 0; ci < n_chunks; ++ci)
             rows[(size_t)entry_of(ci) * 32 + lane] = make_uint4(0u, 0u, 0u, 0xFFFFFFFFu);
