@@ -114,16 +114,21 @@ __device__ __forceinline__ void deq64_2bit(const uint4& w, const Levels& lv, flo
 }
 
 // 4 bits.  The 16 levels are scaled by the block's absmax and rounded to bf16 exactly as the decode
-// kernel does, into a per-lane table in shared memory (entry e of lane l at slut[e * 32 + l], so the
-// warp's lookups never collide on a bank); each code is then one shift/mask and one load.
+// kernel does, into a small table; each code is then one shift/mask and one shared-memory load.  The table
+// (16 words) lives in the thread's own 128-byte destination row, which is only written once all 64
+// elements sit in registers.  Entry e of lane l is word (e ^ (l & 15)) + (l & 16) of the row: rows are 128
+// bytes apart, so the 32 lanes of a warp always hit 32 different banks.
 struct Levels16 { float v[16]; };
 __device__ __forceinline__ void deq64_4bit(const uint4& lo, const uint4& hi, float a, const Levels16& lv,
-                                           uint32_t slut_addr, uint32_t (&o)[32]) {
+                                           uint32_t row_addr, uint32_t (&o)[32]) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t lx = (lane & 15u) << 2;               // byte offset xor-ed into every entry's position
+    const uint32_t tab = row_addr + ((lane & 16u) << 2);
 #pragma unroll
     for (int e = 0; e < 16; e += 2) {
         const uint32_t two = pack_bf16x2(__fmul_rn(lv.v[e], a), __fmul_rn(lv.v[e + 1], a));
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(slut_addr + (uint32_t)e * 128u), "r"(two & 0xFFFFu) : "memory");
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(slut_addr + (uint32_t)(e + 1) * 128u), "r"(two >> 16) : "memory");
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(tab + (((uint32_t)e << 2) ^ lx)), "r"(two & 0xFFFFu) : "memory");
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(tab + (((uint32_t)(e + 1) << 2) ^ lx)), "r"(two >> 16) : "memory");
     }
 #pragma unroll
     for (int q = 0; q < 8; ++q) {  // one 32-bit word = 8 elements
@@ -132,10 +137,9 @@ __device__ __forceinline__ void deq64_4bit(const uint4& lo, const uint4& hi, flo
         uint32_t v[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            // byte offset of entry c = (w >> 4j) & 15 is c * 128
-            const uint32_t off = (j == 0) ? ((w << 7) & 0x780u) : (j == 1) ? ((w << 3) & 0x780u)
-                                                                           : ((w >> (j < 2 ? 0 : 4 * j - 7)) & 0x780u);
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[j]) : "r"(slut_addr + off) : "memory");
+            // byte offset of entry c = (w >> 4j) & 15 is (c << 2) ^ lx
+            const uint32_t c4 = (j == 0) ? (w << 2) : (w >> (4 * j - 2));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[j]) : "r"(tab + ((c4 & 0x3Cu) ^ lx)) : "memory");
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) o[4 * q + j] = __byte_perm(v[2 * j], v[2 * j + 1], 0x5410);
@@ -161,8 +165,8 @@ __device__ __noinline__ void dequant_block_2bit(uint4 w, Levels lv, float a, uin
     deq64_2bit(w, lv, a, o);
     store_row(row_addr, swz, o);
 }
-__device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, const float* mrow, uint32_t slut_addr,
-                                                uint32_t row_addr, int swz) {
+__device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, const float* mrow, uint32_t row_addr,
+                                                int swz) {
     Levels16 lv;   // the row's 16 levels (the caller has prefetched the line)
     const float4* m4 = reinterpret_cast<const float4*>(mrow);
 #pragma unroll
@@ -171,7 +175,7 @@ __device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, con
         lv.v[4 * e] = f.x; lv.v[4 * e + 1] = f.y; lv.v[4 * e + 2] = f.z; lv.v[4 * e + 3] = f.w;
     }
     uint32_t o[32];
-    deq64_4bit(lo, hi, a, lv, slut_addr, o);
+    deq64_4bit(lo, hi, a, lv, row_addr, o);
     store_row(row_addr, swz, o);
 }
 __device__ __noinline__ void zero_row(uint32_t row_addr) {
@@ -197,13 +201,15 @@ template <int MODE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmT,
              const __grid_constant__ CUtensorMap tmFt, const __grid_constant__ CUtensorMap tmFl) {
-    extern __shared__ unsigned char smem_raw[];
-    const uint32_t raw_addr = ptx::smem_u32(smem_raw);
-    unsigned char* base = smem_raw + ((1024u - (raw_addr & 1023u)) & 1023u);
-    unsigned char* out_s = base + kStages * kSmemStage;
-    unsigned char* slut_all = out_s + kSmemOut;   // [8 warps][16 entries][32 lanes] u32: scaled 4-bit tables
-    Barriers* bars = reinterpret_cast<Barriers*>(out_s + kSmemOut + kSmemLut4);
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* base = smem_raw;                   // operand ring (the swizzled tiles need 1024-byte alignment)
+    unsigned char* out_s = base + kSmemRing;          // epilogue staging
+    Barriers* bars = reinterpret_cast<Barriers*>(out_s + kSmemOut);
     volatile uint32_t* abort_flag = &bars->abort;
+    if ((ptx::smem_u32(smem_raw) & 1023u) != 0u) {    // never seen; without it the operand descriptors would be wrong
+        if (threadIdx.x == 0) atomicExch(P.status, (uint32_t)LOWRA_ERR_CUDA);
+        return;
+    }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // Backward: the CTAs of a cluster work on the same weight rows and on neighbouring token tiles, in lock step:
@@ -404,30 +410,32 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 uint32_t v[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileT + chunk * 32, v);
                 ptx::tmem_ld_wait();
-                // thread = operand row (channel), v[j] = token j: transpose through shared memory
+                // thread = operand row (channel), v[j] = token j: transposed through shared memory, eight tokens
+                // at a time (8 tokens x 128 channels = 2 KB: every thread then stores one 16-byte piece)
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const uint32_t two = pack_bf16x2(scale * __uint_as_float(v[j]), 0.0f);
-                    out16[j * kTileR + my_row] = (uint16_t)two;
-                }
-                ptx::named_barrier_sync(1, 128);
+                for (int rnd = 0; rnd < 32 / kEpilogueTokens; ++rnd) {
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int idx = i * 128 + et;
-                    const int row = idx >> 4, ch = idx & 15;
-                    const int m = m0 + chunk * 32 + row, n = r0 + ch * 8;
-                    if (m < P.M && n < R) {
-                        const uint4 val = *reinterpret_cast<const uint4*>(out16 + row * kTileR + ch * 8);
-                        uint16_t* dst = out + (size_t)m * ld + n;
-                        if (vec_ok && n + 8 <= R) {
-                            *reinterpret_cast<uint4*>(dst) = val;
-                        } else {
-                            const uint16_t* e = reinterpret_cast<const uint16_t*>(&val);
-                            for (int k = 0; k < 8 && n + k < R; ++k) dst[k] = e[k];
+                    for (int j = 0; j < kEpilogueTokens; ++j) {
+                        const uint32_t two = pack_bf16x2(scale * __uint_as_float(v[rnd * kEpilogueTokens + j]), 0.0f);
+                        out16[j * kTileR + my_row] = (uint16_t)two;
+                    }
+                    ptx::named_barrier_sync(1, 128);
+                    {
+                        const int row = et >> 4, ch = et & 15;
+                        const int m = m0 + chunk * 32 + rnd * kEpilogueTokens + row, n = r0 + ch * 8;
+                        if (m < P.M && n < R) {
+                            const uint4 val = *reinterpret_cast<const uint4*>(out16 + row * kTileR + ch * 8);
+                            uint16_t* dst = out + (size_t)m * ld + n;
+                            if (vec_ok && n + 8 <= R) {
+                                *reinterpret_cast<uint4*>(dst) = val;
+                            } else {
+                                const uint16_t* e = reinterpret_cast<const uint16_t*>(&val);
+                                for (int k = 0; k < 8 && n + k < R; ++k) dst[k] = e[k];
+                            }
                         }
                     }
+                    ptx::named_barrier_sync(1, 128);
                 }
-                ptx::named_barrier_sync(1, 128);
             }
             ptx::tc_fence_before();
             __syncwarp();
@@ -446,8 +454,6 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // ================================================================== dequant producers
         // The prologue has dealt the rows to these warps (see gemm_prep.cu).  Each thread dequantises one
         // 64-element absmax block per visit of a stage.
-        const int pt = threadIdx.x - kFirstProducerWarp * 32;  // 0..255
-        const uint32_t slut_addr = ptx::smem_u32(slut_all) + (uint32_t)((pt >> 5) * 2048 + lane * 4);
         const int K = P.L.K;
         const int pw = warp - kFirstProducerWarp;               // 0 .. kProducerWarps - 1
         uint32_t it0 = 0;                                       // running stage index at the start of the tile
@@ -564,7 +570,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)row_local * 128u;
                         if (cls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lv.m0, lv.m1, ring[u].a, row_addr, row_local & 7);
                         else if (cls == 1) dequant_block_2bit(ring[u].lo, lv, ring[u].a, row_addr, row_local & 7);
-                        else if (cls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, slut_addr, row_addr, row_local & 7);
+                        else if (cls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, row_addr, row_local & 7);
                         else zero_row(row_addr);
                         ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
                         __syncwarp();
@@ -647,7 +653,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)half * 8192u + col * 128u;
                             if (wcls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lvr[u].m0, lvr[u].m1, ring[u].a, row_addr, col & 7);
                             else if (wcls == 1) dequant_block_2bit(ring[u].lo, lvr[u], ring[u].a, row_addr, col & 7);
-                            else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, slut_addr, row_addr, col & 7);
+                            else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, row_addr, col & 7);
                             else zero_row(row_addr);
                             ptx::fence_proxy_async_smem();   // the tensor core and the copy below read the row
                         }

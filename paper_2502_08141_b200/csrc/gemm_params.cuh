@@ -40,11 +40,11 @@ lowra_status launch_prep(const PrepParams& P, cudaStream_t stream);
 constexpr int kTileR = 128;       // rows of the MMA A operand per tile (output channels fwd, input features bwd)
 constexpr int kTileT = 256;       // tokens per tile (MMA N)
 constexpr int kTileC = 64;        // contraction elements per pipeline stage (= one absmax block, = 128 bytes of bf16)
-constexpr int kStages = 4;        // token-operand (B) slots = weight-operand (A) slots, forward and dense
-// Backward: the dequant warps (and the copies between the CTAs of a cluster) need to run further ahead of the
-// tensor core than the TMA loads do, so the ring is split: more, smaller weight slots and fewer token slots
-// in the same 192 KB.  A weight slot is free once the MMAs of kStagesA stages earlier are complete.
-constexpr int kStagesA = 6, kStagesB = 3;
+constexpr int kStages = 4;        // dense diagnostic: four stages of one weight slot + one token slot
+// Forward / backward: the dequant warps (and the copies between the CTAs of a cluster) need to run further ahead
+// of the tensor core than the TMA loads do, so the ring is split: six 16 KB weight slots and four 32 KB token
+// slots.  A weight slot is free once the MMAs of kStagesA stages earlier are complete.
+constexpr int kStagesA = 6, kStagesB = 4;
 constexpr int kMaxStagesA = 6;
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstProducerWarp = 6;
@@ -80,11 +80,15 @@ struct GemmParams {
 constexpr uint32_t kSmemA = kTileR * kTileC * 2;   // 16 KB
 constexpr uint32_t kSmemB = kTileT * kTileC * 2;   // 32 KB
 constexpr uint32_t kSmemStage = kSmemA + kSmemB;
-static_assert(kStagesA * kSmemA + kStagesB * kSmemB == kStages * kSmemStage, "both ring layouts fill the same space");
-constexpr uint32_t kSmemOut = 32 * kTileR * 2;     // epilogue staging: 32 tokens x 128 channels bf16
-constexpr uint32_t kSmemLut4 = kProducerWarps * 32 * 16 * 4;  // per dequant lane: 16 scaled bf16 levels (one word each)
+constexpr uint32_t kSmemRing = kStagesA * kSmemA + kStagesB * kSmemB;   // 224 KB (the dense ring, 192 KB, lies inside)
+static_assert(kStages * kSmemStage <= kSmemRing, "the dense ring fits into the same space");
+constexpr int kEpilogueTokens = 8;                           // tokens per transposition round of the epilogue
+constexpr uint32_t kSmemOut = kEpilogueTokens * kTileR * 2;  // epilogue staging: 8 tokens x 128 channels bf16
 constexpr uint32_t kSmemBarriers = 1024;
-constexpr uint32_t kGemmSmemBytes = 1024 /*alignment slack*/ + kStages * kSmemStage + kSmemOut + kSmemLut4 + kSmemBarriers;
+// no alignment slack: the dynamic shared memory of a kernel without static shared memory starts 1024-byte
+// aligned (checked by the kernel, which the swizzled operand tiles need)
+constexpr uint32_t kGemmSmemBytes = kSmemRing + kSmemOut + kSmemBarriers;
+static_assert(kGemmSmemBytes <= 232448, "227 KB of shared memory per CTA");
 
 lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
                           const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream);
