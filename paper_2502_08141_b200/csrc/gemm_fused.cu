@@ -165,15 +165,29 @@ __device__ __noinline__ void dequant_block_2bit(uint4 w, Levels lv, float a, uin
     deq64_2bit(w, lv, a, o);
     store_row(row_addr, swz, o);
 }
+// The row's 16 fp32 levels come from global memory (backward: the caller has prefetched the line) ...
 __device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, const float* mrow, uint32_t row_addr,
                                                 int swz) {
-    Levels16 lv;   // the row's 16 levels (the caller has prefetched the line)
+    Levels16 lv;
     const float4* m4 = reinterpret_cast<const float4*>(mrow);
 #pragma unroll
     for (int e = 0; e < 4; ++e) {
         const float4 f = __ldg(m4 + e);
         lv.v[4 * e] = f.x; lv.v[4 * e + 1] = f.y; lv.v[4 * e + 2] = f.z; lv.v[4 * e + 3] = f.w;
     }
+    uint32_t o[32];
+    deq64_4bit(lo, hi, a, lv, row_addr, o);
+    store_row(row_addr, swz, o);
+}
+// ... or from shared memory (forward: `tab_addr`, 64 bytes, parked there for the whole tile)
+__device__ __noinline__ void dequant_block_4bit_smem(uint4 lo, uint4 hi, float a, uint32_t tab_addr, uint32_t row_addr, int swz) {
+    Levels16 lv;
+#pragma unroll
+    for (int e = 0; e < 4; ++e)
+        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(lv.v[4 * e]), "=f"(lv.v[4 * e + 1]), "=f"(lv.v[4 * e + 2]), "=f"(lv.v[4 * e + 3])
+                     : "r"(tab_addr + 16u * e)
+                     : "memory");
     uint32_t o[32];
     deq64_4bit(lo, hi, a, lv, row_addr, o);
     store_row(row_addr, swz, o);
@@ -203,7 +217,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
              const __grid_constant__ CUtensorMap tmFt, const __grid_constant__ CUtensorMap tmFl) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* base = smem_raw;                   // operand ring (the swizzled tiles need 1024-byte alignment)
-    unsigned char* out_s = base + kSmemRing;          // epilogue staging
+    unsigned char* out_s = base + kSmemRingMax;       // epilogue staging
     Barriers* bars = reinterpret_cast<Barriers*>(out_s + kSmemOut);
     volatile uint32_t* abort_flag = &bars->abort;
     if ((ptx::smem_u32(smem_raw) & 1023u) != 0u) {    // never seen; without it the operand descriptors would be wrong
@@ -218,7 +232,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     const uint32_t crank = (CL > 1) ? ptx::cluster_ctarank() : 0u;
     // ring geometry: SA weight-operand slots of 16 KB, then SB token-operand slots of 32 KB
     constexpr int SA = (MODE == kModeDense) ? kStages : kStagesA;
-    constexpr int SB = (MODE == kModeDense) ? kStages : kStagesB;
+    constexpr int SB = (MODE == kModeDense) ? kStages : (MODE == kModeForward) ? kStagesB_fwd : kStagesB_bwd;
+    unsigned char* tab_all = base + SA * kSmemA + SB * kSmemB;   // forward: level tables of 4-bit rows, 2 KB per dequant warp
     auto a_slot = [&](uint32_t it) { return base + (it % SA) * kSmemA; };
     auto b_slot = [&](uint32_t it) { return base + SA * kSmemA + (it % SB) * kSmemB; };
     const int first_tile = (int)blockIdx.x / CL, tile_step = (int)gridDim.x / CL;
@@ -456,6 +471,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // 64-element absmax block per visit of a stage.
         const int K = P.L.K;
         const int pw = warp - kFirstProducerWarp;               // 0 .. kProducerWarps - 1
+        const uint32_t tab_lane = ptx::smem_u32(tab_all) + (uint32_t)pw * 2048u + (uint32_t)lane * 64u;   // forward: this lane's level table
         uint32_t it0 = 0;                                       // running stage index at the start of the tile
         // Backward: a warp only visits the stages it has work on, so it can be several ring revolutions behind
         // or ahead of a stage's "empty" barrier, where a parity wait says nothing.  The TMA producer visits every
@@ -546,6 +562,15 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
                     } else if (cls == 1) {
                         lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
+                    } else {
+                        // the 16 levels of a 4-bit row: parked in shared memory for the whole tile (this lane's
+                        // 64 bytes; only this lane reads them)
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float4 f = __ldg(reinterpret_cast<const float4*>(mrow) + e);
+                            ptx::st_shared_v4(tab_lane + 16u * e,
+                                              make_uint4(__float_as_uint(f.x), __float_as_uint(f.y), __float_as_uint(f.z), __float_as_uint(f.w)));
+                        }
                     }
                 }
                 constexpr int kStep = CL * (kProducerWarps / 4);     // distance between two stages of this warp
@@ -570,7 +595,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)row_local * 128u;
                         if (cls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lv.m0, lv.m1, ring[u].a, row_addr, row_local & 7);
                         else if (cls == 1) dequant_block_2bit(ring[u].lo, lv, ring[u].a, row_addr, row_local & 7);
-                        else if (cls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, row_addr, row_local & 7);
+                        else if (cls == 2) dequant_block_4bit_smem(ring[u].lo, ring[u].hi, ring[u].a, tab_lane, row_addr, row_local & 7);
                         else zero_row(row_addr);
                         ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
                         __syncwarp();
