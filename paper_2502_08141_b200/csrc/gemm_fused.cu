@@ -489,7 +489,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
 #pragma unroll
                     for (int c = 1; c < CL; ++c) v = min(v, ptx::ld_relaxed_cluster(&bars->free_upto[c]));
                     if (v + (uint32_t)(SA - SB) > it) break;
-                    __nanosleep(20);
+                    if (MODE == kModeForward || spin > 64u) __nanosleep(20);
                     if ((spin & 255u) == 255u) {
                         if (t_start == 0) t_start = ptx::globaltimer_ns();
                         if (*abort_flag != 0u || ptx::globaltimer_ns() - t_start > kWaitLimitNs) { v = 0; break; }
@@ -672,6 +672,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         rec_cur[u] = __ldg(rows + (size_t)(j0 + u + 2) * kListWarps * 32);
                         const uint32_t it = it0 + (head & 0xFFFFFFu);
                         const int s = it % SA;
+                        if (((head >> 28) & 3u) == 2u && col != kIdleItem) ptx::prefetch_l1(mrow);   // 4-bit: the wait hides the table's way in
                         if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
                         if (col != kIdleItem) {
                             const int wcls = (int)((head >> 28) & 3u);   // the same for the whole warp
