@@ -115,6 +115,7 @@ size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r);
  *   channel order; all row-major.  r in {16, 32, ..., 128}.  X . A is rounded to bf16 once.
  *   workspace_dev: >= lowra_workspace_bytes(layout, M, r) bytes, 256-byte aligned, contents
  *   overwritten.  Calls that share a workspace must not overlap on the device.
+ *   Limits (LOWRA_ERR_SHAPE otherwise): N % 8 == 0, N <= 524288, N * K / 64 < 2^32, M >= 1.
  */
 lowra_status lowra_lora_forward(const lowra_layout* layout, const uint8_t* packed_dev,
                                 const float* absmax_dev, const float* maps_dev, const uint16_t* X_dev,
@@ -155,7 +156,7 @@ lowra_status lowra_device_status(const void* workspace_dev, void* stream);
  *
  *   - Same arguments, results and errors as lowra_lora_forward, without the workspace.  If
  *     lowra_workspace_bytes(layout, M, r) exceeds LOWRA_STATIC_SCRATCH_BYTES the call launches nothing
- *     and returns LOWRA_ERR_LIMIT (for scale: N = K = 8192, M = 8192, r = 64 needs about 1.2 MB).
+ *     and returns LOWRA_ERR_LIMIT (for scale: N = K = 8192, M = 8192, r = 64 needs about 1.6 MB).
  *   - status_out_dev (optional, may be NULL): a device uint32 that receives the device status word
  *     (LOWRA_OK or LOWRA_ERR_TIMEOUT) once the call's kernels have run, since the built-in scratch cannot
  *     be given to lowra_device_status.
