@@ -1,14 +1,22 @@
 // lowra_encode: fp32 weights -> block absmax + packed 1/2/4-bit codes (paper Appendix A.1).
 //
-// HBM-bound on the 4 bytes read per element.  One warp handles 1024 consecutive elements of one
-// stored row: eight 128-bit loads per lane are issued back to back, each group of 128 elements
-// (two absmax blocks) is reduced with warp shuffles, normalised, pushed through a branch-free
-// threshold search held in registers and packed with shuffles into whole 32-bit words.
+// HBM-bound on the 4 bytes read per element, so the kernel has to get by on a handful of instructions per
+// element.  One warp handles 1024 consecutive elements of one stored row.  Each lane issues eight 128-bit
+// streaming loads back to back (coalesced) and parks them in the warp's slice of shared memory; lane l then
+// owns elements 32 l .. 32 l + 31 (half an absmax block), which it reads back as eight 128-bit loads (the
+// 32-element segments are 144 bytes apart, so neither the writes nor the reads collide on a bank).  The block
+// maximum is one shuffle away; codes are accumulated as bit planes of sign bits:
+//   "thresholds <= n" is counted through the sign of n - t (exact: a difference of two floats has the sign of
+//   the exact difference, and equal values give +0, so a value on a threshold takes the upper bucket; n is
+//   first passed through n + 0.0 so that a negative zero cannot come out below a threshold of +0),
+//   1 bit : one subtract and one funnel shift per element,
+//   2 bits: three sign planes (one per threshold; sorted thresholds) combined into the two code planes with
+//           two logic ops per 32 elements, then interleaved,
+//   4 bits: branch-free binary search over the 15 thresholds held in registers.
+// A lane ends up with 4, 8 or 16 packed bytes: the warp writes 128, 256 or 512 contiguous bytes.
 //
-// Bit-exactness with the definition rests on three things: the block maximum is exact in fp32; the
-// reciprocal is the correctly rounded one (__frcp_rn) and the product a separate rounded multiply
-// (__fmul_rn, never fused); the search returns the number of thresholds <= n, which for sorted
-// thresholds is what the branch-free binary search below computes.
+// Bit-exactness with the definition rests on: the block maximum is exact in fp32; the reciprocal is the
+// correctly rounded one (__frcp_rn) and the product a separate rounded multiply (__fmul_rn, never fused).
 #include "lowra_common.cuh"
 
 namespace lowra {
@@ -16,7 +24,7 @@ namespace lowra {
 constexpr int kEncodeThreads = 256;
 constexpr int kEncodeWarps = kEncodeThreads / 32;
 constexpr int kEncodeChunk = 1024;  // elements per warp task
-constexpr int kGroups = kEncodeChunk / 128;
+constexpr int kSegBytes = 144;      // 32 floats + 16 bytes of padding
 
 struct EncodeParams {
     RowLayout L;
@@ -28,30 +36,20 @@ struct EncodeParams {
     uint32_t n_tasks;
 };
 
-template <int B>
-struct Thresholds;
+// sign bit of (n - t) pushed into `plane` from the right: after 32 pushes (elements 31 .. 0) bit i of the
+// plane says "element i is below t"
+__device__ __forceinline__ uint32_t push_below(uint32_t plane, float n, float t) {
+    return __funnelshift_l(__float_as_uint(__fsub_rn(n, t)), plane, 1);
+}
 
-template <>
-struct Thresholds<1> {
-    float t0;
-    __device__ __forceinline__ void load(const float* t) { t0 = __ldg(t); }
-    __device__ __forceinline__ uint32_t code(float n) const { return t0 <= n ? 1u : 0u; }
-};
-
-template <>
-struct Thresholds<2> {
-    float t[3];
-    __device__ __forceinline__ void load(const float* p) {
-#pragma unroll
-        for (int j = 0; j < 3; ++j) t[j] = __ldg(p + j);
-    }
-    __device__ __forceinline__ uint32_t code(float n) const {
-        const bool c1 = t[1] <= n;
-        const float m = c1 ? t[2] : t[0];
-        const bool c0 = m <= n;
-        return (c1 ? 2u : 0u) | (c0 ? 1u : 0u);
-    }
-};
+// bits of x (16 of them) spread to the even positions
+__device__ __forceinline__ uint32_t spread16(uint32_t x) {
+    x = (x | (x << 8)) & 0x00FF00FFu;
+    x = (x | (x << 4)) & 0x0F0F0F0Fu;
+    x = (x | (x << 2)) & 0x33333333u;
+    x = (x | (x << 1)) & 0x55555555u;
+    return x;
+}
 
 // selp keeps the 15 thresholds in registers (a C ternary tree is turned into an indexed local array)
 __device__ __forceinline__ float sel(bool c, float a, float b) {
@@ -60,8 +58,7 @@ __device__ __forceinline__ float sel(bool c, float a, float b) {
     return r;
 }
 
-template <>
-struct Thresholds<4> {
+struct Thresholds4 {
     float t0, t1, t2, t3, t4, t5, t6, t7, t8, t9, t10, t11, t12, t13, t14;
     __device__ __forceinline__ void load(const float* p) {
         const float4 a = __ldg(reinterpret_cast<const float4*>(p));
@@ -71,6 +68,7 @@ struct Thresholds<4> {
         t0 = a.x; t1 = a.y; t2 = a.z; t3 = a.w; t4 = b.x; t5 = b.y; t6 = b.z; t7 = b.w;
         t8 = c.x; t9 = c.y; t10 = c.z; t11 = c.w; t12 = d.x; t13 = d.y; t14 = d.z;
     }
+    // number of thresholds <= n (sorted thresholds): branch-free binary search
     __device__ __forceinline__ uint32_t code(float n) const {
         const bool c3 = t7 <= n;
         const bool c2 = sel(c3, t11, t3) <= n;
@@ -83,65 +81,105 @@ struct Thresholds<4> {
 };
 
 template <int B>
-__device__ __forceinline__ void encode_chunk(const EncodeParams& P, int p, int chunk, int lane) {
+__device__ __forceinline__ void encode_chunk(const EncodeParams& P, int p, int chunk, int lane, unsigned char* stage) {
     constexpr int c = B >> 1;  // class index of B bits
     const int K = P.L.K;
     const int r = __ldg(P.L.perm + p);
     const float* wrow = P.W + (size_t)r * K;
     const int e0 = chunk * kEncodeChunk;
-    int groups = (K - e0) / 128;
-    if (groups > kGroups) groups = kGroups;
+    const int valid = min(K - e0, kEncodeChunk);   // a multiple of 128
 
-    float4 v[kGroups];
+    // ---- coalesced loads, parked in shared memory: element e of the chunk at segment e / 32, offset e % 32
+    float4 v[8];
 #pragma unroll
-    for (int g = 0; g < kGroups; ++g)
-        v[g] = (g < groups) ? ld_stream_f4(wrow + e0 + g * 128 + lane * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int i = 0; i < 8; ++i) {
+        const int e = (i * 32 + lane) * 4;
+        v[i] = (e < valid) ? ld_stream_f4(wrow + e0 + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const float* trow = P.thresholds + (size_t)r * kTableStride;
+    float t0 = 0.f, t1 = 0.f, t2 = 0.f;
+    Thresholds4 t4;
+    if (B == 1) {
+        t0 = __ldg(trow);
+    } else if (B == 2) {
+        t0 = __ldg(trow); t1 = __ldg(trow + 1); t2 = __ldg(trow + 2);
+    } else {
+        t4.load(trow);
+    }
+    __syncwarp();   // the previous task's reads of the stage are over
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int e = (i * 32 + lane) * 4;
+        *reinterpret_cast<float4*>(stage + (e >> 5) * kSegBytes + (e & 31) * 4) = v[i];
+    }
+    __syncwarp();
 
-    Thresholds<B> thr;
-    thr.load(P.thresholds + (size_t)r * kTableStride);
+    // ---- this lane's 32 elements = half an absmax block
+    float x[32];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const float4 f = *reinterpret_cast<const float4*>(stage + lane * kSegBytes + j * 16);
+        x[4 * j] = f.x; x[4 * j + 1] = f.y; x[4 * j + 2] = f.z; x[4 * j + 3] = f.w;
+    }
+    float m = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(x[i]));
+    m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
+    const bool live = lane * 32 < valid;
+    if (live && (lane & 1) == 0) P.absmax[(size_t)p * P.L.nb + (e0 >> 6) + (lane >> 1)] = m;
+    const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
 
     const size_t row_bytes = (size_t)K * B / 8;
-    uint8_t* prow = P.packed + P.L.seg_off[c] + (size_t)(p - P.L.class_start[c]) * row_bytes;
-    float* arow = P.absmax + (size_t)p * P.L.nb;
-
+    uint8_t* dst = P.packed + P.L.seg_off[c] + (size_t)(p - P.L.class_start[c]) * row_bytes +
+                   (size_t)(e0 + lane * 32) * B / 8;
+    if (B == 1) {
+        uint32_t below = 0u;
 #pragma unroll
-    for (int g = 0; g < kGroups; ++g) {
-        if (g < groups) {  // warp-uniform
-            // block maximum over 64 elements = 16 lanes x 4
-            float m = fmaxf(fmaxf(fabsf(v[g].x), fabsf(v[g].y)), fmaxf(fabsf(v[g].z), fabsf(v[g].w)));
+        for (int i = 31; i >= 0; --i) below = push_below(below, __fadd_rn(__fmul_rn(x[i], inv), 0.0f), t0);
+        if (live) *reinterpret_cast<uint32_t*>(dst) = ~below;
+    } else if (B == 2) {
+        uint32_t s0 = 0u, s1 = 0u, s2 = 0u;   // element i is below threshold 0 / 1 / 2
 #pragma unroll
-            for (int d = 8; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
-            if ((lane & 15) == 0) arow[(e0 + g * 128) / kBlock + (lane >> 4)] = m;
-            const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
-            uint32_t piece = thr.code(__fmul_rn(v[g].x, inv));
-            piece |= thr.code(__fmul_rn(v[g].y, inv)) << B;
-            piece |= thr.code(__fmul_rn(v[g].z, inv)) << (2 * B);
-            piece |= thr.code(__fmul_rn(v[g].w, inv)) << (3 * B);
-            // 4*B bits per lane -> whole 32-bit words: 8 / B lanes per word
-            uint32_t word = piece;
-            word |= __shfl_down_sync(0xffffffffu, word, 1) << (4 * B);
-            if constexpr (B <= 2) word |= __shfl_down_sync(0xffffffffu, word, 2) << (8 * B);
-            if constexpr (B <= 1) word |= __shfl_down_sync(0xffffffffu, word, 4) << (16 * B);
-            constexpr int kLanesPerWord = 8 / B;
-            if ((lane % kLanesPerWord) == 0) {
-                uint32_t* dst = reinterpret_cast<uint32_t*>(prow + (size_t)(e0 + g * 128) * B / 8);
-                dst[lane / kLanesPerWord] = word;
-            }
+        for (int i = 31; i >= 0; --i) {
+            const float n = __fadd_rn(__fmul_rn(x[i], inv), 0.0f);
+            s0 = push_below(s0, n, t0);
+            s1 = push_below(s1, n, t1);
+            s2 = push_below(s2, n, t2);
         }
+        // sorted thresholds: code = number of thresholds <= n; high bit = not below t1, low bit = not below t2
+        // (upper half) or not below t0 (lower half)
+        const uint32_t hi = ~s1;
+        const uint32_t lo = (hi & ~s2) | (s1 & ~s0);
+        uint2 w;
+        w.x = spread16(lo & 0xFFFFu) | (spread16(hi & 0xFFFFu) << 1);
+        w.y = spread16(lo >> 16) | (spread16(hi >> 16) << 1);
+        if (live) *reinterpret_cast<uint2*>(dst) = w;
+    } else {
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            uint32_t acc = 0u;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc |= t4.code(__fmul_rn(x[8 * q + i], inv)) << (4 * i);
+            w[q] = acc;
+        }
+        if (live) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
 __global__ void __launch_bounds__(kEncodeThreads) encode_kernel(const EncodeParams P) {
+    __shared__ __align__(16) unsigned char stage_all[kEncodeWarps][32 * kSegBytes];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
+    unsigned char* stage = stage_all[warp];
     const uint32_t stride = gridDim.x * kEncodeWarps;
     for (uint32_t t = blockIdx.x * kEncodeWarps + warp; t < P.n_tasks; t += stride) {
         const int p = t / P.chunks_per_row;
         const int chunk = t - p * P.chunks_per_row;
         const int c = (p >= P.L.class_start[1]) + (p >= P.L.class_start[2]);
-        if (c == 0) encode_chunk<1>(P, p, chunk, lane);
-        else if (c == 1) encode_chunk<2>(P, p, chunk, lane);
-        else encode_chunk<4>(P, p, chunk, lane);
+        if (c == 0) encode_chunk<1>(P, p, chunk, lane, stage);
+        else if (c == 1) encode_chunk<2>(P, p, chunk, lane, stage);
+        else encode_chunk<4>(P, p, chunk, lane, stage);
     }
 }
 
@@ -169,7 +207,7 @@ extern "C" lowra_status lowra_encode(const lowra_layout* layout, const float* W_
     if (tasks > 0xFFFFFFFFull) return LOWRA_ERR_SHAPE;
     P.n_tasks = (uint32_t)tasks;
     const uint64_t blocks_needed = (tasks + kEncodeWarps - 1) / kEncodeWarps;
-    const uint64_t cap = (uint64_t)kNumSMs * 8;
+    const uint64_t cap = (uint64_t)kNumSMs * 3;   // three CTAs (80 registers, 36 KB of shared memory) are resident per SM
     const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
     encode_kernel<<<grid, kEncodeThreads, 0, (cudaStream_t)stream>>>(P);
     return cudaGetLastError() == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
