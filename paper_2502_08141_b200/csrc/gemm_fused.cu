@@ -146,6 +146,24 @@ __device__ __forceinline__ void deq64_4bit(const uint4& lo, const uint4& hi, flo
     }
 }
 
+// 4 bits, forward: the row's 16 fp32 levels sit in shared memory for the whole tile (`tab`, this lane's 64 bytes),
+// so every element is one table load, one multiply and half a convert, and nothing needs the destination row.
+__device__ __forceinline__ void deq64_4bit_direct(const uint4& lo, const uint4& hi, float a, uint32_t tab, uint32_t (&o)[32]) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {  // one 32-bit word = 8 elements
+        const uint32_t w = q == 0 ? lo.x : q == 1 ? lo.y : q == 2 ? lo.z : q == 3 ? lo.w
+                         : q == 4 ? hi.x : q == 5 ? hi.y : q == 6 ? hi.z : hi.w;
+        float f[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t c4 = (j == 0) ? (w << 2) : (w >> (4 * j - 2));   // byte offset of level c = (w >> 4j) & 15
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(f[j]) : "r"(tab + (c4 & 0x3Cu)) : "memory");
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) o[4 * q + j] = pack_bf16x2(__fmul_rn(f[2 * j], a), __fmul_rn(f[2 * j + 1], a));
+    }
+}
+
 // ---- shared-memory operand (backward): the block is one 128-byte row of the swizzled tile ----------
 // Chunk t (elements 8t .. 8t+7) of the row goes to physical 16-byte slot t ^ swz (128B swizzle).
 __device__ __forceinline__ void store_row(uint32_t row_addr, int swz, const uint32_t (&o)[32]) {
@@ -165,7 +183,7 @@ __device__ __noinline__ void dequant_block_2bit(uint4 w, Levels lv, float a, uin
     deq64_2bit(w, lv, a, o);
     store_row(row_addr, swz, o);
 }
-// The row's 16 fp32 levels come from global memory (backward: the caller has prefetched the line) ...
+// The row's 16 fp32 levels come from global memory (the caller has prefetched the line).
 __device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, const float* mrow, uint32_t row_addr,
                                                 int swz) {
     Levels16 lv;
@@ -175,19 +193,6 @@ __device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, con
         const float4 f = __ldg(m4 + e);
         lv.v[4 * e] = f.x; lv.v[4 * e + 1] = f.y; lv.v[4 * e + 2] = f.z; lv.v[4 * e + 3] = f.w;
     }
-    uint32_t o[32];
-    deq64_4bit(lo, hi, a, lv, row_addr, o);
-    store_row(row_addr, swz, o);
-}
-// ... or from shared memory (forward: `tab_addr`, 64 bytes, parked there for the whole tile)
-__device__ __noinline__ void dequant_block_4bit_smem(uint4 lo, uint4 hi, float a, uint32_t tab_addr, uint32_t row_addr, int swz) {
-    Levels16 lv;
-#pragma unroll
-    for (int e = 0; e < 4; ++e)
-        asm volatile("ld.shared.v4.f32 {%0,%1,%2,%3}, [%4];"
-                     : "=f"(lv.v[4 * e]), "=f"(lv.v[4 * e + 1]), "=f"(lv.v[4 * e + 2]), "=f"(lv.v[4 * e + 3])
-                     : "r"(tab_addr + 16u * e)
-                     : "memory");
     uint32_t o[32];
     deq64_4bit(lo, hi, a, lv, row_addr, o);
     store_row(row_addr, swz, o);
@@ -575,35 +580,39 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 }
                 constexpr int kStep = CL * (kProducerWarps / 4);     // distance between two stages of this warp
                 const int kb_first = (int)crank + CL * wgrp;
-                Block ring[2];
-                ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
-                ring[0].a = ring[1].a = 0.0f;
+                // The block is dequantised into registers BEFORE the wait for the stage (the warps wait most of
+                // the time): once the slot is free only the eight 16-byte stores remain on the critical path.
+                Block cur, nxt;   // codes of this visit and of the next one
+                cur.lo = cur.hi = nxt.lo = nxt.hi = make_uint4(0u, 0u, 0u, 0u);
+                cur.a = nxt.a = 0.0f;
+                if (cls < 3 && kb_first < P.main_blocks)
+                    load_block(cur, bits_ptr + (size_t)kb_first * bits_stride, absmax_ptr + kb_first, cls);
+                if (cls < 3 && kb_first + kStep < P.main_blocks)
+                    load_block(nxt, bits_ptr + (size_t)(kb_first + kStep) * bits_stride, absmax_ptr + kb_first + kStep, cls);
+#pragma unroll 1
+                for (int kb = kb_first; kb < P.main_blocks && !failed; kb += kStep) {
+                    uint32_t o[32];
+                    if (cls == 0) {
+                        deq64_1bit(cur.lo.x, cur.lo.y, lv.m0, lv.m1, cur.a, o);
+                    } else if (cls == 1) {
+                        deq64_2bit(cur.lo, lv, cur.a, o);
+                    } else if (cls == 2) {
+                        deq64_4bit_direct(cur.lo, cur.hi, cur.a, tab_lane, o);
+                    } else {
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {   // ring slot u serves this warp's visits number u, u + 2, ...
-                    const int mb = kb_first + kStep * u;
-                    if (cls < 3 && mb < P.main_blocks)
-                        load_block(ring[u], bits_ptr + (size_t)mb * bits_stride, absmax_ptr + mb, cls);
-                }
-                for (int kb0 = kb_first; kb0 < P.main_blocks && !failed; kb0 += 2 * kStep) {
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const int kb = kb0 + kStep * u;
-                        if (kb >= P.main_blocks) break;
-                        const uint32_t it = it0 + (uint32_t)kb;
-                        const int s = it % SA;
-                        if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
-                        const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)row_local * 128u;
-                        if (cls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lv.m0, lv.m1, ring[u].a, row_addr, row_local & 7);
-                        else if (cls == 1) dequant_block_2bit(ring[u].lo, lv, ring[u].a, row_addr, row_local & 7);
-                        else if (cls == 2) dequant_block_4bit_smem(ring[u].lo, ring[u].hi, ring[u].a, tab_lane, row_addr, row_local & 7);
-                        else zero_row(row_addr);
-                        ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
-                        __syncwarp();
-                        if (lane == 0) finish_stage(it, s, kStageArrivals / 4);
-                        const int nb = kb + 2 * kStep;   // this ring slot's next visit
-                        if (cls < 3 && nb < P.main_blocks)
-                            load_block(ring[u], bits_ptr + (size_t)nb * bits_stride, absmax_ptr + nb, cls);
+                        for (int i = 0; i < 32; ++i) o[i] = 0u;
                     }
+                    cur = nxt;
+                    const int nb = kb + 2 * kStep;
+                    if (cls < 3 && nb < P.main_blocks)
+                        load_block(nxt, bits_ptr + (size_t)nb * bits_stride, absmax_ptr + nb, cls);
+                    const uint32_t it = it0 + (uint32_t)kb;
+                    const int s = it % SA;
+                    if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
+                    store_row(ptx::smem_u32(a_slot(it)) + (uint32_t)row_local * 128u, row_local & 7, o);
+                    ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
+                    __syncwarp();
+                    if (lane == 0) finish_stage(it, s, kStageArrivals / 4);
                 }
                 // LoRA blocks: operands come by TMA; the warps take the stages in turn and arrive for everybody
                 for (int kb = P.main_blocks + pw; kb < t.blocks && !failed; kb += kProducerWarps) {
