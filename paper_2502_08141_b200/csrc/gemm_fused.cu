@@ -3,7 +3,7 @@
 // Persistent CTAs, one per SM, in clusters of two, walk over output tiles of 128 "operand rows" x 256 tokens:
 //   forward : operand rows = output channels n;  Y^T tile [128 n x 256 m]  = W_hat[n, :] . X[m, :]
 //   backward: operand rows = input features k;   dX^T tile [128 k x 256 m] = W_hat[:, k] . dY[m, :]
-// The 128-row operand (the weights) is the A operand of tcgen05.mma.  Twelve dequant warps produce it in shared
+// The 128-row operand (the weights) is the A operand of tcgen05.mma.  Eight dequant warps produce it in shared
 // memory straight from the packed codes (never from HBM as bf16), one 128-byte row per 64-element absmax
 // block: K-major in the forward pass (a thread keeps one output channel for the whole tile), MN-major in the
 // backward pass (every stage brings 64 new channels, dealt to the warps by the prologue).  The two CTAs of a
@@ -21,7 +21,7 @@
 // per-token-tile flag, and the TMA producer of a regular tile waits (bounded) for that flag before it
 // fetches T.  All CTAs are co-resident and walk the tiles in increasing order, so the wait cannot deadlock.
 //
-// Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, 6-17 = dequant.
+// Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, 6-13 = dequant.
 // All mbarrier waits are bounded; a wait that runs out sets the status word and every role leaves.
 #include "gemm_params.cuh"
 #include "ptx.cuh"
@@ -172,17 +172,6 @@ __device__ __forceinline__ void store_row(uint32_t row_addr, int swz, const uint
         ptx::st_shared_v4(row_addr + (uint32_t)((t ^ swz) << 4), make_uint4(o[4 * t], o[4 * t + 1], o[4 * t + 2], o[4 * t + 3]));
 }
 
-__device__ __noinline__ void dequant_block_1bit(uint32_t w0, uint32_t w1, float m0, float m1, float a,
-                                                uint32_t row_addr, int swz) {
-    uint32_t o[32];
-    deq64_1bit(w0, w1, m0, m1, a, o);
-    store_row(row_addr, swz, o);
-}
-__device__ __noinline__ void dequant_block_2bit(uint4 w, Levels lv, float a, uint32_t row_addr, int swz) {
-    uint32_t o[32];
-    deq64_2bit(w, lv, a, o);
-    store_row(row_addr, swz, o);
-}
 // The row's 16 fp32 levels come from global memory (the caller has prefetched the line).
 __device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, const float* mrow, uint32_t row_addr,
                                                 int swz) {
@@ -543,7 +532,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // ---------------------------------------------------------------- forward
                 // The operand tile of a stage is [128 channels][64 input features], K-major: a channel's
                 // 64-element absmax block is one 128-byte row.  The CTAs of the cluster take the stages in turn
-                // (stage kb is produced by CTA kb % CL and copied to the peers); inside the CTA the three groups
+                // (stage kb is produced by CTA kb % CL and copied to the peers); inside the CTA the groups
                 // of four warps take this CTA's stages in turn, and warp q of a group holds rows 32 q .. 32 q + 31
                 // of the tile in precision order (at most two precisions meet in a warp).  A thread keeps its
                 // channel for the whole tile; the packed codes of its next two blocks are already in registers.
@@ -634,13 +623,13 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const uint32_t* heads = P.heads + list;                     // entry j of this warp: heads[j * kListWarps]
                 const uint4* rows = reinterpret_cast<const uint4*>(P.items) + (size_t)list * 32 + lane;   // rows[j * kListWarps * 32]
                 constexpr uint32_t kEnd = 0xFFFFFFFFu;
-                uint32_t head_cur[2];
-                uint4 rec_cur[2];
-                Block ring[2];
-                Levels lvr[2];
-                ring[0].lo = ring[0].hi = ring[1].lo = ring[1].hi = make_uint4(0u, 0u, 0u, 0u);
-                ring[0].a = ring[1].a = 0.0f;
-                lvr[0] = lvr[1] = Levels{0.f, 0.f, 0.f, 0.f};
+                // entry of this visit (0) and of the next one (1): head, row record, codes + absmax, 1/2-bit levels
+                uint32_t head0, head1;
+                uint4 rec0, rec1;
+                Block blk0, blk1;
+                Levels lv0 = {0.f, 0.f, 0.f, 0.f}, lv1 = {0.f, 0.f, 0.f, 0.f};
+                blk0.lo = blk0.hi = blk1.lo = blk1.hi = make_uint4(0u, 0u, 0u, 0u);
+                blk0.a = blk1.a = 0.0f;
 
                 // fetch what an entry needs: codes, absmax, 1/2-bit levels (a 4-bit table is only prefetched)
                 auto fetch = [&](Block& blk, Levels& lv, uint32_t head, const uint4& rec) {
@@ -659,44 +648,48 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     }
                 };
 
-                // prologue: entries 0 and 1
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    head_cur[u] = __ldg(heads + (size_t)u * kListWarps);
-                    rec_cur[u] = __ldg(rows + (size_t)u * kListWarps * 32);
-                }
-#pragma unroll
-                for (int u = 0; u < 2; ++u) fetch(ring[u], lvr[u], head_cur[u], rec_cur[u]);
-                bool list_end = false;
-                for (uint32_t j0 = 0; !list_end && !failed; j0 += 2) {
-#pragma unroll
-                    for (int u = 0; u < 2; ++u) {
-                        const uint32_t head = head_cur[u];
-                        if (head == kEnd) { list_end = true; break; }
-                        const uint32_t col = rec_cur[u].w;   // channel inside the stage = K index of the tile
-                        const float* mrow = P.maps + rec_cur[u].z;
-                        // head and row record of the entry after next (this ring slot's next use) are asked for
-                        // now and consumed after this visit; the lists end with kListSlack all-ones heads
-                        head_cur[u] = __ldg(heads + (size_t)(j0 + u + 2) * kListWarps);
-                        rec_cur[u] = __ldg(rows + (size_t)(j0 + u + 2) * kListWarps * 32);
-                        const uint32_t it = it0 + (head & 0xFFFFFFu);
-                        const int s = it % SA;
-                        if (((head >> 28) & 3u) == 2u && col != kIdleItem) ptx::prefetch_l1(mrow);   // 4-bit: the wait hides the table's way in
-                        if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
-                        if (col != kIdleItem) {
-                            const int wcls = (int)((head >> 28) & 3u);   // the same for the whole warp
-                            const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)half * 8192u + col * 128u;
-                            if (wcls == 0) dequant_block_1bit(ring[u].lo.x, ring[u].lo.y, lvr[u].m0, lvr[u].m1, ring[u].a, row_addr, col & 7);
-                            else if (wcls == 1) dequant_block_2bit(ring[u].lo, lvr[u], ring[u].a, row_addr, col & 7);
-                            else if (wcls == 2) dequant_block_4bit(ring[u].lo, ring[u].hi, ring[u].a, mrow, row_addr, col & 7);
-                            else zero_row(row_addr);
-                            ptx::fence_proxy_async_smem();   // the tensor core and the copy below read the row
-                        }
-                        __syncwarp();
-                        if (lane == 0) finish_stage(it, s, (head >> 24) & 15u);
-                        // refill this ring slot
-                        fetch(ring[u], lvr[u], head_cur[u], rec_cur[u]);
+                head0 = __ldg(heads);
+                rec0 = __ldg(rows);
+                head1 = __ldg(heads + kListWarps);
+                rec1 = __ldg(rows + (size_t)kListWarps * 32);
+                fetch(blk0, lv0, head0, rec0);
+                fetch(blk1, lv1, head1, rec1);
+#pragma unroll 1
+                for (uint32_t j = 0; !failed; ++j) {
+                    const uint32_t head = head0;
+                    if (head == kEnd) break;
+                    const uint32_t col = rec0.w;   // channel inside the stage = K index of the tile
+                    const float* mrow = P.maps + rec0.z;
+                    const int wcls = (int)((head >> 28) & 3u);   // the same for the whole warp
+                    // head and row record of the entry after next are asked for now and consumed after this visit;
+                    // the lists end with kListSlack all-ones heads
+                    const uint32_t head2 = __ldg(heads + (size_t)(j + 2) * kListWarps);
+                    const uint4 rec2 = __ldg(rows + (size_t)(j + 2) * kListWarps * 32);
+                    // 1- and 2-bit blocks are dequantised into registers BEFORE the wait for the stage, so that only
+                    // the eight 16-byte stores remain once the slot is free; a 4-bit block builds its table in the
+                    // destination row and has to wait for it
+                    uint32_t o[32];
+                    if (col != kIdleItem) {
+                        if (wcls == 0) deq64_1bit(blk0.lo.x, blk0.lo.y, lv0.m0, lv0.m1, blk0.a, o);
+                        else if (wcls == 1) deq64_2bit(blk0.lo, lv0, blk0.a, o);
+                        else if (wcls == 2) ptx::prefetch_l1(mrow);
                     }
+                    const uint32_t it = it0 + (head & 0xFFFFFFu);
+                    const int s = it % SA;
+                    if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
+                    if (col != kIdleItem) {
+                        const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)half * 8192u + col * 128u;
+                        if (wcls <= 1) store_row(row_addr, col & 7, o);
+                        else if (wcls == 2) dequant_block_4bit(blk0.lo, blk0.hi, blk0.a, mrow, row_addr, col & 7);
+                        else zero_row(row_addr);
+                        ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
+                    }
+                    __syncwarp();
+                    if (lane == 0) finish_stage(it, s, (head >> 24) & 15u);
+                    // shift, and fetch the data of the entry after next
+                    head0 = head1; rec0 = rec1; blk0 = blk1; lv0 = lv1;
+                    head1 = head2; rec1 = rec2;
+                    fetch(blk1, lv1, head1, rec1);
                 }
                 // LoRA blocks: operands come by TMA; the warps take the stages in turn and arrive for everybody
                 for (int kb = P.main_blocks + pw; kb < t.blocks && !failed; kb += kProducerWarps) {

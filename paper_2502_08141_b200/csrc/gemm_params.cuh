@@ -9,7 +9,8 @@ namespace lowra {
 
 // ---- prologue ------------------------------------------------------------------------------
 constexpr int kPrepThreads = 128;
-constexpr int kProducerWarps = 12;            // dequant warps of the main kernel: three per tensor-memory lane quarter
+constexpr int kProducerWarps = 8;             // dequant warps of the main kernel (14 warps in all: at most four per
+                                              // scheduler, so every thread may hold 128 registers)
 constexpr int kItemStride = 128;              // forward: entries per group of 128 rows in the deal table
 constexpr int kStageArrivals = 8;             // backward: arrivals a stage barrier expects from the dequant warps (>= 7 chunks)
 constexpr int kCluster = 2;                // backward: CTAs per cluster; they share every dequantised weight tile
