@@ -10,9 +10,9 @@ namespace lowra {
 namespace {
 
 // Forward: one warp per group of 128 consecutive output channels (one weight tile of the main kernel).  The
-// rows are ordered by precision class (1 bit, 2 bits, 4 bits, rows past N; stable); entry i of the group is the
-// i-th row in that order = the row held by tensor-memory lane i of the main kernel, so that at most two
-// precisions meet in a warp (32 consecutive lanes).
+// rows are ordered by precision class (1 bit, 2 bits, 4 bits, rows past N); entry i of the group is the i-th row
+// in that order = the row held by lane i % 32 of warp i / 32 of a dequant group of the main kernel, so that at
+// most two precisions meet in a warp.
 __device__ void deal_rows(const PrepParams& P, int blk) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     constexpr int G = 128, per = G / 32;
@@ -36,20 +36,33 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
         class_base[0] = 0;
 #pragma unroll
         for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total[c - 1];
-        int before[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int i = 0; i < per; ++i) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 if (cls[i] == c) {
-                    const int q = before[c] + __popc(mask[i][c] & ((1u << lane) - 1u));  // rank inside the class
+                    // inside the class the rows are taken round-robin over (row offset mod 8), so that eight
+                    // neighbouring lanes hold eight different residues: their 16-byte stores into the swizzled
+                    // operand tile then fall into eight different bank groups
+                    const unsigned res_mask = 0x01010101u << (lane & 7);
+                    int b = 0;   // rank of this row among the rows of its class with the same residue
+#pragma unroll
+                    for (int i2 = 0; i2 < per; ++i2)
+                        if (i2 < i) b += __popc(mask[i2][c] & res_mask);
+                    b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
+                    int q = 0;   // rows of the class taken before this one
+#pragma unroll
+                    for (int res = 0; res < 8; ++res) {
+                        int cnt = 0;
+#pragma unroll
+                        for (int i2 = 0; i2 < per; ++i2) cnt += __popc(mask[i2][c] & (0x01010101u << res));
+                        q += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
+                    }
                     const int off = i * 32 + lane, row = grp * G + off;
                     const uint32_t p = (c < 3) ? (uint32_t)P.inv_perm[row] : 0u;
                     out[class_base[c] + q] = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
                 }
             }
-#pragma unroll
-            for (int c = 0; c < 4; ++c) before[c] += __popc(mask[i][c]);
         }
     }
 }
