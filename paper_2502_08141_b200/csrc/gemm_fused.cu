@@ -225,7 +225,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     constexpr int CL = (MODE == kModeDense) ? 1 : kCluster;
     const uint32_t crank = (CL > 1) ? ptx::cluster_ctarank() : 0u;
     // ring geometry: SA weight-operand slots of 16 KB, then SB token-operand slots of 32 KB
-    constexpr int SA = (MODE == kModeDense) ? kStages : kStagesA;
+    constexpr int SA = (MODE == kModeDense) ? kStages : (MODE == kModeForward) ? kStagesA_fwd : kStagesA_bwd;
     constexpr int SB = (MODE == kModeDense) ? kStages : (MODE == kModeForward) ? kStagesB_fwd : kStagesB_bwd;
     unsigned char* tab_all = base + SA * kSmemA + SB * kSmemB;   // forward: level tables of 4-bit rows, 2 KB per dequant warp
     auto a_slot = [&](uint32_t it) { return base + (it % SA) * kSmemA; };
