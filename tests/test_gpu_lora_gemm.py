@@ -54,6 +54,8 @@ GEMM_CASES = [
     (200, 256, 64, 16, {1: 0.34, 2: 0.33, 4: 0.33}, "llama"),       # N not a multiple of 64
     (640, 1152, 515, 96, {1: 0.6, 2: 0.35, 4: 0.05}, "llama"),      # rank above 64, several tiles each way
     (384, 256, 257, 128, {4: 1.0}, "llama"),                        # 4-bit only, maximum rank
+    (320, 640, 770, 48, {1: 0.5, 2: 0.3, 4: 0.2}, "llama"),         # odd number of 64-channel groups (the CTAs of a
+                                                                    # cluster take them in turn), four token tiles
     (4096, 4096, 2048, 64, {1: 0.3, 2: 0.5, 4: 0.2}, "llama"),      # config 2
 ]
 
