@@ -271,6 +271,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     __syncthreads();
     if (CL > 1) ptx::cluster_sync();   // the peers' barriers and counters exist before anybody touches them
     ptx::tc_fence_after();
+    // Everything above overlapped the prologue kernel (programmatic dependent launch); what follows reads what
+    // that kernel wrote (row deal, cleared flags and status word).
+    if (MODE != kModeDense) ptx::grid_dependency_wait();
     const uint32_t tmem_base = bars->tmem_base;
 
     bool failed = false;
@@ -728,16 +731,20 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
     static bool configured = false;
     static int max_clusters = 0;   // clusters (CL = 1: CTAs) that can be resident at the same time
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = CL;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    // start while the prologue kernel (the previous launch in the stream) is still running; the kernel waits for
+    // it before it reads anything that kernel writes
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(kGemmThreads, 1, 1);
     cfg.dynamicSmemBytes = kGemmSmemBytes;
     cfg.stream = stream;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = (MODE == kModeDense) ? 1 : 2;
     if (!configured) {
         if (cudaFuncSetAttribute(fused_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kGemmSmemBytes) != cudaSuccess)

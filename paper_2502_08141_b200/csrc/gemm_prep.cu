@@ -204,6 +204,7 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
 }  // namespace
 
 __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const PrepParams P) {
+    ptx::grid_launch_dependents();   // the fused kernel may set itself up meanwhile; it waits for this grid before reading
     if (blockIdx.x == 0) {
         if (threadIdx.x == 0) *P.status = 0u;
         for (int i = threadIdx.x; i < P.n_flags; i += kPrepThreads) P.flags[i] = 0u;
