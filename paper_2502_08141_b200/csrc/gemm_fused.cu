@@ -113,41 +113,10 @@ __device__ __forceinline__ void deq64_2bit(const uint4& w, const Levels& lv, flo
     }
 }
 
-// 4 bits.  The 16 levels are scaled by the block's absmax and rounded to bf16 exactly as the decode
-// kernel does, into a small table; each code is then one shift/mask and one shared-memory load.  The table
-// (16 words) lives in the thread's own 128-byte destination row, which is only written once all 64
-// elements sit in registers.  Entry e of lane l is word (e ^ (l & 15)) + (l & 16) of the row: rows are 128
-// bytes apart, so the 32 lanes of a warp always hit 32 different banks.
-struct Levels16 { float v[16]; };
-__device__ __forceinline__ void deq64_4bit(const uint4& lo, const uint4& hi, float a, const Levels16& lv,
-                                           uint32_t row_addr, uint32_t (&o)[32]) {
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t lx = (lane & 15u) << 2;               // byte offset xor-ed into every entry's position
-    const uint32_t tab = row_addr + ((lane & 16u) << 2);
-#pragma unroll
-    for (int e = 0; e < 16; e += 2) {
-        const uint32_t two = pack_bf16x2(__fmul_rn(lv.v[e], a), __fmul_rn(lv.v[e + 1], a));
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(tab + (((uint32_t)e << 2) ^ lx)), "r"(two & 0xFFFFu) : "memory");
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(tab + (((uint32_t)(e + 1) << 2) ^ lx)), "r"(two >> 16) : "memory");
-    }
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {  // one 32-bit word = 8 elements
-        const uint32_t w = q == 0 ? lo.x : q == 1 ? lo.y : q == 2 ? lo.z : q == 3 ? lo.w
-                         : q == 4 ? hi.x : q == 5 ? hi.y : q == 6 ? hi.z : hi.w;
-        uint32_t v[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            // byte offset of entry c = (w >> 4j) & 15 is (c << 2) ^ lx
-            const uint32_t c4 = (j == 0) ? (w << 2) : (w >> (4 * j - 2));
-            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v[j]) : "r"(tab + ((c4 & 0x3Cu) ^ lx)) : "memory");
-        }
-#pragma unroll
-        for (int j = 0; j < 4; ++j) o[4 * q + j] = __byte_perm(v[2 * j], v[2 * j + 1], 0x5410);
-    }
-}
 
-// 4 bits, forward: the row's 16 fp32 levels sit in shared memory for the whole tile (`tab`, this lane's 64 bytes),
-// so every element is one table load, one multiply and half a convert, and nothing needs the destination row.
+// 4 bits: the row's 16 fp32 levels sit in shared memory (`tab`, 64 bytes: parked there for the whole tile in the
+// forward pass, fetched asynchronously two visits ahead in the backward pass), so every element is one table
+// load, one multiply and half a convert - rounded exactly as the decode kernel does.
 __device__ __forceinline__ void deq64_4bit_direct(const uint4& lo, const uint4& hi, float a, uint32_t tab, uint32_t (&o)[32]) {
 #pragma unroll
     for (int q = 0; q < 8; ++q) {  // one 32-bit word = 8 elements
@@ -172,20 +141,6 @@ __device__ __forceinline__ void store_row(uint32_t row_addr, int swz, const uint
         ptx::st_shared_v4(row_addr + (uint32_t)((t ^ swz) << 4), make_uint4(o[4 * t], o[4 * t + 1], o[4 * t + 2], o[4 * t + 3]));
 }
 
-// The row's 16 fp32 levels come from global memory (the caller has prefetched the line).
-__device__ __noinline__ void dequant_block_4bit(uint4 lo, uint4 hi, float a, const float* mrow, uint32_t row_addr,
-                                                int swz) {
-    Levels16 lv;
-    const float4* m4 = reinterpret_cast<const float4*>(mrow);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const float4 f = __ldg(m4 + e);
-        lv.v[4 * e] = f.x; lv.v[4 * e + 1] = f.y; lv.v[4 * e + 2] = f.z; lv.v[4 * e + 3] = f.w;
-    }
-    uint32_t o[32];
-    deq64_4bit(lo, hi, a, lv, row_addr, o);
-    store_row(row_addr, swz, o);
-}
 __device__ __noinline__ void zero_row(uint32_t row_addr) {
 #pragma unroll
     for (int t = 0; t < 8; ++t) ptx::st_shared_v4(row_addr + 16u * t, make_uint4(0u, 0u, 0u, 0u));
@@ -227,7 +182,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     // ring geometry: SA weight-operand slots of 16 KB, then SB token-operand slots of 32 KB
     constexpr int SA = (MODE == kModeDense) ? kStages : (MODE == kModeForward) ? kStagesA_fwd : kStagesA_bwd;
     constexpr int SB = (MODE == kModeDense) ? kStages : (MODE == kModeForward) ? kStagesB_fwd : kStagesB_bwd;
-    unsigned char* tab_all = base + SA * kSmemA + SB * kSmemB;   // forward: level tables of 4-bit rows, 2 KB per dequant warp
+    unsigned char* tab_all = base + SA * kSmemA + SB * kSmemB;   // level tables of 4-bit rows, 2 KB per dequant warp
     auto a_slot = [&](uint32_t it) { return base + (it % SA) * kSmemA; };
     auto b_slot = [&](uint32_t it) { return base + SA * kSmemA + (it % SB) * kSmemB; };
     const int first_tile = (int)blockIdx.x / CL, tile_step = (int)gridDim.x / CL;
@@ -476,7 +431,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // 64-element absmax block per visit of a stage.
         const int K = P.L.K;
         const int pw = warp - kFirstProducerWarp;               // 0 .. kProducerWarps - 1
-        const uint32_t tab_lane = ptx::smem_u32(tab_all) + (uint32_t)pw * 2048u + (uint32_t)lane * 64u;   // forward: this lane's level table
+        const uint32_t tab_warp = ptx::smem_u32(tab_all) + (uint32_t)pw * 2048u;   // this warp's 2 KB of level tables (4-bit rows)
+        const uint32_t tab_lane = tab_warp + (uint32_t)lane * 64u;                  // forward: this lane's table
         uint32_t it0 = 0;                                       // running stage index at the start of the tile
         // Backward: a warp only visits the stages it has work on, so it can be several ring revolutions behind
         // or ahead of a stage's "empty" barrier, where a parity wait says nothing.  The TMA producer visits every
@@ -642,8 +598,10 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 blk0.lo = blk0.hi = blk1.lo = blk1.hi = make_uint4(0u, 0u, 0u, 0u);
                 blk0.a = blk1.a = 0.0f;
 
-                // fetch what an entry needs: codes, absmax, 1/2-bit levels (a 4-bit table is only prefetched)
-                auto fetch = [&](Block& blk, Levels& lv, uint32_t head, const uint4& rec) {
+                // fetch what an entry needs: codes, absmax, 1/2-bit levels in registers; the 16 fp32 levels of a 4-bit
+                // row travel asynchronously into this warp's table cache (two slots of 16 rows x 64 bytes, one per
+                // entry in flight; the two lanes of a row read the same 64 bytes)
+                auto fetch = [&](Block& blk, Levels& lv, uint32_t head, const uint4& rec, uint32_t tab_slot) {
                     const int cls = (head == kEnd || rec.w == kIdleItem) ? 4 : (int)((head >> 28) & 3u);
                     if (cls < 3) {
                         load_block(blk, P.packed + ((size_t)rec.x << 4) + (((size_t)k_first << cls) >> 3),
@@ -653,45 +611,49 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
                         } else if (cls == 1) {
                             lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
-                        } else {
-                            ptx::prefetch_l1(mrow);
+                        } else if (lane < 16) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) ptx::cp_async_16(tab_slot + (uint32_t)lane * 64u + 16u * e, mrow + 4 * e, true);
                         }
                     }
+                    ptx::cp_async_commit();   // one group per entry, empty or not
                 };
 
                 head0 = __ldg(heads);
                 rec0 = __ldg(rows);
                 head1 = __ldg(heads + kListWarps);
                 rec1 = __ldg(rows + (size_t)kListWarps * 32);
-                fetch(blk0, lv0, head0, rec0);
-                fetch(blk1, lv1, head1, rec1);
+                fetch(blk0, lv0, head0, rec0, tab_warp);
+                fetch(blk1, lv1, head1, rec1, tab_warp + 1024u);
 #pragma unroll 1
                 for (uint32_t j = 0; !failed; ++j) {
                     const uint32_t head = head0;
                     if (head == kEnd) break;
                     const uint32_t col = rec0.w;   // channel inside the stage = K index of the tile
-                    const float* mrow = P.maps + rec0.z;
                     const int wcls = (int)((head >> 28) & 3u);   // the same for the whole warp
                     // head and row record of the entry after next are asked for now and consumed after this visit;
                     // the lists end with kListSlack all-ones heads
                     const uint32_t head2 = __ldg(heads + (size_t)(j + 2) * kListWarps);
                     const uint4 rec2 = __ldg(rows + (size_t)(j + 2) * kListWarps * 32);
-                    // 1- and 2-bit blocks are dequantised into registers BEFORE the wait for the stage, so that only
-                    // the eight 16-byte stores remain once the slot is free; a 4-bit block builds its table in the
-                    // destination row and has to wait for it
+                    // the block is dequantised into registers BEFORE the wait for the stage, so that only the eight
+                    // 16-byte stores remain once the slot is free
+                    const uint32_t tab_slot = tab_warp + ((j & 1u) << 10);
+                    if (wcls == 2) {
+                        ptx::cp_async_wait<1>();   // this entry's table has landed (the next entry's may still be under way)
+                        __syncwarp();
+                    }
                     uint32_t o[32];
                     if (col != kIdleItem) {
                         if (wcls == 0) deq64_1bit(blk0.lo.x, blk0.lo.y, lv0.m0, lv0.m1, blk0.a, o);
                         else if (wcls == 1) deq64_2bit(blk0.lo, lv0, blk0.a, o);
-                        else if (wcls == 2) ptx::prefetch_l1(mrow);
+                        else if (wcls == 2) deq64_4bit_direct(blk0.lo, blk0.hi, blk0.a, tab_slot + (lane & 15u) * 64u, o);
                     }
                     const uint32_t it = it0 + (head & 0xFFFFFFu);
                     const int s = it % SA;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
                     if (col != kIdleItem) {
                         const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)half * 8192u + col * 128u;
-                        if (wcls <= 1) store_row(row_addr, col & 7, o);
-                        else if (wcls == 2) dequant_block_4bit(blk0.lo, blk0.hi, blk0.a, mrow, row_addr, col & 7);
+                        if (wcls <= 2) store_row(row_addr, col & 7, o);
                         else zero_row(row_addr);
                         ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
                     }
@@ -700,7 +662,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     // shift, and fetch the data of the entry after next
                     head0 = head1; rec0 = rec1; blk0 = blk1; lv0 = lv1;
                     head1 = head2; rec1 = rec2;
-                    fetch(blk1, lv1, head1, rec1);
+                    fetch(blk1, lv1, head1, rec1, tab_slot);   // entry j + 2 takes over the table slot of entry j
                 }
                 // LoRA blocks: operands come by TMA; the warps take the stages in turn and arrive for everybody
                 for (int kb = P.main_blocks + pw; kb < t.blocks && !failed; kb += kProducerWarps) {

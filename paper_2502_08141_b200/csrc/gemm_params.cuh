@@ -46,7 +46,7 @@ constexpr int kStages = 4;        // dense diagnostic: four stages of one weight
 // of the tensor core than the TMA loads do, so the ring is split into 16 KB weight slots and 32 KB token slots:
 // six + four (backward), five + four (forward, which spends the difference on a cache of the level tables of
 // its 4-bit rows).  A weight slot is free once the MMAs of that many stages earlier are complete.
-constexpr int kStagesA_fwd = 5, kStagesA_bwd = 6;
+constexpr int kStagesA_fwd = 5, kStagesA_bwd = 5;
 constexpr int kStagesB_fwd = 4, kStagesB_bwd = 4;
 constexpr int kMaxStagesA = 6;
 constexpr int kFirstEpilogueWarp = 2;
@@ -83,12 +83,13 @@ struct GemmParams {
 constexpr uint32_t kSmemA = kTileR * kTileC * 2;   // 16 KB
 constexpr uint32_t kSmemB = kTileT * kTileC * 2;   // 32 KB
 constexpr uint32_t kSmemStage = kSmemA + kSmemB;
-constexpr uint32_t kSmemRingMax = kStagesA_bwd * kSmemA + kStagesB_bwd * kSmemB;   // 224 KB
+constexpr uint32_t kSmemRingMax = 224 * 1024;   // operand ring + table cache
 static_assert(kStages * kSmemStage <= kSmemRingMax, "the dense ring fits into the same space");
 constexpr int kEpilogueTokens = 8;                           // tokens per transposition round of the epilogue
 constexpr uint32_t kSmemOut = kEpilogueTokens * kTileR * 2;  // epilogue staging: 8 tokens x 128 channels bf16
 constexpr uint32_t kSmemBarriers = 1024;
-constexpr uint32_t kSmemTab = kProducerWarps * 2048;         // forward: fp32 level tables of the warps' 4-bit rows
+constexpr uint32_t kSmemTab = kProducerWarps * 2048;         // fp32 level tables of the dequant warps' 4-bit rows
+static_assert(kStagesA_bwd * kSmemA + kStagesB_bwd * kSmemB + kSmemTab <= kSmemRingMax, "the backward ring and its table cache fit");
 static_assert(kStagesA_fwd * kSmemA + kStagesB_fwd * kSmemB + kSmemTab <= kSmemRingMax, "the forward ring and its table cache fit");
 // no alignment slack: the dynamic shared memory of a kernel without static shared memory starts 1024-byte
 // aligned (checked by the kernel, which the swizzled operand tiles need)
