@@ -51,7 +51,11 @@ constexpr int kStagesB_fwd = 4, kStagesB_bwd = 4;
 constexpr int kMaxStagesA = 6;
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstProducerWarp = 6;
-constexpr int kGemmThreads = 32 * (kFirstProducerWarp + kProducerWarps);
+// 16 warps, of which two idle (which two depends on the pass, see the kernel): at most four per scheduler, so
+// 128 registers per thread.
+constexpr int kGemmWarps = 16;
+constexpr int kGemmThreads = 32 * kGemmWarps;
+static_assert(kProducerWarps == 8, "the warp map above places eight dequant warps");
 constexpr int kTmemCols = 512;    // two 128 x 256 fp32 accumulators
 
 constexpr int kModeForward = 0, kModeBackward = 1, kModeDense = 2;
