@@ -48,7 +48,8 @@ struct Barriers {
                                        // producer of CTA c of the cluster (every CTA holds a copy of all counters)
 };
 
-// fields of the per-thread row word written by the prologue (see kIdleItem below)
+// fields of the forward row word written by the prologue: bits 0-6 row offset inside the tile, 7-8 class
+// (0, 1, 2 = 1, 2, 4 bits; 3 = row past N, to be zero-filled), 9-31 stored position
 __device__ __forceinline__ int info_row(uint32_t w) { return (int)(w & 127u); }
 __device__ __forceinline__ int info_class(uint32_t w) { return (int)((w >> 7) & 3u); }
 __device__ __forceinline__ int info_pos(uint32_t w) { return (int)(w >> 9); }
@@ -140,16 +141,6 @@ __device__ __forceinline__ void store_row(uint32_t row_addr, int swz, const uint
     for (int t = 0; t < 8; ++t)
         ptx::st_shared_v4(row_addr + (uint32_t)((t ^ swz) << 4), make_uint4(o[4 * t], o[4 * t + 1], o[4 * t + 2], o[4 * t + 3]));
 }
-
-__device__ __noinline__ void zero_row(uint32_t row_addr) {
-#pragma unroll
-    for (int t = 0; t < 8; ++t) ptx::st_shared_v4(row_addr + 16u * t, make_uint4(0u, 0u, 0u, 0u));
-}
-
-// word written by the prologue for every dequant thread and every row group: bits 0-6 row offset inside
-// the group, 7-8 class (0,1,2 = 1,2,4 bits; 3 = row past N, to be zero-filled), 9-31 stored position;
-// all ones = this thread has no row in this group.  All rows of one warp have the same class.
-constexpr uint32_t kIdleItem = 0xFFFFFFFFu;
 
 }  // namespace
 
@@ -606,7 +597,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // row travel asynchronously into this warp's table cache (two slots of 16 rows x 64 bytes, one per
                 // entry in flight; the two lanes of a row read the same 64 bytes)
                 auto fetch = [&](Block& blk, Levels& lv, uint32_t head, const uint4& rec, uint32_t tab_slot) {
-                    const int cls = (head == kEnd || rec.w == kIdleItem) ? 4 : (int)((head >> 28) & 3u);
+                    const int cls = (head == kEnd) ? 4 : (int)((rec.w >> 8) & 3u);   // this lane's row
                     if (cls < 3) {
                         load_block(blk, P.packed + ((size_t)rec.x << 4) + (((size_t)k_first << cls) >> 3),
                                    P.absmax + rec.y + (k_first >> 6), cls);
@@ -633,34 +624,33 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 for (uint32_t j = 0; !failed; ++j) {
                     const uint32_t head = head0;
                     if (head == kEnd) break;
-                    const uint32_t col = rec0.w;   // channel inside the stage = K index of the tile
-                    const int wcls = (int)((head >> 28) & 3u);   // the same for the whole warp
+                    const uint32_t col = rec0.w & 63u;             // channel inside the stage = K index of the tile
+                    const int cls = (int)((rec0.w >> 8) & 3u);     // precision class of this lane's row (3: zeros)
                     // head and row record of the entry after next are asked for now and consumed after this visit;
                     // the lists end with kListSlack all-ones heads
                     const uint32_t head2 = __ldg(heads + (size_t)(j + 2) * kListWarps);
                     const uint4 rec2 = __ldg(rows + (size_t)(j + 2) * kListWarps * 32);
                     // the block is dequantised into registers BEFORE the wait for the stage, so that only the eight
-                    // 16-byte stores remain once the slot is free
+                    // 16-byte stores remain once the slot is free (rows of two precisions may meet in the warp)
                     const uint32_t tab_slot = tab_warp + ((j & 1u) << 10);
-                    if (wcls == 2) {
-                        ptx::cp_async_wait<1>();   // this entry's table has landed (the next entry's may still be under way)
-                        __syncwarp();
-                    }
+                    ptx::cp_async_wait<1>();   // this entry's 4-bit tables have landed (the next entry's may still be under way)
+                    __syncwarp();
                     uint32_t o[32];
-                    if (col != kIdleItem) {
-                        if (wcls == 0) deq64_1bit(blk0.lo.x, blk0.lo.y, lv0.m0, lv0.m1, blk0.a, o);
-                        else if (wcls == 1) deq64_2bit(blk0.lo, lv0, blk0.a, o);
-                        else if (wcls == 2) deq64_4bit_direct(blk0.lo, blk0.hi, blk0.a, tab_slot + (lane & 15u) * 64u, o);
+                    if (cls == 0) {
+                        deq64_1bit(blk0.lo.x, blk0.lo.y, lv0.m0, lv0.m1, blk0.a, o);
+                    } else if (cls == 1) {
+                        deq64_2bit(blk0.lo, lv0, blk0.a, o);
+                    } else if (cls == 2) {
+                        deq64_4bit_direct(blk0.lo, blk0.hi, blk0.a, tab_slot + (lane & 15u) * 64u, o);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] = 0u;
                     }
                     const uint32_t it = it0 + (head & 0xFFFFFFu);
                     const int s = it % SA;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
-                    if (col != kIdleItem) {
-                        const uint32_t row_addr = ptx::smem_u32(a_slot(it)) + (uint32_t)half * 8192u + col * 128u;
-                        if (wcls <= 2) store_row(row_addr, col & 7, o);
-                        else zero_row(row_addr);
-                        ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
-                    }
+                    store_row(ptx::smem_u32(a_slot(it)) + (uint32_t)half * 8192u + col * 128u, (int)(col & 7u), o);
+                    ptx::fence_proxy_async_smem();   // the tensor core and the copy to the peers read the row
                     __syncwarp();
                     if (lane == 0) finish_stage(it, s, (head >> 24) & 15u);
                     // shift, and fetch the data of the entry after next

@@ -26,10 +26,10 @@ Workspace plan_workspace(int N, int K, int M, int r) {
     (void)K;
     Workspace w;
     w.rp = (r + 63) / 64 * 64;
-    // forward: 128 row words per group of 128 channels; backward: at most 7 work-list entries (a head and
-    // 32 row records of 16 bytes each) per group of 64 channels, plus the end markers
+    // forward: 128 row words per group of 128 channels; backward: 4 work-list entries (a head and 32 row records
+    // of 16 bytes each) per group of 64 channels, plus the end markers
     const size_t groups_per_cta = ((size_t)(N + 63) / 64 + kCluster - 1) / kCluster;
-    const size_t entries = kCluster * (7 * groups_per_cta + kListSlack + kProducerWarps);
+    const size_t entries = kCluster * (4 * groups_per_cta + kListSlack + kProducerWarps);
     const size_t fwd_words = (size_t)((N + 127) / 128) * kItemStride;
     w.off_T = kStatusBytes;
     w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);

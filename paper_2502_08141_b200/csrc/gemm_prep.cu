@@ -69,73 +69,37 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
 
 // Backward-input: every pipeline stage of the main kernel brings a group of 64 consecutive output channels.
 // The CTAs of a cluster take the groups in turn (group g is dequantised by CTA g % kCluster, which then copies
-// the finished operand tile to its peers).  The rows of a group are ordered by precision class and cut into
-// chunks of at most 16 rows of one class; a chunk is the work of one dequant warp on one stage (32 lanes =
-// 16 rows x 2 halves of the tile's 128 features).  The chunks of the groups of one CTA are numbered through the
-// whole matrix and chunk n goes to warp n % kProducerWarps of that CTA as entry n / kProducerWarps of the
-// warp's work list, so a warp only ever visits the stages it has work on:
-//   heads[e]         = group index (bits 0-23) | arrivals this entry owes the stage barrier (bits 24-27) |
-//                      precision class of the chunk (bits 28-29; 3 = rows past N, to be zero-filled)
+// the finished operand tile to its peers).  The rows of a group are ordered by precision class (rows past N last)
+// and cut into four chunks of 16 rows; a chunk is the work of one dequant warp on one stage (32 lanes = 16 rows x
+// 2 halves of the tile's 128 features), so most warps see one precision and a few see two.  The chunks of the
+// groups of one CTA are numbered through the whole matrix and chunk n goes to warp n % kProducerWarps of that
+// CTA as entry n / kProducerWarps of the warp's work list, so a warp only ever visits the stages it has work on:
+//   heads[e]         = group index (bits 0-23) | arrivals this entry owes the stage barrier (bits 24-27)
 //   rows[e * 32 + l] = what lane l needs to find its row, ready to use (16 bytes):
 //                      x = byte offset of the row in the packed buffer / 16, y = index of the row's first absmax,
-//                      z = index of the row's first level in the maps table, w = channel inside the group
-//                      (all ones: this lane has no row)
-// with e = entry * kListWarps + warp * kCluster + CTA.  The stage barrier expects kStageArrivals arrivals; the
-// first chunk of a group also arrives for the chunks the group does not have.  Every list ends with all-ones heads.
+//                      z = index of the row's first level in the maps table,
+//                      w = channel inside the group (bits 0-5) | precision class (bits 8-9; 3 = row past N: zeros)
+// with e = entry * kListWarps + warp * kCluster + CTA.  Every list ends with all-ones heads.
 __device__ __forceinline__ uint32_t list_slot(uint32_t n, int cta) {
     return (n / kProducerWarps) * kListWarps + (n % kProducerWarps) * kCluster + (uint32_t)cta;
 }
 
-__device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint32_t* wsum) {
+__device__ void deal_backward(const PrepParams& P, int blk) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
     constexpr int kWarps = kPrepThreads / 32;
+    constexpr int kChunks = 4;   // per group of 64 rows
     const int n_groups = (P.N + 63) / 64;
-    // ---- chunks per group (every block computes all of them: the numbering needs the running sums)
-    for (int grp = warp; grp < n_groups; grp += kWarps) {
-        const int r0 = grp * 64 + lane, r1 = r0 + 32;
-        const int c0 = (r0 < P.N) ? (P.precs[r0] >> 1) : 3, c1 = (r1 < P.N) ? (P.precs[r1] >> 1) : 3;
-        int n = 0;
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            n += (__popc(__ballot_sync(0xffffffffu, c0 == c)) + __popc(__ballot_sync(0xffffffffu, c1 == c)) + 15) / 16;
-        if (lane == 0) pre[grp] = (uint16_t)n;
-    }
-    __syncthreads();
-    // ---- exclusive running sums, one per CTA of the cluster (over the groups g with g % kCluster == cta)
-    for (int cta = 0; cta < kCluster; ++cta) {
-        const int n_mine = (n_groups - cta + kCluster - 1) / kCluster;   // groups of this CTA
-        const int seg = (n_mine + kPrepThreads - 1) / kPrepThreads;
-        const int begin = min(tid * seg, n_mine), end = min(begin + seg, n_mine);
-        uint32_t mine = 0;
-        for (int i = begin; i < end; ++i) mine += pre[i * kCluster + cta];
-        uint32_t incl = mine;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, d);
-            if (lane >= d) incl += v;
-        }
-        if (lane == 31) wsum[warp] = incl;
-        __syncthreads();
-        uint32_t run = incl - mine;
-        uint32_t total = 0;
-#pragma unroll
-        for (int w2 = 0; w2 < kWarps; ++w2) {
-            if (w2 < warp) run += wsum[w2];
-            total += wsum[w2];
-        }
-        for (int i = begin; i < end; ++i) {
-            const uint32_t n = pre[i * kCluster + cta];
-            pre[i * kCluster + cta] = (uint16_t)run;
-            run += n;
-        }
-        if (blk == 0)
+    if (blk == 0) {   // end markers behind the last entry of every CTA's lists
+        for (int cta = 0; cta < kCluster; ++cta) {
+            const uint32_t total = (uint32_t)kChunks * (uint32_t)((n_groups - cta + kCluster - 1) / kCluster);
             for (int i = tid; i < kListSlack; i += kPrepThreads) P.heads[list_slot(total + (uint32_t)i, cta)] = 0xFFFFFFFFu;
-        __syncthreads();
+        }
     }
-
-    // ---- the deal proper: one warp per group
+    uint4* rows = reinterpret_cast<uint4*>(P.items);
+    // one warp per group
     for (int grp = blk * kWarps + warp; grp < n_groups; grp += P.blocks * kWarps) {
-        const uint32_t g0 = pre[grp];
+        const int cta = grp % kCluster;
+        const uint32_t n0 = (uint32_t)kChunks * (uint32_t)(grp / kCluster);   // number of the group's first chunk
         int cls[2];
         unsigned mask[2][4];
         int total_c[4] = {0, 0, 0, 0};
@@ -149,28 +113,19 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
                 total_c[c] += __popc(mask[i][c]);
             }
         }
-        int chunk_base[4];
-        chunk_base[0] = 0;
+        int class_base[4];
+        class_base[0] = 0;
 #pragma unroll
-        for (int c = 1; c < 4; ++c) chunk_base[c] = chunk_base[c - 1] + (total_c[c - 1] + 15) / 16;
-        const int n_chunks = chunk_base[3] + (total_c[3] + 15) / 16;
-        auto entry_of = [&](int ci) { return list_slot(g0 + (uint32_t)ci, grp % kCluster); };
-        uint4* rows = reinterpret_cast<uint4*>(P.items);
-        for (int ci = 0; ci < n_chunks; ++ci)
-            rows[(size_t)entry_of(ci) * 32 + lane] = make_uint4(0u, 0u, 0u, 0xFFFFFFFFu);
-        if (lane < n_chunks) {
-            const int c = (lane >= chunk_base[1]) + (lane >= chunk_base[2]) + (lane >= chunk_base[3]);   // class of chunk `lane`
-            P.heads[entry_of(lane)] = (uint32_t)grp | ((uint32_t)(lane == 0 ? kStageArrivals - n_chunks + 1 : 1) << 24) |
-                                      ((uint32_t)c << 28);
-        }
-        __syncwarp();
+        for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total_c[c - 1];
+        if (lane < kChunks)
+            P.heads[list_slot(n0 + (uint32_t)lane, cta)] = (uint32_t)grp | ((uint32_t)(kStageArrivals / kChunks) << 24);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 if (cls[i] == c) {
                     const int off = i * 32 + lane, row = grp * 64 + off;
-                    uint4 rec = make_uint4(0u, 0u, 0u, (uint32_t)off);
+                    uint4 rec = make_uint4(0u, 0u, 0u, (uint32_t)off | ((uint32_t)c << 8));
                     if (c < 3) {
                         const uint32_t sp = (uint32_t)P.inv_perm[row];   // stored position
                         const uint64_t row_bytes = ((uint64_t)P.L.K << c) >> 3;
@@ -185,13 +140,13 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
                     int b = 0;   // rank of this row among the rows of its class with the same residue
                     if (i == 1) b += __popc(mask[0][c] & res_mask);
                     b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
-                    int pos = 0;  // rows taken before this one
+                    int pos = class_base[c];  // rows taken before this one
 #pragma unroll
                     for (int res = 0; res < 8; ++res) {
                         const int cnt = __popc(mask[0][c] & (0x01010101u << res)) + __popc(mask[1][c] & (0x01010101u << res));
                         pos += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
                     }
-                    uint4* dst = rows + (size_t)entry_of(chunk_base[c] + pos / 16) * 32 + pos % 16;
+                    uint4* dst = rows + (size_t)list_slot(n0 + (uint32_t)(pos / 16), cta) * 32 + pos % 16;
                     dst[0] = rec;
                     dst[16] = rec;
                 }
@@ -199,7 +154,6 @@ __device__ void deal_backward(const PrepParams& P, int blk, uint16_t* pre, uint3
         }
     }
 }
-
 
 }  // namespace
 
@@ -210,9 +164,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const PrepParams P) 
         for (int i = threadIdx.x; i < P.n_flags; i += kPrepThreads) P.flags[i] = 0u;
     }
     if (P.group == 64) {
-        __shared__ uint16_t pre[kMaxGroups64];
-        __shared__ uint32_t wsum[kPrepThreads / 32];
-        deal_backward(P, blockIdx.x, pre, wsum);
+        deal_backward(P, blockIdx.x);
     } else {
         deal_rows(P, blockIdx.x);
     }
