@@ -298,6 +298,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             // pacemaker of the whole CTA: the two barriers of stage it + 1 are probed (non-blocking) before the
             // MMAs of stage it are issued, so the answers are back by the time they are needed.
             bool ready_x = false, ready_w = false;
+            // slots and phases of the two rings, carried along (no division by the ring depths in this loop: the
+            // thread's instructions are one dependent chain)
+            uint32_t sb = 0, phb = 0, sa = 0, pha = 0;
             for (int g = first_tile; g < n_tiles && !failed; g += tile_step, ++tile_iter) {
                 const TileInfo t = decode_tile(g);
                 const uint32_t acc = tile_iter & 1u;            // two accumulators take turns
@@ -306,20 +309,22 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileT;
                 for (int kb = 0; kb < t.blocks; ++kb, ++it) {
-                    const int s = it % SB;
-                    const uint32_t ph = (it / SB) & 1u;
-                    const int sw = (int)(it % SA);              // weight slot
-                    const uint32_t phw = (it / SA) & 1u;
+                    const int s = (int)sb;                      // token slot
+                    const uint32_t ph = phb;
+                    const int sw = (int)sa;                     // weight slot
+                    const uint32_t phw = pha;
                     if (!ready_x)
                         if (!ptx::mbar_wait(&bars->full_x[s], ph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                     if (MODE != kModeDense && !ready_w)
                         if (!ptx::mbar_wait(&bars->full_w[sw], phw, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                     ptx::tc_fence_after();
                     // probe the next stage now (its slots depend on the running stage index only)
-                    ready_x = ptx::mbar_test_wait(&bars->full_x[(it + 1u) % SB], ((it + 1u) / SB) & 1u);
-                    ready_w = (MODE == kModeDense) || ptx::mbar_test_wait(&bars->full_w[(it + 1u) % SA], ((it + 1u) / SA) & 1u);
-                    const uint32_t a_addr = ptx::smem_u32(a_slot(it));
-                    const uint64_t bdesc = ptx::umma_desc_k_sw128(ptx::smem_u32(b_slot(it)));
+                    const uint32_t a_addr = ptx::smem_u32(base + sa * kSmemA);
+                    const uint64_t bdesc = ptx::umma_desc_k_sw128(ptx::smem_u32(base + SA * kSmemA + sb * kSmemB));
+                    if (++sb == (uint32_t)SB) { sb = 0; phb ^= 1u; }
+                    if (++sa == (uint32_t)SA) { sa = 0; pha ^= 1u; }
+                    ready_x = ptx::mbar_test_wait(&bars->full_x[sb], phb);
+                    ready_w = (MODE == kModeDense) || ptx::mbar_test_wait(&bars->full_w[sa], pha);
                     // which weight-operand tiles are MN-major (a contraction index is a 128-byte row of 64 operand
                     // rows): forward - the factor tiles, fetched from A [K, r] (T tiles) and B [r, N] (LoRA blocks);
                     // backward - the dequantised weight tile
