@@ -117,6 +117,7 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const DecodePara
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     WarpStage* ws = &stage_all[warp];
+    pdl_enter();
     const uint32_t n_tasks = P.task_start[3];
     const uint32_t stride = gridDim.x * kDecodeWarps;
     for (uint32_t t = blockIdx.x * kDecodeWarps + warp; t < n_tasks; t += stride) {
@@ -165,6 +166,5 @@ extern "C" lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* 
     const uint64_t blocks_needed = (tasks + kDecodeWarps - 1) / kDecodeWarps;
     const uint64_t cap = (uint64_t)kNumSMs * 8;
     const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
-    decode_kernel<<<grid, kDecodeThreads, 0, (cudaStream_t)stream>>>(P);
-    return cudaGetLastError() == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+    return launch_pdl(decode_kernel, grid, kDecodeThreads, (cudaStream_t)stream, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
 }

@@ -172,6 +172,7 @@ __global__ void __launch_bounds__(kEncodeThreads) encode_kernel(const EncodePara
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     unsigned char* stage = stage_all[warp];
+    pdl_enter();
     const uint32_t stride = gridDim.x * kEncodeWarps;
     for (uint32_t t = blockIdx.x * kEncodeWarps + warp; t < P.n_tasks; t += stride) {
         const int p = t / P.chunks_per_row;
@@ -209,6 +210,5 @@ extern "C" lowra_status lowra_encode(const lowra_layout* layout, const float* W_
     const uint64_t blocks_needed = (tasks + kEncodeWarps - 1) / kEncodeWarps;
     const uint64_t cap = (uint64_t)kNumSMs * 3;   // three CTAs (80 registers, 36 KB of shared memory) are resident per SM
     const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
-    encode_kernel<<<grid, kEncodeThreads, 0, (cudaStream_t)stream>>>(P);
-    return cudaGetLastError() == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+    return launch_pdl(encode_kernel, grid, kEncodeThreads, (cudaStream_t)stream, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
 }

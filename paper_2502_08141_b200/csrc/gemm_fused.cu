@@ -219,7 +219,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     ptx::tc_fence_after();
     // Everything above overlapped the prologue kernel (programmatic dependent launch); what follows reads what
     // that kernel wrote (row deal, cleared flags and status word).
-    if (MODE != kModeDense) ptx::grid_dependency_wait();
+    if (MODE != kModeDense) pdl_enter();
     const uint32_t tmem_base = bars->tmem_base;
 
     bool failed = false;

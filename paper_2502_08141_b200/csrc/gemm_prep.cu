@@ -158,7 +158,7 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
 }  // namespace
 
 __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const PrepParams P) {
-    ptx::grid_launch_dependents();   // the fused kernel may set itself up meanwhile; it waits for this grid before reading
+    pdl_enter();   // the fused kernel may set itself up meanwhile; it waits for this grid before it reads the deal
     if (blockIdx.x == 0) {
         if (threadIdx.x == 0) *P.status = 0u;
         for (int i = threadIdx.x; i < P.n_flags; i += kPrepThreads) P.flags[i] = 0u;
@@ -171,8 +171,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const PrepParams P) 
 }
 
 lowra_status launch_prep(const PrepParams& P, cudaStream_t stream) {
-    prep_kernel<<<P.blocks, kPrepThreads, 0, stream>>>(P);
-    return cudaGetLastError() == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+    return launch_pdl(prep_kernel, (unsigned)P.blocks, kPrepThreads, stream, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
 }
 
 }  // namespace lowra

@@ -1,6 +1,7 @@
 // Shared declarations of the CUDA path: launch-parameter structs, host-side validation helpers and
 // a few device intrinsics.  Nothing in here is used by, or taken from, the CPU oracle.
 #pragma once
+#include <utility>
 
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -28,6 +29,30 @@ lowra_status check_device();
 RowLayout make_row_layout(const lowra_layout* L);
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// -------------------------------------------------------------------------------------------
+// programmatic dependent launch: every kernel of the library lets its successor in the stream start launching
+// right away (so the successor's launch latency and set-up overlap this kernel) and itself waits, before it
+// touches global memory, until its predecessor has completed and flushed - stream order is preserved.
+// -------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, unsigned block, cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(block, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // -------------------------------------------------------------------------------------------
 // device helpers
