@@ -173,6 +173,29 @@ lowra_status lowra_lora_forward_static(const lowra_layout* layout, const uint8_t
                                        float s, uint16_t* Y_dev, uint32_t* status_out_dev, void* stream);
 
 /*
+ * Mapping and threshold learner (Section 5, "Weighted Lloyd's for LoRA Quantization"; appendix "Weighted
+ * Lloyd-Max Algorithm"): for every output channel, at the channel's assigned precision, run `iterations` rounds
+ * of weighted Lloyd-Max on the channel's normalised values (normalised per 64-block exactly as in lowra_encode;
+ * the weight of a value is the absmax of its block):
+ *     assign:  bucket of n = number of current thresholds <= n
+ *     levels:  y_j <- sum(w n) / sum(w) over bucket j   (an empty bucket keeps its level)
+ *     thresholds: t_j <- (y_j + y_{j+1}) / 2
+ * in fp64.  Output tables, fp32 [N, 16], original row order: maps = (float) y (unused entries 0),
+ * thresholds[j] = (float)(((double) maps[j] + (double) maps[j+1]) / 2) (unused entries +infinity) - directly
+ * usable by lowra_encode / lowra_decode.
+ *   W_dev                 fp32 [N, K] row-major, original row order                      (in)
+ *   init_levels_host      fp64 [3][16] HOST: starting levels for 1-, 2-, 4-bit rows      (in; the appendix
+ *   init_thresholds_host  fp64 [3][16] HOST: starting thresholds                          on initialisation)
+ *   iterations            0 .. 1000 (the paper runs 2)
+ * The sums are formed by a fixed parallel tree, not in index order: results are reproducible from run to run
+ * and agree with a serial fp64 implementation to rounding.  K * 4 bytes must fit in shared memory
+ * (K <= 40960), else LOWRA_ERR_SHAPE.  Uses layout->precs_dev only (perm / offsets are not needed).
+ */
+lowra_status lowra_learn_codebooks(const lowra_layout* layout, const float* W_dev, const double* init_levels_host,
+                                   const double* init_thresholds_host, int32_t iterations, float* maps_dev,
+                                   float* thresholds_dev, void* stream);
+
+/*
  * Diagnostic, not part of the method: C = P . Q^T with P bf16 [M, K], Q bf16 [N, K] (both
  * row-major, K % 64 == 0), C bf16 [M, N], run through the same tensor-core pipeline as the fused
  * kernels but with both operands fetched as plain bf16 tiles.  Used to compare "decode, then dense

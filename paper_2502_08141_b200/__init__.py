@@ -27,7 +27,7 @@ LOWRA_STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "lowra_status_string", "lowra_plan", "lowra_encode", "lowra_decode", "lowra_workspace_bytes",
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
-    "lowra_lora_forward_static",
+    "lowra_lora_forward_static", "lowra_learn_codebooks",
 )
 
 
@@ -78,6 +78,8 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_backward_input.restype = ctypes.c_int
         L.lowra_lora_forward_static.argtypes = [lp, vp, vp, vp, vp, i32, vp, vp, i32, ctypes.c_float, vp, vp, vp]
         L.lowra_lora_forward_static.restype = ctypes.c_int
+        L.lowra_learn_codebooks.argtypes = [lp, vp, vp, vp, i32, vp, vp, vp]
+        L.lowra_learn_codebooks.restype = ctypes.c_int
         L.lowra_device_status.argtypes = [vp, vp]
         L.lowra_device_status.restype = ctypes.c_int
         L.lowra_dense_nt.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
@@ -191,6 +193,30 @@ def lowra_decode(layout: Layout, packed: torch.Tensor, absmax: torch.Tensor, map
     code = lib().lowra_decode(layout.ref, _ptr(packed), _ptr(absmax), _ptr(maps), _ptr(out), _stream(stream))
     _check(code, "lowra_decode")
     return out
+
+
+def lowra_learn_codebooks(layout: Layout, W: torch.Tensor, init_levels, init_thresholds, iterations: int,
+                          maps: Optional[torch.Tensor] = None, thresholds: Optional[torch.Tensor] = None,
+                          stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Weighted Lloyd-Max per row at the row's precision -> (maps fp32 [N,16], thresholds fp32 [N,16]).
+
+    init_levels / init_thresholds: host arrays [3, 16] float64 (rows: 1-, 2-, 4-bit starting tables)."""
+    _dev(W, torch.float32, "W")
+    y0 = np.ascontiguousarray(init_levels, dtype=np.float64)
+    t0 = np.ascontiguousarray(init_thresholds, dtype=np.float64)
+    if y0.shape != (3, 16) or t0.shape != (3, 16):
+        raise ValueError("init_levels and init_thresholds must be [3, 16]")
+    if maps is None:
+        maps = torch.empty((layout.N, 16), dtype=torch.float32, device=W.device)
+    if thresholds is None:
+        thresholds = torch.empty((layout.N, 16), dtype=torch.float32, device=W.device)
+    _dev(maps, torch.float32, "maps")
+    _dev(thresholds, torch.float32, "thresholds")
+    code = lib().lowra_learn_codebooks(layout.ref, _ptr(W), y0.ctypes.data_as(ctypes.c_void_p),
+                                       t0.ctypes.data_as(ctypes.c_void_p), int(iterations), _ptr(maps),
+                                       _ptr(thresholds), _stream(stream))
+    _check(code, "lowra_learn_codebooks")
+    return maps, thresholds
 
 
 def lowra_workspace_bytes(layout: Layout, M: int, r: int) -> int:

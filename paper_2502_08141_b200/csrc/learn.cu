@@ -1,0 +1,209 @@
+// lowra_learn_codebooks: weighted Lloyd-Max per output channel (paper Section 5, "Weighted Lloyd's for LoRA
+// Quantization", and the appendix "Weighted Lloyd-Max Algorithm"; the appendix on the learner's initialisation
+// gives the initial tables, which the caller passes in).
+//
+// For every row, at the row's assigned precision b: the data are the row's normalised values n_i (block
+// absmax normalisation exactly as in lowra_encode), each weighted by the absmax of its block; starting from the
+// given levels y and thresholds t, T times: assign every value to its bucket (number of thresholds <= n),
+// replace every level by the weighted mean of its bucket (an empty bucket keeps its level), set the thresholds
+// to the midpoints of neighbouring levels.  All of that in fp64.  Output: the levels rounded to fp32 and the
+// midpoints of those fp32 levels (computed in fp64, rounded to fp32), in [N, 16] tables.
+//
+// One CTA per row at a time (persistent, grid-stride): the row is read from HBM once (4 bytes per element, the
+// kernel's only traffic), normalised and parked in shared memory; the T passes run out of shared memory.
+// Every thread keeps private fp64 sums per bucket: in registers for 1 and 2 bits, in a bank-conflict-free
+// slice of shared memory for 4 bits; a fixed reduction tree adds them up (warp shuffles, then across warps), so
+// results are reproducible from run to run - but the order of the fp64 additions is not the index order of a
+// serial loop, so sums agree with a serial implementation to rounding only.
+#include "lowra_common.cuh"
+
+namespace lowra {
+
+constexpr int kLearnThreads = 128;
+constexpr int kLearnWarps = kLearnThreads / 32;
+
+struct LearnParams {
+    RowLayout L;
+    const float* W;       // [N, K] original order
+    float* maps;          // [N, 16] original order
+    float* thresholds;    // [N, 16] original order
+    int iterations;
+    double init_y[3][16];  // initial levels per class (1, 2, 4 bits)
+    double init_t[3][16];  // initial thresholds per class
+};
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
+    return v;
+}
+
+// number of thresholds <= x among t[0 .. L-2] (sorted): branch-free binary search, L = 2, 4 or 16
+template <int B>
+__device__ __forceinline__ int bucket_of(double x, const double* t) {
+    if (B == 1) return t[0] <= x ? 1 : 0;
+    if (B == 2) {
+        const int hi = t[1] <= x ? 2 : 0;
+        return hi + (t[hi] <= x ? 1 : 0);
+    }
+    int c = t[7] <= x ? 8 : 0;
+    c += t[c + 3] <= x ? 4 : 0;
+    c += t[c + 1] <= x ? 2 : 0;
+    c += t[c] <= x ? 1 : 0;
+    return c;
+}
+
+template <int B>
+__device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, double* acc, double* red, double* yt) {
+    constexpr int Lv = 1 << B;      // levels
+    constexpr int c = B >> 1;       // class index
+    const int K = P.L.K, nb = P.L.nb;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* wrow = P.W + (size_t)r * K;
+    double* y = yt;          // [16] levels
+    double* t = yt + 16;     // [16] thresholds
+
+    // ---- the row: block absmax, normalised values (as in lowra_encode)
+    for (int g = warp; g < nb; g += kLearnWarps) {
+        const float2 v = *reinterpret_cast<const float2*>(wrow + g * kBlock + 2 * lane);
+        float m = fmaxf(fabsf(v.x), fabsf(v.y));
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+        const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
+        xs[g * kBlock + 2 * lane] = __fmul_rn(v.x, inv);
+        xs[g * kBlock + 2 * lane + 1] = __fmul_rn(v.y, inv);
+        if (lane == 0) ws[g] = m;
+    }
+    if (tid < 16) {
+        y[tid] = P.init_y[c][tid];
+        t[tid] = P.init_t[c][tid];
+    }
+    __syncthreads();
+
+    for (int it = 0; it < P.iterations; ++it) {
+        // ---- one pass: private sums of w * n and w per bucket
+        if (B <= 2) {
+            double num[Lv], den[Lv];
+#pragma unroll
+            for (int j = 0; j < Lv; ++j) num[j] = den[j] = 0.0;
+            for (int i = tid; i < K; i += kLearnThreads) {
+                const double x = (double)xs[i], w = (double)ws[i >> 6];
+                const int b = bucket_of<B>(x, t);
+                const double wx = __dmul_rn(w, x);
+#pragma unroll
+                for (int j = 0; j < Lv; ++j) {
+                    num[j] += (b == j) ? wx : 0.0;
+                    den[j] += (b == j) ? w : 0.0;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < Lv; ++j) {
+                const double sn = warp_sum(num[j]), sd = warp_sum(den[j]);
+                if (lane == 0) { red[(2 * j) * kLearnWarps + warp] = sn; red[(2 * j + 1) * kLearnWarps + warp] = sd; }
+            }
+        } else {
+            // 16 buckets: sums live in shared memory, acc[(2 j + which) * kLearnThreads + tid]
+#pragma unroll
+            for (int j = 0; j < 2 * Lv; ++j) acc[j * kLearnThreads + tid] = 0.0;
+            for (int i = tid; i < K; i += kLearnThreads) {
+                const double x = (double)xs[i], w = (double)ws[i >> 6];
+                const int b = bucket_of<B>(x, t);
+                acc[(2 * b) * kLearnThreads + tid] += __dmul_rn(w, x);
+                acc[(2 * b + 1) * kLearnThreads + tid] += w;
+            }
+#pragma unroll 4
+            for (int j = 0; j < 2 * Lv; ++j) {
+                const double s = warp_sum(acc[j * kLearnThreads + tid]);
+                if (lane == 0) red[j * kLearnWarps + warp] = s;
+            }
+        }
+        __syncthreads();
+        // ---- new levels (an empty bucket keeps its level), then midpoints
+        if (tid < Lv) {
+            double sn = 0.0, sd = 0.0;
+#pragma unroll
+            for (int w2 = 0; w2 < kLearnWarps; ++w2) { sn += red[(2 * tid) * kLearnWarps + w2]; sd += red[(2 * tid + 1) * kLearnWarps + w2]; }
+            if (sd > 0.0) y[tid] = sn / sd;
+        }
+        __syncthreads();
+        if (tid + 1 < Lv) t[tid] = (y[tid] + y[tid + 1]) * 0.5;
+        __syncthreads();
+    }
+
+    // ---- tables: fp32 levels, midpoints of the fp32 levels; unused levels 0, unused thresholds +inf
+    if (tid < kTableStride) {
+        const float m = (tid < Lv) ? (float)y[tid] : 0.0f;
+        const float mn = (tid + 1 < Lv) ? (float)y[tid + 1] : 0.0f;
+        P.maps[(size_t)r * kTableStride + tid] = m;
+        P.thresholds[(size_t)r * kTableStride + tid] =
+            (tid + 1 < Lv) ? (float)(((double)m + (double)mn) * 0.5) : __int_as_float(0x7f800000);
+    }
+    __syncthreads();   // the row buffers are reused by the next row
+}
+
+__global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_constant__ LearnParams P) {
+    extern __shared__ __align__(16) unsigned char learn_smem[];
+    // [16 + 16 doubles levels/thresholds][2 * 16 * warps doubles reduction][2 * 16 * threads doubles sums][K floats][nb floats]
+    double* yt = reinterpret_cast<double*>(learn_smem);
+    double* red = yt + 32;
+    double* acc = red + 2 * 16 * kLearnWarps;
+    float* xs = reinterpret_cast<float*>(acc + 2 * 16 * kLearnThreads);
+    float* ws = xs + P.L.K;
+    pdl_enter();
+    for (int r = blockIdx.x; r < P.L.N; r += gridDim.x) {
+        const int b = P.L.precs[r];
+        if (b == 1) learn_row<1>(P, r, xs, ws, acc, red, yt);
+        else if (b == 2) learn_row<2>(P, r, xs, ws, acc, red, yt);
+        else learn_row<4>(P, r, xs, ws, acc, red, yt);
+    }
+}
+
+}  // namespace lowra
+
+extern "C" lowra_status lowra_learn_codebooks(const lowra_layout* layout, const float* W_dev,
+                                              const double* init_levels_host, const double* init_thresholds_host,
+                                              int32_t iterations, float* maps_dev, float* thresholds_dev, void* stream) {
+    using namespace lowra;
+    lowra_status st = check_layout(layout);
+    if (st != LOWRA_OK) return st;
+    if (!W_dev || !init_levels_host || !init_thresholds_host || !maps_dev || !thresholds_dev) return LOWRA_ERR_NULL;
+    if (iterations < 0 || iterations > 1000) return LOWRA_ERR_SHAPE;
+    if (!aligned16(W_dev) || !aligned16(maps_dev) || !aligned16(thresholds_dev)) return LOWRA_ERR_ALIGN;
+    const size_t smem = (32 + 2 * 16 * kLearnWarps + 2 * 16 * kLearnThreads) * sizeof(double) +
+                        ((size_t)layout->K + (size_t)layout->K / kBlock) * sizeof(float);
+    if (smem > 200 * 1024) return LOWRA_ERR_SHAPE;   // the row has to fit into shared memory (K <= 40960)
+    st = check_device();
+    if (st != LOWRA_OK) return st;
+
+    LearnParams P;
+    P.L = make_row_layout(layout);
+    P.W = W_dev;
+    P.maps = maps_dev;
+    P.thresholds = thresholds_dev;
+    P.iterations = iterations;
+    for (int c = 0; c < 3; ++c)
+        for (int j = 0; j < 16; ++j) {
+            P.init_y[c][j] = init_levels_host[c * 16 + j];
+            P.init_t[c][j] = init_thresholds_host[c * 16 + j];
+        }
+    static size_t configured = 0;
+    if (smem > configured) {
+        if (cudaFuncSetAttribute(learn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return LOWRA_ERR_CUDA;
+        configured = smem;
+    }
+    const int per_sm = (int)((220u * 1024u) / (smem + 1024u));
+    const int cap = kNumSMs * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));
+    const unsigned grid = (unsigned)(layout->N < cap ? layout->N : cap);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kLearnThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = (cudaStream_t)stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, learn_kernel, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+}

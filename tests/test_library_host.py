@@ -94,6 +94,14 @@ def test_validation_runs_before_any_device_work(lib):
     sargs[8] = 24
     assert L.lowra_lora_forward_static(*sargs) == lib.LOWRA_ERR_SHAPE
     assert L.lowra_dense_nt(4096, 4096, 16, 16, 100, 4096, 4096, 256, None) == lib.LOWRA_ERR_SHAPE
+    init = (ctypes.c_double * 48)()
+    assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, None, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, init, init, -1, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
+    assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096 + 4, init, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_ALIGN
+    lay.K = 128 * 400                                                    # a row no longer fits into shared memory
+    lay.packed_bytes = 8 * lay.K // 8
+    lay.seg_off[1] = lay.seg_off[2] = lay.packed_bytes
+    assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, init, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
 
 
 def test_missing_library_fails_loudly(lib, monkeypatch, tmp_path):
