@@ -365,6 +365,30 @@ def run_gpu(args):
         e2e = {"value": aggregate_tflops(flops_step, world, ms), "unit": UNIT, "ms_per_step": ms,
                "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e}
 
+    # ---- outside the step: the codebook learner (the stage before encode), timed on the layer's seven matrices
+    extras = None
+    if rank == 0:
+        y0 = np.zeros((3, 16)); t0 = np.zeros((3, 16))        # stand-in starting tables: equally spaced levels
+        for c, b in enumerate((1, 2, 4)):
+            lv = np.linspace(-1.0, 1.0, 1 << b)
+            y0[c, :lv.size] = lv
+            t0[c, :lv.size - 1] = 0.5 * (lv[:-1] + lv[1:])
+        T_learn = 10
+        torch.cuda.synchronize()
+        for d in dev:   # warm-up
+            lw.lowra_learn_codebooks(d["layout"], d["W"], y0, t0, T_learn, maps=d["maps"], thresholds=d["thr"])
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for d in dev:
+            lw.lowra_learn_codebooks(d["layout"], d["W"], y0, t0, T_learn, maps=d["maps"], thresholds=d["thr"])
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_learn = a.elapsed_time(b)
+        extras = {"learn_codebooks": {"ms": ms_learn, "iterations": T_learn, "GB/s": 4.0 * elems / (ms_learn * 1e-3) / 1e9,
+                                      "frac_hbm": 4.0 * elems / (ms_learn * 1e-3) / 1e9 / P["hbm"],
+                                      "element_passes_per_s": elems * T_learn / (ms_learn * 1e-3),
+                                      "note": "not part of the step; algorithmic bytes = one read of W (4 B per element)"}}
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = cpu_baseline_sample()
@@ -377,7 +401,7 @@ def run_gpu(args):
             "config": {"workload": f"config {WORKLOAD}: {cfg.name}, 7 matrices, {M} tokens, rank {r}, "
                                    f"mix {cfg.mix} (avg {bits:.2f} bits), stand-in codebooks",
                        "elements": elems, "l2": "inputs larger than L2 (about 2.7 GB touched per step)"},
-            "phases": phases, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu,
+            "phases": phases, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "extras": extras,
             "gpu_launches": args.steps * len(dev) * 6, "clocks": clocks,
         }
         print(json.dumps(out))

@@ -38,23 +38,25 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
-// number of thresholds <= x among t[0 .. L-2] (sorted): branch-free binary search, L = 2, 4 or 16
+// number of thresholds <= x among t[0 .. L-2] (sorted): branch-free binary search, L = 2, 4 or 16.
+// x is an fp32 value and tf[j] is the least fp32 number >= the fp64 threshold t[j], so "t[j] <= x" (in fp64) and
+// "tf[j] <= x" (in fp32) are the same statement.
 template <int B>
-__device__ __forceinline__ int bucket_of(double x, const double* t) {
-    if (B == 1) return t[0] <= x ? 1 : 0;
+__device__ __forceinline__ int bucket_of(float x, const float* tf) {
+    if (B == 1) return tf[0] <= x ? 1 : 0;
     if (B == 2) {
-        const int hi = t[1] <= x ? 2 : 0;
-        return hi + (t[hi] <= x ? 1 : 0);
+        const int hi = tf[1] <= x ? 2 : 0;
+        return hi + (tf[hi] <= x ? 1 : 0);
     }
-    int c = t[7] <= x ? 8 : 0;
-    c += t[c + 3] <= x ? 4 : 0;
-    c += t[c + 1] <= x ? 2 : 0;
-    c += t[c] <= x ? 1 : 0;
+    int c = tf[7] <= x ? 8 : 0;
+    c += tf[c + 3] <= x ? 4 : 0;
+    c += tf[c + 1] <= x ? 2 : 0;
+    c += tf[c] <= x ? 1 : 0;
     return c;
 }
 
 template <int B>
-__device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, double* acc, double* red, double* yt) {
+__device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, double* acc, double* red, double* yt, float* tf) {
     constexpr int Lv = 1 << B;      // levels
     constexpr int c = B >> 1;       // class index
     const int K = P.L.K, nb = P.L.nb;
@@ -63,58 +65,92 @@ __device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, dou
     double* y = yt;          // [16] levels
     double* t = yt + 16;     // [16] thresholds
 
-    // ---- the row: block absmax, normalised values (as in lowra_encode)
+    // ---- the row: coalesced 128-bit loads into shared memory first (all of a thread's loads are in flight
+    // together), then block absmax and normalised values in place (as in lowra_encode)
+    for (int i0 = 0; i0 < K; i0 += 4 * 4 * kLearnThreads) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + 4 * (u * kLearnThreads + tid);
+            v[u] = (i < K) ? ld_stream_f4(wrow + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = i0 + 4 * (u * kLearnThreads + tid);
+            if (i < K) *reinterpret_cast<float4*>(xs + i) = v[u];
+        }
+    }
+    __syncthreads();
     for (int g = warp; g < nb; g += kLearnWarps) {
-        const float2 v = *reinterpret_cast<const float2*>(wrow + g * kBlock + 2 * lane);
+        const float2 v = *reinterpret_cast<const float2*>(xs + g * kBlock + 2 * lane);
         float m = fmaxf(fabsf(v.x), fabsf(v.y));
 #pragma unroll
         for (int d = 16; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
         const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
-        xs[g * kBlock + 2 * lane] = __fmul_rn(v.x, inv);
-        xs[g * kBlock + 2 * lane + 1] = __fmul_rn(v.y, inv);
+        *reinterpret_cast<float2*>(xs + g * kBlock + 2 * lane) = make_float2(__fmul_rn(v.x, inv), __fmul_rn(v.y, inv));
         if (lane == 0) ws[g] = m;
     }
     if (tid < 16) {
         y[tid] = P.init_y[c][tid];
         t[tid] = P.init_t[c][tid];
+        tf[tid] = __double2float_ru(P.init_t[c][tid]);
     }
     __syncthreads();
 
     for (int it = 0; it < P.iterations; ++it) {
         // ---- one pass: private sums of w * n and w per bucket
         if (B <= 2) {
-            double num[Lv], den[Lv];
+            // four independent sets of sums per thread (the fp64 adds are latency-bound otherwise); a thread walks
+            // over 64-element blocks, four elements at a time, so the block's weight is converted once
+            double num[4][Lv], den[4][Lv];
 #pragma unroll
-            for (int j = 0; j < Lv; ++j) num[j] = den[j] = 0.0;
-            for (int i = tid; i < K; i += kLearnThreads) {
-                const double x = (double)xs[i], w = (double)ws[i >> 6];
-                const int b = bucket_of<B>(x, t);
-                const double wx = __dmul_rn(w, x);
+            for (int u = 0; u < 4; ++u)
 #pragma unroll
-                for (int j = 0; j < Lv; ++j) {
-                    num[j] += (b == j) ? wx : 0.0;
-                    den[j] += (b == j) ? w : 0.0;
+                for (int j = 0; j < Lv; ++j) num[u][j] = den[u][j] = 0.0;
+            for (int q = tid; q < K / 4; q += kLearnThreads) {   // quad q = elements 4 q .. 4 q + 3, all in block q / 16
+                const float4 xv = *reinterpret_cast<const float4*>(xs + 4 * q);
+                const double w = (double)ws[q >> 4];
+                const float xf[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const double x = (double)xf[u];
+                    const int b = bucket_of<B>(xf[u], tf);
+                    const double wx = __dmul_rn(w, x);
+#pragma unroll
+                    for (int j = 0; j < Lv; ++j) {
+                        num[u][j] += (b == j) ? wx : 0.0;
+                        den[u][j] += (b == j) ? w : 0.0;
+                    }
                 }
             }
 #pragma unroll
             for (int j = 0; j < Lv; ++j) {
-                const double sn = warp_sum(num[j]), sd = warp_sum(den[j]);
+                const double sn = warp_sum((num[0][j] + num[1][j]) + (num[2][j] + num[3][j]));
+                const double sd = warp_sum((den[0][j] + den[1][j]) + (den[2][j] + den[3][j]));
                 if (lane == 0) { red[(2 * j) * kLearnWarps + warp] = sn; red[(2 * j + 1) * kLearnWarps + warp] = sd; }
             }
         } else {
-            // 16 buckets: sums live in shared memory, acc[(2 j + which) * kLearnThreads + tid]
+            // 16 buckets: sums live in shared memory, acc[(2 j + which) * kLearnThreads + tid]; four elements at a
+            // time, their bucket searches side by side
 #pragma unroll
             for (int j = 0; j < 2 * Lv; ++j) acc[j * kLearnThreads + tid] = 0.0;
-            for (int i = tid; i < K; i += kLearnThreads) {
-                const double x = (double)xs[i], w = (double)ws[i >> 6];
-                const int b = bucket_of<B>(x, t);
-                acc[(2 * b) * kLearnThreads + tid] += __dmul_rn(w, x);
-                acc[(2 * b + 1) * kLearnThreads + tid] += w;
+            for (int q = tid; q < K / 4; q += kLearnThreads) {
+                const float4 xv = *reinterpret_cast<const float4*>(xs + 4 * q);
+                const double w = (double)ws[q >> 4];
+                const float xf[4] = {xv.x, xv.y, xv.z, xv.w};
+                int b[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) b[u] = bucket_of<B>(xf[u], tf);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    acc[(2 * b[u]) * kLearnThreads + tid] += __dmul_rn(w, (double)xf[u]);
+                    acc[(2 * b[u] + 1) * kLearnThreads + tid] += w;
+                }
             }
 #pragma unroll 4
             for (int j = 0; j < 2 * Lv; ++j) {
-                const double s = warp_sum(acc[j * kLearnThreads + tid]);
-                if (lane == 0) red[j * kLearnWarps + warp] = s;
+                const double s2 = warp_sum(acc[j * kLearnThreads + tid]);
+                if (lane == 0) red[j * kLearnWarps + warp] = s2;
             }
         }
         __syncthreads();
@@ -126,7 +162,11 @@ __device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, dou
             if (sd > 0.0) y[tid] = sn / sd;
         }
         __syncthreads();
-        if (tid + 1 < Lv) t[tid] = (y[tid] + y[tid + 1]) * 0.5;
+        if (tid + 1 < Lv) {
+            const double tm = (y[tid] + y[tid + 1]) * 0.5;
+            t[tid] = tm;
+            tf[tid] = __double2float_ru(tm);
+        }
         __syncthreads();
     }
 
@@ -143,18 +183,19 @@ __device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, dou
 
 __global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_constant__ LearnParams P) {
     extern __shared__ __align__(16) unsigned char learn_smem[];
-    // [16 + 16 doubles levels/thresholds][2 * 16 * warps doubles reduction][2 * 16 * threads doubles sums][K floats][nb floats]
+    // [16 + 16 doubles levels/thresholds][2 * 16 * warps doubles reduction][2 * 16 * threads doubles sums][K floats][nb floats][16 floats]
     double* yt = reinterpret_cast<double*>(learn_smem);
     double* red = yt + 32;
     double* acc = red + 2 * 16 * kLearnWarps;
     float* xs = reinterpret_cast<float*>(acc + 2 * 16 * kLearnThreads);
     float* ws = xs + P.L.K;
+    float* tf = ws + P.L.nb;   // [16] thresholds as fp32 upper neighbours
     pdl_enter();
     for (int r = blockIdx.x; r < P.L.N; r += gridDim.x) {
         const int b = P.L.precs[r];
-        if (b == 1) learn_row<1>(P, r, xs, ws, acc, red, yt);
-        else if (b == 2) learn_row<2>(P, r, xs, ws, acc, red, yt);
-        else learn_row<4>(P, r, xs, ws, acc, red, yt);
+        if (b == 1) learn_row<1>(P, r, xs, ws, acc, red, yt, tf);
+        else if (b == 2) learn_row<2>(P, r, xs, ws, acc, red, yt, tf);
+        else learn_row<4>(P, r, xs, ws, acc, red, yt, tf);
     }
 }
 
@@ -170,7 +211,7 @@ extern "C" lowra_status lowra_learn_codebooks(const lowra_layout* layout, const 
     if (iterations < 0 || iterations > 1000) return LOWRA_ERR_SHAPE;
     if (!aligned16(W_dev) || !aligned16(maps_dev) || !aligned16(thresholds_dev)) return LOWRA_ERR_ALIGN;
     const size_t smem = (32 + 2 * 16 * kLearnWarps + 2 * 16 * kLearnThreads) * sizeof(double) +
-                        ((size_t)layout->K + (size_t)layout->K / kBlock) * sizeof(float);
+                        ((size_t)layout->K + (size_t)layout->K / kBlock + 16) * sizeof(float);
     if (smem > 200 * 1024) return LOWRA_ERR_SHAPE;   // the row has to fit into shared memory (K <= 40960)
     st = check_device();
     if (st != LOWRA_OK) return st;

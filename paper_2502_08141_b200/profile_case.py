@@ -3,6 +3,7 @@
     python -m paper_2502_08141_b200.profile_case forward     # fused forward,  N = K = 4096, 2048 tokens, rank 64
     python -m paper_2502_08141_b200.profile_case backward    # fused backward-input, same shapes
     python -m paper_2502_08141_b200.profile_case codec       # decode + encode of an 11008 x 4096 matrix
+    python -m paper_2502_08141_b200.profile_case learn       # codebook learner, 4096 x 4096, 10 iterations
 
 Each case runs its call three times on seeded synthetic inputs (config-3 precision mix) and checks the
 device status word; a few hundred MB on the device at most.
@@ -15,8 +16,8 @@ import torch
 
 import synth_inputs as si
 
-from . import (Layout, lowra_decode, lowra_device_status, lowra_encode, lowra_lora_backward_input,
-               lowra_lora_forward, lowra_workspace_bytes)
+from . import (Layout, lowra_decode, lowra_device_status, lowra_encode, lowra_learn_codebooks,
+               lowra_lora_backward_input, lowra_lora_forward, lowra_workspace_bytes)
 
 
 def main(case: str) -> None:
@@ -29,6 +30,18 @@ def main(case: str) -> None:
     gen = torch.Generator(device="cuda").manual_seed(1)
     W = torch.randn(N, K, device="cuda", generator=gen) * 0.02
     maps_d, thr_d = torch.from_numpy(maps).cuda(), torch.from_numpy(thr).cuda()
+    if case == "learn":
+        import numpy as np
+        y0 = np.zeros((3, 16)); t0 = np.zeros((3, 16))   # equally spaced starting levels
+        for c, b in enumerate((1, 2, 4)):
+            lv = np.linspace(-1.0, 1.0, 1 << b)
+            y0[c, :lv.size] = lv
+            t0[c, :lv.size - 1] = 0.5 * (lv[:-1] + lv[1:])
+        for _ in range(3):
+            lowra_learn_codebooks(layout, W, y0, t0, 10)
+        torch.cuda.synchronize()
+        print("learn ok")
+        return
     packed, absmax = lowra_encode(layout, W, thr_d)
     if case == "codec":
         out = torch.empty(N, K, dtype=torch.bfloat16, device="cuda")
