@@ -233,3 +233,15 @@ def lora_backward_input(W_hat_bf16: np.ndarray, dY_bf16: np.ndarray, A_bf16: np.
     A = bf16_to_f64(A_bf16)
     B = bf16_to_f64(B_bf16)
     return dY @ W + float(s) * ((dY @ B.T) @ A.T)
+
+
+def lora_backward_adapters(X_bf16: np.ndarray, dY_bf16: np.ndarray, A_bf16: np.ndarray, B_bf16: np.ndarray,
+                           s: float):
+    """Gradients of the trainable low-rank factors (Section 3: only they are trained) of
+    Y = X . W_hat^T + s * (X . A) . B for the output gradient dY:
+        dA = s * X^T . (dY . B^T)  [K, r],      dB = s * (X . A)^T . dY  [r, N],   float64."""
+    X = bf16_to_f64(X_bf16)       # [M, K]
+    dY = bf16_to_f64(dY_bf16)     # [M, N]
+    A = bf16_to_f64(A_bf16)       # [K, r]
+    B = bf16_to_f64(B_bf16)       # [r, N]
+    return float(s) * (X.T @ (dY @ B.T)), float(s) * ((X @ A).T @ dY)

@@ -183,3 +183,41 @@ def test_backward_is_the_adjoint_of_forward():
     lhs = np.sum(f(dY) * oracle.lora_forward(W, X, A, B, 2.0))
     rhs = np.sum(oracle.lora_backward_input(W, dY, A, B, 2.0) * f(X))
     assert abs(lhs - rhs) <= 1e-10 * abs(lhs)
+
+
+def test_adapter_gradients_are_the_derivatives_of_the_forward():
+    """Y is linear in A for fixed B (and in B for fixed A), so for any direction D:
+    <dY, forward(A + D) - forward(A)> = <dA, D> exactly (up to fp64 rounding); same for B.
+    Also a brute-force triple loop on a tiny case, and the trivial cases s = 0, dY = 0."""
+    rng = np.random.default_rng(5)
+    M, K, N, r, s = 12, 16, 10, 4, 1.5
+    bf = lambda a: oracle.f32_to_bf16(a.astype(np.float32))
+    f = oracle.bf16_to_f64
+    X, dY = bf(rng.standard_normal((M, K))), bf(rng.standard_normal((M, N)))
+    A, B = bf(rng.standard_normal((K, r))), bf(rng.standard_normal((r, N)))
+    W = bf(rng.standard_normal((N, K)))
+    dA, dB = oracle.lora_backward_adapters(X, dY, A, B, s)
+    assert dA.shape == (K, r) and dB.shape == (r, N)
+    DA, DB = bf(rng.standard_normal((K, r))), bf(rng.standard_normal((r, N)))
+    # directional derivatives through the forward oracle (exactly representable perturbed factors)
+    A2, B2 = bf(f(A) + f(DA)), bf(f(B) + f(DB))
+    dirA, dirB = f(A2) - f(A), f(B2) - f(B)
+    y0 = oracle.lora_forward(W, X, A, B, s)
+    lhsA = np.sum(f(dY) * (oracle.lora_forward(W, X, A2, B, s) - y0))
+    lhsB = np.sum(f(dY) * (oracle.lora_forward(W, X, A, B2, s) - y0))
+    assert abs(lhsA - np.sum(dA * dirA)) <= 1e-10 * abs(lhsA)
+    assert abs(lhsB - np.sum(dB * dirB)) <= 1e-10 * abs(lhsB)
+    # definition written out with loops
+    Xf, dYf, Af, Bf = f(X), f(dY), f(A), f(B)
+    dA_loop = np.zeros((K, r)); dB_loop = np.zeros((r, N))
+    for k in range(K):
+        for j in range(r):
+            dA_loop[k, j] = s * sum(Xf[m, k] * sum(dYf[m, n] * Bf[j, n] for n in range(N)) for m in range(M))
+    for j in range(r):
+        for n in range(N):
+            dB_loop[j, n] = s * sum(sum(Xf[m, k] * Af[k, j] for k in range(K)) * dYf[m, n] for m in range(M))
+    assert np.allclose(dA, dA_loop, rtol=1e-12, atol=1e-12) and np.allclose(dB, dB_loop, rtol=1e-12, atol=1e-12)
+    z = oracle.lora_backward_adapters(X, dY, A, B, 0.0)
+    assert not z[0].any() and not z[1].any()
+    z = oracle.lora_backward_adapters(X, bf(np.zeros((M, N))), A, B, s)
+    assert not z[0].any() and not z[1].any()
