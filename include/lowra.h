@@ -135,6 +135,30 @@ lowra_status lowra_lora_backward_input(const lowra_layout* layout, const uint8_t
                                        const uint16_t* B_dev, int32_t r, float s, uint16_t* dX_dev,
                                        void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/* Bytes of device scratch that lowra_lora_backward_adapters needs for M tokens and rank r (0 if the
+ * arguments are invalid).  The first 256 bytes hold the device status word. */
+size_t lowra_adapter_workspace_bytes(int32_t M, int32_t r);
+
+/*
+ * Gradients of the trainable low-rank factors of the same layer (Section 3: the base weights stay
+ * frozen, only the adapters are trained).  With Y = X . deq(Wq)^T + s * (X . A) . B:
+ *     dA = s * X^T . (dY . B^T)      [K, r]
+ *     dB = s * (X . A)^T . dY        [r, N]
+ * The quantised weight does not enter.  The two down-projections s X A and s dY B^T are rounded to
+ * bf16 once (as in the forward / backward-input calls), the contractions over the tokens accumulate
+ * in fp32, the results are rounded to bf16.
+ *   X_dev bf16 [M, K];  dY_dev bf16 [M, N];  A_dev bf16 [K, r];  B_dev bf16 [r, N];
+ *   dA_dev bf16 [K, r] (out);  dB_dev bf16 [r, N] (out); all row-major, device, 16-byte aligned.
+ *   r in {16, 32, ..., 128};  K % 8 == 0, N % 8 == 0, M >= 1 (LOWRA_ERR_SHAPE otherwise).
+ *   workspace_dev: >= lowra_adapter_workspace_bytes(M, r) bytes, 256-byte aligned, contents
+ *   overwritten; lowra_device_status reads its status word.
+ */
+lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, const uint16_t* dY_dev, int32_t M,
+                                          int32_t K, int32_t N, const uint16_t* A_dev,
+                                          const uint16_t* B_dev, int32_t r, float s, uint16_t* dA_dev,
+                                          uint16_t* dB_dev, void* workspace_dev, size_t workspace_bytes,
+                                          void* stream);
+
 /*
  * Synchronises `stream` and returns the status word that the last forward / backward call wrote
  * into its workspace: LOWRA_OK, or LOWRA_ERR_TIMEOUT if a bounded wait inside a kernel ran out

@@ -27,7 +27,8 @@ LOWRA_STATIC_SCRATCH_BYTES = 8 << 20
 EXPORTS = (
     "lowra_status_string", "lowra_plan", "lowra_encode", "lowra_decode", "lowra_workspace_bytes",
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
-    "lowra_lora_forward_static", "lowra_learn_codebooks",
+    "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
+    "lowra_lora_backward_adapters",
 )
 
 
@@ -80,6 +81,11 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_forward_static.restype = ctypes.c_int
         L.lowra_learn_codebooks.argtypes = [lp, vp, vp, vp, i32, vp, vp, vp]
         L.lowra_learn_codebooks.restype = ctypes.c_int
+        L.lowra_adapter_workspace_bytes.argtypes = [i32, i32]
+        L.lowra_adapter_workspace_bytes.restype = ctypes.c_size_t
+        L.lowra_lora_backward_adapters.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, ctypes.c_float, vp, vp, vp,
+                                                   ctypes.c_size_t, vp]
+        L.lowra_lora_backward_adapters.restype = ctypes.c_int
         L.lowra_device_status.argtypes = [vp, vp]
         L.lowra_device_status.restype = ctypes.c_int
         L.lowra_dense_nt.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
@@ -290,6 +296,36 @@ def lowra_lora_backward_input(layout: Layout, packed, absmax, maps, dY, A, B, s:
                                            workspace.numel(), _stream(stream))
     _check(code, "lowra_lora_backward_input")
     return dX
+
+
+def lowra_adapter_workspace_bytes(M: int, r: int) -> int:
+    return int(lib().lowra_adapter_workspace_bytes(int(M), int(r)))
+
+
+def lowra_lora_backward_adapters(X, dY, A, B, s: float, dA: Optional[torch.Tensor] = None,
+                                 dB: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                                 stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """dA = s X^T (dY B^T) [K,r] and dB = s (X A)^T dY [r,N]; all operands bf16 on the device."""
+    for t, n in ((X, "X"), (dY, "dY"), (A, "A"), (B, "B")):
+        _dev(t, torch.bfloat16, n)
+    M, K = int(X.shape[0]), int(X.shape[1])
+    N, r = int(dY.shape[1]), int(A.shape[1])
+    if tuple(dY.shape) != (M, N) or tuple(A.shape) != (K, r) or tuple(B.shape) != (r, N):
+        raise ValueError("shape mismatch")
+    if dA is None:
+        dA = torch.empty((K, r), dtype=torch.bfloat16, device=X.device)
+    if dB is None:
+        dB = torch.empty((r, N), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        nbytes = lowra_adapter_workspace_bytes(M, r)
+        if nbytes == 0:
+            raise LowraError(LOWRA_ERR_SHAPE, "lowra_adapter_workspace_bytes")
+        workspace = torch.empty(nbytes, dtype=torch.uint8, device=X.device)
+    code = lib().lowra_lora_backward_adapters(_ptr(X), _ptr(dY), M, K, N, _ptr(A), _ptr(B), r, ctypes.c_float(s),
+                                              _ptr(dA), _ptr(dB), _ptr(workspace), workspace.numel(),
+                                              _stream(stream))
+    _check(code, "lowra_lora_backward_adapters")
+    return dA, dB
 
 
 def lowra_device_status(workspace: torch.Tensor, stream=None) -> int:

@@ -149,6 +149,62 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     return launch_fused(backward ? kModeBackward : kModeForward, G, tmB, tmT, tmFt, tmFl, stream);
 }
 
+// Down-projection alone: T = s act . F (forward form, F = A [C, r]) or U = s act . F^T (backward form, F = B [r, C]),
+// bf16 [M, rp], computed by the down-projection tiles of the fused kernel (a launch without weight tiles).
+lowra_status run_down(bool backward, const uint16_t* act, int M, int C, const uint16_t* F, int r, float s, uint16_t* T,
+                      uint32_t* flags, uint32_t* status, bool clear_status, cudaStream_t stream) {
+    const int rp = (r + 63) / 64 * 64;
+    const int tiles_t = (M + kTileT - 1) / kTileT;
+    PrepParams P;
+    memset(&P, 0, sizeof(P));
+    P.N = 0;                 // nothing to deal: the prologue only clears the status word and the flags
+    P.group = 128;
+    P.status = clear_status ? status : nullptr;
+    P.flags = flags;
+    P.n_flags = tiles_t + kCluster;
+    P.blocks = 1;
+    lowra_status st = launch_prep(P, stream);
+    if (st != LOWRA_OK) return st;
+    GemmParams G;
+    memset(&G, 0, sizeof(G));
+    G.T = T;
+    G.flags = flags;
+    G.status = status;
+    G.s = s;
+    G.rp = rp;
+    G.r = r;
+    G.M = M;
+    G.C = C;
+    G.main_blocks = (C + kTileC - 1) / kTileC;
+    G.lora_blocks = rp / kTileC;
+    G.tiles_r = 0;
+    G.tiles_t = tiles_t;
+    CUtensorMap tmB, tmFt;
+    if (!make_map(&tmB, act, (uint64_t)M, (uint64_t)C, (uint64_t)C, kTileT)) return LOWRA_ERR_CUDA;
+    if (!backward) {
+        if (!make_map(&tmFt, F, (uint64_t)C, (uint64_t)r, (uint64_t)r, 64)) return LOWRA_ERR_CUDA;
+    } else {
+        if (!make_map(&tmFt, F, (uint64_t)r, (uint64_t)C, (uint64_t)C, kTileR)) return LOWRA_ERR_CUDA;
+    }
+    return launch_fused(backward ? kModeBackward : kModeForward, G, tmB, tmB, tmFt, tmB, stream);
+}
+
+struct AdapterWorkspace {
+    size_t off_T, off_U, off_flagsT, off_flagsU, total;
+    int rp;
+};
+AdapterWorkspace plan_adapter_workspace(int M, int r) {
+    AdapterWorkspace w;
+    w.rp = (r + 63) / 64 * 64;
+    const size_t flag_bytes = align256((size_t)((M + kTileT - 1) / kTileT + kCluster) * 4);
+    w.off_T = kStatusBytes;
+    w.off_U = w.off_T + align256((size_t)M * w.rp * 2);
+    w.off_flagsT = w.off_U + align256((size_t)M * w.rp * 2);
+    w.off_flagsU = w.off_flagsT + flag_bytes;
+    w.total = w.off_flagsU + flag_bytes;
+    return w;
+}
+
 __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
 
 }  // namespace
@@ -231,6 +287,47 @@ extern "C" lowra_status lowra_lora_forward_static(const lowra_layout* layout, co
             cudaSuccess)
         return LOWRA_ERR_CUDA;
     return LOWRA_OK;
+}
+
+extern "C" size_t lowra_adapter_workspace_bytes(int32_t M, int32_t r) {
+    using namespace lowra;
+    if (M < 1 || !rank_ok(r)) return 0;
+    return plan_adapter_workspace(M, r).total;
+}
+
+extern "C" lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, const uint16_t* dY_dev, int32_t M, int32_t K,
+                                                     int32_t N, const uint16_t* A_dev, const uint16_t* B_dev, int32_t r,
+                                                     float s, uint16_t* dA_dev, uint16_t* dB_dev, void* workspace_dev,
+                                                     size_t workspace_bytes, void* stream_v) {
+    using namespace lowra;
+    if (!X_dev || !dY_dev || !A_dev || !B_dev || !dA_dev || !dB_dev || !workspace_dev) return LOWRA_ERR_NULL;
+    if (M < 1 || K < 8 || N < 8 || K % 8 != 0 || N % 8 != 0 || !rank_ok(r)) return LOWRA_ERR_SHAPE;
+    if (!aligned16(X_dev) || !aligned16(dY_dev) || !aligned16(A_dev) || !aligned16(B_dev) || !aligned16(dA_dev) ||
+        !aligned16(dB_dev))
+        return LOWRA_ERR_ALIGN;
+    const AdapterWorkspace w = plan_adapter_workspace(M, r);
+    if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) != 0) return LOWRA_ERR_WORKSPACE;
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    cudaStream_t stream = (cudaStream_t)stream_v;
+    unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
+    uint32_t* status = reinterpret_cast<uint32_t*>(ws);
+    uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
+    uint16_t* U = reinterpret_cast<uint16_t*>(ws + w.off_U);
+    // T = s X A and U = s dY B^T; the first launch clears the status word, the later ones only ever set it
+    st = run_down(false, X_dev, M, K, A_dev, r, s, T, reinterpret_cast<uint32_t*>(ws + w.off_flagsT), status, true, stream);
+    if (st != LOWRA_OK) return st;
+    st = run_down(true, dY_dev, M, N, B_dev, r, s, U, reinterpret_cast<uint32_t*>(ws + w.off_flagsU), status, false, stream);
+    if (st != LOWRA_OK) return st;
+    // dA = X^T U [K, r], dB = (dY^T T)^T [r, N]
+    CUtensorMap tmX, tmdY, tmT, tmU;
+    if (!make_map(&tmX, X_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, 64)) return LOWRA_ERR_CUDA;
+    if (!make_map(&tmdY, dY_dev, (uint64_t)M, (uint64_t)N, (uint64_t)N, 64)) return LOWRA_ERR_CUDA;
+    if (!make_map(&tmT, T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, 64)) return LOWRA_ERR_CUDA;
+    if (!make_map(&tmU, U, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, 64)) return LOWRA_ERR_CUDA;
+    st = launch_grad(tmX, tmU, dA_dev, status, K, M, r, w.rp, false, stream);
+    if (st != LOWRA_OK) return st;
+    return launch_grad(tmdY, tmT, dB_dev, status, N, M, r, w.rp, true, stream);
 }
 
 extern "C" lowra_status lowra_device_status(const void* workspace_dev, void* stream) {

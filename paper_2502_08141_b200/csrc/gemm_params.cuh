@@ -103,4 +103,8 @@ static_assert(kGemmSmemBytes <= 232448, "227 KB of shared memory per CTA");
 lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
                           const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream);
 
+// dA = X^T . U or dB = (dY^T . T)^T, see gemm_grad.cu
+lowra_status launch_grad(const CUtensorMap& tmP, const CUtensorMap& tmQ, uint16_t* out, uint32_t* status, int R, int M, int r,
+                         int rp, bool transposed, cudaStream_t stream);
+
 }  // namespace lowra

@@ -98,6 +98,26 @@ def test_validation_runs_before_any_device_work(lib):
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, None, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_NULL
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, init, init, -1, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096 + 4, init, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_ALIGN
+    # adapter gradients: X, dY, M, K, N, A, B, r, s, dA, dB, workspace, bytes, stream
+    big = 1 << 30
+    assert L.lowra_adapter_workspace_bytes(0, 16) == 0
+    assert L.lowra_adapter_workspace_bytes(16, 20) == 0
+    need = L.lowra_adapter_workspace_bytes(300, 48)
+    assert need >= 256 + 2 * 300 * 64 * 2
+    ok = [4096, 4096, 300, 256, 512, 4096, 4096, 48, ctypes.c_float(1.0), 4096, 4096, 4096, big, None]
+    def call(**kw):
+        a = list(ok)
+        for i, v in kw.items():
+            a[int(i[1:])] = v
+        return L.lowra_lora_backward_adapters(*a)
+    assert call(_0=None) == lib.LOWRA_ERR_NULL
+    assert call(_10=None) == lib.LOWRA_ERR_NULL
+    assert call(_2=0) == lib.LOWRA_ERR_SHAPE
+    assert call(_3=100) == lib.LOWRA_ERR_SHAPE       # K not a multiple of 8
+    assert call(_7=8) == lib.LOWRA_ERR_SHAPE
+    assert call(_5=4096 + 2) == lib.LOWRA_ERR_ALIGN
+    assert call(_12=need - 1) == lib.LOWRA_ERR_WORKSPACE
+    assert call(_11=4096 + 16) == lib.LOWRA_ERR_WORKSPACE
     lay.K = 128 * 400                                                    # a row no longer fits into shared memory
     lay.packed_bytes = 8 * lay.K // 8
     lay.seg_off[1] = lay.seg_off[2] = lay.packed_bytes
