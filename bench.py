@@ -389,6 +389,31 @@ def run_gpu(args):
                                       "element_passes_per_s": elems * T_learn / (ms_learn * 1e-3),
                                       "note": "not part of the step; algorithmic bytes = one read of W (4 B per element)"}}
 
+        # the gradients of the low-rank factors (the other half of a training step's backward pass)
+        ws_ad = torch.empty(lw.lowra_adapter_workspace_bytes(M, r), dtype=torch.uint8, device="cuda")
+        grads = [(torch.empty_like(d["A"]), torch.empty_like(d["B"])) for d in dev]
+
+        def adapters():
+            for d, (gA, gB) in zip(dev, grads):
+                lw.lowra_lora_backward_adapters(act_dev[d["m"]["K"]], act_dev[d["m"]["N"]], d["A"], d["B"], s,
+                                                dA=gA, dB=gB, workspace=ws_ad)
+        adapters()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        adapters()
+        b.record(stream)
+        torch.cuda.synchronize()
+        if lw.lowra_device_status(ws_ad) != 0:
+            raise SystemExit("device status after the adapter gradients")
+        ms_ad = a.elapsed_time(b)
+        ad_bytes = sum(2.0 * M * (d["m"]["K"] + d["m"]["N"]) for d in dev)      # X and dY once, bf16
+        ad_flops = sum(4.0 * M * r * (d["m"]["K"] + d["m"]["N"]) for d in dev)
+        extras["adapter_gradients"] = {"ms": ms_ad, "GB/s": ad_bytes / (ms_ad * 1e-3) / 1e9,
+                                       "frac_hbm": ad_bytes / (ms_ad * 1e-3) / 1e9 / P["hbm"],
+                                       "TFLOP/s": ad_flops / (ms_ad * 1e-3) / 1e12, "launches": 6 * len(dev),
+                                       "note": "not part of the step; algorithmic bytes = X and dY read once"}
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = cpu_baseline_sample()

@@ -149,59 +149,17 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     return launch_fused(backward ? kModeBackward : kModeForward, G, tmB, tmT, tmFt, tmFl, stream);
 }
 
-// Down-projection alone: T = s act . F (forward form, F = A [C, r]) or U = s act . F^T (backward form, F = B [r, C]),
-// bf16 [M, rp], computed by the down-projection tiles of the fused kernel (a launch without weight tiles).
-lowra_status run_down(bool backward, const uint16_t* act, int M, int C, const uint16_t* F, int r, float s, uint16_t* T,
-                      uint32_t* flags, uint32_t* status, bool clear_status, cudaStream_t stream) {
-    const int rp = (r + 63) / 64 * 64;
-    const int tiles_t = (M + kTileT - 1) / kTileT;
-    PrepParams P;
-    memset(&P, 0, sizeof(P));
-    P.N = 0;                 // nothing to deal: the prologue only clears the status word and the flags
-    P.group = 128;
-    P.status = clear_status ? status : nullptr;
-    P.flags = flags;
-    P.n_flags = tiles_t + kCluster;
-    P.blocks = 1;
-    lowra_status st = launch_prep(P, stream);
-    if (st != LOWRA_OK) return st;
-    GemmParams G;
-    memset(&G, 0, sizeof(G));
-    G.T = T;
-    G.flags = flags;
-    G.status = status;
-    G.s = s;
-    G.rp = rp;
-    G.r = r;
-    G.M = M;
-    G.C = C;
-    G.main_blocks = (C + kTileC - 1) / kTileC;
-    G.lora_blocks = rp / kTileC;
-    G.tiles_r = 0;
-    G.tiles_t = tiles_t;
-    CUtensorMap tmB, tmFt;
-    if (!make_map(&tmB, act, (uint64_t)M, (uint64_t)C, (uint64_t)C, kTileT)) return LOWRA_ERR_CUDA;
-    if (!backward) {
-        if (!make_map(&tmFt, F, (uint64_t)C, (uint64_t)r, (uint64_t)r, 64)) return LOWRA_ERR_CUDA;
-    } else {
-        if (!make_map(&tmFt, F, (uint64_t)r, (uint64_t)C, (uint64_t)C, kTileR)) return LOWRA_ERR_CUDA;
-    }
-    return launch_fused(backward ? kModeBackward : kModeForward, G, tmB, tmB, tmFt, tmB, stream);
-}
-
+// scratch of the adapter-gradient call: status word | T = s X A | U = s dY B^T  (bf16 [M, rp] each)
 struct AdapterWorkspace {
-    size_t off_T, off_U, off_flagsT, off_flagsU, total;
+    size_t off_T, off_U, total;
     int rp;
 };
 AdapterWorkspace plan_adapter_workspace(int M, int r) {
     AdapterWorkspace w;
     w.rp = (r + 63) / 64 * 64;
-    const size_t flag_bytes = align256((size_t)((M + kTileT - 1) / kTileT + kCluster) * 4);
     w.off_T = kStatusBytes;
     w.off_U = w.off_T + align256((size_t)M * w.rp * 2);
-    w.off_flagsT = w.off_U + align256((size_t)M * w.rp * 2);
-    w.off_flagsU = w.off_flagsT + flag_bytes;
-    w.total = w.off_flagsU + flag_bytes;
+    w.total = w.off_U + align256((size_t)M * w.rp * 2);
     return w;
 }
 
@@ -314,20 +272,37 @@ extern "C" lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, cons
     uint32_t* status = reinterpret_cast<uint32_t*>(ws);
     uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
     uint16_t* U = reinterpret_cast<uint16_t*>(ws + w.off_U);
-    // T = s X A and U = s dY B^T; the first launch clears the status word, the later ones only ever set it
-    st = run_down(false, X_dev, M, K, A_dev, r, s, T, reinterpret_cast<uint32_t*>(ws + w.off_flagsT), status, true, stream);
+    clear_status_kernel<<<1, 1, 0, stream>>>(status);
+    const int rp = w.rp;
+    CUtensorMap tmX, tmXt, tmdY, tmdYt, tmA, tmB, tmT, tmU;
+    if (!make_map(&tmX, X_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, 128) ||      // rows of 64 features (K-major)
+        !make_map(&tmXt, X_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, 64) ||      // 64 tokens x 64 features (MN-major)
+        !make_map(&tmdY, dY_dev, (uint64_t)M, (uint64_t)N, (uint64_t)N, 128) ||
+        !make_map(&tmdYt, dY_dev, (uint64_t)M, (uint64_t)N, (uint64_t)N, 64) ||
+        !make_map(&tmA, A_dev, (uint64_t)K, (uint64_t)r, (uint64_t)r, 64) ||       // 64 features x 64 ranks (MN-major)
+        !make_map(&tmB, B_dev, (uint64_t)r, (uint64_t)N, (uint64_t)N, (uint32_t)rp) ||   // ranks x 64 channels (K-major)
+        !make_map(&tmT, T, (uint64_t)M, (uint64_t)rp, (uint64_t)rp, 64) ||
+        !make_map(&tmU, U, (uint64_t)M, (uint64_t)rp, (uint64_t)rp, 64))
+        return LOWRA_ERR_CUDA;
+    SkinnyArgs a;
+    memset(&a, 0, sizeof(a));
+    a.status = status;
+    a.rp = rp;
+    // T = s X A: rows = tokens, contraction over the K input features
+    a.out = T; a.R = M; a.C = K; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 1; a.transposed = 0; a.scale = s;
+    st = launch_skinny(tmX, tmA, a, stream);
     if (st != LOWRA_OK) return st;
-    st = run_down(true, dY_dev, M, N, B_dev, r, s, U, reinterpret_cast<uint32_t*>(ws + w.off_flagsU), status, false, stream);
+    // U = s dY B^T: rows = tokens, contraction over the N output channels
+    a.out = U; a.C = N; a.b_mn = 0;
+    st = launch_skinny(tmdY, tmB, a, stream);
     if (st != LOWRA_OK) return st;
-    // dA = X^T U [K, r], dB = (dY^T T)^T [r, N]
-    CUtensorMap tmX, tmdY, tmT, tmU;
-    if (!make_map(&tmX, X_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, 64)) return LOWRA_ERR_CUDA;
-    if (!make_map(&tmdY, dY_dev, (uint64_t)M, (uint64_t)N, (uint64_t)N, 64)) return LOWRA_ERR_CUDA;
-    if (!make_map(&tmT, T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, 64)) return LOWRA_ERR_CUDA;
-    if (!make_map(&tmU, U, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, 64)) return LOWRA_ERR_CUDA;
-    st = launch_grad(tmX, tmU, dA_dev, status, K, M, r, w.rp, false, stream);
+    // dA = X^T U: rows = input features, contraction over the tokens
+    a.out = dA_dev; a.R = K; a.C = M; a.n_cols = r; a.ld_out = r; a.a_mn = 1; a.b_mn = 1; a.scale = 1.0f;
+    st = launch_skinny(tmXt, tmU, a, stream);
     if (st != LOWRA_OK) return st;
-    return launch_grad(tmdY, tmT, dB_dev, status, N, M, r, w.rp, true, stream);
+    // dB = (dY^T T)^T: rows = output channels, written transposed
+    a.out = dB_dev; a.R = N; a.ld_out = N; a.transposed = 1;
+    return launch_skinny(tmdYt, tmT, a, stream);
 }
 
 extern "C" lowra_status lowra_device_status(const void* workspace_dev, void* stream) {

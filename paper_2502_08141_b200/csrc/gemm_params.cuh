@@ -103,8 +103,20 @@ static_assert(kGemmSmemBytes <= 232448, "227 KB of shared memory per CTA");
 lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
                           const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream);
 
-// dA = X^T . U or dB = (dY^T . T)^T, see gemm_grad.cu
-lowra_status launch_grad(const CUtensorMap& tmP, const CUtensorMap& tmQ, uint16_t* out, uint32_t* status, int R, int M, int r,
-                         int rp, bool transposed, cudaStream_t stream);
+// One skinny product D [R, rp] = P . Q (see gemm_grad.cu), written in bf16 as out [R, ld_out] or, transposed,
+// as out [n_cols, ld_out].
+struct SkinnyArgs {
+    uint16_t* out;
+    uint32_t* status;
+    int R;            // rows of D
+    int C;            // length of the contraction
+    int rp;           // columns of D (64 or 128)
+    int n_cols;       // columns of D that are written (a multiple of 16)
+    int ld_out;
+    int a_mn, b_mn;   // 1: the row (column) index of P (Q) is the contiguous one in memory
+    int transposed;
+    float scale;
+};
+lowra_status launch_skinny(const CUtensorMap& tmP, const CUtensorMap& tmQ, const SkinnyArgs& a, cudaStream_t stream);
 
 }  // namespace lowra

@@ -294,6 +294,18 @@ __device__ __forceinline__ uint32_t ld_relaxed_cluster(const uint32_t* p) {   //
     asm volatile("ld.relaxed.cluster.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
     return v;
 }
+// Plain loads from the shared memory of any CTA of the cluster (address from map_to_cta); ordered by the
+// cluster barrier around them.
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t caddr) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(caddr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t caddr) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(caddr) : "memory");
+    return v;
+}
 // Arrive (count times) on an mbarrier of any CTA of the cluster.  Relaxed: it orders nothing by itself (the data
 // it announces travels as bulk copies that the same barrier counts in bytes).
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t caddr, uint32_t count) {

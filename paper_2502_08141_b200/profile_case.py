@@ -4,6 +4,7 @@
     python -m paper_2502_08141_b200.profile_case backward    # fused backward-input, same shapes
     python -m paper_2502_08141_b200.profile_case codec       # decode + encode of an 11008 x 4096 matrix
     python -m paper_2502_08141_b200.profile_case learn       # codebook learner, 4096 x 4096, 10 iterations
+    python -m paper_2502_08141_b200.profile_case adapters    # gradients of the low-rank factors, 4096 x 11008, 4096 tokens
 
 Each case runs its call three times on seeded synthetic inputs (config-3 precision mix) and checks the
 device status word; a few hundred MB on the device at most.
@@ -16,11 +17,31 @@ import torch
 
 import synth_inputs as si
 
-from . import (Layout, lowra_decode, lowra_device_status, lowra_encode, lowra_learn_codebooks,
-               lowra_lora_backward_input, lowra_lora_forward, lowra_workspace_bytes)
+from . import (Layout, lowra_adapter_workspace_bytes, lowra_decode, lowra_device_status, lowra_encode, lowra_learn_codebooks,
+               lowra_lora_backward_adapters, lowra_lora_backward_input, lowra_lora_forward, lowra_workspace_bytes)
+
+
+def adapters() -> None:
+    cfg = si.config(3)
+    N, K, M, r = 11008, 4096, 4096, cfg.rank
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    X = torch.randn(M, K, device="cuda", generator=gen).bfloat16()
+    dY = torch.randn(M, N, device="cuda", generator=gen).bfloat16()
+    A = (torch.randn(K, r, device="cuda", generator=gen) * 0.01).bfloat16()
+    B = (torch.randn(r, N, device="cuda", generator=gen) * 0.01).bfloat16()
+    ws = torch.empty(lowra_adapter_workspace_bytes(M, r), dtype=torch.uint8, device="cuda")
+    for _ in range(3):
+        lowra_lora_backward_adapters(X, dY, A, B, cfg.s, workspace=ws)
+    status = lowra_device_status(ws)
+    print("adapters status", status)
+    if status != 0:
+        raise SystemExit(1)
 
 
 def main(case: str) -> None:
+    if case == "adapters":
+        adapters()
+        return
     cfg = si.config(3)
     N, K = (11008, 4096) if case == "codec" else (4096, 4096)
     M, r, s = 2048, cfg.rank, cfg.s
