@@ -28,7 +28,7 @@ constexpr uint32_t kSkinnySmemP = 128 * 64 * 2;        // 16 KB of P per stage
 constexpr uint32_t kSkinnySmemBytes = kSkinnyRing + 256;
 constexpr int kSkinnyMaxStages = 4;
 constexpr int kSkinnyMaxSplit = 8;                     // portable cluster size
-constexpr int kSkinnyTargetCtas = 2 * kNumSMs * 3 / 4; // grow the split until the grid has about this many CTAs
+constexpr int kSkinnySlots = 2 * kNumSMs - 2 * 16;      // CTAs resident at once (two per SM, less what clusters leave unused)
 
 struct SkinnyBarriers {
     uint64_t full[kSkinnyMaxStages];
@@ -179,14 +179,28 @@ skinny_kernel(const SkinnyArgs P, const int S, const __grid_constant__ CUtensorM
                 }
             }
         } else {
-            // out [n_cols, ld_out] = D^T: neighbouring threads take neighbouring rows of D = neighbouring addresses
-            for (int u = t; u < rows_per * P.n_cols; u += 128) {
-                const int row = row_base + u % rows_per, col = u / rows_per;
+            // out [n_cols, ld_out] = D^T.  A warp takes 8 rows x 16 columns of D: its loads read whole 64-byte runs of
+            // a row, its stores write 8 neighbouring elements (rows of D) of 16 rows of out.
+            const int c4n = P.rp / 4;
+            const int lane_row = lane & 7, lane_c4 = lane >> 3;
+            const int units = (rows_per / 8) * (c4n / 4);          // 8 x 16 patches of this CTA's rows
+            for (int u = warp - 2; u < units; u += 4) {
+                const int row = row_base + (u % (rows_per / 8)) * 8 + lane_row;
+                const int col = ((u / (rows_per / 8)) * 4 + lane_c4) * 4;
                 const uint32_t addr = part_addr + (uint32_t)(row * pstride + col) * 4u;
-                float acc = 0.f;
-                for (int p = 0; p < S; ++p) acc += ptx::ld_cluster_f32(ptx::map_to_cta(addr, (uint32_t)p));
+                float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int p = 0; p < S; ++p) {
+                    const float4 v = ptx::ld_cluster_f4(ptx::map_to_cta(addr, (uint32_t)p));
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
                 const int grow = r0 + row;
-                if (grow < P.R) P.out[(size_t)col * P.ld_out + grow] = (uint16_t)pack_bf16x2(acc * P.scale, 0.0f);
+                if (grow < P.R && col < P.n_cols) {
+                    uint16_t* dst = P.out + (size_t)col * P.ld_out + grow;
+                    dst[0] = (uint16_t)pack_bf16x2(acc.x * P.scale, 0.0f);
+                    dst[(size_t)P.ld_out] = (uint16_t)pack_bf16x2(acc.y * P.scale, 0.0f);
+                    dst[2 * (size_t)P.ld_out] = (uint16_t)pack_bf16x2(acc.z * P.scale, 0.0f);
+                    dst[3 * (size_t)P.ld_out] = (uint16_t)pack_bf16x2(acc.w * P.scale, 0.0f);
+                }
             }
         }
     }
@@ -208,8 +222,15 @@ lowra_status launch_skinny(const CUtensorMap& tmP, const CUtensorMap& tmQ, const
         configured = true;
     }
     const int tiles = (a.R + 127) / 128, n_blocks = (a.C + 63) / 64;
+    // split of the contraction: the one with the shortest estimated run = waves of CTAs x (blocks per CTA + a fixed
+    // cost of set-up, pipeline fill and reduction, about six blocks' worth); every slice keeps four blocks or more
     int S = 1;
-    while (S < kSkinnyMaxSplit && tiles * S < kSkinnyTargetCtas && n_blocks >= 4 * S) S *= 2;
+    long best = -1;
+    for (int c = 1; c <= kSkinnyMaxSplit && (c == 1 || n_blocks >= 4 * c); c *= 2) {
+        const long waves = ((long)tiles * c + kSkinnySlots - 1) / kSkinnySlots;
+        const long cost = waves * ((n_blocks + c - 1) / c + 6);
+        if (best < 0 || cost < best) { best = cost; S = c; }
+    }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
