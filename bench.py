@@ -295,9 +295,12 @@ def run_gpu(args):
     flops_step = sum(2 * gemm_flops(M, d["m"]["N"], d["m"]["K"], r) for d in dev)
     value = aggregate_tflops(flops_step, world, ms_per_step)
 
-    phase_ms = {}
-    for phase, e0, e1 in records:
-        phase_ms[phase] = phase_ms.get(phase, 0.0) + e0.elapsed_time(e1)
+    phase_ms, call_ms = {}, {}
+    for idx, (phase, e0, e1) in enumerate(records):
+        ms = e0.elapsed_time(e1)
+        phase_ms[phase] = phase_ms.get(phase, 0.0) + ms
+        per = call_ms.setdefault(phase, [0.0] * len(dev))
+        per[idx % len(dev)] += ms / args.steps          # the calls of a phase run in the order of the matrices
     for k in phase_ms:
         phase_ms[k] /= args.steps
     elems = sum(d["m"]["N"] * d["m"]["K"] for d in dev)
@@ -312,6 +315,12 @@ def run_gpu(args):
         "forward": {"ms": phase_ms["forward"], "TFLOP/s": fwd_tf, "frac_tensor_burst": fwd_tf / P["tensor_burst"]},
         "backward_input": {"ms": phase_ms["backward"], "TFLOP/s": bwd_tf, "frac_tensor_burst": bwd_tf / P["tensor_burst"]},
     }
+    names = [d["m"].get("name", f'{d["m"]["N"]}x{d["m"]["K"]}') for d in dev]
+    for key, phase in (("forward", "forward"), ("backward_input", "backward")):
+        phases[key]["TFLOP/s_per_matrix"] = {
+            f"{i}:{n}": round(gemm_flops(M, d["m"]["N"], d["m"]["K"], r) / (ms * 1e-3) / 1e12, 1)
+            for i, (n, d, ms) in enumerate(zip(names, dev, call_ms[phase]))}
+
     # dominant kernel: the fused tensor-core kernel (forward + backward launches), timed as whole calls
     fused_ms = phase_ms["forward"] + phase_ms["backward"]
     achieved = flops_step / (fused_ms * 1e-3) / 1e12
@@ -411,7 +420,7 @@ def run_gpu(args):
         ad_flops = sum(4.0 * M * r * (d["m"]["K"] + d["m"]["N"]) for d in dev)
         extras["adapter_gradients"] = {"ms": ms_ad, "GB/s": ad_bytes / (ms_ad * 1e-3) / 1e9,
                                        "frac_hbm": ad_bytes / (ms_ad * 1e-3) / 1e9 / P["hbm"],
-                                       "TFLOP/s": ad_flops / (ms_ad * 1e-3) / 1e12, "launches": 6 * len(dev),
+                                       "TFLOP/s": ad_flops / (ms_ad * 1e-3) / 1e12, "launches": 5 * len(dev),
                                        "note": "not part of the step; algorithmic bytes = X and dY read once"}
 
     cpu = None

@@ -144,11 +144,16 @@ __device__ __forceinline__ void store_row(uint32_t row_addr, int swz, const uint
 
 }  // namespace
 
-// Decoded position of a tile in the persistent schedule.
-struct TileInfo {
+// One piece of work of the persistent schedule: a whole tile or, under the stream-K schedule, a slice of the
+// contraction of a weight tile.
+struct Seg {
     bool is_t;     // a LoRA down-projection tile (operand rows = ranks) rather than a weight tile
+    bool part;     // the slice does not start its tile: its fp32 sums go to this cluster's partial-tile slot
+    bool pre;      // the slice starts its tile but does not end it: the accumulator is preloaded with the partial
+                   // tiles of the clusters that hold the rest
     int rt, mt;    // row tile, token tile
-    int blocks;    // contraction blocks of this tile
+    int kb0, kb1;  // contraction blocks [kb0, kb1) of the tile
+    int tile;      // weight tile index (stream-K)
 };
 
 template <int MODE>
@@ -176,19 +181,50 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     unsigned char* tab_all = base + SA * kSmemA + SB * kSmemB;   // level tables of 4-bit rows, 2 KB per dequant warp
     auto a_slot = [&](uint32_t it) { return base + (it % SA) * kSmemA; };
     auto b_slot = [&](uint32_t it) { return base + SA * kSmemA + (it % SB) * kSmemB; };
-    const int first_tile = (int)blockIdx.x / CL, tile_step = (int)gridDim.x / CL;
+    const int cid = (int)blockIdx.x / CL, NC = (int)gridDim.x / CL;   // this cluster, clusters in the grid
     const int super_t = (P.tiles_t + CL - 1) / CL;          // groups of CL token tiles
     const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? super_t : 0;
     const int n_tiles = n_t_tiles + P.tiles_r * super_t;    // per cluster
-    auto decode_tile = [&](int g) {
-        TileInfo t;
-        t.is_t = g < n_t_tiles;
-        if (t.is_t) {
-            t.rt = 0; t.mt = g * CL + (int)crank; t.blocks = P.main_blocks;
-        } else {
+    const int B = P.main_blocks + P.lora_blocks;            // contraction blocks of a weight tile
+    // Schedule.  Whole tiles: cluster c takes tiles c, c + NC, ... (the T tiles come first).  Stream-K (large
+    // problems whose tile count is not a multiple of NC): cluster c < n_t_tiles takes T tile c; the blocks of all
+    // weight tiles, laid end to end, are cut into NC consecutive ranges of equal length (less sk_tau blocks for a
+    // cluster that has a T tile), so a range starts and ends anywhere inside a tile.  A slice that does not start
+    // its tile leaves its sums in the cluster's partial-tile slot; the cluster that starts the tile collects them.
+    const bool sk = MODE != kModeDense && P.sk != 0;
+    auto sk_lo = [&](int c) -> long long {
+        return ((long long)c * P.sk_total) / NC - (long long)min(c, n_t_tiles) * P.sk_tau;
+    };
+    const long long lo = sk ? sk_lo(cid) : 0, hi = sk ? sk_lo(cid + 1) : 0;
+    const int tile0 = sk ? (int)(lo / B) : 0;
+    const int n_t_mine = sk ? (cid < n_t_tiles ? 1 : 0) : 0;
+    const int n_wsegs = (sk && hi > lo) ? (int)((hi - (long long)tile0 * B + B - 1) / B) : 0;
+    // a range that starts inside a tile does that slice second, after its first whole tile: by then T is there
+    // (the slice may hold the tile's LoRA blocks) and the cluster that collects it is far from needing it
+    const bool swap01 = sk && n_wsegs >= 2 && lo > (long long)tile0 * B && hi >= (long long)(tile0 + 2) * B;
+    const int n_segs = sk ? n_t_mine + n_wsegs : (n_tiles > cid ? (n_tiles - cid + NC - 1) / NC : 0);
+    auto seg_at = [&](int i) {
+        Seg t;
+        t.part = t.pre = false;
+        t.tile = 0;
+        const int g = sk ? cid : cid + i * NC;
+        if (sk ? (i < n_t_mine) : (g < n_t_tiles)) {
+            t.is_t = true; t.rt = 0; t.mt = g * CL + (int)crank; t.kb0 = 0; t.kb1 = P.main_blocks;
+        } else if (!sk) {
             const int idx = g - n_t_tiles;
             const int st = idx / P.tiles_r;
-            t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank; t.blocks = P.main_blocks + P.lora_blocks;
+            t.is_t = false; t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank; t.kb0 = 0; t.kb1 = B;
+        } else {
+            int k = i - n_t_mine;
+            if (swap01 && k < 2) k = 1 - k;
+            t.tile = tile0 + k;
+            const long long first = (long long)t.tile * B;
+            t.kb0 = (k == 0) ? (int)(lo - first) : 0;
+            t.kb1 = (hi < first + B) ? (int)(hi - first) : B;
+            const int st = t.tile / P.tiles_r;
+            t.is_t = false; t.rt = t.tile - st * P.tiles_r; t.mt = st * CL + (int)crank;
+            t.part = t.kb0 > 0;
+            t.pre = t.kb0 == 0 && t.kb1 < B;
         }
         return t;
     };
@@ -228,10 +264,10 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // ================================================================== TMA producer
         if (lane == 0) {
             uint32_t it = 0;
-            for (int g = first_tile; g < n_tiles && !failed; g += tile_step) {
-                const TileInfo t = decode_tile(g);
+            for (int i = 0; i < n_segs && !failed; ++i) {
+                const Seg t = seg_at(i);
                 const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
-                for (int kb = 0; kb < t.blocks; ++kb, ++it) {
+                for (int kb = t.kb0; kb < t.kb1; ++kb, ++it) {
                     const int s = it % SB;
                     const uint32_t ph = (it / SB) & 1u;
                     if (!ptx::mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
@@ -264,7 +300,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         ptx::tma_load_2d(b_s, &tmB, c0, m0, bar);
                     } else {
                         const int lb = kb - P.main_blocks;
-                        if (lb == 0) {
+                        if (lb == 0 || kb == t.kb0) {
                             // T of this token tile is written by another CTA: wait for its flag, then make
                             // those generic-proxy writes visible to the TMA (async proxy) reads below
                             if (!ptx::flag_wait(P.flags + t.mt, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
@@ -301,14 +337,16 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             // slots and phases of the two rings, carried along (no division by the ring depths in this loop: the
             // thread's instructions are one dependent chain)
             uint32_t sb = 0, phb = 0, sa = 0, pha = 0;
-            for (int g = first_tile; g < n_tiles && !failed; g += tile_step, ++tile_iter) {
-                const TileInfo t = decode_tile(g);
+            for (int i = 0; i < n_segs && !failed; ++i, ++tile_iter) {
+                const Seg t = seg_at(i);
                 const uint32_t acc = tile_iter & 1u;            // two accumulators take turns
                 const uint32_t aph = (tile_iter >> 1) & 1u;
-                if (!ptx::mbar_wait(&bars->tmem_empty[acc], aph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                // the epilogue warps hand the accumulator over, every time (empty, or preloaded with partial sums)
+                if (!ptx::mbar_wait(&bars->tmem_empty[acc], aph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileT;
-                for (int kb = 0; kb < t.blocks; ++kb, ++it) {
+                const int kb_fresh = t.pre ? -1 : t.kb0;        // the block whose first MMA overwrites the accumulator
+                for (int kb = t.kb0; kb < t.kb1; ++kb, ++it) {
                     const int s = (int)sb;                      // token slot
                     const uint32_t ph = phb;
                     const int sw = (int)sa;                     // weight slot
@@ -335,12 +373,12 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         const uint64_t adesc = ptx::umma_desc_mn_sw128(a_addr, 8192u);
 #pragma unroll
                         for (int kk = 0; kk < kTileC / 16; ++kk)
-                            ptx::umma_bf16(d_tmem, adesc + 128u * kk, bdesc + 2u * kk, kIdescAmn, (kb | kk) != 0 ? 1u : 0u);
+                            ptx::umma_bf16(d_tmem, adesc + 128u * kk, bdesc + 2u * kk, kIdescAmn, (kb != kb_fresh || kk != 0) ? 1u : 0u);
                     } else {
                         const uint64_t adesc = ptx::umma_desc_k_sw128(a_addr);
 #pragma unroll
                         for (int kk = 0; kk < kTileC / 16; ++kk)  // 16 elements = 32 bytes along K per MMA
-                            ptx::umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, kIdesc, (kb | kk) != 0 ? 1u : 0u);
+                            ptx::umma_bf16(d_tmem, adesc + 2u * kk, bdesc + 2u * kk, kIdesc, (kb != kb_fresh || kk != 0) ? 1u : 0u);
                     }
                     ptx::umma_commit(&bars->empty[s]);
                 }
@@ -357,9 +395,62 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         const int et = (warp - kFirstEpilogueWarp) * 32 + lane;
         uint16_t* out16 = reinterpret_cast<uint16_t*>(out_s);
+        const int my_row = q * 32 + lane;
+        // Hand the accumulator of piece i to the MMA warp (four arrivals, one per warp).  A piece that starts a tile
+        // whose later blocks belong to other clusters first gets their partial sums written into the accumulator;
+        // the MMAs then add on top.  `wait` false: look at the partial tiles' flags once and come back later if one
+        // is missing (returns false); true: wait for them (bounded).
+        auto hand_over = [&](int i, bool wait) -> bool {
+            if (i >= n_segs) return true;
+            const Seg t = seg_at(i);
+            const uint32_t acc = (uint32_t)i & 1u;
+            if (t.pre) {
+                const long long tile_end = (long long)(t.tile + 1) * B;
+                int c_end = cid + 1;                                  // clusters cid + 1 .. c_end - 1 hold the rest
+                while (c_end < NC && sk_lo(c_end) < tile_end) ++c_end;
+                for (int c = cid + 1; c < c_end; ++c) {
+                    uint32_t ok = 1u;
+                    if (lane == 0) {
+                        if (wait) {
+                            if (!ptx::flag_wait(P.sk_flags + c * CL + (int)crank, abort_flag, kWaitLimitNs)) { bars->abort = 1u; ok = 2u; }
+                        } else {
+                            ok = ptx::flag_test(P.sk_flags + c * CL + (int)crank) ? 1u : 0u;
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (ok == 0u) return false;
+                    if (ok == 2u) return true;                        // timed out: the abort flag ends the loop below
+                }
+                const int m0 = t.mt * kTileT;
+#pragma unroll 1
+                for (int chunk = 0; chunk < kTileT / 32; ++chunk) {
+                    if (m0 + chunk * 32 >= P.M) break;
+                    float sum[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) sum[j] = 0.0f;
+                    for (int c = cid + 1; c < c_end; ++c) {
+                        const float* src = P.sk_part + ((size_t)c * CL + crank) * ((size_t)kTileT * kTileR) +
+                                           (size_t)(chunk * 32) * kTileR + my_row;
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) sum[j] += __ldcg(src + j * kTileR);
+                    }
+                    uint32_t v[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(sum[j]);
+                    ptx::tmem_st_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileT + chunk * 32, v);
+                }
+                ptx::tmem_st_wait();
+            }
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(&bars->tmem_empty[acc]);
+            return true;
+        };
+        // bit a: accumulator a not handed over yet (its partial tiles were not there at the first look)
+        uint32_t owed = (hand_over(0, false) ? 0u : 1u) | (hand_over(1, false) ? 0u : 2u);
         uint32_t tile_iter = 0;
-        for (int g = first_tile; g < n_tiles && !failed; g += tile_step, ++tile_iter) {
-            const TileInfo t = decode_tile(g);
+        for (int i = 0; i < n_segs && !failed; ++i, ++tile_iter) {
+            const Seg t = seg_at(i);
             const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
             // a T tile writes the down-projected activations [M, rp] (scaled by s); a weight tile writes Y / dX
             uint16_t* out = t.is_t ? P.T : P.out;
@@ -369,18 +460,26 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             const bool vec_ok = (ld % 8) == 0;
             const uint32_t acc = tile_iter & 1u;
             const uint32_t aph = (tile_iter >> 1) & 1u;
-            const int my_row = q * 32 + lane;
+            // everything before this piece is drained, so nobody waits for this warp: now the wait may block
+            if (owed & (1u << acc)) { hand_over(i, true); owed &= ~(1u << acc); }
             // the four epilogue warps share named barriers, so they must agree on leaving
             if (!ptx::mbar_wait_warp(&bars->tmem_full[acc], aph, abort_flag, kWaitLimitNs)) bars->abort = 1u;
             ptx::named_barrier_sync(1, 128);
             if (*abort_flag != 0u) { failed = true; break; }
             ptx::tc_fence_after();
+            float* part = P.sk_part + ((size_t)cid * CL + crank) * ((size_t)kTileT * kTileR) + my_row;
 #pragma unroll 1
             for (int chunk = 0; chunk < kTileT / 32; ++chunk) {
                 if (m0 + chunk * 32 >= P.M) break;
                 uint32_t v[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileT + chunk * 32, v);
                 ptx::tmem_ld_wait();
+                if (t.part) {
+                    // fp32 sums of a slice: [token][row], so that a warp writes 128 consecutive bytes
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) __stcg(part + (size_t)(chunk * 32 + j) * kTileR, __uint_as_float(v[j]));
+                    continue;
+                }
                 // thread = operand row (channel), v[j] = token j: transposed through shared memory, eight tokens
                 // at a time (8 tokens x 128 channels = 2 KB: every thread then stores one 16-byte piece)
 #pragma unroll
@@ -408,16 +507,20 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     ptx::named_barrier_sync(1, 128);
                 }
             }
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(&bars->tmem_empty[acc]);
-            if (t.is_t) {
-                // publish T of this token tile: every writer fences, then one thread raises the flag
+            // the accumulator goes to the piece after next (preloaded if that one collects partial tiles)
+            if (!hand_over(i + 2, false)) owed |= 1u << acc;
+            if (t.is_t || t.part) {
+                // publish T of this token tile, resp. this cluster's partial tile: every writer fences, then one
+                // thread raises the flag
                 __threadfence();
                 ptx::named_barrier_sync(1, 128);
                 if (et == 0) {
-                    ptx::fence_proxy_async_all();
-                    ptx::flag_release(P.flags + t.mt, 1u);
+                    if (t.is_t) {
+                        ptx::fence_proxy_async_all();
+                        ptx::flag_release(P.flags + t.mt, 1u);
+                    } else {
+                        ptx::flag_release(P.sk_flags + cid * CL + (int)crank, 1u);   // one flag per CTA: its half of the slot
+                    }
                 }
             }
         }
@@ -484,14 +587,16 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 }
             }
         };
-        for (int g = first_tile; g < n_tiles && !failed; g += tile_step) {
-            const TileInfo t = decode_tile(g);
+        for (int i = 0; i < n_segs && !failed; ++i) {
+            const Seg t = seg_at(i);
             const int r0 = t.rt * kTileR;
+            const uint32_t itb = it0 - (uint32_t)t.kb0;         // running stage index of block kb: itb + kb
+            const int kb_end = min(t.kb1, P.main_blocks);       // end of this piece's dequantised blocks
             if (t.is_t) {
                 // nothing to dequantise (the operand comes by TMA): the warps take the stages in turn and arrive
                 // for everybody
-                for (int kb = pw; kb < t.blocks; kb += kProducerWarps) {
-                    const uint32_t it = it0 + (uint32_t)kb;
+                for (int kb = pw; kb < t.kb1; kb += kProducerWarps) {
+                    const uint32_t it = itb + (uint32_t)kb;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
                     if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % SA], kStageArrivals);
                 }
@@ -535,18 +640,19 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     }
                 }
                 constexpr int kStep = CL * (kProducerWarps / 4);     // distance between two stages of this warp
-                const int kb_first = (int)crank + CL * wgrp;
+                int kb_first = (int)crank + CL * wgrp;               // this warp's blocks: kb = kb_first (mod kStep)
+                if (kb_first < t.kb0) kb_first += (t.kb0 - kb_first + kStep - 1) / kStep * kStep;
                 // The block is dequantised into registers BEFORE the wait for the stage (the warps wait most of
                 // the time): once the slot is free only the eight 16-byte stores remain on the critical path.
                 Block cur, nxt;   // codes of this visit and of the next one
                 cur.lo = cur.hi = nxt.lo = nxt.hi = make_uint4(0u, 0u, 0u, 0u);
                 cur.a = nxt.a = 0.0f;
-                if (cls < 3 && kb_first < P.main_blocks)
+                if (cls < 3 && kb_first < kb_end)
                     load_block(cur, bits_ptr + (size_t)kb_first * bits_stride, absmax_ptr + kb_first, cls);
-                if (cls < 3 && kb_first + kStep < P.main_blocks)
+                if (cls < 3 && kb_first + kStep < kb_end)
                     load_block(nxt, bits_ptr + (size_t)(kb_first + kStep) * bits_stride, absmax_ptr + kb_first + kStep, cls);
 #pragma unroll 1
-                for (int kb = kb_first; kb < P.main_blocks && !failed; kb += kStep) {
+                for (int kb = kb_first; kb < kb_end && !failed; kb += kStep) {
                     uint32_t o[32];
                     if (cls == 0) {
                         deq64_1bit(cur.lo.x, cur.lo.y, lv.m0, lv.m1, cur.a, o);
@@ -560,9 +666,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     }
                     cur = nxt;
                     const int nb = kb + 2 * kStep;
-                    if (cls < 3 && nb < P.main_blocks)
+                    if (cls < 3 && nb < kb_end)
                         load_block(nxt, bits_ptr + (size_t)nb * bits_stride, absmax_ptr + nb, cls);
-                    const uint32_t it = it0 + (uint32_t)kb;
+                    const uint32_t it = itb + (uint32_t)kb;
                     const int s = it % SA;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
                     store_row(ptx::smem_u32(a_slot(it)) + (uint32_t)row_local * 128u, row_local & 7, o);
@@ -571,8 +677,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     if (lane == 0) finish_stage(it, s, kStageArrivals / 4);
                 }
                 // LoRA blocks: operands come by TMA; the warps take the stages in turn and arrive for everybody
-                for (int kb = P.main_blocks + pw; kb < t.blocks && !failed; kb += kProducerWarps) {
-                    const uint32_t it = it0 + (uint32_t)kb;
+                for (int kb = P.main_blocks + pw; kb < t.kb1 && !failed; kb += kProducerWarps) {
+                    if (kb < t.kb0) continue;
+                    const uint32_t it = itb + (uint32_t)kb;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
                     if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % SA], kStageArrivals);
                 }
@@ -587,8 +694,12 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const int half = (lane >> 4) & 1;
                 const int k_first = r0 + 64 * half;
                 const int list = pw * CL + (int)crank;                      // this warp's work list among the cluster's
-                const uint32_t* heads = P.heads + list;                     // entry j of this warp: heads[j * kListWarps]
-                const uint4* rows = reinterpret_cast<const uint4*>(P.items) + (size_t)list * 32 + lane;   // rows[j * kListWarps * 32]
+                // the piece's first group of this CTA, and the warp's first entry at or behind that group's first chunk
+                const int g_first = t.kb0 + (((int)crank - t.kb0) % CL + CL) % CL;
+                const uint32_t n_first = 4u * (uint32_t)(g_first / CL);
+                const uint32_t j_first = n_first > (uint32_t)pw ? (n_first - (uint32_t)pw + kProducerWarps - 1) / kProducerWarps : 0u;
+                const uint32_t* heads = P.heads + list + (size_t)j_first * kListWarps;   // entry j of the piece: heads[j * kListWarps]
+                const uint4* rows = reinterpret_cast<const uint4*>(P.items) + ((size_t)list + (size_t)j_first * kListWarps) * 32 + lane;
                 constexpr uint32_t kEnd = 0xFFFFFFFFu;
                 // entry of this visit (0) and of the next one (1): head, row record, codes + absmax, 1/2-bit levels
                 uint32_t head0, head1;
@@ -628,7 +739,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
 #pragma unroll 1
                 for (uint32_t j = 0; !failed; ++j) {
                     const uint32_t head = head0;
-                    if (head == kEnd) break;
+                    if ((int)(head & 0xFFFFFFu) >= kb_end) break;   // behind the piece (the end markers are all ones)
                     const uint32_t col = rec0.w & 63u;             // channel inside the stage = K index of the tile
                     const int cls = (int)((rec0.w >> 8) & 3u);     // precision class of this lane's row (3: zeros)
                     // head and row record of the entry after next are asked for now and consumed after this visit;
@@ -651,7 +762,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
 #pragma unroll
                         for (int i = 0; i < 32; ++i) o[i] = 0u;
                     }
-                    const uint32_t it = it0 + (head & 0xFFFFFFu);
+                    const uint32_t it = itb + (head & 0xFFFFFFu);
                     const int s = it % SA;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
                     store_row(ptx::smem_u32(a_slot(it)) + (uint32_t)half * 8192u + col * 128u, (int)(col & 7u), o);
@@ -664,13 +775,14 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     fetch(blk1, lv1, head1, rec1, tab_slot);   // entry j + 2 takes over the table slot of entry j
                 }
                 // LoRA blocks: operands come by TMA; the warps take the stages in turn and arrive for everybody
-                for (int kb = P.main_blocks + pw; kb < t.blocks && !failed; kb += kProducerWarps) {
-                    const uint32_t it = it0 + (uint32_t)kb;
+                for (int kb = P.main_blocks + pw; kb < t.kb1 && !failed; kb += kProducerWarps) {
+                    if (kb < t.kb0) continue;
+                    const uint32_t it = itb + (uint32_t)kb;
                     if (!stage_free(it)) { failed = true; bars->abort = 1u; break; }
                     if (lane == 0) ptx::mbar_arrive_n(&bars->full_w[it % SA], kStageArrivals);
                 }
             }
-            it0 += (uint32_t)t.blocks;
+            it0 += (uint32_t)(t.kb1 - t.kb0);
         }
     }
 
@@ -721,10 +833,29 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
         configured = true;
     }
     const int super_t = (G.tiles_t + CL - 1) / CL;
-    const int n_tiles = G.tiles_r * super_t + ((MODE != kModeDense && G.lora_blocks > 0) ? super_t : 0);
+    const int n_t = (MODE != kModeDense && G.lora_blocks > 0) ? super_t : 0;
+    const int n_tiles = G.tiles_r * super_t + n_t;
     const int clusters = n_tiles < max_clusters ? n_tiles : max_clusters;
     cfg.gridDim = dim3((unsigned)(clusters * CL), 1, 1);
-    if (cudaLaunchKernelEx(&cfg, fused_kernel<MODE>, G, tmB, tmT, tmFt, tmFl) != cudaSuccess) return LOWRA_ERR_CUDA;
+    GemmParams Q = G;
+    Q.sk = 0;
+    // Under stream-K the clusters no longer sweep the contraction in step, so the token operand is not shared in
+    // time any more: it has to stay in L2 between its readers.  Measured on a 90 MB operand: 6.5 times the DRAM
+    // reads of the whole-tile schedule and no gain; so only operands that fit L2 with room to spare.
+    const bool operand_fits_l2 = (size_t)G.M * (size_t)G.C * 2u <= ((size_t)48 << 20);
+    if (MODE != kModeDense && G.sk_part != nullptr && clusters == max_clusters && n_t <= clusters &&
+        n_tiles % clusters != 0 && operand_fits_l2) {
+        // stream-K: equal shares of the weight tiles' blocks; a T tile counts as much as the dequantised blocks of
+        // a weight tile.  Only when every cluster still gets two tiles' worth or more.
+        const int blocks = G.main_blocks + G.lora_blocks;
+        const long long total = (long long)G.tiles_r * super_t * blocks + (long long)n_t * G.main_blocks;
+        if (total / clusters >= (long long)G.main_blocks + 2 * blocks) {
+            Q.sk = 1;
+            Q.sk_tau = G.main_blocks;
+            Q.sk_total = total;
+        }
+    }
+    if (cudaLaunchKernelEx(&cfg, fused_kernel<MODE>, Q, tmB, tmT, tmFt, tmFl) != cudaSuccess) return LOWRA_ERR_CUDA;
     return LOWRA_OK;
 }
 

@@ -16,13 +16,13 @@ constexpr size_t kStatusBytes = 256;
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Workspace {
-    size_t off_T, off_flags, off_items, off_meta, total;
-    int rp;
+    size_t off_T, off_flags, off_items, off_meta, off_part, total;
+    int rp, n_flags;
 };
 
 bool rank_ok(int r) { return r >= 16 && r <= 128 && r % 16 == 0; }
 
-Workspace plan_workspace(int N, int K, int M, int r) {
+Workspace plan_workspace(int N, int K, int M, int r, bool stream_k) {
     (void)K;
     Workspace w;
     w.rp = (r + 63) / 64 * 64;
@@ -33,9 +33,12 @@ Workspace plan_workspace(int N, int K, int M, int r) {
     const size_t fwd_words = (size_t)((N + 127) / 128) * kItemStride;
     w.off_T = kStatusBytes;
     w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);
-    w.off_items = w.off_flags + align256((size_t)((M + kTileT - 1) / kTileT + kCluster) * 4);
+    // "T ready" flags (a cluster's last token tiles may lie past M), then one "partial tile ready" flag per CTA
+    w.n_flags = (M + kTileT - 1) / kTileT + kCluster + kMaxClusters * kCluster;
+    w.off_items = w.off_flags + align256((size_t)w.n_flags * 4);
     w.off_meta = w.off_items + align256((entries * 32 * 4 > fwd_words ? entries * 32 * 4 : fwd_words) * 4);
-    w.total = w.off_meta + align256(entries * 4);
+    w.off_part = w.off_meta + align256(entries * 4);
+    w.total = w.off_part + (stream_k ? align256((size_t)kMaxClusters * kSkSlotFloats * 4) : 0);   // stream-K partial tiles
     return w;
 }
 
@@ -68,7 +71,8 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
 
 lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* packed, const float* absmax,
                       const float* maps, const uint16_t* act, int32_t M, const uint16_t* A, const uint16_t* B,
-                      int32_t r, float s, uint16_t* out, void* workspace, size_t workspace_bytes, void* stream_v) {
+                      int32_t r, float s, uint16_t* out, void* workspace, size_t workspace_bytes, void* stream_v,
+                      bool stream_k = true) {
     lowra_status st = check_layout(layout);
     if (st != LOWRA_OK) return st;
     if (!packed || !absmax || !maps || !act || !A || !B || !out || !workspace) return LOWRA_ERR_NULL;
@@ -78,7 +82,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     if (!aligned16(packed) || !aligned16(absmax) || !aligned16(maps) || !aligned16(act) || !aligned16(A) ||
         !aligned16(B) || !aligned16(out))
         return LOWRA_ERR_ALIGN;
-    const Workspace w = plan_workspace(N, K, M, r);
+    const Workspace w = plan_workspace(N, K, M, r, stream_k);
     if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LOWRA_ERR_WORKSPACE;
     st = check_device();
     if (st != LOWRA_OK) return st;
@@ -104,7 +108,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     P.group = backward ? 64 : 128;
     P.status = status;
     P.flags = flags;
-    P.n_flags = tiles_t + kCluster;   // a cluster's last token tiles may lie past M
+    P.n_flags = w.n_flags;
     P.blocks = ((N + P.group - 1) / P.group + 3) / 4;
     st = launch_prep(P, stream);
     if (st != LOWRA_OK) return st;
@@ -134,6 +138,8 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.lora_blocks = w.rp / kTileC;
     G.tiles_r = (G.R + kTileR - 1) / kTileR;
     G.tiles_t = tiles_t;
+    G.sk_part = stream_k ? reinterpret_cast<float*>(ws + w.off_part) : nullptr;   // null: whole tiles only
+    G.sk_flags = flags + tiles_t + kCluster;
     CUtensorMap tmB, tmT, tmFt, tmFl;
     if (!make_map(&tmB, act, (uint64_t)M, (uint64_t)G.C, (uint64_t)G.C, kTileT)) return LOWRA_ERR_CUDA;
     if (!make_map(&tmT, T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
@@ -171,7 +177,7 @@ __global__ void clear_status_kernel(uint32_t* status) { *status = 0u; }
 extern "C" size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r) {
     using namespace lowra;
     if (!layout || layout->N < 1 || layout->K < 1 || M < 1 || !rank_ok(r)) return 0;
-    return plan_workspace(layout->N, layout->K, M, r).total;
+    return plan_workspace(layout->N, layout->K, M, r, true).total;
 }
 
 extern "C" lowra_status lowra_lora_forward(const lowra_layout* layout, const uint8_t* packed_dev,
@@ -227,8 +233,8 @@ extern "C" lowra_status lowra_lora_forward_static(const lowra_layout* layout, co
                                                   uint32_t* status_out_dev, void* stream) {
     using namespace lowra;
     if (!layout) return LOWRA_ERR_NULL;
-    const size_t need = lowra_workspace_bytes(layout, M, r);
-    if (need == 0) return LOWRA_ERR_SHAPE;
+    if (layout->N < 1 || layout->K < 1 || M < 1 || !rank_ok(r)) return LOWRA_ERR_SHAPE;
+    const size_t need = plan_workspace(layout->N, layout->K, M, r, false).total;   // no room for partial tiles
     if (need > (size_t)LOWRA_STATIC_SCRATCH_BYTES) return LOWRA_ERR_LIMIT;
     lowra_status st = check_device();
     if (st != LOWRA_OK) return st;
@@ -238,7 +244,7 @@ extern "C" lowra_status lowra_lora_forward_static(const lowra_layout* layout, co
     // The prologue kernel rewrites every word the fused kernel reads (status word, down-projection,
     // padded factor, row deal), so nothing left over from an earlier call is ever consumed.
     st = run_lora(false, layout, packed_dev, absmax_dev, maps_dev, X_dev, M, A_dev, B_dev, r, s, Y_dev, scratch,
-                  (size_t)LOWRA_STATIC_SCRATCH_BYTES, stream);
+                  (size_t)LOWRA_STATIC_SCRATCH_BYTES, stream, false);
     if (st != LOWRA_OK) return st;
     if (status_out_dev &&
         cudaMemcpyAsync(status_out_dev, scratch, sizeof(uint32_t), cudaMemcpyDeviceToDevice, (cudaStream_t)stream) !=

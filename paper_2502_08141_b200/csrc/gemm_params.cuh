@@ -82,7 +82,15 @@ struct GemmParams {
     int main_blocks;        // ceil(C / 64)
     int lora_blocks;        // rp / 64 (0 in dense mode)
     int tiles_r, tiles_t;
+    // stream-K schedule (set by the launcher; sk == 0: whole tiles, dealt round-robin to the clusters)
+    float* sk_part;         // fp32 partial tiles, one [kCluster][kTileT][kTileR] slot per cluster
+    uint32_t* sk_flags;     // [clusters] raised when a cluster's partial tile is complete
+    int sk;
+    int sk_tau;             // blocks that a cluster with a T tile takes fewer
+    long long sk_total;     // blocks of all weight tiles + sk_tau per T tile
 };
+constexpr int kMaxClusters = kNumSMs / kCluster;
+constexpr size_t kSkSlotFloats = (size_t)kCluster * kTileT * kTileR;
 
 constexpr uint32_t kSmemA = kTileR * kTileC * 2;   // 16 KB
 constexpr uint32_t kSmemB = kTileT * kTileC * 2;   // 32 KB

@@ -117,6 +117,11 @@ __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.pr
 __device__ __forceinline__ void flag_release(uint32_t* flag, uint32_t value) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
 }
+__device__ __forceinline__ bool flag_test(const uint32_t* flag) {   // one look, no waiting
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    return v != 0u;
+}
 __device__ __forceinline__ bool flag_wait(const uint32_t* flag, volatile uint32_t* abort, uint64_t limit_ns) {
     const uint64_t t0 = globaltimer_ns();
 #pragma unroll 1

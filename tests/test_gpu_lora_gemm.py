@@ -57,6 +57,9 @@ GEMM_CASES = [
     (320, 640, 770, 48, {1: 0.5, 2: 0.3, 4: 0.2}, "llama"),         # odd number of 64-channel groups (the CTAs of a
                                                                     # cluster take them in turn), four token tiles
     (4096, 4096, 2048, 64, {1: 0.3, 2: 0.5, 4: 0.2}, "llama"),      # config 2
+    (1800, 2304, 7500, 80, {1: 0.4, 2: 0.4, 4: 0.2}, "llama"),      # 240 / 285 tiles on 74 clusters: both passes cut the
+                                                                    # contraction of some tiles between clusters; ragged
+                                                                    # channels and tokens, two LoRA blocks
 ]
 
 
