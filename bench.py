@@ -85,7 +85,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
             return
@@ -239,26 +239,30 @@ def run_gpu(args):
     act_dev = {k: bfv(torch.from_numpy(v.view(np.int16)).cuda()) for k, v in acts.items()}
     stream = torch.cuda.current_stream()
 
-    def step(record=None):
-        """One pass; `record` (a list) receives (phase, event_start, event_end) per call."""
-        def timed(phase, fn):
-            if record is None:
-                fn()
-                return
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record(stream); fn(); e1.record(stream)
-            record.append((phase, e0, e1))
-        for d in dev:
-            timed("encode", lambda: lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"]))
-        for d in dev:
-            timed("decode", lambda: lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"]))
-        for d in dev:
-            timed("forward", lambda: lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"],
-                                                           act_dev[d["m"]["K"]], d["A"], d["B"], s, Y=d["Y"], workspace=d["ws"]))
-        for d in dev:
-            timed("backward", lambda: lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"],
-                                                                   act_dev[d["m"]["N"]], d["A"], d["B"], s, dX=d["dX"],
-                                                                   workspace=d["ws"]))
+    def step(record=None, per_call=None):
+        """One pass.  `record` (a list) receives (phase, event_start, event_end) per phase: the calls of a phase
+        run back to back, as a user would issue them; `per_call` receives the same per call (diagnostic pass)."""
+        def phase(name, fn):
+            if record is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            for d in dev:
+                if per_call is not None:
+                    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    c0.record(stream); fn(d); c1.record(stream)
+                    per_call.append((name, c0, c1))
+                else:
+                    fn(d)
+            if record is not None:
+                e1.record(stream)
+                record.append((name, e0, e1))
+        phase("encode", lambda d: lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"]))
+        phase("decode", lambda d: lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"]))
+        phase("forward", lambda d: lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"],
+                                                         act_dev[d["m"]["K"]], d["A"], d["B"], s, Y=d["Y"], workspace=d["ws"]))
+        phase("backward", lambda d: lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"],
+                                                                 act_dev[d["m"]["N"]], d["A"], d["B"], s, dX=d["dX"],
+                                                                 workspace=d["ws"]))
 
     def barrier():
         torch.cuda.synchronize()
@@ -296,13 +300,19 @@ def run_gpu(args):
     value = aggregate_tflops(flops_step, world, ms_per_step)
 
     phase_ms, call_ms = {}, {}
-    for idx, (phase, e0, e1) in enumerate(records):
-        ms = e0.elapsed_time(e1)
-        phase_ms[phase] = phase_ms.get(phase, 0.0) + ms
-        per = call_ms.setdefault(phase, [0.0] * len(dev))
-        per[idx % len(dev)] += ms / args.steps          # the calls of a phase run in the order of the matrices
+    for phase, e0, e1 in records:
+        phase_ms[phase] = phase_ms.get(phase, 0.0) + e0.elapsed_time(e1)
     for k in phase_ms:
         phase_ms[k] /= args.steps
+    # diagnostic pass outside the timed region: the same step with events around every call
+    n_diag = 3
+    calls = []
+    for _ in range(n_diag):
+        step(per_call=calls)
+    torch.cuda.synchronize()
+    for idx, (phase, c0, c1) in enumerate(calls):
+        per = call_ms.setdefault(phase, [0.0] * len(dev))
+        per[idx % len(dev)] += c0.elapsed_time(c1) / n_diag      # the calls of a phase run in the order of the matrices
     elems = sum(d["m"]["N"] * d["m"]["K"] for d in dev)
     P = peaks()
     dec_gbs = sum(decode_bytes(d["m"]["N"], d["m"]["K"], bits) for d in dev) / (phase_ms["decode"] * 1e-3) / 1e9
@@ -317,7 +327,7 @@ def run_gpu(args):
     }
     names = [d["m"].get("name", f'{d["m"]["N"]}x{d["m"]["K"]}') for d in dev]
     for key, phase in (("forward", "forward"), ("backward_input", "backward")):
-        phases[key]["TFLOP/s_per_matrix"] = {
+        phases[key]["TFLOP/s_per_matrix (separate pass, events around every call)"] = {
             f"{i}:{n}": round(gemm_flops(M, d["m"]["N"], d["m"]["K"], r) / (ms * 1e-3) / 1e12, 1)
             for i, (n, d, ms) in enumerate(zip(names, dev, call_ms[phase]))}
 
