@@ -164,6 +164,24 @@ def decode(packed: np.ndarray, absmax_stored: np.ndarray, maps: np.ndarray, prec
     return out
 
 
+def quant_error(W: np.ndarray, precs: np.ndarray, maps: np.ndarray, thresholds: np.ndarray, G: int = 64):
+    """Summed square error per output channel, SSE_i = sum_k (W[i,k] - W_hat[i,k])^2 (the precision
+    assigner's objective, Section 5 and its footnote; the per-channel errors under 1, 2 and 4 bits are
+    what Section 5.1 clusters), and the residual W - W_hat that an iterative low-rank initialiser
+    factorises next (Appendix: LoftQ quantises, then decomposes what is left).
+    W_hat is what decode(encode(W)) gives: bf16(level * absmax) (Appendix A.1, A.2).
+    -> sse float64 [N] (exact differences, squared and summed in float64),
+       residual float32 [N, K] (one fp32 subtraction per element)."""
+    W = _c(W, np.float32)
+    N, K = W.shape
+    packed, a = encode(W, precs, thresholds, G)
+    w_hat = bf16_to_f64(decode(packed, a, maps, precs, K, G))
+    d = W.astype(np.float64) - w_hat
+    sse = np.array([float(np.sum(d[i] * d[i])) for i in range(N)], dtype=np.float64)
+    residual = W - w_hat.astype(np.float32)          # w_hat is exact in fp32; one rounding, in the subtraction
+    return sse, residual
+
+
 def initial_tables(b: int) -> Tuple[np.ndarray, np.ndarray]:
     """Initial levels [2^b] and thresholds [2^b - 1] (float64) of the learner."""
     maps = np.zeros(1 << b, dtype=np.float64)
