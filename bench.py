@@ -433,6 +433,28 @@ def run_gpu(args):
                                        "TFLOP/s": ad_flops / (ms_ad * 1e-3) / 1e12, "launches": 5 * len(dev),
                                        "note": "not part of the step; algorithmic bytes = X and dY read once"}
 
+        # per-channel quantisation error (the precision assigner's input) and the residual W - W_hat
+        sse = [torch.empty(d["m"]["N"], dtype=torch.float64, device="cuda") for d in dev]
+        res = torch.empty(max(d["m"]["N"] * d["m"]["K"] for d in dev), dtype=torch.float32, device="cuda")
+        qe = {}
+        for key, with_res in (("sse_only", False), ("with_residual", True)):
+            def errors():
+                for d, e in zip(dev, sse):
+                    lw.lowra_quant_error(d["layout"], d["W"], d["maps"], d["thr"], sse=e,
+                                         residual=res[:d["m"]["N"] * d["m"]["K"]].view(d["m"]["N"], d["m"]["K"]) if with_res else None)
+            errors()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            errors()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms_q = a.elapsed_time(b)
+            by = (8.0 if with_res else 4.0) * elems
+            qe[key] = {"ms": ms_q, "GB/s": by / (ms_q * 1e-3) / 1e9, "frac_hbm": by / (ms_q * 1e-3) / 1e9 / P["hbm"]}
+        qe["note"] = "not part of the step; algorithmic bytes = W read once (4 B per element) + residual written (4 B)"
+        extras["quant_error"] = qe
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
         cpu = cpu_baseline_sample()

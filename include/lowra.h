@@ -101,6 +101,26 @@ lowra_status lowra_encode(const lowra_layout* layout, const float* W_dev, const 
 lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* packed_dev, const float* absmax_dev,
                           const float* maps_dev, uint16_t* W_bf16_dev, void* stream);
 
+/*
+ * Quantisation error per output channel (Section 5 and its footnote: the precision assigner minimises
+ * the summed square error, SSE = sum_k (W[i,k] - W_hat[i,k])^2; Section 5.1 starts from every channel's
+ * error under 1, 2 and 4 bits) and, optionally, the residual W - W_hat that an iterative low-rank
+ * initialiser decomposes after quantising (appendix on the low-rank initialisers).  One fused pass
+ * over W: W_hat is exactly what lowra_encode followed by lowra_decode gives for this layout and these
+ * tables (bf16), but neither codes nor W_hat are written.
+ *   W_dev          fp32 [N, K] row-major, original row order                        (in)
+ *   maps_dev, thresholds_dev   fp32 [N, 16], original row order                     (in)
+ *   sse_dev        fp64 [N], original row order: sum of the squared fp32 residuals (four at a time in
+ *                  fp32, those partial sums in fp64, fixed order; within 2^-21 relative of the
+ *                  exact sum)                                                       (out)
+ *   residual_dev   fp32 [N, K] = fl32(W - W_hat), or NULL to skip it                (out)
+ * For the error of every channel under each precision, call it once per uniform layout.
+ * Errors: as lowra_encode.
+ */
+lowra_status lowra_quant_error(const lowra_layout* layout, const float* W_dev, const float* maps_dev,
+                               const float* thresholds_dev, double* sse_dev, float* residual_dev,
+                               void* stream);
+
 /* Bytes of device scratch that lowra_lora_forward / lowra_lora_backward_input need for M tokens and
  * LoRA rank r (0 if the arguments are invalid).  The first 256 bytes hold the device status word. */
 size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r);

@@ -28,7 +28,7 @@ EXPORTS = (
     "lowra_status_string", "lowra_plan", "lowra_encode", "lowra_decode", "lowra_workspace_bytes",
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
-    "lowra_lora_backward_adapters",
+    "lowra_lora_backward_adapters", "lowra_quant_error",
 )
 
 
@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_forward_static.restype = ctypes.c_int
         L.lowra_learn_codebooks.argtypes = [lp, vp, vp, vp, i32, vp, vp, vp]
         L.lowra_learn_codebooks.restype = ctypes.c_int
+        L.lowra_quant_error.argtypes = [lp, vp, vp, vp, vp, vp, vp]
+        L.lowra_quant_error.restype = ctypes.c_int
         L.lowra_adapter_workspace_bytes.argtypes = [i32, i32]
         L.lowra_adapter_workspace_bytes.restype = ctypes.c_size_t
         L.lowra_lora_backward_adapters.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, ctypes.c_float, vp, vp, vp,
@@ -296,6 +298,26 @@ def lowra_lora_backward_input(layout: Layout, packed, absmax, maps, dY, A, B, s:
                                            workspace.numel(), _stream(stream))
     _check(code, "lowra_lora_backward_input")
     return dX
+
+
+def lowra_quant_error(layout: Layout, W: torch.Tensor, maps: torch.Tensor, thresholds: torch.Tensor,
+                      sse: Optional[torch.Tensor] = None, residual: Optional[torch.Tensor] = None,
+                      want_residual: bool = False, stream=None):
+    """Per-channel summed square error (fp64 [N]) of quantising W with these tables, and optionally the
+    residual W - W_hat (fp32 [N,K]).  Returns (sse, residual or None)."""
+    _dev(W, torch.float32, "W")
+    _dev(maps, torch.float32, "maps")
+    _dev(thresholds, torch.float32, "thresholds")
+    if tuple(W.shape) != (layout.N, layout.K) or tuple(maps.shape) != (layout.N, 16) or tuple(thresholds.shape) != (layout.N, 16):
+        raise ValueError("shape mismatch")
+    if sse is None:
+        sse = torch.empty(layout.N, dtype=torch.float64, device=W.device)
+    if residual is None and want_residual:
+        residual = torch.empty((layout.N, layout.K), dtype=torch.float32, device=W.device)
+    code = lib().lowra_quant_error(layout.ref, _ptr(W), _ptr(maps), _ptr(thresholds), _ptr(sse),
+                                   _ptr(residual) if residual is not None else None, _stream(stream))
+    _check(code, "lowra_quant_error")
+    return sse, residual
 
 
 def lowra_adapter_workspace_bytes(M: int, r: int) -> int:

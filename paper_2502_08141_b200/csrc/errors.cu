@@ -1,0 +1,162 @@
+// lowra_quant_error: summed square error per output channel and, optionally, the residual W - W_hat.
+//
+// The precision assigner minimises the summed square error between the weights and their quantised
+// counterparts (paper Section 5 and its footnote; Section 5.1 starts from every channel's error under 1, 2 and
+// 4 bits), and an iterative low-rank initialiser factorises the residual W - W_hat after quantising (appendix on
+// the low-rank initialisers).  Both come out of one pass over W, fused: block absmax, normalise, bucket, look the
+// level up, scale and round to bf16 exactly as lowra_encode followed by lowra_decode would - without writing codes
+// or W_hat - then
+//     residual = fl32(x - w_hat)            one fp32 subtraction per element (optional output)
+//     SSE_row  = sum of residual^2          four neighbouring squares are added in fp32, those partial sums in fp64,
+//                                           fixed reduction tree (reproducible)
+// so SSE agrees with the exact sum to 2^-21 relative at worst (residual rounded to fp32: 2^-23; a square and two
+// additions in fp32: 3 * 2^-24 more), typically far closer.
+//
+// One warp per row at a time (grid-stride, no block-wide synchronisation); sixteen lanes with one float4 each cover
+// a 64-element absmax block, so the block maximum is four shuffles.  Traffic: 4 bytes per element read (+ 4 written with the residual).
+#include "lowra_common.cuh"
+
+namespace lowra {
+
+namespace {
+
+constexpr int kErrThreads = 256;
+constexpr int kErrWarps = kErrThreads / 32;
+constexpr int kErrBatch = 4;   // float4 loads per thread and batch; two batches in flight
+
+struct ErrParams {
+    RowLayout L;
+    const float* W;           // [N, K] original order
+    const float* maps;        // [N, 16]
+    const float* thresholds;  // [N, 16]
+    double* sse;              // [N]
+    float* residual;          // [N, K] or null
+};
+
+// level of the bucket of n: the number of thresholds <= n picks the level (thresholds sorted, as the encoder assumes)
+template <int B>
+__device__ __forceinline__ float level_of(float n, const float (&t)[3], const Thresholds4& t4, const float (&y)[4],
+                                          const float* y_smem) {
+    if (B == 1) return t[0] <= n ? y[1] : y[0];
+    if (B == 2) {
+        const bool hi = t[1] <= n;
+        const bool lo = (hi ? t[2] : t[0]) <= n;
+        return hi ? (lo ? y[3] : y[2]) : (lo ? y[1] : y[0]);
+    }
+    return y_smem[t4.code(n)];
+}
+
+template <int B>
+__device__ void error_row(const ErrParams& P, int r, float* y_warp) {
+    const int lane = threadIdx.x & 31;
+    const int K = P.L.K;
+    const float* wrow = P.W + (size_t)r * K;
+    float* rrow = P.residual ? P.residual + (size_t)r * K : nullptr;
+    const float* trow = P.thresholds + (size_t)r * kTableStride;
+    const float* yrow = P.maps + (size_t)r * kTableStride;
+    float t[3] = {0.f, 0.f, 0.f}, y[4] = {0.f, 0.f, 0.f, 0.f};
+    Thresholds4 t4;
+    if (B == 1) {
+        t[0] = __ldg(trow); y[0] = __ldg(yrow); y[1] = __ldg(yrow + 1);
+    } else if (B == 2) {
+        t[0] = __ldg(trow); t[1] = __ldg(trow + 1); t[2] = __ldg(trow + 2);
+        y[0] = __ldg(yrow); y[1] = __ldg(yrow + 1); y[2] = __ldg(yrow + 2); y[3] = __ldg(yrow + 3);
+    } else {
+        t4.load(trow);
+        __syncwarp();   // the previous row's look-ups are over
+        if (lane < 16) y_warp[lane] = __ldg(yrow + lane);
+        __syncwarp();
+    }
+
+    double acc = 0.0;
+    const int n4 = K / 4;   // float4 pieces of the row (a multiple of 32); lane l takes pieces l, l + 32, ...
+    // the loads of the next batch are under way while this one is worked on
+    float4 nxt[kErrBatch];
+#pragma unroll
+    for (int u = 0; u < kErrBatch; ++u) {
+        const int i = lane + u * 32;
+        nxt[u] = (i < n4) ? ld_stream_f4(wrow + (size_t)i * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (int base = lane; base < n4; base += 32 * kErrBatch) {
+        float4 x[kErrBatch];
+#pragma unroll
+        for (int u = 0; u < kErrBatch; ++u) {
+            x[u] = nxt[u];
+            const int i = base + 32 * kErrBatch + u * 32;
+            nxt[u] = (i < n4) ? ld_stream_f4(wrow + (size_t)i * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int u = 0; u < kErrBatch; ++u) {
+            const int i = base + u * 32;
+            // sixteen neighbouring lanes hold one absmax block
+            float m = fmaxf(fmaxf(fabsf(x[u].x), fabsf(x[u].y)), fmaxf(fabsf(x[u].z), fabsf(x[u].w)));
+#pragma unroll
+            for (int d = 8; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+            const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
+            // w_hat of the four elements, rounded to bf16 two at a time
+            const float l0 = __fmul_rn(level_of<B>(__fmul_rn(x[u].x, inv), t, t4, y, y_warp), m);
+            const float l1 = __fmul_rn(level_of<B>(__fmul_rn(x[u].y, inv), t, t4, y, y_warp), m);
+            const float l2 = __fmul_rn(level_of<B>(__fmul_rn(x[u].z, inv), t, t4, y, y_warp), m);
+            const float l3 = __fmul_rn(level_of<B>(__fmul_rn(x[u].w, inv), t, t4, y, y_warp), m);
+            const uint32_t h01 = pack_bf16x2(l0, l1), h23 = pack_bf16x2(l2, l3);
+            float4 res;
+            res.x = __fsub_rn(x[u].x, __uint_as_float(h01 << 16));
+            res.y = __fsub_rn(x[u].y, __uint_as_float(h01 & 0xFFFF0000u));
+            res.z = __fsub_rn(x[u].z, __uint_as_float(h23 << 16));
+            res.w = __fsub_rn(x[u].w, __uint_as_float(h23 & 0xFFFF0000u));
+            if (i < n4) {
+                // four squares in fp32 (three roundings of the partial sum), then into the fp64 sum
+                const float q = __fadd_rn(__fadd_rn(__fmul_rn(res.x, res.x), __fmul_rn(res.y, res.y)),
+                                          __fadd_rn(__fmul_rn(res.z, res.z), __fmul_rn(res.w, res.w)));
+                acc += (double)q;
+                if (rrow) __stcs(reinterpret_cast<float4*>(rrow + (size_t)i * 4), res);
+            }
+        }
+    }
+    // fixed tree over the lanes
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, d);
+    if (lane == 0) P.sse[r] = acc;
+}
+
+__global__ void __launch_bounds__(kErrThreads) error_kernel(const ErrParams P) {
+    __shared__ float y_smem[kErrWarps][16];
+    pdl_enter();
+    const int warp = threadIdx.x >> 5;
+    float* y_warp = y_smem[warp];
+    // one warp per row at a time
+    for (int r = blockIdx.x * kErrWarps + warp; r < P.L.N; r += gridDim.x * kErrWarps) {
+        const int b = P.L.precs[r];
+        if (b == 1) error_row<1>(P, r, y_warp);
+        else if (b == 2) error_row<2>(P, r, y_warp);
+        else error_row<4>(P, r, y_warp);
+    }
+}
+
+}  // namespace
+}  // namespace lowra
+
+extern "C" lowra_status lowra_quant_error(const lowra_layout* layout, const float* W_dev, const float* maps_dev,
+                                          const float* thresholds_dev, double* sse_dev, float* residual_dev,
+                                          void* stream) {
+    using namespace lowra;
+    lowra_status st = check_layout(layout);
+    if (st != LOWRA_OK) return st;
+    if (!W_dev || !maps_dev || !thresholds_dev || !sse_dev) return LOWRA_ERR_NULL;
+    if (!aligned16(W_dev) || !aligned16(maps_dev) || !aligned16(thresholds_dev) || !aligned16(sse_dev) ||
+        (residual_dev && !aligned16(residual_dev)))
+        return LOWRA_ERR_ALIGN;
+    st = check_device();
+    if (st != LOWRA_OK) return st;
+    ErrParams P;
+    P.L = make_row_layout(layout);
+    P.W = W_dev;
+    P.maps = maps_dev;
+    P.thresholds = thresholds_dev;
+    P.sse = sse_dev;
+    P.residual = residual_dev;
+    const int cap = kNumSMs * 4;
+    const int want = (layout->N + kErrWarps - 1) / kErrWarps;
+    const unsigned grid = (unsigned)(want < cap ? want : cap);
+    return launch_pdl(error_kernel, grid, kErrThreads, (cudaStream_t)stream, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+}

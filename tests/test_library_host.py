@@ -98,6 +98,11 @@ def test_validation_runs_before_any_device_work(lib):
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, None, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_NULL
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, init, init, -1, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096 + 4, init, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_ALIGN
+    # quantisation error: layout, W, maps, thresholds, sse, residual (may be NULL), stream
+    assert L.lowra_quant_error(ctypes.byref(lay), 4096, 4096, 4096, None, None, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_quant_error(ctypes.byref(lay), 4096 + 4, 4096, 4096, 4096, None, None) == lib.LOWRA_ERR_ALIGN
+    assert L.lowra_quant_error(ctypes.byref(lay), 4096, 4096, 4096, 4096, 4096 + 8, None) == lib.LOWRA_ERR_ALIGN
+    assert L.lowra_quant_error(None, 4096, 4096, 4096, 4096, None, None) == lib.LOWRA_ERR_NULL
     # adapter gradients: X, dY, M, K, N, A, B, r, s, dA, dB, workspace, bytes, stream
     big = 1 << 30
     assert L.lowra_adapter_workspace_bytes(0, 16) == 0
