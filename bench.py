@@ -160,20 +160,23 @@ def make_host_inputs(cfg, rank: int):
 
 
 # DRAM traffic of one fused_kernel launch measured with ncu on the small profiling case (N = K = 4096,
-# 2048 tokens, rank 64, 1.5 bits on average): forward 22.35 MB, backward-input 22.40 MB, almost all of it reads
-# (the bf16 output is still in L2 when the kernel ends).  That equals the case's input bytes (activations +
-# packed codes + absmax + tables + LoRA factors = 22.1 MB), so traffic is scaled in proportion to input bytes.
-NCU_CASE = dict(N=4096, K=4096, M=2048, r=64, bits=1.5, dram_bytes=0.5 * (22.35e6 + 22.40e6))
+# 2048 tokens, rank 64, 1.5 bits on average; dram__bytes_read.sum + dram__bytes_write.sum): forward 22.4 + 9.2 MB,
+# backward-input 22.5 + 9.0 MB.  The reads equal the case's input bytes (activations + packed codes + absmax +
+# tables + LoRA factors = 22.1 MB: nothing is read twice); of the 16.8 MB of bf16 output a good half has reached
+# DRAM when the kernel ends, the rest is still in L2.  Scaled to a launch of the bench in proportion to its
+# input + output bytes.
+NCU_CASE = dict(N=4096, K=4096, M=2048, r=64, bits=1.5, dram_bytes=0.5 * (22.4e6 + 9.2e6 + 22.5e6 + 9.0e6))
 
 
-def fused_input_bytes(N, K, M, r, bits):
-    return 2.0 * M * K + N * K * (bits / 8 + 4 / 64) + 64.0 * N + 2.0 * (K + N) * r
+def fused_io_bytes(N, K, M, r, bits):
+    """Bytes a fused call has to read and write once: activations, packed codes, absmax, tables, factors; output."""
+    return 2.0 * M * K + N * K * (bits / 8 + 4 / 64) + 64.0 * N + 2.0 * (K + N) * r + 2.0 * M * N
 
 
 def fused_traffic_per_launch(dev, M, r, bits):
-    case = fused_input_bytes(NCU_CASE["N"], NCU_CASE["K"], NCU_CASE["M"], NCU_CASE["r"], NCU_CASE["bits"])
-    per = [fused_input_bytes(d["m"]["N"], d["m"]["K"], M, r, bits) for d in dev] + \
-          [fused_input_bytes(d["m"]["K"], d["m"]["N"], M, r, bits) for d in dev]   # backward reads dY [M, N]
+    case = fused_io_bytes(NCU_CASE["N"], NCU_CASE["K"], NCU_CASE["M"], NCU_CASE["r"], NCU_CASE["bits"])
+    per = [fused_io_bytes(d["m"]["N"], d["m"]["K"], M, r, bits) for d in dev] + \
+          [fused_io_bytes(d["m"]["K"], d["m"]["N"], M, r, bits) for d in dev]   # backward reads dY [M, N], writes dX [M, K]
     return NCU_CASE["dram_bytes"] / case * sum(per) / len(per)
 
 
@@ -340,8 +343,8 @@ def run_gpu(args):
                 "frac_burst": achieved / P["tensor_burst"], "peak_source": P["source"] + " (sustained: timed inside a long step)",
                 "traffic": fused_traffic_per_launch(dev, M, r, bits),
                 "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one fused_kernel launch at "
-                                  "N=K=4096, 2048 tokens (profiles/fused_*_4096x4096_m2048.md), scaled by the input "
-                                  "bytes of an average launch of this workload"}
+                                  "N=K=4096, 2048 tokens (profiles/fused_*_4096x4096_m2048.md), scaled by the input + "
+                                  "output bytes of an average launch of this workload"}
 
     # ---- end to end: host buffers, pinned, copies inside the timed region
     e2e = None

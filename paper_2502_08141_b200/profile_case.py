@@ -5,6 +5,7 @@
     python -m paper_2502_08141_b200.profile_case codec       # decode + encode of an 11008 x 4096 matrix
     python -m paper_2502_08141_b200.profile_case learn       # codebook learner, 4096 x 4096, 10 iterations
     python -m paper_2502_08141_b200.profile_case adapters    # gradients of the low-rank factors, 4096 x 11008, 4096 tokens
+    python -m paper_2502_08141_b200.profile_case errors      # per-channel quantisation error + residual, 11008 x 4096
 
 Each case runs its call three times on seeded synthetic inputs (config-3 precision mix) and checks the
 device status word; a few hundred MB on the device at most.
@@ -18,7 +19,8 @@ import torch
 import synth_inputs as si
 
 from . import (Layout, lowra_adapter_workspace_bytes, lowra_decode, lowra_device_status, lowra_encode, lowra_learn_codebooks,
-               lowra_lora_backward_adapters, lowra_lora_backward_input, lowra_lora_forward, lowra_workspace_bytes)
+               lowra_lora_backward_adapters, lowra_lora_backward_input, lowra_lora_forward, lowra_quant_error,
+               lowra_workspace_bytes)
 
 
 def adapters() -> None:
@@ -43,7 +45,7 @@ def main(case: str) -> None:
         adapters()
         return
     cfg = si.config(3)
-    N, K = (11008, 4096) if case == "codec" else (4096, 4096)
+    N, K = (11008, 4096) if case in ("codec", "errors") else (4096, 4096)
     M, r, s = 2048, cfg.rank, cfg.s
     precs = si.precisions(N, cfg.mix)
     maps, thr = si.standin_codebooks(precs)
@@ -62,6 +64,15 @@ def main(case: str) -> None:
             lowra_learn_codebooks(layout, W, y0, t0, 10)
         torch.cuda.synchronize()
         print("learn ok")
+        return
+    if case == "errors":
+        sse = torch.empty(N, dtype=torch.float64, device="cuda")
+        res = torch.empty(N, K, dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            lowra_quant_error(layout, W, maps_d, thr_d, sse=sse, residual=res)
+            lowra_quant_error(layout, W, maps_d, thr_d, sse=sse)
+        torch.cuda.synchronize()
+        print("errors ok")
         return
     packed, absmax = lowra_encode(layout, W, thr_d)
     if case == "codec":
