@@ -109,3 +109,32 @@ def test_runs_on_a_side_stream(lw):
         out = lw.lowra_decode(layout, packed, absmax, maps, stream=s)
     s.synchronize()
     assert np.array_equal(out.view(torch.int16).cpu().numpy().view(np.uint16), case.W_hat)
+
+
+def test_one_packed_buffer_many_decode_tables(lw):
+    """The production variant of Section 4.1: one set of thresholds (one packed buffer, shared by every
+    adapter), a different decode mapping per adapter.  Decode and the fused forward take the mapping as an
+    argument of its own, so each adapter's table gives that adapter's weights from the same codes."""
+    N, K, M, r = 256, 512, 96, 16
+    case = make_case(N, K, {1: 0.4, 2: 0.4, 4: 0.2}, matrix_id=43)
+    layout = lw.Layout(case.precs, K)
+    packed, absmax = lw.lowra_encode(layout, _dev(case.W), _dev(case.thr))
+    X = si.activations(M, K, matrix_id=43)
+    A, B = si.lora_factors(K, N, r, matrix_id=43)
+    bf = lambda bits: _dev(bits.view(np.int16)).view(torch.bfloat16)
+    rng = np.random.default_rng(43)
+    for adapter in range(3):
+        maps = case.maps.copy()
+        if adapter > 0:   # this adapter's levels: the shared ones moved a little, still sorted
+            for i in range(N):
+                L = 1 << int(case.precs[i])
+                gap = np.diff(maps[i, :L]).min() if L > 1 else 0.0
+                maps[i, :L] += (rng.uniform(-0.3, 0.3, size=L) * gap).astype(np.float32)
+        ref = oracle.decode(case.packed, case.absmax, maps, case.precs, K)
+        out = lw.lowra_decode(layout, packed, absmax, _dev(maps))
+        assert np.array_equal(out.view(torch.int16).cpu().numpy().view(np.uint16), ref)
+        Y = lw.lowra_lora_forward(layout, packed, absmax, _dev(maps), bf(X), bf(A), bf(B), 2.0)
+        Y_ref = oracle.lora_forward(ref, X, A, B, 2.0)
+        got = si.bf16_bits_to_f32(Y.view(torch.int16).cpu().numpy().view(np.uint16))
+        assert np.abs(got - Y_ref).max() <= 1e-2 * np.abs(Y_ref).max()
+        assert np.linalg.norm(got - Y_ref) <= 5e-3 * np.linalg.norm(Y_ref)
