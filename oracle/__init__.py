@@ -164,6 +164,29 @@ def decode(packed: np.ndarray, absmax_stored: np.ndarray, maps: np.ndarray, prec
     return out
 
 
+def natural_layout(codes: np.ndarray, precs: np.ndarray):
+    """The paper's own buffer layout (Appendix A.2: a thread finds its offset into the quantised buffer from the
+    channels' bit precisions): rows in their ORIGINAL order, row r at byte offset sum_{i<r} K*b_i/8, codes packed
+    LSB-first at the row's precision.  codes uint8 [N,K] -> (buffer uint8, offsets uint64 [N+1]).
+    Written with plain shifts on the code matrix, independent of the C packer of the grouped layout."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    precs = np.asarray(precs, dtype=np.int64)
+    N, K = codes.shape
+    row_bytes = K * precs // 8
+    offsets = np.zeros(N + 1, dtype=np.uint64)
+    offsets[1:] = np.cumsum(row_bytes)
+    buf = np.zeros(int(offsets[-1]), dtype=np.uint8)
+    for r in range(N):
+        b = int(precs[r])
+        per = 8 // b                                   # codes per byte
+        c = codes[r].reshape(K // per, per).astype(np.uint32)
+        byte = np.zeros(K // per, dtype=np.uint32)
+        for j in range(per):
+            byte |= (c[:, j] & ((1 << b) - 1)) << (b * j)
+        buf[int(offsets[r]):int(offsets[r + 1])] = byte.astype(np.uint8)
+    return buf, offsets
+
+
 def quant_error(W: np.ndarray, precs: np.ndarray, maps: np.ndarray, thresholds: np.ndarray, G: int = 64):
     """Summed square error per output channel, SSE_i = sum_k (W[i,k] - W_hat[i,k])^2 (the precision
     assigner's objective, Section 5 and its footnote; the per-channel errors under 1, 2 and 4 bits are
