@@ -102,6 +102,26 @@ lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* packed_dev,
                           const float* maps_dev, uint16_t* W_bf16_dev, void* stream);
 
 /*
+ * The paper's own buffer layout as a second storage variant (Appendix A.2: a thread of the
+ * dequantisation kernel finds its offset into the quantised buffer from the channels' bit precisions):
+ * rows in their ORIGINAL order, row r at byte offset sum_{i<r} K * b_i / 8; the absmax rows in original
+ * order too.  A row's bytes are the same in both layouts, so converting is a row permutation.
+ *
+ * lowra_natural_offsets (host only): offsets_host[N + 1] from precs_host[N]; offsets_host[N] is the
+ * buffer size (= the grouped layout's packed_bytes).  Errors as lowra_plan.
+ *
+ * lowra_reorder_rows: to_natural != 0: grouped -> natural; to_natural == 0: natural -> grouped.
+ *   offsets_dev     uint64 [N + 1], device copy of the offsets above                        (in)
+ *   packed_src_dev  uint8 [packed_bytes], absmax_src_dev fp32 [N, K/64] in the source order (in)
+ *   packed_dst_dev, absmax_dst_dev: the same in the destination order; not in place          (out)
+ * Errors: as lowra_encode; source == destination -> LOWRA_ERR_SHAPE.
+ */
+lowra_status lowra_natural_offsets(int32_t N, int32_t K, const uint8_t* precs_host, uint64_t* offsets_host);
+lowra_status lowra_reorder_rows(const lowra_layout* layout, int32_t to_natural, const uint64_t* offsets_dev,
+                                const uint8_t* packed_src_dev, const float* absmax_src_dev,
+                                uint8_t* packed_dst_dev, float* absmax_dst_dev, void* stream);
+
+/*
  * Quantisation error per output channel (Section 5 and its footnote: the precision assigner minimises
  * the summed square error, SSE = sum_k (W[i,k] - W_hat[i,k])^2; Section 5.1 starts from every channel's
  * error under 1, 2 and 4 bits) and, optionally, the residual W - W_hat that an iterative low-rank

@@ -28,7 +28,7 @@ EXPORTS = (
     "lowra_status_string", "lowra_plan", "lowra_encode", "lowra_decode", "lowra_workspace_bytes",
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
-    "lowra_lora_backward_adapters", "lowra_quant_error",
+    "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
 )
 
 
@@ -81,6 +81,10 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_forward_static.restype = ctypes.c_int
         L.lowra_learn_codebooks.argtypes = [lp, vp, vp, vp, i32, vp, vp, vp]
         L.lowra_learn_codebooks.restype = ctypes.c_int
+        L.lowra_natural_offsets.argtypes = [i32, i32, vp, vp]
+        L.lowra_natural_offsets.restype = ctypes.c_int
+        L.lowra_reorder_rows.argtypes = [lp, i32, vp, vp, vp, vp, vp, vp]
+        L.lowra_reorder_rows.restype = ctypes.c_int
         L.lowra_quant_error.argtypes = [lp, vp, vp, vp, vp, vp, vp]
         L.lowra_quant_error.restype = ctypes.c_int
         L.lowra_adapter_workspace_bytes.argtypes = [i32, i32]
@@ -298,6 +302,36 @@ def lowra_lora_backward_input(layout: Layout, packed, absmax, maps, dY, A, B, s:
                                            workspace.numel(), _stream(stream))
     _check(code, "lowra_lora_backward_input")
     return dX
+
+
+def lowra_natural_offsets(precs, K: int):
+    """Byte offsets [N + 1] (numpy uint64) of the rows in the natural-order buffer."""
+    import numpy as np
+    precs = np.ascontiguousarray(precs, dtype=np.uint8)
+    off = np.zeros(precs.size + 1, dtype=np.uint64)
+    code = lib().lowra_natural_offsets(int(precs.size), int(K), ctypes.c_void_p(precs.ctypes.data),
+                                       ctypes.c_void_p(off.ctypes.data))
+    _check(code, "lowra_natural_offsets")
+    return off
+
+
+def lowra_reorder_rows(layout: Layout, to_natural: bool, offsets: torch.Tensor, packed: torch.Tensor,
+                       absmax: torch.Tensor, packed_out: Optional[torch.Tensor] = None,
+                       absmax_out: Optional[torch.Tensor] = None, stream=None):
+    """Grouped <-> natural row order of the packed codes and the absmax rows.  `offsets`: the natural offsets
+    as an int64 / uint64 device tensor [N + 1].  Returns (packed_out, absmax_out)."""
+    _dev(packed, torch.uint8, "packed")
+    _dev(absmax, torch.float32, "absmax")
+    if not offsets.is_cuda or offsets.element_size() != 8 or offsets.numel() != layout.N + 1:
+        raise ValueError("offsets must be a 64-bit device tensor of N + 1 entries")
+    if packed_out is None:
+        packed_out = torch.empty_like(packed)
+    if absmax_out is None:
+        absmax_out = torch.empty_like(absmax)
+    code = lib().lowra_reorder_rows(layout.ref, 1 if to_natural else 0, _ptr(offsets), _ptr(packed), _ptr(absmax),
+                                    _ptr(packed_out), _ptr(absmax_out), _stream(stream))
+    _check(code, "lowra_reorder_rows")
+    return packed_out, absmax_out
 
 
 def lowra_quant_error(layout: Layout, W: torch.Tensor, maps: torch.Tensor, thresholds: torch.Tensor,

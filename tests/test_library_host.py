@@ -98,6 +98,19 @@ def test_validation_runs_before_any_device_work(lib):
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, None, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_NULL
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, init, init, -1, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096 + 4, init, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_ALIGN
+    # natural-order offsets (host only) and the row reordering
+    import numpy as np
+    pr = np.array([1, 4, 2, 2], dtype=np.uint8)
+    off = np.zeros(5, dtype=np.uint64)
+    assert L.lowra_natural_offsets(4, 256, pr.ctypes.data, off.ctypes.data) == lib.LOWRA_OK
+    assert off.tolist() == [0, 32, 160, 224, 288]
+    assert L.lowra_natural_offsets(4, 200, pr.ctypes.data, off.ctypes.data) == lib.LOWRA_ERR_SHAPE
+    pr[1] = 3
+    assert L.lowra_natural_offsets(4, 256, pr.ctypes.data, off.ctypes.data) == lib.LOWRA_ERR_PREC
+    assert L.lowra_natural_offsets(4, 256, None, off.ctypes.data) == lib.LOWRA_ERR_NULL
+    assert L.lowra_reorder_rows(ctypes.byref(lay), 1, None, 4096, 4096, 8192, 8192, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_reorder_rows(ctypes.byref(lay), 1, 4096, 4096, 4096, 4096, 8192, None) == lib.LOWRA_ERR_SHAPE
+    assert L.lowra_reorder_rows(ctypes.byref(lay), 1, 4096, 4096 + 8, 4096, 8192, 8192, None) == lib.LOWRA_ERR_ALIGN
     # quantisation error: layout, W, maps, thresholds, sse, residual (may be NULL), stream
     assert L.lowra_quant_error(ctypes.byref(lay), 4096, 4096, 4096, None, None, None) == lib.LOWRA_ERR_NULL
     assert L.lowra_quant_error(ctypes.byref(lay), 4096 + 4, 4096, 4096, 4096, None, None) == lib.LOWRA_ERR_ALIGN
