@@ -3,6 +3,8 @@
 Encode and decode are compared bit for bit on the whole matrix.  The two products are computed in full
 on the GPU and compared with the fp64 oracle on 128 sampled token rows (always rows 0, 127, 128 and
 M - 1, the rest seeded): the oracle evaluates exactly those rows, all N (resp. K) outputs of each.
+The gradients of the low-rank factors (small outputs) and the per-channel quantisation errors are compared in
+full, the residual bit for bit on 64 sampled rows.
 """
 import numpy as np
 import pytest
@@ -73,3 +75,22 @@ def test_full_size_matrix(name, N, K, mix, mid):
     emax, efro = gemm_errors(got, ref)
     assert emax <= MAX_TOL and efro <= FRO_TOL, ("backward", name, emax, efro)
     assert torch.isfinite(dX.float()).all()
+    del dX
+
+    # gradients of the low-rank factors: small outputs, compared in full (B as spread out as A, so that dA is not zero)
+    B2 = si.bf16_normal((r, N), 0.01, stream=90 + mid)
+    wsa = torch.empty(lw.lowra_adapter_workspace_bytes(M, r), dtype=torch.uint8, device="cuda")
+    dA, dB = lw.lowra_lora_backward_adapters(_bf(X), _bf(dY), _bf(A), _bf(B2), s, workspace=wsa)
+    assert lw.lowra_device_status(wsa) == lw.LOWRA_OK
+    dA_ref, dB_ref = oracle.lora_backward_adapters(X, dY, A, B2, s)
+    for nm, got_t, ref in (("dA", dA, dA_ref), ("dB", dB, dB_ref)):
+        emax, efro = gemm_errors(si.bf16_bits_to_f32(_bits(got_t)), ref)
+        assert emax <= MAX_TOL and efro <= FRO_TOL, (nm, name, emax, efro)
+
+    # per-channel quantisation error on the whole matrix, residual on sampled rows
+    sse, res = lw.lowra_quant_error(layout, _dev(case.W), _dev(case.maps), _dev(case.thr), want_residual=True)
+    sse_ref, res_ref = oracle.quant_error(case.W, case.precs, case.maps, case.thr)
+    got = sse.cpu().numpy()
+    assert np.all(np.abs(got - sse_ref) <= 2.0 ** -21 * sse_ref)
+    rr = np.unique(np.concatenate([[0, N - 1], rng.choice(N, 62, replace=False)]))
+    assert np.array_equal(res[torch.from_numpy(rr).cuda()].cpu().numpy().view(np.uint32), res_ref[rr].view(np.uint32))
