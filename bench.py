@@ -360,32 +360,66 @@ def run_gpu(args):
             + sum(2 * act_host[d["m"]["K"]].numel() + 2 * act_host[d["m"]["N"]].numel() for d in dev)
         d2h = sum(h[k].numel() * h[k].element_size() for h in host for k in ("Y", "dX"))
 
+        # Three streams: uploads, kernels, downloads.  Matrix i + 1 is uploaded while matrix i is computed and
+        # matrix i - 1 is downloaded (the copies of one step are PCIe-bound: 2.1 GB); every buffer has its own
+        # events, so a buffer is never overwritten before its last reader is done, across steps too.
+        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+        xs = [torch.empty_like(act_dev[d["m"]["K"]]) for d in dev]      # per-matrix activations / output gradients
+        gs = [torch.empty_like(act_dev[d["m"]["N"]]) for d in dev]
+        ev_in = [torch.cuda.Event() for _ in dev]
+        ev_done = [None] * len(dev)
+        ev_out = [None] * len(dev)
+
         def e2e_step():
-            for d, h in zip(dev, host):
-                d["W"].copy_(h["W"], non_blocking=True); d["thr"].copy_(h["thr"], non_blocking=True)
-                d["maps"].copy_(h["maps"], non_blocking=True)
-                d["A"].view(torch.int16).copy_(h["A"], non_blocking=True); d["B"].view(torch.int16).copy_(h["B"], non_blocking=True)
-                x = act_dev[d["m"]["K"]]; x.view(torch.int16).copy_(act_host[d["m"]["K"]], non_blocking=True)
-                g = act_dev[d["m"]["N"]]; g.view(torch.int16).copy_(act_host[d["m"]["N"]], non_blocking=True)
+            for i, (d, h) in enumerate(zip(dev, host)):
+                with torch.cuda.stream(s_in):
+                    if ev_done[i] is not None:
+                        s_in.wait_event(ev_done[i])                      # the previous step's kernels have read them
+                    d["W"].copy_(h["W"], non_blocking=True); d["thr"].copy_(h["thr"], non_blocking=True)
+                    d["maps"].copy_(h["maps"], non_blocking=True)
+                    d["A"].view(torch.int16).copy_(h["A"], non_blocking=True)
+                    d["B"].view(torch.int16).copy_(h["B"], non_blocking=True)
+                    xs[i].view(torch.int16).copy_(act_host[d["m"]["K"]], non_blocking=True)
+                    gs[i].view(torch.int16).copy_(act_host[d["m"]["N"]], non_blocking=True)
+                    ev_in[i].record(s_in)
+                stream.wait_event(ev_in[i])
+                if ev_out[i] is not None:
+                    stream.wait_event(ev_out[i])                         # the previous step's results have left
                 lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"])
                 lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"])
-                lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], x, d["A"], d["B"], s, Y=d["Y"], workspace=d["ws"])
-                lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], g, d["A"], d["B"], s, dX=d["dX"], workspace=d["ws"])
-                h["Y"].copy_(d["Y"], non_blocking=True); h["dX"].copy_(d["dX"], non_blocking=True)
+                lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], xs[i], d["A"], d["B"], s, Y=d["Y"], workspace=d["ws"])
+                lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], gs[i], d["A"], d["B"], s, dX=d["dX"], workspace=d["ws"])
+                ev_done[i] = torch.cuda.Event(); ev_done[i].record(stream)
+                with torch.cuda.stream(s_out):
+                    s_out.wait_event(ev_done[i])
+                    h["Y"].copy_(d["Y"], non_blocking=True); h["dX"].copy_(d["dX"], non_blocking=True)
+                    ev_out[i] = torch.cuda.Event(); ev_out[i].record(s_out)
+
+        def e2e_join():   # the step is over when its last download is
+            for e in ev_out:
+                if e is not None:
+                    stream.wait_event(e)
 
         e2e_step()
+        e2e_join()
         barrier()
         n_e2e = max(1, min(args.steps, 3))
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         for _ in range(n_e2e):
             e2e_step()
+        e2e_join()
         b.record(stream)
         barrier()
+        for d in dev:
+            if lw.lowra_device_status(d["ws"]) != 0:
+                raise SystemExit("device status after the end-to-end steps")
         ms = a.elapsed_time(b) / n_e2e
         ms = max_over_ranks(ms, world)
         e2e = {"value": aggregate_tflops(flops_step, world, ms), "unit": UNIT, "ms_per_step": ms,
-               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e}
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e,
+               "note": "uploads, kernels and downloads on three streams: a matrix is computed while the next one "
+                       "arrives and the previous one leaves"}
 
     # ---- outside the step: the codebook learner (the stage before encode), timed on the layer's seven matrices
     extras = None
