@@ -323,10 +323,12 @@ def run_gpu(args):
     fwd_tf = flops_step / 2 / (phase_ms["forward"] * 1e-3) / 1e12
     bwd_tf = flops_step / 2 / (phase_ms["backward"] * 1e-3) / 1e12
     phases = {
-        "encode": {"ms": phase_ms["encode"], "GB/s": enc_gbs, "frac_hbm": enc_gbs / P["hbm"]},
-        "decode": {"ms": phase_ms["decode"], "GB/s": dec_gbs, "frac_hbm": dec_gbs / P["hbm"]},
-        "forward": {"ms": phase_ms["forward"], "TFLOP/s": fwd_tf, "frac_tensor_burst": fwd_tf / P["tensor_burst"]},
-        "backward_input": {"ms": phase_ms["backward"], "TFLOP/s": bwd_tf, "frac_tensor_burst": bwd_tf / P["tensor_burst"]},
+        "encode": {"ms": phase_ms["encode"], "GB/s": enc_gbs, "frac_hbm": enc_gbs / P["hbm"], "frac_hbm_nominal_8TBs": enc_gbs / 8000.0},
+        "decode": {"ms": phase_ms["decode"], "GB/s": dec_gbs, "frac_hbm": dec_gbs / P["hbm"], "frac_hbm_nominal_8TBs": dec_gbs / 8000.0},
+        "forward": {"ms": phase_ms["forward"], "TFLOP/s": fwd_tf, "frac_tensor_burst": fwd_tf / P["tensor_burst"],
+                    "frac_tensor_sustained": fwd_tf / P["tensor_sustained"], "frac_tensor_nominal_2250": fwd_tf / 2250.0},
+        "backward_input": {"ms": phase_ms["backward"], "TFLOP/s": bwd_tf, "frac_tensor_burst": bwd_tf / P["tensor_burst"],
+                           "frac_tensor_sustained": bwd_tf / P["tensor_sustained"], "frac_tensor_nominal_2250": bwd_tf / 2250.0},
     }
     names = [d["m"].get("name", f'{d["m"]["N"]}x{d["m"]["K"]}') for d in dev]
     for key, phase in (("forward", "forward"), ("backward_input", "backward")):
