@@ -11,7 +11,7 @@
 // turn, and the CTA that has dequantised a stage's operand tile sends a copy into its peer's shared memory
 // (one asynchronous 16 KB copy, counted on the peer's stage barrier), so every weight is dequantised once
 // per 512 tokens.  The 256-token operand (activations / output gradients) is the B operand and arrives by
-// TMA.  Shared memory holds six weight slots and three token slots.  Accumulators live in TMEM (two, so the
+// TMA.  Shared memory holds five weight slots and four token slots.  Accumulators live in TMEM (two, so the
 // epilogue of a tile overlaps the main loop of the next).
 // The LoRA term is folded into the same accumulator as extra contraction blocks at the end of every
 // tile: the up-projection factor comes by TMA straight from the caller's matrix, the down-projected
@@ -19,7 +19,10 @@
 // kernel: for every token tile there is one extra "T tile" whose 128 operand rows are the LoRA ranks
 // (factor fetched by TMA, no dequant); T tiles come first in the tile order, their epilogue publishes a
 // per-token-tile flag, and the TMA producer of a regular tile waits (bounded) for that flag before it
-// fetches T.  All CTAs are co-resident and walk the tiles in increasing order, so the wait cannot deadlock.
+// fetches T.  All CTAs are co-resident and a T tile waits for nothing, so the wait cannot deadlock.
+// Schedule: whole tiles dealt round-robin to the clusters, or (launcher's choice) stream-K: equal consecutive
+// ranges of the weight tiles' contraction blocks per cluster, partial tiles handed over through a scratch slot
+// and preloaded into the accumulator of the cluster that starts the tile (see the schedule in the kernel).
 //
 // Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, eight of 6-15 = dequant.
 // All mbarrier waits are bounded; a wait that runs out sets the status word and every role leaves.

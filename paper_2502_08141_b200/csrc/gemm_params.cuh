@@ -9,11 +9,10 @@ namespace lowra {
 
 // ---- prologue ------------------------------------------------------------------------------
 constexpr int kPrepThreads = 128;
-constexpr int kProducerWarps = 8;             // dequant warps of the main kernel (14 warps in all: at most four per
-                                              // scheduler, so every thread may hold 128 registers)
+constexpr int kProducerWarps = 8;             // dequant warps of the main kernel
 constexpr int kItemStride = 128;              // forward: entries per group of 128 rows in the deal table
-constexpr int kStageArrivals = 8;             // backward: arrivals a stage barrier expects from the dequant warps (>= 7 chunks)
-constexpr int kCluster = 2;                // backward: CTAs per cluster; they share every dequantised weight tile
+constexpr int kStageArrivals = 8;             // arrivals a weight-slot barrier expects from the dequant warps (backward: four chunks x 2)
+constexpr int kCluster = 2;                   // CTAs per cluster; they share every dequantised weight tile
 constexpr int kListWarps = kProducerWarps * kCluster;   // backward: work lists (one per dequant warp of the cluster)
 constexpr int kListSlack = 4 * kProducerWarps;  // backward: all-ones heads written behind the last entry of a CTA's lists
 constexpr int kMaxGroups64 = 8192;            // backward: at most this many groups of 64 output channels (N <= 524288)
@@ -44,8 +43,11 @@ constexpr int kTileC = 64;        // contraction elements per pipeline stage (= 
 constexpr int kStages = 4;        // dense diagnostic: four stages of one weight slot + one token slot
 // Forward / backward: the dequant warps (and the copies between the CTAs of a cluster) need to run further ahead
 // of the tensor core than the TMA loads do, so the ring is split into 16 KB weight slots and 32 KB token slots:
-// six + four (backward), five + four (forward, which spends the difference on a cache of the level tables of
-// its 4-bit rows).  A weight slot is free once the MMAs of that many stages earlier are complete.
+// five + four in both passes, plus 16 KB for the level tables of 4-bit rows (the token slots hide the L2
+// latency of the TMA loads; a fifth weight slot was worth +9..13 % in the forward pass, a sixth does not fit beside
+// the table cache, and reading the tables through L1 instead cost more than the sixth slot gave).  A weight slot
+// is free once the MMAs of that many stages earlier are complete; the weight ring must not be shallower than the
+// token ring (the TMA warp also loads factor tiles into weight slots).
 constexpr int kStagesA_fwd = 5, kStagesA_bwd = 5;
 constexpr int kStagesB_fwd = 4, kStagesB_bwd = 4;
 constexpr int kMaxStagesA = 6;
