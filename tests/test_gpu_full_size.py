@@ -94,3 +94,27 @@ def test_full_size_matrix(name, N, K, mix, mid):
     assert np.all(np.abs(got - sse_ref) <= 2.0 ** -21 * sse_ref)
     rr = np.unique(np.concatenate([[0, N - 1], rng.choice(N, 62, replace=False)]))
     assert np.array_equal(res[torch.from_numpy(rr).cuda()].cpu().numpy().view(np.uint32), res_ref[rr].view(np.uint32))
+
+
+@pytest.mark.parametrize("M", [1024, 8192])
+def test_token_sweep_forward(M):
+    """Config 5 (mix of 2 and 4 bits only) runs the forward pass at 1024, 4096 and 8192 tokens; 4096 is covered
+    above.  up_proj shape of the 7B model, sampled token rows."""
+    import paper_2502_08141_b200 as lw
+
+    N, K, r, s, mid = 11008, 4096, 64, 2.0, 5
+    case = make_case(N, K, {2: 0.75, 4: 0.25}, matrix_id=mid, lloyd_iters=2)
+    layout = lw.Layout(case.precs, K)
+    X = si.activations(M, K, matrix_id=500 + M)
+    A, B = si.lora_factors(K, N, r, matrix_id=mid)
+    rng = np.random.default_rng(M)
+    rows = np.unique(np.concatenate([[0, 255, 256, M - 1], rng.choice(M, 60, replace=False)]))
+    ws = torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")
+    Y = lw.lowra_lora_forward(layout, _dev(case.packed), _dev(case.absmax), _dev(case.maps), _bf(X), _bf(A), _bf(B), s,
+                              workspace=ws)
+    assert lw.lowra_device_status(ws) == lw.LOWRA_OK
+    got = si.bf16_bits_to_f32(_bits(Y[torch.from_numpy(rows).cuda()]))
+    ref = oracle.lora_forward(case.W_hat, X[rows], A, B, s)
+    emax, efro = gemm_errors(got, ref)
+    assert emax <= MAX_TOL and efro <= FRO_TOL, (M, emax, efro)
+    assert torch.isfinite(Y.float()).all()
