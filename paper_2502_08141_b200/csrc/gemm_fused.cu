@@ -423,6 +423,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (ok == 0u) return false;
                     if (ok == 2u) return true;                        // timed out: the abort flag ends the loop below
+                    (void)ptx::flag_test(P.sk_flags + c * CL + (int)crank);   // every lane's own acquire before its loads
                 }
                 const int m0 = t.mt * kTileT;
 #pragma unroll 1
