@@ -268,6 +268,14 @@ lowra_status lowra_learn_codebooks(const lowra_layout* layout, const float* W_de
 lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_dev, int32_t M, int32_t N, int32_t K,
                             uint16_t* C_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/*
+ * Diagnostic, not part of the method: the same product as lowra_dense_nt through the two-CTA form of the
+ * tensor-core instruction (two neighbouring SMs share a 256 x 256 tile, each holding half of either operand).
+ * Measures what that form is worth for this pipeline; arguments and errors as lowra_dense_nt.
+ */
+lowra_status lowra_dense_nt_pair(const uint16_t* P_dev, const uint16_t* Q_dev, int32_t M, int32_t N, int32_t K,
+                                 uint16_t* C_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -29,6 +29,7 @@ EXPORTS = (
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
     "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
+    "lowra_dense_nt_pair",
 )
 
 
@@ -96,6 +97,8 @@ def lib() -> ctypes.CDLL:
         L.lowra_device_status.restype = ctypes.c_int
         L.lowra_dense_nt.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
         L.lowra_dense_nt.restype = ctypes.c_int
+        L.lowra_dense_nt_pair.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
+        L.lowra_dense_nt_pair.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -387,6 +390,23 @@ def lowra_lora_backward_adapters(X, dY, A, B, s: float, dA: Optional[torch.Tenso
 def lowra_device_status(workspace: torch.Tensor, stream=None) -> int:
     """Synchronises the stream and returns the status word of the last fused call."""
     return int(lib().lowra_device_status(_ptr(workspace), _stream(stream)))
+
+
+def lowra_dense_nt_pair(P: torch.Tensor, Q: torch.Tensor, C: Optional[torch.Tensor] = None,
+                        workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Diagnostic: C = P . Q^T through the two-CTA form of the tensor-core instruction."""
+    _dev(P, torch.bfloat16, "P")
+    _dev(Q, torch.bfloat16, "Q")
+    M, K = P.shape
+    N = Q.shape[0]
+    if C is None:
+        C = torch.empty((M, N), dtype=torch.bfloat16, device=P.device)
+    if workspace is None:
+        workspace = torch.empty(256, dtype=torch.uint8, device=P.device)
+    code = lib().lowra_dense_nt_pair(_ptr(P), _ptr(Q), int(M), int(N), int(K), _ptr(C), _ptr(workspace),
+                                     workspace.numel(), _stream(stream))
+    _check(code, "lowra_dense_nt_pair")
+    return C
 
 
 def lowra_dense_nt(P: torch.Tensor, Q: torch.Tensor, C: Optional[torch.Tensor] = None,

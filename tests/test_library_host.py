@@ -94,6 +94,8 @@ def test_validation_runs_before_any_device_work(lib):
     sargs[8] = 24
     assert L.lowra_lora_forward_static(*sargs) == lib.LOWRA_ERR_SHAPE
     assert L.lowra_dense_nt(4096, 4096, 16, 16, 100, 4096, 4096, 256, None) == lib.LOWRA_ERR_SHAPE
+    assert L.lowra_dense_nt_pair(4096, 4096, 16, 16, 100, 4096, 4096, 256, None) == lib.LOWRA_ERR_SHAPE
+    assert L.lowra_dense_nt_pair(4096, None, 16, 16, 128, 4096, 4096, 256, None) == lib.LOWRA_ERR_NULL
     init = (ctypes.c_double * 48)()
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, None, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_NULL
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, init, init, -1, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
