@@ -1,4 +1,4 @@
-"""Seeded random shapes through every tensor-core entry point and the error kernel, against the oracle.
+"""Seeded random shapes through the codec, every tensor-core entry point and the error kernel, against the oracle.
 
 Shapes the hand-picked cases do not hit: channel counts that are any multiple of 8, contraction lengths that are
 any multiple of 128, token counts from 1 upwards, every rank from 16 to 128, eight precision mixes (three of them
@@ -46,6 +46,16 @@ def test_random_shape(N, K, M, r, mix_id, mid):
     s = (0.5, 1.0, 2.0)[mid % 3]
     packed, absmax, maps = dev(case.packed), dev(case.absmax), dev(case.maps)
     ws = torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")
+
+    # codec and row reordering: bit-exact
+    p_gpu, a_gpu = lw.lowra_encode(layout, dev(case.W), dev(case.thr))
+    assert np.array_equal(p_gpu.cpu().numpy()[:layout.packed_bytes], case.packed)
+    assert np.array_equal(a_gpu.cpu().numpy().view(np.uint32), case.absmax.view(np.uint32))
+    assert np.array_equal(bits(lw.lowra_decode(layout, packed, absmax, maps)), case.W_hat)
+    off = torch.from_numpy(lw.lowra_natural_offsets(case.precs, K).view(np.int64)).cuda()
+    nat, a_nat = lw.lowra_reorder_rows(layout, True, off, packed, absmax)
+    back, a_back = lw.lowra_reorder_rows(layout, False, off, nat, a_nat)
+    assert torch.equal(back, packed) and torch.equal(a_back, absmax)
 
     Y = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
     lw.lowra_lora_forward(layout, packed, absmax, maps, bf(X), bf(A), bf(B), s, Y=Y, workspace=ws)
