@@ -2,6 +2,7 @@
 
     python -m paper_2502_08141_b200.profile_case forward     # fused forward,  N = K = 4096, 2048 tokens, rank 64
     python -m paper_2502_08141_b200.profile_case backward    # fused backward-input, same shapes
+    python -m paper_2502_08141_b200.profile_case forward4096 # fused forward at 4096 tokens (264 tiles: stream-K schedule)
     python -m paper_2502_08141_b200.profile_case codec       # decode + encode of an 11008 x 4096 matrix
     python -m paper_2502_08141_b200.profile_case learn       # codebook learner, 4096 x 4096, 10 iterations
     python -m paper_2502_08141_b200.profile_case adapters    # gradients of the low-rank factors, 4096 x 11008, 4096 tokens
@@ -46,7 +47,7 @@ def main(case: str) -> None:
         return
     cfg = si.config(3)
     N, K = (11008, 4096) if case in ("codec", "errors") else (4096, 4096)
-    M, r, s = 2048, cfg.rank, cfg.s
+    M, r, s = (4096 if case == "forward4096" else 2048), cfg.rank, cfg.s
     precs = si.precisions(N, cfg.mix)
     maps, thr = si.standin_codebooks(precs)
     layout = Layout(precs, K)
@@ -83,12 +84,12 @@ def main(case: str) -> None:
         torch.cuda.synchronize()
         print("codec ok")
         return
-    act_cols = K if case == "forward" else N
+    act_cols = K if case in ("forward", "forward4096") else N
     act = torch.randn(M, act_cols, device="cuda", generator=gen).bfloat16()
     A = (torch.randn(K, r, device="cuda", generator=gen) * 0.01).bfloat16()
     B = (torch.randn(r, N, device="cuda", generator=gen) * 0.01).bfloat16()
     ws = torch.empty(lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")
-    fn = lowra_lora_forward if case == "forward" else lowra_lora_backward_input
+    fn = lowra_lora_forward if case in ("forward", "forward4096") else lowra_lora_backward_input
     for _ in range(3):
         fn(layout, packed, absmax, maps_d, act, A, B, s, workspace=ws)
     status = lowra_device_status(ws)
