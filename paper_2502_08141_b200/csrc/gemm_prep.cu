@@ -83,6 +83,13 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
 __device__ __forceinline__ uint32_t list_slot(uint32_t n, int cta) {
     return (n / kProducerWarps) * kListWarps + (n % kProducerWarps) * kCluster + (uint32_t)cta;
 }
+// The chunks of a group are sorted by precision, so its last chunk is the dearest one (it holds the group's 4-bit
+// rows, usually next to 2-bit ones: two code paths).  Which of a group's four warps takes which chunk therefore
+// rotates from one group pair to the next; a warp still gets one chunk of every second group of its CTA, in order.
+__device__ __forceinline__ uint32_t chunk_slot(uint32_t n0, uint32_t ci, int cta) {
+    const uint32_t pair = n0 / kProducerWarps;                    // n0 = 4 * (group's number within its CTA)
+    return list_slot((n0 & ~3u) + ((ci + pair) & 3u), cta);
+}
 
 __device__ void deal_backward(const PrepParams& P, int blk) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, tid = threadIdx.x;
@@ -118,7 +125,7 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
 #pragma unroll
         for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total_c[c - 1];
         if (lane < kChunks)
-            P.heads[list_slot(n0 + (uint32_t)lane, cta)] = (uint32_t)grp | ((uint32_t)(kStageArrivals / kChunks) << 24);
+            P.heads[chunk_slot(n0, (uint32_t)lane, cta)] = (uint32_t)grp | ((uint32_t)(kStageArrivals / kChunks) << 24);
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
 #pragma unroll
@@ -146,7 +153,7 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
                         const int cnt = __popc(mask[0][c] & (0x01010101u << res)) + __popc(mask[1][c] & (0x01010101u << res));
                         pos += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
                     }
-                    uint4* dst = rows + (size_t)list_slot(n0 + (uint32_t)(pos / 16), cta) * 32 + pos % 16;
+                    uint4* dst = rows + (size_t)chunk_slot(n0, (uint32_t)(pos / 16), cta) * 32 + pos % 16;
                     dst[0] = rec;
                     dst[16] = rec;
                 }
