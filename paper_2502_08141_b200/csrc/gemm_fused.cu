@@ -44,8 +44,10 @@ struct Barriers {
     uint64_t tmem_full[2];
     uint64_t tmem_empty[2];
     uint64_t drain;
+    uint64_t part_full;   // stream-K: a partial tile has been copied into the (idle) operand ring
     uint32_t tmem_base;
     uint32_t abort;
+    uint32_t epi_leave[2];             // the epilogue warps' common answer to "has somebody given up?"
     uint32_t produced[kMaxStagesA];    // arrivals of this CTA's dequant warps on the stage being filled
     uint32_t free_upto[kCluster];   // stages 0 .. free_upto[c] - 1 have been found free by the TMA
                                        // producer of CTA c of the cluster (every CTA holds a copy of all counters)
@@ -189,47 +191,55 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? super_t : 0;
     const int n_tiles = n_t_tiles + P.tiles_r * super_t;    // per cluster
     const int B = P.main_blocks + P.lora_blocks;            // contraction blocks of a weight tile
-    // Schedule.  Whole tiles: cluster c takes tiles c, c + NC, ... (the T tiles come first).  Stream-K (large
-    // problems whose tile count is not a multiple of NC): cluster c < n_t_tiles takes T tile c; the blocks of all
-    // weight tiles, laid end to end, are cut into NC consecutive ranges of equal length (less sk_tau blocks for a
-    // cluster that has a T tile), so a range starts and ends anywhere inside a tile.  A slice that does not start
-    // its tile leaves its sums in the cluster's partial-tile slot; the cluster that starts the tile collects them.
+    // Schedule.  The pieces of work are numbered g = 0, 1, ...: first the T tiles, then the weight tiles; cluster c
+    // takes g = c, c + NC, c + 2 NC, ... ("rows" of NC pieces; the clusters then sweep the contraction in step and
+    // share the token operand in time).  Whole tiles only: all rows, the last one partly empty.  Stream-K (tile
+    // count not a multiple of NC): only the first sk_dp rows; the contraction blocks of the remaining weight tiles,
+    // laid end to end, are cut into NC equal consecutive ranges, so a range starts and ends anywhere inside a tile.
+    // A slice that does not start its tile leaves its fp32 sums in the cluster's partial-tile slot; the cluster
+    // whose range starts the tile collects them: written into its accumulator before its MMAs begin (sk_late == 0:
+    // hidden behind the whole tiles in between, which needs long ranges) or added in its epilogue (sk_late == 1).
     const bool sk = MODE != kModeDense && P.sk != 0;
-    auto sk_lo = [&](int c) -> long long {
-        return ((long long)c * P.sk_total) / NC - (long long)min(c, n_t_tiles) * P.sk_tau;
-    };
+    const int w_dp = sk ? P.sk_dp : 0;                      // rows of whole pieces before the ranges
+    const int sk_first = w_dp * NC - n_t_tiles;             // first weight tile of the stream-K part
+    auto sk_lo = [&](int c) -> long long { return ((long long)c * P.sk_total) / NC; };
     const long long lo = sk ? sk_lo(cid) : 0, hi = sk ? sk_lo(cid + 1) : 0;
     const int tile0 = sk ? (int)(lo / B) : 0;
-    const int n_t_mine = sk ? (cid < n_t_tiles ? 1 : 0) : 0;
     const int n_wsegs = (sk && hi > lo) ? (int)((hi - (long long)tile0 * B + B - 1) / B) : 0;
-    // a range that starts inside a tile does that slice second, after its first whole tile: by then T is there
-    // (the slice may hold the tile's LoRA blocks) and the cluster that collects it is far from needing it
-    const bool swap01 = sk && n_wsegs >= 2 && lo > (long long)tile0 * B && hi >= (long long)(tile0 + 2) * B;
-    const int n_segs = sk ? n_t_mine + n_wsegs : (n_tiles > cid ? (n_tiles - cid + NC - 1) / NC : 0);
+    const int n_segs = sk ? w_dp + n_wsegs : (n_tiles > cid ? (n_tiles - cid + NC - 1) / NC : 0);
     auto seg_at = [&](int i) {
         Seg t;
         t.part = t.pre = false;
         t.tile = 0;
-        const int g = sk ? cid : cid + i * NC;
-        if (sk ? (i < n_t_mine) : (g < n_t_tiles)) {
-            t.is_t = true; t.rt = 0; t.mt = g * CL + (int)crank; t.kb0 = 0; t.kb1 = P.main_blocks;
-        } else if (!sk) {
-            const int idx = g - n_t_tiles;
-            const int st = idx / P.tiles_r;
-            t.is_t = false; t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank; t.kb0 = 0; t.kb1 = B;
+        if (!sk || i < w_dp) {
+            const int g = cid + i * NC;
+            if (g < n_t_tiles) {
+                t.is_t = true; t.rt = 0; t.mt = g * CL + (int)crank; t.kb0 = 0; t.kb1 = P.main_blocks;
+            } else {
+                const int idx = g - n_t_tiles;
+                const int st = idx / P.tiles_r;
+                t.is_t = false; t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank; t.kb0 = 0; t.kb1 = B;
+            }
         } else {
-            int k = i - n_t_mine;
-            if (swap01 && k < 2) k = 1 - k;
-            t.tile = tile0 + k;
+            const int k = i - w_dp;
+            t.tile = tile0 + k;                             // counted from the first tile of the stream-K part
             const long long first = (long long)t.tile * B;
             t.kb0 = (k == 0) ? (int)(lo - first) : 0;
             t.kb1 = (hi < first + B) ? (int)(hi - first) : B;
-            const int st = t.tile / P.tiles_r;
-            t.is_t = false; t.rt = t.tile - st * P.tiles_r; t.mt = st * CL + (int)crank;
+            const int idx = sk_first + t.tile;
+            const int st = idx / P.tiles_r;
+            t.is_t = false; t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank;
             t.part = t.kb0 > 0;
             t.pre = t.kb0 == 0 && t.kb1 < B;
         }
         return t;
+    };
+    // the clusters cid + 1 .. c_end - 1 hold the rest of the tile that this cluster's range starts
+    auto contributors_end = [&](int tile) {
+        const long long tile_end = (long long)(tile + 1) * B;
+        int c_end = cid + 1;
+        while (c_end < NC && sk_lo(c_end) < tile_end) ++c_end;
+        return c_end;
     };
 
     if (threadIdx.x == 0) {
@@ -243,6 +253,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             ptx::mbar_init(&bars->tmem_empty[a], 4);
         }
         ptx::mbar_init(&bars->drain, 1);
+        ptx::mbar_init(&bars->part_full, 1);
         bars->abort = 0u;
         for (int c = 0; c < kCluster; ++c) bars->free_upto[c] = 0u;
         for (int c = 0; c < kMaxStagesA; ++c) bars->produced[c] = 0u;
@@ -348,7 +359,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 if (!ptx::mbar_wait(&bars->tmem_empty[acc], aph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileT;
-                const int kb_fresh = t.pre ? -1 : t.kb0;        // the block whose first MMA overwrites the accumulator
+                const int kb_fresh = (t.pre && !P.sk_late) ? -1 : t.kb0;   // the block whose first MMA overwrites the accumulator
                 for (int kb = t.kb0; kb < t.kb1; ++kb, ++it) {
                     const int s = (int)sb;                      // token slot
                     const uint32_t ph = phb;
@@ -399,6 +410,17 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         const int et = (warp - kFirstEpilogueWarp) * 32 + lane;
         uint16_t* out16 = reinterpret_cast<uint16_t*>(out_s);
         const int my_row = q * 32 + lane;
+        // The four epilogue warps share named barriers, so they must leave together: one thread reads the abort
+        // flag (any role may raise it at any time), the others take its answer after the barrier.  Two slots in
+        // turn, so that the next question cannot overwrite an answer that a slow warp has not read yet.
+        uint32_t agree_turn = 0;
+        auto agree_abort = [&]() -> bool {
+            if (et == 0) bars->epi_leave[agree_turn & 1u] = *abort_flag;
+            ptx::named_barrier_sync(1, 128);
+            const bool leave = *reinterpret_cast<volatile uint32_t*>(&bars->epi_leave[agree_turn & 1u]) != 0u;
+            ++agree_turn;
+            return leave;
+        };
         // Hand the accumulator of piece i to the MMA warp (four arrivals, one per warp).  A piece that starts a tile
         // whose later blocks belong to other clusters first gets their partial sums written into the accumulator;
         // the MMAs then add on top.  `wait` false: look at the partial tiles' flags once and come back later if one
@@ -407,10 +429,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             if (i >= n_segs) return true;
             const Seg t = seg_at(i);
             const uint32_t acc = (uint32_t)i & 1u;
-            if (t.pre) {
-                const long long tile_end = (long long)(t.tile + 1) * B;
-                int c_end = cid + 1;                                  // clusters cid + 1 .. c_end - 1 hold the rest
-                while (c_end < NC && sk_lo(c_end) < tile_end) ++c_end;
+            if (t.pre && !P.sk_late) {
+                const int c_end = contributors_end(t.tile);
                 for (int c = cid + 1; c < c_end; ++c) {
                     uint32_t ok = 1u;
                     if (lane == 0) {
@@ -468,16 +488,58 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             if (owed & (1u << acc)) { hand_over(i, true); owed &= ~(1u << acc); }
             // the four epilogue warps share named barriers, so they must agree on leaving
             if (!ptx::mbar_wait_warp(&bars->tmem_full[acc], aph, abort_flag, kWaitLimitNs)) bars->abort = 1u;
-            ptx::named_barrier_sync(1, 128);
-            if (*abort_flag != 0u) { failed = true; break; }
+            if (agree_abort()) { failed = true; break; }
             ptx::tc_fence_after();
             float* part = P.sk_part + ((size_t)cid * CL + crank) * ((size_t)kTileT * kTileR) + my_row;
+            // A piece that starts a tile which other clusters finish (sk_late): their partial tiles are added here.
+            // The piece is this cluster's last one and its MMAs are complete, so the operand ring is idle: every
+            // partial tile (128 KB, [token][row] fp32) is copied into it in one go and read from there.
+            const float* add = nullptr;
+            if (t.pre && P.sk_late) {
+                const int c_end = contributors_end(t.tile);
+                const float* ring = reinterpret_cast<const float*>(base) + my_row;
+                bool leave = false;
+                for (int c = cid + 1; c < c_end; ++c) {
+                    if (lane == 0 && !ptx::flag_wait(P.sk_flags + c * CL + (int)crank, abort_flag, kWaitLimitNs)) bars->abort = 1u;
+                    leave = agree_abort();             // also: everybody is done with the previous partial tile in the ring
+                    if (leave) break;
+                    if (et == 0) {
+                        constexpr uint32_t kBytes = (uint32_t)(kTileT * kTileR * 4), kPiece = 16384u;
+                        const unsigned char* src = reinterpret_cast<const unsigned char*>(
+                            P.sk_part + ((size_t)c * CL + crank) * ((size_t)kTileT * kTileR));
+                        ptx::mbar_arrive_expect_tx(&bars->part_full, kBytes);
+                        for (uint32_t off = 0; off < kBytes; off += kPiece)
+                            ptx::bulk_copy_g2s(ptx::smem_u32(base) + off, src + off, kPiece, &bars->part_full);
+                    }
+                    if (!ptx::mbar_wait_warp(&bars->part_full, (uint32_t)(c - cid - 1) & 1u, abort_flag, kWaitLimitNs)) bars->abort = 1u;
+                    leave = agree_abort();
+                    if (leave) break;
+                    if (c + 1 == c_end) { add = ring; break; }          // the last one is added on the way out, below
+#pragma unroll 1
+                    for (int chunk = 0; chunk < kTileT / 32; ++chunk) {   // the others go into the accumulator
+                        if (m0 + chunk * 32 >= P.M) break;
+                        uint32_t v[32];
+                        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileT + chunk * 32;
+                        ptx::tmem_ld_32x32(taddr, v);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + ring[(chunk * 32 + j) * kTileR]);
+                        ptx::tmem_st_32x32(taddr, v);
+                    }
+                    ptx::tmem_st_wait();
+                }
+                if (leave) { failed = true; break; }
+            }
 #pragma unroll 1
             for (int chunk = 0; chunk < kTileT / 32; ++chunk) {
                 if (m0 + chunk * 32 >= P.M) break;
                 uint32_t v[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileT + chunk * 32, v);
                 ptx::tmem_ld_wait();
+                if (add != nullptr) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + add[(chunk * 32 + j) * kTileR]);
+                }
                 if (t.part) {
                     // fp32 sums of a slice: [token][row], so that a warp writes 128 consecutive bytes
 #pragma unroll
@@ -843,20 +905,33 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
     cfg.gridDim = dim3((unsigned)(clusters * CL), 1, 1);
     GemmParams Q = G;
     Q.sk = 0;
-    // Under stream-K the clusters no longer sweep the contraction in step, so the token operand is not shared in
-    // time any more: it has to stay in L2 between its readers.  Measured on a 90 MB operand: 6.5 times the DRAM
-    // reads of the whole-tile schedule and no gain; so only operands that fit L2 with room to spare.
-    const bool operand_fits_l2 = (size_t)G.M * (size_t)G.C * 2u <= ((size_t)48 << 20);
-    if (MODE != kModeDense && G.sk_part != nullptr && clusters == max_clusters && n_t <= clusters &&
-        n_tiles % clusters != 0 && operand_fits_l2) {
-        // stream-K: equal shares of the weight tiles' blocks; a T tile counts as much as the dequantised blocks of
-        // a weight tile.  Only when every cluster still gets two tiles' worth or more.
+    if (MODE != kModeDense && G.sk_part != nullptr && clusters == max_clusters && n_t <= clusters && n_tiles % clusters != 0) {
+        // stream-K for the last rows of pieces.  The clusters' sweeps over the contraction fall out of step inside
+        // the ranges, so the token operand has to stay in L2 there.  If the whole operand does (<= 48 MB) and there
+        // are three rows or more, only the first row stays whole and the partial tiles are preloaded - hidden
+        // behind the whole tiles of the range.  Otherwise all full rows stay whole, only the last, incomplete row
+        // is cut into ranges (little of the operand is live then), and the partial tiles are added in the
+        // epilogue.  (Ranges from the start on a 90 MB operand: 6.5 times the DRAM reads, and no gain.)
         const int blocks = G.main_blocks + G.lora_blocks;
-        const long long total = (long long)G.tiles_r * super_t * blocks + (long long)n_t * G.main_blocks;
-        if (total / clusters >= (long long)G.main_blocks + 2 * blocks) {
+        const int rows = n_tiles / clusters;
+        const int n_last = n_tiles - rows * clusters;                  // pieces of the last, incomplete row
+        const size_t slab = (size_t)CL * kTileT * (size_t)G.C * 2u;    // token operand of one group of token tiles
+        const bool operand_fits_l2 = (size_t)G.M * (size_t)G.C * 2u <= ((size_t)48 << 20);
+        int dp = 0, late = 1;
+        if (operand_fits_l2 && rows >= 3) {
+            dp = 1; late = 0;
+        } else if (2 * n_last >= clusters) {
+            dp = rows;                    // two or three clusters per tile of the last row
+        } else if (rows >= 2 && (size_t)((n_last + clusters) / G.tiles_r + 2) * slab <= ((size_t)40 << 20)) {
+            dp = rows - 1;                // few tiles in the last row: every tile would be cut into many slices, each of
+                                          // which the collecting cluster adds one after the other; cut the last two rows
+        }
+        const long long n_rest = (long long)n_tiles - (long long)dp * clusters;       // weight tiles behind the whole rows
+        if (dp >= 1 && n_rest * blocks >= clusters) {
             Q.sk = 1;
-            Q.sk_tau = G.main_blocks;
-            Q.sk_total = total;
+            Q.sk_dp = dp;
+            Q.sk_late = late;
+            Q.sk_total = n_rest * blocks;
         }
     }
     if (cudaLaunchKernelEx(&cfg, fused_kernel<MODE>, Q, tmB, tmT, tmFt, tmFl) != cudaSuccess) return LOWRA_ERR_CUDA;

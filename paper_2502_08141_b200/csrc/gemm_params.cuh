@@ -88,8 +88,9 @@ struct GemmParams {
     float* sk_part;         // fp32 partial tiles, one [kCluster][kTileT][kTileR] slot per cluster
     uint32_t* sk_flags;     // [clusters] raised when a cluster's partial tile is complete
     int sk;
-    int sk_tau;             // blocks that a cluster with a T tile takes fewer
-    long long sk_total;     // blocks of all weight tiles + sk_tau per T tile
+    int sk_dp;              // rows of whole pieces (T tiles, then weight tiles, round-robin) before the ranges
+    int sk_late;            // 1: partial tiles are added in the collecting piece's epilogue; 0: preloaded into its accumulator
+    long long sk_total;     // contraction blocks of the weight tiles behind the whole rows
 };
 constexpr int kMaxClusters = kNumSMs / kCluster;
 constexpr size_t kSkSlotFloats = (size_t)kCluster * kTileT * kTileR;

@@ -326,6 +326,13 @@ __device__ __forceinline__ void bulk_copy_to_cta(uint32_t cdst, uint32_t src, ui
                  ::"r"(cdst), "r"(src), "r"(bytes), "r"(cbar)
                  : "memory");
 }
+// Asynchronous copy of `bytes` (a multiple of 16) from global memory into this CTA's shared memory, counted in bytes
+// on an mbarrier of this CTA.  Both addresses 16-byte aligned.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
 // All threads of all CTAs of the cluster.
 __device__ __forceinline__ void cluster_sync() {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
