@@ -20,9 +20,10 @@
 // (factor fetched by TMA, no dequant); T tiles come first in the tile order, their epilogue publishes a
 // per-token-tile flag, and the TMA producer of a regular tile waits (bounded) for that flag before it
 // fetches T.  All CTAs are co-resident and a T tile waits for nothing, so the wait cannot deadlock.
-// Schedule: whole tiles dealt round-robin to the clusters, or (launcher's choice) stream-K: equal consecutive
-// ranges of the weight tiles' contraction blocks per cluster, partial tiles handed over through a scratch slot
-// and preloaded into the accumulator of the cluster that starts the tile (see the schedule in the kernel).
+// Schedule: whole tiles dealt round-robin to the clusters, or (launcher's choice) stream-K behind the first rows of
+// whole tiles: equal consecutive ranges of the remaining weight tiles' contraction blocks per cluster, partial tiles
+// handed over through a scratch slot and either preloaded into the accumulator of the cluster that starts the tile
+// or added in its epilogue (see the schedule in the kernel).
 //
 // Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, eight of 6-15 = dequant.
 // All mbarrier waits are bounded; a wait that runs out sets the status word and every role leaves.

@@ -2,7 +2,8 @@
 
     python -m paper_2502_08141_b200.profile_case forward     # fused forward,  N = K = 4096, 2048 tokens, rank 64
     python -m paper_2502_08141_b200.profile_case backward    # fused backward-input, same shapes
-    python -m paper_2502_08141_b200.profile_case forward4096 # fused forward at 4096 tokens (264 tiles: stream-K schedule)
+    python -m paper_2502_08141_b200.profile_case forward4096 # fused forward at 4096 tokens (264 pieces: stream-K, preloaded partial tiles)
+    python -m paper_2502_08141_b200.profile_case backward_gate # fused backward-input, 11008 x 4096, 4096 tokens (stream-K on the last row)
     python -m paper_2502_08141_b200.profile_case codec       # decode + encode of an 11008 x 4096 matrix
     python -m paper_2502_08141_b200.profile_case learn       # codebook learner, 4096 x 4096, 10 iterations
     python -m paper_2502_08141_b200.profile_case adapters    # gradients of the low-rank factors, 4096 x 11008, 4096 tokens
@@ -46,8 +47,8 @@ def main(case: str) -> None:
         adapters()
         return
     cfg = si.config(3)
-    N, K = (11008, 4096) if case in ("codec", "errors") else (4096, 4096)
-    M, r, s = (4096 if case == "forward4096" else 2048), cfg.rank, cfg.s
+    N, K = (11008, 4096) if case in ("codec", "errors", "backward_gate") else (4096, 4096)
+    M, r, s = (4096 if case in ("forward4096", "backward_gate") else 2048), cfg.rank, cfg.s
     precs = si.precisions(N, cfg.mix)
     maps, thr = si.standin_codebooks(precs)
     layout = Layout(precs, K)
