@@ -2,7 +2,8 @@
 
 Shapes the hand-picked cases do not hit: channel counts that are any multiple of 8, contraction lengths that are
 any multiple of 128, token counts from 1 upwards, every rank from 16 to 128, eight precision mixes (three of them
-single-class), and six many-tile / short-contraction problems that run the stream-K schedule in one or both passes.
+single-class), six many-tile / short-contraction problems that run the stream-K schedule with preloaded partial tiles
+in one or both passes, and six with one to seven rows of pieces per cluster (partial tiles added in the epilogue).
 """
 import numpy as np
 import pytest
@@ -28,6 +29,11 @@ def _cases():
     for i, (N, K, M, r) in enumerate([(2304, 256, 6000, 16), (2312, 384, 5900, 48), (1160, 512, 12000, 128),
                                       (3072, 256, 4100, 96), (256, 2304, 6100, 32), (384, 2432, 5800, 64)]):
         out.append((N, K, M, r, (3 + i) % len(MIXES), 200 + i))
+    # between one and seven rows of pieces per cluster: whole rows first, then ranges over the last one or two
+    # (partial tiles added in the epilogue, one to three slices per tile)
+    for i, (N, K, M, r) in enumerate([(2680, 512, 8603, 16), (512, 2176, 3387, 64), (1536, 768, 6550, 96),
+                                      (1408, 256, 8137, 64), (3264, 256, 8757, 80), (2040, 384, 6829, 80)]):
+        out.append((N, K, M, r, (1 + i) % len(MIXES), 300 + i))
     return out
 
 
