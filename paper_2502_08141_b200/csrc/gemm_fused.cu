@@ -508,6 +508,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         constexpr uint32_t kBytes = (uint32_t)(kTileT * kTileR * 4), kPiece = 16384u;
                         const unsigned char* src = reinterpret_cast<const unsigned char*>(
                             P.sk_part + ((size_t)c * CL + crank) * ((size_t)kTileT * kTileR));
+                        // the slices were written with ordinary stores by other SMs and acquired through the flag by
+                        // this very thread: make them visible to the copy engine (async proxy) as well
+                        ptx::fence_proxy_async_all();
                         ptx::mbar_arrive_expect_tx(&bars->part_full, kBytes);
                         for (uint32_t off = 0; off < kBytes; off += kPiece)
                             ptx::bulk_copy_g2s(ptx::smem_u32(base) + off, src + off, kPiece, &bars->part_full);
