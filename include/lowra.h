@@ -142,7 +142,10 @@ lowra_status lowra_quant_error(const lowra_layout* layout, const float* W_dev, c
                                void* stream);
 
 /* Bytes of device scratch that lowra_lora_forward / lowra_lora_backward_input need for M tokens and
- * LoRA rank r (0 if the arguments are invalid).  The first 256 bytes hold the device status word. */
+ * LoRA rank r (0 if the arguments are invalid).  The first 256 bytes hold the device status word; the
+ * rest: the down-projected activations, flags, the deal of the rows to the dequant warps and 19 MB for
+ * the fp32 partial tiles that tiles cut between SMs are handed over in (about 21 MB for a 4096 x 11008
+ * matrix at 4096 tokens). */
 size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r);
 
 /*
@@ -219,8 +222,9 @@ lowra_status lowra_device_status(const void* workspace_dev, void* stream);
  * calls no allocating routine; inputs and outputs are still the caller's.
  *
  *   - Same arguments, results and errors as lowra_lora_forward, without the workspace.  If
- *     lowra_workspace_bytes(layout, M, r) exceeds LOWRA_STATIC_SCRATCH_BYTES the call launches nothing
- *     and returns LOWRA_ERR_LIMIT (for scale: N = K = 8192, M = 8192, r = 64 needs about 1.6 MB).
+ *     the scratch this entry needs (lowra_workspace_bytes(layout, M, r) less the partial tiles, which
+ *     it does without: tiles are never cut here) exceeds LOWRA_STATIC_SCRATCH_BYTES the call launches
+ *     nothing and returns LOWRA_ERR_LIMIT (for scale: N = K = 8192, M = 8192, r = 64 needs about 1.6 MB).
  *   - status_out_dev (optional, may be NULL): a device uint32 that receives the device status word
  *     (LOWRA_OK or LOWRA_ERR_TIMEOUT) once the call's kernels have run, since the built-in scratch cannot
  *     be given to lowra_device_status.
