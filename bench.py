@@ -491,6 +491,28 @@ def run_gpu(args):
             ms_q = a.elapsed_time(b)
             by = (8.0 if with_res else 4.0) * elems
             qe[key] = {"ms": ms_q, "GB/s": by / (ms_q * 1e-3) / 1e9, "frac_hbm": by / (ms_q * 1e-3) / 1e9 / P["hbm"]}
+        # every channel under 1, 2 and 4 bits in one pass (stand-in tables for all three precisions)
+        t3 = []
+        for d in dev:
+            m3 = np.zeros((3, d["m"]["N"], 16), dtype=np.float32); h3 = np.zeros_like(m3)
+            for c, b in enumerate((1, 2, 4)):
+                m3[c], h3[c] = si.standin_codebooks(np.full(d["m"]["N"], b, dtype=np.uint8))
+            t3.append((torch.from_numpy(m3).cuda(), torch.from_numpy(h3).cuda(),
+                       torch.empty((d["m"]["N"], 3), dtype=torch.float64, device="cuda")))
+
+        def errors3():
+            for d, (m3, h3, o3) in zip(dev, t3):
+                lw.lowra_channel_errors(d["W"], m3, h3, sse3=o3)
+        errors3()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        errors3()
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_q = a.elapsed_time(b)
+        qe["three_precisions_one_pass"] = {"ms": ms_q, "GB/s": 4.0 * elems / (ms_q * 1e-3) / 1e9,
+                                           "frac_hbm": 4.0 * elems / (ms_q * 1e-3) / 1e9 / P["hbm"]}
         qe["note"] = "not part of the step; algorithmic bytes = W read once (4 B per element) + residual written (4 B)"
         extras["quant_error"] = qe
 

@@ -141,6 +141,20 @@ lowra_status lowra_quant_error(const lowra_layout* layout, const float* W_dev, c
                                const float* thresholds_dev, double* sse_dev, float* residual_dev,
                                void* stream);
 
+/*
+ * The same error for every channel under 1, 2 and 4 bits in one pass over W (Section 5.1, step 1: each
+ * channel's error under 1-, 2- and 4-bit quantisation is what the channels are clustered by).  No
+ * layout: every row is quantised three times, with its own three codebooks.
+ *   W_dev            fp32 [N, K] row-major, K % 128 == 0                                        (in)
+ *   maps3_dev, thresholds3_dev   fp32 [3][N][16]: plane 0 = the 1-bit tables of every row, plane 1 =
+ *                    the 2-bit tables, plane 2 = the 4-bit tables (as lowra_learn_codebooks writes them
+ *                    for a layout in which every row has that precision)                       (in)
+ *   sse3_dev         fp64 [N][3], the three errors of a row side by side; arithmetic and accuracy as
+ *                    lowra_quant_error                                                          (out)
+ */
+lowra_status lowra_channel_errors(int32_t N, int32_t K, const float* W_dev, const float* maps3_dev,
+                                  const float* thresholds3_dev, double* sse3_dev, void* stream);
+
 /* Bytes of device scratch that lowra_lora_forward / lowra_lora_backward_input need for M tokens and
  * LoRA rank r (0 if the arguments are invalid).  The first 256 bytes hold the device status word; the
  * rest: the down-projected activations, flags, the deal of the rows to the dequant warps and 19 MB for

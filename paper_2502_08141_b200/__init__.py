@@ -29,7 +29,7 @@ EXPORTS = (
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
     "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
-    "lowra_dense_nt_pair",
+    "lowra_dense_nt_pair", "lowra_channel_errors",
 )
 
 
@@ -86,6 +86,8 @@ def lib() -> ctypes.CDLL:
         L.lowra_natural_offsets.restype = ctypes.c_int
         L.lowra_reorder_rows.argtypes = [lp, i32, vp, vp, vp, vp, vp, vp]
         L.lowra_reorder_rows.restype = ctypes.c_int
+        L.lowra_channel_errors.argtypes = [i32, i32, vp, vp, vp, vp, vp]
+        L.lowra_channel_errors.restype = ctypes.c_int
         L.lowra_quant_error.argtypes = [lp, vp, vp, vp, vp, vp, vp]
         L.lowra_quant_error.restype = ctypes.c_int
         L.lowra_adapter_workspace_bytes.argtypes = [i32, i32]
@@ -355,6 +357,22 @@ def lowra_quant_error(layout: Layout, W: torch.Tensor, maps: torch.Tensor, thres
                                    _ptr(residual) if residual is not None else None, _stream(stream))
     _check(code, "lowra_quant_error")
     return sse, residual
+
+
+def lowra_channel_errors(W: torch.Tensor, maps3: torch.Tensor, thresholds3: torch.Tensor,
+                         sse3: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    """Summed square error of every row of W under 1, 2 and 4 bits (fp64 [N,3]); tables fp32 [3,N,16]."""
+    _dev(W, torch.float32, "W")
+    _dev(maps3, torch.float32, "maps3")
+    _dev(thresholds3, torch.float32, "thresholds3")
+    N, K = int(W.shape[0]), int(W.shape[1])
+    if tuple(maps3.shape) != (3, N, 16) or tuple(thresholds3.shape) != (3, N, 16):
+        raise ValueError("shape mismatch")
+    if sse3 is None:
+        sse3 = torch.empty((N, 3), dtype=torch.float64, device=W.device)
+    code = lib().lowra_channel_errors(N, K, _ptr(W), _ptr(maps3), _ptr(thresholds3), _ptr(sse3), _stream(stream))
+    _check(code, "lowra_channel_errors")
+    return sse3
 
 
 def lowra_adapter_workspace_bytes(M: int, r: int) -> int:

@@ -1,4 +1,5 @@
 // lowra_quant_error: summed square error per output channel and, optionally, the residual W - W_hat.
+// lowra_channel_errors: the same error under 1, 2 and 4 bits at once (one read of W), without a layout.
 //
 // The precision assigner minimises the summed square error between the weights and their quantised
 // counterparts (paper Section 5 and its footnote; Section 5.1 starts from every channel's error under 1, 2 and
@@ -133,6 +134,85 @@ __global__ void __launch_bounds__(kErrThreads) error_kernel(const ErrParams P) {
     }
 }
 
+// ---- all three precisions in one pass (the assigner's input: every channel's error under 1, 2 and 4 bits) ----
+struct Err3Params {
+    const float* W;           // [N, K]
+    const float* maps;        // [3][N][16]: tables of the 1-, 2- and 4-bit codebooks of every row
+    const float* thresholds;  // [3][N][16]
+    double* sse;              // [N][3]
+    int N, K;
+};
+
+__global__ void __launch_bounds__(kErrThreads) error3_kernel(const Err3Params P) {
+    __shared__ float y_smem[kErrWarps][16];
+    pdl_enter();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    float* y_warp = y_smem[warp];
+    const int K = P.K, n4 = K / 4;
+    const size_t plane = (size_t)P.N * kTableStride;
+    for (int r = blockIdx.x * kErrWarps + warp; r < P.N; r += gridDim.x * kErrWarps) {
+        const float* wrow = P.W + (size_t)r * K;
+        const float* t1 = P.thresholds + (size_t)r * kTableStride;
+        const float* y1 = P.maps + (size_t)r * kTableStride;
+        const float ta[3] = {__ldg(t1), 0.f, 0.f};
+        const float ya[4] = {__ldg(y1), __ldg(y1 + 1), 0.f, 0.f};
+        const float tb[3] = {__ldg(t1 + plane), __ldg(t1 + plane + 1), __ldg(t1 + plane + 2)};
+        const float yb[4] = {__ldg(y1 + plane), __ldg(y1 + plane + 1), __ldg(y1 + plane + 2), __ldg(y1 + plane + 3)};
+        Thresholds4 t4;
+        t4.load(t1 + 2 * plane);
+        __syncwarp();   // the previous row's look-ups are over
+        if (lane < 16) y_warp[lane] = __ldg(y1 + 2 * plane + lane);
+        __syncwarp();
+        double acc1 = 0.0, acc2 = 0.0, acc4 = 0.0;
+        float4 nxt[kErrBatch];
+#pragma unroll
+        for (int u = 0; u < kErrBatch; ++u) {
+            const int i = lane + u * 32;
+            nxt[u] = (i < n4) ? ld_stream_f4(wrow + (size_t)i * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        for (int base = lane; base < n4; base += 32 * kErrBatch) {
+            float4 x[kErrBatch];
+#pragma unroll
+            for (int u = 0; u < kErrBatch; ++u) {
+                x[u] = nxt[u];
+                const int i = base + 32 * kErrBatch + u * 32;
+                nxt[u] = (i < n4) ? ld_stream_f4(wrow + (size_t)i * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < kErrBatch; ++u) {
+                const int i = base + u * 32;
+                float m = fmaxf(fmaxf(fabsf(x[u].x), fabsf(x[u].y)), fmaxf(fabsf(x[u].z), fabsf(x[u].w)));
+#pragma unroll
+                for (int d = 8; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+                const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
+                const float xs[4] = {x[u].x, x[u].y, x[u].z, x[u].w};
+                float n[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) n[e] = __fmul_rn(xs[e], inv);
+                // squared residuals of the four elements at one precision, added in fp32
+                auto group = [&](auto level) -> float {
+                    const uint32_t h01 = pack_bf16x2(__fmul_rn(level(n[0]), m), __fmul_rn(level(n[1]), m));
+                    const uint32_t h23 = pack_bf16x2(__fmul_rn(level(n[2]), m), __fmul_rn(level(n[3]), m));
+                    const float r0 = __fsub_rn(xs[0], __uint_as_float(h01 << 16)), r1 = __fsub_rn(xs[1], __uint_as_float(h01 & 0xFFFF0000u));
+                    const float r2 = __fsub_rn(xs[2], __uint_as_float(h23 << 16)), r3 = __fsub_rn(xs[3], __uint_as_float(h23 & 0xFFFF0000u));
+                    return __fadd_rn(__fadd_rn(__fmul_rn(r0, r0), __fmul_rn(r1, r1)), __fadd_rn(__fmul_rn(r2, r2), __fmul_rn(r3, r3)));
+                };
+                const float q1 = group([&](float v) { return level_of<1>(v, ta, t4, ya, y_warp); });
+                const float q2 = group([&](float v) { return level_of<2>(v, tb, t4, yb, y_warp); });
+                const float q4 = group([&](float v) { return level_of<4>(v, tb, t4, yb, y_warp); });
+                if (i < n4) { acc1 += (double)q1; acc2 += (double)q2; acc4 += (double)q4; }
+            }
+        }
+#pragma unroll
+        for (int d = 16; d >= 1; d >>= 1) {
+            acc1 += __shfl_xor_sync(0xffffffffu, acc1, d);
+            acc2 += __shfl_xor_sync(0xffffffffu, acc2, d);
+            acc4 += __shfl_xor_sync(0xffffffffu, acc4, d);
+        }
+        if (lane == 0) { P.sse[(size_t)r * 3] = acc1; P.sse[(size_t)r * 3 + 1] = acc2; P.sse[(size_t)r * 3 + 2] = acc4; }
+    }
+}
+
 }  // namespace
 }  // namespace lowra
 
@@ -159,4 +239,26 @@ extern "C" lowra_status lowra_quant_error(const lowra_layout* layout, const floa
     const int want = (layout->N + kErrWarps - 1) / kErrWarps;
     const unsigned grid = (unsigned)(want < cap ? want : cap);
     return launch_pdl(error_kernel, grid, kErrThreads, (cudaStream_t)stream, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+}
+
+extern "C" lowra_status lowra_channel_errors(int32_t N, int32_t K, const float* W_dev, const float* maps3_dev,
+                                             const float* thresholds3_dev, double* sse3_dev, void* stream) {
+    using namespace lowra;
+    if (!W_dev || !maps3_dev || !thresholds3_dev || !sse3_dev) return LOWRA_ERR_NULL;
+    if (N < 1 || K < 128 || K % 128 != 0) return LOWRA_ERR_SHAPE;
+    if (!aligned16(W_dev) || !aligned16(maps3_dev) || !aligned16(thresholds3_dev) || (reinterpret_cast<uintptr_t>(sse3_dev) & 7u) != 0)
+        return LOWRA_ERR_ALIGN;
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    Err3Params P;
+    P.W = W_dev;
+    P.maps = maps3_dev;
+    P.thresholds = thresholds3_dev;
+    P.sse = sse3_dev;
+    P.N = N;
+    P.K = K;
+    const int cap = kNumSMs * 4;
+    const int want = (N + kErrWarps - 1) / kErrWarps;
+    return launch_pdl(error3_kernel, (unsigned)(want < cap ? want : cap), kErrThreads, (cudaStream_t)stream, P) == cudaSuccess
+               ? LOWRA_OK : LOWRA_ERR_CUDA;
 }

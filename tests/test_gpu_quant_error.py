@@ -88,3 +88,24 @@ def test_error_of_the_learned_codebooks_falls_with_the_precision(lw):
         assert np.all(np.abs(sse.cpu().numpy() - ref) <= RTOL * ref)
         errs.append(sse.cpu().numpy())
     assert (errs[1] < errs[0]).all() and (errs[2] < errs[1]).all()
+
+
+@pytest.mark.parametrize("N,K", [(24, 128), (100, 1152), (300, 4096), (40, 11008)])
+def test_three_precisions_in_one_pass(lw, N, K):
+    """Every row under 1, 2 and 4 bits with its own three codebooks: equal to three calls of the oracle with uniform
+    precisions, and bit-identical to three calls of lowra_quant_error (same arithmetic, same order)."""
+    W_np = si.weights(N, K, matrix_id=(N + K) % 50)
+    W = torch.from_numpy(np.ascontiguousarray(W_np)).cuda()
+    maps3 = np.zeros((3, N, 16), dtype=np.float32)
+    thr3 = np.zeros((3, N, 16), dtype=np.float32)
+    ref = np.zeros((N, 3))
+    single = np.zeros((N, 3))
+    for c, b in enumerate((1, 2, 4)):
+        precs = np.full(N, b, dtype=np.uint8)
+        maps3[c], thr3[c] = oracle.lloyd_max(W_np, precs, T=2)
+        ref[:, c], _ = oracle.quant_error(W_np, precs, maps3[c], thr3[c])
+        sse, _ = lw.lowra_quant_error(lw.Layout(precs, K), W, torch.from_numpy(maps3[c]).cuda(), torch.from_numpy(thr3[c]).cuda())
+        single[:, c] = sse.cpu().numpy()
+    got = lw.lowra_channel_errors(W, torch.from_numpy(maps3).cuda(), torch.from_numpy(thr3).cuda()).cpu().numpy()
+    assert np.all(np.abs(got - ref) <= RTOL * ref)
+    assert np.array_equal(got, single)

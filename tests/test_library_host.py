@@ -118,6 +118,10 @@ def test_validation_runs_before_any_device_work(lib):
     assert L.lowra_quant_error(ctypes.byref(lay), 4096 + 4, 4096, 4096, 4096, None, None) == lib.LOWRA_ERR_ALIGN
     assert L.lowra_quant_error(ctypes.byref(lay), 4096, 4096, 4096, 4096, 4096 + 8, None) == lib.LOWRA_ERR_ALIGN
     assert L.lowra_quant_error(None, 4096, 4096, 4096, 4096, None, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_channel_errors(16, 256, 4096, 4096, 4096, None, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_channel_errors(16, 200, 4096, 4096, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
+    assert L.lowra_channel_errors(0, 256, 4096, 4096, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
+    assert L.lowra_channel_errors(16, 256, 4096 + 4, 4096, 4096, 4096, None) == lib.LOWRA_ERR_ALIGN
     # adapter gradients: X, dY, M, K, N, A, B, r, s, dA, dB, workspace, bytes, stream
     big = 1 << 30
     assert L.lowra_adapter_workspace_bytes(0, 16) == 0
