@@ -25,7 +25,7 @@
 // handed over through a scratch slot and either preloaded into the accumulator of the cluster that starts the tile
 // or added in its epilogue (see the schedule in the kernel).
 //
-// Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, eight of 6-15 = dequant.
+// Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, 6-8 / 10-12 / 14-15 = dequant.
 // All mbarrier waits are bounded; a wait that runs out sets the status word and every role leaves.
 #include "gemm_params.cuh"
 #include "ptx.cuh"
@@ -594,16 +594,14 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 }
             }
         }
-    } else if (MODE != kModeDense && ((MODE == kModeForward) ? (warp & 3) != 1 : warp < kFirstProducerWarp + kProducerWarps)) {
+    } else if (MODE != kModeDense && (warp & 3) != 1) {
         // ================================================================== dequant producers
         // The prologue has dealt the rows to these warps (see gemm_prep.cu).  Each thread dequantises one
         // 64-element absmax block per visit of a stage.
-        // Forward: warps 6-8, 10-12, 14, 15 (9 and 13 would share the MMA warp's scheduler and idle instead: the
-        // dequant work is light, the MMA warp's instruction latency is what counts).  Backward: warps 6-13, two
-        // per scheduler (the dequant work is heavier there; 14 and 15 idle).
+        // Warps 6-8, 10-12, 14, 15: warps 9 and 13 would share the MMA warp's scheduler and idle instead (the MMA
+        // warp's instruction latency is what paces the CTA).
         const int K = P.L.K;
-        const int pw = (MODE == kModeForward) ? (warp - kFirstProducerWarp) - (warp > 9 ? 1 : 0) - (warp > 13 ? 1 : 0)
-                                              : warp - kFirstProducerWarp;   // 0 .. kProducerWarps - 1
+        const int pw = (warp - kFirstProducerWarp) - (warp > 9 ? 1 : 0) - (warp > 13 ? 1 : 0);   // 0 .. kProducerWarps - 1
         const uint32_t tab_warp = ptx::smem_u32(tab_all) + (uint32_t)pw * 2048u;   // this warp's 2 KB of level tables (4-bit rows)
         const uint32_t tab_lane = tab_warp + (uint32_t)lane * 64u;                  // forward: this lane's table
         uint32_t it0 = 0;                                       // running stage index at the start of the tile

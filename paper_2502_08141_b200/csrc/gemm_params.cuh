@@ -53,8 +53,8 @@ constexpr int kStagesB_fwd = 4, kStagesB_bwd = 4;
 constexpr int kMaxStagesA = 6;
 constexpr int kFirstEpilogueWarp = 2;
 constexpr int kFirstProducerWarp = 6;
-// 16 warps, of which two idle (which two depends on the pass, see the kernel): at most four per scheduler, so
-// 128 registers per thread.
+// 16 warps, of which two idle (the two that would share the MMA warp's scheduler): at most four per scheduler,
+// so 128 registers per thread.
 constexpr int kGemmWarps = 16;
 constexpr int kGemmThreads = 32 * kGemmWarps;
 static_assert(kProducerWarps == 8, "the warp map above places eight dequant warps");
