@@ -159,13 +159,12 @@ def make_host_inputs(cfg, rank: int):
     return mats, acts
 
 
-# DRAM traffic of one fused_kernel launch measured with ncu on the small profiling case (N = K = 4096,
-# 2048 tokens, rank 64, 1.5 bits on average; dram__bytes_read.sum + dram__bytes_write.sum): forward 22.4 + 9.2 MB,
-# backward-input 22.5 + 9.0 MB.  The reads equal the case's input bytes (activations + packed codes + absmax +
-# tables + LoRA factors = 22.1 MB: nothing is read twice); of the 16.8 MB of bf16 output a good half has reached
-# DRAM when the kernel ends, the rest is still in L2.  Scaled to a launch of the bench in proportion to its
-# input + output bytes.
-NCU_CASE = dict(N=4096, K=4096, M=2048, r=64, bits=1.5, dram_bytes=0.5 * (22.4e6 + 9.2e6 + 22.5e6 + 9.0e6))
+# DRAM traffic of one fused_kernel launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a
+# launch of this very workload: the backward-input pass of gate_proj (dX [4096, 4096] from dY [4096, 11008];
+# profiles/fused_backward_input_11008x4096_m4096_streamk.md): 168.2 MB read + 26.9 MB written.  The bytes the call
+# has to read and write once are 137 MB (the output is partly still in L2 when the kernel ends; the stream-K partial
+# tiles add 19 MB each way).  Scaled to the step's average launch in proportion to those input + output bytes.
+NCU_CASE = dict(N=4096, K=11008, M=4096, r=64, bits=1.5, dram_bytes=168.2e6 + 26.9e6)
 
 
 def fused_io_bytes(N, K, M, r, bits):
@@ -344,9 +343,9 @@ def run_gpu(args):
                 "frac": achieved / P["tensor_sustained"], "peak_burst": P["tensor_burst"],
                 "frac_burst": achieved / P["tensor_burst"], "peak_source": P["source"] + " (sustained: timed inside a long step)",
                 "traffic": fused_traffic_per_launch(dev, M, r, bits),
-                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one fused_kernel launch at "
-                                  "N=K=4096, 2048 tokens (profiles/fused_*_4096x4096_m2048.md), scaled by the input + "
-                                  "output bytes of an average launch of this workload"}
+                "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the gate_proj backward-input launch of "
+                                  "this workload (profiles/fused_backward_input_11008x4096_m4096_streamk.md), scaled by the "
+                                  "input + output bytes of the step's average launch"}
 
     # ---- end to end: host buffers, pinned, copies inside the timed region
     e2e = None
