@@ -929,7 +929,10 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
                                           // which the collecting cluster adds one after the other; cut the last two rows
         }
         const long long n_rest = (long long)n_tiles - (long long)dp * clusters;       // weight tiles behind the whole rows
-        if (dp >= 1 && n_rest * blocks >= clusters) {
+        // adding partial tiles in the epilogue costs about as much as 14 blocks (flag, 128 KB copy, one more pass over
+        // the accumulator): cutting the last row must save more than that over running it as one more row of whole tiles
+        const bool pays = late == 0 || (long long)n_last * blocks / clusters + 14 < blocks;
+        if (dp >= 1 && pays && n_rest * blocks >= clusters) {
             Q.sk = 1;
             Q.sk_dp = dp;
             Q.sk_late = late;
