@@ -20,8 +20,14 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
     for (int grp = blk * (kPrepThreads / 32) + warp; grp < n_groups; grp += P.blocks * (kPrepThreads / 32)) {
         uint32_t* out = P.items + (size_t)grp * kItemStride;
         int cls[per];
+        uint32_t stored[per];   // stored position of the row (asked for now: the answer is needed last)
         unsigned mask[per][4];
         int total[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int i = 0; i < per; ++i) {
+            const int row = grp * G + i * 32 + lane;
+            stored[i] = (row < P.N) ? (uint32_t)P.inv_perm[row] : 0u;
+        }
 #pragma unroll
         for (int i = 0; i < per; ++i) {
             const int row = grp * G + i * 32 + lane;
@@ -58,8 +64,8 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
                         for (int i2 = 0; i2 < per; ++i2) cnt += __popc(mask[i2][c] & (0x01010101u << res));
                         q += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
                     }
-                    const int off = i * 32 + lane, row = grp * G + off;
-                    const uint32_t p = (c < 3) ? (uint32_t)P.inv_perm[row] : 0u;
+                    const int off = i * 32 + lane;
+                    const uint32_t p = (c < 3) ? stored[i] : 0u;
                     out[class_base[c] + q] = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
                 }
             }
@@ -108,8 +114,14 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
         const int cta = grp % kCluster;
         const uint32_t n0 = (uint32_t)kChunks * (uint32_t)(grp / kCluster);   // number of the group's first chunk
         int cls[2];
+        uint32_t stored[2];   // stored position of the row (asked for now: the answer is needed last)
         unsigned mask[2][4];
         int total_c[4] = {0, 0, 0, 0};
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int row = grp * 64 + i * 32 + lane;
+            stored[i] = (row < P.N) ? (uint32_t)P.inv_perm[row] : 0u;
+        }
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int row = grp * 64 + i * 32 + lane;
@@ -134,7 +146,7 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
                     const int off = i * 32 + lane, row = grp * 64 + off;
                     uint4 rec = make_uint4(0u, 0u, 0u, (uint32_t)off | ((uint32_t)c << 8));
                     if (c < 3) {
-                        const uint32_t sp = (uint32_t)P.inv_perm[row];   // stored position
+                        const uint32_t sp = stored[i];   // stored position
                         const uint64_t row_bytes = ((uint64_t)P.L.K << c) >> 3;
                         rec.x = (uint32_t)((P.L.seg_off[c] + (uint64_t)(sp - (uint32_t)P.L.class_start[c]) * row_bytes) >> 4);
                         rec.y = sp * (uint32_t)P.L.nb;
