@@ -42,6 +42,17 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
         class_base[0] = 0;
 #pragma unroll
         for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total[c - 1];
+        // rows of every class by residue (row offset mod 8): the same for all lanes
+        int cnt[4][8];
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int res = 0; res < 8; ++res) {
+                int n = 0;
+#pragma unroll
+                for (int i2 = 0; i2 < per; ++i2) n += __popc(mask[i2][c] & (0x01010101u << res));
+                cnt[c][res] = n;
+            }
 #pragma unroll
         for (int i = 0; i < per; ++i) {
 #pragma unroll
@@ -58,12 +69,8 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
                     b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
                     int q = 0;   // rows of the class taken before this one
 #pragma unroll
-                    for (int res = 0; res < 8; ++res) {
-                        int cnt = 0;
-#pragma unroll
-                        for (int i2 = 0; i2 < per; ++i2) cnt += __popc(mask[i2][c] & (0x01010101u << res));
-                        q += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
-                    }
+                    for (int res = 0; res < 8; ++res)
+                        q += min(cnt[c][res], b) + ((res < (lane & 7) && cnt[c][res] > b) ? 1 : 0);
                     const int off = i * 32 + lane;
                     const uint32_t p = (c < 3) ? stored[i] : 0u;
                     out[class_base[c] + q] = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
