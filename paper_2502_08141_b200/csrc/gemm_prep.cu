@@ -143,6 +143,12 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
         class_base[0] = 0;
 #pragma unroll
         for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total_c[c - 1];
+        int cnt[4][8];   // rows of every class by residue (row offset mod 8): the same for all lanes
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int res = 0; res < 8; ++res)
+                cnt[c][res] = __popc(mask[0][c] & (0x01010101u << res)) + __popc(mask[1][c] & (0x01010101u << res));
         if (lane < kChunks)
             P.heads[chunk_slot(n0, (uint32_t)lane, cta)] = (uint32_t)grp | ((uint32_t)(kStageArrivals / kChunks) << 24);
 #pragma unroll
@@ -168,10 +174,8 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
                     b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
                     int pos = class_base[c];  // rows taken before this one
 #pragma unroll
-                    for (int res = 0; res < 8; ++res) {
-                        const int cnt = __popc(mask[0][c] & (0x01010101u << res)) + __popc(mask[1][c] & (0x01010101u << res));
-                        pos += min(cnt, b) + ((res < (lane & 7) && cnt > b) ? 1 : 0);
-                    }
+                    for (int res = 0; res < 8; ++res)
+                        pos += min(cnt[c][res], b) + ((res < (lane & 7) && cnt[c][res] > b) ? 1 : 0);
                     uint4* dst = rows + (size_t)chunk_slot(n0, (uint32_t)(pos / 16), cta) * 32 + pos % 16;
                     dst[0] = rec;
                     dst[16] = rec;
