@@ -409,7 +409,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // ================================================================== epilogue
         const int q = warp & 3;                 // TMEM lane quarter this warp may read
         const int et = (warp - kFirstEpilogueWarp) * 32 + lane;
-        uint16_t* out16 = reinterpret_cast<uint16_t*>(out_s);
+        uint16_t* stage16 = reinterpret_cast<uint16_t*>(out_s) + (warp - kFirstEpilogueWarp) * (kEpilogueTokens * 32);   // this warp's staging
         const int my_row = q * 32 + lane;
         // The four epilogue warps share named barriers, so they must leave together: one thread reads the abort
         // flag (any role may raise it at any time), the others take its answer after the barrier.  Two slots in
@@ -550,21 +550,22 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     for (int j = 0; j < 32; ++j) __stcg(part + (size_t)(chunk * 32 + j) * kTileR, __uint_as_float(v[j]));
                     continue;
                 }
-                // thread = operand row (channel), v[j] = token j: transposed through shared memory, eight tokens
-                // at a time (8 tokens x 128 channels = 2 KB: every thread then stores one 16-byte piece)
+                // thread = operand row (channel), v[j] = token j: transposed through the warp's own 512 bytes of shared
+                // memory, eight tokens at a time (8 tokens x 32 channels; every lane then stores one 16-byte piece of a
+                // token's 64 bytes) - no barrier between the warps
 #pragma unroll
                 for (int rnd = 0; rnd < 32 / kEpilogueTokens; ++rnd) {
 #pragma unroll
                     for (int j = 0; j < kEpilogueTokens; ++j) {
                         const uint32_t two = pack_bf16x2(scale * __uint_as_float(v[rnd * kEpilogueTokens + j]), 0.0f);
-                        out16[j * kTileR + my_row] = (uint16_t)two;
+                        stage16[j * 32 + lane] = (uint16_t)two;
                     }
-                    ptx::named_barrier_sync(1, 128);
+                    __syncwarp();
                     {
-                        const int row = et >> 4, ch = et & 15;
-                        const int m = m0 + chunk * 32 + rnd * kEpilogueTokens + row, n = r0 + ch * 8;
+                        const int tok = lane >> 2, piece = lane & 3;
+                        const int m = m0 + chunk * 32 + rnd * kEpilogueTokens + tok, n = r0 + q * 32 + piece * 8;
                         if (m < P.M && n < R) {
-                            const uint4 val = *reinterpret_cast<const uint4*>(out16 + row * kTileR + ch * 8);
+                            const uint4 val = *reinterpret_cast<const uint4*>(stage16 + tok * 32 + piece * 8);
                             uint16_t* dst = out + (size_t)m * ld + n;
                             if (vec_ok && n + 8 <= R) {
                                 *reinterpret_cast<uint4*>(dst) = val;
@@ -574,7 +575,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             }
                         }
                     }
-                    ptx::named_barrier_sync(1, 128);
+                    __syncwarp();
                 }
             }
             // the accumulator goes to the piece after next (preloaded if that one collects partial tiles)
