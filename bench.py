@@ -161,10 +161,10 @@ def make_host_inputs(cfg, rank: int):
 
 # DRAM traffic of one fused_kernel launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a
 # launch of this very workload: the backward-input pass of gate_proj (dX [4096, 4096] from dY [4096, 11008];
-# profiles/fused_backward_input_11008x4096_m4096_streamk.md): 168.2 MB read + 26.9 MB written.  The bytes the call
+# profiles/fused_backward_input_11008x4096_m4096_streamk.md): 167.9 MB read + 29.7 MB written.  The bytes the call
 # has to read and write once are 137 MB (the output is partly still in L2 when the kernel ends; the stream-K partial
 # tiles add 19 MB each way).  Scaled to the step's average launch in proportion to those input + output bytes.
-NCU_CASE = dict(N=4096, K=11008, M=4096, r=64, bits=1.5, dram_bytes=168.2e6 + 26.9e6)
+NCU_CASE = dict(N=4096, K=11008, M=4096, r=64, bits=1.5, dram_bytes=167.9e6 + 29.7e6)
 
 
 def fused_io_bytes(N, K, M, r, bits):
