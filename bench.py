@@ -226,7 +226,11 @@ def run_gpu(args):
     # ---- device-resident problem
     dev = []
     for m in mats:
+        # the deal of the rows to the dequant warps depends on the precisions only: built once per weight, like the
+        # storage plan, unless --deal-per-call asks for the prologue launch in every call
         layout = lw.Layout(m["precs"], m["K"])
+        if not args.deal_per_call:
+            layout.build_deal()
         d = dict(m=m, layout=layout,
                  W=torch.from_numpy(m["W"]).cuda(), thr=torch.from_numpy(m["thr"]).cuda(),
                  maps=torch.from_numpy(m["maps"]).cuda(),
@@ -236,7 +240,7 @@ def run_gpu(args):
                  What=torch.empty((m["N"], m["K"]), dtype=torch.bfloat16, device="cuda"),
                  Y=torch.empty((M, m["N"]), dtype=torch.bfloat16, device="cuda"),
                  dX=torch.empty((M, m["K"]), dtype=torch.bfloat16, device="cuda"),
-                 ws=torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda"))
+                 ws=lw.lowra_workspace_init(torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")))
         dev.append(d)
     act_dev = {k: bfv(torch.from_numpy(v.view(np.int16)).cuda()) for k, v in acts.items()}
     stream = torch.cuda.current_stream()
@@ -338,7 +342,7 @@ def run_gpu(args):
     # dominant kernel: the fused tensor-core kernel (forward + backward launches), timed as whole calls
     fused_ms = phase_ms["forward"] + phase_ms["backward"]
     achieved = flops_step / (fused_ms * 1e-3) / 1e12
-    roofline = {"bound": "tensor", "kernel": "fused_kernel (forward + backward-input calls, prologue included)",
+    roofline = {"bound": "tensor", "kernel": "fused_kernel (forward + backward-input calls" + (", prologue launch included)" if args.deal_per_call else ")"),
                 "achieved": achieved, "peak": P["tensor_sustained"], "unit": "TFLOP/s",
                 "frac": achieved / P["tensor_sustained"], "peak_burst": P["tensor_burst"],
                 "frac_burst": achieved / P["tensor_burst"], "peak_source": P["source"] + " (sustained: timed inside a long step)",
@@ -526,9 +530,11 @@ def run_gpu(args):
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": f"config {WORKLOAD}: {cfg.name}, 7 matrices, {M} tokens, rank {r}, "
                                    f"mix {cfg.mix} (avg {bits:.2f} bits), stand-in codebooks",
-                       "elements": elems, "l2": "inputs larger than L2 (about 2.7 GB touched per step)"},
+                       "elements": elems, "l2": "inputs larger than L2 (about 2.7 GB touched per step)",
+                       "row_deal": "in every call (prologue launch)" if args.deal_per_call else
+                                   "once per weight (lowra_deal_build), outside the step like the storage plan"},
             "phases": phases, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "extras": extras,
-            "gpu_launches": args.steps * len(dev) * 6, "clocks": clocks,
+            "gpu_launches": args.steps * len(dev) * (6 if args.deal_per_call else 4), "clocks": clocks,
         }
         print(json.dumps(out))
     if world > 1:
@@ -618,6 +624,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--deal-per-call", action="store_true",
+                    help="fused calls work out the row deal in a prologue launch of their own (no lowra_deal_build)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

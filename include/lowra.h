@@ -66,6 +66,7 @@ typedef struct {
     const uint8_t* precs_dev;    /* [N] bits per row, original order */
     const int32_t* perm_dev;     /* [N] stored position -> original row */
     const int32_t* inv_perm_dev; /* [N] original row -> stored position */
+    const void* deal_dev;        /* NULL, or what lowra_deal_build wrote for this weight (see there) */
 } lowra_layout;
 
 /*
@@ -163,6 +164,29 @@ lowra_status lowra_channel_errors(int32_t N, int32_t K, const float* W_dev, cons
 size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r);
 
 /*
+ * Once per weight instead of once per call (no counterpart in the paper; like the storage planner it depends
+ * on the channels' precisions only).  The fused calls below hand the rows of every group of channels to their
+ * dequantising warps sorted by precision.  With layout->deal_dev == NULL every call works that out again in
+ * a small prologue launch, which also clears the status word and the flags in the workspace.  With
+ * layout->deal_dev pointing at a buffer filled by lowra_deal_build the fused kernel is the only launch
+ * of a call (5-7 us less per call on a B200); the workspace then has to be initialised once with
+ * lowra_workspace_init before its first use, is written by these calls only, and its status word is no
+ * longer cleared per call: lowra_device_status reports the first failure since the initialisation.
+ *   lowra_deal_bytes   size of the buffer for this layout (0 if the layout is invalid); about 40 bytes per
+ *                      channel (0.44 MB for 11008 channels)
+ *   lowra_deal_build   fills deal_dev (256-byte aligned, >= lowra_deal_bytes(layout) bytes) for both the
+ *                      forward and the backward-input call; reads layout->precs_dev / inv_perm_dev and
+ *                      ignores layout->deal_dev.  The buffer is read-only afterwards and may serve any
+ *                      number of calls, streams and workspaces.
+ *   lowra_workspace_init   zero-fills the workspace (status word, call numbering, flags).
+ * Errors: as lowra_lora_forward; LOWRA_ERR_WORKSPACE for a buffer that is too small or not 256-byte aligned
+ * (lowra_deal_build: LOWRA_ERR_ALIGN for the alignment).
+ */
+size_t lowra_deal_bytes(const lowra_layout* layout);
+lowra_status lowra_deal_build(const lowra_layout* layout, void* deal_dev, size_t deal_bytes, void* stream);
+lowra_status lowra_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/*
  * Forward of the quantized-LoRA linear layer (Section 3: the fine-tuning module recovers the base
  * weights with the dequantize kernel; frozen base plus trainable low-rank factors):
  *     Y = X . deq(Wq)^T + s * (X . A) . B
@@ -171,7 +195,9 @@ size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r);
  *   X_dev bf16 [M, K];  A_dev bf16 [K, r];  B_dev bf16 [r, N];  Y_dev bf16 [M, N], original
  *   channel order; all row-major.  r in {16, 32, ..., 128}.  X . A is rounded to bf16 once.
  *   workspace_dev: >= lowra_workspace_bytes(layout, M, r) bytes, 256-byte aligned, contents
- *   overwritten.  Calls that share a workspace must not overlap on the device.
+ *   overwritten.  Calls that share a workspace must not overlap on the device.  With
+ *   layout->deal_dev set: initialised by lowra_workspace_init and since then written by these calls only
+ *   (any mix of forward / backward-input, weights and token counts).
  *   Limits (LOWRA_ERR_SHAPE otherwise): N % 8 == 0, N <= 524288, N * K / 64 < 2^32, M >= 1.
  */
 lowra_status lowra_lora_forward(const lowra_layout* layout, const uint8_t* packed_dev,

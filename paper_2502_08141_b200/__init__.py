@@ -29,7 +29,7 @@ EXPORTS = (
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
     "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
-    "lowra_dense_nt_pair", "lowra_channel_errors",
+    "lowra_dense_nt_pair", "lowra_channel_errors", "lowra_deal_bytes", "lowra_deal_build", "lowra_workspace_init",
 )
 
 
@@ -46,6 +46,7 @@ class _CLayout(ctypes.Structure):
         ("seg_off", ctypes.c_uint64 * 3),
         ("packed_bytes", ctypes.c_uint64),
         ("precs_dev", ctypes.c_void_p), ("perm_dev", ctypes.c_void_p), ("inv_perm_dev", ctypes.c_void_p),
+        ("deal_dev", ctypes.c_void_p),
     ]
 
 
@@ -73,6 +74,12 @@ def lib() -> ctypes.CDLL:
         L.lowra_decode.restype = ctypes.c_int
         L.lowra_workspace_bytes.argtypes = [lp, i32, i32]
         L.lowra_workspace_bytes.restype = ctypes.c_size_t
+        L.lowra_deal_bytes.argtypes = [lp]
+        L.lowra_deal_bytes.restype = ctypes.c_size_t
+        L.lowra_deal_build.argtypes = [lp, vp, ctypes.c_size_t, vp]
+        L.lowra_deal_build.restype = ctypes.c_int
+        L.lowra_workspace_init.argtypes = [vp, ctypes.c_size_t, vp]
+        L.lowra_workspace_init.restype = ctypes.c_int
         gemm_args = [lp, vp, vp, vp, vp, i32, vp, vp, i32, ctypes.c_float, vp, vp, ctypes.c_size_t, vp]
         L.lowra_lora_forward.argtypes = gemm_args
         L.lowra_lora_forward.restype = ctypes.c_int
@@ -172,7 +179,26 @@ class Layout:
         c.precs_dev = self.precs.data_ptr()
         c.perm_dev = self.perm.data_ptr()
         c.inv_perm_dev = self.inv_perm.data_ptr()
+        c.deal_dev = None
         self.c = c
+        self.deal = None
+
+    def build_deal(self, stream=None) -> "Layout":
+        """Deal the rows to the dequantising warps once for this weight (lowra_deal_build): the fused calls on this
+        layout then launch no prologue.  Their workspace must have been through lowra_workspace_init."""
+        n = int(lib().lowra_deal_bytes(self.ref))
+        if n == 0:
+            raise LowraError(LOWRA_ERR_SHAPE, "lowra_deal_bytes")
+        deal = torch.empty(n, dtype=torch.uint8, device=self.device)
+        _check(lib().lowra_deal_build(self.ref, _ptr(deal), n, _stream(stream)), "lowra_deal_build")
+        self.deal = deal
+        self.c.deal_dev = deal.data_ptr()
+        return self
+
+    def drop_deal(self) -> "Layout":
+        self.deal = None
+        self.c.deal_dev = None
+        return self
 
     @property
     def ref(self):
@@ -244,7 +270,17 @@ def _workspace(layout: Layout, M: int, r: int, device) -> torch.Tensor:
     n = lowra_workspace_bytes(layout, M, r)
     if n == 0:
         raise LowraError(LOWRA_ERR_SHAPE, "lowra_workspace_bytes")
-    return torch.empty(n, dtype=torch.uint8, device=device)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    if layout.deal is not None:   # no prologue launch will clear it
+        lowra_workspace_init(ws)
+    return ws
+
+
+def lowra_workspace_init(workspace: torch.Tensor, stream=None) -> torch.Tensor:
+    """Zero-fill a workspace: needed once before calls on a layout that carries a deal (Layout.build_deal)."""
+    _dev(workspace, torch.uint8, "workspace")
+    _check(lib().lowra_workspace_init(_ptr(workspace), workspace.numel(), _stream(stream)), "lowra_workspace_init")
+    return workspace
 
 
 def lowra_lora_forward(layout: Layout, packed, absmax, maps, X, A, B, s: float,

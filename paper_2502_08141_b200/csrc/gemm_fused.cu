@@ -272,6 +272,12 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     // that kernel wrote (row deal, cleared flags and status word).
     if (MODE != kModeDense) pdl_enter();
     const uint32_t tmem_base = bars->tmem_base;
+    // This call's number on the workspace: the value that means "up" in the flags (T ready, partial tile ready).
+    uint32_t want = 1u;
+    if (MODE != kModeDense) {
+        want = *reinterpret_cast<const volatile uint32_t*>(P.epoch) + 1u;
+        if (want == 0u) want = 1u;   // only on a workspace that was never initialised (its flags are cleared per call)
+    }
 
     bool failed = false;
 
@@ -318,7 +324,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         if (lb == 0 || kb == t.kb0) {
                             // T of this token tile is written by another CTA: wait for its flag, then make
                             // those generic-proxy writes visible to the TMA (async proxy) reads below
-                            if (!ptx::flag_wait(P.flags + t.mt, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                            if (!ptx::flag_wait(P.flags + t.mt, want, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
                             ptx::fence_proxy_async_all();
                         }
                         ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
@@ -436,15 +442,15 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     uint32_t ok = 1u;
                     if (lane == 0) {
                         if (wait) {
-                            if (!ptx::flag_wait(P.sk_flags + c * CL + (int)crank, abort_flag, kWaitLimitNs)) { bars->abort = 1u; ok = 2u; }
+                            if (!ptx::flag_wait(P.sk_flags + c * CL + (int)crank, want, abort_flag, kWaitLimitNs)) { bars->abort = 1u; ok = 2u; }
                         } else {
-                            ok = ptx::flag_test(P.sk_flags + c * CL + (int)crank) ? 1u : 0u;
+                            ok = ptx::flag_test(P.sk_flags + c * CL + (int)crank, want) ? 1u : 0u;
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
                     if (ok == 0u) return false;
                     if (ok == 2u) return true;                        // timed out: the abort flag ends the loop below
-                    (void)ptx::flag_test(P.sk_flags + c * CL + (int)crank);   // every lane's own acquire before its loads
+                    (void)ptx::flag_test(P.sk_flags + c * CL + (int)crank, want);   // every lane's own acquire before its loads
                 }
                 const int m0 = t.mt * kTileT;
 #pragma unroll 1
@@ -501,7 +507,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const float* ring = reinterpret_cast<const float*>(base) + my_row;
                 bool leave = false;
                 for (int c = cid + 1; c < c_end; ++c) {
-                    if (lane == 0 && !ptx::flag_wait(P.sk_flags + c * CL + (int)crank, abort_flag, kWaitLimitNs)) bars->abort = 1u;
+                    if (lane == 0 && !ptx::flag_wait(P.sk_flags + c * CL + (int)crank, want, abort_flag, kWaitLimitNs)) bars->abort = 1u;
                     leave = agree_abort();             // also: everybody is done with the previous partial tile in the ring
                     if (leave) break;
                     if (et == 0) {
@@ -588,9 +594,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 if (et == 0) {
                     if (t.is_t) {
                         ptx::fence_proxy_async_all();
-                        ptx::flag_release(P.flags + t.mt, 1u);
+                        ptx::flag_release(P.flags + t.mt, want);
                     } else {
-                        ptx::flag_release(P.sk_flags + cid * CL + (int)crank, 1u);   // one flag per CTA: its half of the slot
+                        ptx::flag_release(P.sk_flags + cid * CL + (int)crank, want);   // one flag per CTA: its half of the slot
                     }
                 }
             }
@@ -863,6 +869,19 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
+    }
+    if (MODE != kModeDense && threadIdx.x == 0) {
+        // the last CTA to leave records the call's number; every CTA has read the old one long before.  Just before
+        // the numbering wraps around, it clears the flags and starts again from zero.
+        __threadfence();
+        if (atomicAdd(P.exits, 1u) == gridDim.x - 1u) {
+            if (want == 0xFFFFFFFFu) {
+                for (int i = 0; i < P.n_flags; ++i) P.flags[i] = 0u;
+                want = 0u;
+            }
+            *P.epoch = want;
+            *P.exits = 0u;
+        }
     }
 }
 

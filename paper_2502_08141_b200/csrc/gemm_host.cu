@@ -11,7 +11,9 @@ namespace lowra {
 
 namespace {
 
-constexpr size_t kStatusBytes = 256;
+constexpr size_t kStatusBytes = 256;   // status word at byte 0, then the two words that number the calls:
+constexpr size_t kEpochOffset = 64;    //   number of the last call that ran on this workspace
+constexpr size_t kExitsOffset = 128;   //   CTAs of the running call that have left
 
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
@@ -22,22 +24,46 @@ struct Workspace {
 
 bool rank_ok(int r) { return r >= 16 && r <= 128 && r % 16 == 0; }
 
+// Sizes of the row deal (see gemm_prep.cu).  Forward: 128 row words per group of 128 channels; backward: 4 work-list
+// entries (a head and 32 row records of 16 bytes each) per group of 64 channels, plus the end markers.
+struct DealSizes {
+    size_t fwd_bytes, rows_bytes, heads_bytes;
+};
+DealSizes deal_sizes(int N) {
+    const size_t groups_per_cta = ((size_t)(N + 63) / 64 + kCluster - 1) / kCluster;
+    const size_t entries = kCluster * (4 * groups_per_cta + kListSlack + kProducerWarps);
+    DealSizes d;
+    d.fwd_bytes = (size_t)((N + 127) / 128) * kItemStride * 4;
+    d.rows_bytes = entries * 32 * 16;
+    d.heads_bytes = entries * 4;
+    return d;
+}
+// A deal kept by the caller (lowra_deal_build): forward row words | backward row records | backward heads
+struct DealBuffer {
+    size_t off_fwd, off_rows, off_heads, total;
+};
+DealBuffer plan_deal(int N) {
+    const DealSizes z = deal_sizes(N);
+    DealBuffer d;
+    d.off_fwd = 0;
+    d.off_rows = align256(z.fwd_bytes);
+    d.off_heads = d.off_rows + align256(z.rows_bytes);
+    d.total = d.off_heads + align256(z.heads_bytes);
+    return d;
+}
+
 Workspace plan_workspace(int N, int K, int M, int r, bool stream_k) {
     (void)K;
     Workspace w;
     w.rp = (r + 63) / 64 * 64;
-    // forward: 128 row words per group of 128 channels; backward: 4 work-list entries (a head and 32 row records
-    // of 16 bytes each) per group of 64 channels, plus the end markers
-    const size_t groups_per_cta = ((size_t)(N + 63) / 64 + kCluster - 1) / kCluster;
-    const size_t entries = kCluster * (4 * groups_per_cta + kListSlack + kProducerWarps);
-    const size_t fwd_words = (size_t)((N + 127) / 128) * kItemStride;
+    const DealSizes z = deal_sizes(N);   // room for the deal of one direction, rebuilt by every call that brings none
     w.off_T = kStatusBytes;
     w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);
     // "T ready" flags (a cluster's last token tiles may lie past M), then one "partial tile ready" flag per CTA
     w.n_flags = (M + kTileT - 1) / kTileT + kCluster + kMaxClusters * kCluster;
     w.off_items = w.off_flags + align256((size_t)w.n_flags * 4);
-    w.off_meta = w.off_items + align256((entries * 32 * 4 > fwd_words ? entries * 32 * 4 : fwd_words) * 4);
-    w.off_part = w.off_meta + align256(entries * 4);
+    w.off_meta = w.off_items + align256(z.rows_bytes > z.fwd_bytes ? z.rows_bytes : z.fwd_bytes);
+    w.off_part = w.off_meta + align256(z.heads_bytes);
     w.total = w.off_part + (stream_k ? align256((size_t)kMaxClusters * kSkSlotFloats * 4) : 0);   // stream-K partial tiles
     return w;
 }
@@ -80,7 +106,7 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     if (M < 1 || !rank_ok(r) || N % 8 != 0 || N > 64 * kMaxGroups64 || (uint64_t)N * (uint64_t)(K / 64) >= (1ull << 32))
         return LOWRA_ERR_SHAPE;
     if (!aligned16(packed) || !aligned16(absmax) || !aligned16(maps) || !aligned16(act) || !aligned16(A) ||
-        !aligned16(B) || !aligned16(out))
+        !aligned16(B) || !aligned16(out) || (reinterpret_cast<uintptr_t>(layout->deal_dev) & 255u) != 0)
         return LOWRA_ERR_ALIGN;
     const Workspace w = plan_workspace(N, K, M, r, stream_k);
     if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LOWRA_ERR_WORKSPACE;
@@ -96,22 +122,32 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     uint32_t* heads = reinterpret_cast<uint32_t*>(ws + w.off_meta);
     const int tiles_t = (M + kTileT - 1) / kTileT;
 
-    // ---- prologue: clear status and flags, deal the rows
-    PrepParams P;
-    memset(&P, 0, sizeof(P));
-    P.L = make_row_layout(layout);
-    P.precs = layout->precs_dev;
-    P.inv_perm = layout->inv_perm_dev;
-    P.items = items;
-    P.heads = heads;
-    P.N = N;
-    P.group = backward ? 64 : 128;
-    P.status = status;
-    P.flags = flags;
-    P.n_flags = w.n_flags;
-    P.blocks = ((N + P.group - 1) / P.group + 3) / 4;
-    st = launch_prep(P, stream);
-    if (st != LOWRA_OK) return st;
+    if (layout->deal_dev != nullptr) {
+        // the rows were dealt once for this weight (lowra_deal_build) and the workspace numbers its calls
+        // (lowra_workspace_init): nothing to prepare, the fused kernel is the only launch
+        const DealBuffer d = plan_deal(N);
+        unsigned char* deal = static_cast<unsigned char*>(const_cast<void*>(layout->deal_dev));
+        items = reinterpret_cast<uint32_t*>(deal + (backward ? d.off_rows : d.off_fwd));
+        heads = reinterpret_cast<uint32_t*>(deal + d.off_heads);
+    } else {
+        // ---- prologue: clear status and flags, deal the rows
+        PrepParams P;
+        memset(&P, 0, sizeof(P));
+        P.L = make_row_layout(layout);
+        P.precs = layout->precs_dev;
+        P.inv_perm = layout->inv_perm_dev;
+        P.items = items;
+        P.heads = heads;
+        P.N = N;
+        P.group = backward ? 64 : 128;
+        P.status = status;
+        P.exits = reinterpret_cast<uint32_t*>(ws + kExitsOffset);
+        P.flags = flags;
+        P.n_flags = w.n_flags;
+        P.blocks = ((N + P.group - 1) / P.group + 3) / 4;
+        st = launch_prep(P, stream);
+        if (st != LOWRA_OK) return st;
+    }
 
     // ---- fused kernel (its first tiles compute T = s X A, resp. U = s dY B^T)
     GemmParams G;
@@ -126,6 +162,9 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.T = T;
     G.flags = flags;
     G.status = status;
+    G.epoch = reinterpret_cast<uint32_t*>(ws + kEpochOffset);
+    G.exits = reinterpret_cast<uint32_t*>(ws + kExitsOffset);
+    G.n_flags = w.n_flags;
     G.s = s;
     G.rp = w.rp;
     G.r = r;
@@ -178,6 +217,51 @@ extern "C" size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, i
     using namespace lowra;
     if (!layout || layout->N < 1 || layout->K < 1 || M < 1 || !rank_ok(r)) return 0;
     return plan_workspace(layout->N, layout->K, M, r, true).total;
+}
+
+extern "C" size_t lowra_deal_bytes(const lowra_layout* layout) {
+    using namespace lowra;
+    if (!layout || layout->N < 1) return 0;
+    return plan_deal(layout->N).total;
+}
+
+extern "C" lowra_status lowra_deal_build(const lowra_layout* layout, void* deal_dev, size_t deal_bytes, void* stream) {
+    using namespace lowra;
+    lowra_status st = check_layout(layout);
+    if (st != LOWRA_OK) return st;
+    if (!deal_dev) return LOWRA_ERR_NULL;
+    const int N = layout->N;
+    if (N % 8 != 0 || N > 64 * kMaxGroups64) return LOWRA_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(deal_dev) & 255u) != 0) return LOWRA_ERR_ALIGN;
+    const DealBuffer d = plan_deal(N);
+    if (deal_bytes < d.total) return LOWRA_ERR_WORKSPACE;
+    st = check_device();
+    if (st != LOWRA_OK) return st;
+    unsigned char* deal = static_cast<unsigned char*>(deal_dev);
+    for (int backward = 0; backward < 2; ++backward) {
+        PrepParams P;
+        memset(&P, 0, sizeof(P));   // no status word, no flags: this launch only deals
+        P.L = make_row_layout(layout);
+        P.precs = layout->precs_dev;
+        P.inv_perm = layout->inv_perm_dev;
+        P.items = reinterpret_cast<uint32_t*>(deal + (backward ? d.off_rows : d.off_fwd));
+        P.heads = reinterpret_cast<uint32_t*>(deal + d.off_heads);
+        P.N = N;
+        P.group = backward ? 64 : 128;
+        P.blocks = ((N + P.group - 1) / P.group + 3) / 4;
+        st = launch_prep(P, (cudaStream_t)stream);
+        if (st != LOWRA_OK) return st;
+    }
+    return LOWRA_OK;
+}
+
+extern "C" lowra_status lowra_workspace_init(void* workspace_dev, size_t workspace_bytes, void* stream) {
+    if (!workspace_dev) return LOWRA_ERR_NULL;
+    if (workspace_bytes < lowra::kStatusBytes || (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) != 0)
+        return LOWRA_ERR_WORKSPACE;
+    // status word, call numbering and every flag start from zero; the rest of the scratch needs no initial value
+    return cudaMemsetAsync(workspace_dev, 0, workspace_bytes, (cudaStream_t)stream) == cudaSuccess ? LOWRA_OK
+                                                                                                   : LOWRA_ERR_CUDA;
 }
 
 extern "C" lowra_status lowra_lora_forward(const lowra_layout* layout, const uint8_t* packed_dev,
@@ -241,8 +325,9 @@ extern "C" lowra_status lowra_lora_forward_static(const lowra_layout* layout, co
     void* scratch = nullptr;
     st = static_scratch(&scratch);
     if (st != LOWRA_OK) return st;
-    // The prologue kernel rewrites every word the fused kernel reads (status word, down-projection,
-    // padded factor, row deal), so nothing left over from an earlier call is ever consumed.
+    // The scratch starts zero-filled (a static array) and only these calls write it, so the numbering of the
+    // calls holds whether or not the layout brings a deal; without one the prologue kernel rewrites the status
+    // word, the flags and the deal on every call.
     st = run_lora(false, layout, packed_dev, absmax_dev, maps_dev, X_dev, M, A_dev, B_dev, r, s, Y_dev, scratch,
                   (size_t)LOWRA_STATIC_SCRATCH_BYTES, stream, false);
     if (st != LOWRA_OK) return st;

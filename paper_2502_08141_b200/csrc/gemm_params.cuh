@@ -28,7 +28,8 @@ struct PrepParams {
     uint32_t* items;      // forward: row words; backward: 16-byte row records of the work-list entries
     uint32_t* heads;      // backward: [7 * ceil(N / 64) + kListSlack] work-list heads
     int N, group;
-    uint32_t* status;     // device status word, cleared
+    uint32_t* status;     // device status word, cleared (null: left alone)
+    uint32_t* exits;      // the fused kernel's count of CTAs that have left, cleared (null: left alone)
     uint32_t* flags;      // [n_flags] "T of this token tile is ready" flags, cleared
     int n_flags;
     int blocks;
@@ -71,8 +72,14 @@ struct GemmParams {
     const uint32_t* heads;    // from the prologue (backward): work-list heads
     uint16_t* out;          // [M, ld_out] bf16
     uint16_t* T;            // [M, rp] bf16: s * X . A (forward) or s * dY . B^T (backward), written by the T tiles
-    uint32_t* flags;        // [tiles_t] raised when T of a token tile is complete
+    uint32_t* flags;        // [tiles_t] set to the call's number when T of a token tile is complete
     uint32_t* status;
+    // Calls on one workspace are numbered: `epoch` holds the number of the last call that ran on it, a call's own
+    // number is that + 1, and a flag is up when it holds the call's number - so flags left over from earlier calls
+    // never need clearing.  The last CTA to leave (counted in `exits`) writes the call's number back.
+    uint32_t* epoch;
+    uint32_t* exits;
+    int n_flags;            // all flags of the workspace (T ready + partial tile ready), for the wrap of the numbering
     float s;
     int rp;                 // LoRA rank rounded up to 64
     int r;                  // LoRA rank

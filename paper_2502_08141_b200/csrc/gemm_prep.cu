@@ -191,6 +191,7 @@ __global__ void __launch_bounds__(kPrepThreads) prep_kernel(const PrepParams P) 
     pdl_enter();   // the fused kernel may set itself up meanwhile; it waits for this grid before it reads the deal
     if (blockIdx.x == 0) {
         if (threadIdx.x == 0 && P.status != nullptr) *P.status = 0u;   // null: keep what earlier launches recorded
+        if (threadIdx.x == 0 && P.exits != nullptr) *P.exits = 0u;
         for (int i = threadIdx.x; i < P.n_flags; i += kPrepThreads) P.flags[i] = 0u;
     }
     if (P.group == 64) {

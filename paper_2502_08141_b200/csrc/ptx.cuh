@@ -113,22 +113,22 @@ __device__ __forceinline__ void fence_proxy_async_smem() {
 // CTA wrote to global memory with ordinary stores)
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
-// Global-memory flag between CTAs: release store / bounded acquire poll.
+// Global-memory flag between CTAs: release store / bounded acquire poll.  A flag is up when it holds `want`.
 __device__ __forceinline__ void flag_release(uint32_t* flag, uint32_t value) {
     asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(flag), "r"(value) : "memory");
 }
-__device__ __forceinline__ bool flag_test(const uint32_t* flag) {   // one look, no waiting
+__device__ __forceinline__ bool flag_test(const uint32_t* flag, uint32_t want) {   // one look, no waiting
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-    return v != 0u;
+    return v == want;
 }
-__device__ __forceinline__ bool flag_wait(const uint32_t* flag, volatile uint32_t* abort, uint64_t limit_ns) {
+__device__ __forceinline__ bool flag_wait(const uint32_t* flag, uint32_t want, volatile uint32_t* abort, uint64_t limit_ns) {
     const uint64_t t0 = globaltimer_ns();
 #pragma unroll 1
     for (;;) {
         uint32_t v;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-        if (v != 0u) return true;
+        if (v == want) return true;
         __nanosleep(64);
         if (abort != nullptr && *abort != 0u) return false;
         if (globaltimer_ns() - t0 > limit_ns) return false;

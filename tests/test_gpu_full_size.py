@@ -1,4 +1,5 @@
-"""Parity at benchmark sizes, in the launch configuration that bench.py times (4096 tokens, rank 64).
+"""Parity at benchmark sizes, in the launch configuration that bench.py times (4096 tokens, rank 64, the rows
+dealt once per weight with lowra_deal_build, the workspace initialised once and then reused by both products).
 
 Encode and decode are compared bit for bit on the whole matrix.  The two products are computed in full
 on the GPU and compared with the fp64 oracle on 128 sampled token rows (always rows 0, 127, 128 and
@@ -42,7 +43,7 @@ def test_full_size_matrix(name, N, K, mix, mid):
 
     M, r, s = 4096, 64, 2.0
     case = make_case(N, K, mix, matrix_id=mid)
-    layout = lw.Layout(case.precs, K)
+    layout = lw.Layout(case.precs, K).build_deal()
 
     packed, absmax = lw.lowra_encode(layout, _dev(case.W), _dev(case.thr))
     what = lw.lowra_decode(layout, packed, absmax, _dev(case.maps))
@@ -57,10 +58,15 @@ def test_full_size_matrix(name, N, K, mix, mid):
     A, B = si.lora_factors(K, N, r, matrix_id=mid)
     rng = np.random.default_rng(mid)
     rows = np.unique(np.concatenate([[0, 127, 128, M - 1], rng.choice(M, 124, replace=False)]))
-    ws = torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")
+    ws = lw.lowra_workspace_init(torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda"))
 
     Y = lw.lowra_lora_forward(layout, packed, absmax, _dev(case.maps), _bf(X), _bf(A), _bf(B), s, workspace=ws)
     assert lw.lowra_device_status(ws) == lw.LOWRA_OK
+    # the same call with the deal worked out in its own prologue launch: bit-identical
+    plain = lw.Layout(case.precs, K)
+    Y2 = lw.lowra_lora_forward(plain, packed, absmax, _dev(case.maps), _bf(X), _bf(A), _bf(B), s, workspace=ws)
+    assert torch.equal(Y.view(torch.int16), Y2.view(torch.int16))
+    del Y2
     got = si.bf16_bits_to_f32(_bits(Y[torch.from_numpy(rows).cuda()]))
     ref = oracle.lora_forward(case.W_hat, X[rows], A, B, s)
     emax, efro = gemm_errors(got, ref)

@@ -89,6 +89,22 @@ def test_validation_runs_before_any_device_work(lib):
     assert L.lowra_lora_forward(*args) == lib.LOWRA_ERR_WORKSPACE
     assert L.lowra_lora_backward_input(*args) == lib.LOWRA_ERR_WORKSPACE
     assert L.lowra_device_status(None, None) == lib.LOWRA_ERR_NULL
+    # a deal kept by the caller and the workspace initialisation that goes with it
+    assert L.lowra_deal_bytes(None) == 0
+    need_deal = L.lowra_deal_bytes(ctypes.byref(lay))
+    assert need_deal >= 8 * 4 and need_deal % 256 == 0
+    assert L.lowra_deal_build(ctypes.byref(lay), None, need_deal, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_deal_build(ctypes.byref(lay), 4096 + 16, need_deal, None) == lib.LOWRA_ERR_ALIGN
+    assert L.lowra_deal_build(ctypes.byref(lay), 4096, need_deal - 1, None) == lib.LOWRA_ERR_WORKSPACE
+    assert L.lowra_deal_build(None, 4096, need_deal, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_workspace_init(None, 1 << 20, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_workspace_init(4096, 16, None) == lib.LOWRA_ERR_WORKSPACE
+    assert L.lowra_workspace_init(4096 + 16, 1 << 20, None) == lib.LOWRA_ERR_WORKSPACE
+    lay.deal_dev = 4096 + 16                                             # a deal that is not 256-byte aligned
+    args[12] = 1 << 30
+    assert L.lowra_lora_forward(*args) == lib.LOWRA_ERR_ALIGN
+    lay.deal_dev = None
+    args[12] = 16
     sargs = [ctypes.byref(lay), 4096, 4096, 4096, 4096, 1 << 20, 4096, 4096, 128, ctypes.c_float(1.0), 4096, None, None]
     assert L.lowra_lora_forward_static(*sargs) == lib.LOWRA_ERR_LIMIT   # 1M tokens x rank 128 needs > 8 MiB of scratch
     sargs[8] = 24
