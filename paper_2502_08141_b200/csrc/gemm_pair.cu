@@ -7,7 +7,7 @@
 // tensor core reading its half of P locally and both halves of Q.  Per FLOP that is two thirds of the one-CTA
 // tile's shared-memory traffic and L2 traffic, which is what bounds the one-CTA pipeline of this library.
 //   - TMA: both CTAs load their halves; the bytes of both are counted on the LEADER's "full" barrier
-//     (cp.async.bulk.tensor with .cta_group::2 and the leader's barrier address; no multicast).
+//     (tiled TMA loads with .cta_group::2 and the leader's barrier address; every CTA loads for itself).
 //   - slot release and "accumulator complete": tcgen05.commit.cta_group::2 with a CTA mask, which arrives on the
 //     barrier at the same offset in both CTAs.
 //   - "accumulator drained": the epilogue warps of both CTAs arrive on the leader's barrier.

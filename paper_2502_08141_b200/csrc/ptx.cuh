@@ -161,7 +161,7 @@ __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
 
-// 2-D tiled load, no multicast: box lands at `dst` (shared), bytes are counted on `bar`.
+// 2-D tiled load into this CTA's shared memory: box lands at `dst`, bytes are counted on `bar`.
 // x = innermost coordinate (elements), y = row.  x * element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
     asm volatile(
