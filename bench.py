@@ -457,6 +457,21 @@ def run_gpu(args):
                                       "frac_hbm": 4.0 * elems / (ms_learn * 1e-3) / 1e9 / P["hbm"],
                                       "element_passes_per_s": elems * T_learn / (ms_learn * 1e-3),
                                       "note": "not part of the step; algorithmic bytes = one read of W (4 B per element)"}}
+        # the same for all three precisions of every row in one pass (what the precision assigner starts from)
+        tabs3 = [(torch.empty((3, d["m"]["N"], 16), dtype=torch.float32, device="cuda"),
+                  torch.empty((3, d["m"]["N"], 16), dtype=torch.float32, device="cuda")) for d in dev]
+        for d, (m3, h3) in zip(dev, tabs3):
+            lw.lowra_learn_codebooks_all(d["W"], y0, t0, T_learn, maps3=m3, thresholds3=h3)
+        a.record(stream)
+        for d, (m3, h3) in zip(dev, tabs3):
+            lw.lowra_learn_codebooks_all(d["W"], y0, t0, T_learn, maps3=m3, thresholds3=h3)
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms_learn3 = a.elapsed_time(b)
+        extras["learn_codebooks_all_precisions"] = {
+            "ms": ms_learn3, "iterations": T_learn, "element_passes_per_s": 3 * elems * T_learn / (ms_learn3 * 1e-3),
+            "note": "not part of the step; every row at 1, 2 and 4 bits from one read of W"}
+        del tabs3
 
         # the gradients of the low-rank factors (the other half of a training step's backward pass)
         ws_ad = torch.empty(lw.lowra_adapter_workspace_bytes(M, r), dtype=torch.uint8, device="cuda")

@@ -304,6 +304,20 @@ lowra_status lowra_learn_codebooks(const lowra_layout* layout, const float* W_de
                                    float* thresholds_dev, void* stream);
 
 /*
+ * The same learner for every channel at all three precisions (Section 5.1 learns each channel's mappings and
+ * thresholds under 1, 2 and 4 bits before it assigns precisions): one read of W, the three runs work on the
+ * one normalised copy of the row in shared memory.  No layout.
+ *   maps3_dev, thresholds3_dev   fp32 [3][N][16]: plane 0 = the 1-bit tables of every row, plane 1 = the 2-bit
+ *                                tables, plane 2 = the 4-bit tables - the input format of lowra_channel_errors;
+ *                                plane c is bit for bit what lowra_learn_codebooks gives for a layout in which
+ *                                every row has 2^c bits                                                  (out)
+ * Other arguments, limits and errors as lowra_learn_codebooks (N >= 1, K % 128 == 0).
+ */
+lowra_status lowra_learn_codebooks_all(int32_t N, int32_t K, const float* W_dev, const double* init_levels_host,
+                                       const double* init_thresholds_host, int32_t iterations, float* maps3_dev,
+                                       float* thresholds3_dev, void* stream);
+
+/*
  * Diagnostic, not part of the method: C = P . Q^T with P bf16 [M, K], Q bf16 [N, K] (both
  * row-major, K % 64 == 0), C bf16 [M, N], run through the same tensor-core pipeline as the fused
  * kernels but with both operands fetched as plain bf16 tiles.  Used to compare "decode, then dense

@@ -30,6 +30,7 @@ EXPORTS = (
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
     "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
     "lowra_dense_nt_pair", "lowra_channel_errors", "lowra_deal_bytes", "lowra_deal_build", "lowra_workspace_init",
+    "lowra_learn_codebooks_all",
 )
 
 
@@ -89,6 +90,8 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_forward_static.restype = ctypes.c_int
         L.lowra_learn_codebooks.argtypes = [lp, vp, vp, vp, i32, vp, vp, vp]
         L.lowra_learn_codebooks.restype = ctypes.c_int
+        L.lowra_learn_codebooks_all.argtypes = [i32, i32, vp, vp, vp, i32, vp, vp, vp]
+        L.lowra_learn_codebooks_all.restype = ctypes.c_int
         L.lowra_natural_offsets.argtypes = [i32, i32, vp, vp]
         L.lowra_natural_offsets.restype = ctypes.c_int
         L.lowra_reorder_rows.argtypes = [lp, i32, vp, vp, vp, vp, vp, vp]
@@ -260,6 +263,32 @@ def lowra_learn_codebooks(layout: Layout, W: torch.Tensor, init_levels, init_thr
                                        _ptr(thresholds), _stream(stream))
     _check(code, "lowra_learn_codebooks")
     return maps, thresholds
+
+
+def lowra_learn_codebooks_all(W: torch.Tensor, init_levels, init_thresholds, iterations: int,
+                              maps3: Optional[torch.Tensor] = None, thresholds3: Optional[torch.Tensor] = None,
+                              stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Every row of W learnt at 1, 2 and 4 bits in one pass -> (maps3, thresholds3) fp32 [3, N, 16], the input
+    format of lowra_channel_errors."""
+    _dev(W, torch.float32, "W")
+    N, K = int(W.shape[0]), int(W.shape[1])
+    y0 = np.ascontiguousarray(init_levels, dtype=np.float64)
+    t0 = np.ascontiguousarray(init_thresholds, dtype=np.float64)
+    if y0.shape != (3, 16) or t0.shape != (3, 16):
+        raise ValueError("init_levels and init_thresholds must be [3, 16]")
+    if maps3 is None:
+        maps3 = torch.empty((3, N, 16), dtype=torch.float32, device=W.device)
+    if thresholds3 is None:
+        thresholds3 = torch.empty((3, N, 16), dtype=torch.float32, device=W.device)
+    _dev(maps3, torch.float32, "maps3")
+    _dev(thresholds3, torch.float32, "thresholds3")
+    if tuple(maps3.shape) != (3, N, 16) or tuple(thresholds3.shape) != (3, N, 16):
+        raise ValueError("maps3 and thresholds3 must be [3, N, 16]")
+    code = lib().lowra_learn_codebooks_all(N, K, _ptr(W), y0.ctypes.data_as(ctypes.c_void_p),
+                                           t0.ctypes.data_as(ctypes.c_void_p), int(iterations), _ptr(maps3),
+                                           _ptr(thresholds3), _stream(stream))
+    _check(code, "lowra_learn_codebooks_all")
+    return maps3, thresholds3
 
 
 def lowra_workspace_bytes(layout: Layout, M: int, r: int) -> int:

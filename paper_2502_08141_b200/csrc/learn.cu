@@ -15,6 +15,8 @@
 // slice of shared memory for 4 bits; a fixed reduction tree adds them up (warp shuffles, then across warps), so
 // results are reproducible from run to run - but the order of the fp64 additions is not the index order of a
 // serial loop, so sums agree with a serial implementation to rounding only.
+#include <string.h>
+
 #include "lowra_common.cuh"
 
 namespace lowra {
@@ -25,9 +27,10 @@ constexpr int kLearnWarps = kLearnThreads / 32;
 struct LearnParams {
     RowLayout L;
     const float* W;       // [N, K] original order
-    float* maps;          // [N, 16] original order
-    float* thresholds;    // [N, 16] original order
+    float* maps;          // [N, 16] original order ([3][N][16] in the three-precision form: plane c = 2^c bits)
+    float* thresholds;    // likewise
     int iterations;
+    int N, K;             // the three-precision form has no layout: every row is learnt at 1, 2 and 4 bits
     double init_y[3][16];  // initial levels per class (1, 2, 4 bits)
     double init_t[3][16];  // initial thresholds per class
 };
@@ -55,18 +58,12 @@ __device__ __forceinline__ int bucket_of(float x, const float* tf) {
     return c;
 }
 
-template <int B>
-__device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, double* acc, double* red, double* yt, float* tf) {
-    constexpr int Lv = 1 << B;      // levels
-    constexpr int c = B >> 1;       // class index
-    const int K = P.L.K, nb = P.L.nb;
+// The row: coalesced 128-bit loads into shared memory first (all of a thread's loads are in flight together), then
+// block absmax and normalised values in place (as in lowra_encode).  Ends with a barrier.
+__device__ void load_row(const LearnParams& P, int r, float* xs, float* ws) {
+    const int K = P.K, nb = K / kBlock;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const float* wrow = P.W + (size_t)r * K;
-    double* y = yt;          // [16] levels
-    double* t = yt + 16;     // [16] thresholds
-
-    // ---- the row: coalesced 128-bit loads into shared memory first (all of a thread's loads are in flight
-    // together), then block absmax and normalised values in place (as in lowra_encode)
     for (int i0 = 0; i0 < K; i0 += 4 * 4 * kLearnThreads) {
         float4 v[4];
 #pragma unroll
@@ -90,6 +87,19 @@ __device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, dou
         *reinterpret_cast<float2*>(xs + g * kBlock + 2 * lane) = make_float2(__fmul_rn(v.x, inv), __fmul_rn(v.y, inv));
         if (lane == 0) ws[g] = m;
     }
+    __syncthreads();
+}
+
+// T rounds on the row parked in shared memory, at B bits; tables to maps_out / thr_out ([16] each).
+template <int B>
+__device__ void learn_row(const LearnParams& P, const float* xs, const float* ws, double* acc, double* red, double* yt,
+                          float* tf, float* maps_out, float* thr_out) {
+    constexpr int Lv = 1 << B;      // levels
+    constexpr int c = B >> 1;       // class index
+    const int K = P.K;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    double* y = yt;          // [16] levels
+    double* t = yt + 16;     // [16] thresholds
     if (tid < 16) {
         y[tid] = P.init_y[c][tid];
         t[tid] = P.init_t[c][tid];
@@ -179,13 +189,13 @@ __device__ void learn_row(const LearnParams& P, int r, float* xs, float* ws, dou
     if (tid < kTableStride) {
         const float m = (tid < Lv) ? (float)y[tid] : 0.0f;
         const float mn = (tid + 1 < Lv) ? (float)y[tid + 1] : 0.0f;
-        P.maps[(size_t)r * kTableStride + tid] = m;
-        P.thresholds[(size_t)r * kTableStride + tid] =
-            (tid + 1 < Lv) ? (float)(((double)m + (double)mn) * 0.5) : __int_as_float(0x7f800000);
+        maps_out[tid] = m;
+        thr_out[tid] = (tid + 1 < Lv) ? (float)(((double)m + (double)mn) * 0.5) : __int_as_float(0x7f800000);
     }
-    __syncthreads();   // the row buffers are reused by the next row
+    __syncthreads();   // the tables and sums in shared memory are reused by the next run, the row buffer by the next row
 }
 
+template <bool ALL3>
 __global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_constant__ LearnParams P) {
     extern __shared__ __align__(16) unsigned char learn_smem[];
     // [16 + 16 doubles levels/thresholds][2 * 16 * warps doubles reduction][2 * 16 * threads doubles sums][K floats][nb floats][16 floats]
@@ -193,17 +203,70 @@ __global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_const
     double* red = yt + 32;
     double* acc = red + 2 * 16 * kLearnWarps;
     float* xs = reinterpret_cast<float*>(acc + 2 * 16 * kLearnThreads);
-    float* ws = xs + P.L.K;
-    float* tf = ws + P.L.nb;   // [16] thresholds as fp32 upper neighbours
+    float* ws = xs + P.K;
+    float* tf = ws + P.K / kBlock;   // [16] thresholds as fp32 upper neighbours
     pdl_enter();
-    for (int r = blockIdx.x; r < P.L.N; r += gridDim.x) {
-        const int b = P.L.precs[r];
-        if (b == 1) learn_row<1>(P, r, xs, ws, acc, red, yt, tf);
-        else if (b == 2) learn_row<2>(P, r, xs, ws, acc, red, yt, tf);
-        else learn_row<4>(P, r, xs, ws, acc, red, yt, tf);
+    for (int r = blockIdx.x; r < P.N; r += gridDim.x) {
+        load_row(P, r, xs, ws);
+        float* m = P.maps + (size_t)r * kTableStride;
+        float* h = P.thresholds + (size_t)r * kTableStride;
+        if (ALL3) {
+            // the row under every precision, from the one copy in shared memory
+            const size_t plane = (size_t)P.N * kTableStride;
+            learn_row<1>(P, xs, ws, acc, red, yt, tf, m, h);
+            learn_row<2>(P, xs, ws, acc, red, yt, tf, m + plane, h + plane);
+            learn_row<4>(P, xs, ws, acc, red, yt, tf, m + 2 * plane, h + 2 * plane);
+        } else {
+            const int b = P.L.precs[r];
+            if (b == 1) learn_row<1>(P, xs, ws, acc, red, yt, tf, m, h);
+            else if (b == 2) learn_row<2>(P, xs, ws, acc, red, yt, tf, m, h);
+            else learn_row<4>(P, xs, ws, acc, red, yt, tf, m, h);
+        }
     }
 }
 
+}  // namespace lowra
+
+namespace lowra {
+namespace {
+
+// validation shared by the two entry points is done by the callers; this fills the tables and launches
+template <bool ALL3>
+lowra_status launch_learn(LearnParams& P, const double* init_levels_host, const double* init_thresholds_host,
+                          void* stream) {
+    const size_t smem = (32 + 2 * 16 * kLearnWarps + 2 * 16 * kLearnThreads) * sizeof(double) +
+                        ((size_t)P.K + (size_t)P.K / kBlock + 16) * sizeof(float);
+    if (smem > 200 * 1024) return LOWRA_ERR_SHAPE;   // the row has to fit into shared memory (K <= 40960)
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    for (int c = 0; c < 3; ++c)
+        for (int j = 0; j < 16; ++j) {
+            P.init_y[c][j] = init_levels_host[c * 16 + j];
+            P.init_t[c][j] = init_thresholds_host[c * 16 + j];
+        }
+    static size_t configured = 0;
+    if (smem > configured) {
+        if (cudaFuncSetAttribute(learn_kernel<ALL3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+            return LOWRA_ERR_CUDA;
+        configured = smem;
+    }
+    const int per_sm = (int)((220u * 1024u) / (smem + 1024u));
+    const int cap = kNumSMs * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));
+    const unsigned grid = (unsigned)(P.N < cap ? P.N : cap);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(grid, 1, 1);
+    cfg.blockDim = dim3(kLearnThreads, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = (cudaStream_t)stream;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, learn_kernel<ALL3>, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+}
+
+}  // namespace
 }  // namespace lowra
 
 extern "C" lowra_status lowra_learn_codebooks(const lowra_layout* layout, const float* W_dev,
@@ -215,41 +278,32 @@ extern "C" lowra_status lowra_learn_codebooks(const lowra_layout* layout, const 
     if (!W_dev || !init_levels_host || !init_thresholds_host || !maps_dev || !thresholds_dev) return LOWRA_ERR_NULL;
     if (iterations < 0 || iterations > 1000) return LOWRA_ERR_SHAPE;
     if (!aligned16(W_dev) || !aligned16(maps_dev) || !aligned16(thresholds_dev)) return LOWRA_ERR_ALIGN;
-    const size_t smem = (32 + 2 * 16 * kLearnWarps + 2 * 16 * kLearnThreads) * sizeof(double) +
-                        ((size_t)layout->K + (size_t)layout->K / kBlock + 16) * sizeof(float);
-    if (smem > 200 * 1024) return LOWRA_ERR_SHAPE;   // the row has to fit into shared memory (K <= 40960)
-    st = check_device();
-    if (st != LOWRA_OK) return st;
-
     LearnParams P;
     P.L = make_row_layout(layout);
     P.W = W_dev;
     P.maps = maps_dev;
     P.thresholds = thresholds_dev;
     P.iterations = iterations;
-    for (int c = 0; c < 3; ++c)
-        for (int j = 0; j < 16; ++j) {
-            P.init_y[c][j] = init_levels_host[c * 16 + j];
-            P.init_t[c][j] = init_thresholds_host[c * 16 + j];
-        }
-    static size_t configured = 0;
-    if (smem > configured) {
-        if (cudaFuncSetAttribute(learn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return LOWRA_ERR_CUDA;
-        configured = smem;
-    }
-    const int per_sm = (int)((220u * 1024u) / (smem + 1024u));
-    const int cap = kNumSMs * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));
-    const unsigned grid = (unsigned)(layout->N < cap ? layout->N : cap);
-    cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.gridDim = dim3(grid, 1, 1);
-    cfg.blockDim = dim3(kLearnThreads, 1, 1);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = (cudaStream_t)stream;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, learn_kernel, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+    P.N = layout->N;
+    P.K = layout->K;
+    return launch_learn<false>(P, init_levels_host, init_thresholds_host, stream);
+}
+
+extern "C" lowra_status lowra_learn_codebooks_all(int32_t N, int32_t K, const float* W_dev,
+                                                  const double* init_levels_host, const double* init_thresholds_host,
+                                                  int32_t iterations, float* maps3_dev, float* thresholds3_dev,
+                                                  void* stream) {
+    using namespace lowra;
+    if (!W_dev || !init_levels_host || !init_thresholds_host || !maps3_dev || !thresholds3_dev) return LOWRA_ERR_NULL;
+    if (N < 1 || K < 128 || K % 128 != 0 || iterations < 0 || iterations > 1000) return LOWRA_ERR_SHAPE;
+    if (!aligned16(W_dev) || !aligned16(maps3_dev) || !aligned16(thresholds3_dev)) return LOWRA_ERR_ALIGN;
+    LearnParams P;
+    memset(&P.L, 0, sizeof(P.L));   // no layout: every row at every precision
+    P.W = W_dev;
+    P.maps = maps3_dev;
+    P.thresholds = thresholds3_dev;
+    P.iterations = iterations;
+    P.N = N;
+    P.K = K;
+    return launch_learn<true>(P, init_levels_host, init_thresholds_host, stream);
 }

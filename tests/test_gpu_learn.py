@@ -121,3 +121,28 @@ def test_learned_tables_feed_the_encoder(lw):
     err_gpu = float(((W_hat - W) ** 2).sum())
     err_ref = float(((W_ref - W) ** 2).sum())
     assert abs(err_gpu - err_ref) <= 1e-4 * err_ref
+
+
+@pytest.mark.parametrize("N,K,T", [(96, 512, 10), (333, 1408, 2), (40, 11008, 3)])
+def test_all_three_precisions_in_one_pass(lw, N, K, T):
+    """lowra_learn_codebooks_all: every row at 1, 2 and 4 bits from one read of W.  Plane c is bit for bit what the
+    per-layout learner gives when every row has 2^c bits (same arithmetic on the same normalised row), and agrees
+    with the oracle like that one; its output feeds lowra_channel_errors as it stands."""
+    W = si.weights(N, K, matrix_id=(N + K) % 53, kind="llama")
+    Wd = torch.from_numpy(W).cuda()
+    y0, t0 = _init_tables()
+    maps3, thr3 = lw.lowra_learn_codebooks_all(Wd, y0, t0, T)
+    torch.cuda.synchronize()
+    sse_ref = np.zeros((N, 3))
+    for c, b in enumerate((1, 2, 4)):
+        precs = np.full(N, b, dtype=np.uint8)
+        m1, h1 = lw.lowra_learn_codebooks(lw.Layout(precs, K), Wd, y0, t0, T)
+        assert torch.equal(maps3[c].view(torch.int32), m1.view(torch.int32)), b
+        assert torch.equal(thr3[c].view(torch.int32), h1.view(torch.int32)), b
+        maps_ref, thr_ref = oracle.lloyd_max(W, precs, T=T)
+        _check(maps3[c].cpu().numpy(), thr3[c].cpu().numpy(), precs, maps_ref, thr_ref)
+        sse_ref[:, c], _ = oracle.quant_error(W, precs, maps3[c].cpu().numpy(), thr3[c].cpu().numpy())
+    # the two calls that give the precision assigner its input: tables for all precisions, then the errors
+    sse3 = lw.lowra_channel_errors(Wd, maps3, thr3).cpu().numpy()
+    assert np.all(np.abs(sse3 - sse_ref) <= 2.0 ** -21 * sse_ref)
+    assert (sse3[:, 1] < sse3[:, 0]).all() and (sse3[:, 2] < sse3[:, 1]).all()

@@ -116,6 +116,10 @@ def test_validation_runs_before_any_device_work(lib):
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, None, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_NULL
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, init, init, -1, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096 + 4, init, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_ALIGN
+    assert L.lowra_learn_codebooks_all(16, 256, 4096, init, None, 10, 4096, 4096, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_learn_codebooks_all(16, 200, 4096, init, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
+    assert L.lowra_learn_codebooks_all(0, 256, 4096, init, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE
+    assert L.lowra_learn_codebooks_all(16, 256, 4096, init, init, 10, 4096 + 4, 4096, None) == lib.LOWRA_ERR_ALIGN
     # natural-order offsets (host only) and the row reordering
     import numpy as np
     pr = np.array([1, 4, 2, 2], dtype=np.uint8)
