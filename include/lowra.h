@@ -169,7 +169,7 @@ size_t lowra_workspace_bytes(const lowra_layout* layout, int32_t M, int32_t r);
  * dequantising warps sorted by precision.  With layout->deal_dev == NULL every call works that out again in
  * a small prologue launch, which also clears the status word and the flags in the workspace.  With
  * layout->deal_dev pointing at a buffer filled by lowra_deal_build the fused kernel is the only launch
- * of a call (5-7 us less per call on a B200); the workspace then has to be initialised once with
+ * of a call (3-6 us less per call on a B200); the workspace then has to be initialised once with
  * lowra_workspace_init before its first use, is written by these calls only, and its status word is no
  * longer cleared per call: lowra_device_status reports the first failure since the initialisation.
  *   lowra_deal_bytes   size of the buffer for this layout (0 if the layout is invalid); about 40 bytes per
