@@ -1,21 +1,33 @@
 #!/usr/bin/env python
 """Benchmark of the LowRA quantized-LoRA hot path on B200.
 
-A *step* is one pass of the whole hot path over one Llama-7B-shaped decoder layer (seven weight
-matrices, 4096 tokens, LoRA rank 64, precision mix averaging 1.5 bits): for every matrix
-lowra_encode, lowra_decode, lowra_lora_forward and lowra_lora_backward_input, through the C ABI.
+A *step* is one pass of the whole hot path over one workload, through the C ABI: for every weight matrix
+lowra_encode, lowra_decode, lowra_lora_forward and (where the workload has it) lowra_lora_backward_input.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload {2,3,4,5}] [--impl reference]
+    python bench.py --case NAME        # one small launch of one kernel family, sized for a profiler capture
 
-Prints ONE JSON line.  `value` is the fused dequant+LoRA product throughput of the step (algorithmic
-FLOPs of the 7 forward + 7 backward products divided by the time of the WHOLE step, encode and decode
-included), measured with CUDA events and inputs resident in HBM; `phases` breaks the step down
-(encode / decode in GB/s, forward / backward in TFLOP/s); `e2e` repeats the step with host buffers and
-the host<->device copies inside the timed region; `roofline` is for the dominant kernel (the fused
-tensor-core kernel); `cpu_baseline` times the CPU oracle on a bounded sample of the same workload.
+Workloads (the configurations of the benchmark spec; 3 is the default and the headline):
+    2  one 4096 x 4096 matrix at 2048 tokens, 2.1 bits on average (run on 8 seeded matrices of that shape per
+       step, so that a step's inputs exceed the L2 cache)
+    3  one Llama-7B-shaped decoder layer (7 matrices), 4096 tokens, 1.5 bits
+    4  one Llama-13B-shaped decoder layer, 4096 tokens, 1.15 bits
+    5  a whole 32-layer Llama-7B-shaped model (224 matrices, 6.5 G parameters), 2.5 bits: encode + decode sweep
+       over every matrix, forward at 1024 / 4096 / 8192 tokens per matrix (no backward)
+Codebooks are learnt on the GPU before the timed region (lowra_learn_codebooks: 10 rounds of weighted Lloyd-Max
+per row from the paper's Appendix-F starting tables), as the configurations say.
 
-With N > 1 (torchrun) every rank runs the same layer shapes on its own seeded weights (independent
-problems, no data-path collective; weak scaling) and rank 0 reports the aggregate.
+Prints ONE JSON line.  `value` is the fused dequant+LoRA product throughput of the step (algorithmic FLOPs of
+the products divided by the time of the WHOLE step, encode and decode included), measured with CUDA events and
+inputs resident in HBM; `phases` breaks the step down; `per_matrix` gives every (matrix, operation) its own
+figure; `e2e` repeats the step with host buffers and the host<->device copies inside the timed region;
+`roofline` is for the dominant kernel (the fused tensor-core kernel) and carries, under `secondary`, the HBM
+figures of decode and encode taken over several GB of distinct buffers (so that what is still in L2 when the
+clock stops is a few per cent); `cpu_baseline` times the CPU oracle on a bounded sample of the same workload and
+holds the GPU's results of that sample against the oracle's.
+
+With N > 1 (torchrun) every rank runs the same shapes on its own seeded weights (independent problems, no
+data-path collective; weak scaling) and rank 0 reports the aggregate.
 
 `--impl reference` times the CPU oracle alone (there is no reference code for this paper).
 """
@@ -23,6 +35,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -39,9 +52,11 @@ if ROOT not in sys.path:
 
 import synth_inputs as si  # noqa: E402
 
-WORKLOAD = 3  # Llama-7B decoder layer, 4096 tokens, avg 1.5 bits
-METRIC = "fused dequant+LoRA fwd+bwd throughput over one Llama-7B layer step (encode+decode+fwd+bwd)"
+METRIC = "fused dequant+LoRA product throughput over one step (encode + decode + forward + backward-input of every matrix)"
 UNIT = "TFLOP/s"
+LLOYD_ITERS = 10
+SWEEP_BYTES = 3.2e9          # decode / encode HBM figures are taken over at least this much output (input)
+L2_BYTES = 126e6
 
 
 def gemm_flops(M, N, K, r):
@@ -135,32 +150,31 @@ class ClockSampler:
 # --------------------------------------------------------------------------------------------------
 # workload
 # --------------------------------------------------------------------------------------------------
-def make_host_inputs(cfg, rank: int):
-    """Seeded host inputs of one layer (matrix ids offset by the rank, so ranks hold different layers)."""
-    M, r = cfg.tokens[0], cfg.rank
+def workload_matrices(workload: int):
+    """(config, list of matrices of one step).  Workload 2 runs its one shape on 8 seeded matrices per step so
+    that the step's inputs exceed L2 between timed iterations."""
+    cfg = si.config(workload)
+    mats = list(cfg.matrices)
+    if workload == 2:
+        mats = [si.Matrix(f"{mats[0].name}#{i}", mats[0].N, mats[0].K, i) for i in range(8)]
+    return cfg, mats
 
-    def one(mat):
-        mid = rank_matrix_id(mat.matrix_id, rank)
-        W = si.weights(mat.N, mat.K, matrix_id=mid, kind=cfg.weight_kind)
-        precs = si.precisions(mat.N, cfg.mix, matrix_id=mid)
-        maps, thr = si.standin_codebooks(precs, matrix_id=mid)
-        A, B = si.lora_factors(mat.K, mat.N, r, matrix_id=mid)
-        return dict(name=mat.name, N=mat.N, K=mat.K, W=W, precs=precs, maps=maps, thr=thr, A=A, B=B)
 
-    with ThreadPoolExecutor(max_workers=min(8, len(cfg.matrices))) as ex:
-        mats = list(ex.map(one, cfg.matrices))
-    # one activation / gradient buffer per distinct width, shared by the matrices of that width
-    acts = {}
-    for m in mats:
-        if m["K"] not in acts:
-            acts[m["K"]] = si.activations(M, m["K"], matrix_id=100 + rank)
-        if m["N"] not in acts:
-            acts[m["N"]] = si.activations(M, m["N"], matrix_id=100 + rank)
-    return mats, acts
+def rank_matrix_id(matrix_id: int, rank: int, per_rank: int = 7) -> int:
+    """Ranks hold different weights: the seed stream of matrix j on rank q is that of matrix j + per_rank * q."""
+    return matrix_id + per_rank * rank
+
+
+def host_matrix(cfg, mat, rank: int, per_rank: int):
+    mid = rank_matrix_id(mat.matrix_id, rank, per_rank)
+    W = si.weights(mat.N, mat.K, matrix_id=mid, kind=cfg.weight_kind)
+    precs = si.precisions(mat.N, cfg.mix, matrix_id=mid)
+    A, B = si.lora_factors(mat.K, mat.N, cfg.rank, matrix_id=mid % 7)      # factors repeat from layer to layer
+    return dict(name=mat.name, N=mat.N, K=mat.K, W=W, precs=precs, A=A, B=B, matrix_id=mid)
 
 
 # DRAM traffic of one fused_kernel launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a
-# launch of this very workload: the backward-input pass of gate_proj (dX [4096, 4096] from dY [4096, 11008];
+# launch of workload 3: the backward-input pass of gate_proj (dX [4096, 4096] from dY [4096, 11008];
 # profiles/fused_backward_input_11008x4096_m4096_streamk.md): 167.9 MB read + 29.7 MB written.  The bytes the call
 # has to read and write once are 137 MB (the output is partly still in L2 when the kernel ends; the stream-K partial
 # tiles add 19 MB each way).  Scaled to the step's average launch in proportion to those input + output bytes.
@@ -172,10 +186,10 @@ def fused_io_bytes(N, K, M, r, bits):
     return 2.0 * M * K + N * K * (bits / 8 + 4 / 64) + 64.0 * N + 2.0 * (K + N) * r + 2.0 * M * N
 
 
-def fused_traffic_per_launch(dev, M, r, bits):
+def fused_traffic_per_launch(calls, r, bits):
+    """calls: (N, K, M) of every fused launch of a step, with N = rows of the operand that is dequantised."""
     case = fused_io_bytes(NCU_CASE["N"], NCU_CASE["K"], NCU_CASE["M"], NCU_CASE["r"], NCU_CASE["bits"])
-    per = [fused_io_bytes(d["m"]["N"], d["m"]["K"], M, r, bits) for d in dev] + \
-          [fused_io_bytes(d["m"]["K"], d["m"]["N"], M, r, bits) for d in dev]   # backward reads dY [M, N], writes dX [M, K]
+    per = [fused_io_bytes(N, K, M, r, bits) for N, K, M in calls]
     return NCU_CASE["dram_bytes"] / case * sum(per) / len(per)
 
 
@@ -191,13 +205,8 @@ def max_over_ranks(ms: float, world: int, device="cuda") -> float:
 
 
 def aggregate_tflops(flops_per_rank_step: float, world: int, ms_per_step: float) -> float:
-    """Whole-job throughput: every rank does one layer step per step (weak scaling)."""
+    """Whole-job throughput: every rank does one step's work per step (weak scaling)."""
     return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
-
-
-def rank_matrix_id(matrix_id: int, rank: int, per_layer: int = 7) -> int:
-    """Ranks hold different layers: the seed stream of matrix j on rank q is that of matrix j + 7 q."""
-    return matrix_id + per_layer * rank
 
 
 def run_gpu(args):
@@ -216,59 +225,115 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     lw.lib()
 
-    cfg = si.config(WORKLOAD)
-    M, r, s = cfg.tokens[0], cfg.rank, cfg.s
+    cfg, mat_list = workload_matrices(args.workload)
+    token_counts = list(cfg.tokens)
+    with_backward = "backward" in cfg.ops
+    r, s = cfg.rank, cfg.s
     bits = si.avg_bits(cfg.mix)
-    mats, acts = make_host_inputs(cfg, rank)
+    per_rank = len(mat_list)
+    y0, t0 = si.initial_codebooks()
 
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
     bfv = lambda t: t.view(torch.bfloat16)
-    # ---- device-resident problem
-    dev = []
-    for m in mats:
-        # the deal of the rows to the dequant warps depends on the precisions only: built once per weight, like the
-        # storage plan, unless --deal-per-call asks for the prologue launch in every call
-        layout = lw.Layout(m["precs"], m["K"])
-        if not args.deal_per_call:
-            layout.build_deal()
-        d = dict(m=m, layout=layout,
-                 W=torch.from_numpy(m["W"]).cuda(), thr=torch.from_numpy(m["thr"]).cuda(),
-                 maps=torch.from_numpy(m["maps"]).cuda(),
-                 A=bfv(torch.from_numpy(m["A"].view(np.int16)).cuda()), B=bfv(torch.from_numpy(m["B"].view(np.int16)).cuda()),
-                 packed=torch.empty(max(layout.packed_bytes, 16), dtype=torch.uint8, device="cuda"),
-                 absmax=torch.empty((m["N"], m["K"] // 64), dtype=torch.float32, device="cuda"),
-                 What=torch.empty((m["N"], m["K"]), dtype=torch.bfloat16, device="cuda"),
-                 Y=torch.empty((M, m["N"]), dtype=torch.bfloat16, device="cuda"),
-                 dX=torch.empty((M, m["K"]), dtype=torch.bfloat16, device="cuda"),
-                 ws=lw.lowra_workspace_init(torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")))
-        dev.append(d)
-    act_dev = {k: bfv(torch.from_numpy(v.view(np.int16)).cuda()) for k, v in acts.items()}
     stream = torch.cuda.current_stream()
+    # ---- device-resident problem: weights are drawn on the host (seeded, one matrix after the other, a few threads
+    # ahead of the uploads) and stay in HBM; codebooks are learnt here, on the GPU, from the Appendix-F tables
+    dev = []
+    t_gen = time.time()
+    with ThreadPoolExecutor(max_workers=min(os.cpu_count() or 8, 32, len(mat_list))) as ex:
+        for m in ex.map(lambda mat: host_matrix(cfg, mat, rank, per_rank), mat_list):
+            layout = lw.Layout(m["precs"], m["K"])
+            if not args.deal_per_call:
+                layout.build_deal()     # the deal of the rows depends on the precisions only: once per weight, like the plan
+            N, K = m["N"], m["K"]
+            d = dict(name=m["name"], N=N, K=K, layout=layout, matrix_id=m["matrix_id"],
+                     W=torch.from_numpy(m["W"]).cuda(),
+                     A=bfv(torch.from_numpy(m["A"].view(np.int16)).cuda()), B=bfv(torch.from_numpy(m["B"].view(np.int16)).cuda()),
+                     maps=torch.empty((N, 16), dtype=torch.float32, device="cuda"),
+                     thr=torch.empty((N, 16), dtype=torch.float32, device="cuda"),
+                     packed=torch.empty(max(layout.packed_bytes, 16), dtype=torch.uint8, device="cuda"),
+                     absmax=torch.empty((N, K // 64), dtype=torch.float32, device="cuda"),
+                     What=torch.empty((N, K), dtype=torch.bfloat16, device="cuda"))
+            lw.lowra_learn_codebooks(layout, d["W"], y0, t0, LLOYD_ITERS, maps=d["maps"], thresholds=d["thr"])
+            if len(dev) < 7:
+                d["host"] = m            # kept for the end-to-end leg and the check against the oracle
+            dev.append(d)
+    torch.cuda.synchronize()
+    t_gen = time.time() - t_gen
+    shapes = sorted({(d["N"], d["K"]) for d in dev})
+    widths = sorted({w for N, K in shapes for w in (N, K)})
+    # one activation / output-gradient buffer per (token count, width), shared by the matrices of that width; one
+    # output buffer per (token count, width) when the workload has many matrices, one per matrix otherwise
+    act_dev = {}
+    for M in token_counts:
+        for wdt in widths:
+            act_dev[(M, wdt)] = bfv(torch.from_numpy(si.activations(M, wdt, matrix_id=100 + rank).view(np.int16)).cuda())
+    shared_out = len(dev) > 8
+    out_shared = {}
+
+    def out_buf(d, M, cols, key):
+        if shared_out:
+            k = (M, cols, key)
+            if k not in out_shared:
+                out_shared[k] = torch.empty((M, cols), dtype=torch.bfloat16, device="cuda")
+            return out_shared[k]
+        return torch.empty((M, cols), dtype=torch.bfloat16, device="cuda")
+
+    for d in dev:
+        d["Y"] = {M: out_buf(d, M, d["N"], "Y") for M in token_counts}
+        d["dX"] = {M: out_buf(d, M, d["K"], "dX") for M in token_counts} if with_backward else None
+    ws_shared = {}
+    for d in dev:
+        d["ws"] = {}
+        for M in token_counts:
+            n = lw.lowra_workspace_bytes(d["layout"], M, r)
+            if shared_out:      # calls on one stream never overlap: one workspace per token count, sized for the largest
+                if M not in ws_shared or ws_shared[M].numel() < n:
+                    ws_shared[M] = torch.empty(n, dtype=torch.uint8, device="cuda")
+                d["ws"][M] = None
+            else:
+                d["ws"][M] = lw.lowra_workspace_init(torch.empty(n, dtype=torch.uint8, device="cuda"))
+    if shared_out:
+        for M in token_counts:
+            lw.lowra_workspace_init(ws_shared[M])
+        for d in dev:
+            for M in token_counts:
+                d["ws"][M] = ws_shared[M]
+    all_ws = list({id(w): w for d in dev for w in d["ws"].values()}.values())
+
+    def check_status(where):
+        for w in all_ws:
+            st = lw.lowra_device_status(w)
+            if st != 0:
+                raise SystemExit(f"device status {st} ({lw.status_string(st)}) {where}")
+
+    f_encode = lambda d, M=None: lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"])
+    f_decode = lambda d, M=None: lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"])
+    f_forward = lambda d, M: lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], act_dev[(M, d["K"])],
+                                                   d["A"], d["B"], s, Y=d["Y"][M], workspace=d["ws"][M])
+    f_backward = lambda d, M: lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], act_dev[(M, d["N"])],
+                                                           d["A"], d["B"], s, dX=d["dX"][M], workspace=d["ws"][M])
+    phase_list = [("encode", f_encode, [None]), ("decode", f_decode, [None]), ("forward", f_forward, token_counts)]
+    if with_backward:
+        phase_list.append(("backward", f_backward, token_counts))
 
     def step(record=None, per_call=None):
         """One pass.  `record` (a list) receives (phase, event_start, event_end) per phase: the calls of a phase
         run back to back, as a user would issue them; `per_call` receives the same per call (diagnostic pass)."""
-        def phase(name, fn):
+        for name, fn, Ms in phase_list:
             if record is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
-            for d in dev:
-                if per_call is not None:
-                    c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    c0.record(stream); fn(d); c1.record(stream)
-                    per_call.append((name, c0, c1))
-                else:
-                    fn(d)
+            for M in Ms:
+                for i, d in enumerate(dev):
+                    if per_call is not None:
+                        c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        c0.record(stream); fn(d, M); c1.record(stream)
+                        per_call.append((name, M, i, c0, c1))
+                    else:
+                        fn(d, M)
             if record is not None:
                 e1.record(stream)
                 record.append((name, e0, e1))
-        phase("encode", lambda d: lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"]))
-        phase("decode", lambda d: lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"]))
-        phase("forward", lambda d: lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"],
-                                                         act_dev[d["m"]["K"]], d["A"], d["B"], s, Y=d["Y"], workspace=d["ws"]))
-        phase("backward", lambda d: lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"],
-                                                                 act_dev[d["m"]["N"]], d["A"], d["B"], s, dX=d["dX"],
-                                                                 workspace=d["ws"]))
 
     def barrier():
         torch.cuda.synchronize()
@@ -276,12 +341,10 @@ def run_gpu(args):
             dist.barrier()
             torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    n_warm = max(args.warmup, 3)
+    for _ in range(n_warm):
         step()
-    for d in dev:
-        st = lw.lowra_device_status(d["ws"])
-        if st != 0:
-            raise SystemExit(f"device status {st} after warm-up")
+    check_status("after warm-up")
 
     # ---- timed region: exactly K steps, device timing with CUDA events, max over ranks
     sampler = ClockSampler(local_rank)
@@ -290,57 +353,119 @@ def run_gpu(args):
     barrier()
     records = []
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    t0 = time.time()
+    t0w = time.time()
     ev0.record(stream)
     for _ in range(args.steps):
         step(records)
     ev1.record(stream)
     barrier()
-    t1 = time.time()
-    clocks = sampler.stop(t0, t1)
+    t1w = time.time()
+    clocks = sampler.stop(t0w, t1w)
     total_ms = ev0.elapsed_time(ev1)
     total_ms = max_over_ranks(total_ms, world)
     ms_per_step = total_ms / args.steps
+    check_status("after the timed steps")
 
-    flops_step = sum(2 * gemm_flops(M, d["m"]["N"], d["m"]["K"], r) for d in dev)
+    dirs = 2 if with_backward else 1
+    flops_dir = sum(gemm_flops(M, d["N"], d["K"], r) for M in token_counts for d in dev)
+    flops_step = dirs * flops_dir
     value = aggregate_tflops(flops_step, world, ms_per_step)
 
-    phase_ms, call_ms = {}, {}
+    phase_ms = {}
     for phase, e0, e1 in records:
         phase_ms[phase] = phase_ms.get(phase, 0.0) + e0.elapsed_time(e1)
     for k in phase_ms:
         phase_ms[k] /= args.steps
     # diagnostic pass outside the timed region: the same step with events around every call
-    n_diag = 3
+    n_diag = 3 if len(dev) <= 8 else 1
     calls = []
     for _ in range(n_diag):
         step(per_call=calls)
     torch.cuda.synchronize()
-    for idx, (phase, c0, c1) in enumerate(calls):
-        per = call_ms.setdefault(phase, [0.0] * len(dev))
-        per[idx % len(dev)] += c0.elapsed_time(c1) / n_diag      # the calls of a phase run in the order of the matrices
-    elems = sum(d["m"]["N"] * d["m"]["K"] for d in dev)
+    call_ms = {}
+    for phase, M, i, c0, c1 in calls:
+        call_ms[(phase, M, i)] = call_ms.get((phase, M, i), 0.0) + c0.elapsed_time(c1) / n_diag
+    elems = sum(d["N"] * d["K"] for d in dev)
     P = peaks()
-    dec_gbs = sum(decode_bytes(d["m"]["N"], d["m"]["K"], bits) for d in dev) / (phase_ms["decode"] * 1e-3) / 1e9
-    enc_gbs = sum(encode_bytes(d["m"]["N"], d["m"]["K"], bits) for d in dev) / (phase_ms["encode"] * 1e-3) / 1e9
-    fwd_tf = flops_step / 2 / (phase_ms["forward"] * 1e-3) / 1e12
-    bwd_tf = flops_step / 2 / (phase_ms["backward"] * 1e-3) / 1e12
+    dec_bytes = sum(decode_bytes(d["N"], d["K"], bits) for d in dev)
+    enc_bytes = sum(encode_bytes(d["N"], d["K"], bits) for d in dev)
+    dec_gbs = dec_bytes / (phase_ms["decode"] * 1e-3) / 1e9
+    enc_gbs = enc_bytes / (phase_ms["encode"] * 1e-3) / 1e9
+    fwd_tf = flops_dir / (phase_ms["forward"] * 1e-3) / 1e12
+    tens = lambda tf: {"TFLOP/s": tf, "frac_tensor_burst": tf / P["tensor_burst"], "frac_tensor_sustained": tf / P["tensor_sustained"],
+                       "frac_tensor_nominal_2250": tf / 2250.0}
     phases = {
         "encode": {"ms": phase_ms["encode"], "GB/s": enc_gbs, "frac_hbm": enc_gbs / P["hbm"], "frac_hbm_nominal_8TBs": enc_gbs / 8000.0},
         "decode": {"ms": phase_ms["decode"], "GB/s": dec_gbs, "frac_hbm": dec_gbs / P["hbm"], "frac_hbm_nominal_8TBs": dec_gbs / 8000.0},
-        "forward": {"ms": phase_ms["forward"], "TFLOP/s": fwd_tf, "frac_tensor_burst": fwd_tf / P["tensor_burst"],
-                    "frac_tensor_sustained": fwd_tf / P["tensor_sustained"], "frac_tensor_nominal_2250": fwd_tf / 2250.0},
-        "backward_input": {"ms": phase_ms["backward"], "TFLOP/s": bwd_tf, "frac_tensor_burst": bwd_tf / P["tensor_burst"],
-                           "frac_tensor_sustained": bwd_tf / P["tensor_sustained"], "frac_tensor_nominal_2250": bwd_tf / 2250.0},
+        "forward": dict(ms=phase_ms["forward"], **tens(fwd_tf)),
     }
-    names = [d["m"].get("name", f'{d["m"]["N"]}x{d["m"]["K"]}') for d in dev]
-    for key, phase in (("forward", "forward"), ("backward_input", "backward")):
-        phases[key]["TFLOP/s_per_matrix (separate pass, events around every call)"] = {
-            f"{i}:{n}": round(gemm_flops(M, d["m"]["N"], d["m"]["K"], r) / (ms * 1e-3) / 1e12, 1)
-            for i, (n, d, ms) in enumerate(zip(names, dev, call_ms[phase]))}
+    if with_backward:
+        bwd_tf = flops_dir / (phase_ms["backward"] * 1e-3) / 1e12
+        phases["backward_input"] = dict(ms=phase_ms["backward"], **tens(bwd_tf))
+    # every (matrix shape, token count, operation): mean over the matrices of that shape (separate pass, events around every call)
+    per_matrix = []
+    for N, K in shapes:
+        idx = [i for i, d in enumerate(dev) if (d["N"], d["K"]) == (N, K)]
+        names = sorted({dev[i]["name"].split("#")[0] for i in idx})
+        row = {"shape": f"{N}x{K}", "matrices": "/".join(names), "count": len(idx)}
+        mean = lambda phase, M: sum(call_ms[(phase, M, i)] for i in idx) / len(idx)
+        row["encode_GB/s"] = round(encode_bytes(N, K, bits) / (mean("encode", None) * 1e-3) / 1e9, 1)
+        row["decode_GB/s"] = round(decode_bytes(N, K, bits) / (mean("decode", None) * 1e-3) / 1e9, 1)
+        for M in token_counts:
+            row[f"forward_TFLOP/s@{M}"] = round(gemm_flops(M, N, K, r) / (mean("forward", M) * 1e-3) / 1e12, 1)
+            if with_backward:
+                row[f"backward_input_TFLOP/s@{M}"] = round(gemm_flops(M, N, K, r) / (mean("backward", M) * 1e-3) / 1e12, 1)
+        per_matrix.append(row)
+
+    # ---- decode and encode as HBM figures: several GB of distinct buffers inside one event pair, so that the part of
+    # the output still dirty in L2 when the clock stops (at most one L2's worth) is a few per cent of the bytes
+    out_layer = sum(d["N"] * d["K"] * 2.0 for d in dev)
+    secondary = {}
+    if out_layer >= SWEEP_BYTES:      # the step's own sweep is long enough (workload 5)
+        for key, gbs, ms, by in (("decode", dec_gbs, phase_ms["decode"], dec_bytes), ("encode", enc_gbs, phase_ms["encode"], enc_bytes)):
+            secondary[key] = {"bound": "hbm", "achieved": gbs, "peak": P["hbm"], "unit": "GB/s", "frac": gbs / P["hbm"],
+                              "frac_nominal_8TBs": gbs / 8000.0, "bytes": by, "ms": ms, "launches": len(dev),
+                              "how": "the step's own sweep over every matrix of the model (one event pair per phase)"}
+    else:
+        n_sets = int(math.ceil(SWEEP_BYTES / out_layer))
+        what_sets = [[torch.empty_like(d["What"]) for d in dev] for _ in range(n_sets)]
+        in_layer = sum(d["N"] * d["K"] * 4.0 for d in dev)
+        n_w = max(1, int(math.ceil(8 * L2_BYTES / in_layer)))           # copies of W so that re-reads never hit L2
+        w_sets = [[d["W"] if j == 0 else d["W"].clone() for d in dev] for j in range(n_w)]
+        pk_sets = [[(torch.empty_like(d["packed"]), torch.empty_like(d["absmax"])) for d in dev] for _ in range(min(n_sets, 4))]
+
+        def decode_sweep():
+            for ws_ in what_sets:
+                for d, o in zip(dev, ws_):
+                    lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=o)
+
+        def encode_sweep():
+            for j in range(n_sets):
+                for i, d in enumerate(dev):
+                    pk, am = pk_sets[j % len(pk_sets)][i]
+                    lw.lowra_encode(d["layout"], w_sets[j % n_w][i], d["thr"], packed=pk, absmax=am)
+
+        for key, fn, by in (("decode", decode_sweep, dec_bytes), ("encode", encode_sweep, enc_bytes)):
+            fn()
+            torch.cuda.synchronize()
+            best = None
+            for _ in range(3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream); fn(); b.record(stream)
+                torch.cuda.synchronize()
+                ms = a.elapsed_time(b)
+                best = ms if best is None else min(best, ms)
+            gbs = n_sets * by / (best * 1e-3) / 1e9
+            secondary[key] = {"bound": "hbm", "achieved": gbs, "peak": P["hbm"], "unit": "GB/s", "frac": gbs / P["hbm"],
+                              "frac_nominal_8TBs": gbs / 8000.0, "bytes": n_sets * by, "ms": best, "launches": n_sets * len(dev),
+                              "how": f"{n_sets} passes over the step's matrices back to back inside one event pair, every pass "
+                                     f"into its own output buffers ({n_sets * out_layer / 1e9:.1f} GB of distinct decode output; "
+                                     f"encode reads {n_w} cop{'y' if n_w == 1 else 'ies'} of the weights in turn); best of 3"}
+        del what_sets, w_sets, pk_sets
+        # the packed codes in d["packed"] were not touched by the sweeps (they wrote their own buffers)
 
     # dominant kernel: the fused tensor-core kernel (forward + backward launches), timed as whole calls
-    fused_ms = phase_ms["forward"] + phase_ms["backward"]
+    fused_ms = phase_ms["forward"] + (phase_ms["backward"] if with_backward else 0.0)
     achieved = flops_step / (fused_ms * 1e-3) / 1e12
     # denominator: the cuBLAS bf16 figure of the clock regime this run was in - the burst figure while the SM clock
     # stayed at its maximum (a timed region of tens of milliseconds), the sustained one when the power cap held it
@@ -348,220 +473,211 @@ def run_gpu(args):
     sm_now, sm_max = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
     capped = bool(sm_now and sm_max and sm_now < 0.95 * sm_max)
     peak = P["tensor_sustained"] if capped else P["tensor_burst"]
-    roofline = {"bound": "tensor", "kernel": "fused_kernel (forward + backward-input calls" + (", prologue launch included)" if args.deal_per_call else ")"),
+    fused_calls = [(d["N"], d["K"], M) for M in token_counts for d in dev]
+    if with_backward:
+        fused_calls += [(d["K"], d["N"], M) for M in token_counts for d in dev]   # backward reads dY [M, N], writes dX [M, K]
+    roofline = {"bound": "tensor", "kernel": "fused_kernel (forward" + (" + backward-input" if with_backward else "") + " calls" +
+                                              (", prologue launch included)" if args.deal_per_call else ")"),
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                 "peak_burst": P["tensor_burst"], "frac_burst": achieved / P["tensor_burst"],
                 "peak_sustained": P["tensor_sustained"], "frac_sustained": achieved / P["tensor_sustained"],
                 "peak_source": P["source"] + (" (sustained figure: the SM clock was held below its maximum during the timed region)"
                                               if capped else " (burst figure: the SM clock stayed at its maximum during the timed region)"),
-                "traffic": fused_traffic_per_launch(dev, M, r, bits),
+                "traffic": fused_traffic_per_launch(fused_calls, r, bits),
                 "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the gate_proj backward-input launch of "
-                                  "this workload (profiles/fused_backward_input_11008x4096_m4096_streamk.md), scaled by the "
-                                  "input + output bytes of the step's average launch"}
+                                  "workload 3 (profiles/fused_backward_input_11008x4096_m4096_streamk.md), scaled by the "
+                                  "input + output bytes of this step's average launch",
+                "secondary": secondary}
 
-    # ---- end to end: host buffers, pinned, copies inside the timed region
+    # ---- end to end: host buffers, pinned, copies inside the timed region (the first seven matrices of the workload)
     e2e = None
     if not args.no_e2e:
-        host = []
-        for m in mats:
-            host.append(dict(W=pin(m["W"]), thr=pin(m["thr"]), maps=pin(m["maps"]), A=pin(m["A"].view(np.int16)),
-                             B=pin(m["B"].view(np.int16)),
-                             Y=torch.empty((M, m["N"]), dtype=torch.bfloat16).pin_memory(),
-                             dX=torch.empty((M, m["K"]), dtype=torch.bfloat16).pin_memory()))
-        act_host = {k: pin(v.view(np.int16)) for k, v in acts.items()}
-        h2d = sum(h[k].numel() * h[k].element_size() for h in host for k in ("W", "thr", "maps", "A", "B")) \
-            + sum(2 * act_host[d["m"]["K"]].numel() + 2 * act_host[d["m"]["N"]].numel() for d in dev)
-        d2h = sum(h[k].numel() * h[k].element_size() for h in host for k in ("Y", "dX"))
+        e2e = run_e2e(args, lw, torch, dev[:7], token_counts[-1] if args.workload != 5 else 4096, act_dev, token_counts, r, s,
+                      with_backward, stream, barrier, world, len(dev))
+        check_status("after the end-to-end steps")
 
-        # Three streams: uploads, kernels, downloads.  Matrix i + 1 is uploaded while matrix i is computed and
-        # matrix i - 1 is downloaded (the copies of one step are PCIe-bound: 2.1 GB); every buffer has its own
-        # events, so a buffer is never overwritten before its last reader is done, across steps too.
-        s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
-        xs = [torch.empty_like(act_dev[d["m"]["K"]]) for d in dev]      # per-matrix activations / output gradients
-        gs = [torch.empty_like(act_dev[d["m"]["N"]]) for d in dev]
-        ev_in = [torch.cuda.Event() for _ in dev]
-        ev_done = [None] * len(dev)
-        ev_out = [None] * len(dev)
-
-        def e2e_step():
-            for i, (d, h) in enumerate(zip(dev, host)):
-                with torch.cuda.stream(s_in):
-                    if ev_done[i] is not None:
-                        s_in.wait_event(ev_done[i])                      # the previous step's kernels have read them
-                    d["W"].copy_(h["W"], non_blocking=True); d["thr"].copy_(h["thr"], non_blocking=True)
-                    d["maps"].copy_(h["maps"], non_blocking=True)
-                    d["A"].view(torch.int16).copy_(h["A"], non_blocking=True)
-                    d["B"].view(torch.int16).copy_(h["B"], non_blocking=True)
-                    xs[i].view(torch.int16).copy_(act_host[d["m"]["K"]], non_blocking=True)
-                    gs[i].view(torch.int16).copy_(act_host[d["m"]["N"]], non_blocking=True)
-                    ev_in[i].record(s_in)
-                stream.wait_event(ev_in[i])
-                if ev_out[i] is not None:
-                    stream.wait_event(ev_out[i])                         # the previous step's results have left
-                lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"])
-                lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"])
-                lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], xs[i], d["A"], d["B"], s, Y=d["Y"], workspace=d["ws"])
-                lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], gs[i], d["A"], d["B"], s, dX=d["dX"], workspace=d["ws"])
-                ev_done[i] = torch.cuda.Event(); ev_done[i].record(stream)
-                with torch.cuda.stream(s_out):
-                    s_out.wait_event(ev_done[i])
-                    h["Y"].copy_(d["Y"], non_blocking=True); h["dX"].copy_(d["dX"], non_blocking=True)
-                    ev_out[i] = torch.cuda.Event(); ev_out[i].record(s_out)
-
-        def e2e_join():   # the step is over when its last download is
-            for e in ev_out:
-                if e is not None:
-                    stream.wait_event(e)
-
-        e2e_step()
-        e2e_join()
-        barrier()
-        n_e2e = max(1, min(args.steps, 3))
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for _ in range(n_e2e):
-            e2e_step()
-        e2e_join()
-        b.record(stream)
-        barrier()
-        for d in dev:
-            if lw.lowra_device_status(d["ws"]) != 0:
-                raise SystemExit("device status after the end-to-end steps")
-        ms = a.elapsed_time(b) / n_e2e
-        ms = max_over_ranks(ms, world)
-        e2e = {"value": aggregate_tflops(flops_step, world, ms), "unit": UNIT, "ms_per_step": ms,
-               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e,
-               "note": "uploads, kernels and downloads on three streams: a matrix is computed while the next one "
-                       "arrives and the previous one leaves"}
-
-    # ---- outside the step: the codebook learner (the stage before encode), timed on the layer's seven matrices
+    # ---- outside the step: learner, adapter gradients, quantisation error on (at most) the first seven matrices
     extras = None
-    if rank == 0:
-        y0 = np.zeros((3, 16)); t0 = np.zeros((3, 16))        # stand-in starting tables: equally spaced levels
-        for c, b in enumerate((1, 2, 4)):
-            lv = np.linspace(-1.0, 1.0, 1 << b)
-            y0[c, :lv.size] = lv
-            t0[c, :lv.size - 1] = 0.5 * (lv[:-1] + lv[1:])
-        T_learn = 10
-        torch.cuda.synchronize()
-        for d in dev:   # warm-up
-            lw.lowra_learn_codebooks(d["layout"], d["W"], y0, t0, T_learn, maps=d["maps"], thresholds=d["thr"])
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for d in dev:
-            lw.lowra_learn_codebooks(d["layout"], d["W"], y0, t0, T_learn, maps=d["maps"], thresholds=d["thr"])
-        b.record(stream)
-        torch.cuda.synchronize()
-        ms_learn = a.elapsed_time(b)
-        extras = {"learn_codebooks": {"ms": ms_learn, "iterations": T_learn, "GB/s": 4.0 * elems / (ms_learn * 1e-3) / 1e9,
-                                      "frac_hbm": 4.0 * elems / (ms_learn * 1e-3) / 1e9 / P["hbm"],
-                                      "element_passes_per_s": elems * T_learn / (ms_learn * 1e-3),
-                                      "note": "not part of the step; algorithmic bytes = one read of W (4 B per element)"}}
-        # the same for all three precisions of every row in one pass (what the precision assigner starts from)
-        tabs3 = [(torch.empty((3, d["m"]["N"], 16), dtype=torch.float32, device="cuda"),
-                  torch.empty((3, d["m"]["N"], 16), dtype=torch.float32, device="cuda")) for d in dev]
-        for d, (m3, h3) in zip(dev, tabs3):
-            lw.lowra_learn_codebooks_all(d["W"], y0, t0, T_learn, maps3=m3, thresholds3=h3)
-        a.record(stream)
-        for d, (m3, h3) in zip(dev, tabs3):
-            lw.lowra_learn_codebooks_all(d["W"], y0, t0, T_learn, maps3=m3, thresholds3=h3)
-        b.record(stream)
-        torch.cuda.synchronize()
-        ms_learn3 = a.elapsed_time(b)
-        extras["learn_codebooks_all_precisions"] = {
-            "ms": ms_learn3, "iterations": T_learn, "element_passes_per_s": 3 * elems * T_learn / (ms_learn3 * 1e-3),
-            "note": "not part of the step; every row at 1, 2 and 4 bits from one read of W"}
-        del tabs3
-
-        # the gradients of the low-rank factors (the other half of a training step's backward pass)
-        ws_ad = torch.empty(lw.lowra_adapter_workspace_bytes(M, r), dtype=torch.uint8, device="cuda")
-        grads = [(torch.empty_like(d["A"]), torch.empty_like(d["B"])) for d in dev]
-
-        def adapters():
-            for d, (gA, gB) in zip(dev, grads):
-                lw.lowra_lora_backward_adapters(act_dev[d["m"]["K"]], act_dev[d["m"]["N"]], d["A"], d["B"], s,
-                                                dA=gA, dB=gB, workspace=ws_ad)
-        adapters()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        adapters()
-        b.record(stream)
-        torch.cuda.synchronize()
-        if lw.lowra_device_status(ws_ad) != 0:
-            raise SystemExit("device status after the adapter gradients")
-        ms_ad = a.elapsed_time(b)
-        ad_bytes = sum(2.0 * M * (d["m"]["K"] + d["m"]["N"]) for d in dev)      # X and dY once, bf16
-        ad_flops = sum(4.0 * M * r * (d["m"]["K"] + d["m"]["N"]) for d in dev)
-        extras["adapter_gradients"] = {"ms": ms_ad, "GB/s": ad_bytes / (ms_ad * 1e-3) / 1e9,
-                                       "frac_hbm": ad_bytes / (ms_ad * 1e-3) / 1e9 / P["hbm"],
-                                       "TFLOP/s": ad_flops / (ms_ad * 1e-3) / 1e12, "launches": 5 * len(dev),
-                                       "note": "not part of the step; algorithmic bytes = X and dY read once"}
-
-        # per-channel quantisation error (the precision assigner's input) and the residual W - W_hat
-        sse = [torch.empty(d["m"]["N"], dtype=torch.float64, device="cuda") for d in dev]
-        res = torch.empty(max(d["m"]["N"] * d["m"]["K"] for d in dev), dtype=torch.float32, device="cuda")
-        qe = {}
-        for key, with_res in (("sse_only", False), ("with_residual", True)):
-            def errors():
-                for d, e in zip(dev, sse):
-                    lw.lowra_quant_error(d["layout"], d["W"], d["maps"], d["thr"], sse=e,
-                                         residual=res[:d["m"]["N"] * d["m"]["K"]].view(d["m"]["N"], d["m"]["K"]) if with_res else None)
-            errors()
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream)
-            errors()
-            b.record(stream)
-            torch.cuda.synchronize()
-            ms_q = a.elapsed_time(b)
-            by = (8.0 if with_res else 4.0) * elems
-            qe[key] = {"ms": ms_q, "GB/s": by / (ms_q * 1e-3) / 1e9, "frac_hbm": by / (ms_q * 1e-3) / 1e9 / P["hbm"]}
-        # every channel under 1, 2 and 4 bits in one pass (stand-in tables for all three precisions)
-        t3 = []
-        for d in dev:
-            m3 = np.zeros((3, d["m"]["N"], 16), dtype=np.float32); h3 = np.zeros_like(m3)
-            for c, b in enumerate((1, 2, 4)):
-                m3[c], h3[c] = si.standin_codebooks(np.full(d["m"]["N"], b, dtype=np.uint8))
-            t3.append((torch.from_numpy(m3).cuda(), torch.from_numpy(h3).cuda(),
-                       torch.empty((d["m"]["N"], 3), dtype=torch.float64, device="cuda")))
-
-        def errors3():
-            for d, (m3, h3, o3) in zip(dev, t3):
-                lw.lowra_channel_errors(d["W"], m3, h3, sse3=o3)
-        errors3()
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        errors3()
-        b.record(stream)
-        torch.cuda.synchronize()
-        ms_q = a.elapsed_time(b)
-        qe["three_precisions_one_pass"] = {"ms": ms_q, "GB/s": 4.0 * elems / (ms_q * 1e-3) / 1e9,
-                                           "frac_hbm": 4.0 * elems / (ms_q * 1e-3) / 1e9 / P["hbm"]}
-        qe["note"] = "not part of the step; algorithmic bytes = W read once (4 B per element) + residual written (4 B)"
-        extras["quant_error"] = qe
+    if rank == 0 and not args.no_extras:
+        extras = run_extras(lw, torch, dev[:7], token_counts[0] if args.workload != 5 else 4096, act_dev, r, s, stream, P, y0, t0)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu:
-        cpu = cpu_baseline_sample()
+        cpu = cpu_baseline_sample(args.workload, gpu=dict(lw=lw, torch=torch, d=dev[0], act=act_dev, M=token_counts[0], r=r, s=s,
+                                                          with_backward=with_backward))
 
     if rank == 0:
+        n_fused = len(fused_calls)
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"config {WORKLOAD}: {cfg.name}, 7 matrices, {M} tokens, rank {r}, "
-                                   f"mix {cfg.mix} (avg {bits:.2f} bits), stand-in codebooks",
-                       "elements": elems, "l2": "inputs larger than L2 (about 2.7 GB touched per step)",
+            "config": {"workload": f"config {args.workload}: {cfg.name}, {len(dev)} matrices, tokens {token_counts}, rank {r}, "
+                                   f"mix {cfg.mix} (avg {bits:.2f} bits), codebooks learnt on the GPU "
+                                   f"({LLOYD_ITERS} rounds of weighted Lloyd-Max per row from the Appendix-F tables)",
+                       "elements": elems,
+                       "l2": f"inputs larger than L2 ({(elems * 4 + out_layer) / 1e9:.1f} GB of weights read and written per step)",
                        "row_deal": "in every call (prologue launch)" if args.deal_per_call else
-                                   "once per weight (lowra_deal_build), outside the step like the storage plan"},
-            "phases": phases, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "extras": extras,
-            "gpu_launches": args.steps * len(dev) * (6 if args.deal_per_call else 4), "clocks": clocks,
+                                   "once per weight (lowra_deal_build), outside the step like the storage plan",
+                       "host_generation_s": round(t_gen, 1)},
+            "phases": phases, "per_matrix": per_matrix, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "extras": extras,
+            "gpu_launches": args.steps * (2 * len(dev) + n_fused * (2 if args.deal_per_call else 1)), "clocks": clocks,
         }
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_e2e(args, lw, torch, dev, M, act_dev, token_counts, r, s, with_backward, stream, barrier, world, n_all):
+    """The same calls with HOST buffers: every step uploads the step's inputs from pinned memory and downloads its
+    results.  Three streams: uploads, kernels, downloads - matrix i + 1 arrives while matrix i is computed and matrix
+    i - 1 leaves; every buffer has its own events, so none is overwritten before its last reader is done."""
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    if M not in token_counts:
+        M = token_counts[0]
+    host = []
+    for d in dev:
+        m = d["host"]
+        h = dict(W=pin(m["W"]), thr=d["thr"].cpu().pin_memory(), maps=d["maps"].cpu().pin_memory(),
+                 A=pin(m["A"].view(np.int16)), B=pin(m["B"].view(np.int16)),
+                 Y=torch.empty((M, d["N"]), dtype=torch.bfloat16).pin_memory())
+        if with_backward:
+            h["dX"] = torch.empty((M, d["K"]), dtype=torch.bfloat16).pin_memory()
+        host.append(h)
+    act_host = {k: act_dev[(M, k)].view(torch.int16).cpu().pin_memory() for k in sorted({w for d in dev for w in (d["N"], d["K"])})}
+    nbytes = lambda t: t.numel() * t.element_size()
+    h2d = sum(nbytes(h[k]) for h in host for k in ("W", "thr", "maps", "A", "B")) \
+        + sum(nbytes(act_host[d["K"]]) + (nbytes(act_host[d["N"]]) if with_backward else 0) for d in dev)
+    d2h = sum(nbytes(h[k]) for h in host for k in ("Y", "dX") if k in h)
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    xs = [torch.empty_like(act_dev[(M, d["K"])]) for d in dev]      # per-matrix activations / output gradients
+    gs = [torch.empty_like(act_dev[(M, d["N"])]) for d in dev] if with_backward else None
+    Ys = [torch.empty((M, d["N"]), dtype=torch.bfloat16, device="cuda") for d in dev]
+    dXs = [torch.empty((M, d["K"]), dtype=torch.bfloat16, device="cuda") for d in dev] if with_backward else None
+    ev_in = [torch.cuda.Event() for _ in dev]
+    ev_done = [None] * len(dev)
+    ev_out = [None] * len(dev)
+
+    def e2e_step():
+        for i, (d, h) in enumerate(zip(dev, host)):
+            with torch.cuda.stream(s_in):
+                if ev_done[i] is not None:
+                    s_in.wait_event(ev_done[i])                      # the previous step's kernels have read them
+                d["W"].copy_(h["W"], non_blocking=True); d["thr"].copy_(h["thr"], non_blocking=True)
+                d["maps"].copy_(h["maps"], non_blocking=True)
+                d["A"].view(torch.int16).copy_(h["A"], non_blocking=True)
+                d["B"].view(torch.int16).copy_(h["B"], non_blocking=True)
+                xs[i].view(torch.int16).copy_(act_host[d["K"]], non_blocking=True)
+                if with_backward:
+                    gs[i].view(torch.int16).copy_(act_host[d["N"]], non_blocking=True)
+                ev_in[i].record(s_in)
+            stream.wait_event(ev_in[i])
+            if ev_out[i] is not None:
+                stream.wait_event(ev_out[i])                         # the previous step's results have left
+            lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"])
+            lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"])
+            lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], xs[i], d["A"], d["B"], s, Y=Ys[i], workspace=d["ws"][M])
+            if with_backward:
+                lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], gs[i], d["A"], d["B"], s, dX=dXs[i],
+                                             workspace=d["ws"][M])
+            ev_done[i] = torch.cuda.Event(); ev_done[i].record(stream)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_done[i])
+                h["Y"].copy_(Ys[i], non_blocking=True)
+                if with_backward:
+                    h["dX"].copy_(dXs[i], non_blocking=True)
+                ev_out[i] = torch.cuda.Event(); ev_out[i].record(s_out)
+
+    def e2e_join():   # the step is over when its last download is
+        for e in ev_out:
+            if e is not None:
+                stream.wait_event(e)
+
+    e2e_step()
+    e2e_join()
+    barrier()
+    n_e2e = max(1, args.steps)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for _ in range(n_e2e):
+        e2e_step()
+    e2e_join()
+    b.record(stream)
+    barrier()
+    ms = a.elapsed_time(b) / n_e2e
+    ms = max_over_ranks(ms, world)
+    flops = (2 if with_backward else 1) * sum(gemm_flops(M, d["N"], d["K"], r) for d in dev)
+    note = ("uploads, kernels and downloads on three streams: a matrix is computed while the next one arrives and the "
+            "previous one leaves")
+    if len(dev) < n_all or len(token_counts) > 1:
+        note += f"; bounded sample of the workload: its first {len(dev)} matrices at {M} tokens"
+    return {"value": aggregate_tflops(flops, world, ms), "unit": UNIT, "ms_per_step": ms,
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": n_e2e, "note": note}
+
+
+def run_extras(lw, torch, dev, M, act_dev, r, s, stream, P, y0, t0):
+    """Kernels around the step, timed on the same matrices: the codebook learner (the stage before encode), the
+    gradients of the low-rank factors, the per-channel quantisation error."""
+    if (M, dev[0]["K"]) not in act_dev:
+        M = sorted({k[0] for k in act_dev})[0]
+    elems = sum(d["N"] * d["K"] for d in dev)
+
+    def timed(fn):
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream); fn(); b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b)
+
+    extras = {"matrices": len(dev), "tokens": M}
+    tabs = [(torch.empty_like(d["maps"]), torch.empty_like(d["thr"])) for d in dev]
+    ms = timed(lambda: [lw.lowra_learn_codebooks(d["layout"], d["W"], y0, t0, LLOYD_ITERS, maps=mp, thresholds=th)
+                        for d, (mp, th) in zip(dev, tabs)])
+    extras["learn_codebooks"] = {"ms": ms, "iterations": LLOYD_ITERS, "GB/s": 4.0 * elems / (ms * 1e-3) / 1e9,
+                                 "frac_hbm": 4.0 * elems / (ms * 1e-3) / 1e9 / P["hbm"],
+                                 "element_passes_per_s": elems * LLOYD_ITERS / (ms * 1e-3),
+                                 "note": "not part of the step; from the Appendix-F starting tables; algorithmic bytes = one read of W (4 B per element)"}
+    # the same for all three precisions of every row in one pass (what the precision assigner starts from)
+    tabs3 = [(torch.empty((3, d["N"], 16), dtype=torch.float32, device="cuda"),
+              torch.empty((3, d["N"], 16), dtype=torch.float32, device="cuda")) for d in dev]
+    ms = timed(lambda: [lw.lowra_learn_codebooks_all(d["W"], y0, t0, LLOYD_ITERS, maps3=m3, thresholds3=h3)
+                        for d, (m3, h3) in zip(dev, tabs3)])
+    extras["learn_codebooks_all_precisions"] = {
+        "ms": ms, "iterations": LLOYD_ITERS, "element_passes_per_s": 3 * elems * LLOYD_ITERS / (ms * 1e-3),
+        "note": "not part of the step; every row at 1, 2 and 4 bits from one read of W"}
+
+    # the gradients of the low-rank factors (the other half of a training step's backward pass)
+    ws_ad = torch.empty(lw.lowra_adapter_workspace_bytes(M, r), dtype=torch.uint8, device="cuda")
+    grads = [(torch.empty_like(d["A"]), torch.empty_like(d["B"])) for d in dev]
+    ms = timed(lambda: [lw.lowra_lora_backward_adapters(act_dev[(M, d["K"])], act_dev[(M, d["N"])], d["A"], d["B"], s,
+                                                        dA=gA, dB=gB, workspace=ws_ad) for d, (gA, gB) in zip(dev, grads)])
+    if lw.lowra_device_status(ws_ad) != 0:
+        raise SystemExit("device status after the adapter gradients")
+    ad_bytes = sum(2.0 * M * (d["K"] + d["N"]) for d in dev)      # X and dY once, bf16
+    ad_flops = sum(4.0 * M * r * (d["K"] + d["N"]) for d in dev)
+    extras["adapter_gradients"] = {"ms": ms, "GB/s": ad_bytes / (ms * 1e-3) / 1e9, "frac_hbm": ad_bytes / (ms * 1e-3) / 1e9 / P["hbm"],
+                                   "TFLOP/s": ad_flops / (ms * 1e-3) / 1e12,
+                                   "note": "not part of the step; algorithmic bytes = X and dY read once"}
+
+    # per-channel quantisation error (the precision assigner's input) and the residual W - W_hat
+    sse = [torch.empty(d["N"], dtype=torch.float64, device="cuda") for d in dev]
+    res = torch.empty(max(d["N"] * d["K"] for d in dev), dtype=torch.float32, device="cuda")
+    qe = {}
+    for key, with_res in (("sse_only", False), ("with_residual", True)):
+        ms = timed(lambda: [lw.lowra_quant_error(d["layout"], d["W"], d["maps"], d["thr"], sse=e,
+                                                 residual=res[:d["N"] * d["K"]].view(d["N"], d["K"]) if with_res else None)
+                            for d, e in zip(dev, sse)])
+        by = (8.0 if with_res else 4.0) * elems
+        qe[key] = {"ms": ms, "GB/s": by / (ms * 1e-3) / 1e9, "frac_hbm": by / (ms * 1e-3) / 1e9 / P["hbm"]}
+    # every channel under 1, 2 and 4 bits in one pass, with the tables learnt above
+    out3 = [torch.empty((d["N"], 3), dtype=torch.float64, device="cuda") for d in dev]
+    ms = timed(lambda: [lw.lowra_channel_errors(d["W"], m3, h3, sse3=o3) for d, (m3, h3), o3 in zip(dev, tabs3, out3)])
+    qe["three_precisions_one_pass"] = {"ms": ms, "GB/s": 4.0 * elems / (ms * 1e-3) / 1e9,
+                                       "frac_hbm": 4.0 * elems / (ms * 1e-3) / 1e9 / P["hbm"]}
+    qe["note"] = "not part of the step; algorithmic bytes = W read once (4 B per element) + residual written (4 B)"
+    extras["quant_error"] = qe
+    return extras
 
 
 # --------------------------------------------------------------------------------------------------
@@ -570,47 +686,131 @@ def run_gpu(args):
 SAMPLE_TOKENS = 512
 
 
-def oracle_sample_step(problem):
-    """The oracle on the bounded sample: q_proj-shaped matrix, encode + decode in full, forward +
-    backward-input on SAMPLE_TOKENS token rows.  Returns per-phase seconds."""
+def oracle_sample_step(problem, with_backward=True, keep=None):
+    """The oracle on the bounded sample: one matrix of the workload, its own codebooks (the learner is input
+    generation and is not timed), encode + decode in full, forward (+ backward-input) on SAMPLE_TOKENS token rows.
+    Returns per-phase seconds; `keep` (a dict) receives the results."""
     import oracle
     W, precs, maps, thr, X, dY, A, B, s = problem
     K = W.shape[1]
     t = {}
     t0 = time.time(); packed, a = oracle.encode(W, precs, thr); t["encode"] = time.time() - t0
     t0 = time.time(); what = oracle.decode(packed, a, maps, precs, K); t["decode"] = time.time() - t0
-    t0 = time.time(); oracle.lora_forward(what, X, A, B, s); t["forward"] = time.time() - t0
-    t0 = time.time(); oracle.lora_backward_input(what, dY, A, B, s); t["backward"] = time.time() - t0
+    t0 = time.time(); Y = oracle.lora_forward(what, X, A, B, s); t["forward"] = time.time() - t0
+    dX = None
+    if with_backward:
+        t0 = time.time(); dX = oracle.lora_backward_input(what, dY, A, B, s); t["backward"] = time.time() - t0
+    if keep is not None:
+        keep.update(packed=packed, absmax=a, what=what, Y=Y, dX=dX)
     return t
 
 
-def make_sample_problem():
-    cfg = si.config(WORKLOAD)
-    mat = cfg.matrices[0]
-    W = si.weights(mat.N, mat.K, matrix_id=mat.matrix_id)
-    precs = si.precisions(mat.N, cfg.mix, matrix_id=mat.matrix_id)
-    maps, thr = si.standin_codebooks(precs, matrix_id=mat.matrix_id)
-    X = si.activations(SAMPLE_TOKENS, mat.K, matrix_id=100)
-    dY = si.activations(SAMPLE_TOKENS, mat.N, matrix_id=101)
-    A, B = si.lora_factors(mat.K, mat.N, cfg.rank, matrix_id=mat.matrix_id)
-    return (W, precs, maps, thr, X, dY, A, B, cfg.s), mat, cfg
+def sample_rows(M):
+    """SAMPLE_TOKENS token rows spread over the M tokens of the step (every tile of 256 tokens is hit)."""
+    return np.unique(np.linspace(0, M - 1, min(SAMPLE_TOKENS, M)).astype(np.int64))
 
 
-def cpu_baseline_sample(reps: int = 3):
+def make_sample_problem(workload):
     import oracle
-    problem, mat, cfg = make_sample_problem()
-    oracle_sample_step(problem)  # warm
-    ts = [oracle_sample_step(problem) for _ in range(reps)]
+    cfg, mats = workload_matrices(workload)
+    mat = mats[0]
+    M = cfg.tokens[0]
+    W = si.weights(mat.N, mat.K, matrix_id=mat.matrix_id, kind=cfg.weight_kind)
+    precs = si.precisions(mat.N, cfg.mix, matrix_id=mat.matrix_id)
+    maps, thr = oracle.lloyd_max(W, precs, T=LLOYD_ITERS)
+    rows = sample_rows(M)
+    X = si.activations(M, mat.K, matrix_id=100)[rows]
+    dY = si.activations(M, mat.N, matrix_id=100)[rows]
+    A, B = si.lora_factors(mat.K, mat.N, cfg.rank, matrix_id=mat.matrix_id % 7)
+    return (W, precs, maps, thr, X, dY, A, B, cfg.s), mat, cfg, rows
+
+
+def cpu_baseline_sample(workload, reps: int = 2, gpu=None):
+    """Times the oracle, as it stands, on a bounded sample of the workload (its first matrix: encode + decode in
+    full, the products on SAMPLE_TOKENS token rows), on all host cores and on one.  With `gpu` (the benchmark's
+    device-resident first matrix) the oracle's results of the sample are also held against what the GPU path - its
+    own learner, encode, decode and fused products, in the launch configuration that was timed - gives for the same
+    matrix and token rows; a mismatch ends the run."""
+    import oracle
+    problem, mat, cfg, rows = make_sample_problem(workload)
+    with_backward = "backward" in cfg.ops
+    keep = {}
+    oracle_sample_step(problem, with_backward, keep)  # warm; its results serve the check below
+    ts = [oracle_sample_step(problem, with_backward) for _ in range(reps)]
     tot = min(sum(t.values()) for t in ts)
     best = min(ts, key=lambda t: sum(t.values()))
-    flops = 2 * gemm_flops(SAMPLE_TOKENS, mat.N, mat.K, cfg.rank)
+    n_rows = len(rows)
+    flops = (2 if with_backward else 1) * gemm_flops(n_rows, mat.N, mat.K, cfg.rank)
     el = mat.N * mat.K
-    return {"value": flops / tot / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-            "sample": f"{mat.name} {mat.N}x{mat.K}: oracle encode + decode in full, forward + backward-input on "
-                      f"{SAMPLE_TOKENS} of {cfg.tokens[0]} token rows (fp64); same value definition as the GPU arm",
-            "seconds_per_sample_step": tot,
-            "encode_ns_per_element": best["encode"] / el * 1e9, "decode_ns_per_element": best["decode"] / el * 1e9,
-            "gemm_fp64_gflops": flops / (best["forward"] + best["backward"]) / 1e9}
+    gemm_s = best["forward"] + best.get("backward", 0.0)
+    out = {"value": flops / tot / 1e12, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+           "sample": f"{mat.name} {mat.N}x{mat.K}: oracle encode + decode in full, forward" + (" + backward-input" if with_backward else "") +
+                     f" on {n_rows} of {cfg.tokens[0]} token rows (fp64); same value definition as the GPU arm",
+           "seconds_per_sample_step": tot,
+           "encode_ns_per_element": best["encode"] / el * 1e9, "decode_ns_per_element": best["decode"] / el * 1e9,
+           "gemm_fp64_gflops": flops / gemm_s / 1e9}
+    # one thread: encode + decode on the first 512 rows of the matrix, the forward product on 32 token rows
+    n_all = oracle.num_threads()
+    oracle.set_threads(1)
+    try:
+        import threadpoolctl
+        limiter = threadpoolctl.threadpool_limits(limits=1)
+    except Exception:
+        limiter = None
+    try:
+        W, precs, maps, thr, X, dY, A, B, s = problem
+        sub = slice(0, min(512, mat.N))
+        t0 = time.time(); pk, am = oracle.encode(W[sub], precs[sub], thr[sub]); t_e = time.time() - t0
+        t0 = time.time(); wh = oracle.decode(pk, am, maps[sub], precs[sub], mat.K); t_d = time.time() - t0
+        t0 = time.time(); oracle.lora_forward(keep["what"], X[:32], A, B, s); t_f = time.time() - t0
+        el1 = W[sub].size
+        out["one_thread"] = {"encode_ns_per_element": t_e / el1 * 1e9, "decode_ns_per_element": t_d / el1 * 1e9,
+                             "gemm_fp64_gflops": gemm_flops(32, mat.N, mat.K, cfg.rank) / t_f / 1e9,
+                             "sample": f"encode + decode of {sub.stop} rows, forward on 32 token rows"}
+    finally:
+        oracle.set_threads(n_all)
+        if limiter is not None:
+            limiter.restore_original_limits()
+
+    if gpu is not None:
+        lw, torch, d, M = gpu["lw"], gpu["torch"], gpu["d"], gpu["M"]
+        bits16 = lambda t: t.view(torch.int16).cpu().numpy().view(np.uint16)
+        idx = torch.from_numpy(rows).cuda()
+        # the step's own calls, once more, on the step's own buffers (same layout, deal, workspace and token count)
+        lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"])
+        lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"])
+        Y = lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], gpu["act"][(M, d["K"])], d["A"], d["B"],
+                                  gpu["s"], Y=d["Y"][M], workspace=d["ws"][M])
+        got = {"forward": si.bf16_bits_to_f32(bits16(Y[idx])).astype(np.float64)}
+        ref = {"forward": keep["Y"]}
+        if gpu["with_backward"]:
+            dX = lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], gpu["act"][(M, d["N"])], d["A"], d["B"],
+                                              gpu["s"], dX=d["dX"][M], workspace=d["ws"][M])
+            got["backward_input"] = si.bf16_bits_to_f32(bits16(dX[idx])).astype(np.float64)
+            ref["backward_input"] = keep["dX"]
+        if lw.lowra_device_status(d["ws"][M]) != 0:
+            raise SystemExit("device status during the check against the oracle")
+        chk = {}
+        # tables: the GPU learner's levels against the oracle's (equal or one ulp apart); codes and decoded weights:
+        # identical wherever the tables are
+        maps_gpu = d["maps"].cpu().numpy()
+        chk["codebook_entries_identical"] = float((maps_gpu == problem[2]).mean())
+        chk["packed_bytes_identical"] = float((d["packed"].cpu().numpy()[:d["layout"].packed_bytes] == keep["packed"]).mean())
+        chk["decoded_elements_identical"] = float((bits16(d["What"]) == keep["what"]).mean())
+        ok = chk["codebook_entries_identical"] >= 0.99 and chk["packed_bytes_identical"] >= 0.999 and chk["decoded_elements_identical"] >= 0.999
+        for k in got:
+            dlt = got[k] - ref[k]
+            emax = float(np.abs(dlt).max() / np.abs(ref[k]).max())
+            efro = float(np.linalg.norm(dlt) / np.linalg.norm(ref[k]))
+            chk[k] = {"max_rel": emax, "fro_rel": efro}
+            ok = ok and emax <= 1e-2 and efro <= 5e-3
+        chk["ok"] = bool(ok)
+        chk["what"] = (f"GPU path of the timed configuration (own learner, encode, decode, fused products) against the oracle's own "
+                       f"pipeline on {mat.name}, {n_rows} token rows; bounds: max 1e-2, Frobenius 5e-3")
+        out["check_against_oracle"] = chk
+        if not ok:
+            raise SystemExit("the GPU results of the timed configuration disagree with the oracle: " + json.dumps(chk))
+    return out
 
 
 def run_reference(args):
@@ -618,25 +818,126 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    problem, mat, cfg = make_sample_problem()
+    problem, mat, cfg, rows = make_sample_problem(args.workload)
+    with_backward = "backward" in cfg.ops
     for _ in range(min(args.warmup, 1)):
-        oracle_sample_step(problem)
+        oracle_sample_step(problem, with_backward)
     t0 = time.time()
     for _ in range(args.steps):
-        oracle_sample_step(problem)
+        oracle_sample_step(problem, with_backward)
     dt = (time.time() - t0) / args.steps
-    flops = 2 * gemm_flops(SAMPLE_TOKENS, mat.N, mat.K, cfg.rank)
+    flops = (2 if with_backward else 1) * gemm_flops(len(rows), mat.N, mat.K, cfg.rank)
     value = flops / dt / 1e12
-    sample = (f"each step = the CPU oracle on {mat.name} {mat.N}x{mat.K}: encode + decode in full, forward + "
-              f"backward-input on {SAMPLE_TOKENS} of {cfg.tokens[0]} token rows (fp64)")
+    sample = (f"each step = the CPU oracle on {mat.name} {mat.N}x{mat.K}: encode + decode in full, forward" +
+              (" + backward-input" if with_backward else "") + f" on {len(rows)} of {cfg.tokens[0]} token rows (fp64)")
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
            "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": min(args.warmup, 1),
            "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
            "dtype": "f64", "data": "synthetic",
-           "config": {"workload": f"config {WORKLOAD}: {cfg.name} (bounded sample: {sample})"},
+           "config": {"workload": f"config {args.workload}: {cfg.name} (bounded sample: {sample})"},
            "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(out))
+
+
+# --------------------------------------------------------------------------------------------------
+# small single-kernel cases for profiler captures (a few hundred MB on the device, three launches each)
+# --------------------------------------------------------------------------------------------------
+CASES = ("forward", "backward", "forward4096", "backward_gate", "forward_4bit", "backward_4bit", "forward_1bit", "backward_1bit",
+         "codec", "decode_layer", "learn", "adapters", "errors")
+
+
+def run_case(case: str) -> None:
+    """forward / backward: fused calls, N = K = 4096, 2048 tokens, rank 64 (config-3 mix; *_4bit, *_1bit: every row
+    at that precision); forward4096: 4096 tokens (264 pieces: tiles cut between SMs, partial tiles preloaded);
+    backward_gate: 11008 x 4096 at 4096 tokens (last row of tiles cut); codec: decode + encode of an 11008 x 4096
+    matrix; decode_layer: the seven decodes of a Llama-7B layer back to back; learn: codebook learner, 4096 x 4096,
+    10 rounds; adapters: gradients of the low-rank factors, 4096 x 11008, 4096 tokens; errors: per-channel
+    quantisation error with and without the residual, 11008 x 4096."""
+    import torch
+
+    import paper_2502_08141_b200 as lw
+
+    cfg = si.config(3)
+    r, s = cfg.rank, cfg.s
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    if case == "adapters":
+        N, K, M = 11008, 4096, 4096
+        X = torch.randn(M, K, device="cuda", generator=gen).bfloat16()
+        dY = torch.randn(M, N, device="cuda", generator=gen).bfloat16()
+        A = (torch.randn(K, r, device="cuda", generator=gen) * 0.01).bfloat16()
+        B = (torch.randn(r, N, device="cuda", generator=gen) * 0.01).bfloat16()
+        ws = torch.empty(lw.lowra_adapter_workspace_bytes(M, r), dtype=torch.uint8, device="cuda")
+        for _ in range(3):
+            lw.lowra_lora_backward_adapters(X, dY, A, B, s, workspace=ws)
+        status = lw.lowra_device_status(ws)
+        print("adapters status", status)
+        if status != 0:
+            raise SystemExit(1)
+        return
+    if case == "decode_layer":
+        mats = []
+        for mat in cfg.matrices:
+            precs = si.precisions(mat.N, cfg.mix, matrix_id=mat.matrix_id)
+            maps, thr = si.standin_codebooks(precs, matrix_id=mat.matrix_id)
+            layout = lw.Layout(precs, mat.K)
+            W = torch.randn(mat.N, mat.K, device="cuda", generator=gen) * 0.02
+            packed, absmax = lw.lowra_encode(layout, W, torch.from_numpy(thr).cuda())
+            mats.append((layout, packed, absmax, torch.from_numpy(maps).cuda(),
+                         torch.empty(mat.N, mat.K, dtype=torch.bfloat16, device="cuda")))
+            del W
+        for _ in range(2):
+            for layout, packed, absmax, maps_d, out in mats:
+                lw.lowra_decode(layout, packed, absmax, maps_d, out=out)
+        torch.cuda.synchronize()
+        print("decode_layer ok")
+        return
+    mix = {4: 1.0} if case.endswith("_4bit") else {1: 1.0} if case.endswith("_1bit") else cfg.mix
+    base = case.split("_")[0] if case.endswith("bit") else case
+    N, K = (11008, 4096) if base in ("codec", "errors", "backward_gate") else (4096, 4096)
+    M = 4096 if base in ("forward4096", "backward_gate") else 2048
+    precs = si.precisions(N, mix)
+    maps, thr = si.standin_codebooks(precs)
+    layout = lw.Layout(precs, K)
+    W = torch.randn(N, K, device="cuda", generator=gen) * 0.02
+    maps_d, thr_d = torch.from_numpy(maps).cuda(), torch.from_numpy(thr).cuda()
+    if base == "learn":
+        y0, t0 = si.initial_codebooks()
+        for _ in range(3):
+            lw.lowra_learn_codebooks(layout, W, y0, t0, LLOYD_ITERS)
+        torch.cuda.synchronize()
+        print("learn ok")
+        return
+    if base == "errors":
+        sse = torch.empty(N, dtype=torch.float64, device="cuda")
+        res = torch.empty(N, K, dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            lw.lowra_quant_error(layout, W, maps_d, thr_d, sse=sse, residual=res)
+            lw.lowra_quant_error(layout, W, maps_d, thr_d, sse=sse)
+        torch.cuda.synchronize()
+        print("errors ok")
+        return
+    packed, absmax = lw.lowra_encode(layout, W, thr_d)
+    if base == "codec":
+        out = torch.empty(N, K, dtype=torch.bfloat16, device="cuda")
+        for _ in range(3):
+            lw.lowra_decode(layout, packed, absmax, maps_d, out=out)
+            lw.lowra_encode(layout, W, thr_d, packed=packed, absmax=absmax)
+        torch.cuda.synchronize()
+        print("codec ok")
+        return
+    fwd = base in ("forward", "forward4096")
+    act = torch.randn(M, K if fwd else N, device="cuda", generator=gen).bfloat16()
+    A = (torch.randn(K, r, device="cuda", generator=gen) * 0.01).bfloat16()
+    B = (torch.randn(r, N, device="cuda", generator=gen) * 0.01).bfloat16()
+    ws = torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda")
+    fn = lw.lowra_lora_forward if fwd else lw.lowra_lora_backward_input
+    for _ in range(3):
+        fn(layout, packed, absmax, maps_d, act, A, B, s, workspace=ws)
+    status = lw.lowra_device_status(ws)
+    print(case, "status", status)
+    if status != 0:
+        raise SystemExit(1)
 
 
 def main():
@@ -645,12 +946,17 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=3, choices=[2, 3, 4, 5])
+    ap.add_argument("--case", default=None, choices=CASES, help="run one small single-kernel case (for a profiler) and exit")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--deal-per-call", action="store_true",
                     help="fused calls work out the row deal in a prologue launch of their own (no lowra_deal_build)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.case is not None:
+        run_case(args.case)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

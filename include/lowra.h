@@ -250,6 +250,15 @@ lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, const uint16_t*
 lowra_status lowra_device_status(const void* workspace_dev, void* stream);
 
 /*
+ * (No counterpart in the paper.)  Every wait inside the tensor-core kernels - on a shared-memory barrier, on a
+ * flag another SM raises - gives up after this long; the kernel then records LOWRA_ERR_TIMEOUT in the status
+ * word, lets what it has in flight land, releases its resources and returns (the output of that call is not
+ * valid; the GPU and the workspace stay usable).  Process-wide, read when a call is made; 1 s unless changed.
+ *   nanoseconds: 1000 .. 10^10, or 0 for the default.  Errors: outside that range -> LOWRA_ERR_SHAPE.
+ */
+lowra_status lowra_set_wait_limit(uint64_t nanoseconds);
+
+/*
  * (No counterpart in the paper: this is a packaging variant of lowra_lora_forward.)
  *
  * lowra_lora_forward for callers that cannot hand over scratch memory.  Some hosts of this library
@@ -267,7 +276,8 @@ lowra_status lowra_device_status(const void* workspace_dev, void* stream);
  *     nothing and returns LOWRA_ERR_LIMIT (for scale: N = K = 8192, M = 8192, r = 64 needs about 1.6 MB).
  *   - status_out_dev (optional, may be NULL): a device uint32 that receives the device status word
  *     (LOWRA_OK or LOWRA_ERR_TIMEOUT) once the call's kernels have run, since the built-in scratch cannot
- *     be given to lowra_device_status.
+ *     be given to lowra_device_status.  It is always this call's own status: the word is cleared at the start of
+ *     every call, also when layout->deal_dev is set (unlike a caller's workspace, whose word is then sticky).
  *   - The first call on each device looks up the device address of the built-in array (once per device,
  *     with that device current).  Make that first call outside any CUDA stream capture.
  *   - All calls on a device share the one array, and it keeps what the previous call left in it (the call
@@ -316,23 +326,6 @@ lowra_status lowra_learn_codebooks(const lowra_layout* layout, const float* W_de
 lowra_status lowra_learn_codebooks_all(int32_t N, int32_t K, const float* W_dev, const double* init_levels_host,
                                        const double* init_thresholds_host, int32_t iterations, float* maps3_dev,
                                        float* thresholds3_dev, void* stream);
-
-/*
- * Diagnostic, not part of the method: C = P . Q^T with P bf16 [M, K], Q bf16 [N, K] (both
- * row-major, K % 64 == 0), C bf16 [M, N], run through the same tensor-core pipeline as the fused
- * kernels but with both operands fetched as plain bf16 tiles.  Used to compare "decode, then dense
- * product" against the fused path.  workspace as above (only the status word is used).
- */
-lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_dev, int32_t M, int32_t N, int32_t K,
-                            uint16_t* C_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
-
-/*
- * Diagnostic, not part of the method: the same product as lowra_dense_nt through the two-CTA form of the
- * tensor-core instruction (two neighbouring SMs share a 256 x 256 tile, each holding half of either operand).
- * Measures what that form is worth for this pipeline; arguments and errors as lowra_dense_nt.
- */
-lowra_status lowra_dense_nt_pair(const uint16_t* P_dev, const uint16_t* Q_dev, int32_t M, int32_t N, int32_t K,
-                                 uint16_t* C_dev, void* workspace_dev, size_t workspace_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -29,8 +29,8 @@ EXPORTS = (
     "lowra_lora_forward", "lowra_lora_backward_input", "lowra_device_status", "lowra_dense_nt",
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
     "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
-    "lowra_dense_nt_pair", "lowra_channel_errors", "lowra_deal_bytes", "lowra_deal_build", "lowra_workspace_init",
-    "lowra_learn_codebooks_all",
+    "lowra_channel_errors", "lowra_deal_bytes", "lowra_deal_build", "lowra_workspace_init",
+    "lowra_learn_codebooks_all", "lowra_set_wait_limit", "lowra_diag_wait_expiry", "lowra_diag_drop_t_flags",
 )
 
 
@@ -109,8 +109,12 @@ def lib() -> ctypes.CDLL:
         L.lowra_device_status.restype = ctypes.c_int
         L.lowra_dense_nt.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
         L.lowra_dense_nt.restype = ctypes.c_int
-        L.lowra_dense_nt_pair.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
-        L.lowra_dense_nt_pair.restype = ctypes.c_int
+        L.lowra_set_wait_limit.argtypes = [ctypes.c_uint64]
+        L.lowra_set_wait_limit.restype = ctypes.c_int
+        L.lowra_diag_wait_expiry.argtypes = [vp, ctypes.c_size_t, ctypes.c_uint64, vp]
+        L.lowra_diag_wait_expiry.restype = ctypes.c_int
+        L.lowra_diag_drop_t_flags.argtypes = [i32]
+        L.lowra_diag_drop_t_flags.restype = ctypes.c_int
         _lib = L
     return _lib
 
@@ -475,21 +479,21 @@ def lowra_device_status(workspace: torch.Tensor, stream=None) -> int:
     return int(lib().lowra_device_status(_ptr(workspace), _stream(stream)))
 
 
-def lowra_dense_nt_pair(P: torch.Tensor, Q: torch.Tensor, C: Optional[torch.Tensor] = None,
-                        workspace: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
-    """Diagnostic: C = P . Q^T through the two-CTA form of the tensor-core instruction."""
-    _dev(P, torch.bfloat16, "P")
-    _dev(Q, torch.bfloat16, "Q")
-    M, K = P.shape
-    N = Q.shape[0]
-    if C is None:
-        C = torch.empty((M, N), dtype=torch.bfloat16, device=P.device)
-    if workspace is None:
-        workspace = torch.empty(256, dtype=torch.uint8, device=P.device)
-    code = lib().lowra_dense_nt_pair(_ptr(P), _ptr(Q), int(M), int(N), int(K), _ptr(C), _ptr(workspace),
-                                     workspace.numel(), _stream(stream))
-    _check(code, "lowra_dense_nt_pair")
-    return C
+def lowra_set_wait_limit(nanoseconds: int) -> None:
+    """Limit of every device-side wait of the tensor-core kernels (0: the default of one second)."""
+    _check(lib().lowra_set_wait_limit(int(nanoseconds)), "lowra_set_wait_limit")
+
+
+def lowra_diag_wait_expiry(workspace: torch.Tensor, limit_ns: int, stream=None) -> None:
+    """Self test: a one-warp kernel whose two waits run out after `limit_ns` each; status word -> LOWRA_ERR_TIMEOUT."""
+    _dev(workspace, torch.uint8, "workspace")
+    _check(lib().lowra_diag_wait_expiry(_ptr(workspace), workspace.numel(), int(limit_ns), _stream(stream)),
+           "lowra_diag_wait_expiry")
+
+
+def lowra_diag_drop_t_flags(calls: int) -> None:
+    """Self test: the next `calls` fused calls do not publish their "down-projection ready" flags and time out."""
+    _check(lib().lowra_diag_drop_t_flags(int(calls)), "lowra_diag_drop_t_flags")
 
 
 def lowra_dense_nt(P: torch.Tensor, Q: torch.Tensor, C: Optional[torch.Tensor] = None,

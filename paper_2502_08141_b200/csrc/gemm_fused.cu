@@ -27,6 +27,8 @@
 //
 // Warp roles: 0 = TMA producer, 1 = MMA issuer (and TMEM owner), 2-5 = epilogue, 6-8 / 10-12 / 14-15 = dequant.
 // All mbarrier waits are bounded; a wait that runs out sets the status word and every role leaves.
+#include <mutex>
+
 #include "gemm_params.cuh"
 #include "ptx.cuh"
 
@@ -34,7 +36,7 @@ namespace lowra {
 
 namespace {
 
-constexpr uint64_t kWaitLimitNs = 1000ull * 1000ull * 1000ull;  // 1 s per wait
+constexpr uint64_t kGraceNs = 50ull * 1000ull;   // after a failure: time for copies and MMAs still in flight to land
 constexpr uint32_t kIdesc = ptx::umma_idesc_bf16(kTileR, kTileT);
 constexpr uint32_t kIdescAmn = kIdesc | (1u << 15);   // A operand MN-major
 
@@ -171,6 +173,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     unsigned char* out_s = base + kSmemRingMax;       // epilogue staging
     Barriers* bars = reinterpret_cast<Barriers*>(out_s + kSmemOut);
     volatile uint32_t* abort_flag = &bars->abort;
+    const uint64_t wait_ns = P.wait_ns;                // limit of every wait below (lowra_set_wait_limit; 1 s by default)
     if ((ptx::smem_u32(smem_raw) & 1023u) != 0u) {    // never seen; without it the operand descriptors would be wrong
         if (threadIdx.x == 0) atomicExch(P.status, (uint32_t)LOWRA_ERR_CUDA);
         return;
@@ -291,7 +294,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 for (int kb = t.kb0; kb < t.kb1; ++kb, ++it) {
                     const int s = it % SB;
                     const uint32_t ph = (it / SB) & 1u;
-                    if (!ptx::mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                    if (!ptx::mbar_wait(&bars->empty[s], ph ^ 1u, abort_flag, wait_ns)) { failed = true; bars->abort = 1u; break; }
                     if (MODE != kModeDense) {   // tell the dequant warps of every CTA of the cluster
 #pragma unroll
                         for (int c = 0; c < CL; ++c)
@@ -324,7 +327,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         if (lb == 0 || kb == t.kb0) {
                             // T of this token tile is written by another CTA: wait for its flag, then make
                             // those generic-proxy writes visible to the TMA (async proxy) reads below
-                            if (!ptx::flag_wait(P.flags + t.mt, want, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                            if (!ptx::flag_wait(P.flags + t.mt, want, abort_flag, wait_ns)) { failed = true; bars->abort = 1u; break; }
                             ptx::fence_proxy_async_all();
                         }
                         ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
@@ -363,7 +366,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const uint32_t acc = tile_iter & 1u;            // two accumulators take turns
                 const uint32_t aph = (tile_iter >> 1) & 1u;
                 // the epilogue warps hand the accumulator over, every time (empty, or preloaded with partial sums)
-                if (!ptx::mbar_wait(&bars->tmem_empty[acc], aph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                if (!ptx::mbar_wait(&bars->tmem_empty[acc], aph, abort_flag, wait_ns)) { failed = true; bars->abort = 1u; break; }
                 ptx::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * kTileT;
                 const int kb_fresh = (t.pre && !P.sk_late) ? -1 : t.kb0;   // the block whose first MMA overwrites the accumulator
@@ -373,9 +376,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     const int sw = (int)sa;                     // weight slot
                     const uint32_t phw = pha;
                     if (!ready_x)
-                        if (!ptx::mbar_wait(&bars->full_x[s], ph, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                        if (!ptx::mbar_wait(&bars->full_x[s], ph, abort_flag, wait_ns)) { failed = true; bars->abort = 1u; break; }
                     if (MODE != kModeDense && !ready_w)
-                        if (!ptx::mbar_wait(&bars->full_w[sw], phw, abort_flag, kWaitLimitNs)) { failed = true; bars->abort = 1u; break; }
+                        if (!ptx::mbar_wait(&bars->full_w[sw], phw, abort_flag, wait_ns)) { failed = true; bars->abort = 1u; break; }
                     ptx::tc_fence_after();
                     // probe the next stage now (its slots depend on the running stage index only)
                     const uint32_t a_addr = ptx::smem_u32(base + sa * kSmemA);
@@ -442,7 +445,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     uint32_t ok = 1u;
                     if (lane == 0) {
                         if (wait) {
-                            if (!ptx::flag_wait(P.sk_flags + c * CL + (int)crank, want, abort_flag, kWaitLimitNs)) { bars->abort = 1u; ok = 2u; }
+                            if (!ptx::flag_wait(P.sk_flags + c * CL + (int)crank, want, abort_flag, wait_ns)) { bars->abort = 1u; ok = 2u; }
                         } else {
                             ok = ptx::flag_test(P.sk_flags + c * CL + (int)crank, want) ? 1u : 0u;
                         }
@@ -494,7 +497,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             // everything before this piece is drained, so nobody waits for this warp: now the wait may block
             if (owed & (1u << acc)) { hand_over(i, true); owed &= ~(1u << acc); }
             // the four epilogue warps share named barriers, so they must agree on leaving
-            if (!ptx::mbar_wait_warp(&bars->tmem_full[acc], aph, abort_flag, kWaitLimitNs)) bars->abort = 1u;
+            if (!ptx::mbar_wait_warp(&bars->tmem_full[acc], aph, abort_flag, wait_ns)) bars->abort = 1u;
             if (agree_abort()) { failed = true; break; }
             ptx::tc_fence_after();
             float* part = P.sk_part + ((size_t)cid * CL + crank) * ((size_t)kTileT * kTileR) + my_row;
@@ -507,7 +510,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const float* ring = reinterpret_cast<const float*>(base) + my_row;
                 bool leave = false;
                 for (int c = cid + 1; c < c_end; ++c) {
-                    if (lane == 0 && !ptx::flag_wait(P.sk_flags + c * CL + (int)crank, want, abort_flag, kWaitLimitNs)) bars->abort = 1u;
+                    if (lane == 0 && !ptx::flag_wait(P.sk_flags + c * CL + (int)crank, want, abort_flag, wait_ns)) bars->abort = 1u;
                     leave = agree_abort();             // also: everybody is done with the previous partial tile in the ring
                     if (leave) break;
                     if (et == 0) {
@@ -521,7 +524,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         for (uint32_t off = 0; off < kBytes; off += kPiece)
                             ptx::bulk_copy_g2s(ptx::smem_u32(base) + off, src + off, kPiece, &bars->part_full);
                     }
-                    if (!ptx::mbar_wait_warp(&bars->part_full, (uint32_t)(c - cid - 1) & 1u, abort_flag, kWaitLimitNs)) bars->abort = 1u;
+                    if (!ptx::mbar_wait_warp(&bars->part_full, (uint32_t)(c - cid - 1) & 1u, abort_flag, wait_ns)) bars->abort = 1u;
                     leave = agree_abort();
                     if (leave) break;
                     if (c + 1 == c_end) { add = ring; break; }          // the last one is added on the way out, below
@@ -594,7 +597,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 if (et == 0) {
                     if (t.is_t) {
                         ptx::fence_proxy_async_all();
-                        ptx::flag_release(P.flags + t.mt, want);
+                        if (!P.diag_drop_t_flags) ptx::flag_release(P.flags + t.mt, want);   // (diagnostic: the waits for T run out)
                     } else {
                         ptx::flag_release(P.sk_flags + cid * CL + (int)crank, want);   // one flag per CTA: its half of the slot
                     }
@@ -631,7 +634,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     if (MODE == kModeForward || spin > 64u) __nanosleep(20);
                     if ((spin & 255u) == 255u) {
                         if (t_start == 0) t_start = ptx::globaltimer_ns();
-                        if (*abort_flag != 0u || ptx::globaltimer_ns() - t_start > kWaitLimitNs) { v = 0; break; }
+                        if (*abort_flag != 0u || ptx::globaltimer_ns() - t_start > wait_ns) { v = 0; break; }
                     }
                 }
             }
@@ -861,11 +864,29 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         }
     }
 
-    if (failed) atomicExch(P.status, (uint32_t)LOWRA_ERR_TIMEOUT);
+    if (failed) {
+        atomicExch(P.status, (uint32_t)LOWRA_ERR_TIMEOUT);
+        // tell the peers as well, so that the CTAs of the cluster agree below on how they leave
+#pragma unroll
+        for (int c = 1; c < CL; ++c)
+            ptx::st_relaxed_cluster(ptx::map_to_cta(ptx::smem_u32(&bars->abort), (crank + (uint32_t)c) % CL), 1u);
+    }
     // ---------------------------------------------------------------------- teardown
     ptx::tc_fence_before();
     __syncthreads();
     if (CL > 1) ptx::cluster_sync();   // no peer writes into this CTA's shared memory (or arrives on its barriers) any more
+    if (*abort_flag != 0u) {
+        // Somebody gave up (the same answer in every CTA of the cluster: the flag was exchanged before the barrier).
+        // Roles that were not waiting on them may have left bulk copies, TMA loads or MMAs in flight; they need
+        // microseconds.  Every role has stopped issuing, so a fixed grace period covers them before shared and
+        // tensor memory are given back.
+        if (threadIdx.x == 0) {
+            const uint64_t t0 = ptx::globaltimer_ns();
+            while (ptx::globaltimer_ns() - t0 < kGraceNs) __nanosleep(1000);
+        }
+        __syncthreads();
+        if (CL > 1) ptx::cluster_sync();
+    }
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc(tmem_base, kTmemCols);
@@ -889,8 +910,10 @@ template <int MODE>
 static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
                                 const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
     constexpr int CL = (MODE == kModeDense) ? 1 : kCluster;
-    static bool configured = false;
-    static int max_clusters = 0;   // clusters (CL = 1: CTAs) that can be resident at the same time
+    // per device: the kernel attribute has been set there, and so many clusters (CL = 1: CTAs) can be resident at once
+    static std::mutex mutex;
+    static bool configured[kMaxDevices] = {false};
+    static int max_clusters_of[kMaxDevices] = {0};
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -906,19 +929,29 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
     cfg.stream = stream;
     cfg.attrs = attr;
     cfg.numAttrs = (MODE == kModeDense) ? 1 : 2;
-    if (!configured) {
-        if (cudaFuncSetAttribute(fused_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)kGemmSmemBytes) != cudaSuccess)
-            return LOWRA_ERR_CUDA;
-        max_clusters = kNumSMs / CL;
-        if (CL > 1) {
-            // the persistent schedule needs every cluster of the grid resident (a tile waits for T of another)
-            cfg.gridDim = dim3(kNumSMs / CL * CL, 1, 1);
-            int n = 0;
-            if (cudaOccupancyMaxActiveClusters(&n, fused_kernel<MODE>, &cfg) != cudaSuccess || n < 1) return LOWRA_ERR_CUDA;
-            if (n < max_clusters) max_clusters = n;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LOWRA_ERR_CUDA;
+    int max_clusters = 0;
+    {
+        std::lock_guard<std::mutex> lock(mutex);
+        if (!configured[dev]) {
+            const int sms = device_sm_count();
+            if (sms < CL) return LOWRA_ERR_CUDA;
+            if (cudaFuncSetAttribute(fused_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)kGemmSmemBytes) != cudaSuccess)
+                return LOWRA_ERR_CUDA;
+            int most = sms / CL;
+            if (CL > 1) {
+                // the persistent schedule needs every cluster of the grid resident (a tile waits for T of another)
+                cfg.gridDim = dim3(sms / CL * CL, 1, 1);
+                int n = 0;
+                if (cudaOccupancyMaxActiveClusters(&n, fused_kernel<MODE>, &cfg) != cudaSuccess || n < 1) return LOWRA_ERR_CUDA;
+                if (n < most) most = n;
+            }
+            max_clusters_of[dev] = most;
+            configured[dev] = true;
         }
-        configured = true;
+        max_clusters = max_clusters_of[dev];
     }
     const int super_t = (G.tiles_t + CL - 1) / CL;
     const int n_t = (MODE != kModeDense && G.lora_blocks > 0) ? super_t : 0;

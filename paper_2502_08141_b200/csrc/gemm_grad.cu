@@ -21,7 +21,6 @@ namespace lowra {
 
 namespace {
 
-constexpr uint64_t kSkinnyWaitNs = 1000ull * 1000ull * 1000ull;
 constexpr int kSkinnyThreads = 192;                    // 6 warps
 constexpr uint32_t kSkinnyRing = 96 * 1024;            // pipeline stages; afterwards the fp32 partial tile
 constexpr uint32_t kSkinnySmemP = 128 * 64 * 2;        // 16 KB of P per stage
@@ -83,7 +82,7 @@ skinny_kernel(const SkinnyArgs P, const int S, const __grid_constant__ CUtensorM
             int issued = 0;
             for (int i = 0; i < n_my; ++i) {
                 const int s = i % stages, kb = kb0 + i;
-                if (!ptx::mbar_wait(&bars->empty[s], ((i / stages) & 1u) ^ 1u, abort_flag, kSkinnyWaitNs)) { failed = true; bars->abort = 1u; break; }
+                if (!ptx::mbar_wait(&bars->empty[s], ((i / stages) & 1u) ^ 1u, abort_flag, P.wait_ns)) { failed = true; bars->abort = 1u; break; }
                 unsigned char* p_s = base + s * stage_bytes;
                 unsigned char* q_s = p_s + kSkinnySmemP;
                 ptx::mbar_arrive_expect_tx(&bars->full[s], stage_bytes);
@@ -112,7 +111,7 @@ skinny_kernel(const SkinnyArgs P, const int S, const __grid_constant__ CUtensorM
             const uint32_t a_step = P.a_mn ? 128u : 2u, b_step = P.b_mn ? 128u : 2u;   // 16 contraction indices further
             for (int i = 0; i < n_my; ++i) {
                 const int s = i % stages;
-                if (!ptx::mbar_wait(&bars->full[s], (i / stages) & 1u, abort_flag, kSkinnyWaitNs)) { failed = true; bars->abort = 1u; break; }
+                if (!ptx::mbar_wait(&bars->full[s], (i / stages) & 1u, abort_flag, P.wait_ns)) { failed = true; bars->abort = 1u; break; }
                 ptx::tc_fence_after();
                 const uint32_t p_addr = ptx::smem_u32(base + s * stage_bytes);
                 const uint32_t q_addr = p_addr + kSkinnySmemP;
@@ -129,7 +128,7 @@ skinny_kernel(const SkinnyArgs P, const int S, const __grid_constant__ CUtensorM
         // ------------------------------------------------------------------ TMEM -> fp32 partial tile in shared memory
         const int q = warp & 3;
         const int row = q * 32 + lane;
-        if (n_my > 0 && !ptx::mbar_wait_warp(&bars->tmem_full, 0u, abort_flag, kSkinnyWaitNs)) { failed = true; bars->abort = 1u; }
+        if (n_my > 0 && !ptx::mbar_wait_warp(&bars->tmem_full, 0u, abort_flag, P.wait_ns)) { failed = true; bars->abort = 1u; }
         if (!failed) {
             ptx::tc_fence_after();
             for (int c0 = 0; c0 < P.rp; c0 += 32) {
@@ -215,12 +214,8 @@ skinny_kernel(const SkinnyArgs P, const int S, const __grid_constant__ CUtensorM
 
 // tmP: box of [64 c][64 rows] (a_mn) or [128 rows][64 c]; tmQ: box of [64 c][64 columns] (b_mn) or [rp columns][64 c].
 lowra_status launch_skinny(const CUtensorMap& tmP, const CUtensorMap& tmQ, const SkinnyArgs& a, cudaStream_t stream) {
-    static bool configured = false;
-    if (!configured) {
-        if (cudaFuncSetAttribute(skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSkinnySmemBytes) != cudaSuccess)
-            return LOWRA_ERR_CUDA;
-        configured = true;
-    }
+    static SmemLimit limit = {};
+    if (ensure_smem_limit(reinterpret_cast<const void*>(skinny_kernel), kSkinnySmemBytes, &limit) != LOWRA_OK) return LOWRA_ERR_CUDA;
     const int tiles = (a.R + 127) / 128, n_blocks = (a.C + 63) / 64;
     // split of the contraction: the one with the shortest estimated run = waves of CTAs x (blocks per CTA + a fixed
     // cost of set-up, pipeline fill and reduction, about six blocks' worth); every slice keeps four blocks or more

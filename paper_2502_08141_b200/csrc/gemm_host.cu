@@ -2,12 +2,23 @@
 // carve-up, TMA descriptors, launches.
 #include <cudaTypedefs.h>
 
+#include <atomic>
 #include <mutex>
 #include <string.h>
 
 #include "gemm_params.cuh"
+#include "lowra_diag.h"
+#include "ptx.cuh"
 
 namespace lowra {
+
+namespace {
+constexpr unsigned long long kDefaultWaitNs = 1000ull * 1000ull * 1000ull;   // 1 s per device-side wait
+std::atomic<unsigned long long> g_wait_ns{kDefaultWaitNs};
+std::atomic<int> g_drop_t_flags{0};   // diagnostic: so many fused calls to come do not publish their "T ready" flags
+}  // namespace
+
+unsigned long long wait_limit_ns() { return g_wait_ns.load(std::memory_order_relaxed); }
 
 namespace {
 
@@ -179,6 +190,12 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.tiles_t = tiles_t;
     G.sk_part = stream_k ? reinterpret_cast<float*>(ws + w.off_part) : nullptr;   // null: whole tiles only
     G.sk_flags = flags + tiles_t + kCluster;
+    G.wait_ns = wait_limit_ns();
+    {   // diagnostic, armed by lowra_diag_drop_t_flags: take one of the calls it asked for
+        int left = g_drop_t_flags.load(std::memory_order_relaxed);
+        while (left > 0 && !g_drop_t_flags.compare_exchange_weak(left, left - 1, std::memory_order_relaxed)) {}
+        G.diag_drop_t_flags = left > 0 ? 1 : 0;
+    }
     CUtensorMap tmB, tmT, tmFt, tmFl;
     if (!make_map(&tmB, act, (uint64_t)M, (uint64_t)G.C, (uint64_t)G.C, kTileT)) return LOWRA_ERR_CUDA;
     if (!make_map(&tmT, T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
@@ -290,7 +307,6 @@ static __device__ __align__(256) unsigned char g_static_scratch[LOWRA_STATIC_SCR
 
 namespace lowra {
 namespace {
-constexpr int kMaxDevices = 64;
 std::mutex g_static_mutex;
 void* g_static_ptr[kMaxDevices] = {nullptr};
 
@@ -327,7 +343,13 @@ extern "C" lowra_status lowra_lora_forward_static(const lowra_layout* layout, co
     if (st != LOWRA_OK) return st;
     // The scratch starts zero-filled (a static array) and only these calls write it, so the numbering of the
     // calls holds whether or not the layout brings a deal; without one the prologue kernel rewrites the status
-    // word, the flags and the deal on every call.
+    // word, the flags and the deal on every call.  With one there is no prologue, and nobody could otherwise reset
+    // the status word of the built-in array: clear it here, in stream order, so that the word handed back below is
+    // this call's own.
+    if (layout->deal_dev != nullptr) {
+        clear_status_kernel<<<1, 1, 0, (cudaStream_t)stream>>>(static_cast<uint32_t*>(scratch));
+        if (cudaGetLastError() != cudaSuccess) return LOWRA_ERR_CUDA;
+    }
     st = run_lora(false, layout, packed_dev, absmax_dev, maps_dev, X_dev, M, A_dev, B_dev, r, s, Y_dev, scratch,
                   (size_t)LOWRA_STATIC_SCRATCH_BYTES, stream, false);
     if (st != LOWRA_OK) return st;
@@ -378,6 +400,7 @@ extern "C" lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, cons
     SkinnyArgs a;
     memset(&a, 0, sizeof(a));
     a.status = status;
+    a.wait_ns = wait_limit_ns();
     a.rp = rp;
     // T = s X A: rows = tokens, contraction over the K input features
     a.out = T; a.R = M; a.C = K; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 1; a.transposed = 0; a.scale = s;
@@ -402,6 +425,62 @@ extern "C" lowra_status lowra_device_status(const void* workspace_dev, void* str
     uint32_t word = 0;
     if (cudaMemcpy(&word, workspace_dev, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return LOWRA_ERR_CUDA;
     return (lowra_status)word;
+}
+
+extern "C" lowra_status lowra_set_wait_limit(uint64_t nanoseconds) {
+    using namespace lowra;
+    if (nanoseconds == 0) nanoseconds = kDefaultWaitNs;
+    if (nanoseconds < 1000ull || nanoseconds > 10ull * kDefaultWaitNs) return LOWRA_ERR_SHAPE;
+    g_wait_ns.store(nanoseconds, std::memory_order_relaxed);
+    return LOWRA_OK;
+}
+
+extern "C" lowra_status lowra_diag_drop_t_flags(int32_t calls) {
+    if (calls < 0 || calls > 1000) return LOWRA_ERR_SHAPE;
+    lowra::g_drop_t_flags.store(calls, std::memory_order_relaxed);
+    return LOWRA_OK;
+}
+
+namespace lowra {
+namespace {
+// One CTA, one warp: lane 0 waits on a shared-memory barrier that nobody ever arrives on, then on a global flag that
+// nobody ever raises, each with the given limit; whatever ran out is recorded and the kernel returns.
+__global__ void wait_expiry_kernel(uint32_t* status, uint32_t* never_raised, uint32_t* report, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        ptx::mbar_init(&bar, 1);
+        ptx::fence_barrier_init();
+    }
+    __syncwarp();
+    uint32_t expired = 0;
+    if (threadIdx.x == 0) {
+        const uint64_t t0 = ptx::globaltimer_ns();
+        if (!ptx::mbar_wait(&bar, 0u, nullptr, limit_ns)) expired |= 1u;
+        const uint64_t t1 = ptx::globaltimer_ns();
+        if (!ptx::flag_wait(never_raised, 0xFFFFFFFFu, nullptr, limit_ns)) expired |= 2u;
+        const uint64_t t2 = ptx::globaltimer_ns();
+        report[0] = expired;
+        report[1] = (uint32_t)((t1 - t0) / 1000ull);   // microseconds spent in either wait
+        report[2] = (uint32_t)((t2 - t1) / 1000ull);
+        if (expired != 0u) atomicExch(status, (uint32_t)LOWRA_ERR_TIMEOUT);
+    }
+    expired = __shfl_sync(0xffffffffu, expired, 0);
+    if (!ptx::mbar_wait_warp(&bar, 0u, nullptr, limit_ns) && threadIdx.x == 0) report[0] |= 4u;
+}
+}  // namespace
+}  // namespace lowra
+
+extern "C" lowra_status lowra_diag_wait_expiry(void* workspace_dev, size_t workspace_bytes, uint64_t limit_ns, void* stream) {
+    using namespace lowra;
+    if (!workspace_dev) return LOWRA_ERR_NULL;
+    if (workspace_bytes < kStatusBytes || (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) != 0) return LOWRA_ERR_WORKSPACE;
+    if (limit_ns < 1000ull || limit_ns > 100ull * 1000ull * 1000ull) return LOWRA_ERR_SHAPE;   // 1 us .. 100 ms
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    uint32_t* w = reinterpret_cast<uint32_t*>(workspace_dev);
+    if (cudaMemsetAsync(workspace_dev, 0, kStatusBytes, (cudaStream_t)stream) != cudaSuccess) return LOWRA_ERR_CUDA;
+    wait_expiry_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(w, w + 4, w + 8, limit_ns);
+    return cudaGetLastError() == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
 }
 
 extern "C" lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_dev, int32_t M, int32_t N, int32_t K,
@@ -430,6 +509,7 @@ extern "C" lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_
     G.lora_blocks = 0;
     G.tiles_r = (N + kTileR - 1) / kTileR;
     G.tiles_t = (M + kTileT - 1) / kTileT;
+    G.wait_ns = wait_limit_ns();
     CUtensorMap tmB, tmFl;
     if (!make_map(&tmB, P_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, kTileT)) return LOWRA_ERR_CUDA;
     if (!make_map(&tmFl, Q_dev, (uint64_t)N, (uint64_t)K, (uint64_t)K, kTileR)) return LOWRA_ERR_CUDA;

@@ -98,7 +98,11 @@ struct GemmParams {
     int sk_dp;              // rows of whole pieces (T tiles, then weight tiles, round-robin) before the ranges
     int sk_late;            // 1: partial tiles are added in the collecting piece's epilogue; 0: preloaded into its accumulator
     long long sk_total;     // contraction blocks of the weight tiles behind the whole rows
+    unsigned long long wait_ns;   // limit of every device-side wait (lowra_set_wait_limit)
+    int diag_drop_t_flags;  // diagnostic (lowra_diag_drop_t_flags): the T tiles do not raise their flags, so the waits
+                            // for them run out and the call ends with LOWRA_ERR_TIMEOUT
 };
+unsigned long long wait_limit_ns();   // the process-wide limit, 1 s unless lowra_set_wait_limit changed it
 constexpr int kMaxClusters = kNumSMs / kCluster;
 constexpr size_t kSkSlotFloats = (size_t)kCluster * kTileT * kTileR;
 
@@ -134,6 +138,7 @@ struct SkinnyArgs {
     int a_mn, b_mn;   // 1: the row (column) index of P (Q) is the contiguous one in memory
     int transposed;
     float scale;
+    unsigned long long wait_ns;   // limit of every device-side wait
 };
 lowra_status launch_skinny(const CUtensorMap& tmP, const CUtensorMap& tmQ, const SkinnyArgs& a, cudaStream_t stream);
 

@@ -1,6 +1,8 @@
 // Host side of the C ABI: status strings, the storage planner and argument validation.
 #include <string.h>
 
+#include <mutex>
+
 #include "lowra_common.cuh"
 
 namespace lowra {
@@ -31,6 +33,33 @@ lowra_status check_device() {
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess)
         return LOWRA_ERR_CUDA;
     return major == 10 ? LOWRA_OK : LOWRA_ERR_ARCH;
+}
+
+lowra_status ensure_smem_limit(const void* kernel, size_t bytes, SmemLimit* state) {
+    static std::mutex mutex;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return LOWRA_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(mutex);
+    if (bytes > state->set[dev]) {
+        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess)
+            return LOWRA_ERR_CUDA;
+        state->set[dev] = bytes;
+    }
+    return LOWRA_OK;
+}
+
+int device_sm_count() {
+    static std::mutex mutex;
+    static int count[kMaxDevices] = {0};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return 0;
+    std::lock_guard<std::mutex> lock(mutex);
+    if (count[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n < 1) return 0;
+        count[dev] = n < kNumSMs ? n : kNumSMs;
+    }
+    return count[dev];
 }
 
 RowLayout make_row_layout(const lowra_layout* L) {

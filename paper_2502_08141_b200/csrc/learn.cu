@@ -244,12 +244,8 @@ lowra_status launch_learn(LearnParams& P, const double* init_levels_host, const 
             P.init_y[c][j] = init_levels_host[c * 16 + j];
             P.init_t[c][j] = init_thresholds_host[c * 16 + j];
         }
-    static size_t configured = 0;
-    if (smem > configured) {
-        if (cudaFuncSetAttribute(learn_kernel<ALL3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-            return LOWRA_ERR_CUDA;
-        configured = smem;
-    }
+    static SmemLimit limit = {};
+    if (ensure_smem_limit(reinterpret_cast<const void*>(learn_kernel<ALL3>), smem, &limit) != LOWRA_OK) return LOWRA_ERR_CUDA;
     const int per_sm = (int)((220u * 1024u) / (smem + 1024u));
     const int cap = kNumSMs * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));
     const unsigned grid = (unsigned)(P.N < cap ? P.N : cap);

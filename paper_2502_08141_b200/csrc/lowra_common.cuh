@@ -12,7 +12,8 @@ namespace lowra {
 
 constexpr int kBlock = 64;        // elements per absmax block (Section 4.1, groupwise normalisation)
 constexpr int kTableStride = 16;  // fp32 entries per row in the mapping / threshold tables
-constexpr int kNumSMs = 148;      // B200
+constexpr int kNumSMs = 148;      // B200: what grids and scratch are sized for; launches use min(this, the device's count)
+constexpr int kMaxDevices = 64;   // per-device host state (launch configuration, built-in scratch) is kept for this many
 
 // Everything a kernel needs to find a stored row; passed by value as a kernel argument.
 struct RowLayout {
@@ -26,6 +27,11 @@ struct RowLayout {
 
 lowra_status check_layout(const lowra_layout* L);
 lowra_status check_device();
+// Raises the dynamic shared-memory limit of `kernel` to `bytes` on the current device unless it already is that high
+// there.  `state`: the caller's record per kernel (a zero-initialised static).  Thread-safe.
+struct SmemLimit { size_t set[kMaxDevices]; };
+lowra_status ensure_smem_limit(const void* kernel, size_t bytes, SmemLimit* state);
+int device_sm_count();            // SMs of the current device, capped at kNumSMs (looked up once per device); 0 on error
 RowLayout make_row_layout(const lowra_layout* L);
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

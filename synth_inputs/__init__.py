@@ -177,6 +177,24 @@ _LEVELS = {
 }
 
 
+# Initial thresholds printed in the same listing (it prints none for 4 bits).
+_THRESHOLDS = {2: [-0.5, 0.16895762, 0.66895762], 1: [0.0]}
+
+
+def initial_codebooks():
+    """Starting tables of a codebook learner, as inputs: the levels and thresholds printed in the paper's
+    Appendix F listing; for 4 bits, where it prints no thresholds, the points halfway between neighbouring
+    levels.  -> (levels, thresholds), float64 [3, 16] each, rows = 1-, 2-, 4-bit tables, unused entries 0."""
+    y0 = np.zeros((3, 16), dtype=np.float64)
+    t0 = np.zeros((3, 16), dtype=np.float64)
+    for c, b in enumerate((1, 2, 4)):
+        lv = np.asarray(_LEVELS[b], dtype=np.float64)
+        y0[c, :lv.size] = lv
+        th = np.asarray(_THRESHOLDS[b], dtype=np.float64) if b in _THRESHOLDS else 0.5 * (lv[:-1] + lv[1:])
+        t0[c, :th.size] = th
+    return y0, t0
+
+
 def standin_codebooks(precs: np.ndarray, *, matrix_id: int = 0, seed: int = BASE_SEED):
     """Per-row tables without running the learner: the listed initial levels, each moved by
     a seeded amount of up to +-20 % of the gap to its neighbour (so rows differ and levels stay

@@ -17,11 +17,17 @@ from helpers import FRO_TOL, MAX_TOL, gemm_errors, make_case
 
 pytestmark = pytest.mark.gpu
 
+MIX3 = {1: 0.60, 2: 0.35, 4: 0.05}     # config 3: 1.5 bits on average
+MIX4 = {1: 0.85, 2: 0.15}              # config 4: 1.15 bits
+MIX5 = {2: 0.75, 4: 0.25}              # config 5: 2.5 bits
 CASES = [
-    # name, N, K, mix, matrix id  -- shapes of configs 3 and 4
-    ("gate_proj-7b", 11008, 4096, {1: 0.60, 2: 0.35, 4: 0.05}, 4),
-    ("down_proj-7b", 4096, 11008, {1: 0.60, 2: 0.35, 4: 0.05}, 6),
-    ("q_proj-13b", 5120, 5120, {1: 0.85, 2: 0.15}, 0),
+    # name, N, K, mix, matrix id  -- every distinct shape of configs 3 and 4
+    ("q_proj-7b", 4096, 4096, MIX3, 0),         # four of the seven matrices of a layer step; 264 pieces on 74 clusters
+    ("gate_proj-7b", 11008, 4096, MIX3, 4),
+    ("down_proj-7b", 4096, 11008, MIX3, 6),
+    ("q_proj-13b", 5120, 5120, MIX4, 0),
+    ("gate_proj-13b", 13824, 5120, MIX4, 4),
+    ("down_proj-13b", 5120, 13824, MIX4, 6),
 ]
 
 
@@ -100,6 +106,49 @@ def test_full_size_matrix(name, N, K, mix, mid):
     assert np.all(np.abs(got - sse_ref) <= 2.0 ** -21 * sse_ref)
     rr = np.unique(np.concatenate([[0, N - 1], rng.choice(N, 62, replace=False)]))
     assert np.array_equal(res[torch.from_numpy(rr).cuda()].cpu().numpy().view(np.uint32), res_ref[rr].view(np.uint32))
+
+
+def test_config5_layer_streamed():
+    """Config 5: the weights of a model go through encode and decode one matrix after the other (here: the seven
+    matrices of one layer at the 2-/4-bit mix, every one bit for bit against the oracle, reusing the same device
+    buffers as a streamed sweep does), and the forward pass runs at 1024, 4096 and 8192 tokens per matrix shape:
+    4096 x 4096 and 4096 x 11008 at 1024 and 8192 tokens here (11008 x 4096: test_token_sweep_forward below;
+    4096 tokens: the cases above)."""
+    import paper_2502_08141_b200 as lw
+
+    cfg = si.config(5)
+    r, s = cfg.rank, cfg.s
+    big = max(m.N * m.K for m in cfg.matrices[:7])
+    W_d = torch.empty(big, dtype=torch.float32, device="cuda")
+    What_d = torch.empty(big, dtype=torch.bfloat16, device="cuda")
+    for mat in cfg.matrices[:7]:
+        N, K = mat.N, mat.K
+        case = make_case(N, K, cfg.mix, matrix_id=mat.matrix_id, lloyd_iters=cfg.lloyd_iters)
+        layout = lw.Layout(case.precs, K).build_deal()
+        W_view = W_d[:N * K].view(N, K)
+        W_view.copy_(torch.from_numpy(case.W))
+        packed, absmax = lw.lowra_encode(layout, W_view, _dev(case.thr))
+        what = lw.lowra_decode(layout, packed, absmax, _dev(case.maps), out=What_d[:N * K].view(N, K))
+        torch.cuda.synchronize()
+        assert np.array_equal(packed.cpu().numpy()[:layout.packed_bytes], case.packed), mat.name
+        assert np.array_equal(absmax.cpu().numpy().view(np.uint32), case.absmax.view(np.uint32)), mat.name
+        assert np.array_equal(_bits(what), case.W_hat), mat.name
+        if mat.name not in ("q_proj", "down_proj"):
+            continue
+        A, B = si.lora_factors(K, N, r, matrix_id=mat.matrix_id)
+        for M in (1024, 8192):
+            X = si.activations(M, K, matrix_id=700 + mat.matrix_id)
+            rng = np.random.default_rng(M + mat.matrix_id)
+            rows = np.unique(np.concatenate([[0, 255, 256, M - 1], rng.choice(M, 60, replace=False)]))
+            ws = lw.lowra_workspace_init(torch.empty(lw.lowra_workspace_bytes(layout, M, r), dtype=torch.uint8, device="cuda"))
+            Y = lw.lowra_lora_forward(layout, packed, absmax, _dev(case.maps), _bf(X), _bf(A), _bf(B), s, workspace=ws)
+            assert lw.lowra_device_status(ws) == lw.LOWRA_OK
+            got = si.bf16_bits_to_f32(_bits(Y[torch.from_numpy(rows).cuda()]))
+            ref = oracle.lora_forward(case.W_hat, X[rows], A, B, s)
+            emax, efro = gemm_errors(got, ref)
+            assert emax <= MAX_TOL and efro <= FRO_TOL, (mat.name, M, emax, efro)
+            assert torch.isfinite(Y.float()).all()
+            del Y, ws
 
 
 @pytest.mark.parametrize("M", [1024, 8192])

@@ -47,20 +47,6 @@ def test_dense_pipeline_matches_fp64(lw):
         assert emax <= MAX_TOL and efro <= FRO_TOL, (M, N, K, emax, efro)
 
 
-def test_two_cta_pipeline_matches_fp64(lw):
-    """The same product through the two-CTA form of the tensor-core instruction (256 x 256 tile per CTA pair)."""
-    for M, N, K in ((256, 256, 64), (300, 200, 256), (1024, 640, 1024), (2048, 1536, 512)):
-        P = si.bf16_normal((M, K), 1.0, stream=42)
-        Q = si.bf16_normal((N, K), 1.0, stream=43)
-        ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
-        C = torch.full((M, N), float("nan"), dtype=torch.bfloat16, device="cuda")
-        lw.lowra_dense_nt_pair(_bf(P), _bf(Q), C=C, workspace=ws)
-        assert lw.lowra_device_status(ws) == lw.LOWRA_OK
-        ref = oracle.bf16_to_f64(P) @ oracle.bf16_to_f64(Q).T
-        emax, efro = gemm_errors(si.bf16_bits_to_f32(_bits(C)), ref)
-        assert emax <= MAX_TOL and efro <= FRO_TOL, (M, N, K, emax, efro)
-
-
 GEMM_CASES = [
     # N, K, M, r, mix, kind
     (512, 512, 16, 16, {1: 0.5, 2: 0.5}, "tiny"),                  # config 1

@@ -22,7 +22,8 @@ def lib():
 
 
 def test_library_exports_every_declared_symbol(lib):
-    header = open(os.path.join(ROOT, "include", "lowra.h")).read()
+    import glob
+    header = "".join(open(h).read() for h in sorted(glob.glob(os.path.join(ROOT, "include", "*.h"))))
     declared = set(re.findall(r"\b(lowra_[a-z_]+)\s*\(", header))
     assert declared == set(lib.EXPORTS)
     L = lib.lib()
@@ -110,8 +111,7 @@ def test_validation_runs_before_any_device_work(lib):
     sargs[8] = 24
     assert L.lowra_lora_forward_static(*sargs) == lib.LOWRA_ERR_SHAPE
     assert L.lowra_dense_nt(4096, 4096, 16, 16, 100, 4096, 4096, 256, None) == lib.LOWRA_ERR_SHAPE
-    assert L.lowra_dense_nt_pair(4096, 4096, 16, 16, 100, 4096, 4096, 256, None) == lib.LOWRA_ERR_SHAPE
-    assert L.lowra_dense_nt_pair(4096, None, 16, 16, 128, 4096, 4096, 256, None) == lib.LOWRA_ERR_NULL
+    assert L.lowra_dense_nt(4096, None, 16, 16, 128, 4096, 4096, 256, None) == lib.LOWRA_ERR_NULL
     init = (ctypes.c_double * 48)()
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, None, init, 10, 4096, 4096, None) == lib.LOWRA_ERR_NULL
     assert L.lowra_learn_codebooks(ctypes.byref(lay), 4096, init, init, -1, 4096, 4096, None) == lib.LOWRA_ERR_SHAPE

@@ -58,3 +58,13 @@ def test_configs():
     assert abs(si.avg_bits(si.config(4).mix) - 1.15) < 1e-9
     assert abs(si.avg_bits(si.config(5).mix) - 2.5) < 1e-9 and len(si.config(5).matrices) == 224
     assert sum(m.N * m.K for m in si.config(5).matrices) == 6_476_005_376
+
+
+def test_initial_codebooks_are_the_printed_tables():
+    """The starting tables handed to the GPU learner by the benchmark are the ones the oracle starts from."""
+    import oracle
+    y0, t0 = si.initial_codebooks()
+    for c, b in enumerate((1, 2, 4)):
+        y, t = oracle.initial_tables(b)
+        assert np.array_equal(y0[c, :y.size], y) and np.all(y0[c, y.size:] == 0)
+        assert np.array_equal(t0[c, :t.size], t) and np.all(t0[c, t.size:] == 0)
