@@ -123,10 +123,18 @@ __device__ __forceinline__ void deq64_2bit(const uint4& w, const Levels& lv, flo
 }
 
 
-// 4 bits: the row's 16 fp32 levels sit in shared memory (`tab`, 64 bytes: parked there for the whole tile in the
-// forward pass, fetched asynchronously two visits ahead in the backward pass), so every element is one table
-// load, one multiply and half a convert - rounded exactly as the decode kernel does.
+// 4 bits: the row's 16 fp32 levels sit in shared memory, entry-major: level c of the row at `tab + c * kStride` bytes
+// (forward: kStride = 128, the 32 lanes of a warp side by side, so a warp's 32 look-ups fall into 32 different banks
+// whatever the codes are; backward: kStride = 64, the 16 rows of an entry side by side, the two lanes of a row read
+// the same table: at most two lanes per bank).  Parked there for the whole tile in the forward pass, fetched
+// asynchronously two visits ahead in the backward pass.  Every element is one table load, one multiply and half a
+// convert - rounded exactly as the decode kernel does.  (Measured instead: the levels scaled and rounded once per
+// block into eight registers and picked with byte permutes, seven per element pair, no table in shared memory: the
+// visits of warps with 4-bit rows became so long that a 60/35/5 mix ran 14 % slower in the forward pass.)
+template <int kStride>
 __device__ __forceinline__ void deq64_4bit_direct(const uint4& lo, const uint4& hi, float a, uint32_t tab, uint32_t (&o)[32]) {
+    constexpr int kShift = (kStride == 128) ? 7 : 6;     // byte offset of level c = c << kShift
+    constexpr uint32_t kMask = 15u << kShift;
 #pragma unroll
     for (int q = 0; q < 8; ++q) {  // one 32-bit word = 8 elements
         const uint32_t w = q == 0 ? lo.x : q == 1 ? lo.y : q == 2 ? lo.z : q == 3 ? lo.w
@@ -134,8 +142,8 @@ __device__ __forceinline__ void deq64_4bit_direct(const uint4& lo, const uint4& 
         float f[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const uint32_t c4 = (j == 0) ? (w << 2) : (w >> (4 * j - 2));   // byte offset of level c = (w >> 4j) & 15
-            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(f[j]) : "r"(tab + (c4 & 0x3Cu)) : "memory");
+            const uint32_t off = (4 * j < kShift) ? (w << (kShift - 4 * j)) : (w >> (4 * j - kShift));   // c = (w >> 4j) & 15
+            asm volatile("ld.shared.f32 %0, [%1];" : "=f"(f[j]) : "r"(tab + (off & kMask)) : "memory");
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) o[4 * q + j] = pack_bf16x2(__fmul_rn(f[2 * j], a), __fmul_rn(f[2 * j + 1], a));
@@ -164,7 +172,8 @@ struct Seg {
     int tile;      // weight tile index (stream-K)
 };
 
-template <int MODE>
+// WIDE: the weight has no 4-bit rows, so nobody needs the level tables and their 16 KB hold a sixth weight slot.
+template <int MODE, bool WIDE>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmT,
              const __grid_constant__ CUtensorMap tmFt, const __grid_constant__ CUtensorMap tmFl) {
@@ -185,7 +194,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     constexpr int CL = (MODE == kModeDense) ? 1 : kCluster;
     const uint32_t crank = (CL > 1) ? ptx::cluster_ctarank() : 0u;
     // ring geometry: SA weight-operand slots of 16 KB, then SB token-operand slots of 32 KB
-    constexpr int SA = (MODE == kModeDense) ? kStages : (MODE == kModeForward) ? kStagesA_fwd : kStagesA_bwd;
+    constexpr int SA = (MODE == kModeDense) ? kStages : ((MODE == kModeForward) ? kStagesA_fwd : kStagesA_bwd) + (WIDE ? 1 : 0);
     constexpr int SB = (MODE == kModeDense) ? kStages : (MODE == kModeForward) ? kStagesB_fwd : kStagesB_bwd;
     unsigned char* tab_all = base + SA * kSmemA + SB * kSmemB;   // level tables of 4-bit rows, 2 KB per dequant warp
     auto a_slot = [&](uint32_t it) { return base + (it % SA) * kSmemA; };
@@ -613,7 +622,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         const int K = P.L.K;
         const int pw = (warp - kFirstProducerWarp) - (warp > 9 ? 1 : 0) - (warp > 13 ? 1 : 0);   // 0 .. kProducerWarps - 1
         const uint32_t tab_warp = ptx::smem_u32(tab_all) + (uint32_t)pw * 2048u;   // this warp's 2 KB of level tables (4-bit rows)
-        const uint32_t tab_lane = tab_warp + (uint32_t)lane * 64u;                  // forward: this lane's table
+        const uint32_t tab_lane = tab_warp + (uint32_t)lane * 4u;                   // forward: level c of this lane's row at tab_lane + 128 c
         uint32_t it0 = 0;                                       // running stage index at the start of the tile
         // Backward: a warp only visits the stages it has work on, so it can be several ring revolutions behind
         // or ahead of a stage's "empty" barrier, where a parity wait says nothing.  The TMA producer visits every
@@ -684,7 +693,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // 64-element absmax block is one 128-byte row.  The CTAs of the cluster take the stages in turn
                 // (stage kb is produced by CTA kb % CL and copied to the peers); inside the CTA the groups
                 // of four warps take this CTA's stages in turn, and warp q of a group holds rows 32 q .. 32 q + 31
-                // of the tile in precision order (at most two precisions meet in a warp).  A thread keeps its
+                // of the tile, roughly in precision order (see the deal in gemm_prep.cu).  A thread keeps its
                 // channel for the whole tile; the packed codes of its next two blocks are already in registers.
                 const int q = pw & 3, wgrp = pw >> 2;
                 const uint32_t item = __ldg(P.items + (size_t)t.rt * kItemStride + q * 32 + lane);
@@ -706,14 +715,16 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
                     } else if (cls == 1) {
                         lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
-                    } else {
-                        // the 16 levels of a 4-bit row: parked in shared memory for the whole tile (this lane's
-                        // 64 bytes; only this lane reads them)
+                    } else if (!WIDE) {
+                        // the 16 levels of a 4-bit row: parked in shared memory for the whole tile (entry-major: the warp's
+                        // 32 tables interleaved word by word; only this lane reads its own)
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             const float4 f = __ldg(reinterpret_cast<const float4*>(mrow) + e);
-                            ptx::st_shared_v4(tab_lane + 16u * e,
-                                              make_uint4(__float_as_uint(f.x), __float_as_uint(f.y), __float_as_uint(f.z), __float_as_uint(f.w)));
+                            ptx::st_shared_f32(tab_lane + 128u * (4 * e), f.x);
+                            ptx::st_shared_f32(tab_lane + 128u * (4 * e + 1), f.y);
+                            ptx::st_shared_f32(tab_lane + 128u * (4 * e + 2), f.z);
+                            ptx::st_shared_f32(tab_lane + 128u * (4 * e + 3), f.w);
                         }
                     }
                 }
@@ -736,8 +747,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         deq64_1bit(cur.lo.x, cur.lo.y, lv.m0, lv.m1, cur.a, o);
                     } else if (cls == 1) {
                         deq64_2bit(cur.lo, lv, cur.a, o);
-                    } else if (cls == 2) {
-                        deq64_4bit_direct(cur.lo, cur.hi, cur.a, tab_lane, o);
+                    } else if (!WIDE && cls == 2) {
+                        deq64_4bit_direct<128>(cur.lo, cur.hi, cur.a, tab_lane, o);
                     } else {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) o[i] = 0u;
@@ -800,9 +811,13 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                             lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
                         } else if (cls == 1) {
                             lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1); lv.m2 = __ldg(mrow + 2); lv.m3 = __ldg(mrow + 3);
-                        } else if (lane < 16) {
+                        } else if (!WIDE) {
+                            // entry-major: level c of row (lane & 15) at tab_slot + 64 c + 4 (lane & 15); the two lanes of
+                            // a row fetch eight levels each
+                            const uint32_t c0 = (uint32_t)(lane >> 4) * 8u;
 #pragma unroll
-                            for (int e = 0; e < 4; ++e) ptx::cp_async_16(tab_slot + (uint32_t)lane * 64u + 16u * e, mrow + 4 * e, true);
+                            for (uint32_t e = 0; e < 8; ++e)
+                                ptx::cp_async_4(tab_slot + 64u * (c0 + e) + 4u * (uint32_t)(lane & 15), mrow + c0 + e);
                         }
                     }
                     ptx::cp_async_commit();   // one group per entry, empty or not
@@ -834,8 +849,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         deq64_1bit(blk0.lo.x, blk0.lo.y, lv0.m0, lv0.m1, blk0.a, o);
                     } else if (cls == 1) {
                         deq64_2bit(blk0.lo, lv0, blk0.a, o);
-                    } else if (cls == 2) {
-                        deq64_4bit_direct(blk0.lo, blk0.hi, blk0.a, tab_slot + (lane & 15u) * 64u, o);
+                    } else if (!WIDE && cls == 2) {
+                        deq64_4bit_direct<64>(blk0.lo, blk0.hi, blk0.a, tab_slot + (lane & 15u) * 4u, o);
                     } else {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) o[i] = 0u;
@@ -906,7 +921,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     }
 }
 
-template <int MODE>
+template <int MODE, bool WIDE>
 static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
                                 const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
     constexpr int CL = (MODE == kModeDense) ? 1 : kCluster;
@@ -937,7 +952,7 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
         if (!configured[dev]) {
             const int sms = device_sm_count();
             if (sms < CL) return LOWRA_ERR_CUDA;
-            if (cudaFuncSetAttribute(fused_kernel<MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(fused_kernel<MODE, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)kGemmSmemBytes) != cudaSuccess)
                 return LOWRA_ERR_CUDA;
             int most = sms / CL;
@@ -945,7 +960,7 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
                 // the persistent schedule needs every cluster of the grid resident (a tile waits for T of another)
                 cfg.gridDim = dim3(sms / CL * CL, 1, 1);
                 int n = 0;
-                if (cudaOccupancyMaxActiveClusters(&n, fused_kernel<MODE>, &cfg) != cudaSuccess || n < 1) return LOWRA_ERR_CUDA;
+                if (cudaOccupancyMaxActiveClusters(&n, fused_kernel<MODE, WIDE>, &cfg) != cudaSuccess || n < 1) return LOWRA_ERR_CUDA;
                 if (n < most) most = n;
             }
             max_clusters_of[dev] = most;
@@ -992,15 +1007,20 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
             Q.sk_total = n_rest * blocks;
         }
     }
-    if (cudaLaunchKernelEx(&cfg, fused_kernel<MODE>, Q, tmB, tmT, tmFt, tmFl) != cudaSuccess) return LOWRA_ERR_CUDA;
+    if (cudaLaunchKernelEx(&cfg, fused_kernel<MODE, WIDE>, Q, tmB, tmT, tmFt, tmFl) != cudaSuccess) return LOWRA_ERR_CUDA;
     return LOWRA_OK;
 }
 
 lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
                           const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
-    if (mode == kModeForward) return launch_mode<kModeForward>(G, tmB, tmT, tmFt, tmFl, stream);
-    if (mode == kModeBackward) return launch_mode<kModeBackward>(G, tmB, tmT, tmFt, tmFl, stream);
-    return launch_mode<kModeDense>(G, tmB, tmT, tmFt, tmFl, stream);
+    const bool wide = G.L.class_start[3] == G.L.class_start[2];   // no 4-bit rows: the table cache becomes a weight slot
+    if (mode == kModeForward)
+        return wide ? launch_mode<kModeForward, true>(G, tmB, tmT, tmFt, tmFl, stream)
+                    : launch_mode<kModeForward, false>(G, tmB, tmT, tmFt, tmFl, stream);
+    if (mode == kModeBackward)
+        return wide ? launch_mode<kModeBackward, true>(G, tmB, tmT, tmFt, tmFl, stream)
+                    : launch_mode<kModeBackward, false>(G, tmB, tmT, tmFt, tmFl, stream);
+    return launch_mode<kModeDense, false>(G, tmB, tmT, tmFt, tmFl, stream);
 }
 
 }  // namespace lowra

@@ -45,8 +45,9 @@ constexpr int kStages = 4;        // dense diagnostic: four stages of one weight
 // Forward / backward: the dequant warps (and the copies between the CTAs of a cluster) need to run further ahead
 // of the tensor core than the TMA loads do, so the ring is split into 16 KB weight slots and 32 KB token slots:
 // five + four in both passes, plus 16 KB for the level tables of 4-bit rows (the token slots hide the L2
-// latency of the TMA loads; a fifth weight slot was worth +9..13 % in the forward pass, a sixth does not fit beside
-// the table cache, and reading the tables through L1 instead cost more than the sixth slot gave).  A weight slot
+// latency of the TMA loads; a fifth weight slot was worth +9..13 % in the forward pass; a sixth is worth another
+// +3..5 % and takes the place of the table cache in calls on weights without 4-bit rows; reading the tables through
+// L1 instead, or keeping the levels in registers, cost more than the sixth slot gives).  A weight slot
 // is free once the MMAs of that many stages earlier are complete; the weight ring must not be shallower than the
 // token ring (the TMA warp also loads factor tiles into weight slots).
 constexpr int kStagesA_fwd = 5, kStagesA_bwd = 5;

@@ -22,7 +22,6 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
         int cls[per];
         uint32_t stored[per];   // stored position of the row (asked for now: the answer is needed last)
         unsigned mask[per][4];
-        int total[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int i = 0; i < per; ++i) {
             const int row = grp * G + i * 32 + lane;
@@ -35,45 +34,29 @@ __device__ void deal_rows(const PrepParams& P, int blk) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 mask[i][c] = __ballot_sync(0xffffffffu, cls[i] == c);
-                total[c] += __popc(mask[i][c]);
             }
         }
-        int class_base[4];
-        class_base[0] = 0;
-#pragma unroll
-        for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total[c - 1];
-        // rows of every class by residue (row offset mod 8): the same for all lanes
-        int cnt[4][8];
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-            for (int res = 0; res < 8; ++res) {
-                int n = 0;
-#pragma unroll
-                for (int i2 = 0; i2 < per; ++i2) n += __popc(mask[i2][c] & (0x01010101u << res));
-                cnt[c][res] = n;
-            }
+        // Order: the rows with the same offset mod 8 (16 of them; a lane's rows all share its lane & 7) are ranked by
+        // (class, offset), and entry 8 * rank + (offset mod 8) takes the row.  Eight neighbouring lanes of a dequant warp
+        // therefore always hold eight different offsets mod 8 - their 16-byte stores into the swizzled operand tile fall
+        // into eight different bank groups whatever the precisions are - and the entries still run from the lowest
+        // class to the highest, exactly sorted wherever the classes are spread evenly over the eight residues.
+        const unsigned res_mask = 0x01010101u << (lane & 7);
 #pragma unroll
         for (int i = 0; i < per; ++i) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 if (cls[i] == c) {
-                    // inside the class the rows are taken round-robin over (row offset mod 8), so that eight
-                    // neighbouring lanes hold eight different residues: their 16-byte stores into the swizzled
-                    // operand tile then fall into eight different bank groups
-                    const unsigned res_mask = 0x01010101u << (lane & 7);
-                    int b = 0;   // rank of this row among the rows of its class with the same residue
+                    int rank = 0;   // rows of the same residue that come before this one
 #pragma unroll
-                    for (int i2 = 0; i2 < per; ++i2)
-                        if (i2 < i) b += __popc(mask[i2][c] & res_mask);
-                    b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
-                    int q = 0;   // rows of the class taken before this one
+                    for (int c2 = 0; c2 < 4; ++c2)
 #pragma unroll
-                    for (int res = 0; res < 8; ++res)
-                        q += min(cnt[c][res], b) + ((res < (lane & 7) && cnt[c][res] > b) ? 1 : 0);
+                        for (int i2 = 0; i2 < per; ++i2)
+                            if (c2 < c || (c2 == c && i2 < i)) rank += __popc(mask[i2][c2] & res_mask);
+                    rank += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
                     const int off = i * 32 + lane;
                     const uint32_t p = (c < 3) ? stored[i] : 0u;
-                    out[class_base[c] + q] = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
+                    out[rank * 8 + (lane & 7)] = (uint32_t)off | ((uint32_t)c << 7) | (p << 9);
                 }
             }
         }
@@ -123,7 +106,6 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
         int cls[2];
         uint32_t stored[2];   // stored position of the row (asked for now: the answer is needed last)
         unsigned mask[2][4];
-        int total_c[4] = {0, 0, 0, 0};
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
             const int row = grp * 64 + i * 32 + lane;
@@ -136,19 +118,8 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 mask[i][c] = __ballot_sync(0xffffffffu, cls[i] == c);
-                total_c[c] += __popc(mask[i][c]);
             }
         }
-        int class_base[4];
-        class_base[0] = 0;
-#pragma unroll
-        for (int c = 1; c < 4; ++c) class_base[c] = class_base[c - 1] + total_c[c - 1];
-        int cnt[4][8];   // rows of every class by residue (row offset mod 8): the same for all lanes
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-#pragma unroll
-            for (int res = 0; res < 8; ++res)
-                cnt[c][res] = __popc(mask[0][c] & (0x01010101u << res)) + __popc(mask[1][c] & (0x01010101u << res));
         if (lane < kChunks)
             P.heads[chunk_slot(n0, (uint32_t)lane, cta)] = (uint32_t)grp | ((uint32_t)(kStageArrivals / kChunks) << 24);
 #pragma unroll
@@ -165,17 +136,19 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
                         rec.y = sp * (uint32_t)P.L.nb;
                         rec.z = (uint32_t)row * (uint32_t)kTableStride;
                     }
-                    // inside the class the rows are taken round-robin over (row offset mod 8), so that eight
-                    // neighbouring lanes hold eight different residues: their 16-byte stores into the swizzled
-                    // operand tile then fall into eight different bank groups
+                    // the eight rows with the same offset mod 8 are ranked by (class, offset); position 8 * rank +
+                    // (offset mod 8): eight neighbouring lanes always hold eight different residues, so their 16-byte
+                    // stores into the swizzled operand tile fall into eight different bank groups whatever the
+                    // precisions are, and the positions still run from the lowest class to the highest
                     const unsigned res_mask = 0x01010101u << (lane & 7);
-                    int b = 0;   // rank of this row among the rows of its class with the same residue
-                    if (i == 1) b += __popc(mask[0][c] & res_mask);
-                    b += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
-                    int pos = class_base[c];  // rows taken before this one
+                    int rank = 0;
 #pragma unroll
-                    for (int res = 0; res < 8; ++res)
-                        pos += min(cnt[c][res], b) + ((res < (lane & 7) && cnt[c][res] > b) ? 1 : 0);
+                    for (int c2 = 0; c2 < 4; ++c2)
+#pragma unroll
+                        for (int i2 = 0; i2 < 2; ++i2)
+                            if (c2 < c || (c2 == c && i2 < i)) rank += __popc(mask[i2][c2] & res_mask);
+                    rank += __popc(mask[i][c] & res_mask & ((1u << lane) - 1u));
+                    const int pos = rank * 8 + (lane & 7);
                     uint4* dst = rows + (size_t)chunk_slot(n0, (uint32_t)(pos / 16), cta) * 32 + pos % 16;
                     dst[0] = rec;
                     dst[16] = rec;
