@@ -67,6 +67,12 @@ typedef struct {
     const int32_t* perm_dev;     /* [N] stored position -> original row */
     const int32_t* inv_perm_dev; /* [N] original row -> stored position */
     const void* deal_dev;        /* NULL, or what lowra_deal_build wrote for this weight (see there) */
+    const uint64_t* natural_offsets_dev;   /* NULL: packed codes and absmax rows in the grouped order described above.
+                                    Otherwise [N + 1] byte offsets (a device copy of what lowra_natural_offsets
+                                    writes): the packed buffer and the absmax rows are in the paper's own order
+                                    (Appendix A.2) - rows in their ORIGINAL order, row r at byte natural_offsets[r],
+                                    absmax row r = original row r - and every call that takes this layout (encode,
+                                    decode, deal_build, forward, backward-input) reads or writes that buffer directly */
 } lowra_layout;
 
 /*
@@ -110,6 +116,10 @@ lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* packed_dev,
  *
  * lowra_natural_offsets (host only): offsets_host[N + 1] from precs_host[N]; offsets_host[N] is the
  * buffer size (= the grouped layout's packed_bytes).  Errors as lowra_plan.
+ *
+ * Nothing has to be converted to use such a buffer: point layout->natural_offsets_dev at the offsets and every kernel
+ * finds a row at its offset there (the perm / inv_perm / counts of the layout are still needed: work is still handed
+ * out precision by precision).  lowra_reorder_rows converts an existing buffer from one order to the other:
  *
  * lowra_reorder_rows: to_natural != 0: grouped -> natural; to_natural == 0: natural -> grouped.
  *   offsets_dev     uint64 [N + 1], device copy of the offsets above                        (in)

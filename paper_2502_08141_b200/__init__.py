@@ -47,7 +47,7 @@ class _CLayout(ctypes.Structure):
         ("seg_off", ctypes.c_uint64 * 3),
         ("packed_bytes", ctypes.c_uint64),
         ("precs_dev", ctypes.c_void_p), ("perm_dev", ctypes.c_void_p), ("inv_perm_dev", ctypes.c_void_p),
-        ("deal_dev", ctypes.c_void_p),
+        ("deal_dev", ctypes.c_void_p), ("natural_offsets_dev", ctypes.c_void_p),
     ]
 
 
@@ -168,7 +168,9 @@ def lowra_plan(precs_host: np.ndarray, K: int) -> dict:
 class Layout:
     """A ``lowra_layout`` plus the device arrays it points to (kept alive here)."""
 
-    def __init__(self, precs_host: np.ndarray, K: int, device="cuda"):
+    def __init__(self, precs_host: np.ndarray, K: int, device="cuda", natural: bool = False):
+        """natural=True: packed codes and absmax rows are kept in the paper's own order (rows in original order at
+        offsets that follow from their precisions); every call on this layout then reads / writes that buffer."""
         self.precs_host = np.ascontiguousarray(precs_host, dtype=np.uint8)
         self.N, self.K = int(self.precs_host.shape[0]), int(K)
         self.plan = lowra_plan(self.precs_host, K)
@@ -187,8 +189,14 @@ class Layout:
         c.perm_dev = self.perm.data_ptr()
         c.inv_perm_dev = self.inv_perm.data_ptr()
         c.deal_dev = None
+        c.natural_offsets_dev = None
         self.c = c
         self.deal = None
+        self.natural_offsets = None
+        if natural:
+            off = lowra_natural_offsets(self.precs_host, K)
+            self.natural_offsets = torch.from_numpy(off.view(np.int64)).to(self.device)
+            c.natural_offsets_dev = self.natural_offsets.data_ptr()
 
     def build_deal(self, stream=None) -> "Layout":
         """Deal the rows to the dequantising warps once for this weight (lowra_deal_build): the fused calls on this

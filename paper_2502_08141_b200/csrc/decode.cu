@@ -51,10 +51,10 @@ __device__ __forceinline__ void decode_piece(const DecodeParams& P, int p, int p
     const int K = P.L.K;
     const int r = __ldg(P.L.perm + p);
     const size_t row_bytes = (size_t)K * B / 8;
-    const uint8_t* row = P.packed + P.L.seg_off[c] + (size_t)(p - P.L.class_start[c]) * row_bytes;
+    const uint8_t* row = P.packed + packed_row_offset(P.L, c, p, r);
     const size_t byte0 = (size_t)piece * 512 + (size_t)lane * 16;
     const int e0 = piece * kElemsPiece;                         // first element of the piece
-    const float* arow = P.absmax + (size_t)p * P.L.nb + e0 / kBlock;
+    const float* arow = P.absmax + (size_t)absmax_row_of(P.L, p, r) * P.L.nb + e0 / kBlock;
     const int blocks_left = P.L.nb - e0 / kBlock;               // blocks of the row from e0 on
     const float* mrow = P.maps + (size_t)r * kTableStride;
 

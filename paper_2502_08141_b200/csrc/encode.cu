@@ -97,12 +97,10 @@ __device__ __forceinline__ void encode_chunk(const EncodeParams& P, int p, int c
     for (int i = 0; i < 32; ++i) m = fmaxf(m, fabsf(x[i]));
     m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, 1));
     const bool live = lane * 32 < valid;
-    if (live && (lane & 1) == 0) P.absmax[(size_t)p * P.L.nb + (e0 >> 6) + (lane >> 1)] = m;
+    if (live && (lane & 1) == 0) P.absmax[(size_t)absmax_row_of(P.L, p, r) * P.L.nb + (e0 >> 6) + (lane >> 1)] = m;
     const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
 
-    const size_t row_bytes = (size_t)K * B / 8;
-    uint8_t* dst = P.packed + P.L.seg_off[c] + (size_t)(p - P.L.class_start[c]) * row_bytes +
-                   (size_t)(e0 + lane * 32) * B / 8;
+    uint8_t* dst = P.packed + packed_row_offset(P.L, c, p, r) + (size_t)(e0 + lane * 32) * B / 8;
     if (B == 1) {
         uint32_t below = 0u;
 #pragma unroll

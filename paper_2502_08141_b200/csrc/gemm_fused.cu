@@ -708,8 +708,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                     const int p = info_pos(item);
                     const int b = 1 << cls;
                     bits_stride = 8 * b;
-                    bits_ptr = P.packed + P.L.seg_off[cls] + (size_t)(p - P.L.class_start[cls]) * ((size_t)K * b / 8);
-                    absmax_ptr = P.absmax + (size_t)p * P.L.nb;
+                    bits_ptr = P.packed + packed_row_offset(P.L, cls, p, r0 + row_local);
+                    absmax_ptr = P.absmax + (size_t)absmax_row_of(P.L, p, r0 + row_local) * P.L.nb;
                     mrow = P.maps + (size_t)(r0 + row_local) * kTableStride;
                     if (cls == 0) {
                         lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);

@@ -402,21 +402,31 @@ extern "C" lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, cons
     a.status = status;
     a.wait_ns = wait_limit_ns();
     a.rp = rp;
-    // T = s X A: rows = tokens, contraction over the K input features
-    a.out = T; a.R = M; a.C = K; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 1; a.transposed = 0; a.scale = s;
-    st = launch_skinny(tmX, tmA, a, stream);
-    if (st != LOWRA_OK) return st;
-    // U = s dY B^T: rows = tokens, contraction over the N output channels
-    a.out = U; a.C = N; a.b_mn = 0;
-    st = launch_skinny(tmdY, tmB, a, stream);
-    if (st != LOWRA_OK) return st;
-    // dA = X^T U: rows = input features, contraction over the tokens
-    a.out = dA_dev; a.R = K; a.C = M; a.n_cols = r; a.ld_out = r; a.a_mn = 1; a.b_mn = 1; a.scale = 1.0f;
-    st = launch_skinny(tmXt, tmU, a, stream);
-    if (st != LOWRA_OK) return st;
-    // dB = (dY^T T)^T: rows = output channels, written transposed
-    a.out = dB_dev; a.R = N; a.ld_out = N; a.transposed = 1;
-    return launch_skinny(tmdYt, tmT, a, stream);
+    // Four skinny products; X and dY are each needed by two of them.  The two uses of the larger operand run back to
+    // back, so that its second reading comes from L2 (126 MB hold a 4096-token operand of up to 11008 columns), and
+    // the smaller operand is read first and last: T, U, dB, dA when dY is the larger one, U, T, dA, dB otherwise.
+    auto down_T = [&]() {   // T = s X A: rows = tokens, contraction over the K input features
+        a.out = T; a.R = M; a.C = K; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 1; a.transposed = 0; a.scale = s;
+        return launch_skinny(tmX, tmA, a, stream);
+    };
+    auto down_U = [&]() {   // U = s dY B^T: rows = tokens, contraction over the N output channels
+        a.out = U; a.R = M; a.C = N; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 0; a.transposed = 0; a.scale = s;
+        return launch_skinny(tmdY, tmB, a, stream);
+    };
+    auto grad_A = [&]() {   // dA = X^T U: rows = input features, contraction over the tokens
+        a.out = dA_dev; a.R = K; a.C = M; a.n_cols = r; a.ld_out = r; a.a_mn = 1; a.b_mn = 1; a.transposed = 0; a.scale = 1.0f;
+        return launch_skinny(tmXt, tmU, a, stream);
+    };
+    auto grad_B = [&]() {   // dB = (dY^T T)^T: rows = output channels, written transposed
+        a.out = dB_dev; a.R = N; a.C = M; a.n_cols = r; a.ld_out = N; a.a_mn = 1; a.b_mn = 1; a.transposed = 1; a.scale = 1.0f;
+        return launch_skinny(tmdYt, tmT, a, stream);
+    };
+    if (N > K) {
+        if ((st = down_T()) != LOWRA_OK || (st = down_U()) != LOWRA_OK || (st = grad_B()) != LOWRA_OK) return st;
+        return grad_A();
+    }
+    if ((st = down_U()) != LOWRA_OK || (st = down_T()) != LOWRA_OK || (st = grad_A()) != LOWRA_OK) return st;
+    return grad_B();
 }
 
 extern "C" lowra_status lowra_device_status(const void* workspace_dev, void* stream) {

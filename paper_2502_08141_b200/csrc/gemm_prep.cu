@@ -131,9 +131,8 @@ __device__ void deal_backward(const PrepParams& P, int blk) {
                     uint4 rec = make_uint4(0u, 0u, 0u, (uint32_t)off | ((uint32_t)c << 8));
                     if (c < 3) {
                         const uint32_t sp = stored[i];   // stored position
-                        const uint64_t row_bytes = ((uint64_t)P.L.K << c) >> 3;
-                        rec.x = (uint32_t)((P.L.seg_off[c] + (uint64_t)(sp - (uint32_t)P.L.class_start[c]) * row_bytes) >> 4);
-                        rec.y = sp * (uint32_t)P.L.nb;
+                        rec.x = (uint32_t)(packed_row_offset(P.L, c, (int)sp, row) >> 4);
+                        rec.y = (uint32_t)absmax_row_of(P.L, (int)sp, row) * (uint32_t)P.L.nb;
                         rec.z = (uint32_t)row * (uint32_t)kTableStride;
                     }
                     // the eight rows with the same offset mod 8 are ranked by (class, offset); position 8 * rank +

@@ -23,6 +23,7 @@ lowra_status check_layout(const lowra_layout* L) {
     if (L->seg_off[0] != 0 || L->seg_off[1] != o1 || L->seg_off[2] != o2 || L->packed_bytes != total)
         return LOWRA_ERR_PREC;
     if (!aligned16(L->perm_dev) || !aligned16(L->inv_perm_dev)) return LOWRA_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(L->natural_offsets_dev) & 7u) != 0) return LOWRA_ERR_ALIGN;
     return LOWRA_OK;
 }
 
@@ -75,6 +76,7 @@ RowLayout make_row_layout(const lowra_layout* L) {
     R.precs = L->precs_dev;
     R.perm = L->perm_dev;
     R.inv_perm = L->inv_perm_dev;
+    R.nat = L->natural_offsets_dev;
     return R;
 }
 

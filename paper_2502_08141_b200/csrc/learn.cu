@@ -12,8 +12,9 @@
 // One CTA per row at a time (persistent, grid-stride): the row is read from HBM once (4 bytes per element, the
 // kernel's only traffic), normalised and parked in shared memory; the T passes run out of shared memory.
 // Every thread keeps private fp64 sums per bucket: in registers for 1 and 2 bits, in a bank-conflict-free
-// slice of shared memory for 4 bits; a fixed reduction tree adds them up (warp shuffles, then across warps), so
-// results are reproducible from run to run - but the order of the fp64 additions is not the index order of a
+// slice of shared memory for 4 bits; the block's weight enters once per four elements (they are added up exactly
+// first); a fixed reduction tree adds the threads' sums up (warp shuffles, then across warps), so
+// results are reproducible from run to run - but the order of the fp64 operations is not the index order of a
 // serial loop, so sums agree with a serial implementation to rounding only.
 #include <string.h>
 
@@ -108,47 +109,56 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
     __syncthreads();
 
     for (int it = 0; it < P.iterations; ++it) {
-        // ---- one pass: private sums of w * n and w per bucket
+        // ---- one pass: private sums of w * n and w per bucket.  The weight is the same for the four elements a thread
+        // takes at a time (they lie in one 64-element block), so the elements themselves are added up per bucket first
+        // (exactly: four fp32 values in fp64) and counted, and the weight enters once per four elements and bucket.
         if (B <= 2) {
-            // four independent sets of sums per thread (the fp64 adds are latency-bound otherwise); a thread walks
-            // over 64-element blocks, four elements at a time, so the block's weight is converted once
-            double num[4][Lv], den[4][Lv];
+            // Few buckets: no bucket index at all.  cn[0] / cd[0] take the elements below the first threshold, cn[j] /
+            // cd[j] (j >= 1) everything at or above threshold j - 1 - predicated adds - and a bucket's sums are the
+            // difference of two neighbours (which were added up over the same elements in the same order wherever the
+            // bucket is empty, so that an empty bucket has exactly zero weight).
+            double cn[Lv], cd[Lv];
+            float th[Lv - 1];
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int j = 0; j < Lv; ++j) cn[j] = cd[j] = 0.0;
 #pragma unroll
-                for (int j = 0; j < Lv; ++j) num[u][j] = den[u][j] = 0.0;
+            for (int j = 0; j < Lv - 1; ++j) th[j] = tf[j];
             for (int q = tid; q < K / 4; q += kLearnThreads) {   // quad q = elements 4 q .. 4 q + 3, all in block q / 16
                 const float4 xv = *reinterpret_cast<const float4*>(xs + 4 * q);
                 const double w = (double)ws[q >> 4];
                 const float xf[4] = {xv.x, xv.y, xv.z, xv.w};
+                double sq[Lv];
+                int cq[Lv];
+#pragma unroll
+                for (int j = 0; j < Lv; ++j) { sq[j] = 0.0; cq[j] = 0; }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const double x = (double)xf[u];
-                    const int b = bucket_of<B>(xf[u], tf);
-                    const double wx = __dmul_rn(w, x);
-                    if (B == 1) {
-                        // two buckets: a branch (measured 29 % faster than adding a selected 0.0 to both)
-                        if (b == 0) { num[u][0] += wx; den[u][0] += w; } else { num[u][Lv - 1] += wx; den[u][Lv - 1] += w; }
-                    } else {
+                    if (th[0] <= xf[u]) { sq[1] += x; ++cq[1]; } else { sq[0] += x; ++cq[0]; }
 #pragma unroll
-                        for (int j = 0; j < Lv; ++j) {   // four buckets: branches were slower on long rows
-                            num[u][j] += (b == j) ? wx : 0.0;
-                            den[u][j] += (b == j) ? w : 0.0;
-                        }
-                    }
+                    for (int j = 2; j < Lv; ++j)
+                        if (th[j - 1] <= xf[u]) { sq[j] += x; ++cq[j]; }
+                }
+#pragma unroll
+                for (int j = 0; j < Lv; ++j) {
+                    cn[j] = fma(w, sq[j], cn[j]);
+                    cd[j] = fma(w, (double)cq[j], cd[j]);
                 }
             }
 #pragma unroll
             for (int j = 0; j < Lv; ++j) {
-                const double sn = warp_sum((num[0][j] + num[1][j]) + (num[2][j] + num[3][j]));
-                const double sd = warp_sum((den[0][j] + den[1][j]) + (den[2][j] + den[3][j]));
+                const double pn = (j == 0 || j == Lv - 1) ? cn[j] : cn[j] - cn[j + 1];
+                const double pd = (j == 0 || j == Lv - 1) ? cd[j] : cd[j] - cd[j + 1];
+                const double sn = warp_sum(pn);
+                const double sd = warp_sum(pd);
                 if (lane == 0) { red[(2 * j) * kLearnWarps + warp] = sn; red[(2 * j + 1) * kLearnWarps + warp] = sd; }
             }
         } else {
-            // 16 buckets: sums live in shared memory, acc[(2 j + which) * kLearnThreads + tid]; four elements at a
+            // 16 buckets: the sums live in shared memory, one (w n, w) pair per thread and bucket; four elements at a
             // time, their bucket searches side by side
+            double2* acc2 = reinterpret_cast<double2*>(acc);
 #pragma unroll
-            for (int j = 0; j < 2 * Lv; ++j) acc[j * kLearnThreads + tid] = 0.0;
+            for (int j = 0; j < Lv; ++j) acc2[j * kLearnThreads + tid] = make_double2(0.0, 0.0);
             for (int q = tid; q < K / 4; q += kLearnThreads) {
                 const float4 xv = *reinterpret_cast<const float4*>(xs + 4 * q);
                 const double w = (double)ws[q >> 4];
@@ -158,29 +168,36 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
                 for (int u = 0; u < 4; ++u) b[u] = bucket_of<B>(xf[u], tf);
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    acc[(2 * b[u]) * kLearnThreads + tid] += __dmul_rn(w, (double)xf[u]);
-                    acc[(2 * b[u] + 1) * kLearnThreads + tid] += w;
+                    double2 a = acc2[b[u] * kLearnThreads + tid];
+                    a.x = fma(w, (double)xf[u], a.x);
+                    a.y += w;
+                    acc2[b[u] * kLearnThreads + tid] = a;
                 }
             }
 #pragma unroll 4
-            for (int j = 0; j < 2 * Lv; ++j) {
-                const double s2 = warp_sum(acc[j * kLearnThreads + tid]);
-                if (lane == 0) red[j * kLearnWarps + warp] = s2;
+            for (int j = 0; j < Lv; ++j) {
+                const double2 a = acc2[j * kLearnThreads + tid];
+                const double sn = warp_sum(a.x), sd = warp_sum(a.y);
+                if (lane == 0) { red[(2 * j) * kLearnWarps + warp] = sn; red[(2 * j + 1) * kLearnWarps + warp] = sd; }
             }
         }
         __syncthreads();
-        // ---- new levels (an empty bucket keeps its level), then midpoints
-        if (tid < Lv) {
-            double sn = 0.0, sd = 0.0;
+        // ---- new levels (an empty bucket keeps its level), then midpoints: the first warp, a shuffle in between
+        if (warp == 0) {
+            double yv = 0.0;
+            if (lane < Lv) {
+                double sn = 0.0, sd = 0.0;
 #pragma unroll
-            for (int w2 = 0; w2 < kLearnWarps; ++w2) { sn += red[(2 * tid) * kLearnWarps + w2]; sd += red[(2 * tid + 1) * kLearnWarps + w2]; }
-            if (sd > 0.0) y[tid] = sn / sd;
-        }
-        __syncthreads();
-        if (tid + 1 < Lv) {
-            const double tm = (y[tid] + y[tid + 1]) * 0.5;
-            t[tid] = tm;
-            tf[tid] = __double2float_ru(tm);
+                for (int w2 = 0; w2 < kLearnWarps; ++w2) { sn += red[(2 * lane) * kLearnWarps + w2]; sd += red[(2 * lane + 1) * kLearnWarps + w2]; }
+                yv = (sd > 0.0) ? sn / sd : y[lane];
+                y[lane] = yv;
+            }
+            const double yn = __shfl_down_sync(0xffffffffu, yv, 1);
+            if (lane + 1 < Lv) {
+                const double tm = (yv + yn) * 0.5;
+                t[lane] = tm;
+                tf[lane] = __double2float_ru(tm);
+            }
         }
         __syncthreads();
     }
@@ -195,14 +212,19 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
     __syncthreads();   // the tables and sums in shared memory are reused by the next run, the row buffer by the next row
 }
 
-template <bool ALL3>
+// FOUR = false: for weights without 4-bit rows.  Only the 4-bit runs need the 32 KB of per-thread bucket sums in shared
+// memory, and the rounds of a row are a chain of short phases between barriers, so what hides their latency is the number
+// of CTAs per SM: without those 32 KB three times as many fit (all-1-bit rows: 0.52 -> 0.34 ms on 4096 x 11008 at ten
+// rounds).  (Running the 4-bit rows of a mixed weight in a kernel of their own was slower: the few rows leave most SMs
+// idle for the length of a row.)
+template <bool ALL3, bool FOUR>
 __global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_constant__ LearnParams P) {
     extern __shared__ __align__(16) unsigned char learn_smem[];
-    // [16 + 16 doubles levels/thresholds][2 * 16 * warps doubles reduction][2 * 16 * threads doubles sums][K floats][nb floats][16 floats]
+    // [16 + 16 doubles levels/thresholds][2 * 16 * warps doubles reduction][FOUR: 2 * 16 * threads doubles sums][K floats][nb floats][16 floats]
     double* yt = reinterpret_cast<double*>(learn_smem);
     double* red = yt + 32;
     double* acc = red + 2 * 16 * kLearnWarps;
-    float* xs = reinterpret_cast<float*>(acc + 2 * 16 * kLearnThreads);
+    float* xs = reinterpret_cast<float*>(acc + (FOUR ? 2 * 16 * kLearnThreads : 0));
     float* ws = xs + P.K;
     float* tf = ws + P.K / kBlock;   // [16] thresholds as fp32 upper neighbours
     pdl_enter();
@@ -215,12 +237,12 @@ __global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_const
             const size_t plane = (size_t)P.N * kTableStride;
             learn_row<1>(P, xs, ws, acc, red, yt, tf, m, h);
             learn_row<2>(P, xs, ws, acc, red, yt, tf, m + plane, h + plane);
-            learn_row<4>(P, xs, ws, acc, red, yt, tf, m + 2 * plane, h + 2 * plane);
+            if (FOUR) learn_row<4>(P, xs, ws, acc, red, yt, tf, m + 2 * plane, h + 2 * plane);
         } else {
             const int b = P.L.precs[r];
             if (b == 1) learn_row<1>(P, xs, ws, acc, red, yt, tf, m, h);
             else if (b == 2) learn_row<2>(P, xs, ws, acc, red, yt, tf, m, h);
-            else learn_row<4>(P, xs, ws, acc, red, yt, tf, m, h);
+            else if (FOUR) learn_row<4>(P, xs, ws, acc, red, yt, tf, m, h);
         }
     }
 }
@@ -231,23 +253,17 @@ namespace lowra {
 namespace {
 
 // validation shared by the two entry points is done by the callers; this fills the tables and launches
-template <bool ALL3>
-lowra_status launch_learn(LearnParams& P, const double* init_levels_host, const double* init_thresholds_host,
-                          void* stream) {
-    const size_t smem = (32 + 2 * 16 * kLearnWarps + 2 * 16 * kLearnThreads) * sizeof(double) +
+template <bool ALL3, bool FOUR>
+lowra_status launch_learn_kernel(const LearnParams& P, void* stream) {
+    const size_t smem = (32 + 2 * 16 * kLearnWarps + (FOUR ? 2 * 16 * kLearnThreads : 0)) * sizeof(double) +
                         ((size_t)P.K + (size_t)P.K / kBlock + 16) * sizeof(float);
     if (smem > 200 * 1024) return LOWRA_ERR_SHAPE;   // the row has to fit into shared memory (K <= 40960)
-    lowra_status st = check_device();
-    if (st != LOWRA_OK) return st;
-    for (int c = 0; c < 3; ++c)
-        for (int j = 0; j < 16; ++j) {
-            P.init_y[c][j] = init_levels_host[c * 16 + j];
-            P.init_t[c][j] = init_thresholds_host[c * 16 + j];
-        }
     static SmemLimit limit = {};
-    if (ensure_smem_limit(reinterpret_cast<const void*>(learn_kernel<ALL3>), smem, &limit) != LOWRA_OK) return LOWRA_ERR_CUDA;
+    if (ensure_smem_limit(reinterpret_cast<const void*>(learn_kernel<ALL3, FOUR>), smem, &limit) != LOWRA_OK) return LOWRA_ERR_CUDA;
     const int per_sm = (int)((220u * 1024u) / (smem + 1024u));
-    const int cap = kNumSMs * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));
+    const int sms = device_sm_count();
+    if (sms < 1) return LOWRA_ERR_CUDA;
+    const int cap = sms * (per_sm < 1 ? 1 : (per_sm > 16 ? 16 : per_sm));
     const unsigned grid = (unsigned)(P.N < cap ? P.N : cap);
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -259,7 +275,23 @@ lowra_status launch_learn(LearnParams& P, const double* init_levels_host, const 
     cfg.stream = (cudaStream_t)stream;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, learn_kernel<ALL3>, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, learn_kernel<ALL3, FOUR>, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+}
+
+// validation shared by the two entry points is done by the callers; this fills the tables and launches (`four`: whether
+// any run at 4 bits is asked for)
+template <bool ALL3>
+lowra_status launch_learn(LearnParams& P, const double* init_levels_host, const double* init_thresholds_host,
+                          bool four, void* stream) {
+    if (((size_t)P.K + (size_t)P.K / kBlock) * sizeof(float) > 160 * 1024) return LOWRA_ERR_SHAPE;   // K <= 40960: the row has to fit
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    for (int c = 0; c < 3; ++c)
+        for (int j = 0; j < 16; ++j) {
+            P.init_y[c][j] = init_levels_host[c * 16 + j];
+            P.init_t[c][j] = init_thresholds_host[c * 16 + j];
+        }
+    return four ? launch_learn_kernel<ALL3, true>(P, stream) : launch_learn_kernel<ALL3, false>(P, stream);
 }
 
 }  // namespace
@@ -282,7 +314,7 @@ extern "C" lowra_status lowra_learn_codebooks(const lowra_layout* layout, const 
     P.iterations = iterations;
     P.N = layout->N;
     P.K = layout->K;
-    return launch_learn<false>(P, init_levels_host, init_thresholds_host, stream);
+    return launch_learn<false>(P, init_levels_host, init_thresholds_host, layout->counts[2] > 0, stream);
 }
 
 extern "C" lowra_status lowra_learn_codebooks_all(int32_t N, int32_t K, const float* W_dev,
@@ -301,5 +333,5 @@ extern "C" lowra_status lowra_learn_codebooks_all(int32_t N, int32_t K, const fl
     P.iterations = iterations;
     P.N = N;
     P.K = K;
-    return launch_learn<true>(P, init_levels_host, init_thresholds_host, stream);
+    return launch_learn<true>(P, init_levels_host, init_thresholds_host, true, stream);
 }

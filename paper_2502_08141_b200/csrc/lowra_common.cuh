@@ -23,6 +23,7 @@ struct RowLayout {
     const uint8_t* precs;         // [N] original order
     const int32_t* perm;          // stored -> original
     const int32_t* inv_perm;      // original -> stored
+    const uint64_t* nat;          // null: grouped order; else [N + 1] byte offsets of the rows in the natural-order buffer
 };
 
 lowra_status check_layout(const lowra_layout* L);
@@ -63,6 +64,12 @@ static inline cudaError_t launch_pdl(void (*kernel)(KArgs...), unsigned grid, un
 // -------------------------------------------------------------------------------------------
 // device helpers
 // -------------------------------------------------------------------------------------------
+// Where stored row p (original row r, class c) lies: byte offset of its codes in the packed buffer, and its absmax row.
+__device__ __forceinline__ size_t packed_row_offset(const RowLayout& L, int c, int p, int r) {
+    return L.nat != nullptr ? (size_t)__ldg(L.nat + r) : (size_t)L.seg_off[c] + (size_t)(p - L.class_start[c]) * (((size_t)L.K << c) >> 3);
+}
+__device__ __forceinline__ int absmax_row_of(const RowLayout& L, int p, int r) { return L.nat != nullptr ? r : p; }
+
 __device__ __forceinline__ int class_of_stored_row(const RowLayout& L, int p) {
     return (p >= L.class_start[1]) + (p >= L.class_start[2]);
 }
