@@ -228,6 +228,27 @@ lowra_status lowra_lora_backward_input(const lowra_layout* layout, const uint8_t
                                        const uint16_t* B_dev, int32_t r, float s, uint16_t* dX_dev,
                                        void* workspace_dev, size_t workspace_bytes, void* stream);
 
+/*
+ * Forward pass for several adapters that share one quantised base weight (Section 4.1, "Adapting LowRA to Production
+ * Use Cases": the thresholds are shared, so there is one packed buffer, and every adapter brings its own mapping
+ * table and its own low-rank factors).  The tokens of the batch are sorted by adapter: adapter a owns the token rows
+ * [group_start_host[a], group_start_host[a + 1]) of X and Y, and for those rows
+ *     Y = X . deq_a(Wq)^T + s * (X . A_a) . B_a
+ * with deq_a the dequantisation through adapter a's mappings.  One call routes every group to its tables; the groups
+ * run back to back on the stream as one fused launch each (a dequantised weight tile depends on the adapter's
+ * mappings, so groups cannot share tiles), empty groups are skipped.
+ *   maps_dev         fp32 [n_adapters][N][16]
+ *   A_dev            bf16 [n_adapters][K][r];   B_dev  bf16 [n_adapters][r][N]
+ *   group_start_host int32 [n_adapters + 1], HOST, non-decreasing, [0] = 0, [n_adapters] = M
+ *   X_dev bf16 [M, K];  Y_dev bf16 [M, N];  workspace_dev: as lowra_lora_forward for M tokens.
+ * Errors: as lowra_lora_forward; n_adapters < 1 or group_start_host not as described -> LOWRA_ERR_SHAPE.
+ */
+lowra_status lowra_lora_forward_adapters(const lowra_layout* layout, const uint8_t* packed_dev, const float* absmax_dev,
+                                         const float* maps_dev, int32_t n_adapters, const uint16_t* X_dev, int32_t M,
+                                         const int32_t* group_start_host, const uint16_t* A_dev, const uint16_t* B_dev,
+                                         int32_t r, float s, uint16_t* Y_dev, void* workspace_dev, size_t workspace_bytes,
+                                         void* stream);
+
 /* Bytes of device scratch that lowra_lora_backward_adapters needs for M tokens and rank r (0 if the
  * arguments are invalid).  The first 256 bytes hold the device status word. */
 size_t lowra_adapter_workspace_bytes(int32_t M, int32_t r);

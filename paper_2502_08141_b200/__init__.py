@@ -30,7 +30,7 @@ EXPORTS = (
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
     "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
     "lowra_channel_errors", "lowra_deal_bytes", "lowra_deal_build", "lowra_workspace_init",
-    "lowra_learn_codebooks_all", "lowra_set_wait_limit", "lowra_diag_wait_expiry", "lowra_diag_drop_t_flags",
+    "lowra_learn_codebooks_all", "lowra_lora_forward_adapters", "lowra_set_wait_limit", "lowra_diag_wait_expiry", "lowra_diag_drop_t_flags",
 )
 
 
@@ -86,6 +86,9 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_forward.restype = ctypes.c_int
         L.lowra_lora_backward_input.argtypes = gemm_args
         L.lowra_lora_backward_input.restype = ctypes.c_int
+        L.lowra_lora_forward_adapters.argtypes = [lp, vp, vp, vp, i32, vp, i32, vp, vp, vp, i32, ctypes.c_float, vp, vp,
+                                                  ctypes.c_size_t, vp]
+        L.lowra_lora_forward_adapters.restype = ctypes.c_int
         L.lowra_lora_forward_static.argtypes = [lp, vp, vp, vp, vp, i32, vp, vp, i32, ctypes.c_float, vp, vp, vp]
         L.lowra_lora_forward_static.restype = ctypes.c_int
         L.lowra_learn_codebooks.argtypes = [lp, vp, vp, vp, i32, vp, vp, vp]
@@ -341,6 +344,32 @@ def lowra_lora_forward(layout: Layout, packed, absmax, maps, X, A, B, s: float,
                                     _ptr(B), r, ctypes.c_float(s), _ptr(Y), _ptr(workspace),
                                     workspace.numel(), _stream(stream))
     _check(code, "lowra_lora_forward")
+    return Y
+
+
+def lowra_lora_forward_adapters(layout: Layout, packed, absmax, maps, X, group_start, A, B, s: float,
+                                Y: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                                stream=None) -> torch.Tensor:
+    """Several adapters on one quantised base weight: maps fp32 [n, N, 16], A bf16 [n, K, r], B bf16 [n, r, N];
+    adapter a owns the token rows group_start[a] .. group_start[a + 1] of X (host sequence of n + 1 ints)."""
+    for t, nm in ((X, "X"), (A, "A"), (B, "B")):
+        _dev(t, torch.bfloat16, nm)
+    _dev(maps, torch.float32, "maps")
+    n, M, r = int(maps.shape[0]), int(X.shape[0]), int(A.shape[2])
+    if (tuple(maps.shape) != (n, layout.N, 16) or tuple(X.shape) != (M, layout.K) or tuple(A.shape) != (n, layout.K, r)
+            or tuple(B.shape) != (n, r, layout.N)):
+        raise ValueError("shape mismatch")
+    gs = np.ascontiguousarray(group_start, dtype=np.int32)
+    if gs.shape != (n + 1,):
+        raise ValueError("group_start must have n_adapters + 1 entries")
+    if Y is None:
+        Y = torch.empty((M, layout.N), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = _workspace(layout, M, r, X.device)
+    code = lib().lowra_lora_forward_adapters(layout.ref, _ptr(packed), _ptr(absmax), _ptr(maps), n, _ptr(X), M,
+                                             gs.ctypes.data_as(ctypes.c_void_p), _ptr(A), _ptr(B), r, ctypes.c_float(s),
+                                             _ptr(Y), _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(code, "lowra_lora_forward_adapters")
     return Y
 
 

@@ -298,6 +298,33 @@ extern "C" lowra_status lowra_lora_backward_input(const lowra_layout* layout, co
                            workspace_dev, workspace_bytes, stream);
 }
 
+extern "C" lowra_status lowra_lora_forward_adapters(const lowra_layout* layout, const uint8_t* packed_dev,
+                                                    const float* absmax_dev, const float* maps_dev, int32_t n_adapters,
+                                                    const uint16_t* X_dev, int32_t M, const int32_t* group_start_host,
+                                                    const uint16_t* A_dev, const uint16_t* B_dev, int32_t r, float s,
+                                                    uint16_t* Y_dev, void* workspace_dev, size_t workspace_bytes,
+                                                    void* stream) {
+    using namespace lowra;
+    lowra_status st = check_layout(layout);
+    if (st != LOWRA_OK) return st;
+    if (!maps_dev || !X_dev || !A_dev || !B_dev || !Y_dev || !group_start_host) return LOWRA_ERR_NULL;
+    if (n_adapters < 1 || M < 1 || !rank_ok(r) || group_start_host[0] != 0 || group_start_host[n_adapters] != M)
+        return LOWRA_ERR_SHAPE;
+    for (int a = 0; a < n_adapters; ++a)
+        if (group_start_host[a + 1] < group_start_host[a]) return LOWRA_ERR_SHAPE;
+    const size_t N = (size_t)layout->N, K = (size_t)layout->K;
+    if (workspace_bytes < lowra_workspace_bytes(layout, M, r)) return LOWRA_ERR_WORKSPACE;
+    for (int a = 0; a < n_adapters; ++a) {
+        const int m0 = group_start_host[a], m = group_start_host[a + 1] - m0;
+        if (m == 0) continue;
+        st = run_lora(false, layout, packed_dev, absmax_dev, maps_dev + (size_t)a * N * kTableStride, X_dev + (size_t)m0 * K, m,
+                      A_dev + (size_t)a * K * (size_t)r, B_dev + (size_t)a * (size_t)r * N, r, s, Y_dev + (size_t)m0 * N,
+                      workspace_dev, workspace_bytes, stream);
+        if (st != LOWRA_OK) return st;
+    }
+    return LOWRA_OK;
+}
+
 // ---------------------------------------------------------------------------------------------------
 // Forward without caller-provided scratch, for callers that may not allocate device memory.
 // The scratch is this fixed array: part of the library image, present on every GPU that loads it.
