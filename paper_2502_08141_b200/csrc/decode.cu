@@ -42,42 +42,61 @@ struct WarpStage {
     float lut[16];       // 4-bit rows: the row's levels
 };
 
-template <int B>
-__device__ __forceinline__ void decode_piece(const DecodeParams& P, int p, int piece, int lane, WarpStage* ws) {
-    constexpr int c = B >> 1;              // class index of B bits
-    constexpr int kElemsPiece = 4096 / B;  // elements in a full piece
-    constexpr int kIters = 8 / B;          // 512 elements per iteration
-    constexpr int kBlocks = kElemsPiece / kBlock;
+// What a warp fetches for one piece, held in registers while the previous piece is being expanded.
+struct Fetched {
+    uint4 packed;        // this lane's 16 packed bytes
+    float a0, a1;        // absmax of blocks lane and lane + 32 of the piece
+    float m0, m1, m2, m3;   // 1 bit: levels 0, 1; 2 bits: levels 0 .. 3; 4 bits: m0 = level `lane` (lanes 0 .. 15)
+    int c, r, e0;        // class, original row, first element of the piece
+};
+
+__device__ __forceinline__ void locate(const DecodeParams& P, uint32_t t, int& c, int& p, int& piece) {
+    c = (t >= P.task_start[1]) + (t >= P.task_start[2]);
+    const uint32_t local = t - P.task_start[c];
+    const uint32_t ppr = P.pieces_per_row[c];
+    const int q = local / ppr;
+    piece = local - q * ppr;
+    p = P.L.class_start[c] + q;
+}
+
+__device__ __forceinline__ void fetch_piece(const DecodeParams& P, uint32_t t, int lane, Fetched& f) {
+    int c, p, piece;
+    locate(P, t, c, p, piece);
     const int K = P.L.K;
     const int r = __ldg(P.L.perm + p);
-    const size_t row_bytes = (size_t)K * B / 8;
+    const size_t row_bytes = ((size_t)K << c) >> 3;
     const uint8_t* row = P.packed + packed_row_offset(P.L, c, p, r);
     const size_t byte0 = (size_t)piece * 512 + (size_t)lane * 16;
-    const int e0 = piece * kElemsPiece;                         // first element of the piece
+    const int e0 = piece * (4096 >> c);                          // first element of the piece
+    const int kBlocks = 64 >> c;                                 // blocks in a full piece
     const float* arow = P.absmax + (size_t)absmax_row_of(P.L, p, r) * P.L.nb + e0 / kBlock;
-    const int blocks_left = P.L.nb - e0 / kBlock;               // blocks of the row from e0 on
+    const int blocks_left = P.L.nb - e0 / kBlock;                // blocks of the row from e0 on
     const float* mrow = P.maps + (size_t)r * kTableStride;
-
-    // stage the piece
-    ws->packed[lane] = (byte0 < row_bytes) ? ld_stream_v4(row + byte0) : make_uint4(0u, 0u, 0u, 0u);
-#pragma unroll
-    for (int i = 0; i < kBlocks; i += 32)
-        if (i + lane < kBlocks) ws->absmax[i + lane] = (i + lane < blocks_left) ? __ldg(arow + i + lane) : 0.0f;
-    float m0 = 0.f, m1 = 0.f, m2 = 0.f, m3 = 0.f;
-    if (B == 4) {
-        if (lane < 16) ws->lut[lane] = __ldg(mrow + lane);
+    f.packed = (byte0 < row_bytes) ? ld_stream_v4(row + byte0) : make_uint4(0u, 0u, 0u, 0u);
+    f.a0 = (lane < kBlocks && lane < blocks_left) ? __ldg(arow + lane) : 0.0f;
+    f.a1 = (lane + 32 < kBlocks && lane + 32 < blocks_left) ? __ldg(arow + lane + 32) : 0.0f;
+    f.m0 = f.m1 = f.m2 = f.m3 = 0.0f;
+    if (c == 2) {
+        if (lane < 16) f.m0 = __ldg(mrow + lane);
     } else {
-        m0 = __ldg(mrow); m1 = __ldg(mrow + 1);
-        if (B == 2) { m2 = __ldg(mrow + 2); m3 = __ldg(mrow + 3); }
+        f.m0 = __ldg(mrow); f.m1 = __ldg(mrow + 1);
+        if (c == 1) { f.m2 = __ldg(mrow + 2); f.m3 = __ldg(mrow + 3); }
     }
-    __syncwarp();
+    f.c = c; f.r = r; f.e0 = e0;
+}
 
-    uint16_t* dst = P.out + (size_t)r * K + e0 + lane * 16;
+// Expands the piece parked in the warp's stage: lane l, in round j, elements e0 + 512 j + 16 l .. + 15.
+template <int B>
+__device__ __forceinline__ void expand_piece(const DecodeParams& P, const Fetched& f, int lane, const WarpStage* ws) {
+    constexpr int kIters = 8 / B;          // 512 elements per iteration
+    const int K = P.L.K;
+    uint16_t* dst = P.out + (size_t)f.r * K + f.e0 + lane * 16;
     const unsigned char* bytes = reinterpret_cast<const unsigned char*>(ws->packed);
+    const float m0 = f.m0, m1 = f.m1, m2 = f.m2, m3 = f.m3;
 #pragma unroll
     for (int j = 0; j < kIters; ++j) {
         // lane l: elements e0 + 512 j + 16 l .. + 15, i.e. bits [(512 j + 16 l) B, + 16 B) of the piece
-        const int e = e0 + 512 * j + 16 * lane;
+        const int e = f.e0 + 512 * j + 16 * lane;
         const float a = ws->absmax[8 * j + (lane >> 2)];
         uint32_t o[8];
         if (B == 1) {
@@ -85,10 +104,10 @@ __device__ __forceinline__ void decode_piece(const DecodeParams& P, int p, int p
             const uint32_t LH = pack_bf16x2(__fmul_rn(m0, a), __fmul_rn(m1, a));
             const uint32_t L = LH & 0xFFFFu, H = LH >> 16;
             const uint32_t lo = min(L, H);
-            const uint32_t BB = lo * 0x10001u, d = max(L, H) - lo, f = (L > H) ? 0x10001u : 0u;
+            const uint32_t BB = lo * 0x10001u, d = max(L, H) - lo, fl = (L > H) ? 0x10001u : 0u;
             const uint32_t z = h | (h << 15);   // pair i at bits 0 and 16 of z >> 2i
 #pragma unroll
-            for (int i = 0; i < 8; ++i) o[i] = (((z >> (2 * i)) & 0x10001u) ^ f) * d + BB;
+            for (int i = 0; i < 8; ++i) o[i] = (((z >> (2 * i)) & 0x10001u) ^ fl) * d + BB;
         } else if (B == 2) {
             const uint32_t w = *reinterpret_cast<const uint32_t*>(bytes + 128 * j + 4 * lane);
             const uint32_t E01 = pack_bf16x2(__fmul_rn(m0, a), __fmul_rn(m1, a));
@@ -109,7 +128,6 @@ __device__ __forceinline__ void decode_piece(const DecodeParams& P, int p, int p
         }
         if (e < K) st_stream_v8(dst + 512 * j, o);
     }
-    __syncwarp();  // the stage is reused by the warp's next piece
 }
 
 __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const DecodeParams P) {
@@ -120,16 +138,27 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const DecodePara
     pdl_enter();
     const uint32_t n_tasks = P.task_start[3];
     const uint32_t stride = gridDim.x * kDecodeWarps;
-    for (uint32_t t = blockIdx.x * kDecodeWarps + warp; t < n_tasks; t += stride) {
-        const int c = (t >= P.task_start[1]) + (t >= P.task_start[2]);
-        const uint32_t local = t - P.task_start[c];
-        const uint32_t ppr = P.pieces_per_row[c];
-        const int q = local / ppr;
-        const int piece = local - q * ppr;
-        const int p = P.L.class_start[c] + q;
-        if (c == 0) decode_piece<1>(P, p, piece, lane, ws);
-        else if (c == 1) decode_piece<2>(P, p, piece, lane, ws);
-        else decode_piece<4>(P, p, piece, lane, ws);
+    uint32_t t = blockIdx.x * kDecodeWarps + warp;
+    if (t >= n_tasks) return;
+    // The loads of the warp's next piece are in flight while the current one is expanded and written.
+    Fetched cur, nxt;
+    fetch_piece(P, t, lane, cur);
+    for (;;) {
+        ws->packed[lane] = cur.packed;
+        ws->absmax[lane] = cur.a0;
+        ws->absmax[lane + 32] = cur.a1;
+        if (cur.c == 2 && lane < 16) ws->lut[lane] = cur.m0;
+        __syncwarp();
+        const uint32_t tn = t + stride;
+        const bool more = tn < n_tasks;
+        if (more) fetch_piece(P, tn, lane, nxt);
+        if (cur.c == 0) expand_piece<1>(P, cur, lane, ws);
+        else if (cur.c == 1) expand_piece<2>(P, cur, lane, ws);
+        else expand_piece<4>(P, cur, lane, ws);
+        if (!more) break;
+        __syncwarp();  // the stage is reused by the warp's next piece
+        cur = nxt;
+        t = tn;
     }
 }
 

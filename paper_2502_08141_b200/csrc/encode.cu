@@ -136,7 +136,7 @@ __device__ __forceinline__ void encode_chunk(const EncodeParams& P, int p, int c
     }
 }
 
-__global__ void __launch_bounds__(kEncodeThreads) encode_kernel(const EncodeParams P) {
+__global__ void __launch_bounds__(kEncodeThreads, 3) encode_kernel(const EncodeParams P) {
     __shared__ __align__(16) unsigned char stage_all[kEncodeWarps][32 * kSegBytes];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
