@@ -205,7 +205,10 @@ lowra_status lowra_workspace_init(void* workspace_dev, size_t workspace_bytes, v
  *   X_dev bf16 [M, K];  A_dev bf16 [K, r];  B_dev bf16 [r, N];  Y_dev bf16 [M, N], original
  *   channel order; all row-major.  r in {16, 32, ..., 128}.  X . A is rounded to bf16 once.
  *   workspace_dev: >= lowra_workspace_bytes(layout, M, r) bytes, 256-byte aligned, contents
- *   overwritten.  Calls that share a workspace must not overlap on the device.  With
+ *   overwritten.  Calls that share a workspace must not overlap on the device; and a call must have the
+ *   device's SMs to itself while it runs: its grid is persistent (one CTA per SM) and its CTAs wait for one
+ *   another, so they all have to be resident - do not run another kernel beside it on a second stream (the
+ *   call would sit in its bounded waits and end with LOWRA_ERR_TIMEOUT).  With
  *   layout->deal_dev set: initialised by lowra_workspace_init and since then written by these calls only
  *   (any mix of forward / backward-input, weights and token counts).
  *   Limits (LOWRA_ERR_SHAPE otherwise): N % 8 == 0, N <= 524288, N * K / 64 < 2^32, M >= 1.
