@@ -267,6 +267,25 @@ def run_gpu(args):
     for M in token_counts:
         for wdt in widths:
             act_dev[(M, wdt)] = bfv(torch.from_numpy(si.activations(M, wdt, matrix_id=100 + rank).view(np.int16)).cuda())
+    # Inputs per matrix: the projections that read the same activations in a decoder layer share X (q, k, v; gate and
+    # up), every other matrix has its own; every matrix has its own output gradient.  Distinct buffers are the width's
+    # seeded buffer rotated by a few token rows (the first matrix of the workload keeps the unrotated one).
+    GROUPS = {"q_proj": "qkv", "k_proj": "qkv", "v_proj": "qkv", "gate_proj": "gate_up", "up_proj": "gate_up"}
+    x_groups, x_bufs, g_bufs = [], {}, {}
+    for i, d in enumerate(dev):
+        d["group"] = GROUPS.get(d["name"], d["name"])
+        if d["group"] not in x_groups:
+            x_groups.append(d["group"])
+        gi, j = x_groups.index(d["group"]) % 7, i % 7
+        d["X"], d["G"] = {}, {}
+        for M in token_counts:
+            kx, kg = (M, d["K"], gi), (M, d["N"], j)
+            if kx not in x_bufs:
+                x_bufs[kx] = act_dev[(M, d["K"])] if gi == 0 else torch.roll(act_dev[(M, d["K"])], 37 * gi, dims=0)
+            if kg not in g_bufs and with_backward:
+                g_bufs[kg] = act_dev[(M, d["N"])] if j == 0 else torch.roll(act_dev[(M, d["N"])], 53 * j, dims=0)
+            d["X"][M] = x_bufs[kx]
+            d["G"][M] = g_bufs.get(kg)
     shared_out = len(dev) > 8
     out_shared = {}
 
@@ -308,13 +327,43 @@ def run_gpu(args):
 
     f_encode = lambda d, M=None: lw.lowra_encode(d["layout"], d["W"], d["thr"], packed=d["packed"], absmax=d["absmax"])
     f_decode = lambda d, M=None: lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=d["What"])
-    f_forward = lambda d, M: lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], act_dev[(M, d["K"])],
+    f_forward = lambda d, M: lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], d["X"][M],
                                                    d["A"], d["B"], s, Y=d["Y"][M], workspace=d["ws"][M])
-    f_backward = lambda d, M: lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], act_dev[(M, d["N"])],
+    f_backward = lambda d, M: lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], d["G"][M],
                                                            d["A"], d["B"], s, dX=d["dX"][M], workspace=d["ws"][M])
     phase_list = [("encode", f_encode, [None]), ("decode", f_decode, [None]), ("forward", f_forward, token_counts)]
     if with_backward:
         phase_list.append(("backward", f_backward, token_counts))
+    # The q, k and v projections of a layer (one shape, one input) go through the one-launch batch calls, as a layer
+    # would issue them; everything else is a call per matrix.  units: lists of matrix indices, one list per launch.
+    units, i = [], 0
+    while i < len(dev):
+        j = i + 1
+        if dev[i]["group"] == "qkv" and not args.deal_per_call and not args.no_batch and not shared_out:
+            while (j < len(dev) and j - i < 4 and dev[j]["group"] == "qkv" and (dev[j]["N"], dev[j]["K"]) == (dev[i]["N"], dev[i]["K"])):
+                j += 1
+        units.append(list(range(i, j)))
+        i = j
+    batch_ws, batch_members = {}, {}
+    for u in units:
+        if len(u) > 1:
+            for M in token_counts:
+                n = lw.lowra_batch_workspace_bytes(dev[u[0]]["layout"], len(u), M, r)
+                batch_ws[(u[0], M)] = lw.lowra_workspace_init(torch.empty(n, dtype=torch.uint8, device="cuda"))
+                common = lambda d: dict(layout=d["layout"], packed=d["packed"], absmax=d["absmax"], maps=d["maps"], A=d["A"], B=d["B"])
+                batch_members[("forward", u[0], M)] = [dict(common(dev[k]), act=dev[k]["X"][M], out=dev[k]["Y"][M]) for k in u]
+                if with_backward:
+                    batch_members[("backward", u[0], M)] = [dict(common(dev[k]), act=dev[k]["G"][M], out=dev[k]["dX"][M]) for k in u]
+            all_ws.extend(batch_ws[(u[0], M)] for M in token_counts)
+
+    def run_unit(name, fn, u, M):
+        if len(u) == 1 or name in ("encode", "decode"):
+            for k in u:
+                fn(dev[k], M)
+        elif name == "forward":
+            lw.lowra_lora_forward_batch(batch_members[(name, u[0], M)], s, batch_ws[(u[0], M)])
+        else:
+            lw.lowra_lora_backward_input_batch(batch_members[(name, u[0], M)], s, batch_ws[(u[0], M)])
 
     def step(record=None, per_call=None):
         """One pass.  `record` (a list) receives (phase, event_start, event_end) per phase: the calls of a phase
@@ -324,13 +373,14 @@ def run_gpu(args):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(stream)
             for M in Ms:
-                for i, d in enumerate(dev):
-                    if per_call is not None:
+                if per_call is not None:          # diagnostic pass: a call per matrix, events around each
+                    for i, d in enumerate(dev):
                         c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                         c0.record(stream); fn(d, M); c1.record(stream)
                         per_call.append((name, M, i, c0, c1))
-                    else:
-                        fn(d, M)
+                else:
+                    for u in units:
+                        run_unit(name, fn, u, M)
             if record is not None:
                 e1.record(stream)
                 record.append((name, e0, e1))
@@ -513,7 +563,7 @@ def run_gpu(args):
                                                           with_backward=with_backward))
 
     if rank == 0:
-        n_fused = len(fused_calls)
+        n_fused = len(units) * len(token_counts) * (2 if with_backward else 1)     # fused launches per step
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": n_warm, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
@@ -525,6 +575,11 @@ def run_gpu(args):
                        "l2": f"inputs larger than L2 ({(elems * 4 + out_layer) / 1e9:.1f} GB of weights read and written per step)",
                        "row_deal": "in every call (prologue launch)" if args.deal_per_call else
                                    "once per weight (lowra_deal_build), outside the step like the storage plan",
+                       "launches": "one call per matrix" if all(len(u) == 1 for u in units) else
+                                   "q, k and v projections (one shape, one input) through lowra_lora_forward_batch / "
+                                   "lowra_lora_backward_input_batch, one launch per direction; every other matrix a call "
+                                   "of its own; per_matrix figures are single calls",
+                       "inputs": "q/k/v share X, gate/up share X, every other matrix its own; one output gradient per matrix",
                        "host_generation_s": round(t_gen, 1)},
             "phases": phases, "per_matrix": per_matrix, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "extras": extras,
             "gpu_launches": args.steps * (2 * len(dev) + n_fused * (2 if args.deal_per_call else 1)), "clocks": clocks,
@@ -957,6 +1012,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-batch", action="store_true", help="a fused call per matrix, also for the q, k and v projections")
     ap.add_argument("--deal-per-call", action="store_true",
                     help="fused calls work out the row deal in a prologue launch of their own (no lowra_deal_build)")
     args = ap.parse_args()

@@ -30,7 +30,8 @@ EXPORTS = (
     "lowra_lora_forward_static", "lowra_learn_codebooks", "lowra_adapter_workspace_bytes",
     "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
     "lowra_channel_errors", "lowra_deal_bytes", "lowra_deal_build", "lowra_workspace_init",
-    "lowra_learn_codebooks_all", "lowra_lora_forward_adapters", "lowra_set_wait_limit", "lowra_diag_wait_expiry", "lowra_diag_drop_t_flags",
+    "lowra_learn_codebooks_all", "lowra_lora_forward_adapters", "lowra_batch_workspace_bytes",
+    "lowra_lora_forward_batch", "lowra_lora_backward_input_batch", "lowra_set_wait_limit", "lowra_diag_wait_expiry", "lowra_diag_drop_t_flags",
 )
 
 
@@ -49,6 +50,12 @@ class _CLayout(ctypes.Structure):
         ("precs_dev", ctypes.c_void_p), ("perm_dev", ctypes.c_void_p), ("inv_perm_dev", ctypes.c_void_p),
         ("deal_dev", ctypes.c_void_p), ("natural_offsets_dev", ctypes.c_void_p),
     ]
+
+
+class _CMember(ctypes.Structure):
+    _fields_ = [("layout", ctypes.POINTER(_CLayout)), ("packed_dev", ctypes.c_void_p), ("absmax_dev", ctypes.c_void_p),
+                ("maps_dev", ctypes.c_void_p), ("act_dev", ctypes.c_void_p), ("A_dev", ctypes.c_void_p),
+                ("B_dev", ctypes.c_void_p), ("out_dev", ctypes.c_void_p)]
 
 
 _lib = None
@@ -89,6 +96,13 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_forward_adapters.argtypes = [lp, vp, vp, vp, i32, vp, i32, vp, vp, vp, i32, ctypes.c_float, vp, vp,
                                                   ctypes.c_size_t, vp]
         L.lowra_lora_forward_adapters.restype = ctypes.c_int
+        L.lowra_batch_workspace_bytes.argtypes = [lp, i32, i32, i32]
+        L.lowra_batch_workspace_bytes.restype = ctypes.c_size_t
+        batch_args = [ctypes.POINTER(_CMember), i32, i32, i32, ctypes.c_float, vp, ctypes.c_size_t, vp]
+        L.lowra_lora_forward_batch.argtypes = batch_args
+        L.lowra_lora_forward_batch.restype = ctypes.c_int
+        L.lowra_lora_backward_input_batch.argtypes = batch_args
+        L.lowra_lora_backward_input_batch.restype = ctypes.c_int
         L.lowra_lora_forward_static.argtypes = [lp, vp, vp, vp, vp, i32, vp, vp, i32, ctypes.c_float, vp, vp, vp]
         L.lowra_lora_forward_static.restype = ctypes.c_int
         L.lowra_learn_codebooks.argtypes = [lp, vp, vp, vp, i32, vp, vp, vp]
@@ -345,6 +359,44 @@ def lowra_lora_forward(layout: Layout, packed, absmax, maps, X, A, B, s: float,
                                     workspace.numel(), _stream(stream))
     _check(code, "lowra_lora_forward")
     return Y
+
+
+def lowra_batch_workspace_bytes(layout: Layout, count: int, M: int, r: int) -> int:
+    return int(lib().lowra_batch_workspace_bytes(layout.ref, int(count), int(M), int(r)))
+
+
+def _batch(fn_name: str, members, s: float, workspace: torch.Tensor, backward: bool, stream=None):
+    """members: sequence of dicts with layout, packed, absmax, maps, act, A, B, out (device tensors)."""
+    n = len(members)
+    arr = (_CMember * n)()
+    M = int(members[0]["act"].shape[0])
+    r = int(members[0]["A"].shape[1])
+    for i, m in enumerate(members):
+        lay = m["layout"]
+        for key in ("act", "A", "B", "out"):
+            _dev(m[key], torch.bfloat16, key)
+        act_cols, out_cols = (lay.N, lay.K) if backward else (lay.K, lay.N)
+        if (tuple(m["act"].shape) != (M, act_cols) or tuple(m["out"].shape) != (M, out_cols) or
+                tuple(m["A"].shape) != (lay.K, r) or tuple(m["B"].shape) != (r, lay.N)):
+            raise ValueError("shape mismatch in member %d" % i)
+        arr[i].layout = ctypes.pointer(lay.c)
+        arr[i].packed_dev, arr[i].absmax_dev, arr[i].maps_dev = m["packed"].data_ptr(), m["absmax"].data_ptr(), m["maps"].data_ptr()
+        arr[i].act_dev, arr[i].A_dev, arr[i].B_dev, arr[i].out_dev = (m["act"].data_ptr(), m["A"].data_ptr(), m["B"].data_ptr(),
+                                                                     m["out"].data_ptr())
+    code = getattr(lib(), fn_name)(arr, n, M, r, ctypes.c_float(s), _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(code, fn_name)
+    return [m["out"] for m in members]
+
+
+def lowra_lora_forward_batch(members, s: float, workspace: torch.Tensor, stream=None):
+    """Several weights of one shape in one launch: Y_i = X_i deq(Wq_i)^T + s (X_i A_i) B_i.  `members`: dicts with
+    layout (carrying a deal), packed, absmax, maps, act (X_i), A, B, out (Y_i).  Returns the outputs."""
+    return _batch("lowra_lora_forward_batch", members, s, workspace, False, stream)
+
+
+def lowra_lora_backward_input_batch(members, s: float, workspace: torch.Tensor, stream=None):
+    """The input gradients of several weights of one shape in one launch; act = dY_i, out = dX_i."""
+    return _batch("lowra_lora_backward_input_batch", members, s, workspace, True, stream)
 
 
 def lowra_lora_forward_adapters(layout: Layout, packed, absmax, maps, X, group_start, A, B, s: float,

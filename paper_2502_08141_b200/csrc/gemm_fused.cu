@@ -167,16 +167,17 @@ struct Seg {
     bool part;     // the slice does not start its tile: its fp32 sums go to this cluster's partial-tile slot
     bool pre;      // the slice starts its tile but does not end it: the accumulator is preloaded with the partial
                    // tiles of the clusters that hold the rest
+    int prob;      // which weight of the batch
     int rt, mt;    // row tile, token tile
     int kb0, kb1;  // contraction blocks [kb0, kb1) of the tile
     int tile;      // weight tile index (stream-K)
 };
 
 // WIDE: the weight has no 4-bit rows, so nobody needs the level tables and their 16 KB hold a sixth weight slot.
-template <int MODE, bool WIDE>
+// NB: members the kernel's parameters have room for (1: the plain calls; kMaxBatch: the batch calls).
+template <int MODE, bool WIDE, int NB>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmT,
-             const __grid_constant__ CUtensorMap tmFt, const __grid_constant__ CUtensorMap tmFl) {
+fused_kernel(const __grid_constant__ KParams<NB> P, const __grid_constant__ KMaps<NB> TM) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* base = smem_raw;                   // operand ring (the swizzled tiles need 1024-byte alignment)
     unsigned char* out_s = base + kSmemRingMax;       // epilogue staging
@@ -201,8 +202,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     auto b_slot = [&](uint32_t it) { return base + SA * kSmemA + (it % SB) * kSmemB; };
     const int cid = (int)blockIdx.x / CL, NC = (int)gridDim.x / CL;   // this cluster, clusters in the grid
     const int super_t = (P.tiles_t + CL - 1) / CL;          // groups of CL token tiles
-    const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? super_t : 0;
-    const int n_tiles = n_t_tiles + P.tiles_r * super_t;    // per cluster
+    const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? P.count * super_t : 0;   // all members' T tiles come first
+    const int tiles_w = P.tiles_r * super_t;                // weight tiles of one member (per cluster)
+    const int n_tiles = n_t_tiles + P.count * tiles_w;      // per cluster
     const int B = P.main_blocks + P.lora_blocks;            // contraction blocks of a weight tile
     // Schedule.  The pieces of work are numbered g = 0, 1, ...: first the T tiles, then the weight tiles; cluster c
     // takes g = c, c + NC, c + 2 NC, ... ("rows" of NC pieces; the clusters then sweep the contraction in step and
@@ -224,12 +226,16 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         Seg t;
         t.part = t.pre = false;
         t.tile = 0;
+        t.prob = 0;
         if (!sk || i < w_dp) {
             const int g = cid + i * NC;
             if (g < n_t_tiles) {
-                t.is_t = true; t.rt = 0; t.mt = g * CL + (int)crank; t.kb0 = 0; t.kb1 = P.main_blocks;
+                t.prob = (NB == 1) ? 0 : g / super_t;
+                t.is_t = true; t.rt = 0; t.mt = (g - t.prob * super_t) * CL + (int)crank; t.kb0 = 0; t.kb1 = P.main_blocks;
             } else {
-                const int idx = g - n_t_tiles;
+                int idx = g - n_t_tiles;
+                t.prob = (NB == 1) ? 0 : idx / tiles_w;
+                idx -= t.prob * tiles_w;
                 const int st = idx / P.tiles_r;
                 t.is_t = false; t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank; t.kb0 = 0; t.kb1 = B;
             }
@@ -239,7 +245,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             const long long first = (long long)t.tile * B;
             t.kb0 = (k == 0) ? (int)(lo - first) : 0;
             t.kb1 = (hi < first + B) ? (int)(hi - first) : B;
-            const int idx = sk_first + t.tile;
+            int idx = sk_first + t.tile;
+            t.prob = (NB == 1) ? 0 : idx / tiles_w;
+            idx -= t.prob * tiles_w;
             const int st = idx / P.tiles_r;
             t.is_t = false; t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank;
             t.part = t.kb0 > 0;
@@ -271,9 +279,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         for (int c = 0; c < kCluster; ++c) bars->free_upto[c] = 0u;
         for (int c = 0; c < kMaxStagesA; ++c) bars->produced[c] = 0u;
         ptx::fence_barrier_init();
-        ptx::prefetch_tensormap(&tmB);
-        if (P.lora_blocks > 0) { ptx::prefetch_tensormap(&tmT); ptx::prefetch_tensormap(&tmFt); }
-        if (P.lora_blocks > 0 || MODE == kModeDense) ptx::prefetch_tensormap(&tmFl);
+        ptx::prefetch_tensormap(&TM.m[0].tmB);
+        if (P.lora_blocks > 0) { ptx::prefetch_tensormap(&TM.m[0].tmT); ptx::prefetch_tensormap(&TM.m[0].tmFt); }
+        if (P.lora_blocks > 0 || MODE == kModeDense) ptx::prefetch_tensormap(&TM.m[0].tmFl);
     }
     if (warp == 1) ptx::tmem_alloc(&bars->tmem_base, kTmemCols);
     ptx::tc_fence_before();
@@ -300,6 +308,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             for (int i = 0; i < n_segs && !failed; ++i) {
                 const Seg t = seg_at(i);
                 const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
+                const MemberMaps& tm = TM.m[t.prob];
                 for (int kb = t.kb0; kb < t.kb1; ++kb, ++it) {
                     const int s = it % SB;
                     const uint32_t ph = (it / SB) & 1u;
@@ -316,38 +325,38 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                         const int c0 = kb * kTileC;
                         if (MODE == kModeForward) {   // ranks x features from A [K, r]: one 64x64 box per 64 ranks
                             ptx::mbar_arrive_expect_tx(bar, (uint32_t)P.lora_blocks * 8192u + kSmemB);
-                            for (int jb = 0; jb < P.lora_blocks; ++jb) ptx::tma_load_2d(a_s + jb * 8192, &tmFt, jb * 64, c0, bar);
+                            for (int jb = 0; jb < P.lora_blocks; ++jb) ptx::tma_load_2d(a_s + jb * 8192, &tm.tmFt, jb * 64, c0, bar);
                         } else {                      // ranks x channels from B [r, N]: one 64 x 128 box
                             ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
-                            ptx::tma_load_2d(a_s, &tmFt, c0, 0, bar);
+                            ptx::tma_load_2d(a_s, &tm.tmFt, c0, 0, bar);
                         }
-                        ptx::tma_load_2d(b_s, &tmB, c0, m0, bar);
+                        ptx::tma_load_2d(b_s, &tm.tmB, c0, m0, bar);
                     } else if (kb < P.main_blocks) {
                         const int c0 = kb * kTileC;
                         if (MODE == kModeDense) {
                             ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
-                            ptx::tma_load_2d(a_s, &tmFl, c0, r0, bar);
+                            ptx::tma_load_2d(a_s, &tm.tmFl, c0, r0, bar);
                         } else {
                             ptx::mbar_arrive_expect_tx(bar, kSmemB);
                         }
-                        ptx::tma_load_2d(b_s, &tmB, c0, m0, bar);
+                        ptx::tma_load_2d(b_s, &tm.tmB, c0, m0, bar);
                     } else {
                         const int lb = kb - P.main_blocks;
                         if (lb == 0 || kb == t.kb0) {
                             // T of this token tile is written by another CTA: wait for its flag, then make
                             // those generic-proxy writes visible to the TMA (async proxy) reads below
-                            if (!ptx::flag_wait(P.flags + t.mt, want, abort_flag, wait_ns)) { failed = true; bars->abort = 1u; break; }
+                            if (!ptx::flag_wait(P.mem[t.prob].flags + t.mt, want, abort_flag, wait_ns)) { failed = true; bars->abort = 1u; break; }
                             ptx::fence_proxy_async_all();
                         }
                         ptx::mbar_arrive_expect_tx(bar, kSmemA + kSmemB);
                         if (MODE == kModeForward) {   // channels x ranks from B [r, N]: two 64-channel boxes; the dequant
                                                       // warps move the rows into tensor memory in their own row order
-                            ptx::tma_load_2d(a_s, &tmFl, r0, lb * 64, bar);
-                            ptx::tma_load_2d(a_s + 8192, &tmFl, r0 + 64, lb * 64, bar);
+                            ptx::tma_load_2d(a_s, &tm.tmFl, r0, lb * 64, bar);
+                            ptx::tma_load_2d(a_s + 8192, &tm.tmFl, r0 + 64, lb * 64, bar);
                         } else {                      // features x ranks from A [K, r], K-major: one 64 x 128 box
-                            ptx::tma_load_2d(a_s, &tmFl, lb * 64, r0, bar);
+                            ptx::tma_load_2d(a_s, &tm.tmFl, lb * 64, r0, bar);
                         }
-                        ptx::tma_load_2d(b_s, &tmT, lb * 64, m0, bar);
+                        ptx::tma_load_2d(b_s, &tm.tmT, lb * 64, m0, bar);
                     }
                 }
             }
@@ -496,7 +505,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
             const Seg t = seg_at(i);
             const int r0 = t.rt * kTileR, m0 = t.mt * kTileT;
             // a T tile writes the down-projected activations [M, rp] (scaled by s); a weight tile writes Y / dX
-            uint16_t* out = t.is_t ? P.T : P.out;
+            uint16_t* out = t.is_t ? P.mem[t.prob].T : P.mem[t.prob].out;
             const int ld = t.is_t ? P.rp : P.ld_out;
             const int R = t.is_t ? P.rp : P.R;
             const float scale = t.is_t ? P.s : 1.0f;
@@ -606,7 +615,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 if (et == 0) {
                     if (t.is_t) {
                         ptx::fence_proxy_async_all();
-                        if (!P.diag_drop_t_flags) ptx::flag_release(P.flags + t.mt, want);   // (diagnostic: the waits for T run out)
+                        if (!P.diag_drop_t_flags) ptx::flag_release(P.mem[t.prob].flags + t.mt, want);   // (diagnostic: the waits for T run out)
                     } else {
                         ptx::flag_release(P.sk_flags + cid * CL + (int)crank, want);   // one flag per CTA: its half of the slot
                     }
@@ -619,7 +628,6 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         // 64-element absmax block per visit of a stage.
         // Warps 6-8, 10-12, 14, 15: warps 9 and 13 would share the MMA warp's scheduler and idle instead (the MMA
         // warp's instruction latency is what paces the CTA).
-        const int K = P.L.K;
         const int pw = (warp - kFirstProducerWarp) - (warp > 9 ? 1 : 0) - (warp > 13 ? 1 : 0);   // 0 .. kProducerWarps - 1
         const uint32_t tab_warp = ptx::smem_u32(tab_all) + (uint32_t)pw * 2048u;   // this warp's 2 KB of level tables (4-bit rows)
         const uint32_t tab_lane = tab_warp + (uint32_t)lane * 4u;                   // forward: level c of this lane's row at tab_lane + 128 c
@@ -677,6 +685,7 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
         for (int i = 0; i < n_segs && !failed; ++i) {
             const Seg t = seg_at(i);
             const int r0 = t.rt * kTileR;
+            const Member& W = P.mem[t.prob];                    // the weight this piece belongs to
             const uint32_t itb = it0 - (uint32_t)t.kb0;         // running stage index of block kb: itb + kb
             const int kb_end = min(t.kb1, P.main_blocks);       // end of this piece's dequantised blocks
             if (t.is_t) {
@@ -696,21 +705,21 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 // of the tile, roughly in precision order (see the deal in gemm_prep.cu).  A thread keeps its
                 // channel for the whole tile; the packed codes of its next two blocks are already in registers.
                 const int q = pw & 3, wgrp = pw >> 2;
-                const uint32_t item = __ldg(P.items + (size_t)t.rt * kItemStride + q * 32 + lane);
+                const uint32_t item = __ldg(W.items + (size_t)t.rt * kItemStride + q * 32 + lane);
                 const int cls = info_class(item);
                 const int row_local = info_row(item);
                 Levels lv = {0.f, 0.f, 0.f, 0.f};
-                const uint8_t* bits_ptr = P.packed;
-                const float* absmax_ptr = P.absmax;
-                const float* mrow = P.maps;
+                const uint8_t* bits_ptr = W.packed;
+                const float* absmax_ptr = W.absmax;
+                const float* mrow = W.maps;
                 int bits_stride = 0;  // packed bytes per 64-element block
                 if (cls < 3) {
                     const int p = info_pos(item);
                     const int b = 1 << cls;
                     bits_stride = 8 * b;
-                    bits_ptr = P.packed + packed_row_offset(P.L, cls, p, r0 + row_local);
-                    absmax_ptr = P.absmax + (size_t)absmax_row_of(P.L, p, r0 + row_local) * P.L.nb;
-                    mrow = P.maps + (size_t)(r0 + row_local) * kTableStride;
+                    bits_ptr = W.packed + packed_row_offset(W.L, cls, p, r0 + row_local);
+                    absmax_ptr = W.absmax + (size_t)absmax_row_of(W.L, p, r0 + row_local) * W.L.nb;
+                    mrow = W.maps + (size_t)(r0 + row_local) * kTableStride;
                     if (cls == 0) {
                         lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
                     } else if (cls == 1) {
@@ -787,8 +796,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 const int g_first = t.kb0 + (((int)crank - t.kb0) % CL + CL) % CL;
                 const uint32_t n_first = 4u * (uint32_t)(g_first / CL);
                 const uint32_t j_first = n_first > (uint32_t)pw ? (n_first - (uint32_t)pw + kProducerWarps - 1) / kProducerWarps : 0u;
-                const uint32_t* heads = P.heads + list + (size_t)j_first * kListWarps;   // entry j of the piece: heads[j * kListWarps]
-                const uint4* rows = reinterpret_cast<const uint4*>(P.items) + ((size_t)list + (size_t)j_first * kListWarps) * 32 + lane;
+                const uint32_t* heads = W.heads + list + (size_t)j_first * kListWarps;   // entry j of the piece: heads[j * kListWarps]
+                const uint4* rows = reinterpret_cast<const uint4*>(W.items) + ((size_t)list + (size_t)j_first * kListWarps) * 32 + lane;
                 constexpr uint32_t kEnd = 0xFFFFFFFFu;
                 // entry of this visit (0) and of the next one (1): head, row record, codes + absmax, 1/2-bit levels
                 uint32_t head0, head1;
@@ -804,9 +813,9 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
                 auto fetch = [&](Block& blk, Levels& lv, uint32_t head, const uint4& rec, uint32_t tab_slot) {
                     const int cls = (head == kEnd) ? 4 : (int)((rec.w >> 8) & 3u);   // this lane's row
                     if (cls < 3) {
-                        load_block(blk, P.packed + ((size_t)rec.x << 4) + (((size_t)k_first << cls) >> 3),
-                                   P.absmax + rec.y + (k_first >> 6), cls);
-                        const float* mrow = P.maps + rec.z;
+                        load_block(blk, W.packed + ((size_t)rec.x << 4) + (((size_t)k_first << cls) >> 3),
+                                   W.absmax + rec.y + (k_first >> 6), cls);
+                        const float* mrow = W.maps + rec.z;
                         if (cls == 0) {
                             lv.m0 = __ldg(mrow); lv.m1 = __ldg(mrow + 1);
                         } else if (cls == 1) {
@@ -921,9 +930,8 @@ fused_kernel(const GemmParams P, const __grid_constant__ CUtensorMap tmB, const 
     }
 }
 
-template <int MODE, bool WIDE>
-static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
-                                const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
+template <int MODE, bool WIDE, int NB>
+static lowra_status launch_mode(const GemmParams& G, const BatchMaps& TM, cudaStream_t stream) {
     constexpr int CL = (MODE == kModeDense) ? 1 : kCluster;
     // per device: the kernel attribute has been set there, and so many clusters (CL = 1: CTAs) can be resident at once
     static std::mutex mutex;
@@ -952,7 +960,7 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
         if (!configured[dev]) {
             const int sms = device_sm_count();
             if (sms < CL) return LOWRA_ERR_CUDA;
-            if (cudaFuncSetAttribute(fused_kernel<MODE, WIDE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            if (cudaFuncSetAttribute(fused_kernel<MODE, WIDE, NB>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)kGemmSmemBytes) != cudaSuccess)
                 return LOWRA_ERR_CUDA;
             int most = sms / CL;
@@ -960,7 +968,7 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
                 // the persistent schedule needs every cluster of the grid resident (a tile waits for T of another)
                 cfg.gridDim = dim3(sms / CL * CL, 1, 1);
                 int n = 0;
-                if (cudaOccupancyMaxActiveClusters(&n, fused_kernel<MODE, WIDE>, &cfg) != cudaSuccess || n < 1) return LOWRA_ERR_CUDA;
+                if (cudaOccupancyMaxActiveClusters(&n, fused_kernel<MODE, WIDE, NB>, &cfg) != cudaSuccess || n < 1) return LOWRA_ERR_CUDA;
                 if (n < most) most = n;
             }
             max_clusters_of[dev] = most;
@@ -969,8 +977,8 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
         max_clusters = max_clusters_of[dev];
     }
     const int super_t = (G.tiles_t + CL - 1) / CL;
-    const int n_t = (MODE != kModeDense && G.lora_blocks > 0) ? super_t : 0;
-    const int n_tiles = G.tiles_r * super_t + n_t;
+    const int n_t = (MODE != kModeDense && G.lora_blocks > 0) ? G.count * super_t : 0;
+    const int n_tiles = G.count * G.tiles_r * super_t + n_t;
     const int clusters = n_tiles < max_clusters ? n_tiles : max_clusters;
     cfg.gridDim = dim3((unsigned)(clusters * CL), 1, 1);
     GemmParams Q = G;
@@ -986,7 +994,7 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
         const int rows = n_tiles / clusters;
         const int n_last = n_tiles - rows * clusters;                  // pieces of the last, incomplete row
         const size_t slab = (size_t)CL * kTileT * (size_t)G.C * 2u;    // token operand of one group of token tiles
-        const bool operand_fits_l2 = (size_t)G.M * (size_t)G.C * 2u <= ((size_t)48 << 20);
+        const bool operand_fits_l2 = (size_t)G.operand_bytes <= ((size_t)48 << 20);
         int dp = 0, late = 1;
         if (operand_fits_l2 && rows >= 3) {
             dp = 1; late = 0;
@@ -1007,20 +1015,31 @@ static lowra_status launch_mode(const GemmParams& G, const CUtensorMap& tmB, con
             Q.sk_total = n_rest * blocks;
         }
     }
-    if (cudaLaunchKernelEx(&cfg, fused_kernel<MODE, WIDE>, Q, tmB, tmT, tmFt, tmFl) != cudaSuccess) return LOWRA_ERR_CUDA;
+    KParams<NB> QP;
+    KMaps<NB> QM;
+    static_cast<GemmCommon&>(QP) = static_cast<const GemmCommon&>(Q);
+    for (int i = 0; i < NB; ++i) { QP.mem[i] = Q.mem[i]; QM.m[i] = TM.m[i]; }
+    if (cudaLaunchKernelEx(&cfg, fused_kernel<MODE, WIDE, NB>, QP, QM) != cudaSuccess) return LOWRA_ERR_CUDA;
     return LOWRA_OK;
 }
 
-lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
-                          const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream) {
-    const bool wide = G.L.class_start[3] == G.L.class_start[2];   // no 4-bit rows: the table cache becomes a weight slot
-    if (mode == kModeForward)
-        return wide ? launch_mode<kModeForward, true>(G, tmB, tmT, tmFt, tmFl, stream)
-                    : launch_mode<kModeForward, false>(G, tmB, tmT, tmFt, tmFl, stream);
-    if (mode == kModeBackward)
-        return wide ? launch_mode<kModeBackward, true>(G, tmB, tmT, tmFt, tmFl, stream)
-                    : launch_mode<kModeBackward, false>(G, tmB, tmT, tmFt, tmFl, stream);
-    return launch_mode<kModeDense, false>(G, tmB, tmT, tmFt, tmFl, stream);
+template <int MODE>
+static lowra_status launch_variant(const GemmParams& G, const BatchMaps& TM, cudaStream_t stream) {
+    bool wide = MODE != kModeDense;   // no member has 4-bit rows: the table cache becomes a weight slot
+    for (int i = 0; i < G.count; ++i) wide = wide && G.mem[i].L.class_start[3] == G.mem[i].L.class_start[2];
+    if constexpr (MODE == kModeDense) {
+        return launch_mode<kModeDense, false, 1>(G, TM, stream);
+    } else {
+        if (G.count == 1)
+            return wide ? launch_mode<MODE, true, 1>(G, TM, stream) : launch_mode<MODE, false, 1>(G, TM, stream);
+        return wide ? launch_mode<MODE, true, kMaxBatch>(G, TM, stream) : launch_mode<MODE, false, kMaxBatch>(G, TM, stream);
+    }
+}
+
+lowra_status launch_fused(int mode, const GemmParams& G, const BatchMaps& TM, cudaStream_t stream) {
+    if (mode == kModeForward) return launch_variant<kModeForward>(G, TM, stream);
+    if (mode == kModeBackward) return launch_variant<kModeBackward>(G, TM, stream);
+    return launch_variant<kModeDense>(G, TM, stream);
 }
 
 }  // namespace lowra

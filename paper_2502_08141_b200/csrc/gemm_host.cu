@@ -29,8 +29,8 @@ constexpr size_t kExitsOffset = 128;   //   CTAs of the running call that have l
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Workspace {
-    size_t off_T, off_flags, off_items, off_meta, off_part, total;
-    int rp, n_flags;
+    size_t off_T, t_bytes, off_flags, off_items, off_meta, off_part, total;
+    int rp, t_flags, n_flags;
 };
 
 bool rank_ok(int r) { return r >= 16 && r <= 128 && r % 16 == 0; }
@@ -63,15 +63,18 @@ DealBuffer plan_deal(int N) {
     return d;
 }
 
-Workspace plan_workspace(int N, int K, int M, int r, bool stream_k) {
+Workspace plan_workspace(int N, int K, int M, int r, bool stream_k, int count = 1) {
     (void)K;
     Workspace w;
     w.rp = (r + 63) / 64 * 64;
     const DealSizes z = deal_sizes(N);   // room for the deal of one direction, rebuilt by every call that brings none
     w.off_T = kStatusBytes;
-    w.off_flags = w.off_T + align256((size_t)M * w.rp * 2);
-    // "T ready" flags (a cluster's last token tiles may lie past M), then one "partial tile ready" flag per CTA
-    w.n_flags = (M + kTileT - 1) / kTileT + kCluster + kMaxClusters * kCluster;
+    w.t_bytes = align256((size_t)M * w.rp * 2);                      // per member
+    w.off_flags = w.off_T + (size_t)count * w.t_bytes;
+    // per member the "T ready" flags (a cluster's last token tiles may lie past M), then one "partial tile ready"
+    // flag per CTA
+    w.t_flags = (M + kTileT - 1) / kTileT + kCluster;
+    w.n_flags = count * w.t_flags + kMaxClusters * kCluster;
     w.off_items = w.off_flags + align256((size_t)w.n_flags * 4);
     w.off_meta = w.off_items + align256(z.rows_bytes > z.fwd_bytes ? z.rows_bytes : z.fwd_bytes);
     w.off_part = w.off_meta + align256(z.heads_bytes);
@@ -106,71 +109,98 @@ bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols, u
     return rc == CUDA_SUCCESS;
 }
 
-lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* packed, const float* absmax,
-                      const float* maps, const uint16_t* act, int32_t M, const uint16_t* A, const uint16_t* B,
-                      int32_t r, float s, uint16_t* out, void* workspace, size_t workspace_bytes, void* stream_v,
-                      bool stream_k = true) {
-    lowra_status st = check_layout(layout);
-    if (st != LOWRA_OK) return st;
-    if (!packed || !absmax || !maps || !act || !A || !B || !out || !workspace) return LOWRA_ERR_NULL;
-    const int N = layout->N, K = layout->K;
+// One weight of a fused call, as the entry points receive it.
+struct MemberArgs {
+    const lowra_layout* layout;
+    const uint8_t* packed;
+    const float* absmax;
+    const float* maps;
+    const uint16_t* act;   // X (forward) or dY (backward-input)
+    const uint16_t* A;
+    const uint16_t* B;
+    uint16_t* out;
+};
+
+// Forward / backward-input for `count` weights of one shape in one launch (count == 1: the plain calls).
+lowra_status run_members(bool backward, const MemberArgs* mem, int count, int32_t M, int32_t r, float s, void* workspace,
+                         size_t workspace_bytes, void* stream_v, bool stream_k = true) {
+    if (count < 1 || count > kMaxBatch) return LOWRA_ERR_SHAPE;
+    for (int i = 0; i < count; ++i) {
+        lowra_status st = check_layout(mem[i].layout);
+        if (st != LOWRA_OK) return st;
+        if (!mem[i].packed || !mem[i].absmax || !mem[i].maps || !mem[i].act || !mem[i].A || !mem[i].B || !mem[i].out) return LOWRA_ERR_NULL;
+    }
+    if (!workspace) return LOWRA_ERR_NULL;
+    const int N = mem[0].layout->N, K = mem[0].layout->K;
     if (M < 1 || !rank_ok(r) || N % 8 != 0 || N > 64 * kMaxGroups64 || (uint64_t)N * (uint64_t)(K / 64) >= (1ull << 32))
         return LOWRA_ERR_SHAPE;
-    if (!aligned16(packed) || !aligned16(absmax) || !aligned16(maps) || !aligned16(act) || !aligned16(A) ||
-        !aligned16(B) || !aligned16(out) || (reinterpret_cast<uintptr_t>(layout->deal_dev) & 255u) != 0)
-        return LOWRA_ERR_ALIGN;
-    const Workspace w = plan_workspace(N, K, M, r, stream_k);
+    for (int i = 0; i < count; ++i) {
+        const MemberArgs& m = mem[i];
+        if (m.layout->N != N || m.layout->K != K) return LOWRA_ERR_SHAPE;                 // one shape per launch
+        if (count > 1 && m.layout->deal_dev == nullptr) return LOWRA_ERR_NULL;            // a batch has no prologue launch
+        if (!aligned16(m.packed) || !aligned16(m.absmax) || !aligned16(m.maps) || !aligned16(m.act) || !aligned16(m.A) ||
+            !aligned16(m.B) || !aligned16(m.out) || (reinterpret_cast<uintptr_t>(m.layout->deal_dev) & 255u) != 0)
+            return LOWRA_ERR_ALIGN;
+    }
+    const Workspace w = plan_workspace(N, K, M, r, stream_k, count);
     if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LOWRA_ERR_WORKSPACE;
-    st = check_device();
+    lowra_status st = check_device();
     if (st != LOWRA_OK) return st;
     cudaStream_t stream = (cudaStream_t)stream_v;
 
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     uint32_t* status = reinterpret_cast<uint32_t*>(ws);
-    uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
     uint32_t* flags = reinterpret_cast<uint32_t*>(ws + w.off_flags);
-    uint32_t* items = reinterpret_cast<uint32_t*>(ws + w.off_items);
-    uint32_t* heads = reinterpret_cast<uint32_t*>(ws + w.off_meta);
     const int tiles_t = (M + kTileT - 1) / kTileT;
 
-    if (layout->deal_dev != nullptr) {
-        // the rows were dealt once for this weight (lowra_deal_build) and the workspace numbers its calls
-        // (lowra_workspace_init): nothing to prepare, the fused kernel is the only launch
-        const DealBuffer d = plan_deal(N);
-        unsigned char* deal = static_cast<unsigned char*>(const_cast<void*>(layout->deal_dev));
-        items = reinterpret_cast<uint32_t*>(deal + (backward ? d.off_rows : d.off_fwd));
-        heads = reinterpret_cast<uint32_t*>(deal + d.off_heads);
-    } else {
-        // ---- prologue: clear status and flags, deal the rows
-        PrepParams P;
-        memset(&P, 0, sizeof(P));
-        P.L = make_row_layout(layout);
-        P.precs = layout->precs_dev;
-        P.inv_perm = layout->inv_perm_dev;
-        P.items = items;
-        P.heads = heads;
-        P.N = N;
-        P.group = backward ? 64 : 128;
-        P.status = status;
-        P.exits = reinterpret_cast<uint32_t*>(ws + kExitsOffset);
-        P.flags = flags;
-        P.n_flags = w.n_flags;
-        P.blocks = ((N + P.group - 1) / P.group + 3) / 4;
-        st = launch_prep(P, stream);
-        if (st != LOWRA_OK) return st;
-    }
-
-    // ---- fused kernel (its first tiles compute T = s X A, resp. U = s dY B^T)
     GemmParams G;
     memset(&G, 0, sizeof(G));
-    G.L = make_row_layout(layout);
-    G.packed = packed;
-    G.absmax = absmax;
-    G.maps = maps;
-    G.items = items;
-    G.heads = heads;
-    G.out = out;
-    G.T = T;
+    BatchMaps TM;
+    memset(&TM, 0, sizeof(TM));
+    G.count = count;
+    for (int i = 0; i < count; ++i) {
+        const MemberArgs& m = mem[i];
+        Member& g = G.mem[i];
+        g.L = make_row_layout(m.layout);
+        g.packed = m.packed;
+        g.absmax = m.absmax;
+        g.maps = m.maps;
+        g.out = m.out;
+        g.T = reinterpret_cast<uint16_t*>(ws + w.off_T + (size_t)i * w.t_bytes);
+        g.flags = flags + (size_t)i * w.t_flags;
+        if (m.layout->deal_dev != nullptr) {
+            // the rows were dealt once for this weight (lowra_deal_build) and the workspace numbers its calls
+            // (lowra_workspace_init): nothing to prepare, the fused kernel is the only launch
+            const DealBuffer d = plan_deal(N);
+            const unsigned char* deal = static_cast<const unsigned char*>(m.layout->deal_dev);
+            g.items = reinterpret_cast<const uint32_t*>(deal + (backward ? d.off_rows : d.off_fwd));
+            g.heads = reinterpret_cast<const uint32_t*>(deal + d.off_heads);
+        } else {
+            // ---- prologue: clear status and flags, deal the rows (plain calls only)
+            uint32_t* items = reinterpret_cast<uint32_t*>(ws + w.off_items);
+            uint32_t* heads = reinterpret_cast<uint32_t*>(ws + w.off_meta);
+            PrepParams P;
+            memset(&P, 0, sizeof(P));
+            P.L = g.L;
+            P.precs = m.layout->precs_dev;
+            P.inv_perm = m.layout->inv_perm_dev;
+            P.items = items;
+            P.heads = heads;
+            P.N = N;
+            P.group = backward ? 64 : 128;
+            P.status = status;
+            P.exits = reinterpret_cast<uint32_t*>(ws + kExitsOffset);
+            P.flags = flags;
+            P.n_flags = w.n_flags;
+            P.blocks = ((N + P.group - 1) / P.group + 3) / 4;
+            st = launch_prep(P, stream);
+            if (st != LOWRA_OK) return st;
+            g.items = items;
+            g.heads = heads;
+        }
+    }
+
+    // ---- fused kernel (its first tiles compute T = s X A, resp. U = s dY B^T, of every member)
     G.flags = flags;
     G.status = status;
     G.epoch = reinterpret_cast<uint32_t*>(ws + kEpochOffset);
@@ -179,7 +209,6 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.s = s;
     G.rp = w.rp;
     G.r = r;
-    G.lora_up = B;
     G.M = M;
     G.R = backward ? K : N;
     G.C = backward ? N : K;
@@ -188,27 +217,43 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
     G.lora_blocks = w.rp / kTileC;
     G.tiles_r = (G.R + kTileR - 1) / kTileR;
     G.tiles_t = tiles_t;
+    for (int i = 0; i < count; ++i) {   // token operands: every distinct one once (q, k, v share X in the forward pass)
+        bool seen = false;
+        for (int j = 0; j < i; ++j) seen = seen || mem[j].act == mem[i].act;
+        if (!seen) G.operand_bytes += (long long)M * G.C * 2;
+    }
     G.sk_part = stream_k ? reinterpret_cast<float*>(ws + w.off_part) : nullptr;   // null: whole tiles only
-    G.sk_flags = flags + tiles_t + kCluster;
+    G.sk_flags = flags + (size_t)count * w.t_flags;
     G.wait_ns = wait_limit_ns();
     {   // diagnostic, armed by lowra_diag_drop_t_flags: take one of the calls it asked for
         int left = g_drop_t_flags.load(std::memory_order_relaxed);
         while (left > 0 && !g_drop_t_flags.compare_exchange_weak(left, left - 1, std::memory_order_relaxed)) {}
         G.diag_drop_t_flags = left > 0 ? 1 : 0;
     }
-    CUtensorMap tmB, tmT, tmFt, tmFl;
-    if (!make_map(&tmB, act, (uint64_t)M, (uint64_t)G.C, (uint64_t)G.C, kTileT)) return LOWRA_ERR_CUDA;
-    if (!make_map(&tmT, T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
-    if (!backward) {
-        // T tiles take ranks x features from A [K, r] (64 x 64 boxes); LoRA blocks take channels x ranks from B [r, N]
-        if (!make_map(&tmFt, A, (uint64_t)K, (uint64_t)r, (uint64_t)r, 64)) return LOWRA_ERR_CUDA;
-        if (!make_map(&tmFl, B, (uint64_t)r, (uint64_t)N, (uint64_t)N, 64)) return LOWRA_ERR_CUDA;
-    } else {
-        // T tiles take ranks x channels from B [r, N]; LoRA blocks take features x ranks from A [K, r] (64 x 128 boxes)
-        if (!make_map(&tmFt, B, (uint64_t)r, (uint64_t)N, (uint64_t)N, kTileR)) return LOWRA_ERR_CUDA;
-        if (!make_map(&tmFl, A, (uint64_t)K, (uint64_t)r, (uint64_t)r, kTileR)) return LOWRA_ERR_CUDA;
+    for (int i = 0; i < count; ++i) {
+        const MemberArgs& m = mem[i];
+        MemberMaps& t = TM.m[i];
+        if (!make_map(&t.tmB, m.act, (uint64_t)M, (uint64_t)G.C, (uint64_t)G.C, kTileT)) return LOWRA_ERR_CUDA;
+        if (!make_map(&t.tmT, G.mem[i].T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
+        if (!backward) {
+            // T tiles take ranks x features from A [K, r] (64 x 64 boxes); LoRA blocks take channels x ranks from B [r, N]
+            if (!make_map(&t.tmFt, m.A, (uint64_t)K, (uint64_t)r, (uint64_t)r, 64)) return LOWRA_ERR_CUDA;
+            if (!make_map(&t.tmFl, m.B, (uint64_t)r, (uint64_t)N, (uint64_t)N, 64)) return LOWRA_ERR_CUDA;
+        } else {
+            // T tiles take ranks x channels from B [r, N]; LoRA blocks take features x ranks from A [K, r] (64 x 128 boxes)
+            if (!make_map(&t.tmFt, m.B, (uint64_t)r, (uint64_t)N, (uint64_t)N, kTileR)) return LOWRA_ERR_CUDA;
+            if (!make_map(&t.tmFl, m.A, (uint64_t)K, (uint64_t)r, (uint64_t)r, kTileR)) return LOWRA_ERR_CUDA;
+        }
     }
-    return launch_fused(backward ? kModeBackward : kModeForward, G, tmB, tmT, tmFt, tmFl, stream);
+    return launch_fused(backward ? kModeBackward : kModeForward, G, TM, stream);
+}
+
+lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* packed, const float* absmax,
+                      const float* maps, const uint16_t* act, int32_t M, const uint16_t* A, const uint16_t* B,
+                      int32_t r, float s, uint16_t* out, void* workspace, size_t workspace_bytes, void* stream_v,
+                      bool stream_k = true) {
+    const MemberArgs m = {layout, packed, absmax, maps, act, A, B, out};
+    return run_members(backward, &m, 1, M, r, s, workspace, workspace_bytes, stream_v, stream_k);
 }
 
 // scratch of the adapter-gradient call: status word | T = s X A | U = s dY B^T  (bf16 [M, rp] each)
@@ -296,6 +341,42 @@ extern "C" lowra_status lowra_lora_backward_input(const lowra_layout* layout, co
                                                   void* workspace_dev, size_t workspace_bytes, void* stream) {
     return lowra::run_lora(true, layout, packed_dev, absmax_dev, maps_dev, dY_dev, M, A_dev, B_dev, r, s, dX_dev,
                            workspace_dev, workspace_bytes, stream);
+}
+
+static_assert(LOWRA_MAX_BATCH == lowra::kMaxBatch, "header and kernel agree on the batch limit");
+
+extern "C" size_t lowra_batch_workspace_bytes(const lowra_layout* layout, int32_t count, int32_t M, int32_t r) {
+    using namespace lowra;
+    if (!layout || layout->N < 1 || layout->K < 1 || M < 1 || !rank_ok(r) || count < 1 || count > kMaxBatch) return 0;
+    return plan_workspace(layout->N, layout->K, M, r, true, count).total;
+}
+
+namespace lowra {
+namespace {
+lowra_status run_batch(bool backward, const lowra_member* members, int32_t count, int32_t M, int32_t r, float s,
+                       void* workspace, size_t workspace_bytes, void* stream) {
+    if (!members) return LOWRA_ERR_NULL;
+    if (count < 1 || count > kMaxBatch) return LOWRA_ERR_SHAPE;
+    MemberArgs mem[kMaxBatch];
+    for (int i = 0; i < count; ++i) {
+        const lowra_member& m = members[i];
+        mem[i] = MemberArgs{m.layout, m.packed_dev, m.absmax_dev, m.maps_dev, m.act_dev, m.A_dev, m.B_dev, m.out_dev};
+        if (m.layout != nullptr && m.layout->deal_dev == nullptr) return LOWRA_ERR_NULL;   // also for a batch of one
+    }
+    return run_members(backward, mem, count, M, r, s, workspace, workspace_bytes, stream);
+}
+}  // namespace
+}  // namespace lowra
+
+extern "C" lowra_status lowra_lora_forward_batch(const lowra_member* members_host, int32_t count, int32_t M, int32_t r,
+                                                 float s, void* workspace_dev, size_t workspace_bytes, void* stream) {
+    return lowra::run_batch(false, members_host, count, M, r, s, workspace_dev, workspace_bytes, stream);
+}
+
+extern "C" lowra_status lowra_lora_backward_input_batch(const lowra_member* members_host, int32_t count, int32_t M,
+                                                        int32_t r, float s, void* workspace_dev, size_t workspace_bytes,
+                                                        void* stream) {
+    return lowra::run_batch(true, members_host, count, M, r, s, workspace_dev, workspace_bytes, stream);
 }
 
 extern "C" lowra_status lowra_lora_forward_adapters(const lowra_layout* layout, const uint8_t* packed_dev,
@@ -536,7 +617,10 @@ extern "C" lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_
 
     GemmParams G;
     memset(&G, 0, sizeof(G));
-    G.out = C_dev;
+    BatchMaps TM;
+    memset(&TM, 0, sizeof(TM));
+    G.count = 1;
+    G.mem[0].out = C_dev;
     G.status = status;
     G.M = M;
     G.R = N;
@@ -547,8 +631,9 @@ extern "C" lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_
     G.tiles_r = (N + kTileR - 1) / kTileR;
     G.tiles_t = (M + kTileT - 1) / kTileT;
     G.wait_ns = wait_limit_ns();
-    CUtensorMap tmB, tmFl;
-    if (!make_map(&tmB, P_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, kTileT)) return LOWRA_ERR_CUDA;
-    if (!make_map(&tmFl, Q_dev, (uint64_t)N, (uint64_t)K, (uint64_t)K, kTileR)) return LOWRA_ERR_CUDA;
-    return launch_fused(kModeDense, G, tmB, tmB, tmB, tmFl, stream);
+    if (!make_map(&TM.m[0].tmB, P_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, kTileT)) return LOWRA_ERR_CUDA;
+    if (!make_map(&TM.m[0].tmFl, Q_dev, (uint64_t)N, (uint64_t)K, (uint64_t)K, kTileR)) return LOWRA_ERR_CUDA;
+    TM.m[0].tmT = TM.m[0].tmB;
+    TM.m[0].tmFt = TM.m[0].tmB;
+    return launch_fused(kModeDense, G, TM, stream);
 }

@@ -64,16 +64,36 @@ constexpr int kTmemCols = 512;    // two 128 x 256 fp32 accumulators
 
 constexpr int kModeForward = 0, kModeBackward = 1, kModeDense = 2;
 
-struct GemmParams {
+constexpr int kMaxBatch = 4;      // weights of the same shape that one launch can walk (lowra_lora_*_batch)
+
+// One weight of a call: its quantised state, the deal of its rows, its output, its down-projected activations.
+struct Member {
     RowLayout L;
     const uint8_t* packed;
     const float* absmax;
     const float* maps;
-    const uint32_t* items;    // from the prologue: row words (forward: per tile; backward: per work-list entry)
-    const uint32_t* heads;    // from the prologue (backward): work-list heads
-    uint16_t* out;          // [M, ld_out] bf16
-    uint16_t* T;            // [M, rp] bf16: s * X . A (forward) or s * dY . B^T (backward), written by the T tiles
-    uint32_t* flags;        // [tiles_t] set to the call's number when T of a token tile is complete
+    const uint32_t* items;    // from the deal: row words (forward: per tile; backward: per work-list entry)
+    const uint32_t* heads;    // from the deal (backward): work-list heads
+    uint16_t* out;            // [M, ld_out] bf16
+    uint16_t* T;              // [M, rp] bf16: s * X . A (forward) or s * dY . B^T (backward), written by the T tiles
+    uint32_t* flags;          // [tiles_t + kCluster] set to the call's number when T of a token tile is complete
+};
+
+// Tensor maps of one member: token operand, T, factor of the T tiles, factor of the LoRA blocks.
+struct MemberMaps {
+    CUtensorMap tmB, tmT, tmFt, tmFl;
+};
+template <int NB>
+struct KMaps {
+    MemberMaps m[NB];
+};
+using BatchMaps = KMaps<kMaxBatch>;
+
+// What a launch needs beside its members.  (The kernel is instantiated for one member and for kMaxBatch members: a
+// plain call then carries 0.7 KB of kernel parameters instead of 2.8 KB, which its launch latency shows.)
+struct GemmCommon {
+    int count;              // members (1 for the plain calls); all of one shape
+    uint32_t* flags;        // all flags of the workspace (the members' T flags, then the partial-tile flags)
     uint32_t* status;
     // Calls on one workspace are numbered: `epoch` holds the number of the last call that ran on it, a call's own
     // number is that + 1, and a flag is up when it holds the call's number - so flags left over from earlier calls
@@ -84,14 +104,14 @@ struct GemmParams {
     float s;
     int rp;                 // LoRA rank rounded up to 64
     int r;                  // LoRA rank
-    const uint16_t* lora_up;  // forward: B [r, N] (read by the dequant warps for the LoRA blocks)
     int M;                  // tokens
     int R;                  // A-operand rows in total: N (forward, dense) or K (backward)
     int C;                  // main contraction length: K (forward, dense) or N (backward)
     int ld_out;             // = R
     int main_blocks;        // ceil(C / 64)
     int lora_blocks;        // rp / 64 (0 in dense mode)
-    int tiles_r, tiles_t;
+    int tiles_r, tiles_t;   // per member
+    long long operand_bytes;   // token operands of the call, each distinct one counted once (host: schedule choice)
     // stream-K schedule (set by the launcher; sk == 0: whole tiles, dealt round-robin to the clusters)
     float* sk_part;         // fp32 partial tiles, one [kCluster][kTileT][kTileR] slot per cluster
     uint32_t* sk_flags;     // [clusters] raised when a cluster's partial tile is complete
@@ -103,6 +123,11 @@ struct GemmParams {
     int diag_drop_t_flags;  // diagnostic (lowra_diag_drop_t_flags): the T tiles do not raise their flags, so the waits
                             // for them run out and the call ends with LOWRA_ERR_TIMEOUT
 };
+template <int NB>
+struct KParams : GemmCommon {
+    Member mem[NB];
+};
+using GemmParams = KParams<kMaxBatch>;
 unsigned long long wait_limit_ns();   // the process-wide limit, 1 s unless lowra_set_wait_limit changed it
 constexpr int kMaxClusters = kNumSMs / kCluster;
 constexpr size_t kSkSlotFloats = (size_t)kCluster * kTileT * kTileR;
@@ -123,8 +148,7 @@ static_assert(kStagesA_fwd * kSmemA + kStagesB_fwd * kSmemB + kSmemTab <= kSmemR
 constexpr uint32_t kGemmSmemBytes = kSmemRingMax + kSmemOut + kSmemBarriers;
 static_assert(kGemmSmemBytes <= 232448, "227 KB of shared memory per CTA");
 
-lowra_status launch_fused(int mode, const GemmParams& G, const CUtensorMap& tmB, const CUtensorMap& tmT,
-                          const CUtensorMap& tmFt, const CUtensorMap& tmFl, cudaStream_t stream);
+lowra_status launch_fused(int mode, const GemmParams& G, const BatchMaps& TM, cudaStream_t stream);
 
 // One skinny product D [R, rp] = P . Q (see gemm_grad.cu), written in bf16 as out [R, ld_out] or, transposed,
 // as out [n_cols, ld_out].
