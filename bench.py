@@ -721,6 +721,25 @@ def run_extras(lw, torch, dev, M, act_dev, r, s, stream, P, y0, t0):
                                    "TFLOP/s": ad_flops / (ms * 1e-3) / 1e12,
                                    "note": "not part of the step; algorithmic bytes = X and dY read once"}
 
+    # the same gradients from the down-projections that forward and backward-input leave in their workspaces: X and dY
+    # are read once.  One workspace per direction, so that both projections survive; the fused calls run outside the timing.
+    ws_f = [lw.lowra_workspace_init(torch.empty(lw.lowra_workspace_bytes(d["layout"], M, r), dtype=torch.uint8, device="cuda")) for d in dev]
+    for d, w in zip(dev, ws_f):
+        lw.lowra_lora_forward(d["layout"], d["packed"], d["absmax"], d["maps"], act_dev[(M, d["K"])], d["A"], d["B"], s,
+                              Y=d["Y"][M], workspace=w)
+        lw.lowra_lora_backward_input(d["layout"], d["packed"], d["absmax"], d["maps"], act_dev[(M, d["N"])], d["A"], d["B"], s,
+                                     dX=d["dX"][M] if d["dX"] else None, workspace=d["ws"][M])
+    proj = [(lw.lowra_workspace_projection(w, M, r), lw.lowra_workspace_projection(d["ws"][M], M, r)) for d, w in zip(dev, ws_f)]
+    ms = timed(lambda: [lw.lowra_lora_backward_adapters_reuse(act_dev[(M, d["K"])], act_dev[(M, d["N"])], T, U, r,
+                                                              dA=gA, dB=gB, workspace=ws_ad) for d, (T, U), (gA, gB) in zip(dev, proj, grads)])
+    if lw.lowra_device_status(ws_ad) != 0:
+        raise SystemExit("device status after the adapter gradients (reusing the projections)")
+    extras["adapter_gradients_reusing_projections"] = {
+        "ms": ms, "GB/s": ad_bytes / (ms * 1e-3) / 1e9, "frac_hbm": ad_bytes / (ms * 1e-3) / 1e9 / P["hbm"],
+        "note": "not part of the step; dA and dB from the s X A and s dY B^T that lowra_lora_forward / lowra_lora_backward_input "
+                "left in their workspaces: two products instead of four, X and dY read once"}
+    del ws_f, proj
+
     # per-channel quantisation error (the precision assigner's input) and the residual W - W_hat
     sse = [torch.empty(d["N"], dtype=torch.float64, device="cuda") for d in dev]
     res = torch.empty(max(d["N"] * d["K"] for d in dev), dtype=torch.float32, device="cuda")
@@ -905,7 +924,7 @@ def run_reference(args):
 # small single-kernel cases for profiler captures (a few hundred MB on the device, three launches each)
 # --------------------------------------------------------------------------------------------------
 CASES = ("forward", "backward", "forward4096", "backward_gate", "forward_4bit", "backward_4bit", "forward_1bit", "backward_1bit",
-         "codec", "decode_layer", "learn", "adapters", "errors")
+         "codec", "decode_layer", "learn", "adapters", "adapters_reuse", "errors")
 
 
 def run_case(case: str) -> None:
@@ -913,7 +932,7 @@ def run_case(case: str) -> None:
     at that precision); forward4096: 4096 tokens (264 pieces: tiles cut between SMs, partial tiles preloaded);
     backward_gate: 11008 x 4096 at 4096 tokens (last row of tiles cut); codec: decode + encode of an 11008 x 4096
     matrix; decode_layer: the seven decodes of a Llama-7B layer back to back; learn: codebook learner, 4096 x 4096,
-    10 rounds; adapters: gradients of the low-rank factors, 4096 x 11008, 4096 tokens; errors: per-channel
+    10 rounds; adapters: gradients of the low-rank factors, 4096 x 11008, 4096 tokens (adapters_reuse: from given projections); errors: per-channel
     quantisation error with and without the residual, 11008 x 4096."""
     import torch
 
@@ -922,15 +941,21 @@ def run_case(case: str) -> None:
     cfg = si.config(3)
     r, s = cfg.rank, cfg.s
     gen = torch.Generator(device="cuda").manual_seed(1)
-    if case == "adapters":
+    if case in ("adapters", "adapters_reuse"):
         N, K, M = 11008, 4096, 4096
         X = torch.randn(M, K, device="cuda", generator=gen).bfloat16()
         dY = torch.randn(M, N, device="cuda", generator=gen).bfloat16()
         A = (torch.randn(K, r, device="cuda", generator=gen) * 0.01).bfloat16()
         B = (torch.randn(r, N, device="cuda", generator=gen) * 0.01).bfloat16()
         ws = torch.empty(lw.lowra_adapter_workspace_bytes(M, r), dtype=torch.uint8, device="cuda")
-        for _ in range(3):
-            lw.lowra_lora_backward_adapters(X, dY, A, B, s, workspace=ws)
+        if case == "adapters_reuse":     # the projections as a forward / backward-input call leaves them: bf16 [M, 64]
+            T = (s * (X.float() @ A.float())).bfloat16()
+            U = (s * (dY.float() @ B.float().T)).bfloat16()
+            for _ in range(3):
+                lw.lowra_lora_backward_adapters_reuse(X, dY, T, U, r, workspace=ws)
+        else:
+            for _ in range(3):
+                lw.lowra_lora_backward_adapters(X, dY, A, B, s, workspace=ws)
         status = lw.lowra_device_status(ws)
         print("adapters status", status)
         if status != 0:

@@ -312,6 +312,26 @@ lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, const uint16_t*
                                           void* stream);
 
 /*
+ * The same gradients from the down-projections that the two calls above have already formed (Section 3: forward and
+ * backward of the layer come before the factors' gradients in a training step): lowra_lora_forward leaves
+ * T = bf16(s X A) in its workspace, lowra_lora_backward_input leaves U = bf16(s dY B^T) in its own, both [M, rp] with
+ * rp = r rounded up to 64.  With them only dA = X^T U and dB = T^T dY remain: X and dY are read once instead of twice
+ * and two of the four products fall away.
+ *   lowra_workspace_projection  device pointer to that matrix inside a workspace of the fused calls (member: 0 for the
+ *                               plain calls, the member's index for the batch calls); valid from the moment that call
+ *                               has run (stream order) until the next call on the same workspace - so forward and
+ *                               backward-input need a workspace each for both to survive.  NULL for invalid arguments.
+ *   T_dev, U_dev                bf16 [M, rp] as above (any device memory: the caller may also keep copies)
+ *   workspace_dev               256-byte aligned, >= 256 bytes (status word only)
+ * Other arguments, limits and errors as lowra_lora_backward_adapters; A, B and s are not needed (T and U carry them).
+ */
+const uint16_t* lowra_workspace_projection(const void* workspace_dev, int32_t member, int32_t M, int32_t r);
+lowra_status lowra_lora_backward_adapters_reuse(const uint16_t* X_dev, const uint16_t* dY_dev, int32_t M, int32_t K,
+                                                int32_t N, const uint16_t* T_dev, const uint16_t* U_dev, int32_t r,
+                                                uint16_t* dA_dev, uint16_t* dB_dev, void* workspace_dev,
+                                                size_t workspace_bytes, void* stream);
+
+/*
  * Synchronises `stream` and returns the status word that the last forward / backward call wrote
  * into its workspace: LOWRA_OK, or LOWRA_ERR_TIMEOUT if a bounded wait inside a kernel ran out
  * (the kernel then released its resources and returned; the output is not valid).

@@ -31,7 +31,8 @@ EXPORTS = (
     "lowra_lora_backward_adapters", "lowra_quant_error", "lowra_natural_offsets", "lowra_reorder_rows",
     "lowra_channel_errors", "lowra_deal_bytes", "lowra_deal_build", "lowra_workspace_init",
     "lowra_learn_codebooks_all", "lowra_lora_forward_adapters", "lowra_batch_workspace_bytes",
-    "lowra_lora_forward_batch", "lowra_lora_backward_input_batch", "lowra_set_wait_limit", "lowra_diag_wait_expiry", "lowra_diag_drop_t_flags",
+    "lowra_lora_forward_batch", "lowra_lora_backward_input_batch", "lowra_lora_backward_adapters_reuse",
+    "lowra_workspace_projection", "lowra_set_wait_limit", "lowra_diag_wait_expiry", "lowra_diag_drop_t_flags",
 )
 
 
@@ -122,6 +123,10 @@ def lib() -> ctypes.CDLL:
         L.lowra_lora_backward_adapters.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, ctypes.c_float, vp, vp, vp,
                                                    ctypes.c_size_t, vp]
         L.lowra_lora_backward_adapters.restype = ctypes.c_int
+        L.lowra_lora_backward_adapters_reuse.argtypes = [vp, vp, i32, i32, i32, vp, vp, i32, vp, vp, vp, ctypes.c_size_t, vp]
+        L.lowra_lora_backward_adapters_reuse.restype = ctypes.c_int
+        L.lowra_workspace_projection.argtypes = [vp, i32, i32, i32]
+        L.lowra_workspace_projection.restype = ctypes.c_void_p
         L.lowra_device_status.argtypes = [vp, vp]
         L.lowra_device_status.restype = ctypes.c_int
         L.lowra_dense_nt.argtypes = [vp, vp, i32, i32, i32, vp, vp, ctypes.c_size_t, vp]
@@ -560,6 +565,41 @@ def lowra_lora_backward_adapters(X, dY, A, B, s: float, dA: Optional[torch.Tenso
                                               _ptr(dA), _ptr(dB), _ptr(workspace), workspace.numel(),
                                               _stream(stream))
     _check(code, "lowra_lora_backward_adapters")
+    return dA, dB
+
+
+def lowra_workspace_projection(workspace: torch.Tensor, M: int, r: int, member: int = 0) -> torch.Tensor:
+    """The down-projection (s X A after a forward call, s dY B^T after a backward-input call) that the last fused call
+    left in `workspace`: a bf16 [M, rp] view into the workspace, rp = r rounded up to 64."""
+    _dev(workspace, torch.uint8, "workspace")
+    p = lib().lowra_workspace_projection(_ptr(workspace), int(member), int(M), int(r))
+    if not p:
+        raise LowraError(LOWRA_ERR_SHAPE, "lowra_workspace_projection")
+    rp = (int(r) + 63) // 64 * 64
+    off = int(p) - workspace.data_ptr()
+    return workspace[off:off + int(M) * rp * 2].view(torch.bfloat16).view(int(M), rp)
+
+
+def lowra_lora_backward_adapters_reuse(X, dY, T, U, r: int, dA: Optional[torch.Tensor] = None,
+                                       dB: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                                       stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """dA = X^T U [K, r] and dB = T^T dY [r, N] from the down-projections T, U (bf16 [M, rp]) that the forward and the
+    backward-input call left in their workspaces (lowra_workspace_projection): X and dY are read once."""
+    for t, n in ((X, "X"), (dY, "dY"), (T, "T"), (U, "U")):
+        _dev(t, torch.bfloat16, n)
+    M, K, N = int(X.shape[0]), int(X.shape[1]), int(dY.shape[1])
+    rp = (int(r) + 63) // 64 * 64
+    if tuple(dY.shape) != (M, N) or tuple(T.shape) != (M, rp) or tuple(U.shape) != (M, rp):
+        raise ValueError("shape mismatch")
+    if dA is None:
+        dA = torch.empty((K, r), dtype=torch.bfloat16, device=X.device)
+    if dB is None:
+        dB = torch.empty((r, N), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = torch.empty(256, dtype=torch.uint8, device=X.device)
+    code = lib().lowra_lora_backward_adapters_reuse(_ptr(X), _ptr(dY), M, K, N, _ptr(T), _ptr(U), int(r), _ptr(dA), _ptr(dB),
+                                                    _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(code, "lowra_lora_backward_adapters_reuse")
     return dA, dB
 
 

@@ -474,36 +474,43 @@ extern "C" size_t lowra_adapter_workspace_bytes(int32_t M, int32_t r) {
     return plan_adapter_workspace(M, r).total;
 }
 
-extern "C" lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, const uint16_t* dY_dev, int32_t M, int32_t K,
-                                                     int32_t N, const uint16_t* A_dev, const uint16_t* B_dev, int32_t r,
-                                                     float s, uint16_t* dA_dev, uint16_t* dB_dev, void* workspace_dev,
-                                                     size_t workspace_bytes, void* stream_v) {
-    using namespace lowra;
-    if (!X_dev || !dY_dev || !A_dev || !B_dev || !dA_dev || !dB_dev || !workspace_dev) return LOWRA_ERR_NULL;
+namespace lowra {
+namespace {
+// dA = X^T U and dB = (dY^T T)^T, with the down-projections T = s X A and U = s dY B^T either computed here (T_in ==
+// nullptr: four skinny products, X and dY read twice) or taken from the caller (two products, X and dY read once).
+lowra_status run_adapters(const uint16_t* X_dev, const uint16_t* dY_dev, int32_t M, int32_t K, int32_t N, const uint16_t* A_dev,
+                          const uint16_t* B_dev, int32_t r, float s, const uint16_t* T_in, const uint16_t* U_in, uint16_t* dA_dev,
+                          uint16_t* dB_dev, void* workspace_dev, size_t workspace_bytes, void* stream_v) {
+    const bool reuse = T_in != nullptr;
+    if (!X_dev || !dY_dev || !dA_dev || !dB_dev || !workspace_dev) return LOWRA_ERR_NULL;
+    if (reuse ? !U_in : (!A_dev || !B_dev)) return LOWRA_ERR_NULL;
     if (M < 1 || K < 8 || N < 8 || K % 8 != 0 || N % 8 != 0 || !rank_ok(r)) return LOWRA_ERR_SHAPE;
     if (!aligned16(X_dev) || !aligned16(dY_dev) || !aligned16(A_dev) || !aligned16(B_dev) || !aligned16(dA_dev) ||
-        !aligned16(dB_dev))
+        !aligned16(dB_dev) || !aligned16(T_in) || !aligned16(U_in))
         return LOWRA_ERR_ALIGN;
     const AdapterWorkspace w = plan_adapter_workspace(M, r);
-    if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) != 0) return LOWRA_ERR_WORKSPACE;
+    if (workspace_bytes < (reuse ? kStatusBytes : w.total) || (reinterpret_cast<uintptr_t>(workspace_dev) & 255u) != 0)
+        return LOWRA_ERR_WORKSPACE;
     lowra_status st = check_device();
     if (st != LOWRA_OK) return st;
     cudaStream_t stream = (cudaStream_t)stream_v;
     unsigned char* ws = static_cast<unsigned char*>(workspace_dev);
     uint32_t* status = reinterpret_cast<uint32_t*>(ws);
-    uint16_t* T = reinterpret_cast<uint16_t*>(ws + w.off_T);
-    uint16_t* U = reinterpret_cast<uint16_t*>(ws + w.off_U);
+    const uint16_t* T = reuse ? T_in : reinterpret_cast<uint16_t*>(ws + w.off_T);
+    const uint16_t* U = reuse ? U_in : reinterpret_cast<uint16_t*>(ws + w.off_U);
     clear_status_kernel<<<1, 1, 0, stream>>>(status);
     const int rp = w.rp;
     CUtensorMap tmX, tmXt, tmdY, tmdYt, tmA, tmB, tmT, tmU;
-    if (!make_map(&tmX, X_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, 128) ||      // rows of 64 features (K-major)
-        !make_map(&tmXt, X_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, 64) ||      // 64 tokens x 64 features (MN-major)
-        !make_map(&tmdY, dY_dev, (uint64_t)M, (uint64_t)N, (uint64_t)N, 128) ||
+    if (!make_map(&tmXt, X_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, 64) ||      // 64 tokens x 64 features (MN-major)
         !make_map(&tmdYt, dY_dev, (uint64_t)M, (uint64_t)N, (uint64_t)N, 64) ||
-        !make_map(&tmA, A_dev, (uint64_t)K, (uint64_t)r, (uint64_t)r, 64) ||       // 64 features x 64 ranks (MN-major)
-        !make_map(&tmB, B_dev, (uint64_t)r, (uint64_t)N, (uint64_t)N, (uint32_t)rp) ||   // ranks x 64 channels (K-major)
         !make_map(&tmT, T, (uint64_t)M, (uint64_t)rp, (uint64_t)rp, 64) ||
         !make_map(&tmU, U, (uint64_t)M, (uint64_t)rp, (uint64_t)rp, 64))
+        return LOWRA_ERR_CUDA;
+    if (!reuse &&
+        (!make_map(&tmX, X_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, 128) ||      // rows of 64 features (K-major)
+         !make_map(&tmdY, dY_dev, (uint64_t)M, (uint64_t)N, (uint64_t)N, 128) ||
+         !make_map(&tmA, A_dev, (uint64_t)K, (uint64_t)r, (uint64_t)r, 64) ||       // 64 features x 64 ranks (MN-major)
+         !make_map(&tmB, B_dev, (uint64_t)r, (uint64_t)N, (uint64_t)N, (uint32_t)rp)))   // ranks x 64 channels (K-major)
         return LOWRA_ERR_CUDA;
     SkinnyArgs a;
     memset(&a, 0, sizeof(a));
@@ -511,14 +518,14 @@ extern "C" lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, cons
     a.wait_ns = wait_limit_ns();
     a.rp = rp;
     // Four skinny products; X and dY are each needed by two of them.  The two uses of the larger operand run back to
-    // back, so that its second reading comes from L2 (126 MB hold a 4096-token operand of up to 11008 columns), and
-    // the smaller operand is read first and last: T, U, dB, dA when dY is the larger one, U, T, dA, dB otherwise.
+    // back, so that its second reading can come from L2, and the smaller operand is read first and last: T, U, dB, dA
+    // when dY is the larger one, U, T, dA, dB otherwise.  With the caller's T and U only the two gradients are left.
     auto down_T = [&]() {   // T = s X A: rows = tokens, contraction over the K input features
-        a.out = T; a.R = M; a.C = K; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 1; a.transposed = 0; a.scale = s;
+        a.out = const_cast<uint16_t*>(T); a.R = M; a.C = K; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 1; a.transposed = 0; a.scale = s;
         return launch_skinny(tmX, tmA, a, stream);
     };
     auto down_U = [&]() {   // U = s dY B^T: rows = tokens, contraction over the N output channels
-        a.out = U; a.R = M; a.C = N; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 0; a.transposed = 0; a.scale = s;
+        a.out = const_cast<uint16_t*>(U); a.R = M; a.C = N; a.n_cols = rp; a.ld_out = rp; a.a_mn = 0; a.b_mn = 0; a.transposed = 0; a.scale = s;
         return launch_skinny(tmdY, tmB, a, stream);
     };
     auto grad_A = [&]() {   // dA = X^T U: rows = input features, contraction over the tokens
@@ -529,12 +536,42 @@ extern "C" lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, cons
         a.out = dB_dev; a.R = N; a.C = M; a.n_cols = r; a.ld_out = N; a.a_mn = 1; a.b_mn = 1; a.transposed = 1; a.scale = 1.0f;
         return launch_skinny(tmdYt, tmT, a, stream);
     };
+    if (reuse) {
+        if ((st = grad_A()) != LOWRA_OK) return st;
+        return grad_B();
+    }
     if (N > K) {
         if ((st = down_T()) != LOWRA_OK || (st = down_U()) != LOWRA_OK || (st = grad_B()) != LOWRA_OK) return st;
         return grad_A();
     }
     if ((st = down_U()) != LOWRA_OK || (st = down_T()) != LOWRA_OK || (st = grad_A()) != LOWRA_OK) return st;
     return grad_B();
+}
+}  // namespace
+}  // namespace lowra
+
+extern "C" lowra_status lowra_lora_backward_adapters(const uint16_t* X_dev, const uint16_t* dY_dev, int32_t M, int32_t K,
+                                                     int32_t N, const uint16_t* A_dev, const uint16_t* B_dev, int32_t r,
+                                                     float s, uint16_t* dA_dev, uint16_t* dB_dev, void* workspace_dev,
+                                                     size_t workspace_bytes, void* stream) {
+    return lowra::run_adapters(X_dev, dY_dev, M, K, N, A_dev, B_dev, r, s, nullptr, nullptr, dA_dev, dB_dev, workspace_dev,
+                               workspace_bytes, stream);
+}
+
+extern "C" lowra_status lowra_lora_backward_adapters_reuse(const uint16_t* X_dev, const uint16_t* dY_dev, int32_t M, int32_t K,
+                                                           int32_t N, const uint16_t* T_dev, const uint16_t* U_dev, int32_t r,
+                                                           uint16_t* dA_dev, uint16_t* dB_dev, void* workspace_dev,
+                                                           size_t workspace_bytes, void* stream) {
+    if (!T_dev || !U_dev) return LOWRA_ERR_NULL;
+    return lowra::run_adapters(X_dev, dY_dev, M, K, N, nullptr, nullptr, r, 1.0f, T_dev, U_dev, dA_dev, dB_dev, workspace_dev,
+                               workspace_bytes, stream);
+}
+
+extern "C" const uint16_t* lowra_workspace_projection(const void* workspace_dev, int32_t member, int32_t M, int32_t r) {
+    using namespace lowra;
+    if (!workspace_dev || member < 0 || member >= kMaxBatch || M < 1 || !rank_ok(r)) return nullptr;
+    const size_t t_bytes = align256((size_t)M * (size_t)((r + 63) / 64 * 64) * 2);
+    return reinterpret_cast<const uint16_t*>(static_cast<const unsigned char*>(workspace_dev) + kStatusBytes + (size_t)member * t_bytes);
 }
 
 extern "C" lowra_status lowra_device_status(const void* workspace_dev, void* stream) {
