@@ -272,13 +272,16 @@ lowra_status lowra_lora_backward_input_batch(const lowra_member* members_host, i
  * table and its own low-rank factors).  The tokens of the batch are sorted by adapter: adapter a owns the token rows
  * [group_start_host[a], group_start_host[a + 1]) of X and Y, and for those rows
  *     Y = X . deq_a(Wq)^T + s * (X . A_a) . B_a
- * with deq_a the dequantisation through adapter a's mappings.  One call routes every group to its tables; the groups
- * run back to back on the stream as one fused launch each (a dequantised weight tile depends on the adapter's
- * mappings, so groups cannot share tiles), empty groups are skipped.
+ * with deq_a the dequantisation through adapter a's mappings.  One call routes every group to its tables.  Up to
+ * LOWRA_MAX_BATCH groups run in one fused launch (their tiles dealt to the SMs together, so that small groups fill the
+ * GPU between them) when the layout carries a deal and the workspace has lowra_batch_workspace_bytes(layout,
+ * LOWRA_MAX_BATCH, M, r) bytes; otherwise every group is a launch of its own.  A dequantised weight tile depends on
+ * the adapter's mappings, so groups never share tiles; empty groups are skipped.
  *   maps_dev         fp32 [n_adapters][N][16]
  *   A_dev            bf16 [n_adapters][K][r];   B_dev  bf16 [n_adapters][r][N]
  *   group_start_host int32 [n_adapters + 1], HOST, non-decreasing, [0] = 0, [n_adapters] = M
- *   X_dev bf16 [M, K];  Y_dev bf16 [M, N];  workspace_dev: as lowra_lora_forward for M tokens.
+ *   X_dev bf16 [M, K];  Y_dev bf16 [M, N];  workspace_dev: at least as lowra_lora_forward for M tokens (see above);
+ *   with a deal in the layout, initialised by lowra_workspace_init.
  * Errors: as lowra_lora_forward; n_adapters < 1 or group_start_host not as described -> LOWRA_ERR_SHAPE.
  */
 lowra_status lowra_lora_forward_adapters(const lowra_layout* layout, const uint8_t* packed_dev, const float* absmax_dev,

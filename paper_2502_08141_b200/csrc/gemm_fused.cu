@@ -201,10 +201,19 @@ fused_kernel(const __grid_constant__ KParams<NB> P, const __grid_constant__ KMap
     auto a_slot = [&](uint32_t it) { return base + (it % SA) * kSmemA; };
     auto b_slot = [&](uint32_t it) { return base + SA * kSmemA + (it % SB) * kSmemB; };
     const int cid = (int)blockIdx.x / CL, NC = (int)gridDim.x / CL;   // this cluster, clusters in the grid
-    const int super_t = (P.tiles_t + CL - 1) / CL;          // groups of CL token tiles
-    const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? P.count * super_t : 0;   // all members' T tiles come first
-    const int tiles_w = P.tiles_r * super_t;                // weight tiles of one member (per cluster)
-    const int n_tiles = n_t_tiles + P.count * tiles_w;      // per cluster
+    const int super_t = P.super_total;                      // groups of CL token tiles, all members one after the other
+    const int n_t_tiles = (MODE != kModeDense && P.lora_blocks > 0) ? super_t : 0;   // all members' T tiles come first
+    const int n_tiles = n_t_tiles + P.tiles_r * super_t;    // per cluster
+    // token-tile group gst of the call -> member and group inside the member
+    auto member_of = [&](int gst, int& prob, int& st) {
+        prob = 0;
+        if (NB > 1) {
+#pragma unroll
+            for (int i = 1; i < NB; ++i)
+                if (i < P.count && gst >= P.mem[i].st0) prob = i;
+        }
+        st = gst - P.mem[prob].st0;
+    };
     const int B = P.main_blocks + P.lora_blocks;            // contraction blocks of a weight tile
     // Schedule.  The pieces of work are numbered g = 0, 1, ...: first the T tiles, then the weight tiles; cluster c
     // takes g = c, c + NC, c + 2 NC, ... ("rows" of NC pieces; the clusters then sweep the contraction in step and
@@ -229,15 +238,15 @@ fused_kernel(const __grid_constant__ KParams<NB> P, const __grid_constant__ KMap
         t.prob = 0;
         if (!sk || i < w_dp) {
             const int g = cid + i * NC;
+            int st;
             if (g < n_t_tiles) {
-                t.prob = (NB == 1) ? 0 : g / super_t;
-                t.is_t = true; t.rt = 0; t.mt = (g - t.prob * super_t) * CL + (int)crank; t.kb0 = 0; t.kb1 = P.main_blocks;
+                member_of(g, t.prob, st);
+                t.is_t = true; t.rt = 0; t.mt = st * CL + (int)crank; t.kb0 = 0; t.kb1 = P.main_blocks;
             } else {
-                int idx = g - n_t_tiles;
-                t.prob = (NB == 1) ? 0 : idx / tiles_w;
-                idx -= t.prob * tiles_w;
-                const int st = idx / P.tiles_r;
-                t.is_t = false; t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank; t.kb0 = 0; t.kb1 = B;
+                const int idx = g - n_t_tiles;
+                const int gst = idx / P.tiles_r;
+                member_of(gst, t.prob, st);
+                t.is_t = false; t.rt = idx - gst * P.tiles_r; t.mt = st * CL + (int)crank; t.kb0 = 0; t.kb1 = B;
             }
         } else {
             const int k = i - w_dp;
@@ -245,11 +254,11 @@ fused_kernel(const __grid_constant__ KParams<NB> P, const __grid_constant__ KMap
             const long long first = (long long)t.tile * B;
             t.kb0 = (k == 0) ? (int)(lo - first) : 0;
             t.kb1 = (hi < first + B) ? (int)(hi - first) : B;
-            int idx = sk_first + t.tile;
-            t.prob = (NB == 1) ? 0 : idx / tiles_w;
-            idx -= t.prob * tiles_w;
-            const int st = idx / P.tiles_r;
-            t.is_t = false; t.rt = idx - st * P.tiles_r; t.mt = st * CL + (int)crank;
+            const int idx = sk_first + t.tile;
+            const int gst = idx / P.tiles_r;
+            int st;
+            member_of(gst, t.prob, st);
+            t.is_t = false; t.rt = idx - gst * P.tiles_r; t.mt = st * CL + (int)crank;
             t.part = t.kb0 > 0;
             t.pre = t.kb0 == 0 && t.kb1 < B;
         }
@@ -476,7 +485,7 @@ fused_kernel(const __grid_constant__ KParams<NB> P, const __grid_constant__ KMap
                 const int m0 = t.mt * kTileT;
 #pragma unroll 1
                 for (int chunk = 0; chunk < kTileT / 32; ++chunk) {
-                    if (m0 + chunk * 32 >= P.M) break;
+                    if (m0 + chunk * 32 >= P.mem[t.prob].M) break;
                     float sum[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) sum[j] = 0.0f;
@@ -548,7 +557,7 @@ fused_kernel(const __grid_constant__ KParams<NB> P, const __grid_constant__ KMap
                     if (c + 1 == c_end) { add = ring; break; }          // the last one is added on the way out, below
 #pragma unroll 1
                     for (int chunk = 0; chunk < kTileT / 32; ++chunk) {   // the others go into the accumulator
-                        if (m0 + chunk * 32 >= P.M) break;
+                        if (m0 + chunk * 32 >= P.mem[t.prob].M) break;
                         uint32_t v[32];
                         const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileT + chunk * 32;
                         ptx::tmem_ld_32x32(taddr, v);
@@ -563,7 +572,7 @@ fused_kernel(const __grid_constant__ KParams<NB> P, const __grid_constant__ KMap
             }
 #pragma unroll 1
             for (int chunk = 0; chunk < kTileT / 32; ++chunk) {
-                if (m0 + chunk * 32 >= P.M) break;
+                if (m0 + chunk * 32 >= P.mem[t.prob].M) break;
                 uint32_t v[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileT + chunk * 32, v);
                 ptx::tmem_ld_wait();
@@ -591,7 +600,7 @@ fused_kernel(const __grid_constant__ KParams<NB> P, const __grid_constant__ KMap
                     {
                         const int tok = lane >> 2, piece = lane & 3;
                         const int m = m0 + chunk * 32 + rnd * kEpilogueTokens + tok, n = r0 + q * 32 + piece * 8;
-                        if (m < P.M && n < R) {
+                        if (m < P.mem[t.prob].M && n < R) {
                             const uint4 val = *reinterpret_cast<const uint4*>(stage16 + tok * 32 + piece * 8);
                             uint16_t* dst = out + (size_t)m * ld + n;
                             if (vec_ok && n + 8 <= R) {
@@ -976,9 +985,9 @@ static lowra_status launch_mode(const GemmParams& G, const BatchMaps& TM, cudaSt
         }
         max_clusters = max_clusters_of[dev];
     }
-    const int super_t = (G.tiles_t + CL - 1) / CL;
-    const int n_t = (MODE != kModeDense && G.lora_blocks > 0) ? G.count * super_t : 0;
-    const int n_tiles = G.count * G.tiles_r * super_t + n_t;
+    const int super_t = G.super_total;
+    const int n_t = (MODE != kModeDense && G.lora_blocks > 0) ? super_t : 0;
+    const int n_tiles = G.tiles_r * super_t + n_t;
     const int clusters = n_tiles < max_clusters ? n_tiles : max_clusters;
     cfg.gridDim = dim3((unsigned)(clusters * CL), 1, 1);
     GemmParams Q = G;

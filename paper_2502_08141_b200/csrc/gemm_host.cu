@@ -29,8 +29,10 @@ constexpr size_t kExitsOffset = 128;   //   CTAs of the running call that have l
 size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
 
 struct Workspace {
-    size_t off_T, t_bytes, off_flags, off_items, off_meta, off_part, total;
-    int rp, t_flags, n_flags;
+    size_t off_T[kMaxBatch];      // per member: its down-projected activations
+    int flag0[kMaxBatch];         // per member: index of its first "T ready" flag
+    size_t off_flags, off_items, off_meta, off_part, total;
+    int rp, n_flags, sk_flag0;
 };
 
 bool rank_ok(int r) { return r >= 16 && r <= 128 && r % 16 == 0; }
@@ -63,23 +65,35 @@ DealBuffer plan_deal(int N) {
     return d;
 }
 
-Workspace plan_workspace(int N, int K, int M, int r, bool stream_k, int count = 1) {
+// Ms: the members' token counts (the plain and the batch calls: all equal).
+Workspace plan_workspace(int N, int K, const int* Ms, int count, int r, bool stream_k) {
     (void)K;
     Workspace w;
+    memset(&w, 0, sizeof(w));
     w.rp = (r + 63) / 64 * 64;
     const DealSizes z = deal_sizes(N);   // room for the deal of one direction, rebuilt by every call that brings none
-    w.off_T = kStatusBytes;
-    w.t_bytes = align256((size_t)M * w.rp * 2);                      // per member
-    w.off_flags = w.off_T + (size_t)count * w.t_bytes;
-    // per member the "T ready" flags (a cluster's last token tiles may lie past M), then one "partial tile ready"
-    // flag per CTA
-    w.t_flags = (M + kTileT - 1) / kTileT + kCluster;
-    w.n_flags = count * w.t_flags + kMaxClusters * kCluster;
+    size_t off = kStatusBytes;
+    int flags = 0;
+    for (int i = 0; i < count; ++i) {
+        w.off_T[i] = off;
+        off += align256((size_t)Ms[i] * w.rp * 2);
+        // the member's "T ready" flags (a cluster's last token tiles may lie past its tokens)
+        w.flag0[i] = flags;
+        flags += (Ms[i] + kTileT - 1) / kTileT + kCluster;
+    }
+    w.off_flags = off;
+    w.sk_flag0 = flags;                                  // then one "partial tile ready" flag per CTA
+    w.n_flags = flags + kMaxClusters * kCluster;
     w.off_items = w.off_flags + align256((size_t)w.n_flags * 4);
     w.off_meta = w.off_items + align256(z.rows_bytes > z.fwd_bytes ? z.rows_bytes : z.fwd_bytes);
     w.off_part = w.off_meta + align256(z.heads_bytes);
     w.total = w.off_part + (stream_k ? align256((size_t)kMaxClusters * kSkSlotFloats * 4) : 0);   // stream-K partial tiles
     return w;
+}
+Workspace plan_workspace(int N, int K, int M, int r, bool stream_k, int count = 1) {
+    int Ms[kMaxBatch];
+    for (int i = 0; i < kMaxBatch; ++i) Ms[i] = M;
+    return plan_workspace(N, K, Ms, count, r, stream_k);
 }
 
 PFN_cuTensorMapEncodeTiled_v12000 encode_fn() {
@@ -119,10 +133,12 @@ struct MemberArgs {
     const uint16_t* A;
     const uint16_t* B;
     uint16_t* out;
+    int32_t M;             // tokens of this member
 };
 
-// Forward / backward-input for `count` weights of one shape in one launch (count == 1: the plain calls).
-lowra_status run_members(bool backward, const MemberArgs* mem, int count, int32_t M, int32_t r, float s, void* workspace,
+// Forward / backward-input for `count` weights of one shape in one launch (count == 1: the plain calls).  The members
+// may have different token counts (several adapters on one weight: one member per token group).
+lowra_status run_members(bool backward, const MemberArgs* mem, int count, int32_t r, float s, void* workspace,
                          size_t workspace_bytes, void* stream_v, bool stream_k = true) {
     if (count < 1 || count > kMaxBatch) return LOWRA_ERR_SHAPE;
     for (int i = 0; i < count; ++i) {
@@ -132,17 +148,21 @@ lowra_status run_members(bool backward, const MemberArgs* mem, int count, int32_
     }
     if (!workspace) return LOWRA_ERR_NULL;
     const int N = mem[0].layout->N, K = mem[0].layout->K;
-    if (M < 1 || !rank_ok(r) || N % 8 != 0 || N > 64 * kMaxGroups64 || (uint64_t)N * (uint64_t)(K / 64) >= (1ull << 32))
+    if (!rank_ok(r) || N % 8 != 0 || N > 64 * kMaxGroups64 || (uint64_t)N * (uint64_t)(K / 64) >= (1ull << 32))
         return LOWRA_ERR_SHAPE;
+    int Ms[kMaxBatch], M = 0;
     for (int i = 0; i < count; ++i) {
         const MemberArgs& m = mem[i];
+        if (m.M < 1) return LOWRA_ERR_SHAPE;
+        Ms[i] = m.M;
+        M = m.M > M ? m.M : M;
         if (m.layout->N != N || m.layout->K != K) return LOWRA_ERR_SHAPE;                 // one shape per launch
         if (count > 1 && m.layout->deal_dev == nullptr) return LOWRA_ERR_NULL;            // a batch has no prologue launch
         if (!aligned16(m.packed) || !aligned16(m.absmax) || !aligned16(m.maps) || !aligned16(m.act) || !aligned16(m.A) ||
             !aligned16(m.B) || !aligned16(m.out) || (reinterpret_cast<uintptr_t>(m.layout->deal_dev) & 255u) != 0)
             return LOWRA_ERR_ALIGN;
     }
-    const Workspace w = plan_workspace(N, K, M, r, stream_k, count);
+    const Workspace w = plan_workspace(N, K, Ms, count, r, stream_k);
     if (workspace_bytes < w.total || (reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return LOWRA_ERR_WORKSPACE;
     lowra_status st = check_device();
     if (st != LOWRA_OK) return st;
@@ -151,7 +171,6 @@ lowra_status run_members(bool backward, const MemberArgs* mem, int count, int32_
     unsigned char* ws = static_cast<unsigned char*>(workspace);
     uint32_t* status = reinterpret_cast<uint32_t*>(ws);
     uint32_t* flags = reinterpret_cast<uint32_t*>(ws + w.off_flags);
-    const int tiles_t = (M + kTileT - 1) / kTileT;
 
     GemmParams G;
     memset(&G, 0, sizeof(G));
@@ -166,8 +185,11 @@ lowra_status run_members(bool backward, const MemberArgs* mem, int count, int32_
         g.absmax = m.absmax;
         g.maps = m.maps;
         g.out = m.out;
-        g.T = reinterpret_cast<uint16_t*>(ws + w.off_T + (size_t)i * w.t_bytes);
-        g.flags = flags + (size_t)i * w.t_flags;
+        g.T = reinterpret_cast<uint16_t*>(ws + w.off_T[i]);
+        g.flags = flags + w.flag0[i];
+        g.M = m.M;
+        g.st0 = G.super_total;
+        G.super_total += ((m.M + kTileT - 1) / kTileT + kCluster - 1) / kCluster;
         if (m.layout->deal_dev != nullptr) {
             // the rows were dealt once for this weight (lowra_deal_build) and the workspace numbers its calls
             // (lowra_workspace_init): nothing to prepare, the fused kernel is the only launch
@@ -216,14 +238,13 @@ lowra_status run_members(bool backward, const MemberArgs* mem, int count, int32_
     G.main_blocks = (G.C + kTileC - 1) / kTileC;
     G.lora_blocks = w.rp / kTileC;
     G.tiles_r = (G.R + kTileR - 1) / kTileR;
-    G.tiles_t = tiles_t;
     for (int i = 0; i < count; ++i) {   // token operands: every distinct one once (q, k, v share X in the forward pass)
         bool seen = false;
         for (int j = 0; j < i; ++j) seen = seen || mem[j].act == mem[i].act;
-        if (!seen) G.operand_bytes += (long long)M * G.C * 2;
+        if (!seen) G.operand_bytes += (long long)mem[i].M * G.C * 2;
     }
     G.sk_part = stream_k ? reinterpret_cast<float*>(ws + w.off_part) : nullptr;   // null: whole tiles only
-    G.sk_flags = flags + (size_t)count * w.t_flags;
+    G.sk_flags = flags + w.sk_flag0;
     G.wait_ns = wait_limit_ns();
     {   // diagnostic, armed by lowra_diag_drop_t_flags: take one of the calls it asked for
         int left = g_drop_t_flags.load(std::memory_order_relaxed);
@@ -233,8 +254,8 @@ lowra_status run_members(bool backward, const MemberArgs* mem, int count, int32_
     for (int i = 0; i < count; ++i) {
         const MemberArgs& m = mem[i];
         MemberMaps& t = TM.m[i];
-        if (!make_map(&t.tmB, m.act, (uint64_t)M, (uint64_t)G.C, (uint64_t)G.C, kTileT)) return LOWRA_ERR_CUDA;
-        if (!make_map(&t.tmT, G.mem[i].T, (uint64_t)M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
+        if (!make_map(&t.tmB, m.act, (uint64_t)m.M, (uint64_t)G.C, (uint64_t)G.C, kTileT)) return LOWRA_ERR_CUDA;
+        if (!make_map(&t.tmT, G.mem[i].T, (uint64_t)m.M, (uint64_t)w.rp, (uint64_t)w.rp, kTileT)) return LOWRA_ERR_CUDA;
         if (!backward) {
             // T tiles take ranks x features from A [K, r] (64 x 64 boxes); LoRA blocks take channels x ranks from B [r, N]
             if (!make_map(&t.tmFt, m.A, (uint64_t)K, (uint64_t)r, (uint64_t)r, 64)) return LOWRA_ERR_CUDA;
@@ -252,8 +273,8 @@ lowra_status run_lora(bool backward, const lowra_layout* layout, const uint8_t* 
                       const float* maps, const uint16_t* act, int32_t M, const uint16_t* A, const uint16_t* B,
                       int32_t r, float s, uint16_t* out, void* workspace, size_t workspace_bytes, void* stream_v,
                       bool stream_k = true) {
-    const MemberArgs m = {layout, packed, absmax, maps, act, A, B, out};
-    return run_members(backward, &m, 1, M, r, s, workspace, workspace_bytes, stream_v, stream_k);
+    const MemberArgs m = {layout, packed, absmax, maps, act, A, B, out, M};
+    return run_members(backward, &m, 1, r, s, workspace, workspace_bytes, stream_v, stream_k);
 }
 
 // scratch of the adapter-gradient call: status word | T = s X A | U = s dY B^T  (bf16 [M, rp] each)
@@ -360,10 +381,10 @@ lowra_status run_batch(bool backward, const lowra_member* members, int32_t count
     MemberArgs mem[kMaxBatch];
     for (int i = 0; i < count; ++i) {
         const lowra_member& m = members[i];
-        mem[i] = MemberArgs{m.layout, m.packed_dev, m.absmax_dev, m.maps_dev, m.act_dev, m.A_dev, m.B_dev, m.out_dev};
+        mem[i] = MemberArgs{m.layout, m.packed_dev, m.absmax_dev, m.maps_dev, m.act_dev, m.A_dev, m.B_dev, m.out_dev, M};
         if (m.layout != nullptr && m.layout->deal_dev == nullptr) return LOWRA_ERR_NULL;   // also for a batch of one
     }
-    return run_members(backward, mem, count, M, r, s, workspace, workspace_bytes, stream);
+    return run_members(backward, mem, count, r, s, workspace, workspace_bytes, stream);
 }
 }  // namespace
 }  // namespace lowra
@@ -395,13 +416,25 @@ extern "C" lowra_status lowra_lora_forward_adapters(const lowra_layout* layout, 
         if (group_start_host[a + 1] < group_start_host[a]) return LOWRA_ERR_SHAPE;
     const size_t N = (size_t)layout->N, K = (size_t)layout->K;
     if (workspace_bytes < lowra_workspace_bytes(layout, M, r)) return LOWRA_ERR_WORKSPACE;
-    for (int a = 0; a < n_adapters; ++a) {
-        const int m0 = group_start_host[a], m = group_start_host[a + 1] - m0;
-        if (m == 0) continue;
-        st = run_lora(false, layout, packed_dev, absmax_dev, maps_dev + (size_t)a * N * kTableStride, X_dev + (size_t)m0 * K, m,
-                      A_dev + (size_t)a * K * (size_t)r, B_dev + (size_t)a * (size_t)r * N, r, s, Y_dev + (size_t)m0 * N,
-                      workspace_dev, workspace_bytes, stream);
-        if (st != LOWRA_OK) return st;
+    // Up to kMaxBatch token groups go into one launch (one member per group: the same packed weight, the group's
+    // mappings, factors and token rows) when the layout carries a deal and the workspace has room for it; otherwise
+    // every group is a launch of its own.
+    const bool together = layout->deal_dev != nullptr &&
+                          workspace_bytes >= plan_workspace(layout->N, layout->K, M, r, true, kMaxBatch).total;
+    MemberArgs mem[kMaxBatch];
+    int n = 0;
+    for (int a = 0; a <= n_adapters; ++a) {
+        if (a < n_adapters) {
+            const int m0 = group_start_host[a], m = group_start_host[a + 1] - m0;
+            if (m == 0) continue;
+            mem[n++] = MemberArgs{layout, packed_dev, absmax_dev, maps_dev + (size_t)a * N * kTableStride, X_dev + (size_t)m0 * K,
+                                  A_dev + (size_t)a * K * (size_t)r, B_dev + (size_t)a * (size_t)r * N, Y_dev + (size_t)m0 * N, m};
+        }
+        if (n > 0 && (a == n_adapters || n == (together ? kMaxBatch : 1))) {
+            st = run_members(false, mem, n, r, s, workspace_dev, workspace_bytes, stream);
+            if (st != LOWRA_OK) return st;
+            n = 0;
+        }
     }
     return LOWRA_OK;
 }
@@ -570,7 +603,7 @@ extern "C" lowra_status lowra_lora_backward_adapters_reuse(const uint16_t* X_dev
 extern "C" const uint16_t* lowra_workspace_projection(const void* workspace_dev, int32_t member, int32_t M, int32_t r) {
     using namespace lowra;
     if (!workspace_dev || member < 0 || member >= kMaxBatch || M < 1 || !rank_ok(r)) return nullptr;
-    const size_t t_bytes = align256((size_t)M * (size_t)((r + 63) / 64 * 64) * 2);
+    const size_t t_bytes = align256((size_t)M * (size_t)((r + 63) / 64 * 64) * 2);   // as plan_workspace lays equal members out
     return reinterpret_cast<const uint16_t*>(static_cast<const unsigned char*>(workspace_dev) + kStatusBytes + (size_t)member * t_bytes);
 }
 
@@ -666,7 +699,8 @@ extern "C" lowra_status lowra_dense_nt(const uint16_t* P_dev, const uint16_t* Q_
     G.main_blocks = K / kTileC;
     G.lora_blocks = 0;
     G.tiles_r = (N + kTileR - 1) / kTileR;
-    G.tiles_t = (M + kTileT - 1) / kTileT;
+    G.super_total = (M + kTileT - 1) / kTileT;     // one CTA per "cluster" in the dense mode
+    G.mem[0].M = M;
     G.wait_ns = wait_limit_ns();
     if (!make_map(&TM.m[0].tmB, P_dev, (uint64_t)M, (uint64_t)K, (uint64_t)K, kTileT)) return LOWRA_ERR_CUDA;
     if (!make_map(&TM.m[0].tmFl, Q_dev, (uint64_t)N, (uint64_t)K, (uint64_t)K, kTileR)) return LOWRA_ERR_CUDA;

@@ -77,6 +77,8 @@ struct Member {
     uint16_t* out;            // [M, ld_out] bf16
     uint16_t* T;              // [M, rp] bf16: s * X . A (forward) or s * dY . B^T (backward), written by the T tiles
     uint32_t* flags;          // [tiles_t + kCluster] set to the call's number when T of a token tile is complete
+    int M;                    // this member's tokens (the batch calls: the same for all; several adapters: a group's)
+    int st0;                  // token-tile groups (kCluster tiles each) of the members before this one
 };
 
 // Tensor maps of one member: token operand, T, factor of the T tiles, factor of the LoRA blocks.
@@ -104,13 +106,14 @@ struct GemmCommon {
     float s;
     int rp;                 // LoRA rank rounded up to 64
     int r;                  // LoRA rank
-    int M;                  // tokens
+    int M;                  // tokens of the largest member (host: schedule choice)
+    int super_total;        // token-tile groups (kCluster tiles each) of all members
     int R;                  // A-operand rows in total: N (forward, dense) or K (backward)
     int C;                  // main contraction length: K (forward, dense) or N (backward)
     int ld_out;             // = R
     int main_blocks;        // ceil(C / 64)
     int lora_blocks;        // rp / 64 (0 in dense mode)
-    int tiles_r, tiles_t;   // per member
+    int tiles_r;            // row tiles of a member (all members have one shape)
     long long operand_bytes;   // token operands of the call, each distinct one counted once (host: schedule choice)
     // stream-K schedule (set by the launcher; sk == 0: whole tiles, dealt round-robin to the clusters)
     float* sk_part;         // fp32 partial tiles, one [kCluster][kTileT][kTileR] slot per cluster
