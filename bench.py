@@ -121,21 +121,26 @@ class ClockSampler:
         except Exception:
             self.proc.kill()
         sm, smax, reasons = [], [], set()
-        for ts, line in self.lines:
-            parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 9:
-                continue
-            try:
-                clk, mx = float(parts[1]), float(parts[2])
-            except ValueError:
-                continue
-            if t0 - 0.05 <= ts <= t1 + 0.15:
-                sm.append(clk)
-                smax.append(mx)
-                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
-                                     parts[5:9]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
+        # samples taken while the GPU was working: a line arrives a few milliseconds after it was sampled; when the
+        # region is shorter than that allows, the window is widened by one sampling period on either side
+        for lo, hi in ((t0 + 0.004, t1 + 0.004), (t0 - 0.02, t1 + 0.03)):
+            for ts, line in self.lines:
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    clk, mx = float(parts[1]), float(parts[2])
+                except ValueError:
+                    continue
+                if lo <= ts <= hi:
+                    sm.append(clk)
+                    smax.append(mx)
+                    for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                         parts[5:9]):
+                        if val.lower().startswith("active"):
+                            reasons.add(name)
+            if len(sm) >= 2:
+                break
         if not sm:  # region shorter than the sampling period: take everything seen
             for ts, line in self.lines:
                 parts = [p.strip() for p in line.split(",")]
@@ -144,7 +149,7 @@ class ClockSampler:
                 except Exception:
                     pass
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+                "sm_min_mhz": min(sm) if sm else None, "reasons": sorted(reasons), "samples": len(sm)}
 
 
 # --------------------------------------------------------------------------------------------------
@@ -426,6 +431,10 @@ def run_gpu(args):
         phase_ms[phase] = phase_ms.get(phase, 0.0) + e0.elapsed_time(e1)
     for k in phase_ms:
         phase_ms[k] /= args.steps
+    # the fused phases step by step: the power cap sets in some tens of milliseconds into a run of tensor-core calls
+    n_ph = len(phase_list)
+    fused_ms_by_step = [round(sum(e0.elapsed_time(e1) for ph, e0, e1 in records[i * n_ph:(i + 1) * n_ph] if ph in ("forward", "backward")), 3)
+                        for i in range(args.steps)]
     # diagnostic pass outside the timed region: the same step with events around every call
     n_diag = 3 if len(dev) <= 8 else 1
     calls = []
@@ -543,6 +552,7 @@ def run_gpu(args):
                 "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of the gate_proj backward-input launch of "
                                   "workload 3 (profiles/fused_backward_input_11008x4096_m4096_streamk.md), scaled by the "
                                   "input + output bytes of this step's average launch",
+                "ms_by_step": fused_ms_by_step if args.steps <= 64 else fused_ms_by_step[:32] + fused_ms_by_step[-32:],
                 "secondary": secondary}
 
     # ---- end to end: host buffers, pinned, copies inside the timed region (the first seven matrices of the workload)
