@@ -36,10 +36,25 @@ struct LearnParams {
     double init_t[3][16];  // initial thresholds per class
 };
 
-__device__ __forceinline__ double warp_sum(double v) {
+// NV sums per lane (NV = 4, 8 or 16) added up over the warp: instead of NV butterflies over all 32 lanes, every step
+// hands half of a lane's values to its partner and adds the partner's other half to its own, so that the number of
+// values halves with the distance; once a lane holds one value the remaining steps are plain butterflies.  Afterwards
+// the lanes whose low bits are zero hold the totals: value number lane / (32 / NV) in v[0].  A fixed order of additions.
+template <int NV>
+__device__ __forceinline__ void warp_sums(double (&v)[NV], int lane) {
+    int d = 16;
 #pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) v += __shfl_xor_sync(0xffffffffu, v, d);
-    return v;
+    for (int n = NV; n > 1; n >>= 1, d >>= 1) {
+        const bool upper = (lane & d) != 0;
+#pragma unroll
+        for (int k = 0; k < n / 2; ++k) {
+            const double send = upper ? v[k] : v[k + n / 2];
+            const double keep = upper ? v[k + n / 2] : v[k];
+            v[k] = keep + __shfl_xor_sync(0xffffffffu, send, d);
+        }
+    }
+#pragma unroll
+    for (; d >= 1; d >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], d);
 }
 
 // number of thresholds <= x among t[0 .. L-2] (sorted): branch-free binary search, L = 2, 4 or 16.
@@ -59,11 +74,12 @@ __device__ __forceinline__ int bucket_of(float x, const float* tf) {
     return c;
 }
 
-// The row: coalesced 128-bit loads into shared memory first (all of a thread's loads are in flight together), then
-// block absmax and normalised values in place (as in lowra_encode).  Ends with a barrier.
+// The row: coalesced 128-bit loads (all of a thread's loads in flight together); sixteen neighbouring lanes hold one
+// 64-element block between them, so the block's absmax is four shuffles away and the values go to shared memory
+// already normalised (as in lowra_encode: reciprocal rounded to nearest, one multiplication).  Ends with a barrier.
 __device__ void load_row(const LearnParams& P, int r, float* xs, float* ws) {
-    const int K = P.K, nb = K / kBlock;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K = P.K;
+    const int tid = threadIdx.x;
     const float* wrow = P.W + (size_t)r * K;
     for (int i0 = 0; i0 < K; i0 += 4 * 4 * kLearnThreads) {
         float4 v[4];
@@ -74,19 +90,17 @@ __device__ void load_row(const LearnParams& P, int r, float* xs, float* ws) {
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const int i = i0 + 4 * (u * kLearnThreads + tid);
-            if (i < K) *reinterpret_cast<float4*>(xs + i) = v[u];
-        }
-    }
-    __syncthreads();
-    for (int g = warp; g < nb; g += kLearnWarps) {
-        const float2 v = *reinterpret_cast<const float2*>(xs + g * kBlock + 2 * lane);
-        float m = fmaxf(fabsf(v.x), fabsf(v.y));
+            const int i = i0 + 4 * (u * kLearnThreads + tid);   // K is a multiple of 128: a warp is in or out as a whole
+            float m = fmaxf(fmaxf(fabsf(v[u].x), fabsf(v[u].y)), fmaxf(fabsf(v[u].z), fabsf(v[u].w)));
 #pragma unroll
-        for (int d = 16; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
-        const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
-        *reinterpret_cast<float2*>(xs + g * kBlock + 2 * lane) = make_float2(__fmul_rn(v.x, inv), __fmul_rn(v.y, inv));
-        if (lane == 0) ws[g] = m;
+            for (int d = 8; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
+            const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
+            if (i < K) {
+                *reinterpret_cast<float4*>(xs + i) =
+                    make_float4(__fmul_rn(v[u].x, inv), __fmul_rn(v[u].y, inv), __fmul_rn(v[u].z, inv), __fmul_rn(v[u].w, inv));
+                if ((tid & 15) == 0) ws[i / kBlock] = m;
+            }
+        }
     }
     __syncthreads();
 }
@@ -145,14 +159,14 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
                     cd[j] = fma(w, (double)cq[j], cd[j]);
                 }
             }
+            double v[2 * Lv];
 #pragma unroll
             for (int j = 0; j < Lv; ++j) {
-                const double pn = (j == 0 || j == Lv - 1) ? cn[j] : cn[j] - cn[j + 1];
-                const double pd = (j == 0 || j == Lv - 1) ? cd[j] : cd[j] - cd[j + 1];
-                const double sn = warp_sum(pn);
-                const double sd = warp_sum(pd);
-                if (lane == 0) { red[(2 * j) * kLearnWarps + warp] = sn; red[(2 * j + 1) * kLearnWarps + warp] = sd; }
+                v[2 * j] = (j == 0 || j == Lv - 1) ? cn[j] : cn[j] - cn[j + 1];
+                v[2 * j + 1] = (j == 0 || j == Lv - 1) ? cd[j] : cd[j] - cd[j + 1];
             }
+            warp_sums<2 * Lv>(v, lane);
+            if ((lane & (32 / (2 * Lv) - 1)) == 0) red[(lane / (32 / (2 * Lv))) * kLearnWarps + warp] = v[0];
         } else {
             // 16 buckets: the sums live in shared memory, one (w n, w) pair per thread and bucket; four elements at a
             // time, their bucket searches side by side
@@ -174,11 +188,17 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
                     acc2[b[u] * kLearnThreads + tid] = a;
                 }
             }
-#pragma unroll 4
-            for (int j = 0; j < Lv; ++j) {
-                const double2 a = acc2[j * kLearnThreads + tid];
-                const double sn = warp_sum(a.x), sd = warp_sum(a.y);
-                if (lane == 0) { red[(2 * j) * kLearnWarps + warp] = sn; red[(2 * j + 1) * kLearnWarps + warp] = sd; }
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {   // eight buckets = sixteen sums at a time
+                double v[16];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    const double2 a = acc2[(8 * half + j) * kLearnThreads + tid];
+                    v[2 * j] = a.x;
+                    v[2 * j + 1] = a.y;
+                }
+                warp_sums<16>(v, lane);
+                if ((lane & 1) == 0) red[(16 * half + lane / 2) * kLearnWarps + warp] = v[0];
             }
         }
         __syncthreads();
@@ -193,13 +213,21 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
                 y[lane] = yv;
             }
             const double yn = __shfl_down_sync(0xffffffffu, yv, 1);
+            bool same = true;
             if (lane + 1 < Lv) {
                 const double tm = (yv + yn) * 0.5;
+                const float tn = __double2float_ru(tm);
+                same = tn == tf[lane];
                 t[lane] = tm;
-                tf[lane] = __double2float_ru(tm);
+                tf[lane] = tn;
             }
+            // thresholds that have not moved (as the fp32 numbers the elements are compared with) assign every element
+            // as before: the next round would add the same sums up in the same order and change nothing, nor any later one
+            const bool settled = __all_sync(0xffffffffu, same);
+            if (lane == 0) tf[16] = settled ? 1.0f : 0.0f;
         }
         __syncthreads();
+        if (tf[16] != 0.0f) break;
     }
 
     // ---- tables: fp32 levels, midpoints of the fp32 levels; unused levels 0, unused thresholds +inf
@@ -226,7 +254,7 @@ __global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_const
     double* acc = red + 2 * 16 * kLearnWarps;
     float* xs = reinterpret_cast<float*>(acc + (FOUR ? 2 * 16 * kLearnThreads : 0));
     float* ws = xs + P.K;
-    float* tf = ws + P.K / kBlock;   // [16] thresholds as fp32 upper neighbours
+    float* tf = ws + P.K / kBlock;   // [16] thresholds as fp32 upper neighbours, [16] "this row has settled"
     pdl_enter();
     for (int r = blockIdx.x; r < P.N; r += gridDim.x) {
         load_row(P, r, xs, ws);
@@ -256,7 +284,7 @@ namespace {
 template <bool ALL3, bool FOUR>
 lowra_status launch_learn_kernel(const LearnParams& P, void* stream) {
     const size_t smem = (32 + 2 * 16 * kLearnWarps + (FOUR ? 2 * 16 * kLearnThreads : 0)) * sizeof(double) +
-                        ((size_t)P.K + (size_t)P.K / kBlock + 16) * sizeof(float);
+                        ((size_t)P.K + (size_t)P.K / kBlock + 20) * sizeof(float);
     if (smem > 200 * 1024) return LOWRA_ERR_SHAPE;   // the row has to fit into shared memory (K <= 40960)
     static SmemLimit limit = {};
     if (ensure_smem_limit(reinterpret_cast<const void*>(learn_kernel<ALL3, FOUR>), smem, &limit) != LOWRA_OK) return LOWRA_ERR_CUDA;
