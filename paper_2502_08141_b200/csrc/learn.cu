@@ -10,12 +10,13 @@
 // midpoints of those fp32 levels (computed in fp64, rounded to fp32), in [N, 16] tables.
 //
 // One CTA per row at a time (persistent, grid-stride): the row is read from HBM once (4 bytes per element, the
-// kernel's only traffic), normalised and parked in shared memory; the T passes run out of shared memory.
+// kernel's only traffic), normalised on its way into shared memory; the T passes run out of shared memory.
 // Every thread keeps private fp64 sums per bucket: in registers for 1 and 2 bits, in a bank-conflict-free
 // slice of shared memory for 4 bits; the block's weight enters once per four elements (they are added up exactly
-// first); a fixed reduction tree adds the threads' sums up (warp shuffles, then across warps), so
+// first); a fixed reduction tree adds the threads' sums up (a halving exchange inside a warp, then across warps), so
 // results are reproducible from run to run - but the order of the fp64 operations is not the index order of a
-// serial loop, so sums agree with a serial implementation to rounding only.
+// serial loop, so sums agree with a serial implementation to rounding only.  One barrier per round; every warp forms
+// the new levels and thresholds itself; a row whose thresholds have settled (as fp32 numbers) skips its remaining rounds.
 #include <string.h>
 
 #include "lowra_common.cuh"
@@ -106,23 +107,31 @@ __device__ void load_row(const LearnParams& P, int r, float* xs, float* ws) {
 }
 
 // T rounds on the row parked in shared memory, at B bits; tables to maps_out / thr_out ([16] each).
+// One barrier per round: the warps leave their partial sums in shared memory (two buffers, used in turn), meet once, and
+// then EVERY warp forms the new levels and thresholds for itself - lane j holds level j and threshold j in registers, the
+// same numbers in every warp since they come from the same partial sums in the same order - so nobody waits for a
+// first warp to publish them.
 template <int B>
-__device__ void learn_row(const LearnParams& P, const float* xs, const float* ws, double* acc, double* red, double* yt,
-                          float* tf, float* maps_out, float* thr_out) {
+__device__ void learn_row(const LearnParams& P, const float* xs, const float* ws, double* acc, double* red2, float* tfw_all,
+                          float* maps_out, float* thr_out) {
     constexpr int Lv = 1 << B;      // levels
     constexpr int c = B >> 1;       // class index
     const int K = P.K;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    double* y = yt;          // [16] levels
-    double* t = yt + 16;     // [16] thresholds
-    if (tid < 16) {
-        y[tid] = P.init_y[c][tid];
-        t[tid] = P.init_t[c][tid];
-        tf[tid] = __double2float_ru(P.init_t[c][tid]);
+    float* tf = tfw_all + warp * 16;                      // 4 bits: this warp's copy of the thresholds (bucket search by index)
+    double ylane = lane < Lv ? P.init_y[c][lane] : 0.0;   // level `lane`
+    float tlane = lane + 1 < Lv ? __double2float_ru(P.init_t[c][lane]) : 0.0f;   // threshold `lane`: the least fp32 number >= it
+    float th[B <= 2 ? Lv - 1 : 1];                        // 1 and 2 bits: all thresholds in registers
+    if (B <= 2) {
+#pragma unroll
+        for (int j = 0; j < Lv - 1; ++j) th[j] = __double2float_ru(P.init_t[c][j]);
+    } else {
+        if (lane < 16) tf[lane] = tlane;
+        __syncwarp();
     }
-    __syncthreads();
 
     for (int it = 0; it < P.iterations; ++it) {
+        double* red = red2 + (it & 1) * (2 * 16 * kLearnWarps);
         // ---- one pass: private sums of w * n and w per bucket.  The weight is the same for the four elements a thread
         // takes at a time (they lie in one 64-element block), so the elements themselves are added up per bucket first
         // (exactly: four fp32 values in fp64) and counted, and the weight enters once per four elements and bucket.
@@ -132,11 +141,8 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
             // difference of two neighbours (which were added up over the same elements in the same order wherever the
             // bucket is empty, so that an empty bucket has exactly zero weight).
             double cn[Lv], cd[Lv];
-            float th[Lv - 1];
 #pragma unroll
             for (int j = 0; j < Lv; ++j) cn[j] = cd[j] = 0.0;
-#pragma unroll
-            for (int j = 0; j < Lv - 1; ++j) th[j] = tf[j];
             for (int q = tid; q < K / 4; q += kLearnThreads) {   // quad q = elements 4 q .. 4 q + 3, all in block q / 16
                 const float4 xv = *reinterpret_cast<const float4*>(xs + 4 * q);
                 const double w = (double)ws[q >> 4];
@@ -202,42 +208,42 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
             }
         }
         __syncthreads();
-        // ---- new levels (an empty bucket keeps its level), then midpoints: the first warp, a shuffle in between
-        if (warp == 0) {
-            double yv = 0.0;
-            if (lane < Lv) {
-                double sn = 0.0, sd = 0.0;
+        // ---- new levels (an empty bucket keeps its level), then midpoints with a shuffle in between: every warp
+        if (lane < Lv) {
+            double sn = 0.0, sd = 0.0;
 #pragma unroll
-                for (int w2 = 0; w2 < kLearnWarps; ++w2) { sn += red[(2 * lane) * kLearnWarps + w2]; sd += red[(2 * lane + 1) * kLearnWarps + w2]; }
-                yv = (sd > 0.0) ? sn / sd : y[lane];
-                y[lane] = yv;
-            }
-            const double yn = __shfl_down_sync(0xffffffffu, yv, 1);
-            bool same = true;
-            if (lane + 1 < Lv) {
-                const double tm = (yv + yn) * 0.5;
-                const float tn = __double2float_ru(tm);
-                same = tn == tf[lane];
-                t[lane] = tm;
-                tf[lane] = tn;
-            }
-            // thresholds that have not moved (as the fp32 numbers the elements are compared with) assign every element
-            // as before: the next round would add the same sums up in the same order and change nothing, nor any later one
-            const bool settled = __all_sync(0xffffffffu, same);
-            if (lane == 0) tf[16] = settled ? 1.0f : 0.0f;
+            for (int w2 = 0; w2 < kLearnWarps; ++w2) { sn += red[(2 * lane) * kLearnWarps + w2]; sd += red[(2 * lane + 1) * kLearnWarps + w2]; }
+            if (sd > 0.0) ylane = sn / sd;
         }
-        __syncthreads();
-        if (tf[16] != 0.0f) break;
+        const double yn = __shfl_down_sync(0xffffffffu, ylane, 1);
+        bool same = true;
+        if (lane + 1 < Lv) {
+            const float tn = __double2float_ru((ylane + yn) * 0.5);
+            same = tn == tlane;
+            tlane = tn;
+        }
+        if (B <= 2) {
+#pragma unroll
+            for (int j = 0; j < Lv - 1; ++j) th[j] = __shfl_sync(0xffffffffu, tlane, j);
+        } else {
+            if (lane < 16) tf[lane] = tlane;
+            __syncwarp();
+        }
+        // thresholds that have not moved (as the fp32 numbers the elements are compared with) assign every element
+        // as before: the next round would add the same sums up in the same order and change nothing, nor any later one
+        if (__all_sync(0xffffffffu, same)) break;
     }
 
     // ---- tables: fp32 levels, midpoints of the fp32 levels; unused levels 0, unused thresholds +inf
-    if (tid < kTableStride) {
-        const float m = (tid < Lv) ? (float)y[tid] : 0.0f;
-        const float mn = (tid + 1 < Lv) ? (float)y[tid + 1] : 0.0f;
-        maps_out[tid] = m;
-        thr_out[tid] = (tid + 1 < Lv) ? (float)(((double)m + (double)mn) * 0.5) : __int_as_float(0x7f800000);
+    if (warp == 0) {
+        const float m = (lane < Lv) ? (float)ylane : 0.0f;
+        const float mn = __shfl_down_sync(0xffffffffu, m, 1);
+        if (lane < kTableStride) {
+            maps_out[lane] = m;
+            thr_out[lane] = (lane + 1 < Lv) ? (float)(((double)m + (double)mn) * 0.5) : __int_as_float(0x7f800000);
+        }
     }
-    __syncthreads();   // the tables and sums in shared memory are reused by the next run, the row buffer by the next row
+    __syncthreads();   // the sums in shared memory are reused by the next run, the row buffer by the next row
 }
 
 // FOUR = false: for weights without 4-bit rows.  Only the 4-bit runs need the 32 KB of per-thread bucket sums in shared
@@ -248,13 +254,12 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
 template <bool ALL3, bool FOUR>
 __global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_constant__ LearnParams P) {
     extern __shared__ __align__(16) unsigned char learn_smem[];
-    // [16 + 16 doubles levels/thresholds][2 * 16 * warps doubles reduction][FOUR: 2 * 16 * threads doubles sums][K floats][nb floats][16 floats]
-    double* yt = reinterpret_cast<double*>(learn_smem);
-    double* red = yt + 32;
-    double* acc = red + 2 * 16 * kLearnWarps;
+    // [2 x 2 * 16 * warps doubles partial sums][FOUR: 2 * 16 * threads doubles sums][K floats][nb floats][warps x 16 floats]
+    double* red2 = reinterpret_cast<double*>(learn_smem);
+    double* acc = red2 + 2 * 2 * 16 * kLearnWarps;
     float* xs = reinterpret_cast<float*>(acc + (FOUR ? 2 * 16 * kLearnThreads : 0));
     float* ws = xs + P.K;
-    float* tf = ws + P.K / kBlock;   // [16] thresholds as fp32 upper neighbours, [16] "this row has settled"
+    float* tfw = ws + P.K / kBlock;   // 4-bit runs: a copy of the thresholds (fp32 upper neighbours) per warp
     pdl_enter();
     for (int r = blockIdx.x; r < P.N; r += gridDim.x) {
         load_row(P, r, xs, ws);
@@ -263,14 +268,14 @@ __global__ void __launch_bounds__(kLearnThreads) learn_kernel(const __grid_const
         if (ALL3) {
             // the row under every precision, from the one copy in shared memory
             const size_t plane = (size_t)P.N * kTableStride;
-            learn_row<1>(P, xs, ws, acc, red, yt, tf, m, h);
-            learn_row<2>(P, xs, ws, acc, red, yt, tf, m + plane, h + plane);
-            if (FOUR) learn_row<4>(P, xs, ws, acc, red, yt, tf, m + 2 * plane, h + 2 * plane);
+            learn_row<1>(P, xs, ws, acc, red2, tfw, m, h);
+            learn_row<2>(P, xs, ws, acc, red2, tfw, m + plane, h + plane);
+            if (FOUR) learn_row<4>(P, xs, ws, acc, red2, tfw, m + 2 * plane, h + 2 * plane);
         } else {
             const int b = P.L.precs[r];
-            if (b == 1) learn_row<1>(P, xs, ws, acc, red, yt, tf, m, h);
-            else if (b == 2) learn_row<2>(P, xs, ws, acc, red, yt, tf, m, h);
-            else if (FOUR) learn_row<4>(P, xs, ws, acc, red, yt, tf, m, h);
+            if (b == 1) learn_row<1>(P, xs, ws, acc, red2, tfw, m, h);
+            else if (b == 2) learn_row<2>(P, xs, ws, acc, red2, tfw, m, h);
+            else if (FOUR) learn_row<4>(P, xs, ws, acc, red2, tfw, m, h);
         }
     }
 }
@@ -283,15 +288,15 @@ namespace {
 // validation shared by the two entry points is done by the callers; this fills the tables and launches
 template <bool ALL3, bool FOUR>
 lowra_status launch_learn_kernel(const LearnParams& P, void* stream) {
-    const size_t smem = (32 + 2 * 16 * kLearnWarps + (FOUR ? 2 * 16 * kLearnThreads : 0)) * sizeof(double) +
-                        ((size_t)P.K + (size_t)P.K / kBlock + 20) * sizeof(float);
+    const size_t smem = (2 * 2 * 16 * kLearnWarps + (FOUR ? 2 * 16 * kLearnThreads : 0)) * sizeof(double) +
+                        ((size_t)P.K + (size_t)P.K / kBlock + 16 * kLearnWarps) * sizeof(float);
     if (smem > 200 * 1024) return LOWRA_ERR_SHAPE;   // the row has to fit into shared memory (K <= 40960)
     static SmemLimit limit = {};
     if (ensure_smem_limit(reinterpret_cast<const void*>(learn_kernel<ALL3, FOUR>), smem, &limit) != LOWRA_OK) return LOWRA_ERR_CUDA;
     const int per_sm = (int)((220u * 1024u) / (smem + 1024u));
     const int sms = device_sm_count();
     if (sms < 1) return LOWRA_ERR_CUDA;
-    const int cap = sms * (per_sm < 1 ? 1 : (per_sm > 16 ? 16 : per_sm));
+    const int cap = sms * (per_sm < 1 ? 1 : (per_sm > 8 ? 8 : per_sm));   // 64 registers per thread: eight CTAs per SM at most
     const unsigned grid = (unsigned)(P.N < cap ? P.N : cap);
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
