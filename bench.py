@@ -541,6 +541,12 @@ def run_gpu(args):
     fused_calls = [(d["N"], d["K"], M) for M in token_counts for d in dev]
     if with_backward:
         fused_calls += [(d["K"], d["N"], M) for M in token_counts for d in dev]   # backward reads dY [M, N], writes dX [M, K]
+    # the steps that ran before the power limiter set in (within 2 % of the fastest step): the same figure over those alone
+    fastest = min(fused_ms_by_step)
+    quick = [m for m in fused_ms_by_step if m <= 1.02 * fastest]
+    tf_quick = flops_step / (sum(quick) / len(quick) * 1e-3) / 1e12
+    before_limit = {"steps": len(quick), "of": args.steps, "achieved": tf_quick, "frac_burst": tf_quick / P["tensor_burst"],
+                    "what": "fused phases of the steps within 2 % of the fastest one (the power limiter slows the later steps of a run, see ms_by_step)"}
     roofline = {"bound": "tensor", "kernel": "fused_kernel (forward" + (" + backward-input" if with_backward else "") + " calls" +
                                               (", prologue launch included)" if args.deal_per_call else ")"),
                 "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
@@ -553,6 +559,7 @@ def run_gpu(args):
                                   "workload 3 (profiles/fused_backward_input_11008x4096_m4096_streamk.md), scaled by the "
                                   "input + output bytes of this step's average launch",
                 "ms_by_step": fused_ms_by_step if args.steps <= 64 else fused_ms_by_step[:32] + fused_ms_by_step[-32:],
+                "before_power_limit": before_limit,
                 "secondary": secondary}
 
     # ---- end to end: host buffers, pinned, copies inside the timed region (the first seven matrices of the workload)
