@@ -12,7 +12,7 @@
 // One CTA per row at a time (persistent, grid-stride): the row is read from HBM once (4 bytes per element, the
 // kernel's only traffic), normalised on its way into shared memory; the T passes run out of shared memory.
 // Every thread keeps private fp64 sums per bucket: in registers for 1 and 2 bits, in a bank-conflict-free
-// slice of shared memory for 4 bits; the block's weight enters once per four elements (they are added up exactly
+// slice of shared memory for 4 bits; the block's weight enters once per sixteen elements (they are added up exactly
 // first); a fixed reduction tree adds the threads' sums up (a halving exchange inside a warp, then across warps), so
 // results are reproducible from run to run - but the order of the fp64 operations is not the index order of a
 // serial loop, so sums agree with a serial implementation to rounding only.  One barrier per round; every warp forms
@@ -75,6 +75,12 @@ __device__ __forceinline__ int bucket_of(float x, const float* tf) {
     return c;
 }
 
+// Where group of four elements number q of a row lies in shared memory (in units of 16 bytes).  The rounds read the row
+// sixteen elements = four groups per thread at a time (eight in the 4-bit rounds); with the groups of every set of four
+// exchanged among themselves by the number of the pair of sets they are in, the eight lanes that share a shared-memory
+// wavefront fall into eight different 16-byte columns, in the rounds' reads and in the loader's writes alike.
+__device__ __forceinline__ int quad_slot(int q) { return q ^ ((q >> 3) & 3); }
+
 // The row: coalesced 128-bit loads (all of a thread's loads in flight together); sixteen neighbouring lanes hold one
 // 64-element block between them, so the block's absmax is four shuffles away and the values go to shared memory
 // already normalised (as in lowra_encode: reciprocal rounded to nearest, one multiplication).  Ends with a barrier.
@@ -97,7 +103,7 @@ __device__ void load_row(const LearnParams& P, int r, float* xs, float* ws) {
             for (int d = 8; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
             const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
             if (i < K) {
-                *reinterpret_cast<float4*>(xs + i) =
+                *reinterpret_cast<float4*>(xs + 4 * quad_slot(i >> 2)) =
                     make_float4(__fmul_rn(v[u].x, inv), __fmul_rn(v[u].y, inv), __fmul_rn(v[u].z, inv), __fmul_rn(v[u].w, inv));
                 if ((tid & 15) == 0) ws[i / kBlock] = m;
             }
@@ -132,9 +138,9 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
 
     for (int it = 0; it < P.iterations; ++it) {
         double* red = red2 + (it & 1) * (2 * 16 * kLearnWarps);
-        // ---- one pass: private sums of w * n and w per bucket.  The weight is the same for the four elements a thread
-        // takes at a time (they lie in one 64-element block), so the elements themselves are added up per bucket first
-        // (exactly: four fp32 values in fp64) and counted, and the weight enters once per four elements and bucket.
+        // ---- one pass: private sums of w * n and w per bucket.  The weight is the same for the sixteen elements a thread
+        // takes at a time (a quarter of a 64-element block), so the elements themselves are added up per bucket first
+        // (exactly: sixteen fp32 values in fp64) and counted, and the weight enters once per sixteen elements and bucket.
         if (B <= 2) {
             // Few buckets: no bucket index at all.  cn[0] / cd[0] take the elements below the first threshold, cn[j] /
             // cd[j] (j >= 1) everything at or above threshold j - 1 - predicated adds - and a bucket's sums are the
@@ -143,16 +149,19 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
             double cn[Lv], cd[Lv];
 #pragma unroll
             for (int j = 0; j < Lv; ++j) cn[j] = cd[j] = 0.0;
-            for (int q = tid; q < K / 4; q += kLearnThreads) {   // quad q = elements 4 q .. 4 q + 3, all in block q / 16
-                const float4 xv = *reinterpret_cast<const float4*>(xs + 4 * q);
-                const double w = (double)ws[q >> 4];
-                const float xf[4] = {xv.x, xv.y, xv.z, xv.w};
+            for (int run = tid; run < K / 16; run += kLearnThreads) {   // elements 16 run .. 16 run + 15, all in block run / 4
+                const float4 xa = *reinterpret_cast<const float4*>(xs + 4 * quad_slot(4 * run));
+                const float4 xb = *reinterpret_cast<const float4*>(xs + 4 * quad_slot(4 * run + 1));
+                const float4 xc = *reinterpret_cast<const float4*>(xs + 4 * quad_slot(4 * run + 2));
+                const float4 xd = *reinterpret_cast<const float4*>(xs + 4 * quad_slot(4 * run + 3));
+                const double w = (double)ws[run >> 2];
+                const float xf[16] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w, xc.x, xc.y, xc.z, xc.w, xd.x, xd.y, xd.z, xd.w};
                 double sq[Lv];
                 int cq[Lv];
 #pragma unroll
                 for (int j = 0; j < Lv; ++j) { sq[j] = 0.0; cq[j] = 0; }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < 16; ++u) {
                     const double x = (double)xf[u];
                     if (th[0] <= xf[u]) { sq[1] += x; ++cq[1]; } else { sq[0] += x; ++cq[0]; }
 #pragma unroll
@@ -174,20 +183,21 @@ __device__ void learn_row(const LearnParams& P, const float* xs, const float* ws
             warp_sums<2 * Lv>(v, lane);
             if ((lane & (32 / (2 * Lv) - 1)) == 0) red[(lane / (32 / (2 * Lv))) * kLearnWarps + warp] = v[0];
         } else {
-            // 16 buckets: the sums live in shared memory, one (w n, w) pair per thread and bucket; four elements at a
+            // 16 buckets: the sums live in shared memory, one (w n, w) pair per thread and bucket; eight elements at a
             // time, their bucket searches side by side
             double2* acc2 = reinterpret_cast<double2*>(acc);
 #pragma unroll
             for (int j = 0; j < Lv; ++j) acc2[j * kLearnThreads + tid] = make_double2(0.0, 0.0);
-            for (int q = tid; q < K / 4; q += kLearnThreads) {
-                const float4 xv = *reinterpret_cast<const float4*>(xs + 4 * q);
-                const double w = (double)ws[q >> 4];
-                const float xf[4] = {xv.x, xv.y, xv.z, xv.w};
-                int b[4];
+            for (int run = tid; run < K / 8; run += kLearnThreads) {
+                const float4 xa = *reinterpret_cast<const float4*>(xs + 4 * quad_slot(2 * run));
+                const float4 xb = *reinterpret_cast<const float4*>(xs + 4 * quad_slot(2 * run + 1));
+                const double w = (double)ws[run >> 3];
+                const float xf[8] = {xa.x, xa.y, xa.z, xa.w, xb.x, xb.y, xb.z, xb.w};
+                int b[8];
 #pragma unroll
-                for (int u = 0; u < 4; ++u) b[u] = bucket_of<B>(xf[u], tf);
+                for (int u = 0; u < 8; ++u) b[u] = bucket_of<B>(xf[u], tf);
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
+                for (int u = 0; u < 8; ++u) {
                     double2 a = acc2[b[u] * kLearnThreads + tid];
                     a.x = fma(w, (double)xf[u], a.x);
                     a.y += w;
