@@ -318,10 +318,6 @@ __device__ __forceinline__ void st_shared_f32(uint32_t saddr, float v) {
 __device__ __forceinline__ void cp_async_4(uint32_t saddr, const void* gptr) {
     asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(saddr), "l"(gptr) : "memory");
 }
-__device__ __forceinline__ void cp_async_16(uint32_t saddr, const void* gptr, bool valid) {
-    const int sz = valid ? 16 : 0;  // zero-fill when out of range
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(saddr), "l"(gptr), "r"(sz) : "memory");
-}
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
