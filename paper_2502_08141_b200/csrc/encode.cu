@@ -12,7 +12,9 @@
 //   1 bit : one subtract and one funnel shift per element,
 //   2 bits: three sign planes (one per threshold; sorted thresholds) combined into the two code planes with
 //           two logic ops per 32 elements, then interleaved,
-//   4 bits: branch-free binary search over the 15 thresholds held in registers.
+//   4 bits: branch-free binary search over the row's 15 thresholds, which lie in the warp's slice of shared memory
+//           (four look-ups by index per element; kept in registers and picked with selects, a search costs 20
+//           instructions on the half-rate pipe).
 // A lane ends up with 4, 8 or 16 packed bytes: the warp writes 128, 256 or 512 contiguous bytes.
 //
 // Bit-exactness with the definition rests on: the block maximum is exact in fp32; the reciprocal is the
@@ -69,15 +71,16 @@ __device__ __forceinline__ void encode_chunk(const EncodeParams& P, int p, int c
     }
     const float* trow = P.thresholds + (size_t)r * kTableStride;
     float t0 = 0.f, t1 = 0.f, t2 = 0.f;
-    Thresholds4 t4;
+    float* ts = reinterpret_cast<float*>(stage + 32 * kSegBytes);   // 4 bits: the row's 15 thresholds, searched by index
     if (B == 1) {
         t0 = __ldg(trow);
     } else if (B == 2) {
         t0 = __ldg(trow); t1 = __ldg(trow + 1); t2 = __ldg(trow + 2);
-    } else {
-        t4.load(trow);
+    } else if (lane < 16) {
+        t0 = __ldg(trow + lane);
     }
     __syncwarp();   // the previous task's reads of the stage are over
+    if (B == 4 && lane < 16) ts[lane] = t0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         const int e = (i * 32 + lane) * 4;
@@ -129,7 +132,15 @@ __device__ __forceinline__ void encode_chunk(const EncodeParams& P, int p, int c
         for (int q = 0; q < 4; ++q) {
             uint32_t acc = 0u;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) acc |= t4.code(__fmul_rn(x[8 * q + i], inv)) << (4 * i);
+            for (int i = 0; i < 8; ++i) {
+                // number of thresholds <= n (sorted thresholds): branch-free binary search, four look-ups by index
+                const float n = __fmul_rn(x[8 * q + i], inv);
+                uint32_t k = ts[7] <= n ? 8u : 0u;
+                k += ts[k + 3] <= n ? 4u : 0u;
+                k += ts[k + 1] <= n ? 2u : 0u;
+                k += ts[k] <= n ? 1u : 0u;
+                acc |= k << (4 * i);
+            }
             w[q] = acc;
         }
         if (live) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -137,7 +148,7 @@ __device__ __forceinline__ void encode_chunk(const EncodeParams& P, int p, int c
 }
 
 __global__ void __launch_bounds__(kEncodeThreads, 3) encode_kernel(const EncodeParams P) {
-    __shared__ __align__(16) unsigned char stage_all[kEncodeWarps][32 * kSegBytes];
+    __shared__ __align__(16) unsigned char stage_all[kEncodeWarps][32 * kSegBytes + 64];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     unsigned char* stage = stage_all[warp];

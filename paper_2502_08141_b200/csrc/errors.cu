@@ -34,17 +34,23 @@ struct ErrParams {
     float* residual;          // [N, K] or null
 };
 
-// level of the bucket of n: the number of thresholds <= n picks the level (thresholds sorted, as the encoder assumes)
+// level of the bucket of n: the number of thresholds <= n picks the level (thresholds sorted, as the encoder assumes).
+// 4 bits: levels at tab[0 .. 15], thresholds at tab[16 .. 30] of the warp's table in shared memory; branch-free binary
+// search, four look-ups by index (the same search as lowra_encode's).
 template <int B>
-__device__ __forceinline__ float level_of(float n, const float (&t)[3], const Thresholds4& t4, const float (&y)[4],
-                                          const float* y_smem) {
+__device__ __forceinline__ float level_of(float n, const float (&t)[3], const float (&y)[4], const float* tab) {
     if (B == 1) return t[0] <= n ? y[1] : y[0];
     if (B == 2) {
         const bool hi = t[1] <= n;
         const bool lo = (hi ? t[2] : t[0]) <= n;
         return hi ? (lo ? y[3] : y[2]) : (lo ? y[1] : y[0]);
     }
-    return y_smem[t4.code(n)];
+    const float* ts = tab + 16;
+    int k = ts[7] <= n ? 8 : 0;
+    k += ts[k + 3] <= n ? 4 : 0;
+    k += ts[k + 1] <= n ? 2 : 0;
+    k += ts[k] <= n ? 1 : 0;
+    return tab[k];
 }
 
 template <int B>
@@ -56,16 +62,14 @@ __device__ void error_row(const ErrParams& P, int r, float* y_warp) {
     const float* trow = P.thresholds + (size_t)r * kTableStride;
     const float* yrow = P.maps + (size_t)r * kTableStride;
     float t[3] = {0.f, 0.f, 0.f}, y[4] = {0.f, 0.f, 0.f, 0.f};
-    Thresholds4 t4;
     if (B == 1) {
         t[0] = __ldg(trow); y[0] = __ldg(yrow); y[1] = __ldg(yrow + 1);
     } else if (B == 2) {
         t[0] = __ldg(trow); t[1] = __ldg(trow + 1); t[2] = __ldg(trow + 2);
         y[0] = __ldg(yrow); y[1] = __ldg(yrow + 1); y[2] = __ldg(yrow + 2); y[3] = __ldg(yrow + 3);
     } else {
-        t4.load(trow);
         __syncwarp();   // the previous row's look-ups are over
-        if (lane < 16) y_warp[lane] = __ldg(yrow + lane);
+        if (lane < 16) { y_warp[lane] = __ldg(yrow + lane); y_warp[16 + lane] = __ldg(trow + lane); }
         __syncwarp();
     }
 
@@ -95,10 +99,10 @@ __device__ void error_row(const ErrParams& P, int r, float* y_warp) {
             for (int d = 8; d >= 1; d >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, d));
             const float inv = (m == 0.0f) ? 0.0f : __frcp_rn(m);
             // w_hat of the four elements, rounded to bf16 two at a time
-            const float l0 = __fmul_rn(level_of<B>(__fmul_rn(x[u].x, inv), t, t4, y, y_warp), m);
-            const float l1 = __fmul_rn(level_of<B>(__fmul_rn(x[u].y, inv), t, t4, y, y_warp), m);
-            const float l2 = __fmul_rn(level_of<B>(__fmul_rn(x[u].z, inv), t, t4, y, y_warp), m);
-            const float l3 = __fmul_rn(level_of<B>(__fmul_rn(x[u].w, inv), t, t4, y, y_warp), m);
+            const float l0 = __fmul_rn(level_of<B>(__fmul_rn(x[u].x, inv), t, y, y_warp), m);
+            const float l1 = __fmul_rn(level_of<B>(__fmul_rn(x[u].y, inv), t, y, y_warp), m);
+            const float l2 = __fmul_rn(level_of<B>(__fmul_rn(x[u].z, inv), t, y, y_warp), m);
+            const float l3 = __fmul_rn(level_of<B>(__fmul_rn(x[u].w, inv), t, y, y_warp), m);
             const uint32_t h01 = pack_bf16x2(l0, l1), h23 = pack_bf16x2(l2, l3);
             float4 res;
             res.x = __fsub_rn(x[u].x, __uint_as_float(h01 << 16));
@@ -121,7 +125,7 @@ __device__ void error_row(const ErrParams& P, int r, float* y_warp) {
 }
 
 __global__ void __launch_bounds__(kErrThreads) error_kernel(const ErrParams P) {
-    __shared__ float y_smem[kErrWarps][16];
+    __shared__ float y_smem[kErrWarps][32];   // per warp: the 16 levels and 15 thresholds of a 4-bit row
     pdl_enter();
     const int warp = threadIdx.x >> 5;
     float* y_warp = y_smem[warp];
@@ -144,7 +148,7 @@ struct Err3Params {
 };
 
 __global__ void __launch_bounds__(kErrThreads) error3_kernel(const Err3Params P) {
-    __shared__ float y_smem[kErrWarps][16];
+    __shared__ float y_smem[kErrWarps][32];   // per warp: the 16 levels and 15 thresholds of the row's 4-bit codebook
     pdl_enter();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     float* y_warp = y_smem[warp];
@@ -158,10 +162,8 @@ __global__ void __launch_bounds__(kErrThreads) error3_kernel(const Err3Params P)
         const float ya[4] = {__ldg(y1), __ldg(y1 + 1), 0.f, 0.f};
         const float tb[3] = {__ldg(t1 + plane), __ldg(t1 + plane + 1), __ldg(t1 + plane + 2)};
         const float yb[4] = {__ldg(y1 + plane), __ldg(y1 + plane + 1), __ldg(y1 + plane + 2), __ldg(y1 + plane + 3)};
-        Thresholds4 t4;
-        t4.load(t1 + 2 * plane);
         __syncwarp();   // the previous row's look-ups are over
-        if (lane < 16) y_warp[lane] = __ldg(y1 + 2 * plane + lane);
+        if (lane < 16) { y_warp[lane] = __ldg(y1 + 2 * plane + lane); y_warp[16 + lane] = __ldg(t1 + 2 * plane + lane); }
         __syncwarp();
         double acc1 = 0.0, acc2 = 0.0, acc4 = 0.0;
         float4 nxt[kErrBatch];
@@ -197,9 +199,9 @@ __global__ void __launch_bounds__(kErrThreads) error3_kernel(const Err3Params P)
                     const float r2 = __fsub_rn(xs[2], __uint_as_float(h23 << 16)), r3 = __fsub_rn(xs[3], __uint_as_float(h23 & 0xFFFF0000u));
                     return __fadd_rn(__fadd_rn(__fmul_rn(r0, r0), __fmul_rn(r1, r1)), __fadd_rn(__fmul_rn(r2, r2), __fmul_rn(r3, r3)));
                 };
-                const float q1 = group([&](float v) { return level_of<1>(v, ta, t4, ya, y_warp); });
-                const float q2 = group([&](float v) { return level_of<2>(v, tb, t4, yb, y_warp); });
-                const float q4 = group([&](float v) { return level_of<4>(v, tb, t4, yb, y_warp); });
+                const float q1 = group([&](float v) { return level_of<1>(v, ta, ya, y_warp); });
+                const float q2 = group([&](float v) { return level_of<2>(v, tb, yb, y_warp); });
+                const float q4 = group([&](float v) { return level_of<4>(v, tb, yb, y_warp); });
                 if (i < n4) { acc1 += (double)q1; acc2 += (double)q2; acc4 += (double)q4; }
             }
         }

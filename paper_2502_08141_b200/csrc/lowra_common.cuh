@@ -81,35 +81,6 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return r;
 }
 
-// selp keeps the 15 thresholds in registers (a C ternary tree is turned into an indexed local array)
-__device__ __forceinline__ float sel(bool c, float a, float b) {
-    float r;
-    asm("{ .reg .pred p; setp.ne.u32 p, %3, 0; selp.f32 %0, %1, %2, p; }" : "=f"(r) : "f"(a), "f"(b), "r"((uint32_t)c));
-    return r;
-}
-
-struct Thresholds4 {
-    float t0, t1, t2, t3, t4, t5, t6, t7, t8, t9, t10, t11, t12, t13, t14;
-    __device__ __forceinline__ void load(const float* p) {
-        const float4 a = __ldg(reinterpret_cast<const float4*>(p));
-        const float4 b = __ldg(reinterpret_cast<const float4*>(p) + 1);
-        const float4 c = __ldg(reinterpret_cast<const float4*>(p) + 2);
-        const float4 d = __ldg(reinterpret_cast<const float4*>(p) + 3);
-        t0 = a.x; t1 = a.y; t2 = a.z; t3 = a.w; t4 = b.x; t5 = b.y; t6 = b.z; t7 = b.w;
-        t8 = c.x; t9 = c.y; t10 = c.z; t11 = c.w; t12 = d.x; t13 = d.y; t14 = d.z;
-    }
-    // number of thresholds <= n (sorted thresholds): branch-free binary search
-    __device__ __forceinline__ uint32_t code(float n) const {
-        const bool c3 = t7 <= n;
-        const bool c2 = sel(c3, t11, t3) <= n;
-        const float hi1 = sel(c2, t13, t9), lo1 = sel(c2, t5, t1);
-        const bool c1 = sel(c3, hi1, lo1) <= n;
-        const float q3 = sel(c1, t14, t12), q2 = sel(c1, t10, t8), q1 = sel(c1, t6, t4), q0 = sel(c1, t2, t0);
-        const bool c0 = sel(c3, sel(c2, q3, q2), sel(c2, q1, q0)) <= n;
-        return (c3 ? 8u : 0u) | (c2 ? 4u : 0u) | (c1 ? 2u : 0u) | (c0 ? 1u : 0u);
-    }
-};
-
 __device__ __forceinline__ uint4 ld_stream_v4(const void* p) {
     uint4 v;
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
