@@ -361,6 +361,17 @@ def run_gpu(args):
                     batch_members[("backward", u[0], M)] = [dict(common(dev[k]), act=dev[k]["G"][M], out=dev[k]["dX"][M]) for k in u]
             all_ws.extend(batch_ws[(u[0], M)] for M in token_counts)
 
+    # encode and decode: the matrices of a layer in one launch each (lowra_encode_group / lowra_decode_group, up to eight
+    # members, the largest first), as a layer or a model is quantised; --no-batch: a call per matrix
+    codec_groups = []
+    if not args.no_batch:
+        gsz = 7 if len(dev) > lw.LOWRA_MAX_GROUP else lw.LOWRA_MAX_GROUP      # a model: layer by layer (seven matrices)
+        for g0 in range(0, len(dev), gsz):
+            idx = sorted(range(g0, min(g0 + gsz, len(dev))), key=lambda i: -dev[i]["N"] * dev[i]["K"])
+            codec_groups.append((
+                [dict(layout=dev[i]["layout"], W=dev[i]["W"], thresholds=dev[i]["thr"], packed=dev[i]["packed"], absmax=dev[i]["absmax"]) for i in idx],
+                [dict(layout=dev[i]["layout"], packed=dev[i]["packed"], absmax=dev[i]["absmax"], maps=dev[i]["maps"], out=dev[i]["What"]) for i in idx]))
+
     def run_unit(name, fn, u, M):
         if len(u) == 1 or name in ("encode", "decode"):
             for k in u:
@@ -383,6 +394,12 @@ def run_gpu(args):
                         c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                         c0.record(stream); fn(d, M); c1.record(stream)
                         per_call.append((name, M, i, c0, c1))
+                elif codec_groups and name == "encode":
+                    for enc_members, _ in codec_groups:
+                        lw.lowra_encode_group(enc_members)
+                elif codec_groups and name == "decode":
+                    for _, dec_members in codec_groups:
+                        lw.lowra_decode_group(dec_members)
                 else:
                     for u in units:
                         run_unit(name, fn, u, M)
@@ -483,7 +500,7 @@ def run_gpu(args):
     if out_layer >= SWEEP_BYTES:      # the step's own sweep is long enough (workload 5)
         for key, gbs, ms, by in (("decode", dec_gbs, phase_ms["decode"], dec_bytes), ("encode", enc_gbs, phase_ms["encode"], enc_bytes)):
             secondary[key] = {"bound": "hbm", "achieved": gbs, "peak": P["hbm"], "unit": "GB/s", "frac": gbs / P["hbm"],
-                              "frac_nominal_8TBs": gbs / 8000.0, "bytes": by, "ms": ms, "launches": len(dev),
+                              "frac_nominal_8TBs": gbs / 8000.0, "bytes": by, "ms": ms, "launches": len(codec_groups) if codec_groups else len(dev),
                               "how": "the step's own sweep over every matrix of the model (one event pair per phase)"}
     else:
         n_sets = int(math.ceil(SWEEP_BYTES / out_layer))
@@ -497,35 +514,55 @@ def run_gpu(args):
         # short launches come, so that the figure is the kernels' and not the interpreter's
         order = sorted(range(len(dev)), key=lambda i: -dev[i]["N"] * dev[i]["K"])
 
-        def decode_sweep():
+        def decode_sweep(grouped):
             for ws_ in what_sets:
-                for i in order:
-                    d = dev[i]
-                    lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=ws_[i])
+                if grouped:
+                    lw.lowra_decode_group([dict(layout=dev[i]["layout"], packed=dev[i]["packed"], absmax=dev[i]["absmax"],
+                                                maps=dev[i]["maps"], out=ws_[i]) for i in order])
+                else:
+                    for i in order:
+                        d = dev[i]
+                        lw.lowra_decode(d["layout"], d["packed"], d["absmax"], d["maps"], out=ws_[i])
 
-        def encode_sweep():
+        def encode_sweep(grouped):
             for j in range(n_sets):
-                for i in order:
-                    d = dev[i]
-                    pk, am = pk_sets[j % len(pk_sets)][i]
-                    lw.lowra_encode(d["layout"], w_sets[j % n_w][i], d["thr"], packed=pk, absmax=am)
+                if grouped:
+                    lw.lowra_encode_group([dict(layout=dev[i]["layout"], W=w_sets[j % n_w][i], thresholds=dev[i]["thr"],
+                                                packed=pk_sets[j % len(pk_sets)][i][0], absmax=pk_sets[j % len(pk_sets)][i][1])
+                                           for i in order])
+                else:
+                    for i in order:
+                        d = dev[i]
+                        pk, am = pk_sets[j % len(pk_sets)][i]
+                        lw.lowra_encode(d["layout"], w_sets[j % n_w][i], d["thr"], packed=pk, absmax=am)
 
-        for key, fn, by in (("decode", decode_sweep, dec_bytes), ("encode", encode_sweep, enc_bytes)):
-            fn()
+        def best_of_three(fn, grouped):
+            fn(grouped)
             torch.cuda.synchronize()
             best = None
             for _ in range(3):
                 a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record(stream); fn(); b.record(stream)
+                a.record(stream); fn(grouped); b.record(stream)
                 torch.cuda.synchronize()
                 ms = a.elapsed_time(b)
                 best = ms if best is None else min(best, ms)
+            return best
+
+        grouped = bool(codec_groups) and len(dev) <= lw.LOWRA_MAX_GROUP
+        for key, fn, by in (("decode", decode_sweep, dec_bytes), ("encode", encode_sweep, enc_bytes)):
+            best = best_of_three(fn, grouped)
             gbs = n_sets * by / (best * 1e-3) / 1e9
             secondary[key] = {"bound": "hbm", "achieved": gbs, "peak": P["hbm"], "unit": "GB/s", "frac": gbs / P["hbm"],
-                              "frac_nominal_8TBs": gbs / 8000.0, "bytes": n_sets * by, "ms": best, "launches": n_sets * len(dev),
+                              "frac_nominal_8TBs": gbs / 8000.0, "bytes": n_sets * by, "ms": best,
+                              "launches": n_sets * (1 if grouped else len(dev)),
                               "how": f"{n_sets} passes over the step's matrices back to back inside one event pair, every pass "
                                      f"into its own output buffers ({n_sets * out_layer / 1e9:.1f} GB of distinct decode output; "
-                                     f"encode reads {n_w} cop{'y' if n_w == 1 else 'ies'} of the weights in turn); best of 3"}
+                                     f"encode reads {n_w} cop{'y' if n_w == 1 else 'ies'} of the weights in turn); best of 3; " +
+                                     ("the matrices of a pass in one launch (lowra_%s_group)" % key if grouped else "a launch per matrix")}
+            if grouped:          # the same sweep with a launch per matrix, for comparison
+                single = best_of_three(fn, False)
+                secondary[key]["a_launch_per_matrix"] = {"achieved": n_sets * by / (single * 1e-3) / 1e9,
+                                                         "frac": n_sets * by / (single * 1e-3) / 1e9 / P["hbm"], "ms": single}
         del what_sets, w_sets, pk_sets
         # the packed codes in d["packed"] were not touched by the sweeps (they wrote their own buffers)
 
@@ -596,10 +633,12 @@ def run_gpu(args):
                                    "q, k and v projections (one shape, one input) through lowra_lora_forward_batch / "
                                    "lowra_lora_backward_input_batch, one launch per direction; every other matrix a call "
                                    "of its own; per_matrix figures are single calls",
+                       "codec_launches": ("encode and decode: the matrices of a layer in one launch each (lowra_encode_group / "
+                                          "lowra_decode_group); per_matrix figures are single calls") if codec_groups else "a launch per matrix",
                        "inputs": "q/k/v share X, gate/up share X, every other matrix its own; one output gradient per matrix",
                        "host_generation_s": round(t_gen, 1)},
             "phases": phases, "per_matrix": per_matrix, "roofline": roofline, "e2e": e2e, "cpu_baseline": cpu, "extras": extras,
-            "gpu_launches": args.steps * (2 * len(dev) + n_fused * (2 if args.deal_per_call else 1)), "clocks": clocks,
+            "gpu_launches": args.steps * ((2 * len(codec_groups) if codec_groups else 2 * len(dev)) + n_fused * (2 if args.deal_per_call else 1)), "clocks": clocks,
         }
         print(json.dumps(out))
     if world > 1:

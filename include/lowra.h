@@ -109,6 +109,30 @@ lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* packed_dev,
                           const float* maps_dev, uint16_t* W_bf16_dev, void* stream);
 
 /*
+ * Several matrices per launch (no counterpart in the paper; Appendix A.1 / A.2 describe one matrix): the weights of a
+ * layer, or of a model, are quantised and dequantised together, and a launch per matrix spends a good part of a small
+ * matrix's time (a 4096 x 4096 decode is 7 us of work) filling and draining the GPU.  lowra_encode_group and
+ * lowra_decode_group hand the chunks of up to LOWRA_MAX_GROUP matrices - any shapes, any layouts - to the warps of ONE
+ * launch, matrix after matrix in the order given (put the largest first).  Every member's result is bit for bit what the
+ * single call gives.  The array of members is host memory and is read before the call returns; the pointers inside it
+ * are device pointers with the meaning, layout and alignment of the arguments of lowra_encode / lowra_decode:
+ *   encode: W_dev, tables_dev = thresholds (in);  packed_dev, absmax_dev (out);  W_bf16_dev unused
+ *   decode: packed_dev, absmax_dev, tables_dev = mappings (in);  W_bf16_dev (out);  W_dev unused
+ * Errors: as the single calls, for the first member that is at fault; count < 1 or > LOWRA_MAX_GROUP -> LOWRA_ERR_SHAPE.
+ */
+#define LOWRA_MAX_GROUP 8
+typedef struct lowra_group_member {
+    const lowra_layout* layout;
+    const float* W_dev;
+    const float* tables_dev;
+    uint8_t* packed_dev;
+    float* absmax_dev;
+    uint16_t* W_bf16_dev;
+} lowra_group_member;
+lowra_status lowra_encode_group(const lowra_group_member* members_host, int32_t count, void* stream);
+lowra_status lowra_decode_group(const lowra_group_member* members_host, int32_t count, void* stream);
+
+/*
  * The paper's own buffer layout as a second storage variant (Appendix A.2: a thread of the
  * dequantisation kernel finds its offset into the quantised buffer from the channels' bit precisions):
  * rows in their ORIGINAL order, row r at byte offset sum_{i<r} K * b_i / 8; the absmax rows in original

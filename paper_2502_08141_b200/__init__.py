@@ -33,6 +33,7 @@ EXPORTS = (
     "lowra_learn_codebooks_all", "lowra_lora_forward_adapters", "lowra_batch_workspace_bytes",
     "lowra_lora_forward_batch", "lowra_lora_backward_input_batch", "lowra_lora_backward_adapters_reuse",
     "lowra_workspace_projection", "lowra_set_wait_limit", "lowra_diag_wait_expiry", "lowra_diag_drop_t_flags",
+    "lowra_encode_group", "lowra_decode_group",
 )
 
 
@@ -51,6 +52,11 @@ class _CLayout(ctypes.Structure):
         ("precs_dev", ctypes.c_void_p), ("perm_dev", ctypes.c_void_p), ("inv_perm_dev", ctypes.c_void_p),
         ("deal_dev", ctypes.c_void_p), ("natural_offsets_dev", ctypes.c_void_p),
     ]
+
+
+class _CGroupMember(ctypes.Structure):
+    _fields_ = [("layout", ctypes.POINTER(_CLayout)), ("W_dev", ctypes.c_void_p), ("tables_dev", ctypes.c_void_p),
+                ("packed_dev", ctypes.c_void_p), ("absmax_dev", ctypes.c_void_p), ("W_bf16_dev", ctypes.c_void_p)]
 
 
 class _CMember(ctypes.Structure):
@@ -81,6 +87,9 @@ def lib() -> ctypes.CDLL:
         L.lowra_encode.restype = ctypes.c_int
         L.lowra_decode.argtypes = [lp, vp, vp, vp, vp, vp]
         L.lowra_decode.restype = ctypes.c_int
+        for fn in (L.lowra_encode_group, L.lowra_decode_group):
+            fn.argtypes = [ctypes.POINTER(_CGroupMember), i32, vp]
+            fn.restype = ctypes.c_int
         L.lowra_workspace_bytes.argtypes = [lp, i32, i32]
         L.lowra_workspace_bytes.restype = ctypes.c_size_t
         L.lowra_deal_bytes.argtypes = [lp]
@@ -273,6 +282,61 @@ def lowra_decode(layout: Layout, packed: torch.Tensor, absmax: torch.Tensor, map
     code = lib().lowra_decode(layout.ref, _ptr(packed), _ptr(absmax), _ptr(maps), _ptr(out), _stream(stream))
     _check(code, "lowra_decode")
     return out
+
+
+LOWRA_MAX_GROUP = 8
+
+
+def lowra_encode_group(members, stream=None):
+    """Several matrices in one launch.  `members`: up to LOWRA_MAX_GROUP dicts with layout, W (fp32 [N, K]), thresholds
+    (fp32 [N, 16]) and, optionally, packed / absmax to write into.  Returns the list of (packed, absmax) pairs; every
+    pair is bit for bit what lowra_encode gives."""
+    n = len(members)
+    arr = (_CGroupMember * max(n, 1))()
+    outs = []
+    for i, m in enumerate(members):
+        layout, W, thr = m["layout"], m["W"], m["thresholds"]
+        _dev(W, torch.float32, "W")
+        _dev(thr, torch.float32, "thresholds")
+        if tuple(W.shape) != (layout.N, layout.K) or tuple(thr.shape) != (layout.N, 16):
+            raise ValueError("shape mismatch")
+        packed = m.get("packed")
+        absmax = m.get("absmax")
+        if packed is None:
+            packed = torch.empty(max(layout.packed_bytes, 16), dtype=torch.uint8, device=W.device)
+        if absmax is None:
+            absmax = torch.empty((layout.N, layout.K // 64), dtype=torch.float32, device=W.device)
+        _dev(packed, torch.uint8, "packed")
+        _dev(absmax, torch.float32, "absmax")
+        arr[i].layout = ctypes.pointer(layout.c)
+        arr[i].W_dev, arr[i].tables_dev = W.data_ptr(), thr.data_ptr()
+        arr[i].packed_dev, arr[i].absmax_dev, arr[i].W_bf16_dev = packed.data_ptr(), absmax.data_ptr(), None
+        outs.append((packed, absmax))
+    _check(lib().lowra_encode_group(arr, n, _stream(stream)), "lowra_encode_group")
+    return outs
+
+
+def lowra_decode_group(members, stream=None):
+    """Several matrices in one launch.  `members`: up to LOWRA_MAX_GROUP dicts with layout, packed, absmax, maps and,
+    optionally, out (bf16 [N, K]).  Returns the list of outputs; every one is bit for bit what lowra_decode gives."""
+    n = len(members)
+    arr = (_CGroupMember * max(n, 1))()
+    outs = []
+    for i, m in enumerate(members):
+        layout, packed, absmax, maps = m["layout"], m["packed"], m["absmax"], m["maps"]
+        _dev(packed, torch.uint8, "packed")
+        _dev(absmax, torch.float32, "absmax")
+        _dev(maps, torch.float32, "maps")
+        out = m.get("out")
+        if out is None:
+            out = torch.empty((layout.N, layout.K), dtype=torch.bfloat16, device=packed.device)
+        _dev(out, torch.bfloat16, "out")
+        arr[i].layout = ctypes.pointer(layout.c)
+        arr[i].W_dev, arr[i].tables_dev = None, maps.data_ptr()
+        arr[i].packed_dev, arr[i].absmax_dev, arr[i].W_bf16_dev = packed.data_ptr(), absmax.data_ptr(), out.data_ptr()
+        outs.append(out)
+    _check(lib().lowra_decode_group(arr, n, _stream(stream)), "lowra_decode_group")
+    return outs
 
 
 def lowra_learn_codebooks(layout: Layout, W: torch.Tensor, init_levels, init_thresholds, iterations: int,

@@ -47,7 +47,8 @@ struct Fetched {
     uint4 packed;        // this lane's 16 packed bytes
     float a0, a1;        // absmax of blocks lane and lane + 32 of the piece
     float m0, m1, m2, m3;   // 1 bit: levels 0, 1; 2 bits: levels 0 .. 3; 4 bits: m0 = level `lane` (lanes 0 .. 15)
-    int c, r, e0;        // class, original row, first element of the piece
+    int c, e0, K;        // class, first element of the piece, row length
+    uint16_t* dst;       // where element e0 of the row goes
 };
 
 __device__ __forceinline__ void locate(const DecodeParams& P, uint32_t t, int& c, int& p, int& piece) {
@@ -82,15 +83,16 @@ __device__ __forceinline__ void fetch_piece(const DecodeParams& P, uint32_t t, i
         f.m0 = __ldg(mrow); f.m1 = __ldg(mrow + 1);
         if (c == 1) { f.m2 = __ldg(mrow + 2); f.m3 = __ldg(mrow + 3); }
     }
-    f.c = c; f.r = r; f.e0 = e0;
+    f.c = c; f.e0 = e0; f.K = K;
+    f.dst = P.out + (size_t)r * K + e0;
 }
 
 // Expands the piece parked in the warp's stage: lane l, in round j, elements e0 + 512 j + 16 l .. + 15.
 template <int B>
-__device__ __forceinline__ void expand_piece(const DecodeParams& P, const Fetched& f, int lane, const WarpStage* ws) {
+__device__ __forceinline__ void expand_piece(const Fetched& f, int lane, const WarpStage* ws) {
     constexpr int kIters = 8 / B;          // 512 elements per iteration
-    const int K = P.L.K;
-    uint16_t* dst = P.out + (size_t)f.r * K + f.e0 + lane * 16;
+    const int K = f.K;
+    uint16_t* dst = f.dst + lane * 16;
     const unsigned char* bytes = reinterpret_cast<const unsigned char*>(ws->packed);
     const float m0 = f.m0, m1 = f.m1, m2 = f.m2, m3 = f.m3;
 #pragma unroll
@@ -130,19 +132,35 @@ __device__ __forceinline__ void expand_piece(const DecodeParams& P, const Fetche
     }
 }
 
-__global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const DecodeParams P) {
+// The tasks of up to NM matrices, numbered through: matrix after matrix, inside a matrix class after class.
+template <int NM>
+struct DecodeGroup {
+    DecodeParams m[NM];
+    uint32_t first_task[NM + 1];   // first task of every member; [NM] (and the entries of unused members) = number of tasks
+};
+
+template <int NM>
+__device__ __forceinline__ void fetch_task(const DecodeGroup<NM>& G, uint32_t t, int lane, Fetched& f) {
+    int mi = 0;
+#pragma unroll
+    for (int i = 1; i < NM; ++i) mi += (t >= G.first_task[i]) ? 1 : 0;
+    fetch_piece(G.m[mi], t - G.first_task[mi], lane, f);
+}
+
+template <int NM>
+__global__ void __launch_bounds__(kDecodeThreads, 5) decode_kernel(const __grid_constant__ DecodeGroup<NM> G) {
     __shared__ __align__(16) WarpStage stage_all[kDecodeWarps];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     WarpStage* ws = &stage_all[warp];
     pdl_enter();
-    const uint32_t n_tasks = P.task_start[3];
+    const uint32_t n_tasks = G.first_task[NM];
     const uint32_t stride = gridDim.x * kDecodeWarps;
     uint32_t t = blockIdx.x * kDecodeWarps + warp;
     if (t >= n_tasks) return;
     // The loads of the warp's next piece are in flight while the current one is expanded and written.
     Fetched cur, nxt;
-    fetch_piece(P, t, lane, cur);
+    fetch_task<NM>(G, t, lane, cur);
     for (;;) {
         ws->packed[lane] = cur.packed;
         ws->absmax[lane] = cur.a0;
@@ -151,10 +169,10 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const DecodePara
         __syncwarp();
         const uint32_t tn = t + stride;
         const bool more = tn < n_tasks;
-        if (more) fetch_piece(P, tn, lane, nxt);
-        if (cur.c == 0) expand_piece<1>(P, cur, lane, ws);
-        else if (cur.c == 1) expand_piece<2>(P, cur, lane, ws);
-        else expand_piece<4>(P, cur, lane, ws);
+        if (more) fetch_task<NM>(G, tn, lane, nxt);
+        if (cur.c == 0) expand_piece<1>(cur, lane, ws);
+        else if (cur.c == 1) expand_piece<2>(cur, lane, ws);
+        else expand_piece<4>(cur, lane, ws);
         if (!more) break;
         __syncwarp();  // the stage is reused by the warp's next piece
         cur = nxt;
@@ -162,28 +180,23 @@ __global__ void __launch_bounds__(kDecodeThreads) decode_kernel(const DecodePara
     }
 }
 
-}  // namespace lowra
+namespace {
 
-extern "C" lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* packed_dev,
-                                     const float* absmax_dev, const float* maps_dev, uint16_t* W_bf16_dev,
-                                     void* stream) {
-    using namespace lowra;
+// checks one matrix's arguments and fills its entry; `tasks` receives the number of its tasks
+lowra_status decode_member(const lowra_layout* layout, const uint8_t* packed_dev, const float* absmax_dev, const float* maps_dev,
+                           uint16_t* W_bf16_dev, DecodeParams& P, uint64_t& tasks) {
     lowra_status st = check_layout(layout);
     if (st != LOWRA_OK) return st;
     if (!packed_dev || !absmax_dev || !maps_dev || !W_bf16_dev) return LOWRA_ERR_NULL;
     if (!aligned16(packed_dev) || !aligned16(absmax_dev) || !aligned16(maps_dev) ||
         (reinterpret_cast<uintptr_t>(W_bf16_dev) & 31u) != 0)
         return LOWRA_ERR_ALIGN;
-    st = check_device();
-    if (st != LOWRA_OK) return st;
-
-    DecodeParams P;
     P.L = make_row_layout(layout);
     P.packed = packed_dev;
     P.absmax = absmax_dev;
     P.maps = maps_dev;
     P.out = W_bf16_dev;
-    uint64_t tasks = 0;
+    tasks = 0;
     for (int c = 0; c < 3; ++c) {
         const uint64_t row_bytes = (uint64_t)layout->K * (1u << c) / 8u;
         P.pieces_per_row[c] = (uint32_t)((row_bytes + 511) / 512);
@@ -192,8 +205,57 @@ extern "C" lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* 
     }
     if (tasks > 0xFFFFFFFFull) return LOWRA_ERR_SHAPE;
     P.task_start[3] = (uint32_t)tasks;
+    return LOWRA_OK;
+}
+
+template <int NM>
+lowra_status launch_decode(const DecodeGroup<NM>& G, void* stream) {
+    const uint64_t tasks = G.first_task[NM];
     const uint64_t blocks_needed = (tasks + kDecodeWarps - 1) / kDecodeWarps;
     const uint64_t cap = (uint64_t)kNumSMs * 8;
     const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
-    return launch_pdl(decode_kernel, grid, kDecodeThreads, (cudaStream_t)stream, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+    return launch_pdl(decode_kernel<NM>, grid, kDecodeThreads, (cudaStream_t)stream, G) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+}
+
+}  // namespace
+
+}  // namespace lowra
+
+extern "C" lowra_status lowra_decode(const lowra_layout* layout, const uint8_t* packed_dev,
+                                     const float* absmax_dev, const float* maps_dev, uint16_t* W_bf16_dev,
+                                     void* stream) {
+    using namespace lowra;
+    DecodeGroup<1> G;
+    uint64_t tasks = 0;
+    lowra_status st = decode_member(layout, packed_dev, absmax_dev, maps_dev, W_bf16_dev, G.m[0], tasks);
+    if (st != LOWRA_OK) return st;
+    st = check_device();
+    if (st != LOWRA_OK) return st;
+    G.first_task[0] = 0;
+    G.first_task[1] = (uint32_t)tasks;
+    return launch_decode<1>(G, stream);
+}
+
+extern "C" lowra_status lowra_decode_group(const lowra_group_member* members_host, int32_t count, void* stream) {
+    using namespace lowra;
+    if (!members_host) return LOWRA_ERR_NULL;
+    if (count < 1 || count > LOWRA_MAX_GROUP) return LOWRA_ERR_SHAPE;
+    DecodeGroup<LOWRA_MAX_GROUP> G;
+    uint64_t total = 0;
+    for (int i = 0; i < count; ++i) {
+        const lowra_group_member& m = members_host[i];
+        uint64_t tasks = 0;
+        lowra_status st = decode_member(m.layout, m.packed_dev, m.absmax_dev, m.tables_dev, m.W_bf16_dev, G.m[i], tasks);
+        if (st != LOWRA_OK) return st;
+        G.first_task[i] = (uint32_t)total;
+        total += tasks;
+        if (total > 0xFFFFFFFFull) return LOWRA_ERR_SHAPE;
+    }
+    for (int i = count; i <= LOWRA_MAX_GROUP; ++i) {
+        if (i < LOWRA_MAX_GROUP) G.m[i] = G.m[0];
+        G.first_task[i] = (uint32_t)total;
+    }
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    return launch_decode<LOWRA_MAX_GROUP>(G, stream);
 }

@@ -147,16 +147,29 @@ __device__ __forceinline__ void encode_chunk(const EncodeParams& P, int p, int c
     }
 }
 
-__global__ void __launch_bounds__(kEncodeThreads, 3) encode_kernel(const EncodeParams P) {
+// The tasks of up to NM matrices, numbered through, matrix after matrix.
+template <int NM>
+struct EncodeGroup {
+    EncodeParams m[NM];
+    uint32_t first_task[NM + 1];   // first task of every member; [NM] (and the entries of unused members) = number of tasks
+};
+
+template <int NM>
+__global__ void __launch_bounds__(kEncodeThreads, 3) encode_kernel(const __grid_constant__ EncodeGroup<NM> G) {
     __shared__ __align__(16) unsigned char stage_all[kEncodeWarps][32 * kSegBytes + 64];
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
     unsigned char* stage = stage_all[warp];
     pdl_enter();
     const uint32_t stride = gridDim.x * kEncodeWarps;
-    for (uint32_t t = blockIdx.x * kEncodeWarps + warp; t < P.n_tasks; t += stride) {
-        const int p = t / P.chunks_per_row;
-        const int chunk = t - p * P.chunks_per_row;
+    for (uint32_t t = blockIdx.x * kEncodeWarps + warp; t < G.first_task[NM]; t += stride) {
+        int mi = 0;
+#pragma unroll
+        for (int i = 1; i < NM; ++i) mi += (t >= G.first_task[i]) ? 1 : 0;
+        const EncodeParams& P = G.m[mi];
+        const uint32_t local = t - G.first_task[mi];
+        const int p = local / P.chunks_per_row;
+        const int chunk = local - p * P.chunks_per_row;
         const int c = (p >= P.L.class_start[1]) + (p >= P.L.class_start[2]);
         if (c == 0) encode_chunk<1>(P, p, chunk, lane, stage);
         else if (c == 1) encode_chunk<2>(P, p, chunk, lane, stage);
@@ -164,20 +177,16 @@ __global__ void __launch_bounds__(kEncodeThreads, 3) encode_kernel(const EncodeP
     }
 }
 
-}  // namespace lowra
+namespace {
 
-extern "C" lowra_status lowra_encode(const lowra_layout* layout, const float* W_dev, const float* thresholds_dev,
-                                     uint8_t* packed_dev, float* absmax_dev, void* stream) {
-    using namespace lowra;
+// checks one matrix's arguments and fills its entry
+lowra_status encode_member(const lowra_layout* layout, const float* W_dev, const float* thresholds_dev, uint8_t* packed_dev,
+                           float* absmax_dev, EncodeParams& P) {
     lowra_status st = check_layout(layout);
     if (st != LOWRA_OK) return st;
     if (!W_dev || !thresholds_dev || !packed_dev || !absmax_dev) return LOWRA_ERR_NULL;
     if (!aligned16(W_dev) || !aligned16(thresholds_dev) || !aligned16(packed_dev) || !aligned16(absmax_dev))
         return LOWRA_ERR_ALIGN;
-    st = check_device();
-    if (st != LOWRA_OK) return st;
-
-    EncodeParams P;
     P.L = make_row_layout(layout);
     P.W = W_dev;
     P.thresholds = thresholds_dev;
@@ -187,8 +196,54 @@ extern "C" lowra_status lowra_encode(const lowra_layout* layout, const float* W_
     const uint64_t tasks = (uint64_t)layout->N * P.chunks_per_row;
     if (tasks > 0xFFFFFFFFull) return LOWRA_ERR_SHAPE;
     P.n_tasks = (uint32_t)tasks;
+    return LOWRA_OK;
+}
+
+template <int NM>
+lowra_status launch_encode(const EncodeGroup<NM>& G, void* stream) {
+    const uint64_t tasks = G.first_task[NM];
     const uint64_t blocks_needed = (tasks + kEncodeWarps - 1) / kEncodeWarps;
     const uint64_t cap = (uint64_t)kNumSMs * 3;   // three CTAs (80 registers, 36 KB of shared memory) are resident per SM
     const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
-    return launch_pdl(encode_kernel, grid, kEncodeThreads, (cudaStream_t)stream, P) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+    return launch_pdl(encode_kernel<NM>, grid, kEncodeThreads, (cudaStream_t)stream, G) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
+}
+
+}  // namespace
+
+}  // namespace lowra
+
+extern "C" lowra_status lowra_encode(const lowra_layout* layout, const float* W_dev, const float* thresholds_dev,
+                                     uint8_t* packed_dev, float* absmax_dev, void* stream) {
+    using namespace lowra;
+    EncodeGroup<1> G;
+    lowra_status st = encode_member(layout, W_dev, thresholds_dev, packed_dev, absmax_dev, G.m[0]);
+    if (st != LOWRA_OK) return st;
+    st = check_device();
+    if (st != LOWRA_OK) return st;
+    G.first_task[0] = 0;
+    G.first_task[1] = G.m[0].n_tasks;
+    return launch_encode<1>(G, stream);
+}
+
+extern "C" lowra_status lowra_encode_group(const lowra_group_member* members_host, int32_t count, void* stream) {
+    using namespace lowra;
+    if (!members_host) return LOWRA_ERR_NULL;
+    if (count < 1 || count > LOWRA_MAX_GROUP) return LOWRA_ERR_SHAPE;
+    EncodeGroup<LOWRA_MAX_GROUP> G;
+    uint64_t total = 0;
+    for (int i = 0; i < count; ++i) {
+        const lowra_group_member& m = members_host[i];
+        lowra_status st = encode_member(m.layout, m.W_dev, m.tables_dev, m.packed_dev, m.absmax_dev, G.m[i]);
+        if (st != LOWRA_OK) return st;
+        G.first_task[i] = (uint32_t)total;
+        total += G.m[i].n_tasks;
+        if (total > 0xFFFFFFFFull) return LOWRA_ERR_SHAPE;
+    }
+    for (int i = count; i <= LOWRA_MAX_GROUP; ++i) {
+        if (i < LOWRA_MAX_GROUP) G.m[i] = G.m[0];
+        G.first_task[i] = (uint32_t)total;
+    }
+    lowra_status st = check_device();
+    if (st != LOWRA_OK) return st;
+    return launch_encode<LOWRA_MAX_GROUP>(G, stream);
 }
