@@ -82,3 +82,29 @@ def test_group_argument_checks(lw):
     with pytest.raises(lw.LowraError) as e:
         lw.lowra_encode_group(nine)
     assert e.value.code == lw.LOWRA_ERR_SHAPE
+
+
+@pytest.mark.parametrize("config", [3, 4])
+def test_a_whole_layer_in_one_launch_equals_the_single_calls(lw, config):
+    """The launch configuration bench.py times: the seven matrices of a layer (full size, the config's precision mix,
+    largest first) through one lowra_encode_group and one lowra_decode_group launch; bit for bit the single calls, which
+    tests/test_gpu_full_size.py holds against the oracle on the same shapes."""
+    cfg = si.config(config)
+    mats = sorted(cfg.matrices, key=lambda m: -m.N * m.K)
+    gen = torch.Generator(device="cuda").manual_seed(config)
+    ms = []
+    for m in mats:
+        precs = si.precisions(m.N, cfg.mix, matrix_id=m.matrix_id)
+        maps, thr = si.standin_codebooks(precs, matrix_id=m.matrix_id)
+        W = torch.randn(m.N, m.K, device="cuda", generator=gen) * 0.02
+        W[::97, ::61] *= 10.0                                   # a few outliers, as in the weight recipe
+        ms.append(dict(layout=lw.Layout(precs, m.K), W=W, thresholds=torch.from_numpy(thr).cuda(), maps=torch.from_numpy(maps).cuda()))
+    group = lw.lowra_encode_group([dict(layout=m["layout"], W=m["W"], thresholds=m["thresholds"]) for m in ms])
+    outs = lw.lowra_decode_group([dict(layout=m["layout"], packed=p, absmax=a, maps=m["maps"]) for m, (p, a) in zip(ms, group)])
+    for m, (p, a), o in zip(ms, group, outs):
+        p1, a1 = lw.lowra_encode(m["layout"], m["W"], m["thresholds"])
+        assert torch.equal(p1[:m["layout"].packed_bytes], p[:m["layout"].packed_bytes])
+        assert torch.equal(a1.view(torch.int32), a.view(torch.int32))
+        o1 = lw.lowra_decode(m["layout"], p1, a1, m["maps"])
+        assert torch.equal(o1.view(torch.int16), o.view(torch.int16))
+        del p1, a1, o1
