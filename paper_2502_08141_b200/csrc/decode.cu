@@ -42,7 +42,7 @@ struct WarpStage {
     float lut[16];       // 4-bit rows: the row's levels
 };
 
-// What a warp fetches for one piece, held in registers while the previous piece is being expanded.
+// What a warp fetches for its piece.
 struct Fetched {
     uint4 packed;        // this lane's 16 packed bytes
     float a0, a1;        // absmax of blocks lane and lane + 32 of the piece
@@ -147,6 +147,9 @@ __device__ __forceinline__ void fetch_task(const DecodeGroup<NM>& G, uint32_t t,
     fetch_piece(G.m[mi], t - G.first_task[mi], lane, f);
 }
 
+// One piece per warp, one CTA per eight pieces: the hardware hands fresh CTAs to the SMs as others finish, which keeps the
+// SMs evenly loaded although the pieces differ in length by a factor of four (a persistent grid whose warps walked over
+// several pieces each, the next one's loads in flight, was 8 % slower).
 template <int NM>
 __global__ void __launch_bounds__(kDecodeThreads, 5) decode_kernel(const __grid_constant__ DecodeGroup<NM> G) {
     __shared__ __align__(16) WarpStage stage_all[kDecodeWarps];
@@ -154,30 +157,18 @@ __global__ void __launch_bounds__(kDecodeThreads, 5) decode_kernel(const __grid_
     const int warp = threadIdx.x >> 5;
     WarpStage* ws = &stage_all[warp];
     pdl_enter();
-    const uint32_t n_tasks = G.first_task[NM];
-    const uint32_t stride = gridDim.x * kDecodeWarps;
-    uint32_t t = blockIdx.x * kDecodeWarps + warp;
-    if (t >= n_tasks) return;
-    // The loads of the warp's next piece are in flight while the current one is expanded and written.
-    Fetched cur, nxt;
+    const uint32_t t = blockIdx.x * kDecodeWarps + warp;
+    if (t >= G.first_task[NM]) return;
+    Fetched cur;
     fetch_task<NM>(G, t, lane, cur);
-    for (;;) {
-        ws->packed[lane] = cur.packed;
-        ws->absmax[lane] = cur.a0;
-        ws->absmax[lane + 32] = cur.a1;
-        if (cur.c == 2 && lane < 16) ws->lut[lane] = cur.m0;
-        __syncwarp();
-        const uint32_t tn = t + stride;
-        const bool more = tn < n_tasks;
-        if (more) fetch_task<NM>(G, tn, lane, nxt);
-        if (cur.c == 0) expand_piece<1>(cur, lane, ws);
-        else if (cur.c == 1) expand_piece<2>(cur, lane, ws);
-        else expand_piece<4>(cur, lane, ws);
-        if (!more) break;
-        __syncwarp();  // the stage is reused by the warp's next piece
-        cur = nxt;
-        t = tn;
-    }
+    ws->packed[lane] = cur.packed;
+    ws->absmax[lane] = cur.a0;
+    ws->absmax[lane + 32] = cur.a1;
+    if (cur.c == 2 && lane < 16) ws->lut[lane] = cur.m0;
+    __syncwarp();
+    if (cur.c == 0) expand_piece<1>(cur, lane, ws);
+    else if (cur.c == 1) expand_piece<2>(cur, lane, ws);
+    else expand_piece<4>(cur, lane, ws);
 }
 
 namespace {
@@ -211,9 +202,7 @@ lowra_status decode_member(const lowra_layout* layout, const uint8_t* packed_dev
 template <int NM>
 lowra_status launch_decode(const DecodeGroup<NM>& G, void* stream) {
     const uint64_t tasks = G.first_task[NM];
-    const uint64_t blocks_needed = (tasks + kDecodeWarps - 1) / kDecodeWarps;
-    const uint64_t cap = (uint64_t)kNumSMs * 8;
-    const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
+    const unsigned grid = (unsigned)((tasks + kDecodeWarps - 1) / kDecodeWarps);   // < 2^29: the tasks were counted in 32 bits
     return launch_pdl(decode_kernel<NM>, grid, kDecodeThreads, (cudaStream_t)stream, G) == cudaSuccess ? LOWRA_OK : LOWRA_ERR_CUDA;
 }
 
