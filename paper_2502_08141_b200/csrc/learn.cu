@@ -25,6 +25,7 @@ namespace lowra {
 
 constexpr int kLearnThreads = 128;
 constexpr int kLearnWarps = kLearnThreads / 32;
+constexpr int kLoadsInFlight = 8;   // 128-bit loads a thread issues before it looks at the first one (a 4096-element row in one go)
 
 struct LearnParams {
     RowLayout L;
@@ -88,15 +89,15 @@ __device__ void load_row(const LearnParams& P, int r, float* xs, float* ws) {
     const int K = P.K;
     const int tid = threadIdx.x;
     const float* wrow = P.W + (size_t)r * K;
-    for (int i0 = 0; i0 < K; i0 += 4 * 4 * kLearnThreads) {
-        float4 v[4];
+    for (int i0 = 0; i0 < K; i0 += 4 * kLoadsInFlight * kLearnThreads) {
+        float4 v[kLoadsInFlight];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kLoadsInFlight; ++u) {
             const int i = i0 + 4 * (u * kLearnThreads + tid);
             v[u] = (i < K) ? ld_stream_f4(wrow + i) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kLoadsInFlight; ++u) {
             const int i = i0 + 4 * (u * kLearnThreads + tid);   // K is a multiple of 128: a warp is in or out as a whole
             float m = fmaxf(fmaxf(fabsf(v[u].x), fabsf(v[u].y)), fmaxf(fabsf(v[u].z), fabsf(v[u].w)));
 #pragma unroll
