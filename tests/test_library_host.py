@@ -173,3 +173,20 @@ def test_missing_library_fails_loudly(lib, monkeypatch, tmp_path):
     monkeypatch.setattr(lib, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(RuntimeError, match="no fallback"):
         lib.lib()
+
+
+def test_public_headers_compile_as_plain_c(tmp_path):
+    """The boundary is a C ABI: both headers must go through a C99 compiler on their own (no C++ in the signatures)."""
+    import shutil
+    import subprocess
+
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "h.c"
+    src.write_text('#include "lowra.h"\n#include "lowra_diag.h"\n'
+                   "int main(void) { lowra_layout l; lowra_member m; lowra_group_member g; (void)l; (void)m; (void)g; return 0; }\n")
+    out = subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(root, "include"),
+                          "-c", str(src), "-o", str(tmp_path / "h.o")], capture_output=True, text=True)
+    assert out.returncode == 0, out.stderr
